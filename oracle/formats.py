@@ -1,0 +1,168 @@
+"""Format oracle: BCSR, WCSR and the long-window split plan.  TEST INFRASTRUCTURE ONLY.
+
+Each function writes out the definition from the paper (Sec. 2.3 "Sparse
+Formats"; Sec. 3.3 for the task decomposition) with numpy primitives
+(repeat, unique, bincount, cumsum, fancy-index scatter).  There is no
+blocking, threading or device code here, and nothing is shared with the
+CUDA library's own format construction.
+
+Readings taken where the paper is silent or garbled (all listed again in the
+design notes):
+  * a block / a window column is kept when any *stored* CSR entry falls in
+    it, whatever its value (structural, Sec. 2.3 "contain at least one
+    nonzero");
+  * m and k need not be multiples of the block / window size: counts use
+    ceilings and the ragged edge is zero padded;
+  * blocks inside a block-row and columns inside a window are ascending;
+  * WCSR ``values`` is ONE row-major 2-D array [b_row, padded_nnz_cols]
+    (the second of the two shapes printed in Sec. 2.3);
+  * an empty window has length 0 (no pad group);
+  * a long window is cut into consecutive chunks of T columns (Sec. 3.3
+    "fixed-size sub-tasks"); T is a multiple of b_col.
+
+Values are moved, never computed with, so any dtype works (bf16 travels as
+uint16 bit patterns).
+
+Pins (tests/test_oracle_formats.py): brute-force per-element Python
+constructions on tiny inputs, round trips to dense, the array-length and
+fill-ratio formulas of Sec. 2.3, dense / block-diagonal / diagonal /
+identical-row special cases, wh = 1 degenerating to padded CSR.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def _csr_rows(row_ptr):
+    row_ptr = np.asarray(row_ptr, dtype=np.int64)
+    m = row_ptr.shape[0] - 1
+    return np.repeat(np.arange(m, dtype=np.int64), np.diff(row_ptr))
+
+
+def _cdiv(a, b):
+    return -(-a // b)
+
+
+# --------------------------------------------------------------------------- BCSR
+
+
+def bcsr_from_csr(m, k, row_ptr, col_idx, vals, b):
+    """CSR -> BCSR with b x b blocks (Sec. 2.3, BCSR paragraph).
+
+    Returns dict(block_row_ptr int32 [ceil(m/b)+1], block_col_idx int32 [nnzb],
+    blocks [nnzb, b, b] of vals.dtype, zero filled).
+    """
+    vals = np.asarray(vals)
+    col = np.asarray(col_idx, dtype=np.int64)
+    rows = _csr_rows(row_ptr)
+    nbr, nbc = _cdiv(m, b), _cdiv(k, b)
+    key = (rows // b) * nbc + (col // b)
+    ukeys = np.unique(key)                       # ascending => block-row major, block-col ascending
+    nnzb = ukeys.shape[0]
+    counts = np.bincount(ukeys // nbc, minlength=nbr)
+    block_row_ptr = np.zeros(nbr + 1, dtype=np.int64)
+    block_row_ptr[1:] = np.cumsum(counts)
+    blocks = np.zeros((nnzb, b, b), dtype=vals.dtype)
+    pos = np.searchsorted(ukeys, key)
+    blocks[pos, rows % b, col % b] = vals
+    return dict(
+        block_row_ptr=block_row_ptr.astype(np.int32),
+        block_col_idx=(ukeys % nbc).astype(np.int32),
+        blocks=blocks,
+    )
+
+
+def bcsr_to_dense(m, k, b, block_row_ptr, block_col_idx, blocks):
+    """Expand BCSR back to a dense m x k array (stored zeros become zeros)."""
+    nbr = block_row_ptr.shape[0] - 1
+    nbc = _cdiv(k, b)
+    D = np.zeros((nbr * b, nbc * b), dtype=blocks.dtype)
+    for I in range(nbr):
+        for p in range(block_row_ptr[I], block_row_ptr[I + 1]):
+            J = int(block_col_idx[p])
+            D[I * b:(I + 1) * b, J * b:(J + 1) * b] = blocks[p]
+    return D[:m, :k]
+
+
+def fill_ratio_bcsr(nnz, nnzb, b):
+    """nnz / (nnz_blocks * b_row * b_col)  (Sec. 2.3)."""
+    return nnz / float(nnzb * b * b) if nnzb else 0.0
+
+
+# --------------------------------------------------------------------------- WCSR
+
+
+def wcsr_from_csr(m, k, row_ptr, col_idx, vals, wh, b_col):
+    """CSR -> WCSR with window height wh and column padding b_col (Sec. 2.3, WCSR paragraph).
+
+    Returns dict(window_row_ptr int32 [ceil(m/wh)+1] in units of columns,
+    window_col_idx int32 [P] (-1 on pads), values [wh, P] of vals.dtype).
+    """
+    vals = np.asarray(vals)
+    col = np.asarray(col_idx, dtype=np.int64)
+    rows = _csr_rows(row_ptr)
+    nwin = _cdiv(m, wh)
+    key = (rows // wh) * k + col
+    ukeys = np.unique(key)                        # window major, columns ascending
+    uwin = ukeys // k
+    cnt = np.bincount(uwin, minlength=nwin).astype(np.int64)
+    length = _cdiv(cnt, b_col) * b_col            # 0 stays 0
+    wptr = np.zeros(nwin + 1, dtype=np.int64)
+    wptr[1:] = np.cumsum(length)
+    P = int(wptr[-1])
+    if P >= 2 ** 31:
+        raise ValueError("padded column count does not fit int32")
+    first = np.zeros(nwin + 1, dtype=np.int64)
+    first[1:] = np.cumsum(cnt)
+    rank = np.arange(ukeys.shape[0], dtype=np.int64) - first[uwin]
+    ppos = wptr[uwin] + rank                      # padded position of every kept column
+    wcol = np.full(P, -1, dtype=np.int32)
+    wcol[ppos] = (ukeys % k).astype(np.int32)
+    values = np.zeros((wh, P), dtype=vals.dtype)
+    values[rows % wh, ppos[np.searchsorted(ukeys, key)]] = vals
+    return dict(window_row_ptr=wptr.astype(np.int32), window_col_idx=wcol, values=values)
+
+
+def wcsr_to_dense(m, k, wh, window_row_ptr, window_col_idx, values):
+    """Expand WCSR back to a dense m x k array."""
+    nwin = window_row_ptr.shape[0] - 1
+    D = np.zeros((nwin * wh, k), dtype=values.dtype)
+    for w in range(nwin):
+        for q in range(window_row_ptr[w], window_row_ptr[w + 1]):
+            c = int(window_col_idx[q])
+            if c >= 0:
+                D[w * wh:(w + 1) * wh, c] = values[:, q]
+    return D[:m]
+
+
+def fill_ratio_wcsr(nnz, P, wh):
+    """Stored-value analogue of the BCSR fill ratio: nnz / (wh * padded columns)."""
+    return nnz / float(wh * P) if P else 0.0
+
+
+# --------------------------------------------------------------------------- split plan
+
+
+def split_plan(window_row_ptr, T):
+    """Task decomposition of Sec. 3.3: windows longer than T columns are cut
+    into consecutive chunks of T columns; every chunk is one task.
+
+    Returns int32 array [ntasks, 4] with rows (window, q0, count, slot):
+    q0 is the chunk's first column relative to the window start, count its
+    number of columns, slot the index of the partial-sum tile the task writes
+    (running index over all chunks of windows that have more than one chunk,
+    in task order) or -1 when the window is a single task that writes C
+    directly.  Empty windows produce no task.
+    """
+    wptr = np.asarray(window_row_ptr, dtype=np.int64)
+    length = np.diff(wptr)
+    nchunk = _cdiv(length, T)
+    win = np.repeat(np.arange(length.shape[0], dtype=np.int64), nchunk)
+    firsttask = np.zeros(length.shape[0] + 1, dtype=np.int64)
+    firsttask[1:] = np.cumsum(nchunk)
+    cidx = np.arange(win.shape[0], dtype=np.int64) - firsttask[win]
+    q0 = cidx * T
+    count = np.minimum(T, length[win] - q0)
+    is_split = nchunk[win] > 1
+    slot = np.where(is_split, np.cumsum(is_split) - 1, -1)
+    return np.stack([win, q0, count, slot], axis=1).astype(np.int32)

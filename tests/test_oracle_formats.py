@@ -1,0 +1,218 @@
+"""Pins for the format oracle (Sec. 2.3 BCSR / WCSR, Sec. 3.3 split plan).
+
+The numpy definitions in oracle/formats.py are compared with per-element
+Python constructions written here from the paper's text, with round trips,
+with the array-length and fill-ratio formulas the paper prints, and with
+special cases whose answer is known in closed form.
+"""
+import numpy as np
+import pytest
+
+from oracle import formats as F
+from paper_2604_17834_b200 import workloads as wl
+
+
+def _dense(a):
+    m, k = a["m"], a["k"]
+    D = np.zeros((m, k), dtype=a["vals"].dtype)
+    mask = np.zeros((m, k), dtype=bool)
+    for i in range(m):
+        for p in range(a["row_ptr"][i], a["row_ptr"][i + 1]):
+            D[i, a["col_idx"][p]] = a["vals"][p]
+            mask[i, a["col_idx"][p]] = True
+    return D, mask
+
+
+def _brute_bcsr(D, mask, b):
+    m, k = D.shape
+    nbr, nbc = -(-m // b), -(-k // b)
+    ptr, idx, blocks = [0], [], []
+    for I in range(nbr):
+        for J in range(nbc):
+            sub = mask[I * b:(I + 1) * b, J * b:(J + 1) * b]
+            if sub.any():
+                blk = np.zeros((b, b), dtype=D.dtype)
+                d = D[I * b:(I + 1) * b, J * b:(J + 1) * b]
+                blk[:d.shape[0], :d.shape[1]] = d
+                idx.append(J)
+                blocks.append(blk)
+        ptr.append(len(idx))
+    return ptr, idx, blocks
+
+
+def _brute_wcsr(D, mask, wh, b_col):
+    m, k = D.shape
+    nwin = -(-m // wh)
+    ptr, idx, cols_vals = [0], [], []
+    for w in range(nwin):
+        rows = range(w * wh, min(m, (w + 1) * wh))
+        kept = [c for c in range(k) if any(mask[r, c] for r in rows)]
+        for c in kept:
+            v = np.zeros(wh, dtype=D.dtype)
+            for r in rows:
+                v[r - w * wh] = D[r, c]
+            idx.append(c)
+            cols_vals.append(v)
+        while len(idx) % b_col:
+            idx.append(-1)
+            cols_vals.append(np.zeros(wh, dtype=D.dtype))
+        ptr.append(len(idx))
+    vals = np.stack(cols_vals, axis=1) if cols_vals else np.zeros((wh, 0), dtype=D.dtype)
+    return ptr, idx, vals
+
+
+CASES = [(37, 29, 0.15), (64, 64, 0.05), (16, 50, 0.5), (70, 130, 0.02)]
+
+
+@pytest.mark.parametrize("m,k,dens", CASES)
+@pytest.mark.parametrize("b", [4, 16, 32])
+def test_bcsr_matches_brute_force_and_round_trips(m, k, dens, b):
+    a = wl.random_csr(100 + m + b, m, k, dens, "fp16", empty_rows=(0, m - 1))
+    D, mask = _dense(a)
+    f = F.bcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], b)
+    ptr, idx, blocks = _brute_bcsr(D, mask, b)
+    assert f["block_row_ptr"].tolist() == ptr
+    assert f["block_col_idx"].tolist() == idx
+    assert f["block_row_ptr"].shape[0] == -(-m // b) + 1            # Sec. 2.3 array lengths
+    assert f["blocks"].shape == (len(idx), b, b)
+    if blocks:
+        assert np.array_equal(f["blocks"].view(np.uint16), np.stack(blocks).view(np.uint16))
+    back = F.bcsr_to_dense(m, k, b, f["block_row_ptr"], f["block_col_idx"], f["blocks"])
+    assert np.array_equal(back.view(np.uint16), D.view(np.uint16))
+    # every stored CSR entry is found again: nnz preserved
+    assert int(mask.sum()) == a["col_idx"].shape[0]
+    nb = -(-m // b) * -(-k // b)
+    assert len(idx) == sum(
+        mask[I * b:(I + 1) * b, J * b:(J + 1) * b].any()
+        for I in range(-(-m // b)) for J in range(-(-k // b)))
+    assert len(idx) <= nb
+
+
+def test_bcsr_structural_zero_keeps_block():
+    # an explicitly stored 0.0 marks its block (structural reading)
+    row_ptr = np.array([0, 1, 1, 1, 1], np.int64)
+    f = F.bcsr_from_csr(4, 4, row_ptr, np.array([3], np.int32), np.array([0.0], np.float32), 2)
+    assert f["block_row_ptr"].tolist() == [0, 1, 1] and f["block_col_idx"].tolist() == [1]
+
+
+def test_bcsr_dense_and_block_diagonal_and_fill_ratio():
+    m = k = 24
+    b = 8
+    a = wl.random_csr(1, m, k, 2.0, "tf32")                 # density >= 1 -> fully dense
+    f = F.bcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], b)
+    assert f["block_col_idx"].shape[0] == 9
+    assert F.fill_ratio_bcsr(m * k, 9, b) == 1.0
+    mask = np.eye(3, dtype=bool)
+    rp, ci = wl.csr_from_block_mask(mask, b, m, k)
+    f = F.bcsr_from_csr(m, k, rp, ci, np.ones(ci.shape[0], np.float32), b)
+    assert f["block_col_idx"].tolist() == [0, 1, 2]
+    assert f["block_row_ptr"].tolist() == [0, 1, 2, 3]
+    # one entry per block: fill ratio = nnz / (nnzb * b * b)
+    rp = np.array([0, 1] + [1] * 7 + [2] + [2] * 15, np.int64)
+    f = F.bcsr_from_csr(m, k, rp, np.array([0, 9], np.int32), np.ones(2, np.float32), b)
+    assert F.fill_ratio_bcsr(2, f["block_col_idx"].shape[0], b) == 2 / (2 * 64)
+
+
+@pytest.mark.parametrize("m,k,dens", CASES)
+@pytest.mark.parametrize("wh,b_col", [(4, 2), (16, 8), (16, 16), (1, 4)])
+def test_wcsr_matches_brute_force_and_round_trips(m, k, dens, wh, b_col):
+    a = wl.random_csr(200 + m + wh, m, k, dens, "fp16", empty_rows=tuple(range(min(wh, m))))
+    D, mask = _dense(a)
+    f = F.wcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], wh, b_col)
+    ptr, idx, vals = _brute_wcsr(D, mask, wh, b_col)
+    assert f["window_row_ptr"].tolist() == ptr
+    assert f["window_col_idx"].tolist() == idx
+    assert f["values"].shape == (wh, len(idx))               # one 2-D array [b_row, padded cols]
+    assert np.array_equal(f["values"].view(np.uint16), vals.view(np.uint16))
+    assert f["window_row_ptr"][1] == 0                        # first window emptied above
+    lens = np.diff(f["window_row_ptr"])
+    assert np.all(lens % b_col == 0)
+    pads = f["window_col_idx"] < 0
+    assert np.all(f["window_col_idx"][pads] == -1)
+    assert not f["values"][:, pads].any()
+    for w in range(len(ptr) - 1):
+        c = f["window_col_idx"][ptr[w]:ptr[w + 1]]
+        c = c[c >= 0]
+        assert np.all(np.diff(c) > 0)                         # strictly ascending
+    back = F.wcsr_to_dense(m, k, wh, f["window_row_ptr"], f["window_col_idx"], f["values"])
+    assert np.array_equal(back.view(np.uint16), D.view(np.uint16))
+
+
+def test_wcsr_height_one_is_padded_csr():
+    a = wl.random_csr(5, 20, 33, 0.2, "tf32")
+    f = F.wcsr_from_csr(20, 33, a["row_ptr"], a["col_idx"], a["vals"], 1, 4)
+    for i in range(20):
+        lo, hi = a["row_ptr"][i], a["row_ptr"][i + 1]
+        q0, q1 = f["window_row_ptr"][i], f["window_row_ptr"][i + 1]
+        n = hi - lo
+        assert q1 - q0 == -(-n // 4) * 4
+        assert np.array_equal(f["window_col_idx"][q0:q0 + n], a["col_idx"][lo:hi])
+        assert np.array_equal(f["values"][0, q0:q0 + n], a["vals"][lo:hi])
+
+
+def test_wcsr_identical_rows_and_diagonal():
+    wh, b_col, k = 8, 4, 40
+    cols = np.array([1, 5, 6, 20, 39], np.int32)
+    rp = np.arange(0, 5 * wh + 1, 5, dtype=np.int64)
+    f = F.wcsr_from_csr(wh, k, rp, np.tile(cols, wh), np.ones(5 * wh, np.float32), wh, b_col)
+    assert f["window_row_ptr"].tolist() == [0, 8]              # pad(5) = 8
+    assert f["window_col_idx"].tolist() == [1, 5, 6, 20, 39, -1, -1, -1]
+    n = 24
+    f = F.wcsr_from_csr(n, n, np.arange(n + 1, dtype=np.int64), np.arange(n, dtype=np.int32),
+                        np.arange(1, n + 1, dtype=np.float32), wh, b_col)
+    assert np.all(np.diff(f["window_row_ptr"]) == wh)          # pad(wh) = wh columns per window
+    assert np.array_equal(f["values"][np.arange(n) % wh, np.arange(n)], np.arange(1, n + 1))
+
+
+def _brute_plan(wptr, T):
+    tasks, slot = [], 0
+    for w in range(len(wptr) - 1):
+        L = wptr[w + 1] - wptr[w]
+        chunks = [(q0, min(T, L - q0)) for q0 in range(0, L, T)]
+        for q0, c in chunks:
+            if len(chunks) > 1:
+                tasks.append((w, q0, c, slot))
+                slot += 1
+            else:
+                tasks.append((w, q0, c, -1))
+    return tasks
+
+
+@pytest.mark.parametrize("T", [8, 16, 64, 4096])
+def test_split_plan(T):
+    rng = np.random.default_rng(T)
+    lens = rng.choice([0, 8, 16, 24, 64, 72, 200, 1000], size=60)
+    wptr = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    plan = F.split_plan(wptr, T)
+    assert plan.dtype == np.int32
+    assert [tuple(r) for r in plan.tolist()] == _brute_plan(wptr.tolist(), T)
+    assert plan[:, 2].sum() == wptr[-1]                        # chunks tile all padded columns
+    assert np.all(plan[:, 2] <= T) and np.all(plan[:, 2] % 8 == 0) and np.all(plan[:, 2] > 0)
+    if T >= lens.max():
+        assert np.all(plan[:, 3] == -1)                        # nothing split
+    # chunks of one window are consecutive, in order, and tile [0, len)
+    for w in np.unique(plan[:, 0]):
+        rows = plan[plan[:, 0] == w]
+        assert rows[0, 1] == 0
+        assert np.all(rows[1:, 1] == rows[:-1, 1] + rows[:-1, 2])
+        assert rows[-1, 1] + rows[-1, 2] == lens[w]
+
+
+def test_generators_are_deterministic_and_shaped():
+    a1, a2 = wl.bcsr_tiny(), wl.bcsr_tiny()
+    assert np.array_equal(a1["col_idx"], a2["col_idx"]) and np.array_equal(a1["vals"], a2["vals"])
+    g = wl.bcsr_llm(m=1024, k=512)
+    f = F.bcsr_from_csr(1024, 512, g["row_ptr"], g["col_idx"], g["vals"], 64)
+    assert f["block_col_idx"].shape[0] == 128 - int(np.floor(0.9 * 128))
+    s = wl.bcsr_sweep(9, m=1024, k=1024, b=32, density=0.2)
+    f = F.bcsr_from_csr(1024, 1024, s["row_ptr"], s["col_idx"], s["vals"], 32)
+    per_row = np.diff(f["block_row_ptr"])
+    assert (per_row == 32).sum() >= 3 and (per_row == 0).sum() >= 6
+    r = wl.rmat(scale=10, edge_factor=8)
+    assert r["m"] == 1024 and np.all(np.diff(r["row_ptr"]) >= 0)
+    keys = np.repeat(np.arange(1024), np.diff(r["row_ptr"])) * 1024 + r["col_idx"]
+    assert np.all(np.diff(keys) > 0)                           # sorted, duplicates merged
+    w = wl.wcsr_irregular(m=2000)
+    keys = np.repeat(np.arange(2000), np.diff(w["row_ptr"])) * 2000 + w["col_idx"]
+    assert np.all(np.diff(keys) > 0)
+    assert np.diff(w["row_ptr"]).min() >= 1
