@@ -1,0 +1,202 @@
+/*
+ * spmm_b200 -- sparse x dense matrix multiplication C = A x B on one NVIDIA
+ * B200 (sm_100a), with A held in one of the two formats of the AsyncSparse
+ * paper (Sec. 2.3 "Sparse Formats"):
+ *
+ *   BCSR  Block Compressed Sparse Row: A is tiled into b x b blocks and only
+ *         blocks holding at least one stored entry are kept, each as a dense
+ *         tile.  The kernel runs one tensor-core micro-GEMM per stored block
+ *         (Sec. 3.1 - 3.3).
+ *   WCSR  Window Compressed Sparse Row: rows are grouped into windows of
+ *         fixed height; per window the union of the column indices is kept
+ *         and padded to a multiple of b_col.  The kernel gathers the matching
+ *         rows of B and multiplies them with the packed window tile; long
+ *         windows are cut into fixed-size sub-tasks (Sec. 3.2 - 3.3).
+ *
+ * Conventions
+ *   - A is m x k, B is k x N row-major (B[r*N + c]), C is m x N row-major,
+ *     fp32.  C is overwritten completely (no alpha / beta; Sec. 2.3 states
+ *     the problem as C = A x B).
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA
+ *     device memory of the current device.  The library never frees or keeps
+ *     a caller's pointer beyond the call that receives it.
+ *   - Every function returns 0 (SPMM_OK) or a negative spmm_status_t.  No
+ *     exception crosses this boundary.
+ *   - There is no CPU fallback: without a CUDA device every create call that
+ *     is not host_only, and every run call, fails with SPMM_ERR_CUDA.
+ */
+#ifndef SPMM_B200_H
+#define SPMM_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct spmm_handle_s *spmm_handle_t;
+
+typedef enum {
+    SPMM_OK = 0,
+    SPMM_ERR_INVALID_ARG = -1,   /* null pointer, negative size, bad enum value              */
+    SPMM_ERR_UNSORTED = -2,      /* CSR columns not strictly ascending / duplicate COO entry  */
+    SPMM_ERR_OUT_OF_RANGE = -3,  /* row or column index outside the matrix                    */
+    SPMM_ERR_UNSUPPORTED = -4,   /* block / window size, N, dtype or alignment not supported  */
+    SPMM_ERR_ALLOC = -5,         /* host or device allocation failed                          */
+    SPMM_ERR_CUDA = -6,          /* a CUDA call or a launch failed (no device, bad context)   */
+    SPMM_ERR_DEV_TIMEOUT = -7,   /* a bounded wait inside a kernel ran out (see spmm_check)   */
+    SPMM_ERR_HOST_ONLY = -8,     /* the handle was created host_only and cannot run           */
+    SPMM_ERR_TOO_LARGE = -9      /* a size exceeds a fixed capacity (int32 index, scratch)    */
+} spmm_status_t;
+
+/* Value type of A and B.  Accumulation and C are always fp32. */
+typedef enum {
+    SPMM_BF16 = 0,               /* 2-byte bfloat16 storage                                   */
+    SPMM_FP16 = 1,               /* 2-byte IEEE half storage                                  */
+    SPMM_TF32 = 2                /* 4-byte fp32 storage, TF32 tensor-core arithmetic          */
+} spmm_dtype_t;
+
+/* Optional creation parameters; pass NULL for all defaults.  Zero = default. */
+typedef struct {
+    int32_t b_col;       /* WCSR: pad every window to a multiple of this many columns.
+                            Default (and only supported value): 16 for 2-byte types, 8 for
+                            TF32 -- the K extent of one tensor-core instruction (Sec. 2.3,
+                            Sec. 4.1 uses 8 with TF32).                                      */
+    int32_t split_cols;  /* WCSR: sub-task size T in columns (Sec. 3.3); multiple of b_col.
+                            Default 1024.                                                    */
+    int32_t host_only;   /* 1: build the format on the host only (no CUDA call at all); the
+                            handle serves spmm_export / spmm_get_info, spmm_run fails.       */
+    int32_t n_ctas;      /* persistent grid size the schedule is built for; default = the
+                            device's SM count (148 when host_only).                          */
+    int32_t reserved[12];
+} spmm_opts_t;
+
+typedef struct {
+    int32_t format;          /* 0 = BCSR, 1 = WCSR                                            */
+    int32_t dtype;           /* spmm_dtype_t                                                  */
+    int64_t m, k, nnz;       /* matrix shape and number of stored CSR/COO entries             */
+    int32_t block;           /* BCSR block size b, or WCSR window height                      */
+    int32_t b_col;           /* WCSR column padding (0 for BCSR)                              */
+    int64_t n_units;         /* BCSR: stored blocks; WCSR: padded columns P                   */
+    int64_t stored_values;   /* BCSR: blocks*b*b; WCSR: height*P  ("nnz_stored")              */
+    double  fill_ratio;      /* nnz / stored_values (Sec. 2.3)                                */
+    int64_t n_rows_units;    /* BCSR: block-rows; WCSR: windows                               */
+    int64_t n_empty;         /* empty block-rows / windows                                    */
+    int64_t n_tasks;         /* WCSR sub-tasks (0 for BCSR)                                   */
+    int64_t n_split;         /* WCSR windows cut into more than one task                      */
+    int64_t n_slots;         /* WCSR partial-sum tiles                                        */
+    int32_t split_cols;      /* WCSR T in effect                                              */
+    int32_t n_ctas;          /* grid size the schedule was built for                          */
+    int64_t distinct_b_rows; /* rows of B that A touches (distinct stored columns)            */
+    /* bytes the roofline model charges for one spmm_run at the given N: */
+    double  bytes_a, bytes_idx, bytes_b_touched, bytes_c;
+    double  bytes_gather;    /* B bytes that must enter shared memory (no reuse assumed)      */
+    double  flops_stored;    /* 2 * stored_values * N                                         */
+    int64_t workspace_bytes; /* device scratch spmm_run needs at this N (WCSR partial tiles)  */
+} spmm_info_t;
+
+/* Arrays spmm_export can return, in their canonical (paper) layout. */
+typedef enum {
+    SPMM_X_BCSR_BLOCK_ROW_PTR = 0,  /* int32 [ceil(m/b)+1]                                   */
+    SPMM_X_BCSR_BLOCK_COL_IDX = 1,  /* int32 [n_blocks], ascending inside a block-row         */
+    SPMM_X_BCSR_BLOCKS = 2,         /* dtype [n_blocks][b][b] row-major, zero filled          */
+    SPMM_X_BCSR_ROW_ORDER = 3,      /* int32 [block-rows]: schedule order, longest first      */
+    SPMM_X_WCSR_WINDOW_ROW_PTR = 10,/* int32 [ceil(m/h)+1], in columns                        */
+    SPMM_X_WCSR_WINDOW_COL_IDX = 11,/* int32 [P], -1 on padding                               */
+    SPMM_X_WCSR_VALUES = 12,        /* dtype [h][P] row-major                                 */
+    SPMM_X_WCSR_TASKS = 13,         /* int32 [n_tasks][4]: window, first col in window,
+                                       column count, partial slot (-1 = writes C directly)    */
+    SPMM_X_WCSR_SPANS = 14          /* int32 [n_spans+1]: task ranges handed to the CTAs      */
+} spmm_export_t;
+
+/*
+ * Create a BCSR handle from CSR (Sec. 2.3, BCSR paragraph).
+ *   out      receives the handle (NULL on failure).
+ *   m, k     matrix shape; need not be multiples of `block` (ragged edge is zero padded).
+ *   row_ptr  host int64 [m+1], row_ptr[0] = 0, non-decreasing.
+ *   col_idx  host int32 [nnz], strictly ascending inside each row, in [0, k).
+ *   vals     host, nnz elements of `dtype` (2 or 4 bytes each; bf16/fp16 as raw 16-bit).
+ *   block    16, 32, 64 or 128.
+ * A block is kept when any stored entry falls inside it, whatever its value.
+ * The arrays are copied; the caller keeps ownership.  The handle owns its device memory.
+ */
+int spmm_bcsr_create_csr(spmm_handle_t *out, int64_t m, int64_t k, const int64_t *row_ptr,
+                         const int32_t *col_idx, const void *vals, int dtype, int block,
+                         const spmm_opts_t *opts);
+
+/* Same from COO: host int32 rows[nnz], cols[nnz] in any order, no duplicate (row, col). */
+int spmm_bcsr_create_coo(spmm_handle_t *out, int64_t m, int64_t k, int64_t nnz,
+                         const int32_t *rows, const int32_t *cols, const void *vals, int dtype,
+                         int block, const spmm_opts_t *opts);
+
+/*
+ * Create a WCSR handle (Sec. 2.3, WCSR paragraph; task split of Sec. 3.3).
+ * Arguments as above; window_height is 16 (the only supported value; Sec. 5
+ * names finer-than-64 windows as the redesign this library performs).
+ * Per window the kept columns are ascending, then -1 pads up to a multiple of b_col.
+ */
+int spmm_wcsr_create_csr(spmm_handle_t *out, int64_t m, int64_t k, const int64_t *row_ptr,
+                         const int32_t *col_idx, const void *vals, int dtype, int window_height,
+                         const spmm_opts_t *opts);
+
+int spmm_wcsr_create_coo(spmm_handle_t *out, int64_t m, int64_t k, int64_t nnz,
+                         const int32_t *rows, const int32_t *cols, const void *vals, int dtype,
+                         int window_height, const spmm_opts_t *opts);
+
+/*
+ * C = A x B (Sec. 2.3; kernels of Sec. 3).  Asynchronous on `stream` (a cudaStream_t passed
+ * as void*; NULL = the default stream); never synchronises.
+ *   B_dev  device, k x N row-major, elements of the handle's dtype, 16-byte aligned.
+ *   C_dev  device, m x N row-major fp32, 16-byte aligned; every element is written.
+ *   N      dense width; N * element size must be a multiple of 16 bytes.
+ * WCSR keeps the partial tiles of split windows in a device workspace owned by the handle;
+ * it is (re)allocated here the first time a given N needs more than it holds, so two runs
+ * of one handle must not overlap on the GPU, and the first run at a new N may synchronise.
+ * Split windows are merged by a fixed-order sum, so results are run-to-run identical.
+ */
+int spmm_run(spmm_handle_t h, const void *B_dev, void *C_dev, int64_t N, void *stream);
+
+/*
+ * Same result as spmm_run, for callers that hold HOST buffers: copies B to the device,
+ * runs, copies C back and synchronises `stream` before returning.  B_host / C_host are
+ * ordinary or pinned host memory of k*N elements / m*N floats; the device staging buffers
+ * belong to the handle and are reused between calls.
+ */
+int spmm_run_host(spmm_handle_t h, const void *B_host, void *C_host, int64_t N, void *stream);
+
+/*
+ * After the caller has synchronised the stream: reads the handle's device status word.
+ * Every wait inside the kernels is bounded; a wait that ran out makes the kernel leave
+ * early and this call return SPMM_ERR_DEV_TIMEOUT (the output is then undefined).
+ * The status word is cleared by the call.
+ */
+int spmm_check(spmm_handle_t h);
+
+/* Fill *info; the byte / flop model fields are evaluated for dense width N (N may be 0). */
+int spmm_get_info(spmm_handle_t h, int64_t N, spmm_info_t *info);
+
+/*
+ * Copy one canonical array to host memory.  *need receives its size in bytes; when
+ * host_dst is NULL or cap < *need nothing is copied (SPMM_ERR_INVALID_ARG if cap is too
+ * small and host_dst non-NULL).  Arrays are read back from the device copy the kernels
+ * use (and un-permuted where the device layout is private), so what is checked is what runs.
+ */
+int spmm_export(spmm_handle_t h, int which, void *host_dst, size_t cap, size_t *need);
+
+/* Free the handle and everything it owns.  NULL is accepted. */
+int spmm_destroy(spmm_handle_t h);
+
+/* Static, never-NULL description of a status code. */
+const char *spmm_status_string(int code);
+
+/*
+ * Upper bound, in nanoseconds, of any single wait inside a kernel (default 2e9).  Process
+ * wide; meant for tests of the timeout path.  Values below 1000 are raised to 1000.
+ */
+int spmm_set_wait_limit_ns(uint64_t ns);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPMM_B200_H */

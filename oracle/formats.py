@@ -166,3 +166,37 @@ def split_plan(window_row_ptr, T):
     is_split = nchunk[win] > 1
     slot = np.where(is_split, np.cumsum(is_split) - 1, -1)
     return np.stack([win, q0, count, slot], axis=1).astype(np.int32)
+
+
+# --------------------------------------------------------------------------- schedules
+
+
+def bcsr_row_order(block_row_ptr):
+    """Order in which block-rows are scheduled: most stored blocks first, ties by index.
+
+    This is the longest-processing-time-first rule applied to the imbalance
+    Sec. 3.5 / Sec. 4.2 (opt6) describe for a persistent kernel with a static
+    tile order: a block-row's work is proportional to its number of stored blocks.
+    """
+    lens = np.diff(np.asarray(block_row_ptr, dtype=np.int64))
+    return np.argsort(-lens, kind="stable").astype(np.int32)
+
+
+def task_spans(plan, n_spans, fixed_cost=32):
+    """Cut the task list into n_spans consecutive ranges of near-equal cost.
+
+    cost(task) = its column count + fixed_cost.  Span j ends after the first
+    task at which the running cost c satisfies c * n_spans >= (j + 1) * total
+    (integer arithmetic); spans may be empty.  Returns int32 [n_spans + 1].
+    """
+    cost = plan[:, 2].astype(np.int64) + fixed_cost
+    total = int(cost.sum())
+    spans = [0]
+    run, ti, nt = 0, 0, plan.shape[0]
+    for j in range(n_spans):
+        while ti < nt and run * n_spans < (j + 1) * total:
+            run += int(cost[ti])
+            ti += 1
+        spans.append(ti)
+    spans[-1] = nt
+    return np.asarray(spans, dtype=np.int32)

@@ -1,0 +1,639 @@
+// C-ABI layer: handles, format upload, tensor maps, launches (see include/spmm_b200.h).
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "format.h"
+#include "kernels.h"
+#include "spmm_b200.h"
+
+using namespace spmm;
+
+namespace {
+
+std::atomic<uint64_t> g_wait_limit_ns{2000000000ull};
+
+inline int elem_size(int dtype) { return dtype == SPMM_TF32 ? 4 : 2; }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// 2-D row-major tensor [rows][cols] of 16-bit elements, box [box_rows][box_cols].
+int encode_2d_16bit(CUtensorMap* map, int dtype, const void* base, uint64_t rows, uint64_t cols,
+                    uint32_t box_rows, uint32_t box_cols, CUtensorMapSwizzle swz) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return SPMM_ERR_CUDA;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {box_cols, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapDataType dt = dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+    CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SPMM_OK : SPMM_ERR_CUDA;
+}
+
+template <class T>
+int upload(T** dptr, const void* src, size_t bytes) {
+    *dptr = nullptr;
+    const size_t alloc = bytes ? bytes : 16;
+    if (cudaMalloc(reinterpret_cast<void**>(dptr), alloc) != cudaSuccess) return SPMM_ERR_ALLOC;
+    if (bytes && cudaMemcpy(*dptr, src, bytes, cudaMemcpyHostToDevice) != cudaSuccess) return SPMM_ERR_CUDA;
+    return SPMM_OK;
+}
+
+}  // namespace
+
+struct spmm_handle_s {
+    int format = 0;      // 0 BCSR, 1 WCSR
+    int dtype = 0;
+    int es = 2;
+    int64_t m = 0, k = 0, nnz = 0;
+    bool host_only = false;
+    int n_ctas = 148;
+    int sms = 148;
+    int device = 0;
+
+    BcsrHost bcsr;       // index arrays kept; value array dropped after upload unless host_only
+    WcsrHost wcsr;
+
+    // device copies
+    int32_t* d_ptr = nullptr;        // block_row_ptr / window_row_ptr
+    int32_t* d_idx = nullptr;        // block_col_idx / window_col_idx
+    uint8_t* d_vals = nullptr;       // blocks / packed values
+    int32_t* d_order = nullptr;      // BCSR row order
+    WcsrDevTask* d_tasks = nullptr;
+    int32_t* d_spans = nullptr;
+    int32_t* d_merge = nullptr;      // window | first | nparts, each [n_merge]
+    int n_merge = 0;
+    int* d_status = nullptr;
+
+    float* d_partial = nullptr;      // WCSR workspace
+    size_t partial_bytes = 0;
+
+    // BCSR tensor maps
+    CUtensorMap tmA;
+    bool tmA_ok = false;
+    CUtensorMap tmB;
+    const void* tmB_ptr = nullptr;
+    int64_t tmB_N = -1;
+
+    // staging for spmm_run_host
+    void* d_Bstage = nullptr;
+    size_t Bstage_bytes = 0;
+    float* d_Cstage = nullptr;
+    size_t Cstage_bytes = 0;
+};
+
+namespace {
+
+void free_handle(spmm_handle_s* h) {
+    if (!h) return;
+    if (!h->host_only) {
+        cudaFree(h->d_ptr);
+        cudaFree(h->d_idx);
+        cudaFree(h->d_vals);
+        cudaFree(h->d_order);
+        cudaFree(h->d_tasks);
+        cudaFree(h->d_spans);
+        cudaFree(h->d_merge);
+        cudaFree(h->d_status);
+        cudaFree(h->d_partial);
+        cudaFree(h->d_Bstage);
+        cudaFree(h->d_Cstage);
+    }
+    delete h;
+}
+
+int device_setup(spmm_handle_s* h, const spmm_opts_t* opts) {
+    if (h->host_only) {
+        h->sms = 148;
+        h->n_ctas = (opts && opts->n_ctas > 0) ? opts->n_ctas : 148;
+        return SPMM_OK;
+    }
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SPMM_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SPMM_ERR_CUDA;
+    if (prop.major != 10) return SPMM_ERR_UNSUPPORTED;   // sm_100a code only
+    h->device = dev;
+    h->sms = prop.multiProcessorCount;
+    h->n_ctas = (opts && opts->n_ctas > 0) ? opts->n_ctas : h->sms;
+    if (cudaMalloc(reinterpret_cast<void**>(&h->d_status), 4 * sizeof(int)) != cudaSuccess) return SPMM_ERR_ALLOC;
+    if (cudaMemset(h->d_status, 0, 4 * sizeof(int)) != cudaSuccess) return SPMM_ERR_CUDA;
+    return SPMM_OK;
+}
+
+int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, const spmm_opts_t* opts) {
+    if (dtype != SPMM_BF16 && dtype != SPMM_FP16) return SPMM_ERR_UNSUPPORTED;
+    int rc = validate_csr(a);
+    if (rc) return rc;
+    spmm_handle_s* h = new (std::nothrow) spmm_handle_s;
+    if (!h) return SPMM_ERR_ALLOC;
+    h->format = 0;
+    h->dtype = dtype;
+    h->es = a.es;
+    h->m = a.m;
+    h->k = a.k;
+    h->nnz = a.nnz;
+    h->host_only = opts && opts->host_only;
+    rc = device_setup(h, opts);
+    if (rc) { free_handle(h); return rc; }
+    try {
+        rc = build_bcsr(a, block, &h->bcsr);
+    } catch (const std::bad_alloc&) {
+        rc = SPMM_ERR_ALLOC;
+    }
+    if (rc) { free_handle(h); return rc; }
+    if (!h->host_only) {
+        const BcsrHost& f = h->bcsr;
+        if (static_cast<int64_t>(f.nnzb) * f.b >= (int64_t{1} << 31)) { free_handle(h); return SPMM_ERR_TOO_LARGE; }
+        rc = upload(&h->d_ptr, f.block_row_ptr.data(), f.block_row_ptr.size() * 4);
+        if (!rc) rc = upload(&h->d_idx, f.block_col_idx.data(), f.block_col_idx.size() * 4);
+        if (!rc) rc = upload(&h->d_vals, f.blocks.data(), f.blocks.size());
+        if (!rc) rc = upload(&h->d_order, f.row_order.data(), f.row_order.size() * 4);
+        if (!rc && f.nnzb > 0) {
+            const int bw = f.b < 64 ? f.b : 64;
+            const CUtensorMapSwizzle swz = bw == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                          : (bw == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+            rc = encode_2d_16bit(&h->tmA, dtype, h->d_vals, static_cast<uint64_t>(f.nnzb) * f.b, f.b, f.b, bw, swz);
+            h->tmA_ok = rc == SPMM_OK;
+        }
+        if (rc) { free_handle(h); return rc; }
+        std::vector<uint8_t>().swap(h->bcsr.blocks);   // the device copy is the one that counts
+    }
+    *out = h;
+    return SPMM_OK;
+}
+
+int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const spmm_opts_t* opts) {
+    if (dtype != SPMM_BF16 && dtype != SPMM_FP16 && dtype != SPMM_TF32) return SPMM_ERR_UNSUPPORTED;
+    int rc = validate_csr(a);
+    if (rc) return rc;
+    const int b_col_default = 32 / a.es;
+    const int b_col = (opts && opts->b_col > 0) ? opts->b_col : b_col_default;
+    if (b_col != b_col_default) return SPMM_ERR_UNSUPPORTED;
+    const int T = (opts && opts->split_cols > 0) ? opts->split_cols : 1024;
+    if (T % b_col != 0) return SPMM_ERR_INVALID_ARG;
+    spmm_handle_s* h = new (std::nothrow) spmm_handle_s;
+    if (!h) return SPMM_ERR_ALLOC;
+    h->format = 1;
+    h->dtype = dtype;
+    h->es = a.es;
+    h->m = a.m;
+    h->k = a.k;
+    h->nnz = a.nnz;
+    h->host_only = opts && opts->host_only;
+    rc = device_setup(h, opts);
+    if (rc) { free_handle(h); return rc; }
+    try {
+        rc = build_wcsr(a, wh, b_col, T, h->n_ctas * 8, &h->wcsr);
+    } catch (const std::bad_alloc&) {
+        rc = SPMM_ERR_ALLOC;
+    }
+    if (rc) { free_handle(h); return rc; }
+    if (!h->host_only) {
+        const WcsrHost& f = h->wcsr;
+        std::vector<WcsrDevTask> dt(f.tasks.size());
+        for (size_t i = 0; i < f.tasks.size(); ++i) {
+            dt[i].col_begin = f.window_row_ptr[f.tasks[i].window] + f.tasks[i].q0;
+            dt[i].count = f.tasks[i].count;
+            dt[i].window = f.tasks[i].window;
+            dt[i].slot = f.tasks[i].slot;
+        }
+        const size_t nm = f.merge_window.size();
+        std::vector<int32_t> mg(3 * nm);
+        for (size_t i = 0; i < nm; ++i) {
+            mg[i] = f.merge_window[i];
+            mg[nm + i] = f.merge_first[i];
+            mg[2 * nm + i] = f.merge_nparts[i];
+        }
+        h->n_merge = static_cast<int>(nm);
+        rc = upload(&h->d_ptr, f.window_row_ptr.data(), f.window_row_ptr.size() * 4);
+        if (!rc) rc = upload(&h->d_idx, f.window_col_idx.data(), f.window_col_idx.size() * 4);
+        if (!rc) rc = upload(&h->d_vals, f.packed.data(), f.packed.size());
+        if (!rc) rc = upload(&h->d_tasks, dt.data(), dt.size() * sizeof(WcsrDevTask));
+        if (!rc) rc = upload(&h->d_spans, f.spans.data(), f.spans.size() * 4);
+        if (!rc) rc = upload(&h->d_merge, mg.data(), mg.size() * 4);
+        if (rc) { free_handle(h); return rc; }
+        std::vector<uint8_t>().swap(h->wcsr.packed);
+    }
+    *out = h;
+    return SPMM_OK;
+}
+
+int make_view(CsrView* v, int64_t m, int64_t k, const int64_t* row_ptr, const int32_t* col_idx, const void* vals,
+              int dtype) {
+    if (dtype < 0 || dtype > 2) return SPMM_ERR_INVALID_ARG;
+    if (m < 0 || k < 0 || !row_ptr) return SPMM_ERR_INVALID_ARG;
+    if (m >= (int64_t{1} << 31) || k >= (int64_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
+    v->m = m;
+    v->k = k;
+    v->row_ptr = row_ptr;
+    v->nnz = row_ptr[m];
+    v->col_idx = col_idx;
+    v->vals = static_cast<const uint8_t*>(vals);
+    v->es = elem_size(dtype);
+    return SPMM_OK;
+}
+
+int ensure_tmB(spmm_handle_s* h, const void* B, int64_t N, int groups) {
+    (void)groups;
+    if (h->tmB_ptr == B && h->tmB_N == N) return SPMM_OK;
+    int rc = encode_2d_16bit(&h->tmB, h->dtype, B, static_cast<uint64_t>(h->k), static_cast<uint64_t>(N),
+                             static_cast<uint32_t>(h->bcsr.b), 64, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+    h->tmB_ptr = B;
+    h->tmB_N = N;
+    return SPMM_OK;
+}
+
+int run_bcsr(spmm_handle_s* h, const void* B, float* C, int64_t N, cudaStream_t stream) {
+    const BcsrHost& f = h->bcsr;
+    if (N < 64) return SPMM_ERR_UNSUPPORTED;   // the B box is 64 tokens wide
+    // token tile: the largest of 512 / 256 / 128 columns that divides N (Sec. 4.3: pick a tile
+    // width that divides the dense width so that no padded columns are computed); otherwise
+    // the largest tile, whose ragged last tile is predicated.
+    const int gmax = bcsr_token_groups_max(f.b);
+    int groups = 0;
+    for (int g = gmax; g >= 1; g >>= 1)
+        if (N % (128 * g) == 0) { groups = g; break; }
+    if (!groups) groups = N >= 128 * gmax ? gmax : (N > 128 ? 2 : 1);
+    // keep at least ~4 tiles per CTA when the matrix is small
+    while (groups > 1 && f.nbr * ((N + 128 * groups - 1) / (128 * groups)) < 4 * h->n_ctas) groups >>= 1;
+    const int bnt = 128 * groups;
+    BcsrParams p;
+    p.block_row_ptr = h->d_ptr;
+    p.block_col_idx = h->d_idx;
+    p.row_order = h->d_order;
+    p.C = C;
+    p.m = h->m;
+    p.N = N;
+    p.nbr = static_cast<int32_t>(f.nbr);
+    p.n_tt = static_cast<int32_t>((N + bnt - 1) / bnt);
+    // slab: token tiles whose B rows (k x slab columns) stay within ~48 MB of L2
+    const int64_t slab_cols = (int64_t{48} << 20) / (h->k * h->es > 0 ? h->k * h->es : 1);
+    int64_t sw = slab_cols / bnt;
+    if (sw < 1) sw = 1;
+    if (sw > p.n_tt) sw = p.n_tt;
+    p.slab_w = static_cast<int32_t>(sw);
+    p.total_tiles = static_cast<int64_t>(p.nbr) * p.n_tt;
+    p.status = h->d_status;
+    p.wait_limit_ns = g_wait_limit_ns.load();
+    if (p.total_tiles == 0) return SPMM_OK;
+    CUtensorMap tmA = h->tmA;
+    if (!h->tmA_ok) {
+        // no stored block at all: the kernel never touches A, any valid map will do
+        int rc = encode_2d_16bit(&tmA, h->dtype, h->d_vals, 8, 8, 8, 8, CU_TENSOR_MAP_SWIZZLE_NONE);
+        if (rc) return rc;
+    }
+    int rc = ensure_tmB(h, B, N, groups);
+    if (rc) return rc;
+    int grid = h->n_ctas;
+    if (grid > p.total_tiles) grid = static_cast<int>(p.total_tiles);
+    cudaError_t e = launch_bcsr(h->dtype, f.b, groups, tmA, h->tmB, p, grid, stream);
+    return e == cudaSuccess ? SPMM_OK : SPMM_ERR_CUDA;
+}
+
+int64_t wcsr_workspace_bytes(const spmm_handle_s* h, int64_t N) {
+    return h->wcsr.n_slots * int64_t{16} * N * 4;
+}
+
+int launch_wcsr_all(spmm_handle_s* h, const void* B, float* C, float* partial, int64_t N, cudaStream_t stream) {
+    const WcsrHost& f = h->wcsr;
+    const int groups = N > 128 ? 2 : 1;
+    const int bnt = 128 * groups;
+    WcsrParams p;
+    p.tasks = h->d_tasks;
+    p.spans = h->d_spans;
+    p.col_idx = h->d_idx;
+    p.packed = h->d_vals;
+    p.B = B;
+    p.C = C;
+    p.partial = partial;
+    p.m = h->m;
+    p.N = N;
+    p.n_spans = static_cast<int32_t>(f.spans.size()) - 1;
+    p.n_tt = static_cast<int32_t>((N + bnt - 1) / bnt);
+    p.status = h->d_status;
+    p.wait_limit_ns = g_wait_limit_ns.load();
+    if (!f.tasks.empty()) {
+        cudaError_t e = launch_wcsr(h->dtype, groups, p, h->sms, stream);
+        if (e != cudaSuccess) return SPMM_ERR_CUDA;
+    }
+    MergeParams mp;
+    mp.window = h->d_merge;
+    mp.first = h->d_merge + h->n_merge;
+    mp.nparts = h->d_merge + 2 * h->n_merge;
+    mp.partial = partial;
+    mp.C = C;
+    mp.m = h->m;
+    mp.N = N;
+    mp.n = h->n_merge;
+    cudaError_t e = launch_wcsr_merge(mp, stream);
+    return e == cudaSuccess ? SPMM_OK : SPMM_ERR_CUDA;
+}
+
+int run_wcsr(spmm_handle_s* h, const void* B, float* C, int64_t N, cudaStream_t stream) {
+    const size_t need = static_cast<size_t>(wcsr_workspace_bytes(h, N));
+    if (need > h->partial_bytes) {
+        if (h->d_partial) {
+            if (cudaDeviceSynchronize() != cudaSuccess) return SPMM_ERR_CUDA;
+            cudaFree(h->d_partial);
+            h->d_partial = nullptr;
+            h->partial_bytes = 0;
+        }
+        if (cudaMalloc(reinterpret_cast<void**>(&h->d_partial), need) != cudaSuccess) return SPMM_ERR_ALLOC;
+        h->partial_bytes = need;
+    }
+    return launch_wcsr_all(h, B, C, h->d_partial, N, stream);
+}
+
+int check_run_args(spmm_handle_s* h, const void* B, const void* C, int64_t N) {
+    if (!h || !B || !C || N <= 0) return SPMM_ERR_INVALID_ARG;
+    if (h->host_only) return SPMM_ERR_HOST_ONLY;
+    if ((N * h->es) % 16 != 0) return SPMM_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(B) & 15) || (reinterpret_cast<uintptr_t>(C) & 15)) return SPMM_ERR_UNSUPPORTED;
+    if (N >= (int64_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
+    return SPMM_OK;
+}
+
+}  // namespace
+
+// ============================================================================= C ABI
+
+extern "C" {
+
+int spmm_bcsr_create_csr(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* row_ptr, const int32_t* col_idx,
+                         const void* vals, int dtype, int block, const spmm_opts_t* opts) {
+    if (!out) return SPMM_ERR_INVALID_ARG;
+    *out = nullptr;
+    CsrView v;
+    int rc = make_view(&v, m, k, row_ptr, col_idx, vals, dtype);
+    if (rc) return rc;
+    return create_bcsr(out, v, dtype, block, opts);
+}
+
+int spmm_bcsr_create_coo(spmm_handle_t* out, int64_t m, int64_t k, int64_t nnz, const int32_t* rows,
+                         const int32_t* cols, const void* vals, int dtype, int block, const spmm_opts_t* opts) {
+    if (!out) return SPMM_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (dtype < 0 || dtype > 2) return SPMM_ERR_INVALID_ARG;
+    CsrOwned o;
+    int rc;
+    try {
+        rc = coo_to_csr(m, k, nnz, rows, cols, static_cast<const uint8_t*>(vals), elem_size(dtype), &o);
+    } catch (const std::bad_alloc&) {
+        rc = SPMM_ERR_ALLOC;
+    }
+    if (rc) return rc;
+    return spmm_bcsr_create_csr(out, m, k, o.row_ptr.data(), o.col_idx.data(), o.vals.data(), dtype, block, opts);
+}
+
+int spmm_wcsr_create_csr(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* row_ptr, const int32_t* col_idx,
+                         const void* vals, int dtype, int window_height, const spmm_opts_t* opts) {
+    if (!out) return SPMM_ERR_INVALID_ARG;
+    *out = nullptr;
+    CsrView v;
+    int rc = make_view(&v, m, k, row_ptr, col_idx, vals, dtype);
+    if (rc) return rc;
+    return create_wcsr(out, v, dtype, window_height, opts);
+}
+
+int spmm_wcsr_create_coo(spmm_handle_t* out, int64_t m, int64_t k, int64_t nnz, const int32_t* rows,
+                         const int32_t* cols, const void* vals, int dtype, int window_height,
+                         const spmm_opts_t* opts) {
+    if (!out) return SPMM_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (dtype < 0 || dtype > 2) return SPMM_ERR_INVALID_ARG;
+    CsrOwned o;
+    int rc;
+    try {
+        rc = coo_to_csr(m, k, nnz, rows, cols, static_cast<const uint8_t*>(vals), elem_size(dtype), &o);
+    } catch (const std::bad_alloc&) {
+        rc = SPMM_ERR_ALLOC;
+    }
+    if (rc) return rc;
+    return spmm_wcsr_create_csr(out, m, k, o.row_ptr.data(), o.col_idx.data(), o.vals.data(), dtype, window_height,
+                                opts);
+}
+
+int spmm_run(spmm_handle_t h, const void* B_dev, void* C_dev, int64_t N, void* stream) {
+    int rc = check_run_args(h, B_dev, C_dev, N);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (h->format == 0) return run_bcsr(h, B_dev, static_cast<float*>(C_dev), N, st);
+    return run_wcsr(h, B_dev, static_cast<float*>(C_dev), N, st);
+}
+
+int spmm_run_host(spmm_handle_t h, const void* B_host, void* C_host, int64_t N, void* stream) {
+    if (!h || !B_host || !C_host || N <= 0) return SPMM_ERR_INVALID_ARG;
+    if (h->host_only) return SPMM_ERR_HOST_ONLY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t bbytes = static_cast<size_t>(h->k) * N * h->es;
+    const size_t cbytes = static_cast<size_t>(h->m) * N * 4;
+    if (bbytes > h->Bstage_bytes) {
+        cudaFree(h->d_Bstage);
+        h->d_Bstage = nullptr;
+        h->Bstage_bytes = 0;
+        if (cudaMalloc(&h->d_Bstage, bbytes ? bbytes : 16) != cudaSuccess) return SPMM_ERR_ALLOC;
+        h->Bstage_bytes = bbytes;
+    }
+    if (cbytes > h->Cstage_bytes) {
+        cudaFree(h->d_Cstage);
+        h->d_Cstage = nullptr;
+        h->Cstage_bytes = 0;
+        if (cudaMalloc(reinterpret_cast<void**>(&h->d_Cstage), cbytes ? cbytes : 16) != cudaSuccess) return SPMM_ERR_ALLOC;
+        h->Cstage_bytes = cbytes;
+    }
+    if (cudaMemcpyAsync(h->d_Bstage, B_host, bbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SPMM_ERR_CUDA;
+    int rc = spmm_run(h, h->d_Bstage, h->d_Cstage, N, stream);
+    if (rc) return rc;
+    if (cudaMemcpyAsync(C_host, h->d_Cstage, cbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SPMM_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SPMM_ERR_CUDA;
+    return SPMM_OK;
+}
+
+int spmm_check(spmm_handle_t h) {
+    if (!h) return SPMM_ERR_INVALID_ARG;
+    if (h->host_only) return SPMM_ERR_HOST_ONLY;
+    int st[4] = {0, 0, 0, 0};
+    if (cudaMemcpy(st, h->d_status, sizeof(st), cudaMemcpyDeviceToHost) != cudaSuccess) return SPMM_ERR_CUDA;
+    if (st[0] != 0) {
+        cudaMemset(h->d_status, 0, sizeof(st));
+        return SPMM_ERR_DEV_TIMEOUT;
+    }
+    return SPMM_OK;
+}
+
+int spmm_get_info(spmm_handle_t h, int64_t N, spmm_info_t* info) {
+    if (!h || !info || N < 0) return SPMM_ERR_INVALID_ARG;
+    std::memset(info, 0, sizeof(*info));
+    info->format = h->format;
+    info->dtype = h->dtype;
+    info->m = h->m;
+    info->k = h->k;
+    info->nnz = h->nnz;
+    info->n_ctas = h->n_ctas;
+    const double s = h->es, n = static_cast<double>(N);
+    if (h->format == 0) {
+        const BcsrHost& f = h->bcsr;
+        info->block = f.b;
+        info->n_units = f.nnzb;
+        info->stored_values = f.nnzb * f.b * f.b;
+        info->n_rows_units = f.nbr;
+        info->n_empty = f.n_empty;
+        int64_t rows_touched = f.distinct_bcols * f.b;
+        if (rows_touched > h->k) rows_touched = h->k;
+        info->distinct_b_rows = rows_touched;
+        info->bytes_a = static_cast<double>(info->stored_values) * s;
+        info->bytes_idx = static_cast<double>(f.nbr + 1 + f.nnzb) * 4.0;
+        info->bytes_gather = static_cast<double>(f.nnzb) * f.b * n * s;
+    } else {
+        const WcsrHost& f = h->wcsr;
+        info->block = f.wh;
+        info->b_col = f.b_col;
+        info->n_units = f.P;
+        info->stored_values = f.P * f.wh;
+        info->n_rows_units = f.nwin;
+        info->n_empty = f.n_empty;
+        info->n_tasks = static_cast<int64_t>(f.tasks.size());
+        info->n_split = f.n_split;
+        info->n_slots = f.n_slots;
+        info->split_cols = f.T;
+        info->distinct_b_rows = f.distinct_cols;
+        info->bytes_a = static_cast<double>(info->stored_values) * s;
+        info->bytes_idx = static_cast<double>(f.nwin + 1 + f.P) * 4.0;
+        info->bytes_gather = static_cast<double>(f.P) * n * s;
+        info->workspace_bytes = wcsr_workspace_bytes(h, N);
+    }
+    info->fill_ratio = info->stored_values ? static_cast<double>(h->nnz) / static_cast<double>(info->stored_values) : 0.0;
+    info->bytes_b_touched = static_cast<double>(info->distinct_b_rows) * n * s;
+    info->bytes_c = static_cast<double>(h->m) * n * 4.0;
+    info->flops_stored = 2.0 * static_cast<double>(info->stored_values) * n;
+    return SPMM_OK;
+}
+
+int spmm_export(spmm_handle_t h, int which, void* host_dst, size_t cap, size_t* need) {
+    if (!h || !need) return SPMM_ERR_INVALID_ARG;
+    const void* dev_src = nullptr;    // device array in canonical layout, or
+    const void* host_src = nullptr;   // host array in canonical layout
+    size_t bytes = 0;
+    bool unpack_wcsr = false;
+    std::vector<int32_t> tmp;
+    if (h->format == 0) {
+        const BcsrHost& f = h->bcsr;
+        switch (which) {
+            case SPMM_X_BCSR_BLOCK_ROW_PTR: bytes = f.block_row_ptr.size() * 4; dev_src = h->d_ptr; host_src = f.block_row_ptr.data(); break;
+            case SPMM_X_BCSR_BLOCK_COL_IDX: bytes = f.block_col_idx.size() * 4; dev_src = h->d_idx; host_src = f.block_col_idx.data(); break;
+            case SPMM_X_BCSR_BLOCKS: bytes = static_cast<size_t>(f.nnzb) * f.b * f.b * h->es; dev_src = h->d_vals; host_src = f.blocks.data(); break;
+            case SPMM_X_BCSR_ROW_ORDER: bytes = f.row_order.size() * 4; dev_src = h->d_order; host_src = f.row_order.data(); break;
+            default: return SPMM_ERR_INVALID_ARG;
+        }
+    } else {
+        const WcsrHost& f = h->wcsr;
+        switch (which) {
+            case SPMM_X_WCSR_WINDOW_ROW_PTR: bytes = f.window_row_ptr.size() * 4; dev_src = h->d_ptr; host_src = f.window_row_ptr.data(); break;
+            case SPMM_X_WCSR_WINDOW_COL_IDX: bytes = f.window_col_idx.size() * 4; dev_src = h->d_idx; host_src = f.window_col_idx.data(); break;
+            case SPMM_X_WCSR_VALUES: bytes = static_cast<size_t>(f.P) * f.wh * h->es; unpack_wcsr = true; break;
+            case SPMM_X_WCSR_TASKS: bytes = f.tasks.size() * 16; break;
+            case SPMM_X_WCSR_SPANS: bytes = f.spans.size() * 4; dev_src = h->d_spans; host_src = f.spans.data(); break;
+            default: return SPMM_ERR_INVALID_ARG;
+        }
+    }
+    *need = bytes;
+    if (!host_dst) return SPMM_OK;
+    if (cap < bytes) return SPMM_ERR_INVALID_ARG;
+    if (bytes == 0) return SPMM_OK;
+    if (unpack_wcsr) {
+        const WcsrHost& f = h->wcsr;
+        std::vector<uint8_t> packed_dl;
+        const uint8_t* packed = f.packed.data();
+        if (!h->host_only) {
+            packed_dl.resize(bytes);
+            if (cudaMemcpy(packed_dl.data(), h->d_vals, bytes, cudaMemcpyDeviceToHost) != cudaSuccess) return SPMM_ERR_CUDA;
+            packed = packed_dl.data();
+        }
+        uint8_t* dst = static_cast<uint8_t*>(host_dst);
+        for (int r = 0; r < f.wh; ++r)
+            for (int64_t q = 0; q < f.P; ++q)
+                std::memcpy(dst + (static_cast<size_t>(r) * f.P + q) * h->es,
+                            packed + wcsr_packed_offset(f.wh, f.b_col, h->es, r, q), h->es);
+        return SPMM_OK;
+    }
+    if (h->format == 1 && which == SPMM_X_WCSR_TASKS) {
+        const WcsrHost& f = h->wcsr;
+        int32_t* dst = static_cast<int32_t*>(host_dst);
+        if (h->host_only) {
+            for (size_t i = 0; i < f.tasks.size(); ++i) {
+                dst[4 * i + 0] = f.tasks[i].window;
+                dst[4 * i + 1] = f.tasks[i].q0;
+                dst[4 * i + 2] = f.tasks[i].count;
+                dst[4 * i + 3] = f.tasks[i].slot;
+            }
+        } else {
+            std::vector<WcsrDevTask> dt(f.tasks.size());
+            if (cudaMemcpy(dt.data(), h->d_tasks, bytes, cudaMemcpyDeviceToHost) != cudaSuccess) return SPMM_ERR_CUDA;
+            for (size_t i = 0; i < dt.size(); ++i) {
+                dst[4 * i + 0] = dt[i].window;
+                dst[4 * i + 1] = dt[i].col_begin - f.window_row_ptr[dt[i].window];
+                dst[4 * i + 2] = dt[i].count;
+                dst[4 * i + 3] = dt[i].slot;
+            }
+        }
+        return SPMM_OK;
+    }
+    if (h->host_only) {
+        std::memcpy(host_dst, host_src, bytes);
+        return SPMM_OK;
+    }
+    return cudaMemcpy(host_dst, dev_src, bytes, cudaMemcpyDeviceToHost) == cudaSuccess ? SPMM_OK : SPMM_ERR_CUDA;
+}
+
+int spmm_destroy(spmm_handle_t h) {
+    free_handle(h);
+    return SPMM_OK;
+}
+
+const char* spmm_status_string(int code) {
+    switch (code) {
+        case SPMM_OK: return "ok";
+        case SPMM_ERR_INVALID_ARG: return "invalid argument";
+        case SPMM_ERR_UNSORTED: return "unsorted or duplicate entries";
+        case SPMM_ERR_OUT_OF_RANGE: return "index out of range";
+        case SPMM_ERR_UNSUPPORTED: return "unsupported size, dtype, alignment or device";
+        case SPMM_ERR_ALLOC: return "allocation failed";
+        case SPMM_ERR_CUDA: return "CUDA call failed (is there a B200 and a usable context?)";
+        case SPMM_ERR_DEV_TIMEOUT: return "a bounded wait inside a kernel ran out";
+        case SPMM_ERR_HOST_ONLY: return "handle was created host_only";
+        case SPMM_ERR_TOO_LARGE: return "size exceeds a fixed capacity";
+        default: return "unknown status";
+    }
+}
+
+int spmm_set_wait_limit_ns(uint64_t ns) {
+    g_wait_limit_ns.store(ns < 1000 ? 1000 : ns);
+    return SPMM_OK;
+}
+
+}  // extern "C"

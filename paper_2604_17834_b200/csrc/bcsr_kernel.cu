@@ -1,0 +1,288 @@
+// BCSR SpMM kernel for sm_100a (Sec. 3.1 - 3.3 of the paper, re-designed for Blackwell).
+//
+// Work unit ("tile"): one block-row I of A times BN_T = 128 * GROUPS columns of B
+// ("tokens").  For every stored block p of the block-row the tile accumulates
+//     D[n, r] += sum_c  B[J_p*b + c, n0 + n] * A_p[r, c]
+// i.e. the tokens sit on the 128 TMEM lanes (MMA M side, operand read MN-major straight
+// from row-major B) and the b rows of the block are the MMA N side (operand = the stored
+// block, K-major).  One shape therefore serves b = 16, 32, 64 and 128, and the epilogue
+// writes C rows with fully coalesced 128-byte warp stores.
+//
+// Roles (192 threads, one CTA per SM, persistent):
+//   warp 0      TMA producer: per stored block one A-block load plus 2*GROUPS B boxes into a
+//               STAGES-deep shared-memory ring, full/empty mbarriers with phase bits.
+//   warp 1      MMA issuer: one thread issues tcgen05.mma into one of two TMEM accumulator
+//               buffers; tcgen05.commit frees the ring slot / publishes the accumulator.
+//   warps 2-5   epilogue: tcgen05.ld -> registers -> global C (zeros for empty block-rows),
+//               overlapping the next tile's MMAs thanks to the second TMEM buffer.
+// Tiles are enumerated slab-major (a slab = a group of token tiles whose B rows fit in L2)
+// and, inside a slab, block-rows longest first; CTA c takes tiles c, c + grid, ...
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace spmm {
+
+namespace {
+
+template <int B, int GROUPS, int STAGES>
+struct BcsrCfg {
+    static constexpr int kBnT = 128 * GROUPS;
+    static constexpr int kNBox = 2 * GROUPS;                 // 64-token boxes per stage
+    static constexpr int kBoxBytes = B * 128;                // b k-rows x 128 B
+    static constexpr int kDenseBytes = kNBox * kBoxBytes;
+    static constexpr int kABytes = B * B * 2;
+    static constexpr int kStageBytes = ((kDenseBytes + kABytes + 1023) / 1024) * 1024;
+    static constexpr int kARowBytes = (B < 64 ? B : 64) * 2;
+    static constexpr uint32_t kASwizzle = kARowBytes == 128 ? SWZ_128B : (kARowBytes == 64 ? SWZ_64B : SWZ_32B);
+    static constexpr int kAccCols = GROUPS * B;
+    static constexpr int kTmemCols = (2 * kAccCols <= 32) ? 32 : (2 * kAccCols <= 64 ? 64 : (2 * kAccCols <= 128 ? 128 : (2 * kAccCols <= 256 ? 256 : 512)));
+    static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+    static_assert(2 * kAccCols <= 512, "accumulators exceed TMEM");
+};
+
+struct TileCoord { int I; int t; };
+
+__device__ __forceinline__ TileCoord tile_coord(int64_t L, const BcsrParams& p) {
+    const int64_t per_slab = static_cast<int64_t>(p.nbr) * p.slab_w;
+    const int s = static_cast<int>(L / per_slab);
+    const int64_t u = L - s * per_slab;
+    const int t0 = s * p.slab_w;
+    const int w = min(p.slab_w, p.n_tt - t0);
+    TileCoord c;
+    c.I = p.row_order[static_cast<int>(u / w)];
+    c.t = t0 + static_cast<int>(u % w);
+    return c;
+}
+
+template <int B, int GROUPS, int STAGES, int FMT>
+__global__ void __launch_bounds__(192, 1)
+bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const BcsrParams p) {
+    using Cfg = BcsrCfg<B, GROUPS, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * Cfg::kStageBytes);
+    // barrier slots: full[STAGES], empty[STAGES], acc_full[2], acc_empty[2]
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+    auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+    auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * STAGES + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * STAGES + 5);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    WaitCtl ctl{abort_flag, p.status, p.wait_limit_ns};
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(accf_bar(a), 1); mbar_init(acce_bar(a), 4); }
+        *abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tmap(&tmA);
+        prefetch_tmap(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int64_t N = p.N;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t L = blockIdx.x; L < p.total_tiles && ok; L += gridDim.x) {
+                const TileCoord tc = tile_coord(L, p);
+                const int n0 = tc.t * Cfg::kBnT;
+                const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
+                const int nbox = (nvalid + 63) >> 6;
+                const uint32_t tx = Cfg::kABytes + nbox * Cfg::kBoxBytes;
+                const int pb = p.block_row_ptr[tc.I], pe = p.block_row_ptr[tc.I + 1];
+                for (int q = pb; q < pe; ++q, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, ctl, 1)) { ok = false; break; }
+                    const uint32_t sb = smem_base + s * Cfg::kStageBytes;
+                    mbar_arrive_expect_tx(full_bar(s), tx);
+                    const int J = p.block_col_idx[q];
+                    if constexpr (B <= 64) {
+                        tma_load_2d(sb + Cfg::kDenseBytes, &tmA, full_bar(s), 0, q * B);
+                    } else {
+                        tma_load_2d(sb + Cfg::kDenseBytes, &tmA, full_bar(s), 0, q * B);
+                        tma_load_2d(sb + Cfg::kDenseBytes + B * 128, &tmA, full_bar(s), 64, q * B);
+                    }
+                    for (int x = 0; x < nbox; ++x)
+                        tma_load_2d(sb + x * Cfg::kBoxBytes, &tmB, full_bar(s), n0 + x * 64, J * B);
+                }
+            }
+            if (!ok) {
+                // leave no bulk copy in flight: wait (bounded) for the fills already issued
+                const uint32_t first = it > STAGES ? it - STAGES : 0;
+                for (uint32_t j = first; j < it; ++j) {
+                    const uint64_t t0 = globaltimer_ns();
+                    while (!mbar_try_wait(full_bar(j % STAGES), (j / STAGES) & 1u) &&
+                           globaltimer_ns() - t0 < 2000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(FMT, 128, B, 1, 0);
+            uint32_t it = 0, tile_i = 0;
+            bool ok = true;
+            for (int64_t L = blockIdx.x; L < p.total_tiles && ok; L += gridDim.x, ++tile_i) {
+                const TileCoord tc = tile_coord(L, p);
+                const int n0 = tc.t * Cfg::kBnT;
+                const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
+                const int ngrp = (nvalid + 127) >> 7;
+                const int acc = tile_i & 1;
+                const uint32_t aph = (tile_i >> 1) & 1u;
+                if (!mbar_wait(acce_bar(acc), aph ^ 1u, ctl, 2)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d0 = tmem_base + acc * Cfg::kAccCols;
+                const int pb = p.block_row_ptr[tc.I], pe = p.block_row_ptr[tc.I + 1];
+                for (int q = pb; q < pe; ++q, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, ctl, 3)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t sb = smem_base + s * Cfg::kStageBytes;
+                    const uint32_t ab = sb + Cfg::kDenseBytes;
+#pragma unroll
+                    for (int ks = 0; ks < B / 16; ++ks) {
+                        uint32_t a_addr;
+                        if constexpr (B <= 64) a_addr = ab + ks * 32;
+                        else a_addr = ab + (ks >> 2) * (B * 128) + (ks & 3) * 32;
+                        const uint64_t bdesc = make_smem_desc(a_addr, 16, 8 * Cfg::kARowBytes, Cfg::kASwizzle);
+                        const uint32_t accum = (q > pb || ks > 0) ? 1u : 0u;
+                        for (int g = 0; g < ngrp; ++g) {
+                            const uint64_t adesc = make_smem_desc(sb + g * 2 * Cfg::kBoxBytes + ks * 2048,
+                                                                  Cfg::kBoxBytes, 1024, SWZ_128B);
+                            umma_ss<false>(d0 + g * B, adesc, bdesc, idesc, accum);
+                        }
+                    }
+                    tc_commit(empty_bar(s));
+                }
+                if (!ok) break;
+                if (pe > pb) tc_commit(accf_bar(acc));
+                else mbar_arrive(accf_bar(acc));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int qd = warp & 3;                    // TMEM lane quarter this warp may read
+        uint32_t tile_i = 0;
+        bool ok = true;
+        for (int64_t L = blockIdx.x; L < p.total_tiles && ok; L += gridDim.x, ++tile_i) {
+            const TileCoord tc = tile_coord(L, p);
+            const int n0 = tc.t * Cfg::kBnT;
+            const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
+            const int ngrp = (nvalid + 127) >> 7;
+            const int acc = tile_i & 1;
+            const uint32_t aph = (tile_i >> 1) & 1u;
+            const bool has_blocks = p.block_row_ptr[tc.I + 1] > p.block_row_ptr[tc.I];
+            if (!mbar_wait(accf_bar(acc), aph, ctl, 4)) { ok = false; break; }
+            tc_fence_after_sync();
+            const int64_t row0 = static_cast<int64_t>(tc.I) * B;
+            const int rows = static_cast<int>(min_i64(B, p.m - row0));
+            for (int g = 0; g < ngrp; ++g) {
+                const int n = n0 + g * 128 + qd * 32 + lane;
+                const bool nok = n < N;
+                float* cp = p.C + row0 * N + n;
+#pragma unroll
+                for (int c0 = 0; c0 < B; c0 += 32) {
+                    constexpr int W = B < 32 ? B : 32;
+                    uint32_t v[32];
+                    if (has_blocks) {
+                        const uint32_t ta = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) +
+                                            acc * Cfg::kAccCols + g * B + c0;
+                        if constexpr (W == 16) {
+                            uint32_t v16[16];
+                            tmem_ld_x16(ta, v16);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) v[j] = v16[j];
+                        } else {
+                            tmem_ld_x32(ta, v);
+                            tmem_ld_wait();
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < W; ++j) v[j] = 0u;
+                    }
+                    if (nok) {
+#pragma unroll
+                        for (int j = 0; j < W; ++j)
+                            if (c0 + j < rows) cp[static_cast<int64_t>(c0 + j) * N] = __uint_as_float(v[j]);
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acce_bar(acc));
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    }
+}
+
+template <int B, int GROUPS, int STAGES, int FMT>
+cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const BcsrParams& p, int grid,
+                       cudaStream_t stream) {
+    using Cfg = BcsrCfg<B, GROUPS, STAGES>;
+    auto kfn = bcsr_spmm_kernel<B, GROUPS, STAGES, FMT>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    kfn<<<grid, 192, Cfg::kSmemBytes, stream>>>(tmA, tmB, p);
+    return cudaGetLastError();
+}
+
+template <int FMT>
+cudaError_t launch_fmt(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                       const BcsrParams& p, int grid, cudaStream_t stream) {
+    switch (b * 10 + groups) {
+        case 161: return launch_one<16, 1, 8, FMT>(tmA, tmB, p, grid, stream);
+        case 162: return launch_one<16, 2, 8, FMT>(tmA, tmB, p, grid, stream);
+        case 164: return launch_one<16, 4, 8, FMT>(tmA, tmB, p, grid, stream);
+        case 321: return launch_one<32, 1, 8, FMT>(tmA, tmB, p, grid, stream);
+        case 322: return launch_one<32, 2, 8, FMT>(tmA, tmB, p, grid, stream);
+        case 324: return launch_one<32, 4, 6, FMT>(tmA, tmB, p, grid, stream);
+        case 641: return launch_one<64, 1, 8, FMT>(tmA, tmB, p, grid, stream);
+        case 642: return launch_one<64, 2, 5, FMT>(tmA, tmB, p, grid, stream);
+        case 644: return launch_one<64, 4, 3, FMT>(tmA, tmB, p, grid, stream);
+        case 1281: return launch_one<128, 1, 3, FMT>(tmA, tmB, p, grid, stream);
+        case 1282: return launch_one<128, 2, 2, FMT>(tmA, tmB, p, grid, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+int bcsr_token_groups_max(int b) { return b == 128 ? 2 : 4; }
+
+cudaError_t launch_bcsr(int dtype, int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                        const BcsrParams& p, int grid, cudaStream_t stream) {
+    if (dtype == 1) return launch_fmt<0>(b, groups, tmA, tmB, p, grid, stream);   // fp16
+    if (dtype == 0) return launch_fmt<1>(b, groups, tmA, tmB, p, grid, stream);   // bf16
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace spmm

@@ -1,0 +1,235 @@
+// Host-side format construction (Sec. 2.3 "Sparse Formats", Sec. 3.3 task split).
+#include "format.h"
+
+#include <algorithm>
+#include <cstring>
+#include <numeric>
+
+#include "spmm_b200.h"
+
+namespace spmm {
+
+static inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+int validate_csr(const CsrView& a) {
+    if (a.m < 0 || a.k < 0 || !a.row_ptr) return SPMM_ERR_INVALID_ARG;
+    if (a.row_ptr[0] != 0) return SPMM_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < a.m; ++i)
+        if (a.row_ptr[i + 1] < a.row_ptr[i]) return SPMM_ERR_INVALID_ARG;
+    if (a.row_ptr[a.m] != a.nnz) return SPMM_ERR_INVALID_ARG;
+    if (a.nnz > 0 && (!a.col_idx || !a.vals)) return SPMM_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < a.m; ++i) {
+        int64_t prev = -1;
+        for (int64_t p = a.row_ptr[i]; p < a.row_ptr[i + 1]; ++p) {
+            const int64_t c = a.col_idx[p];
+            if (c < 0 || c >= a.k) return SPMM_ERR_OUT_OF_RANGE;
+            if (c <= prev) return SPMM_ERR_UNSORTED;
+            prev = c;
+        }
+    }
+    return SPMM_OK;
+}
+
+int coo_to_csr(int64_t m, int64_t k, int64_t nnz, const int32_t* rows, const int32_t* cols,
+               const uint8_t* vals, int es, CsrOwned* out) {
+    if (m < 0 || k < 0 || nnz < 0) return SPMM_ERR_INVALID_ARG;
+    if (nnz > 0 && (!rows || !cols || !vals)) return SPMM_ERR_INVALID_ARG;
+    for (int64_t p = 0; p < nnz; ++p)
+        if (rows[p] < 0 || rows[p] >= m || cols[p] < 0 || cols[p] >= k) return SPMM_ERR_OUT_OF_RANGE;
+    std::vector<int64_t> perm(static_cast<size_t>(nnz));
+    std::iota(perm.begin(), perm.end(), int64_t{0});
+    std::stable_sort(perm.begin(), perm.end(), [&](int64_t x, int64_t y) {
+        if (rows[x] != rows[y]) return rows[x] < rows[y];
+        return cols[x] < cols[y];
+    });
+    for (int64_t p = 1; p < nnz; ++p)
+        if (rows[perm[p]] == rows[perm[p - 1]] && cols[perm[p]] == cols[perm[p - 1]])
+            return SPMM_ERR_UNSORTED;
+    out->row_ptr.assign(static_cast<size_t>(m) + 1, 0);
+    out->col_idx.resize(static_cast<size_t>(nnz));
+    out->vals.resize(static_cast<size_t>(nnz) * es);
+    for (int64_t p = 0; p < nnz; ++p) {
+        const int64_t s = perm[p];
+        out->row_ptr[static_cast<size_t>(rows[s]) + 1]++;
+        out->col_idx[p] = cols[s];
+        std::memcpy(&out->vals[static_cast<size_t>(p) * es], vals + static_cast<size_t>(s) * es, es);
+    }
+    for (int64_t i = 0; i < m; ++i) out->row_ptr[i + 1] += out->row_ptr[i];
+    return SPMM_OK;
+}
+
+// ----------------------------------------------------------------------------- BCSR
+
+int build_bcsr(const CsrView& a, int b, BcsrHost* out) {
+    if (b != 16 && b != 32 && b != 64 && b != 128) return SPMM_ERR_UNSUPPORTED;
+    out->b = b;
+    const int64_t nbr = cdiv(a.m, b), nbc = cdiv(a.k, b);
+    out->nbr = nbr;
+    out->nbc = nbc;
+    out->block_row_ptr.assign(static_cast<size_t>(nbr) + 1, 0);
+    out->block_col_idx.clear();
+
+    // pass 1: which block columns each block-row touches (structural: any stored entry)
+    std::vector<int64_t> stamp(static_cast<size_t>(nbc), -1);
+    std::vector<uint8_t> col_used(static_cast<size_t>(nbc), 0);
+    std::vector<int32_t> found;
+    for (int64_t I = 0; I < nbr; ++I) {
+        found.clear();
+        const int64_t r1 = std::min<int64_t>(a.m, (I + 1) * b);
+        for (int64_t i = I * b; i < r1; ++i)
+            for (int64_t p = a.row_ptr[i]; p < a.row_ptr[i + 1]; ++p) {
+                const int64_t J = a.col_idx[p] / b;
+                if (stamp[J] != I) {
+                    stamp[J] = I;
+                    found.push_back(static_cast<int32_t>(J));
+                }
+            }
+        std::sort(found.begin(), found.end());
+        for (int32_t J : found) col_used[J] = 1;
+        out->block_col_idx.insert(out->block_col_idx.end(), found.begin(), found.end());
+        if (out->block_col_idx.size() >= (size_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
+        out->block_row_ptr[I + 1] = static_cast<int32_t>(out->block_col_idx.size());
+    }
+    const int64_t nnzb = static_cast<int64_t>(out->block_col_idx.size());
+    out->nnzb = nnzb;
+    out->distinct_bcols = std::count(col_used.begin(), col_used.end(), uint8_t{1});
+
+    // pass 2: scatter the values into their dense tiles
+    const size_t tile_bytes = static_cast<size_t>(b) * b * a.es;
+    out->blocks.assign(static_cast<size_t>(nnzb) * tile_bytes, 0);
+    std::vector<int32_t> slot_of(static_cast<size_t>(nbc), -1);
+    for (int64_t I = 0; I < nbr; ++I) {
+        for (int32_t p = out->block_row_ptr[I]; p < out->block_row_ptr[I + 1]; ++p)
+            slot_of[out->block_col_idx[p]] = p;
+        const int64_t r1 = std::min<int64_t>(a.m, (I + 1) * b);
+        for (int64_t i = I * b; i < r1; ++i)
+            for (int64_t p = a.row_ptr[i]; p < a.row_ptr[i + 1]; ++p) {
+                const int64_t c = a.col_idx[p];
+                const size_t dst = static_cast<size_t>(slot_of[c / b]) * tile_bytes +
+                                   (static_cast<size_t>(i - I * b) * b + static_cast<size_t>(c % b)) * a.es;
+                std::memcpy(&out->blocks[dst], a.vals + static_cast<size_t>(p) * a.es, a.es);
+            }
+    }
+
+    // schedule: block-rows with the most stored blocks first, ties by index
+    out->row_order.resize(static_cast<size_t>(nbr));
+    std::iota(out->row_order.begin(), out->row_order.end(), 0);
+    std::stable_sort(out->row_order.begin(), out->row_order.end(), [&](int32_t x, int32_t y) {
+        const int32_t lx = out->block_row_ptr[x + 1] - out->block_row_ptr[x];
+        const int32_t ly = out->block_row_ptr[y + 1] - out->block_row_ptr[y];
+        return lx > ly;
+    });
+    out->n_empty = 0;
+    for (int64_t I = 0; I < nbr; ++I)
+        if (out->block_row_ptr[I + 1] == out->block_row_ptr[I]) out->n_empty++;
+    return SPMM_OK;
+}
+
+// ----------------------------------------------------------------------------- WCSR
+
+int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_spans, WcsrHost* out) {
+    if (wh != 16) return SPMM_ERR_UNSUPPORTED;
+    if (b_col * a.es != 32) return SPMM_ERR_UNSUPPORTED;
+    if (T <= 0 || T % b_col != 0 || n_spans <= 0) return SPMM_ERR_INVALID_ARG;
+    out->wh = wh;
+    out->b_col = b_col;
+    out->T = T;
+    const int64_t nwin = cdiv(a.m, wh);
+    out->nwin = nwin;
+    out->window_row_ptr.assign(static_cast<size_t>(nwin) + 1, 0);
+    out->window_col_idx.clear();
+
+    // pass 1: per window, the ascending union of its rows' columns, padded with -1
+    std::vector<int32_t> cols;
+    std::vector<uint8_t> col_used(static_cast<size_t>(a.k), 0);
+    int64_t P = 0;
+    for (int64_t w = 0; w < nwin; ++w) {
+        const int64_t r0 = w * wh, r1 = std::min<int64_t>(a.m, r0 + wh);
+        cols.assign(a.col_idx + a.row_ptr[r0], a.col_idx + a.row_ptr[r1]);
+        std::sort(cols.begin(), cols.end());
+        cols.erase(std::unique(cols.begin(), cols.end()), cols.end());
+        const int64_t len = cdiv(static_cast<int64_t>(cols.size()), b_col) * b_col;
+        if (P + len >= (int64_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
+        for (int32_t c : cols) col_used[c] = 1;
+        out->window_col_idx.insert(out->window_col_idx.end(), cols.begin(), cols.end());
+        out->window_col_idx.insert(out->window_col_idx.end(), static_cast<size_t>(len) - cols.size(), -1);
+        P += len;
+        out->window_row_ptr[w + 1] = static_cast<int32_t>(P);
+    }
+    out->P = P;
+    out->distinct_cols = std::count(col_used.begin(), col_used.end(), uint8_t{1});
+
+    // pass 2: values, straight into the packed device layout
+    out->packed.assign(static_cast<size_t>(P) * wh * a.es, 0);
+    for (int64_t w = 0; w < nwin; ++w) {
+        const int64_t r0 = w * wh, r1 = std::min<int64_t>(a.m, r0 + wh);
+        const int32_t* wc = out->window_col_idx.data() + out->window_row_ptr[w];
+        const int64_t base = out->window_row_ptr[w];
+        for (int64_t i = r0; i < r1; ++i) {
+            int64_t q = 0;   // both lists ascend: walk them together
+            for (int64_t p = a.row_ptr[i]; p < a.row_ptr[i + 1]; ++p) {
+                const int32_t c = a.col_idx[p];
+                while (wc[q] != c) ++q;
+                std::memcpy(&out->packed[wcsr_packed_offset(wh, b_col, a.es, static_cast<int>(i - r0), base + q)],
+                            a.vals + static_cast<size_t>(p) * a.es, a.es);
+            }
+        }
+    }
+
+    // split plan: consecutive chunks of T columns; a window with one chunk writes C itself
+    out->tasks.clear();
+    out->merge_window.clear();
+    out->merge_first.clear();
+    out->merge_nparts.clear();
+    out->n_empty = out->n_split = out->n_slots = 0;
+    std::vector<int32_t> empty_windows;
+    for (int64_t w = 0; w < nwin; ++w) {
+        const int32_t len = out->window_row_ptr[w + 1] - out->window_row_ptr[w];
+        if (len == 0) {
+            empty_windows.push_back(static_cast<int32_t>(w));
+            continue;
+        }
+        const int32_t nchunk = static_cast<int32_t>(cdiv(len, T));
+        if (nchunk > 1) {
+            out->merge_window.push_back(static_cast<int32_t>(w));
+            out->merge_first.push_back(static_cast<int32_t>(out->n_slots));
+            out->merge_nparts.push_back(nchunk);
+            out->n_split++;
+        }
+        for (int32_t c = 0; c < nchunk; ++c) {
+            WcsrTask t;
+            t.window = static_cast<int32_t>(w);
+            t.q0 = c * T;
+            t.count = std::min(T, len - c * T);
+            t.slot = nchunk > 1 ? static_cast<int32_t>(out->n_slots++) : -1;
+            out->tasks.push_back(t);
+        }
+    }
+    out->n_empty = static_cast<int64_t>(empty_windows.size());
+    for (int32_t w : empty_windows) {
+        out->merge_window.push_back(w);
+        out->merge_first.push_back(-1);
+        out->merge_nparts.push_back(0);
+    }
+
+    // spans: cut the task list into n_spans consecutive ranges of near-equal cost
+    // (cost of a task = its columns + kTaskFixedCost); span j ends at the first task where
+    // the running cost reaches (j+1)/n_spans of the total.
+    const int64_t ntasks = static_cast<int64_t>(out->tasks.size());
+    int64_t total = 0;
+    for (const WcsrTask& t : out->tasks) total += t.count + kTaskFixedCost;
+    out->spans.assign(static_cast<size_t>(n_spans) + 1, 0);
+    int64_t run = 0, ti = 0;
+    for (int j = 0; j < n_spans; ++j) {
+        // smallest ti with run * n_spans >= (j+1) * total
+        while (ti < ntasks && run * n_spans < static_cast<int64_t>(j + 1) * total) {
+            run += out->tasks[ti].count + kTaskFixedCost;
+            ++ti;
+        }
+        out->spans[j + 1] = static_cast<int32_t>(ti);
+    }
+    out->spans[n_spans] = static_cast<int32_t>(ntasks);
+    return SPMM_OK;
+}
+
+}  // namespace spmm

@@ -1,0 +1,76 @@
+// Host-side format construction: CSR/COO canonicalisation, BCSR block mask and
+// packing, WCSR window condensation and column remap, long-window split plan and
+// the static schedules (Sec. 2.3 formats; Sec. 3.3 task decomposition).
+#pragma once
+
+#include <cstdint>
+#include <vector>
+
+namespace spmm {
+
+struct CsrView {
+    int64_t m = 0, k = 0, nnz = 0;
+    const int64_t* row_ptr = nullptr;
+    const int32_t* col_idx = nullptr;
+    const uint8_t* vals = nullptr;   // nnz * es bytes
+    int es = 2;                      // element size in bytes
+};
+
+// Owning CSR, produced from COO.
+struct CsrOwned {
+    std::vector<int64_t> row_ptr;
+    std::vector<int32_t> col_idx;
+    std::vector<uint8_t> vals;
+};
+
+struct BcsrHost {
+    int b = 0;
+    int64_t nbr = 0, nbc = 0, nnzb = 0, n_empty = 0, distinct_bcols = 0;
+    std::vector<int32_t> block_row_ptr;   // [nbr+1]
+    std::vector<int32_t> block_col_idx;   // [nnzb], ascending inside a block-row
+    std::vector<uint8_t> blocks;          // [nnzb][b][b] * es, zero filled
+    std::vector<int32_t> row_order;       // [nbr] block-rows, most stored blocks first (stable)
+};
+
+struct WcsrTask { int32_t window, q0, count, slot; };
+
+struct WcsrHost {
+    int wh = 0, b_col = 0, T = 0;
+    int64_t nwin = 0, P = 0, n_empty = 0, n_split = 0, n_slots = 0, distinct_cols = 0;
+    std::vector<int32_t> window_row_ptr;  // [nwin+1], in columns
+    std::vector<int32_t> window_col_idx;  // [P], -1 on pads
+    // Device-private packing of values[wh][P]: one chunk of wh x b_col values per group of
+    // b_col consecutive padded columns; inside a chunk the order is
+    // [16-byte K half (2)][8-row group (wh/8)][row in group (8)][16 bytes], which is the
+    // un-swizzled K-major core-matrix layout tcgen05.mma reads.  chunk bytes = wh * 32.
+    std::vector<uint8_t> packed;
+    std::vector<WcsrTask> tasks;          // window order; chunks of a window consecutive
+    std::vector<int32_t> spans;           // [n_spans+1] task ranges, balanced by cost
+    // finalisation lists: windows whose C rows the merge kernel writes
+    std::vector<int32_t> merge_window;    // split windows then empty windows
+    std::vector<int32_t> merge_first;     // first slot (split) or -1 (empty)
+    std::vector<int32_t> merge_nparts;    // number of slots (split) or 0 (empty)
+};
+
+// All return 0 or a negative spmm_status_t value.
+int validate_csr(const CsrView& a);
+int coo_to_csr(int64_t m, int64_t k, int64_t nnz, const int32_t* rows, const int32_t* cols,
+               const uint8_t* vals, int es, CsrOwned* out);
+int build_bcsr(const CsrView& a, int b, BcsrHost* out);
+int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_spans, WcsrHost* out);
+
+// Byte offset of element (row r, padded column q) inside the packed WCSR value array.
+inline size_t wcsr_packed_offset(int wh, int b_col, int es, int r, int64_t q) {
+    const int64_t chunk = q / b_col;
+    const int c = static_cast<int>(q % b_col);
+    const int byte_in_row = c * es;                  // 0 .. 31
+    return static_cast<size_t>(chunk) * (static_cast<size_t>(wh) * 32) +
+           static_cast<size_t>(byte_in_row / 16) * (static_cast<size_t>(wh) * 16) +
+           static_cast<size_t>(r / 8) * 128 + static_cast<size_t>(r % 8) * 16 +
+           static_cast<size_t>(byte_in_row % 16);
+}
+
+// Cost, in column equivalents, that the span partition charges per task on top of its columns.
+constexpr int kTaskFixedCost = 32;
+
+}  // namespace spmm

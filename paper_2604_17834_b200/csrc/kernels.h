@@ -1,0 +1,66 @@
+// Launch interfaces between the C-ABI layer (api.cu) and the kernels.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace spmm {
+
+struct BcsrParams {
+    const int32_t* block_row_ptr;
+    const int32_t* block_col_idx;
+    const int32_t* row_order;
+    float* C;
+    int64_t m, N;
+    int32_t nbr;        // block-rows
+    int32_t n_tt;       // token tiles = ceil(N / (128 * groups))
+    int32_t slab_w;     // token tiles per L2 slab
+    int64_t total_tiles;
+    int* status;
+    uint64_t wait_limit_ns;
+};
+
+// dtype: 0 bf16, 1 fp16.  groups: token tile = 128 * groups columns of B (1, 2 or 4).
+cudaError_t launch_bcsr(int dtype, int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                        const BcsrParams& p, int grid, cudaStream_t stream);
+int bcsr_token_groups_max(int b);
+
+// Device task descriptor of the WCSR kernel (one per sub-task of the split plan).
+struct WcsrDevTask {
+    int32_t col_begin;   // absolute position of the task's first padded column
+    int32_t count;       // columns (multiple of b_col)
+    int32_t window;
+    int32_t slot;        // partial tile index, or -1: write C directly
+};
+
+struct WcsrParams {
+    const WcsrDevTask* tasks;
+    const int32_t* spans;        // [n_spans+1]
+    const int32_t* col_idx;      // window_col_idx [P]
+    const uint8_t* packed;       // packed A values
+    const void* B;               // k x N row-major
+    float* C;
+    float* partial;              // [n_slots][16][N]
+    int64_t m, N;
+    int32_t n_spans;
+    int32_t n_tt;                // token tiles = ceil(N / (128 * groups))
+    int* status;
+    uint64_t wait_limit_ns;
+};
+
+// dtype: 0 bf16, 1 fp16, 2 tf32.  groups: 1 or 2.
+cudaError_t launch_wcsr(int dtype, int groups, const WcsrParams& p, int grid, cudaStream_t stream);
+
+struct MergeParams {
+    const int32_t* window;   // [n] windows the merge writes
+    const int32_t* first;    // first slot or -1
+    const int32_t* nparts;   // slots to add (0 = zero fill)
+    const float* partial;
+    float* C;
+    int64_t m, N;
+    int32_t n;
+};
+cudaError_t launch_wcsr_merge(const MergeParams& p, cudaStream_t stream);
+
+}  // namespace spmm

@@ -1,0 +1,341 @@
+// WCSR SpMM kernel for sm_100a (Sec. 3.2 - 3.3 of the paper, re-designed for Blackwell).
+//
+// Work item: one sub-task of the split plan (a run of `count` condensed columns of one
+// 16-row window) times BN_T = 128 * GROUPS columns of B ("tokens").  It accumulates
+//     D[n, r] += sum_q  B[window_col_idx[q], n0 + n] * values[r, q]
+// with the tokens on the 128 TMEM lanes (MMA M side; the gathered B rows are written to
+// shared memory in the MN-major 128-byte-swizzled layout tcgen05.mma reads) and the 16
+// window rows as the MMA N side (operand = the packed window tile, K-major, un-swizzled).
+//
+// Roles (288 threads, persistent CTAs):
+//   warps 0-3   gather producers: per stage read KT column indices and copy the matching
+//               B rows with 16-byte cp.async (zero fill for -1 pads) into a STAGES-deep
+//               ring; thread 0 also bulk-copies the contiguous packed A tile.  A stage is
+//               published LAG fills later (wait_group + proxy fence + mbarrier arrive), so
+//               LAG + 1 stages of loads stay in flight per thread.
+//   warp 4      MMA issuer (one thread): count / b_col tcgen05.mma per group and stage.
+//   warps 5-8   epilogue: tcgen05.ld, release the TMEM buffer, store to C (unsplit window)
+//               or to the task's partial tile (split window).
+// CTA c walks spans c, c + grid, ... of the cost-balanced span list; tasks inside a span are
+// consecutive, so neighbouring windows (which share B rows in banded matrices) run together.
+// Split windows are summed in slot order by wcsr_merge_kernel, which also zero-fills the C
+// rows of empty windows: results are run-to-run identical.
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace spmm {
+
+namespace {
+
+constexpr int kWH = 16;
+constexpr int kProducerThreads = 128;
+constexpr int kNAcc = 4;
+
+template <int ES, int GROUPS, int KT, int STAGES>
+struct WcsrCfg {
+    static constexpr int kE16 = 16 / ES;                    // elements per 16-byte chunk
+    static constexpr int kKStep = 32 / ES;                  // columns per MMA (= b_col)
+    static constexpr int kBnT = 128 * GROUPS;
+    static constexpr int kRowBytes = kBnT * ES;
+    static constexpr int kCh = kRowBytes / 16;              // 16-byte chunks per gathered row
+    static constexpr int kRpp = kProducerThreads / kCh;     // rows per pass
+    static constexpr int kPasses = KT / kRpp;
+    static constexpr int kAtomStride = KT * 128;            // bytes between MN atoms
+    static constexpr int kAtomsPerGroup = ES;               // 128 tokens * ES / 128 B
+    static constexpr int kDenseBytes = KT * kRowBytes;
+    static constexpr int kABytes = (KT / kKStep) * (kWH * 32);
+    static constexpr int kStageBytes = kDenseBytes + kABytes;
+    static constexpr int kAccCols = GROUPS * kWH;
+    static constexpr int kTmemCols = kNAcc * kAccCols < 32 ? 32 : kNAcc * kAccCols;
+    static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 + 256;
+    static_assert(kCh <= kProducerThreads && kProducerThreads % kCh == 0, "chunk mapping");
+    static_assert(KT % 8 == 0 && KT % kRpp == 0 && KT % kKStep == 0, "stage shape");
+    static_assert(kStageBytes % 1024 == 0, "stage alignment");
+};
+
+template <int ES, int FMT, int GROUPS, int KT, int STAGES, int LAG>
+__global__ void __launch_bounds__(288)
+wcsr_spmm_kernel(const WcsrParams p) {
+    using Cfg = WcsrCfg<ES, GROUPS, KT, STAGES>;
+    static_assert(LAG >= 1 && LAG < STAGES, "publish lag must leave a free stage");
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * Cfg::kStageBytes);
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+    auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+    auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + kNAcc + a); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * STAGES + 2 * kNAcc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * STAGES + 2 * kNAcc + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    WaitCtl ctl{abort_flag, p.status, p.wait_limit_ns};
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), kProducerThreads); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < kNAcc; ++a) { mbar_init(accf_bar(a), 1); mbar_init(acce_bar(a), 4); }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 4) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    const int64_t N = p.N;
+
+    if (warp < 4) {
+        // ------------------------------------------------------------------ gather producers
+        const int tid = threadIdx.x;
+        const int c = tid % Cfg::kCh;              // my 16-byte chunk inside a gathered row
+        const int rsub = tid / Cfg::kCh;           // my row inside a pass
+        const uint32_t dst_c = (c >> 3) * Cfg::kAtomStride;
+        const uint8_t* Bp = static_cast<const uint8_t*>(p.B);
+        uint32_t it = 0;
+        bool ok = true;
+        for (int sp = blockIdx.x; sp < p.n_spans && ok; sp += gridDim.x) {
+            const int t_end = p.spans[sp + 1];
+            for (int t = p.spans[sp]; t < t_end && ok; ++t) {
+                const WcsrDevTask task = p.tasks[t];
+                for (int tt = 0; tt < p.n_tt && ok; ++tt) {
+                    const int n0 = tt * Cfg::kBnT;
+                    const bool chunk_ok = n0 + c * Cfg::kE16 < N;
+                    const size_t col_byte = (static_cast<size_t>(n0) + c * Cfg::kE16) * ES;
+                    for (int done = 0; done < task.count; done += KT, ++it) {
+                        const int s = it % STAGES;
+                        const uint32_t ph = (it / STAGES) & 1u;
+                        const int q = task.col_begin + done;
+                        const int cnt = min(KT, task.count - done);
+                        if (!mbar_wait(empty_bar(s), ph ^ 1u, ctl, 11)) { ok = false; break; }
+                        const uint32_t sb = smem_base + s * Cfg::kStageBytes;
+                        if (tid == 0) {
+                            const uint32_t abytes = (cnt / Cfg::kKStep) * (kWH * 32);
+                            mbar_expect_tx(full_bar(s), abytes);
+                            bulk_load_1d(sb + Cfg::kDenseBytes,
+                                         p.packed + static_cast<size_t>(q / Cfg::kKStep) * (kWH * 32),
+                                         abytes, full_bar(s));
+                        }
+                        if (chunk_ok) {
+                            int idx[Cfg::kPasses];
+#pragma unroll
+                            for (int ps = 0; ps < Cfg::kPasses; ++ps) {
+                                const int r = ps * Cfg::kRpp + rsub;
+                                idx[ps] = r < cnt ? __ldg(p.col_idx + q + r) : -2;
+                            }
+#pragma unroll
+                            for (int ps = 0; ps < Cfg::kPasses; ++ps) {
+                                const int r = ps * Cfg::kRpp + rsub;
+                                if (idx[ps] != -2) {
+                                    uint32_t dst = sb + dst_c + r * 128;
+                                    if constexpr (ES == 2) {
+                                        // 128-byte swizzle: 16-byte chunk index ^= row % 8
+                                        dst += ((c & 7) ^ (r & 7)) << 4;
+                                    } else {
+                                        // 128-byte swizzle with 32-byte atoms (the only MN-major
+                                        // layout for 32-bit operands): 32-byte chunk index ^= row % 4
+                                        dst += ((((c & 7) >> 1) ^ (r & 3)) << 5) + ((c & 1) << 4);
+                                    }
+                                    const bool valid = idx[ps] >= 0;
+                                    const uint8_t* src = Bp + (valid ? static_cast<size_t>(idx[ps]) * N * ES + col_byte : 0);
+                                    cp_async_16(dst, src, valid);
+                                }
+                            }
+                        }
+                        cp_async_commit();
+                        if (it >= LAG) {
+                            cp_async_wait<LAG>();
+                            fence_proxy_async_smem();
+                            mbar_arrive(full_bar((it - LAG) % STAGES));
+                        }
+                    }
+                }
+            }
+        }
+        // publish what is still pending (also on the abort path: never leave copies in flight)
+        cp_async_wait<0>();
+        fence_proxy_async_smem();
+        for (uint32_t j = it > LAG ? it - LAG : 0; j < it; ++j) mbar_arrive(full_bar(j % STAGES));
+        if (!ok && tid == 0) {
+            const uint32_t first = it > STAGES ? it - STAGES : 0;
+            for (uint32_t j = first; j < it; ++j) {
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(full_bar(j % STAGES), (j / STAGES) & 1u) &&
+                       globaltimer_ns() - t0 < 2000000ull) {}
+            }
+        }
+    } else if (warp == 4) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(FMT, 128, kWH, 1, 0);
+            uint32_t it = 0, item = 0;
+            bool ok = true;
+            for (int sp = blockIdx.x; sp < p.n_spans && ok; sp += gridDim.x) {
+                const int t_end = p.spans[sp + 1];
+                for (int t = p.spans[sp]; t < t_end && ok; ++t) {
+                    const WcsrDevTask task = p.tasks[t];
+                    for (int tt = 0; tt < p.n_tt && ok; ++tt, ++item) {
+                        const int n0 = tt * Cfg::kBnT;
+                        const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
+                        const int ngrp = (nvalid + 127) >> 7;
+                        const int acc = item % kNAcc;
+                        const uint32_t aph = (item / kNAcc) & 1u;
+                        if (!mbar_wait(acce_bar(acc), aph ^ 1u, ctl, 12)) { ok = false; break; }
+                        tc_fence_after_sync();
+                        const uint32_t d0 = tmem_base + acc * Cfg::kAccCols;
+                        for (int done = 0; done < task.count; done += KT, ++it) {
+                            const int s = it % STAGES;
+                            const uint32_t ph = (it / STAGES) & 1u;
+                            const int cnt = min(KT, task.count - done);
+                            if (!mbar_wait(full_bar(s), ph, ctl, 13)) { ok = false; break; }
+                            tc_fence_after_sync();
+                            const uint32_t sb = smem_base + s * Cfg::kStageBytes;
+                            const int nks = cnt / Cfg::kKStep;
+                            for (int ks = 0; ks < nks; ++ks) {
+                                const uint64_t bdesc = make_smem_desc(sb + Cfg::kDenseBytes + ks * (kWH * 32),
+                                                                      kWH * 16, 128, SWZ_NONE);
+                                const uint32_t accum = (done > 0 || ks > 0) ? 1u : 0u;
+                                for (int g = 0; g < ngrp; ++g) {
+                                    const uint64_t adesc = make_smem_desc(
+                                        sb + g * Cfg::kAtomsPerGroup * Cfg::kAtomStride + ks * (Cfg::kKStep / 8) * 1024,
+                                        Cfg::kAtomStride, ES == 2 ? 1024 : 512, ES == 2 ? SWZ_128B : SWZ_128B_BASE32B);
+                                    umma_ss<FMT == 2>(d0 + g * kWH, adesc, bdesc, idesc, accum);
+                                }
+                            }
+                            tc_commit(empty_bar(s));
+                        }
+                        if (!ok) break;
+                        tc_commit(accf_bar(acc));
+                    }
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int qd = warp & 3;
+        uint32_t item = 0;
+        bool ok = true;
+        for (int sp = blockIdx.x; sp < p.n_spans && ok; sp += gridDim.x) {
+            const int t_end = p.spans[sp + 1];
+            for (int t = p.spans[sp]; t < t_end && ok; ++t) {
+                const WcsrDevTask task = p.tasks[t];
+                float* out;
+                int rows;
+                if (task.slot < 0) {
+                    const int64_t row0 = static_cast<int64_t>(task.window) * kWH;
+                    out = p.C + row0 * N;
+                    rows = static_cast<int>(min_i64(kWH, p.m - row0));
+                } else {
+                    out = p.partial + static_cast<int64_t>(task.slot) * kWH * N;
+                    rows = kWH;
+                }
+                for (int tt = 0; tt < p.n_tt && ok; ++tt, ++item) {
+                    const int n0 = tt * Cfg::kBnT;
+                    const int acc = item % kNAcc;
+                    const uint32_t aph = (item / kNAcc) & 1u;
+                    if (!mbar_wait(accf_bar(acc), aph, ctl, 14)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    uint32_t v[GROUPS][16];
+#pragma unroll
+                    for (int g = 0; g < GROUPS; ++g)
+                        tmem_ld_x16(tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + acc * Cfg::kAccCols + g * kWH, v[g]);
+                    tmem_ld_wait();
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(acce_bar(acc));
+#pragma unroll
+                    for (int g = 0; g < GROUPS; ++g) {
+                        const int n = n0 + g * 128 + qd * 32 + lane;
+                        if (n < N) {
+#pragma unroll
+                            for (int j = 0; j < kWH; ++j)
+                                if (j < rows) out[static_cast<int64_t>(j) * N + n] = __uint_as_float(v[g][j]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 4) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    }
+}
+
+// C rows of split windows = sum of their partial tiles in slot order; C rows of empty
+// windows = 0.  One CTA per listed window.
+__global__ void __launch_bounds__(256)
+wcsr_merge_kernel(const MergeParams p) {
+    const int i = blockIdx.x;
+    const int w = p.window[i];
+    const int first = p.first[i];
+    const int nparts = p.nparts[i];
+    const int64_t N = p.N;
+    const int64_t row0 = static_cast<int64_t>(w) * kWH;
+    const int rows = static_cast<int>(min_i64(kWH, p.m - row0));
+    const int64_t n4 = N >> 2;     // N is a multiple of 4
+    const int64_t total = static_cast<int64_t>(rows) * n4;
+    const float4* part = reinterpret_cast<const float4*>(p.partial);
+    float4* out = reinterpret_cast<float4*>(p.C + row0 * N);
+    for (int64_t e = threadIdx.x; e < total; e += blockDim.x) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < nparts; ++s) {
+            const float4 v = part[static_cast<int64_t>(first + s) * kWH * n4 + e];
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        out[e] = acc;
+    }
+}
+
+template <int ES, int FMT, int GROUPS, int KT, int STAGES, int LAG>
+cudaError_t launch_one(const WcsrParams& p, int sms, cudaStream_t stream) {
+    using Cfg = WcsrCfg<ES, GROUPS, KT, STAGES>;
+    auto kfn = wcsr_spmm_kernel<ES, FMT, GROUPS, KT, STAGES, LAG>;
+    static int occ = 0;
+    if (occ == 0) {
+        cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        int o = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kfn, 288, Cfg::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        // TMEM: every resident CTA holds kTmemCols of the SM's 512 columns
+        o = o < 512 / Cfg::kTmemCols ? o : 512 / Cfg::kTmemCols;
+        occ = o < 1 ? 1 : (o > 2 ? 2 : o);
+    }
+    int grid = sms * occ;
+    if (grid > p.n_spans) grid = p.n_spans;
+    if (grid < 1) return cudaSuccess;
+    kfn<<<grid, 288, Cfg::kSmemBytes, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_wcsr(int dtype, int groups, const WcsrParams& p, int sms, cudaStream_t stream) {
+    if (dtype == 2) {
+        if (groups == 1) return launch_one<4, 2, 1, 32, 6, 3>(p, sms, stream);
+        if (groups == 2) return launch_one<4, 2, 2, 32, 6, 3>(p, sms, stream);
+    } else if (dtype == 1) {
+        if (groups == 1) return launch_one<2, 0, 1, 64, 6, 3>(p, sms, stream);
+        if (groups == 2) return launch_one<2, 0, 2, 64, 6, 3>(p, sms, stream);
+    } else if (dtype == 0) {
+        if (groups == 1) return launch_one<2, 1, 1, 64, 6, 3>(p, sms, stream);
+        if (groups == 2) return launch_one<2, 1, 2, 64, 6, 3>(p, sms, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_wcsr_merge(const MergeParams& p, cudaStream_t stream) {
+    if (p.n <= 0) return cudaSuccess;
+    wcsr_merge_kernel<<<p.n, 256, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace spmm

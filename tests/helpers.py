@@ -1,0 +1,53 @@
+"""Shared pieces of the GPU parity tests: run the CUDA path through the C ABI and
+compare it element by element with the fp64 oracle under the stated bound
+
+    |C_gpu - C_ref| <= tau * sum_k |a_ik b_kj| + 1e-6,
+
+tau = 8e-3 for bf16 / fp16 inputs, 2e-3 for the TF32 path (fp32 accumulation).
+"""
+import numpy as np
+
+from oracle import spmm_ref
+from paper_2604_17834_b200 import workloads as wl
+
+TAU = {"bf16": 8e-3, "fp16": 8e-3, "tf32": 2e-3}
+
+
+def to_device(arr):
+    """numpy storage array -> torch CUDA tensor holding the same bytes."""
+    import torch
+    a = np.ascontiguousarray(arr)
+    if a.dtype == np.uint16:
+        a = a.view(np.int16)
+    return torch.from_numpy(a).cuda()
+
+
+def run_gpu(lib, h, B_storage, m, N, fill=float("nan"), check=True):
+    """One spmm_run on device buffers; C is pre-filled with NaN so unwritten elements show."""
+    import torch
+    Bd = to_device(B_storage)
+    C = torch.full((m, N), fill, dtype=torch.float32, device="cuda")
+    lib.spmm_run(h, Bd.data_ptr(), C.data_ptr(), N, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    if check:
+        lib.spmm_check(h)
+    return C.cpu().numpy()
+
+
+def reference(a, B_storage, dtype, cols=None, rows=None):
+    v64 = wl.widen(a["vals"], dtype)
+    B64 = wl.widen(B_storage if cols is None else B_storage[:, cols], dtype)
+    return spmm_ref(a["row_ptr"], a["col_idx"], v64, B64, rows=rows)
+
+
+def assert_close(C_gpu, C_ref, S, dtype, what=""):
+    assert C_gpu.shape == C_ref.shape
+    assert np.all(np.isfinite(C_gpu)), "%s: %d non-finite / unwritten outputs" % (what, int((~np.isfinite(C_gpu)).sum()))
+    err = np.abs(C_gpu.astype(np.float64) - C_ref)
+    bound = TAU[dtype] * S + 1e-6
+    bad = err > bound
+    if bad.any():
+        i, j = np.unravel_index(np.argmax(err - bound), err.shape)
+        raise AssertionError("%s: %d of %d outside the bound; worst at (%d,%d): gpu %.6g ref %.6g err %.3g bound %.3g"
+                             % (what, int(bad.sum()), err.size, i, j, C_gpu[i, j], C_ref[i, j], err[i, j], bound[i, j]))
+    return float(np.max(err / bound))

@@ -1,0 +1,164 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle,
+element by element on the same seeded inputs.  Sizes span several tiles, ragged
+tails, empty block-rows / windows, split windows, and every supported block size
+and dtype.  Format arrays exported from the device copy are compared bit for bit.
+"""
+import numpy as np
+import pytest
+
+from oracle import formats as F
+from paper_2604_17834_b200 import workloads as wl
+
+from helpers import assert_close, reference, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2604_17834_b200 import binding
+    return binding
+
+
+def _bcsr_case(lib, a, dtype, b, N, Bdist=("uniform", -1.0, 1.0), seed=9):
+    Bs = wl.dense(seed, a["k"], N, Bdist, dtype)
+    h = lib.spmm_bcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], dtype, b)
+    try:
+        f = F.bcsr_from_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], b)
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCK_ROW_PTR, np.int32), f["block_row_ptr"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCK_COL_IDX, np.int32), f["block_col_idx"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCKS, np.uint16), f["blocks"].view(np.uint16).ravel())
+        C = run_gpu(lib, h, Bs, a["m"], N)
+        Cr, S = reference(a, Bs, dtype)
+        worst = assert_close(C, Cr, S, dtype, "bcsr b=%d N=%d" % (b, N))
+        C2 = run_gpu(lib, h, Bs, a["m"], N)
+        assert np.array_equal(C, C2)                   # run-to-run identical
+        return worst
+    finally:
+        lib.spmm_destroy(h)
+
+
+def test_bcsr_tiny_config(lib):
+    """configs[0]: 512 x 512 bf16, 64 x 64 blocks kept w.p. 0.5, B 512 x 256."""
+    a = wl.bcsr_tiny()
+    _bcsr_case(lib, a, "bf16", 64, 256)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp16"])
+@pytest.mark.parametrize("b", [16, 32, 64, 128])
+def test_bcsr_block_sizes(lib, dtype, b):
+    a = wl.bcsr_sweep(300 + b, m=1024, k=768, b=b, density=0.2, dtype=dtype)
+    _bcsr_case(lib, a, dtype, b, 640)                  # 640 = 512 + 128: several token tiles
+
+
+@pytest.mark.parametrize("m,k,b,N", [(500, 300, 64, 200), (130, 70, 32, 72), (1000, 1000, 16, 1032),
+                                      (257, 640, 128, 328), (64, 64, 64, 64)])
+def test_bcsr_ragged_shapes(lib, m, k, b, N):
+    """m, k not multiples of b; N not a multiple of the token tile; scattered entries."""
+    a = wl.random_csr(7 + m, m, k, 0.02, "fp16", empty_rows=tuple(range(min(b, m // 2))))
+    _bcsr_case(lib, a, "fp16", b, N)
+
+
+def test_bcsr_all_empty_and_identity(lib):
+    rp = np.zeros(129, np.int64)
+    a = dict(m=128, k=128, row_ptr=rp, col_idx=np.zeros(0, np.int32), vals=np.zeros(0, np.uint16))
+    Bs = wl.dense(1, 128, 128, ("normal", 0.0, 1.0), "bf16")
+    h = lib.spmm_bcsr_create_csr(128, 128, rp, a["col_idx"], a["vals"], "bf16", 64)
+    assert not run_gpu(lib, h, Bs, 128, 128).any()
+    lib.spmm_destroy(h)
+    one = wl.to_storage(np.ones(128), "bf16")
+    h = lib.spmm_bcsr_create_csr(128, 128, np.arange(129, dtype=np.int64), np.arange(128, dtype=np.int32), one, "bf16", 32)
+    C = run_gpu(lib, h, Bs, 128, 128)
+    assert np.array_equal(C.astype(np.float64), wl.widen(Bs, "bf16"))   # identity: exact
+    lib.spmm_destroy(h)
+
+
+def _wcsr_case(lib, a, dtype, N, T=0, Bdist=("normal", 0.0, 1.0), seed=19):
+    Bs = wl.dense(seed, a["k"], N, Bdist, dtype)
+    h = lib.spmm_wcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], dtype, 16, split_cols=T)
+    try:
+        b_col = 8 if dtype == "tf32" else 16
+        info = lib.spmm_get_info(h, N)
+        f = F.wcsr_from_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], 16, b_col)
+        np_dt = wl.storage_np_dtype(dtype)
+        bits = np.uint32 if dtype == "tf32" else np.uint16
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_ROW_PTR, np.int32), f["window_row_ptr"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_COL_IDX, np.int32), f["window_col_idx"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_VALUES, np_dt).view(bits), f["values"].view(bits).ravel())
+        plan = F.split_plan(f["window_row_ptr"], info["split_cols"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_TASKS, np.int32).reshape(-1, 4), plan)
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_SPANS, np.int32), F.task_spans(plan, info["n_ctas"] * 8))
+        C = run_gpu(lib, h, Bs, a["m"], N)
+        Cr, S = reference(a, Bs, dtype)
+        worst = assert_close(C, Cr, S, dtype, "wcsr %s N=%d T=%d" % (dtype, N, T))
+        C2 = run_gpu(lib, h, Bs, a["m"], N)
+        assert np.array_equal(C, C2)                   # deterministic merge
+        return worst, info
+    finally:
+        lib.spmm_destroy(h)
+
+
+@pytest.mark.parametrize("dtype", ["tf32", "fp16", "bf16"])
+@pytest.mark.parametrize("N", [128, 32, 256, 72])
+def test_wcsr_small(lib, dtype, N):
+    a = wl.random_csr(51, 1000, 900, 0.02, dtype, empty_rows=tuple(range(32, 64)))
+    _, info = _wcsr_case(lib, a, dtype, N, T=64)
+    assert info["n_split"] > 0 and info["n_empty"] >= 2
+
+
+@pytest.mark.parametrize("T", [16, 256, 4096])
+def test_wcsr_split_sizes_agree(lib, T):
+    a = wl.wcsr_irregular(seed=5, m=4000, dtype="tf32")
+    _wcsr_case(lib, a, "tf32", 128, T=T)
+
+
+def test_wcsr_irregular_scaled(lib):
+    """configs[1] recipe at 20,000 rows (the oracle finishes in seconds)."""
+    a = wl.wcsr_irregular(seed=1002, m=20_000, dtype="tf32")
+    worst, _ = _wcsr_case(lib, a, "tf32", 128)
+    assert worst < 1.0
+
+
+def test_wcsr_rmat_scaled(lib):
+    """configs[4] recipe at 2^14 rows, fp16, N = 32 / 128."""
+    a = wl.rmat(scale=14, dtype="fp16")
+    for N in (32, 128):
+        _wcsr_case(lib, a, "fp16", N, T=512)
+
+
+def test_wcsr_ragged_rows_and_identity(lib):
+    a = wl.random_csr(61, 1003, 77, 0.1, "fp16")
+    _wcsr_case(lib, a, "fp16", 40)
+    n = 100
+    one = np.ones(n, np.float32)
+    Bs = wl.dense(2, n, 64, ("normal", 0.0, 1.0), "tf32")
+    h = lib.spmm_wcsr_create_csr(n, n, np.arange(n + 1, dtype=np.int64), np.arange(n, dtype=np.int32), one, "tf32", 16)
+    C = run_gpu(lib, h, Bs, n, 64)
+    lib.spmm_destroy(h)
+    # identity: each output is one product 1.0 * b, exact up to the TF32 rounding of b
+    assert np.max(np.abs(C - Bs) / np.maximum(np.abs(Bs), 1e-30)) <= 2.0 ** -10
+
+
+def test_run_host_matches_device_run(lib):
+    a = wl.bcsr_tiny()
+    Bs = wl.dense(3, 512, 256, ("uniform", -1.0, 1.0), "bf16")
+    h = lib.spmm_bcsr_create_csr(512, 512, a["row_ptr"], a["col_idx"], a["vals"], "bf16", 64)
+    C = run_gpu(lib, h, Bs, 512, 256)
+    Ch = np.full((512, 256), np.nan, np.float32)
+    lib.spmm_run_host(h, Bs, Ch, 256)
+    assert np.array_equal(C, Ch)
+    lib.spmm_destroy(h)
+
+
+def test_bad_run_arguments(lib):
+    import torch
+    a = wl.bcsr_tiny()
+    h = lib.spmm_bcsr_create_csr(512, 512, a["row_ptr"], a["col_idx"], a["vals"], "bf16", 64)
+    buf = torch.zeros(1 << 20, dtype=torch.float32, device="cuda")
+    for args, code in (((buf.data_ptr(), buf.data_ptr(), 100), lib.SPMM_ERR_UNSUPPORTED),      # N*2 % 16 != 0
+                       ((buf.data_ptr() + 2, buf.data_ptr(), 256), lib.SPMM_ERR_UNSUPPORTED),  # misaligned
+                       ((0, buf.data_ptr(), 256), lib.SPMM_ERR_INVALID_ARG)):
+        with pytest.raises(lib.SpmmError) as e:
+            lib.spmm_run(h, *args)
+        assert e.value.code == code
+    lib.spmm_destroy(h)

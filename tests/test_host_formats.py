@@ -1,0 +1,199 @@
+"""CPU tests of the library's host logic through the C ABI (host_only handles):
+format construction, split plan and schedules must equal the oracle bit for bit;
+malformed input must be rejected with the documented codes; every symbol the
+header declares must be exported.  No CUDA call is made here.
+"""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import formats as F
+from paper_2604_17834_b200 import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2604_17834_b200 import build
+    build.build()
+    from paper_2604_17834_b200 import binding
+    return binding
+
+
+def test_library_exports_every_declared_symbol(lib):
+    import ctypes
+    header = open(os.path.join(ROOT, "include", "spmm_b200.h")).read()
+    declared = set(re.findall(r"\b(spmm_[a-z0-9_]+)\s*\(", header))
+    assert declared == set(lib.EXPORTED_SYMBOLS)
+    so = ctypes.CDLL(lib.LIB_PATH)
+    for name in declared:
+        assert getattr(so, name) is not None
+    assert lib.spmm_status_string(0) == "ok"
+    assert "wait" in lib.spmm_status_string(lib.SPMM_ERR_DEV_TIMEOUT)
+
+
+def _bits(a):
+    a = np.ascontiguousarray(a)
+    return a.view({2: np.uint16, 4: np.uint32}[a.dtype.itemsize])
+
+
+BCSR_CASES = [
+    ("bf16", 512, 512, 64), ("fp16", 300, 410, 16), ("fp16", 257, 129, 32),
+    ("bf16", 640, 384, 128), ("fp16", 64, 64, 64),
+]
+
+
+@pytest.mark.parametrize("dtype,m,k,b", BCSR_CASES)
+def test_bcsr_format_is_bit_exact(lib, dtype, m, k, b):
+    a = wl.random_csr(31 + m, m, k, 0.01, dtype, empty_rows=tuple(range(min(b, m))))
+    h = lib.spmm_bcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, b, host_only=True)
+    try:
+        f = F.bcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], b)
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCK_ROW_PTR, np.int32), f["block_row_ptr"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCK_COL_IDX, np.int32), f["block_col_idx"])
+        got = lib.spmm_export(h, lib.X_BCSR_BLOCKS, wl.storage_np_dtype(dtype))
+        assert np.array_equal(_bits(got), _bits(f["blocks"]).ravel())
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_ROW_ORDER, np.int32), F.bcsr_row_order(f["block_row_ptr"]))
+        info = lib.spmm_get_info(h, 256)
+        nnzb = f["block_col_idx"].shape[0]
+        assert info["n_units"] == nnzb and info["stored_values"] == nnzb * b * b
+        assert info["nnz"] == a["col_idx"].shape[0]
+        assert info["fill_ratio"] == pytest.approx(F.fill_ratio_bcsr(info["nnz"], nnzb, b))
+        assert info["n_empty"] == int((np.diff(f["block_row_ptr"]) == 0).sum()) >= 1
+        assert info["flops_stored"] == 2.0 * nnzb * b * b * 256
+        rows_touched = min(k, np.unique(f["block_col_idx"]).shape[0] * b)
+        assert info["bytes_b_touched"] == rows_touched * 256 * 2
+        assert info["bytes_c"] == m * 256 * 4
+        with pytest.raises(lib.SpmmError) as e:
+            lib.spmm_run(h, 16, 16, 256)
+        assert e.value.code == lib.SPMM_ERR_HOST_ONLY
+    finally:
+        lib.spmm_destroy(h)
+
+
+def test_bcsr_workload_generators_round_trip(lib):
+    a = wl.bcsr_tiny()
+    h = lib.spmm_bcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "bf16", 64, host_only=True)
+    f = F.bcsr_from_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], 64)
+    assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCKS, np.uint16), f["blocks"].ravel())
+    assert lib.spmm_get_info(h)["fill_ratio"] == 1.0
+    lib.spmm_destroy(h)
+    s = wl.bcsr_sweep(77, m=2048, k=2048, b=32, density=0.1)
+    h = lib.spmm_bcsr_create_csr(2048, 2048, s["row_ptr"], s["col_idx"], s["vals"], "fp16", 32, host_only=True)
+    f = F.bcsr_from_csr(2048, 2048, s["row_ptr"], s["col_idx"], s["vals"], 32)
+    order = lib.spmm_export(h, lib.X_BCSR_ROW_ORDER, np.int32)
+    assert np.array_equal(order, F.bcsr_row_order(f["block_row_ptr"]))
+    lens = np.diff(f["block_row_ptr"])[order]
+    assert np.all(np.diff(lens) <= 0) and lens[0] == 64 and lens[-1] == 0
+    lib.spmm_destroy(h)
+
+
+WCSR_CASES = [("tf32", 1000, 900, 0.01, 64), ("fp16", 333, 517, 0.05, 32), ("bf16", 160, 4000, 0.2, 128),
+              ("fp16", 16, 40, 0.5, 16)]
+
+
+@pytest.mark.parametrize("dtype,m,k,dens,T", WCSR_CASES)
+def test_wcsr_format_plan_and_spans_are_bit_exact(lib, dtype, m, k, dens, T):
+    a = wl.random_csr(41 + m, m, k, dens, dtype, empty_rows=tuple(range(16, min(32, m))))
+    b_col = 8 if dtype == "tf32" else 16
+    h = lib.spmm_wcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, 16, split_cols=T,
+                                 host_only=True, n_ctas=5)
+    try:
+        f = F.wcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], 16, b_col)
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_ROW_PTR, np.int32), f["window_row_ptr"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_COL_IDX, np.int32), f["window_col_idx"])
+        got = lib.spmm_export(h, lib.X_WCSR_VALUES, wl.storage_np_dtype(dtype))
+        assert np.array_equal(_bits(got), _bits(f["values"]).ravel())
+        plan = F.split_plan(f["window_row_ptr"], T)
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_TASKS, np.int32).reshape(-1, 4), plan)
+        spans = lib.spmm_export(h, lib.X_WCSR_SPANS, np.int32)
+        assert np.array_equal(spans, F.task_spans(plan, 5 * 8))
+        assert spans[0] == 0 and spans[-1] == plan.shape[0] and np.all(np.diff(spans) >= 0)
+        info = lib.spmm_get_info(h, 128)
+        P = f["window_col_idx"].shape[0]
+        assert info["n_units"] == P and info["stored_values"] == 16 * P
+        assert info["n_tasks"] == plan.shape[0]
+        assert info["n_slots"] == int((plan[:, 3] >= 0).sum())
+        assert info["n_split"] == np.unique(plan[plan[:, 3] >= 0, 0]).shape[0]
+        assert info["n_empty"] == int((np.diff(f["window_row_ptr"]) == 0).sum())
+        assert info["distinct_b_rows"] == np.unique(a["col_idx"]).shape[0]
+        assert info["workspace_bytes"] == info["n_slots"] * 16 * 128 * 4
+        assert info["fill_ratio"] == pytest.approx(F.fill_ratio_wcsr(info["nnz"], P, 16))
+    finally:
+        lib.spmm_destroy(h)
+
+
+def test_wcsr_irregular_workload(lib):
+    a = wl.wcsr_irregular(seed=3, m=5000, dtype="tf32")
+    h = lib.spmm_wcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "tf32", 16, split_cols=256,
+                                 host_only=True)
+    f = F.wcsr_from_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], 16, 8)
+    assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_COL_IDX, np.int32), f["window_col_idx"])
+    assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_VALUES, np.float32).view(np.uint32),
+                          f["values"].ravel().view(np.uint32))
+    assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_TASKS, np.int32).reshape(-1, 4),
+                          F.split_plan(f["window_row_ptr"], 256))
+    lib.spmm_destroy(h)
+
+
+def test_coo_entry_points_match_csr(lib):
+    a = wl.random_csr(5, 200, 300, 0.05, "fp16")
+    rows = np.repeat(np.arange(200), np.diff(a["row_ptr"])).astype(np.int32)
+    perm = np.random.default_rng(0).permutation(rows.shape[0])
+    h1 = lib.spmm_bcsr_create_csr(200, 300, a["row_ptr"], a["col_idx"], a["vals"], "fp16", 32, host_only=True)
+    h2 = lib.spmm_bcsr_create_coo(200, 300, rows[perm], a["col_idx"][perm], a["vals"][perm], "fp16", 32, host_only=True)
+    for which, dt in ((lib.X_BCSR_BLOCK_ROW_PTR, np.int32), (lib.X_BCSR_BLOCK_COL_IDX, np.int32), (lib.X_BCSR_BLOCKS, np.uint16)):
+        assert np.array_equal(lib.spmm_export(h1, which, dt), lib.spmm_export(h2, which, dt))
+    lib.spmm_destroy(h1)
+    lib.spmm_destroy(h2)
+    w1 = lib.spmm_wcsr_create_csr(200, 300, a["row_ptr"], a["col_idx"], a["vals"], "fp16", 16, host_only=True)
+    w2 = lib.spmm_wcsr_create_coo(200, 300, rows[perm], a["col_idx"][perm], a["vals"][perm], "fp16", 16, host_only=True)
+    for which, dt in ((lib.X_WCSR_WINDOW_ROW_PTR, np.int32), (lib.X_WCSR_WINDOW_COL_IDX, np.int32), (lib.X_WCSR_VALUES, np.uint16)):
+        assert np.array_equal(lib.spmm_export(w1, which, dt), lib.spmm_export(w2, which, dt))
+    lib.spmm_destroy(w1)
+    lib.spmm_destroy(w2)
+
+
+def test_malformed_input_is_rejected(lib):
+    rp = np.array([0, 2, 3], np.int64)
+    v = np.ones(3, np.float16)
+
+    def code(fn, *args, **kw):
+        with pytest.raises(lib.SpmmError) as e:
+            fn(*args, **kw)
+        return e.value.code
+
+    mk = lib.spmm_bcsr_create_csr
+    assert code(mk, 2, 4, rp, np.array([1, 0, 2], np.int32), v, "fp16", 16, host_only=True) == lib.SPMM_ERR_UNSORTED
+    assert code(mk, 2, 4, rp, np.array([1, 1, 2], np.int32), v, "fp16", 16, host_only=True) == lib.SPMM_ERR_UNSORTED
+    assert code(mk, 2, 4, rp, np.array([0, 4, 2], np.int32), v, "fp16", 16, host_only=True) == lib.SPMM_ERR_OUT_OF_RANGE
+    assert code(mk, 2, 4, rp, np.array([-1, 1, 2], np.int32), v, "fp16", 16, host_only=True) == lib.SPMM_ERR_OUT_OF_RANGE
+    assert code(mk, 2, 4, np.array([0, 3, 2], np.int64), np.array([0, 1, 2], np.int32), v, "fp16", 16,
+                host_only=True) == lib.SPMM_ERR_INVALID_ARG
+    assert code(mk, 2, 4, rp, np.array([0, 1, 2], np.int32), v, "fp16", 48, host_only=True) == lib.SPMM_ERR_UNSUPPORTED
+    assert code(mk, 2, 4, rp, np.array([0, 1, 2], np.int32), np.ones(3, np.float32), "tf32", 16,
+                host_only=True) == lib.SPMM_ERR_UNSUPPORTED
+    mw = lib.spmm_wcsr_create_csr
+    assert code(mw, 2, 4, rp, np.array([0, 1, 2], np.int32), v, "fp16", 8, host_only=True) == lib.SPMM_ERR_UNSUPPORTED
+    assert code(mw, 2, 4, rp, np.array([0, 1, 2], np.int32), v, "fp16", 16, split_cols=24,
+                host_only=True) == lib.SPMM_ERR_INVALID_ARG
+    assert code(mw, 2, 4, rp, np.array([0, 1, 2], np.int32), v, "fp16", 16, b_col=8,
+                host_only=True) == lib.SPMM_ERR_UNSUPPORTED
+    dup_r, dup_c = np.array([0, 0], np.int32), np.array([1, 1], np.int32)
+    assert code(lib.spmm_bcsr_create_coo, 2, 4, dup_r, dup_c, v[:2], "fp16", 16, host_only=True) == lib.SPMM_ERR_UNSORTED
+    lib.spmm_destroy(None)                                     # NULL is accepted
+
+
+def test_empty_matrix(lib):
+    rp = np.zeros(33, np.int64)
+    h = lib.spmm_wcsr_create_csr(32, 10, rp, np.zeros(0, np.int32), np.zeros(0, np.float32), "tf32", 16, host_only=True)
+    info = lib.spmm_get_info(h, 8)
+    assert info["n_units"] == 0 and info["n_tasks"] == 0 and info["n_empty"] == 2
+    assert lib.spmm_export(h, lib.X_WCSR_WINDOW_ROW_PTR, np.int32).tolist() == [0, 0, 0]
+    lib.spmm_destroy(h)
+    h = lib.spmm_bcsr_create_csr(32, 10, rp, np.zeros(0, np.int32), np.zeros(0, np.uint16), "bf16", 16, host_only=True)
+    assert lib.spmm_get_info(h)["n_units"] == 0
+    lib.spmm_destroy(h)
