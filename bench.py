@@ -1,0 +1,410 @@
+#!/usr/bin/env python
+"""Benchmark of the B200 SpMM hot path (BCSR and WCSR kernels behind the C ABI).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+                    [--only NAME] [--skip-others] [--with-graph]
+
+A step is one ``spmm_run`` (the SpMM kernel, plus the merge kernel for WCSR) on
+inputs already resident in HBM.  The headline workload is configs[1] (WCSR,
+100,000 x 100,000 TF32, N = 128); the other configurations are measured the same
+way and reported under "others".  Throughput is GFLOP/s over stored nonzeros,
+2 * nnz_stored * N / t.  L2 is flushed (a 512 MB write) before every timed
+launch and each launch is timed with its own pair of CUDA events on the
+launching stream.  With N > 1 GPUs every rank runs an independent replica of the
+same workload (the path has no exchange step); value = total flops / max time.
+
+``--impl reference`` times the fp64 CPU oracle (oracle/) on the host cores on a
+bounded sample of the same workload and prints the same line with
+"impl": "reference".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2604_17834_b200 import workloads as wl  # noqa: E402
+
+METRIC = "SpMM GFLOP/s over stored nonzeros (2*nnz_stored*N/time)"
+UNIT = "GFLOP/s"
+
+
+# --------------------------------------------------------------------------- workloads
+
+
+def workload_table():
+    """name -> (description, builder).  builder() -> dict(kind, a, dtype, size, N, Bdist, opts)."""
+    def cfg1():
+        return dict(kind="bcsr", a=wl.bcsr_tiny(), dtype="bf16", size=64, N=256, Bdist=("uniform", -1.0, 1.0))
+
+    def cfg2():
+        return dict(kind="wcsr", a=wl.wcsr_irregular(), dtype="tf32", size=16, N=128, Bdist=("normal", 0.0, 1.0))
+
+    def cfg3_gate():
+        return dict(kind="bcsr", a=wl.bcsr_llm(), dtype="bf16", size=64, N=65536, Bdist=("normal", 0.0, 1.0))
+
+    def cfg3_down():
+        return dict(kind="bcsr", a=wl.bcsr_llm(seed=1013, m=3584, k=18944), dtype="bf16", size=64, N=65536,
+                    Bdist=("normal", 0.0, 1.0))
+
+    def cfg4(b, d, skewed=True):
+        def f():
+            return dict(kind="bcsr", a=wl.bcsr_sweep(1004 + b + int(d * 1000), b=b, density=d, skewed=skewed),
+                        dtype="fp16", size=b, N=4096, Bdist=("uniform", -1.0, 1.0))
+        return f
+
+    def cfg5(N):
+        def f():
+            return dict(kind="wcsr", a=wl.rmat(), dtype="fp16", size=16, N=N, Bdist=("normal", 0.0, 1.0))
+        return f
+
+    t = {
+        "cfg1_bcsr_tiny": ("configs[0] BCSR 512x512 bf16 b=64 keep 0.5, N=256", cfg1),
+        "cfg2_wcsr_irregular": ("configs[1] WCSR 100000x100000 tf32 zipf(2) rows, 50% band, wh=16, N=128", cfg2),
+        "cfg3_bcsr_llm_gate": ("configs[2] BCSR 18944x3584 bf16 b=64 90% blocks zero, N=65536", cfg3_gate),
+        "cfg3_bcsr_llm_down": ("configs[2] BCSR 3584x18944 bf16 b=64 90% blocks zero, N=65536", cfg3_down),
+        "cfg5_wcsr_rmat_n32": ("configs[4] WCSR R-MAT 2^21 deg 16 fp16 wh=16, N=32", cfg5(32)),
+        "cfg5_wcsr_rmat_n128": ("configs[4] WCSR R-MAT 2^21 deg 16 fp16 wh=16, N=128", cfg5(128)),
+        "cfg5_wcsr_rmat_n256": ("configs[4] WCSR R-MAT 2^21 deg 16 fp16 wh=16, N=256", cfg5(256)),
+    }
+    for b in (16, 32, 64, 128):
+        for d in (0.5, 0.2, 0.1, 0.05, 0.01):
+            t["cfg4_bcsr_sweep_b%d_d%g" % (b, d)] = (
+                "configs[3] BCSR 8192x8192 fp16 b=%d skewed rows, keep %g in the rest, N=4096" % (b, d), cfg4(b, d))
+        for d in (0.05, 0.01):
+            t["cfg4_bcsr_flat_b%d_d%g" % (b, d)] = (
+                "configs[3] BCSR 8192x8192 fp16 b=%d flat Bernoulli(%g), N=4096" % (b, d), cfg4(b, d, False))
+    return t
+
+
+HEADLINE = "cfg2_wcsr_irregular"
+DEFAULT_OTHERS = ["cfg1_bcsr_tiny", "cfg3_bcsr_llm_gate", "cfg4_bcsr_sweep_b64_d0.1", "cfg4_bcsr_sweep_b16_d0.1",
+                  "cfg4_bcsr_sweep_b128_d0.1", "cfg4_bcsr_flat_b64_d0.05"]
+
+
+# --------------------------------------------------------------------------- helpers
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nme, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nme)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def create_handle(lib, w, **opt):
+    a = w["a"]
+    t0 = time.perf_counter()
+    if w["kind"] == "bcsr":
+        h = lib.spmm_bcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], w["dtype"], w["size"], **opt)
+    else:
+        h = lib.spmm_wcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], w["dtype"], w["size"], **opt)
+    return h, (time.perf_counter() - t0) * 1e3
+
+
+def device_B(torch, w, seed=7):
+    """Seeded synthetic dense operand, generated on the device in storage dtype."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+    k, N = w["a"]["k"], w["N"]
+    tdt = {"bf16": torch.bfloat16, "fp16": torch.float16, "tf32": torch.float32}[w["dtype"]]
+    B = torch.empty((k, N), dtype=tdt, device="cuda")
+    rows = max(1, (1 << 26) // N)
+    for r0 in range(0, k, rows):
+        r1 = min(k, r0 + rows)
+        if w["Bdist"][0] == "normal":
+            x = torch.randn((r1 - r0, N), generator=g, device="cuda", dtype=torch.float32) * w["Bdist"][2] + w["Bdist"][1]
+        else:
+            x = torch.rand((r1 - r0, N), generator=g, device="cuda", dtype=torch.float32) * (w["Bdist"][2] - w["Bdist"][1]) + w["Bdist"][1]
+        B[r0:r1] = x.to(tdt)
+    return B
+
+
+def roofline_of(info, ms, pk):
+    """Roofline of one spmm_run: slower of tensor time for the stored flops and HBM time for the model bytes."""
+    model_bytes = info["bytes_a"] + info["bytes_idx"] + info["bytes_b_touched"] + info["bytes_c"]
+    tc_peak = pk["bf16_tflops"] * (0.5 if info["dtype"] == 2 else 1.0)       # TF32 = half the bf16 rate (nominal ratio)
+    t_hbm = model_bytes / (pk["hbm_gbs"] * 1e9)
+    t_tc = info["flops_stored"] / (tc_peak * 1e12)
+    t = ms * 1e-3
+    if t_hbm >= t_tc:
+        ach = model_bytes / t / 1e9
+        r = {"bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"]}
+    else:
+        ach = info["flops_stored"] / t / 1e12
+        r = {"bound": "tensor", "achieved": ach, "peak": tc_peak, "unit": "TFLOP/s", "frac": ach / tc_peak}
+    r.update({"peak_source": pk["source"], "model_bytes": model_bytes, "t_roof_us": max(t_hbm, t_tc) * 1e6,
+              "gather_bytes": info["bytes_gather"], "traffic": None})
+    return r
+
+
+def time_workload(torch, lib, w, steps, warmup, flush):
+    """-> dict with per-launch median / mean ms (device events), GFLOP/s, roofline, info."""
+    h, create_ms = create_handle(lib, w)
+    try:
+        N = w["N"]
+        info = lib.spmm_get_info(h, N)
+        B = device_B(torch, w)
+        C = torch.empty((w["a"]["m"], N), dtype=torch.float32, device="cuda")
+        st = torch.cuda.current_stream().cuda_stream
+        for _ in range(max(3, warmup)):
+            lib.spmm_run(h, B.data_ptr(), C.data_ptr(), N, st)
+        torch.cuda.synchronize()
+        lib.spmm_check(h)
+        evs = []
+        for _ in range(steps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            lib.spmm_run(h, B.data_ptr(), C.data_ptr(), N, st)
+            e1.record()
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        lib.spmm_check(h)
+        ms = np.array([a.elapsed_time(b) for a, b in evs])
+        launches = 1 + (1 if (w["kind"] == "wcsr" and (info["n_split"] + info["n_empty"]) > 0) else 0)
+        return dict(h=None, info=info, ms_mean=float(ms.mean()), ms_median=float(np.median(ms)), ms_min=float(ms.min()),
+                    create_ms=create_ms, launches_per_step=launches, B=B, C=C)
+    finally:
+        lib.spmm_destroy(h)
+
+
+def summarize(name, desc, res, pk, N):
+    info = res["info"]
+    ms = res["ms_mean"]
+    gf = info["flops_stored"] / (ms * 1e-3) / 1e9
+    return {
+        "workload": name, "description": desc, "ms_per_step": ms, "ms_median": res["ms_median"], "ms_min": res["ms_min"],
+        "gflops_stored": gf, "gflops_useful": 2.0 * info["nnz"] * N / (ms * 1e-3) / 1e9,
+        "fill_ratio": info["fill_ratio"], "stored_values": info["stored_values"], "n_units": info["n_units"],
+        "create_ms": res["create_ms"], "roofline": roofline_of(info, ms, pk),
+    }
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+
+
+def cpu_oracle_time(w, budget_s=15.0):
+    """Time the oracle (as it stands, one thread) on a bounded sample: all rows x a column slab."""
+    from oracle import spmm_ref
+    a, N, dtype = w["a"], w["N"], w["dtype"]
+    nnz = int(a["row_ptr"][-1])
+    # ~0.35 G multiply-add pairs per second per core with the |.| sum: size the slab for the budget
+    cols = int(max(1, min(N, budget_s * 2.0e8 / max(1, nnz))))
+    Bs = wl.dense(11, a["k"], cols, w["Bdist"], dtype)
+    v64, B64 = wl.widen(a["vals"], dtype), wl.widen(Bs, dtype)
+    t0 = time.perf_counter()
+    spmm_ref(a["row_ptr"], a["col_idx"], v64, B64)
+    dt = time.perf_counter() - t0
+    return dt * (N / cols), cols, dt
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    name = args.only or HEADLINE
+    desc, builder = workload_table()[name]
+    w = builder()
+    from paper_2604_17834_b200 import build
+    build.build()
+    from paper_2604_17834_b200 import binding as lib
+    h, _ = create_handle(lib, w, host_only=True)
+    info = lib.spmm_get_info(h, w["N"])
+    lib.spmm_destroy(h)
+    times = []
+    for i in range(args.warmup + args.steps):
+        t_full, cols, dt = cpu_oracle_time(w, budget_s=max(1.0, 60.0 / (args.warmup + args.steps)))
+        if i >= args.warmup:
+            times.append(t_full)
+    t = float(np.mean(times))
+    val = info["flops_stored"] / t / 1e9
+    sample = "all %d rows x %d of %d columns per step, scaled linearly in N" % (w["a"]["m"], cols, w["N"])
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "config": {"workload": name, "description": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- main arm
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="b200")
+    ap.add_argument("--only", default=None, help="time just this workload as the headline (see workload_table)")
+    ap.add_argument("--skip-others", action="store_true")
+    ap.add_argument("--others", default=None, help="comma-separated workload names to report beside the headline")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    from paper_2604_17834_b200 import binding as lib
+
+    pk = peaks()
+    table = workload_table()
+    name = args.only or HEADLINE
+    desc, builder = table[name]
+    w = builder()
+    warmup = max(3, args.warmup)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    res = time_workload(torch, lib, w, args.steps, warmup, flush)
+    barrier()
+    clocks = sampler.stop()
+    ms = res["ms_mean"]
+    if world > 1:
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    info = res["info"]
+    value = world * info["flops_stored"] / (ms * 1e-3) / 1e9
+    head = summarize(name, desc, res, pk, w["N"])
+
+    # end to end through the C ABI with host buffers (pinned), copies inside the timed region
+    a, N = w["a"], w["N"]
+    Bh = torch.empty((a["k"], N), dtype=res["B"].dtype).pin_memory()
+    Bh.copy_(res["B"])
+    Ch = torch.empty((a["m"], N), dtype=torch.float32).pin_memory()
+    h, _ = create_handle(lib, w)
+    st = torch.cuda.current_stream().cuda_stream
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        lib.spmm_run_host(h, Bh.data_ptr(), Ch.data_ptr(), N, st)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        lib.spmm_run_host(h, Bh.data_ptr(), Ch.data_ptr(), N, st)
+    torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    lib.spmm_destroy(h)
+    if world > 1:
+        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = {"value": world * info["flops_stored"] / e2e_s / 1e9, "unit": UNIT, "ms_per_step": e2e_s * 1e3,
+           "h2d_bytes_per_step": int(Bh.numel() * Bh.element_size()), "d2h_bytes_per_step": int(Ch.numel() * 4)}
+    del res["B"], res["C"]
+
+    others = []
+    if rank == 0 and not args.skip_others and args.only is None:
+        names = args.others.split(",") if args.others else DEFAULT_OTHERS
+        for nm in names:
+            d2, b2 = table[nm]
+            w2 = b2()
+            r2 = time_workload(torch, lib, w2, max(5, args.steps // 3), 3, flush)
+            r2.pop("B"), r2.pop("C")
+            others.append(summarize(nm, d2, r2, pk, w2["N"]))
+            del w2
+            torch.cuda.empty_cache()
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        t_full, cols, dt = cpu_oracle_time(w)
+        cpu = {"value": info["flops_stored"] / t_full / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": "all %d rows x %d of %d columns (%.1f s), scaled linearly in N" % (a["m"], cols, N, dt),
+               "useful_gflops": 2.0 * info["nnz"] * N / t_full / 1e9}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": w["dtype"], "data": "synthetic",
+            "config": {"workload": name, "description": desc, "l2": "flushed before every timed launch (512 MB write)",
+                       "timing": "one CUDA-event pair per launch on the launching stream; mean over steps",
+                       "multi_gpu": "independent replicas, no collective"},
+            "clocks": clocks, "e2e": e2e,
+            "gpu_launches": int(res["launches_per_step"] * args.steps),
+            "roofline": head["roofline"], "cpu_baseline": cpu,
+            "headline_detail": {k: head[k] for k in ("ms_median", "ms_min", "gflops_useful", "fill_ratio", "create_ms")},
+            "others": others,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
