@@ -158,6 +158,29 @@ int spmm_wcsr_create_coo(spmm_handle_t *out, int64_t m, int64_t k, int64_t nnz,
 int spmm_run(spmm_handle_t h, const void *B_dev, void *C_dev, int64_t N, void *stream);
 
 /*
+ * WCSR only; the paper has no counterpart (an addition of this library).  Same result as
+ * spmm_run, but the call allocates nothing: the partial tiles of split windows go to a
+ * scratch array that is built into the library (8 MiB of device memory, held by every GPU
+ * that loads the library until the process exits) instead of a workspace allocated on
+ * demand.  It is meant for callers that must not allocate device memory at the time of the
+ * call: code that runs inside a framework whose memory pool already owns the device, or a
+ * latency-critical loop that cannot afford the device-wide synchronisation an allocation
+ * or a free can cause.
+ *   - The partial tiles need n_slots * 16 * N * 4 bytes (spmm_get_info: workspace_bytes).
+ *     More than 8 MiB returns SPMM_ERR_TOO_LARGE and nothing is launched; choose a larger
+ *     split_cols at creation, a smaller N, or use spmm_run.
+ *   - The first call on each device looks up the scratch array's device address; make that
+ *     first call outside any stream capture.  Later calls only launch kernels.
+ *   - The array is shared by all handles and all calls and keeps the previous call's
+ *     contents; every partial tile a call reads is first written by that same call, so
+ *     nothing needs clearing.  Two calls that overlap on the GPU (different streams, or
+ *     different host threads) race on it: serialise them.
+ *   - Returns SPMM_ERR_INVALID_ARG for a BCSR handle.
+ * Arguments and all other behaviour as spmm_run.
+ */
+int spmm_wcsr_run_static(spmm_handle_t h, const void *B_dev, void *C_dev, int64_t N, void *stream);
+
+/*
  * Same result as spmm_run, for callers that hold HOST buffers: copies B to the device,
  * runs, copies C back and synchronises `stream` before returning.  B_host / C_host are
  * ordinary or pinned host memory of k*N elements / m*N floats; the device staging buffers

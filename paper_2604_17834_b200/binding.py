@@ -41,7 +41,7 @@ X_WCSR_WINDOW_ROW_PTR, X_WCSR_WINDOW_COL_IDX, X_WCSR_VALUES, X_WCSR_TASKS, X_WCS
 
 EXPORTED_SYMBOLS = (
     "spmm_bcsr_create_csr", "spmm_bcsr_create_coo", "spmm_wcsr_create_csr", "spmm_wcsr_create_coo",
-    "spmm_run", "spmm_run_host", "spmm_check", "spmm_get_info", "spmm_export", "spmm_destroy",
+    "spmm_run", "spmm_wcsr_run_static", "spmm_run_host", "spmm_check", "spmm_get_info", "spmm_export", "spmm_destroy",
     "spmm_status_string", "spmm_set_wait_limit_ns",
 )
 
@@ -79,6 +79,7 @@ _lib.spmm_bcsr_create_coo.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _vp
 _lib.spmm_wcsr_create_coo.argtypes = _lib.spmm_bcsr_create_coo.argtypes
 _lib.spmm_run.argtypes = [_vp, _vp, _vp, _i64, _vp]
 _lib.spmm_run_host.argtypes = [_vp, _vp, _vp, _i64, _vp]
+_lib.spmm_wcsr_run_static.argtypes = [_vp, _vp, _vp, _i64, _vp]
 _lib.spmm_check.argtypes = [_vp]
 _lib.spmm_get_info.argtypes = [_vp, _i64, ctypes.POINTER(SpmmInfo)]
 _lib.spmm_export.argtypes = [_vp, _i32, _vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
@@ -170,6 +171,17 @@ def spmm_run(h, B_dev_ptr, C_dev_ptr, N, stream=0):
     rc = _lib.spmm_run(h, _vp(B_dev_ptr), _vp(C_dev_ptr), N, _vp(stream))
     if rc != SPMM_OK:
         raise SpmmError(rc, "spmm_run")
+
+
+def spmm_wcsr_run_static(h, B_dev_ptr, C_dev_ptr, N, stream=0):
+    """WCSR only: like spmm_run, but allocates nothing -- the partial tiles of split windows
+    use the 8 MiB scratch array built into the library.  For callers that may not allocate
+    device memory when they call (a framework's pool owns the device, or an allocation's
+    synchronisation is not acceptable).  Raises SpmmError(SPMM_ERR_TOO_LARGE) when the
+    partial tiles do not fit; calls that overlap on the GPU race on the shared array."""
+    rc = _lib.spmm_wcsr_run_static(h, _vp(B_dev_ptr), _vp(C_dev_ptr), N, _vp(stream))
+    if rc != SPMM_OK:
+        raise SpmmError(rc, "spmm_wcsr_run_static")
 
 
 def spmm_run_host(h, B_host, C_host, N, stream=0):

@@ -446,6 +446,17 @@ int spmm_run(spmm_handle_t h, const void* B_dev, void* C_dev, int64_t N, void* s
     return run_wcsr(h, B_dev, static_cast<float*>(C_dev), N, st);
 }
 
+int spmm_wcsr_run_static(spmm_handle_t h, const void* B_dev, void* C_dev, int64_t N, void* stream) {
+    int rc = check_run_args(h, B_dev, C_dev, N);
+    if (rc) return rc;
+    if (h->format != 1) return SPMM_ERR_INVALID_ARG;
+    float* scratch = nullptr;
+    size_t cap = 0;
+    if (wcsr_static_scratch(&scratch, &cap) != cudaSuccess) return SPMM_ERR_CUDA;
+    if (static_cast<size_t>(wcsr_workspace_bytes(h, N)) > cap) return SPMM_ERR_TOO_LARGE;
+    return launch_wcsr_all(h, B_dev, static_cast<float*>(C_dev), scratch, N, static_cast<cudaStream_t>(stream));
+}
+
 int spmm_run_host(spmm_handle_t h, const void* B_host, void* C_host, int64_t N, void* stream) {
     if (!h || !B_host || !C_host || N <= 0) return SPMM_ERR_INVALID_ARG;
     if (h->host_only) return SPMM_ERR_HOST_ONLY;

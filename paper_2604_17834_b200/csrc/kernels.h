@@ -63,4 +63,8 @@ struct MergeParams {
 };
 cudaError_t launch_wcsr_merge(const MergeParams& p, cudaStream_t stream);
 
+// Device address and size in bytes of the library's built-in partial-tile scratch on the
+// current device (resolved on the first call per device).
+cudaError_t wcsr_static_scratch(float** ptr, size_t* bytes);
+
 }  // namespace spmm

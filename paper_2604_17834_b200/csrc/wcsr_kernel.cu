@@ -20,6 +20,8 @@
 // consecutive, so neighbouring windows (which share B rows in banded matrices) run together.
 // Split windows are summed in slot order by wcsr_merge_kernel, which also zero-fills the C
 // rows of empty windows: results are run-to-run identical.
+#include <mutex>
+
 #include "kernels.h"
 #include "ptx.cuh"
 
@@ -330,6 +332,34 @@ cudaError_t launch_wcsr(int dtype, int groups, const WcsrParams& p, int sms, cud
         if (groups == 2) return launch_one<2, 1, 2, 64, 6, 3>(p, sms, stream);
     }
     return cudaErrorInvalidValue;
+}
+
+// Built-in scratch for spmm_wcsr_run_static: partial tiles of split windows, for callers
+// that may not allocate device memory.  Every GPU that loads the library holds these
+// kStaticScratchBytes until the process exits.  All handles and all calls share it.
+constexpr size_t kStaticScratchBytes = size_t{8} << 20;
+static __device__ __align__(256) float g_static_scratch[kStaticScratchBytes / sizeof(float)];
+
+cudaError_t wcsr_static_scratch(float** ptr, size_t* bytes) {
+    // In host code the array's name is only a stand-in for the device symbol, never a
+    // device address: resolve it once per device, with that device current.
+    constexpr int kMaxDevices = 64;
+    static float* resolved[kMaxDevices] = {};
+    static std::mutex mu;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!resolved[dev]) {
+        float* p = nullptr;
+        e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_scratch);
+        if (e != cudaSuccess) return e;
+        resolved[dev] = p;
+    }
+    *ptr = resolved[dev];
+    *bytes = kStaticScratchBytes;
+    return cudaSuccess;
 }
 
 cudaError_t launch_wcsr_merge(const MergeParams& p, cudaStream_t stream) {
