@@ -64,7 +64,8 @@ typedef struct {
                             TF32 -- the K extent of one tensor-core instruction (Sec. 2.3,
                             Sec. 4.1 uses 8 with TF32).                                      */
     int32_t split_cols;  /* WCSR: sub-task size T in columns (Sec. 3.3); multiple of b_col.
-                            Default 1024.                                                    */
+                            Default: about a quarter of one bin's share of the padded columns,
+                            rounded down to a multiple of 64 and clamped to [128, 4096].      */
     int32_t host_only;   /* 1: build the format on the host only (no CUDA call at all); the
                             handle serves spmm_export / spmm_get_info, spmm_run fails.       */
     int32_t n_ctas;      /* persistent grid size the schedule is built for; default = the
@@ -107,7 +108,9 @@ typedef enum {
     SPMM_X_WCSR_VALUES = 12,        /* dtype [h][P] row-major                                 */
     SPMM_X_WCSR_TASKS = 13,         /* int32 [n_tasks][4]: window, first col in window,
                                        column count, partial slot (-1 = writes C directly)    */
-    SPMM_X_WCSR_SPANS = 14          /* int32 [n_spans+1]: task ranges handed to the CTAs      */
+    SPMM_X_WCSR_BIN_PTR = 14,       /* int32 [n_bins+1]: ranges of BIN_TASKS, n_bins = 2*n_ctas */
+    SPMM_X_WCSR_BIN_TASKS = 15      /* int32 [n_tasks]: task indices bin by bin (the static
+                                       schedule: CTA c runs bins c, c + grid, ...)            */
 } spmm_export_t;
 
 /*

@@ -182,21 +182,33 @@ def bcsr_row_order(block_row_ptr):
     return np.argsort(-lens, kind="stable").astype(np.int32)
 
 
-def task_spans(plan, n_spans, fixed_cost=32):
-    """Cut the task list into n_spans consecutive ranges of near-equal cost.
+def default_split_cols(P, n_bins):
+    """Sub-task size used when the caller gives none: a quarter of one bin's share of the
+    padded columns, rounded down to a multiple of 64, clamped to [128, 4096]."""
+    t = (P // (n_bins * 4)) // 64 * 64
+    return int(min(4096, max(128, t)))
 
-    cost(task) = its column count + fixed_cost.  Span j ends after the first
-    task at which the running cost c satisfies c * n_spans >= (j + 1) * total
-    (integer arithmetic); spans may be empty.  Returns int32 [n_spans + 1].
+
+def task_bins(plan, n_bins, fixed_cost=32):
+    """Static schedule of the sub-tasks of Sec. 3.3 over n_bins bins: the
+    longest-processing-time rule.  cost(task) = its column count + fixed_cost.
+    Tasks are taken heaviest first (ties: lower task index first); each goes to
+    the bin whose load is smallest at that moment (ties: lowest bin index).
+    Inside a bin tasks are listed in ascending task index.
+
+    Returns (bin_ptr int32 [n_bins+1], bin_tasks int32 [ntasks]).
     """
+    import heapq
     cost = plan[:, 2].astype(np.int64) + fixed_cost
-    total = int(cost.sum())
-    spans = [0]
-    run, ti, nt = 0, 0, plan.shape[0]
-    for j in range(n_spans):
-        while ti < nt and run * n_spans < (j + 1) * total:
-            run += int(cost[ti])
-            ti += 1
-        spans.append(ti)
-    spans[-1] = nt
-    return np.asarray(spans, dtype=np.int32)
+    order = np.argsort(-plan[:, 2].astype(np.int64), kind="stable")
+    heap = [(0, b) for b in range(n_bins)]
+    heapq.heapify(heap)
+    members = [[] for _ in range(n_bins)]
+    for t in order.tolist():
+        load, b = heapq.heappop(heap)
+        members[b].append(t)
+        heapq.heappush(heap, (load + int(cost[t]), b))
+    bin_ptr = np.zeros(n_bins + 1, dtype=np.int64)
+    bin_ptr[1:] = np.cumsum([len(x) for x in members])
+    tasks = [t for x in members for t in sorted(x)]
+    return bin_ptr.astype(np.int32), np.asarray(tasks, dtype=np.int32)

@@ -37,7 +37,8 @@ SPMM_ERR_HOST_ONLY = -8
 SPMM_ERR_TOO_LARGE = -9
 
 X_BCSR_BLOCK_ROW_PTR, X_BCSR_BLOCK_COL_IDX, X_BCSR_BLOCKS, X_BCSR_ROW_ORDER = 0, 1, 2, 3
-X_WCSR_WINDOW_ROW_PTR, X_WCSR_WINDOW_COL_IDX, X_WCSR_VALUES, X_WCSR_TASKS, X_WCSR_SPANS = 10, 11, 12, 13, 14
+X_WCSR_WINDOW_ROW_PTR, X_WCSR_WINDOW_COL_IDX, X_WCSR_VALUES, X_WCSR_TASKS = 10, 11, 12, 13
+X_WCSR_BIN_PTR, X_WCSR_BIN_TASKS = 14, 15
 
 EXPORTED_SYMBOLS = (
     "spmm_bcsr_create_csr", "spmm_bcsr_create_coo", "spmm_wcsr_create_csr", "spmm_wcsr_create_coo",

@@ -83,7 +83,10 @@ struct spmm_handle_s {
     uint8_t* d_vals = nullptr;       // blocks / packed values
     int32_t* d_order = nullptr;      // BCSR row order
     WcsrDevTask* d_tasks = nullptr;
-    int32_t* d_spans = nullptr;
+    int32_t* d_bin_ptr = nullptr;
+    int32_t* d_bin_tasks = nullptr;
+    int32_t* d_fills = nullptr;
+    int32_t* d_bin_fill = nullptr;
     int32_t* d_merge = nullptr;      // window | first | nparts, each [n_merge]
     int n_merge = 0;
     int* d_status = nullptr;
@@ -115,7 +118,10 @@ void free_handle(spmm_handle_s* h) {
         cudaFree(h->d_vals);
         cudaFree(h->d_order);
         cudaFree(h->d_tasks);
-        cudaFree(h->d_spans);
+        cudaFree(h->d_bin_ptr);
+        cudaFree(h->d_bin_tasks);
+        cudaFree(h->d_fills);
+        cudaFree(h->d_bin_fill);
         cudaFree(h->d_merge);
         cudaFree(h->d_status);
         cudaFree(h->d_partial);
@@ -193,7 +199,7 @@ int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const s
     const int b_col_default = 32 / a.es;
     const int b_col = (opts && opts->b_col > 0) ? opts->b_col : b_col_default;
     if (b_col != b_col_default) return SPMM_ERR_UNSUPPORTED;
-    const int T = (opts && opts->split_cols > 0) ? opts->split_cols : 1024;
+    const int T = (opts && opts->split_cols > 0) ? opts->split_cols : 0;   // 0: chosen from the matrix
     if (T % b_col != 0) return SPMM_ERR_INVALID_ARG;
     spmm_handle_s* h = new (std::nothrow) spmm_handle_s;
     if (!h) return SPMM_ERR_ALLOC;
@@ -207,7 +213,7 @@ int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const s
     rc = device_setup(h, opts);
     if (rc) { free_handle(h); return rc; }
     try {
-        rc = build_wcsr(a, wh, b_col, T, h->n_ctas * 8, &h->wcsr);
+        rc = build_wcsr(a, wh, b_col, T, h->n_ctas * 2, &h->wcsr);
     } catch (const std::bad_alloc&) {
         rc = SPMM_ERR_ALLOC;
     }
@@ -233,7 +239,10 @@ int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const s
         if (!rc) rc = upload(&h->d_idx, f.window_col_idx.data(), f.window_col_idx.size() * 4);
         if (!rc) rc = upload(&h->d_vals, f.packed.data(), f.packed.size());
         if (!rc) rc = upload(&h->d_tasks, dt.data(), dt.size() * sizeof(WcsrDevTask));
-        if (!rc) rc = upload(&h->d_spans, f.spans.data(), f.spans.size() * 4);
+        if (!rc) rc = upload(&h->d_bin_ptr, f.bin_ptr.data(), f.bin_ptr.size() * 4);
+        if (!rc) rc = upload(&h->d_bin_tasks, f.bin_tasks.data(), f.bin_tasks.size() * 4);
+        if (!rc) rc = upload(&h->d_fills, f.fills.data(), f.fills.size() * 4);
+        if (!rc) rc = upload(&h->d_bin_fill, f.bin_fill.data(), f.bin_fill.size() * 4);
         if (!rc) rc = upload(&h->d_merge, mg.data(), mg.size() * 4);
         if (rc) { free_handle(h); return rc; }
         std::vector<uint8_t>().swap(h->wcsr.packed);
@@ -325,7 +334,10 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, float* C, float* partial, i
     const int bnt = 128 * groups;
     WcsrParams p;
     p.tasks = h->d_tasks;
-    p.spans = h->d_spans;
+    p.bin_ptr = h->d_bin_ptr;
+    p.bin_tasks = h->d_bin_tasks;
+    p.fills = reinterpret_cast<const int2*>(h->d_fills);
+    p.bin_fill = h->d_bin_fill;
     p.col_idx = h->d_idx;
     p.packed = h->d_vals;
     p.B = B;
@@ -333,7 +345,7 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, float* C, float* partial, i
     p.partial = partial;
     p.m = h->m;
     p.N = N;
-    p.n_spans = static_cast<int32_t>(f.spans.size()) - 1;
+    p.n_bins = static_cast<int32_t>(f.bin_ptr.size()) - 1;
     p.n_tt = static_cast<int32_t>((N + bnt - 1) / bnt);
     p.status = h->d_status;
     p.wait_limit_ns = g_wait_limit_ns.load();
@@ -568,7 +580,8 @@ int spmm_export(spmm_handle_t h, int which, void* host_dst, size_t cap, size_t* 
             case SPMM_X_WCSR_WINDOW_COL_IDX: bytes = f.window_col_idx.size() * 4; dev_src = h->d_idx; host_src = f.window_col_idx.data(); break;
             case SPMM_X_WCSR_VALUES: bytes = static_cast<size_t>(f.P) * f.wh * h->es; unpack_wcsr = true; break;
             case SPMM_X_WCSR_TASKS: bytes = f.tasks.size() * 16; break;
-            case SPMM_X_WCSR_SPANS: bytes = f.spans.size() * 4; dev_src = h->d_spans; host_src = f.spans.data(); break;
+            case SPMM_X_WCSR_BIN_PTR: bytes = f.bin_ptr.size() * 4; dev_src = h->d_bin_ptr; host_src = f.bin_ptr.data(); break;
+            case SPMM_X_WCSR_BIN_TASKS: bytes = f.bin_tasks.size() * 4; dev_src = h->d_bin_tasks; host_src = f.bin_tasks.data(); break;
             default: return SPMM_ERR_INVALID_ARG;
         }
     }

@@ -4,6 +4,8 @@
 #include <algorithm>
 #include <cstring>
 #include <numeric>
+#include <queue>
+#include <utility>
 
 #include "spmm_b200.h"
 
@@ -127,13 +129,12 @@ int build_bcsr(const CsrView& a, int b, BcsrHost* out) {
 
 // ----------------------------------------------------------------------------- WCSR
 
-int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_spans, WcsrHost* out) {
+int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost* out) {
     if (wh != 16) return SPMM_ERR_UNSUPPORTED;
     if (b_col * a.es != 32) return SPMM_ERR_UNSUPPORTED;
-    if (T <= 0 || T % b_col != 0 || n_spans <= 0) return SPMM_ERR_INVALID_ARG;
+    if (T < 0 || T % b_col != 0 || n_bins <= 0) return SPMM_ERR_INVALID_ARG;
     out->wh = wh;
     out->b_col = b_col;
-    out->T = T;
     const int64_t nwin = cdiv(a.m, wh);
     out->nwin = nwin;
     out->window_row_ptr.assign(static_cast<size_t>(nwin) + 1, 0);
@@ -176,6 +177,13 @@ int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_spans, WcsrHost
         }
     }
 
+    if (T == 0) {
+        int64_t t = P / (static_cast<int64_t>(n_bins) * 4);
+        t = (t / 64) * 64;
+        T = static_cast<int>(std::min<int64_t>(4096, std::max<int64_t>(128, t)));
+    }
+    out->T = T;
+
     // split plan: consecutive chunks of T columns; a window with one chunk writes C itself
     out->tasks.clear();
     out->merge_window.clear();
@@ -212,23 +220,52 @@ int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_spans, WcsrHost
         out->merge_nparts.push_back(0);
     }
 
-    // spans: cut the task list into n_spans consecutive ranges of near-equal cost
-    // (cost of a task = its columns + kTaskFixedCost); span j ends at the first task where
-    // the running cost reaches (j+1)/n_spans of the total.
+    // bins: longest-processing-time assignment of tasks
     const int64_t ntasks = static_cast<int64_t>(out->tasks.size());
-    int64_t total = 0;
-    for (const WcsrTask& t : out->tasks) total += t.count + kTaskFixedCost;
-    out->spans.assign(static_cast<size_t>(n_spans) + 1, 0);
-    int64_t run = 0, ti = 0;
-    for (int j = 0; j < n_spans; ++j) {
-        // smallest ti with run * n_spans >= (j+1) * total
-        while (ti < ntasks && run * n_spans < static_cast<int64_t>(j + 1) * total) {
-            run += out->tasks[ti].count + kTaskFixedCost;
-            ++ti;
-        }
-        out->spans[j + 1] = static_cast<int32_t>(ti);
+    std::vector<int32_t> order(static_cast<size_t>(ntasks));
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(),
+                     [&](int32_t x, int32_t y) { return out->tasks[x].count > out->tasks[y].count; });
+    using Load = std::pair<int64_t, int32_t>;   // (load, bin): smallest load, then lowest bin, on top
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+    for (int32_t bsel = 0; bsel < n_bins; ++bsel) heap.push(Load(0, bsel));
+    std::vector<int32_t> bin_of(static_cast<size_t>(ntasks));
+    std::vector<int32_t> bin_count(static_cast<size_t>(n_bins), 0);
+    for (int32_t t : order) {
+        Load top = heap.top();
+        heap.pop();
+        bin_of[t] = top.second;
+        bin_count[top.second]++;
+        top.first += out->tasks[t].count + kTaskFixedCost;
+        heap.push(top);
     }
-    out->spans[n_spans] = static_cast<int32_t>(ntasks);
+    out->bin_ptr.assign(static_cast<size_t>(n_bins) + 1, 0);
+    for (int j = 0; j < n_bins; ++j) out->bin_ptr[j + 1] = out->bin_ptr[j] + bin_count[j];
+    out->bin_tasks.assign(static_cast<size_t>(ntasks), 0);
+    {
+        std::vector<int32_t> fillpos(out->bin_ptr.begin(), out->bin_ptr.end() - 1);
+        for (int64_t t = 0; t < ntasks; ++t) out->bin_tasks[fillpos[bin_of[t]]++] = static_cast<int32_t>(t);
+    }
+
+    // pipeline schedule: one fill per stage-sized run of columns (16 KB of gathered B rows at
+    // 128 tokens: 64 columns of a 2-byte type, 32 of a 4-byte type), bin-major
+    out->kt = 128 / a.es;
+    out->fills.clear();
+    out->bin_fill.assign(static_cast<size_t>(n_bins) + 1, 0);
+    for (int j = 0; j < n_bins; ++j) {
+        for (int32_t i = out->bin_ptr[j]; i < out->bin_ptr[j + 1]; ++i) {
+            const WcsrTask& tk = out->tasks[out->bin_tasks[i]];
+            const int32_t base = out->window_row_ptr[tk.window] + tk.q0;
+            for (int32_t done = 0; done < tk.count; done += out->kt) {
+                const int32_t cnt = std::min(out->kt, tk.count - done);
+                const int32_t first = done == 0, last = done + out->kt >= tk.count;
+                out->fills.push_back(base + done);
+                out->fills.push_back(cnt | (first << 16) | (last << 17));
+            }
+        }
+        if (out->fills.size() / 2 >= (size_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
+        out->bin_fill[j + 1] = static_cast<int32_t>(out->fills.size() / 2);
+    }
     return SPMM_OK;
 }
 

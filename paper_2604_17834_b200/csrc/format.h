@@ -45,7 +45,19 @@ struct WcsrHost {
     // un-swizzled K-major core-matrix layout tcgen05.mma reads.  chunk bytes = wh * 32.
     std::vector<uint8_t> packed;
     std::vector<WcsrTask> tasks;          // window order; chunks of a window consecutive
-    std::vector<int32_t> spans;           // [n_spans+1] task ranges, balanced by cost
+    // Static schedule: tasks are dealt to n_bins bins by the longest-processing-time rule
+    // (cost = columns + kTaskFixedCost; heaviest task first, always into the lightest bin, ties
+    // to the lowest bin index); inside a bin tasks run in ascending order.  CTA c runs bins
+    // c, c + grid, ...
+    std::vector<int32_t> bin_ptr;         // [n_bins+1]
+    std::vector<int32_t> bin_tasks;       // [n_tasks] task indices, bin-major
+    // Device-private pipeline schedule: every task cut into "fills" of at most kt columns (one
+    // shared-memory stage each), stored bin-major in the bins' task order.
+    // fills[i] = {first padded column, count | first<<16 | last<<17} where first / last mark
+    // the first / last fill of a task; bin_fill[j] = index of the first fill of bin j.
+    int kt = 0;
+    std::vector<int32_t> fills;           // 2 * n_fills
+    std::vector<int32_t> bin_fill;        // [n_bins+1]
     // finalisation lists: windows whose C rows the merge kernel writes
     std::vector<int32_t> merge_window;    // split windows then empty windows
     std::vector<int32_t> merge_first;     // first slot (split) or -1 (empty)
@@ -57,7 +69,9 @@ int validate_csr(const CsrView& a);
 int coo_to_csr(int64_t m, int64_t k, int64_t nnz, const int32_t* rows, const int32_t* cols,
                const uint8_t* vals, int es, CsrOwned* out);
 int build_bcsr(const CsrView& a, int b, BcsrHost* out);
-int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_spans, WcsrHost* out);
+// T = 0 picks the sub-task size from the matrix: about a quarter of one bin's share of the
+// padded columns, rounded down to a multiple of 64 and clamped to [128, 4096].
+int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost* out);
 
 // Byte offset of element (row r, padded column q) inside the packed WCSR value array.
 inline size_t wcsr_packed_offset(int wh, int b_col, int es, int r, int64_t q) {

@@ -36,14 +36,17 @@ struct WcsrDevTask {
 
 struct WcsrParams {
     const WcsrDevTask* tasks;
-    const int32_t* spans;        // [n_spans+1]
+    const int32_t* bin_ptr;      // [n_bins+1] ranges of bin_tasks
+    const int32_t* bin_tasks;    // task indices, bin-major
+    const int2* fills;           // {first padded column, count | first<<16 | last<<17}, bin-major
+    const int32_t* bin_fill;     // [n_bins+1] fill ranges
     const int32_t* col_idx;      // window_col_idx [P]
     const uint8_t* packed;       // packed A values
     const void* B;               // k x N row-major
     float* C;
     float* partial;              // [n_slots][16][N]
     int64_t m, N;
-    int32_t n_spans;
+    int32_t n_bins;
     int32_t n_tt;                // token tiles = ceil(N / (128 * groups))
     int* status;
     uint64_t wait_limit_ns;

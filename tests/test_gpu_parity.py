@@ -87,7 +87,9 @@ def _wcsr_case(lib, a, dtype, N, T=0, Bdist=("normal", 0.0, 1.0), seed=19):
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_VALUES, np_dt).view(bits), f["values"].view(bits).ravel())
         plan = F.split_plan(f["window_row_ptr"], info["split_cols"])
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_TASKS, np.int32).reshape(-1, 4), plan)
-        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_SPANS, np.int32), F.task_spans(plan, info["n_ctas"] * 8))
+        bin_ptr, bin_tasks = F.task_bins(plan, info["n_ctas"] * 2)
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_BIN_PTR, np.int32), bin_ptr)
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_BIN_TASKS, np.int32), bin_tasks)
         C = run_gpu(lib, h, Bs, a["m"], N)
         Cr, S = reference(a, Bs, dtype)
         worst = assert_close(C, Cr, S, dtype, "wcsr %s N=%d T=%d" % (dtype, N, T))

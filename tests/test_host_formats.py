@@ -96,7 +96,7 @@ WCSR_CASES = [("tf32", 1000, 900, 0.01, 64), ("fp16", 333, 517, 0.05, 32), ("bf1
 
 
 @pytest.mark.parametrize("dtype,m,k,dens,T", WCSR_CASES)
-def test_wcsr_format_plan_and_spans_are_bit_exact(lib, dtype, m, k, dens, T):
+def test_wcsr_format_plan_and_bins_are_bit_exact(lib, dtype, m, k, dens, T):
     a = wl.random_csr(41 + m, m, k, dens, dtype, empty_rows=tuple(range(16, min(32, m))))
     b_col = 8 if dtype == "tf32" else 16
     h = lib.spmm_wcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, 16, split_cols=T,
@@ -109,9 +109,16 @@ def test_wcsr_format_plan_and_spans_are_bit_exact(lib, dtype, m, k, dens, T):
         assert np.array_equal(_bits(got), _bits(f["values"]).ravel())
         plan = F.split_plan(f["window_row_ptr"], T)
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_TASKS, np.int32).reshape(-1, 4), plan)
-        spans = lib.spmm_export(h, lib.X_WCSR_SPANS, np.int32)
-        assert np.array_equal(spans, F.task_spans(plan, 5 * 8))
-        assert spans[0] == 0 and spans[-1] == plan.shape[0] and np.all(np.diff(spans) >= 0)
+        bin_ptr = lib.spmm_export(h, lib.X_WCSR_BIN_PTR, np.int32)
+        bin_tasks = lib.spmm_export(h, lib.X_WCSR_BIN_TASKS, np.int32)
+        want_ptr, want_tasks = F.task_bins(plan, 5 * 2)
+        assert np.array_equal(bin_ptr, want_ptr) and np.array_equal(bin_tasks, want_tasks)
+        assert sorted(bin_tasks.tolist()) == list(range(plan.shape[0]))      # every task exactly once
+        cost = plan[:, 2].astype(np.int64) + 32
+        loads = np.array([cost[bin_tasks[bin_ptr[j]:bin_ptr[j + 1]]].sum() for j in range(10)])
+        assert loads.max() - loads.min() <= cost.max()                       # LPT balance property
+        for j in range(10):
+            assert np.all(np.diff(bin_tasks[bin_ptr[j]:bin_ptr[j + 1]]) > 0)
         info = lib.spmm_get_info(h, 128)
         P = f["window_col_idx"].shape[0]
         assert info["n_units"] == P and info["stored_values"] == 16 * P
@@ -124,6 +131,16 @@ def test_wcsr_format_plan_and_spans_are_bit_exact(lib, dtype, m, k, dens, T):
         assert info["fill_ratio"] == pytest.approx(F.fill_ratio_wcsr(info["nnz"], P, 16))
     finally:
         lib.spmm_destroy(h)
+
+
+def test_default_split_size(lib):
+    a = wl.wcsr_irregular(seed=4, m=30000, dtype="fp16")
+    h = lib.spmm_wcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "fp16", 16, host_only=True, n_ctas=3)
+    info = lib.spmm_get_info(h)
+    assert info["split_cols"] == F.default_split_cols(info["n_units"], 6)
+    assert 128 <= info["split_cols"] <= 4096 and info["split_cols"] % 64 == 0
+    lib.spmm_destroy(h)
+    assert F.default_split_cols(100, 8) == 128 and F.default_split_cols(10 ** 9, 8) == 4096
 
 
 def test_wcsr_irregular_workload(lib):
