@@ -17,6 +17,9 @@ using namespace spmm;
 namespace {
 
 std::atomic<uint64_t> g_wait_limit_ns{2000000000ull};
+#ifdef SPMM_TRACE
+long long* g_trace = nullptr;
+#endif
 
 inline int elem_size(int dtype) { return dtype == SPMM_TF32 ? 4 : 2; }
 
@@ -85,6 +88,7 @@ struct spmm_handle_s {
     WcsrDevTask* d_tasks = nullptr;
     int32_t* d_bin_ptr = nullptr;
     int32_t* d_bin_tasks = nullptr;
+    int32_t* d_items = nullptr;
     int32_t* d_fills = nullptr;
     int32_t* d_bin_fill = nullptr;
     int32_t* d_merge = nullptr;      // window | first | nparts, each [n_merge]
@@ -120,6 +124,7 @@ void free_handle(spmm_handle_s* h) {
         cudaFree(h->d_tasks);
         cudaFree(h->d_bin_ptr);
         cudaFree(h->d_bin_tasks);
+        cudaFree(h->d_items);
         cudaFree(h->d_fills);
         cudaFree(h->d_bin_fill);
         cudaFree(h->d_merge);
@@ -241,6 +246,15 @@ int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const s
         if (!rc) rc = upload(&h->d_tasks, dt.data(), dt.size() * sizeof(WcsrDevTask));
         if (!rc) rc = upload(&h->d_bin_ptr, f.bin_ptr.data(), f.bin_ptr.size() * 4);
         if (!rc) rc = upload(&h->d_bin_tasks, f.bin_tasks.data(), f.bin_tasks.size() * 4);
+        if (!rc) {
+            std::vector<int32_t> items(4 * f.bin_tasks.size(), 0);
+            for (size_t i = 0; i < f.bin_tasks.size(); ++i) {
+                items[4 * i] = f.tasks[f.bin_tasks[i]].window;
+                items[4 * i + 1] = f.tasks[f.bin_tasks[i]].slot;
+                items[4 * i + 2] = f.tasks[f.bin_tasks[i]].count;
+            }
+            rc = upload(&h->d_items, items.data(), items.size() * 4);
+        }
         if (!rc) rc = upload(&h->d_fills, f.fills.data(), f.fills.size() * 4);
         if (!rc) rc = upload(&h->d_bin_fill, f.bin_fill.data(), f.bin_fill.size() * 4);
         if (!rc) rc = upload(&h->d_merge, mg.data(), mg.size() * 4);
@@ -266,10 +280,32 @@ int make_view(CsrView* v, int64_t m, int64_t k, const int64_t* row_ptr, const in
     return SPMM_OK;
 }
 
+// Map of B for the WCSR row gather: box = one row x 128 bytes.
+int encode_gather_map(CUtensorMap* map, int dtype, const void* base, uint64_t rows, uint64_t cols) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return SPMM_ERR_CUDA;
+    const uint32_t es = dtype == SPMM_TF32 ? 4 : 2;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * es};
+    const cuuint32_t box[2] = {128 / es, 1};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapDataType dt = dtype == SPMM_TF32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                 : (dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
+    const CUtensorMapSwizzle swz = dtype == SPMM_TF32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B;
+    const CUtensorMapL2promotion promo = cols * es >= 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_NONE;
+    CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                    promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SPMM_OK : SPMM_ERR_CUDA;
+}
+
 int ensure_tmB(spmm_handle_s* h, const void* B, int64_t N, int groups) {
     (void)groups;
     if (h->tmB_ptr == B && h->tmB_N == N) return SPMM_OK;
-    int rc = encode_2d_16bit(&h->tmB, h->dtype, B, static_cast<uint64_t>(h->k), static_cast<uint64_t>(N),
+    int rc;
+    if (h->format == 1)
+        rc = encode_gather_map(&h->tmB, h->dtype, B, static_cast<uint64_t>(h->k), static_cast<uint64_t>(N));
+    else
+        rc = encode_2d_16bit(&h->tmB, h->dtype, B, static_cast<uint64_t>(h->k), static_cast<uint64_t>(N),
                              static_cast<uint32_t>(h->bcsr.b), 64, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
     h->tmB_ptr = B;
@@ -333,9 +369,8 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, float* C, float* partial, i
     const int groups = N > 128 ? 2 : 1;
     const int bnt = 128 * groups;
     WcsrParams p;
-    p.tasks = h->d_tasks;
     p.bin_ptr = h->d_bin_ptr;
-    p.bin_tasks = h->d_bin_tasks;
+    p.items = reinterpret_cast<const int4*>(h->d_items);
     p.fills = reinterpret_cast<const int2*>(h->d_fills);
     p.bin_fill = h->d_bin_fill;
     p.col_idx = h->d_idx;
@@ -349,8 +384,14 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, float* C, float* partial, i
     p.n_tt = static_cast<int32_t>((N + bnt - 1) / bnt);
     p.status = h->d_status;
     p.wait_limit_ns = g_wait_limit_ns.load();
+    p.trace = nullptr;
+#ifdef SPMM_TRACE
+    p.trace = g_trace;
+#endif
     if (!f.tasks.empty()) {
-        cudaError_t e = launch_wcsr(h->dtype, groups, p, h->sms, stream);
+        int rc = ensure_tmB(h, B, N, groups);
+        if (rc) return rc;
+        cudaError_t e = launch_wcsr(h->dtype, groups, h->tmB, p, h->sms, stream);
         if (e != cudaSuccess) return SPMM_ERR_CUDA;
     }
     MergeParams mp;
@@ -654,6 +695,10 @@ const char* spmm_status_string(int code) {
         default: return "unknown status";
     }
 }
+
+#ifdef SPMM_TRACE
+void spmm_debug_set_trace(long long* dev_buf) { g_trace = dev_buf; }
+#endif
 
 int spmm_set_wait_limit_ns(uint64_t ns) {
     g_wait_limit_ns.store(ns < 1000 ? 1000 : ns);

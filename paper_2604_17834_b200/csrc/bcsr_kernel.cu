@@ -137,6 +137,8 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(FMT, 128, B, 1, 0);
+            const uint64_t adesc0 = make_smem_desc(0, Cfg::kBoxBytes, 1024, SWZ_128B);
+            const uint64_t bdesc0 = make_smem_desc(0, 16, 8 * Cfg::kARowBytes, Cfg::kASwizzle);
             uint32_t it = 0, tile_i = 0;
             bool ok = true;
             for (int64_t L = blockIdx.x; L < p.total_tiles && ok; L += gridDim.x, ++tile_i) {
@@ -156,19 +158,18 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (!mbar_wait(full_bar(s), ph, ctl, 3)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t sb = smem_base + s * Cfg::kStageBytes;
-                    const uint32_t ab = sb + Cfg::kDenseBytes;
+                    // descriptors differ only in their start-address field (bytes >> 4)
+                    const uint64_t a0 = adesc0 + (sb >> 4);
+                    const uint64_t b0 = bdesc0 + ((sb + Cfg::kDenseBytes) >> 4);
 #pragma unroll
                     for (int ks = 0; ks < B / 16; ++ks) {
-                        uint32_t a_addr;
-                        if constexpr (B <= 64) a_addr = ab + ks * 32;
-                        else a_addr = ab + (ks >> 2) * (B * 128) + (ks & 3) * 32;
-                        const uint64_t bdesc = make_smem_desc(a_addr, 16, 8 * Cfg::kARowBytes, Cfg::kASwizzle);
+                        const uint32_t boff = B <= 64 ? ks * 32 : (ks >> 2) * (B * 128) + (ks & 3) * 32;
                         const uint32_t accum = (q > pb || ks > 0) ? 1u : 0u;
-                        for (int g = 0; g < ngrp; ++g) {
-                            const uint64_t adesc = make_smem_desc(sb + g * 2 * Cfg::kBoxBytes + ks * 2048,
-                                                                  Cfg::kBoxBytes, 1024, SWZ_128B);
-                            umma_ss<false>(d0 + g * B, adesc, bdesc, idesc, accum);
-                        }
+#pragma unroll
+                        for (int g = 0; g < GROUPS; ++g)
+                            if (g < ngrp)
+                                umma_ss<false>(d0 + g * B, a0 + ((g * 2 * Cfg::kBoxBytes + ks * 2048) >> 4),
+                                               b0 + (boff >> 4), idesc, accum);
                     }
                     tc_commit(empty_bar(s));
                 }
@@ -190,7 +191,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const int acc = tile_i & 1;
             const uint32_t aph = (tile_i >> 1) & 1u;
             const bool has_blocks = p.block_row_ptr[tc.I + 1] > p.block_row_ptr[tc.I];
-            if (!mbar_wait(accf_bar(acc), aph, ctl, 4)) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(accf_bar(acc), aph, ctl, 4))) { ok = false; break; }
             tc_fence_after_sync();
             const int64_t row0 = static_cast<int64_t>(tc.I) * B;
             const int rows = static_cast<int>(min_i64(B, p.m - row0));

@@ -35,9 +35,8 @@ struct WcsrDevTask {
 };
 
 struct WcsrParams {
-    const WcsrDevTask* tasks;
-    const int32_t* bin_ptr;      // [n_bins+1] ranges of bin_tasks
-    const int32_t* bin_tasks;    // task indices, bin-major
+    const int32_t* bin_ptr;      // [n_bins+1] ranges of items
+    const int4* items;           // {window, partial slot or -1, columns, 0} of every task, bin-major
     const int2* fills;           // {first padded column, count | first<<16 | last<<17}, bin-major
     const int32_t* bin_fill;     // [n_bins+1] fill ranges
     const int32_t* col_idx;      // window_col_idx [P]
@@ -50,10 +49,13 @@ struct WcsrParams {
     int32_t n_tt;                // token tiles = ceil(N / (128 * groups))
     int* status;
     uint64_t wait_limit_ns;
+    long long* trace;            // tuning builds only (SPMM_TRACE); nullptr otherwise
 };
 
-// dtype: 0 bf16, 1 fp16, 2 tf32.  groups: 1 or 2.
-cudaError_t launch_wcsr(int dtype, int groups, const WcsrParams& p, int grid, cudaStream_t stream);
+// dtype: 0 bf16, 1 fp16, 2 tf32.  groups: 1 or 2.  tmB: 2-D map of B (k rows x N), box = 128
+// bytes x 1 row, 128-byte swizzle (32-byte atoms for tf32), used in row-gather mode.
+cudaError_t launch_wcsr(int dtype, int groups, const CUtensorMap& tmB, const WcsrParams& p, int sms,
+                        cudaStream_t stream);
 
 struct MergeParams {
     const int32_t* window;   // [n] windows the merge writes

@@ -8,11 +8,11 @@
 // window rows as the MMA N side (operand = the packed window tile, K-major, un-swizzled).
 //
 // Roles (288 threads, persistent CTAs):
-//   warps 0-3   gather producers: per stage read KT column indices and copy the matching
-//               B rows with 16-byte cp.async (zero fill for -1 pads) into a STAGES-deep
-//               ring; thread 0 also bulk-copies the contiguous packed A tile.  A stage is
-//               published LAG fills later (wait_group + proxy fence + mbarrier arrive), so
-//               LAG + 1 stages of loads stay in flight per thread.
+//   warps 0-3   gather producers: warp w owns the CTA's fills w, w + 4, ...; per fill every
+//               lane reads four column indices and issues one TMA row-gather (four B rows x
+//               128 bytes, hardware swizzle, zero fill for -1 pads) into a STAGES-deep ring;
+//               lane 0 also bulk-copies the contiguous packed A tile.  Completion is counted
+//               in bytes on the stage's mbarrier, so producers never wait for data.
 //   warp 4      MMA issuer (one thread): count / b_col tcgen05.mma per group and stage.
 //   warps 5-8   epilogue: tcgen05.ld, release the TMEM buffer, store to C (unsplit window)
 //               or to the task's partial tile (split window).
@@ -30,9 +30,26 @@ namespace spmm {
 
 namespace {
 
+// Optional per-CTA cycle accounting for kernel tuning (compiled out unless SPMM_TRACE is
+// defined; the buffer is WcsrParams::trace, 16 counters per CTA).
+#ifdef SPMM_TRACE
+#define TRACE_DECL(name) long long name = 0
+#define TRACE_T0(t) const long long t = clock64()
+#define TRACE_ADD(acc, t) acc += clock64() - t
+#define TRACE_PUT(slot, val) do { if (p.trace) p.trace[blockIdx.x * 16 + (slot)] = (val); } while (0)
+#else
+#define TRACE_DECL(name)
+#define TRACE_T0(t)
+#define TRACE_ADD(acc, t)
+#define TRACE_PUT(slot, val)
+#endif
+
 constexpr int kWH = 16;
 constexpr int kProducerWarps = 4;
-constexpr int kNAcc = 4;
+// A 128 x 16 x K MMA is tiny, and MMAs that accumulate into the same TMEM tile serialise on
+// it, so the K steps of an item rotate over kNSub independent partial accumulators that the
+// epilogue adds (in index order).
+constexpr int kNSub = 4;
 
 template <int ES, int GROUPS, int KT, int STAGES>
 struct WcsrCfg {
@@ -40,60 +57,44 @@ struct WcsrCfg {
     static constexpr int kKStep = 32 / ES;                  // columns per MMA (= b_col)
     static constexpr int kBnT = 128 * GROUPS;
     static constexpr int kRowBytes = kBnT * ES;
-    static constexpr int kCh = kRowBytes / 16;              // 16-byte chunks per gathered row
-    static constexpr int kIssues = KT * kCh / 32;           // cp.async per lane per fill
-    static constexpr int kIdxRegs = (KT + 31) / 32;         // column indices held per lane
+    static constexpr int kSegs = kRowBytes / 128;           // 128-byte segments per gathered row
+    static constexpr int kGathers = (KT / 4) * kSegs;       // row-gather instructions per full fill
+    static constexpr int kRounds = (kGathers + 31) / 32;    // per lane
     static constexpr int kAtomStride = KT * 128;            // bytes between MN atoms
     static constexpr int kAtomsPerGroup = ES;               // 128 tokens * ES / 128 B
     static constexpr int kDenseBytes = KT * kRowBytes;
     static constexpr int kABytes = (KT / kKStep) * (kWH * 32);
     static constexpr int kStageBytes = kDenseBytes + kABytes;
-    static constexpr int kAccCols = GROUPS * kWH;
-    static constexpr int kTmemCols = kNAcc * kAccCols < 32 ? 32 : kNAcc * kAccCols;
+    static constexpr int kNAcc = GROUPS == 1 ? 4 : 2;       // items with live accumulators
+    static constexpr int kAccCols = GROUPS * kNSub * kWH;   // TMEM columns of one item
+    static constexpr int kTmemCols = kNAcc * kAccCols;      // 256
     static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 + 256;
     static_assert(KT % 8 == 0 && KT % kKStep == 0 && KT <= 64, "stage shape");
+    static_assert(kGathers % 32 == 0, "gather instructions are dealt to whole warps");
     static_assert(kStageBytes % 1024 == 0, "stage alignment");
 };
 
-// Walks the fills a CTA owns, in the order every role uses: bins blockIdx.x, +grid, ...;
-// inside a bin all token tiles; inside a token tile the bin's fills.
-struct FillCursor {
-    int sp, tt, f, f_end;
-    __device__ __forceinline__ void load_bin(const WcsrParams& p) {
-        if (sp < p.n_bins) {
-            f = __ldg(p.bin_fill + sp);
-            f_end = __ldg(p.bin_fill + sp + 1);
+// Every role of a CTA walks the same sequence of segments: bins blockIdx.x, +grid, ...; per
+// bin one segment per token tile.  A segment is a contiguous range of the (bin-major) fill
+// and item arrays, so descriptors are fetched 32 at a time with one coalesced load and
+// handed out with warp shuffles.
+struct SegIter {
+    int b, tt;
+    __device__ __forceinline__ void init() { b = blockIdx.x; tt = -1; }
+    // advance to the next segment; false when the CTA has no more work
+    __device__ __forceinline__ bool next(const WcsrParams& p) {
+        if (b >= p.n_bins) return false;
+        if (++tt >= p.n_tt) {
+            tt = 0;
+            b += gridDim.x;
         }
-    }
-    __device__ __forceinline__ void normalise(const WcsrParams& p) {
-        while (sp < p.n_bins && f >= f_end) {
-            if (f_end > __ldg(p.bin_fill + sp) && tt + 1 < p.n_tt) {
-                ++tt;
-                f = __ldg(p.bin_fill + sp);
-            } else {
-                tt = 0;
-                sp += gridDim.x;
-                load_bin(p);
-            }
-        }
-    }
-    __device__ __forceinline__ void init(const WcsrParams& p) {
-        sp = blockIdx.x;
-        tt = 0;
-        f = f_end = 0;
-        load_bin(p);
-        normalise(p);
-    }
-    __device__ __forceinline__ bool done(const WcsrParams& p) const { return sp >= p.n_bins; }
-    __device__ __forceinline__ void step(const WcsrParams& p) {
-        ++f;
-        normalise(p);
+        return b < p.n_bins;
     }
 };
 
 template <int ES, int FMT, int GROUPS, int KT, int STAGES>
 __global__ void __launch_bounds__(288, (WcsrCfg<ES, GROUPS, KT, STAGES>::kSmemBytes + 1024) * 2 <= 227 * 1024 ? 2 : 1)
-wcsr_spmm_kernel(const WcsrParams p) {
+wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
     using Cfg = WcsrCfg<ES, GROUPS, KT, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -103,18 +104,19 @@ wcsr_spmm_kernel(const WcsrParams p) {
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
     auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
-    auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + kNAcc + a); };
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * STAGES + 2 * kNAcc);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * STAGES + 2 * kNAcc + 1);
+    auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + Cfg::kNAcc + a); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * STAGES + 2 * Cfg::kNAcc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * STAGES + 2 * Cfg::kNAcc + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     WaitCtl ctl{abort_flag, p.status, p.wait_limit_ns};
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 32); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < kNAcc; ++a) { mbar_init(accf_bar(a), 1); mbar_init(acce_bar(a), 4); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < Cfg::kNAcc; ++a) { mbar_init(accf_bar(a), 1); mbar_init(acce_bar(a), 4); }
         *abort_flag = 0;
         fence_mbar_init();
+        prefetch_tmap(&tmB);
     }
     if (warp == 4) {
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);
@@ -125,202 +127,264 @@ wcsr_spmm_kernel(const WcsrParams p) {
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     const int64_t N = p.N;
+    const int2 kNoDesc = make_int2(0, 0);
 
     if (warp < kProducerWarps) {
         // ------------------------------------------------------------------ gather producers
-        // Warp w fills stages for the CTA's fills w, w + 4, ...; a fill is one warp's job from
-        // the index loads to the mbarrier arrive, so four fills are always in progress.
-        const int c = lane % Cfg::kCh;               // my 16-byte chunk inside a gathered row
-        const int rsub = lane / Cfg::kCh;            // my row inside one issue (kCh < 32)
-        constexpr int kRowsPerIssue = Cfg::kCh >= 32 ? 1 : 32 / Cfg::kCh;
-        constexpr int kIssuesPerRow = Cfg::kCh > 32 ? Cfg::kCh / 32 : 1;
-        const uint8_t* Bp = static_cast<const uint8_t*>(p.B);
-        const size_t row_pitch = static_cast<size_t>(N) * ES;
-
-        // Three fills are tracked per warp: `cur` (indices in registers, rows being copied),
-        // `n1` (descriptor in registers, indices requested while cur's rows travel) and `n2`
-        // (descriptor requested), so neither a descriptor nor an index load stalls the copy loop.
-        FillCursor cur;
-        cur.init(p);
-        for (int i = 0; i < warp && !cur.done(p); ++i) cur.step(p);
-        FillCursor n1 = cur;
-        for (int i = 0; i < kProducerWarps && !n1.done(p); ++i) n1.step(p);
-        uint32_t it = warp;
-        bool have = !cur.done(p), have1 = !n1.done(p);
-        int2 d_cur = make_int2(0, 0), d_n1 = make_int2(0, 0);
-        int idx_cur[Cfg::kIdxRegs];
-        if (have) d_cur = __ldg(p.fills + cur.f);
-        if (have1) d_n1 = __ldg(p.fills + n1.f);
-        if (have) {
-            const int cnt = d_cur.y & 0xFFFF;
+        // Lane l of the owning warp issues gather u = l (+32 per round): row group u / kSegs
+        // (rows 4*rg .. 4*rg+3 of the fill), 128-byte segment u % kSegs of those rows.
+        auto load_idx = [&](const int2 d, int4 (&idx)[Cfg::kRounds]) {
+            const int cnt = d.y & 0xFFFF;
 #pragma unroll
-            for (int j = 0; j < Cfg::kIdxRegs; ++j)
-                idx_cur[j] = (j * 32 + lane < cnt) ? __ldg(p.col_idx + d_cur.x + j * 32 + lane) : -1;
-        }
-        bool ok = true;
-        while (have) {
-            FillCursor n2 = n1;
-            for (int i = 0; i < kProducerWarps && !n2.done(p); ++i) n2.step(p);
-            const bool have2 = have1 && !n2.done(p);
-            int2 d_n2 = make_int2(0, 0);
-            if (have2) d_n2 = __ldg(p.fills + n2.f);
-
-            const int s = it % STAGES;
-            const uint32_t ph = (it / STAGES) & 1u;
-            const int q = d_cur.x;
-            const int cnt = d_cur.y & 0xFFFF;
-            const int n0 = cur.tt * Cfg::kBnT;
-            if (!mbar_wait(empty_bar(s), ph ^ 1u, ctl, 11)) { ok = false; break; }
-            const uint32_t sb = smem_base + s * Cfg::kStageBytes;
-            if (lane == 0) {
-                const uint32_t abytes = (cnt / Cfg::kKStep) * (kWH * 32);
-                mbar_expect_tx(full_bar(s), abytes);
-                bulk_load_1d(sb + Cfg::kDenseBytes, p.packed + static_cast<size_t>(q / Cfg::kKStep) * (kWH * 32),
-                             abytes, full_bar(s));
+            for (int r = 0; r < Cfg::kRounds; ++r) {
+                const int rg = (lane + 32 * r) / Cfg::kSegs;
+                idx[r] = (rg * 4 < cnt) ? __ldg(reinterpret_cast<const int4*>(p.col_idx + d.x) + rg)
+                                        : make_int4(-1, -1, -1, -1);
             }
-#pragma unroll
-            for (int i = 0; i < Cfg::kIssues; ++i) {
-                const int r = (i / kIssuesPerRow) * kRowsPerIssue + rsub;
-                const int cc = c + (i % kIssuesPerRow) * 32;        // chunk inside the row
-                // (the register holding row r's index is known at compile time: rsub < kRowsPerIssue)
-                const int idx = __shfl_sync(0xffffffffu, idx_cur[((i / kIssuesPerRow) * kRowsPerIssue) >> 5], r & 31);
-                if (r < cnt && n0 + cc * Cfg::kE16 < N) {
-                    uint32_t dst = sb + (cc >> 3) * Cfg::kAtomStride + r * 128;
-                    if constexpr (ES == 2) {
-                        // 128-byte swizzle: 16-byte chunk index ^= row % 8
-                        dst += ((cc & 7) ^ (r & 7)) << 4;
-                    } else {
-                        // 128-byte swizzle with 32-byte atoms (the only MN-major layout for
-                        // 32-bit operands): 32-byte chunk index ^= row % 4
-                        dst += ((((cc & 7) >> 1) ^ (r & 3)) << 5) + ((cc & 1) << 4);
+        };
+
+        TRACE_DECL(tr_empty);
+        TRACE_DECL(tr_copy);
+        TRACE_DECL(tr_issue_p);
+        TRACE_DECL(tr_fills);
+        TRACE_T0(tr_start);
+        SegIter seg;
+        seg.init();
+        uint32_t it0 = 0;                            // CTA-wide number of fills before this segment
+        uint32_t last_it = 0;
+        bool issued_any = false, ok = true;
+        // column indices of this warp's current fill and of its next two fills (requested two
+        // fills ahead, so their latency never sits in the issue loop)
+        int4 idx_cur[Cfg::kRounds], idx_n1[Cfg::kRounds], idx_n2[Cfg::kRounds];
+        bool rdy0 = false, rdy1 = false;
+        while (ok && seg.next(p)) {
+            const int f0 = __ldg(p.bin_fill + seg.b), f1 = __ldg(p.bin_fill + seg.b + 1);
+            const int n0 = seg.tt * Cfg::kBnT;
+            const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
+            const int nseg = (nvalid * ES + 127) >> 7;       // 128-byte segments that hold tokens < N
+            int2 win = (f0 + lane < f1) ? __ldg(p.fills + f0 + lane) : kNoDesc;
+            for (int wbase = f0; wbase < f1 && ok; wbase += 32) {
+                const int2 nwin = (wbase + 32 + lane < f1) ? __ldg(p.fills + wbase + 32 + lane) : kNoDesc;
+                const uint32_t itw = it0 + static_cast<uint32_t>(wbase - f0);   // counter of window slot 0
+                int j = static_cast<int>((static_cast<uint32_t>(warp) - itw) & 3u);
+                for (; j < 32 && wbase + j < f1; j += kProducerWarps) {
+                    const uint32_t it = itw + j;
+                    int2 d;
+                    d.x = __shfl_sync(0xffffffffu, win.x, j);
+                    d.y = __shfl_sync(0xffffffffu, win.y, j);
+                    // this warp's next two fills, if they are in this segment
+                    const int j1 = j + kProducerWarps, j2 = j + 2 * kProducerWarps;
+                    const bool have1 = wbase + j1 < f1, have2 = wbase + j2 < f1;
+                    int2 d1, d2;
+                    d1.x = __shfl_sync(0xffffffffu, j1 < 32 ? win.x : nwin.x, j1 & 31);
+                    d1.y = __shfl_sync(0xffffffffu, j1 < 32 ? win.y : nwin.y, j1 & 31);
+                    d2.x = __shfl_sync(0xffffffffu, j2 < 32 ? win.x : nwin.x, j2 & 31);
+                    d2.y = __shfl_sync(0xffffffffu, j2 < 32 ? win.y : nwin.y, j2 & 31);
+                    if (!rdy0) load_idx(d, idx_cur);
+                    if (have1 && !rdy1) load_idx(d1, idx_n1);
+                    if (have2) load_idx(d2, idx_n2);
+
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    const int q = d.x;
+                    const int cnt = d.y & 0xFFFF;
+                    TRACE_T0(tr_a);
+                    if (!__all_sync(0xffffffffu, mbar_wait(empty_bar(s), ph ^ 1u, ctl, 11))) { ok = false; break; }
+                    TRACE_ADD(tr_empty, tr_a);
+                    const uint32_t sb = smem_base + s * Cfg::kStageBytes;
+                    TRACE_T0(tr_e);
+                    if (lane == 0) {
+                        const uint32_t abytes = (cnt / Cfg::kKStep) * (kWH * 32);
+                        mbar_arrive_expect_tx(full_bar(s), abytes + (cnt / 4) * nseg * 512);
+                        bulk_load_1d(sb + Cfg::kDenseBytes,
+                                     p.packed + static_cast<size_t>(q / Cfg::kKStep) * (kWH * 32), abytes, full_bar(s));
                     }
-                    const bool valid = idx >= 0;
-                    const uint8_t* src = Bp + (valid ? static_cast<size_t>(idx) * row_pitch +
-                                                           (static_cast<size_t>(n0) + cc * Cfg::kE16) * ES
-                                                     : 0);
-                    cp_async_16(dst, src, valid);
+                    __syncwarp();
+                    issued_any = true;
+                    last_it = it;
+#pragma unroll
+                    for (int r = 0; r < Cfg::kRounds; ++r) {
+                        const int u = lane + 32 * r;
+                        const int rg = u / Cfg::kSegs, sg = u % Cfg::kSegs;
+                        if (rg * 4 < cnt && sg < nseg)
+                            tma_gather4_2d(sb + sg * Cfg::kAtomStride + rg * 512, &tmB, full_bar(s),
+                                           n0 + sg * (128 / ES), idx_cur[r].x, idx_cur[r].y, idx_cur[r].z, idx_cur[r].w);
+                    }
+                    TRACE_ADD(tr_issue_p, tr_e);
+#ifdef SPMM_TRACE
+                    ++tr_fills;
+#endif
+#pragma unroll
+                    for (int r = 0; r < Cfg::kRounds; ++r) {
+                        idx_cur[r] = idx_n1[r];
+                        idx_n1[r] = idx_n2[r];
+                    }
+                    rdy0 = have1;
+                    rdy1 = have2;
                 }
+                win = nwin;
             }
-            cp_async_commit();
-            // the next fill's indices travel while this fill's rows do
-            int idx_n1[Cfg::kIdxRegs];
-#pragma unroll
-            for (int j = 0; j < Cfg::kIdxRegs; ++j) idx_n1[j] = -1;
-            if (have1) {
-                const int cn = d_n1.y & 0xFFFF;
-#pragma unroll
-                for (int j = 0; j < Cfg::kIdxRegs; ++j)
-                    if (j * 32 + lane < cn) idx_n1[j] = __ldg(p.col_idx + d_n1.x + j * 32 + lane);
-            }
-            cp_async_wait<0>();
-            fence_proxy_async_smem();
-            mbar_arrive(full_bar(s));
-            cur = n1;
-            n1 = n2;
-            d_cur = d_n1;
-            d_n1 = d_n2;
-#pragma unroll
-            for (int j = 0; j < Cfg::kIdxRegs; ++j) idx_cur[j] = idx_n1[j];
-            have = have1;
-            have1 = have2;
-            it += kProducerWarps;
+            it0 += static_cast<uint32_t>(f1 - f0);
         }
-        cp_async_wait<0>();
-        if (!ok && lane == 0 && it >= kProducerWarps) {
-            // abort path: the A tile of this warp's previous fill may still be in flight
-            const uint32_t j = it - kProducerWarps;
+#ifdef SPMM_TRACE
+        if (warp == 0 && lane == 0) {
+            TRACE_PUT(0, clock64() - tr_start);
+            TRACE_PUT(1, tr_empty);
+            TRACE_PUT(2, tr_copy);
+            TRACE_PUT(3, tr_fills);
+            TRACE_PUT(14, tr_issue_p);
+        }
+#endif
+        if (!ok && lane == 0 && issued_any) {
+            // abort path: this warp's last fill may still be in flight
             const uint64_t t0 = globaltimer_ns();
-            while (!mbar_try_wait(full_bar(j % STAGES), (j / STAGES) & 1u) && globaltimer_ns() - t0 < 2000000ull) {}
+            while (!mbar_try_wait(full_bar(last_it % STAGES), (last_it / STAGES) & 1u) &&
+                   globaltimer_ns() - t0 < 2000000ull) {}
         }
     } else if (warp == 4) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(FMT, 128, kWH, 1, 0);
-            FillCursor cur;
-            cur.init(p);
-            uint32_t it = 0, item = 0;
-            bool have = !cur.done(p);
-            int2 d_cur = make_int2(0, 0);
-            if (have) d_cur = __ldg(p.fills + cur.f);
-            uint32_t d0 = 0;
-            int acc = 0;
-            while (have) {
-                FillCursor nxt = cur;
-                nxt.step(p);
-                const bool have_n = !nxt.done(p);
-                int2 d_nxt = make_int2(0, 0);
-                if (have_n) d_nxt = __ldg(p.fills + nxt.f);
-
-                const int cnt = d_cur.y & 0xFFFF;
-                const bool first = (d_cur.y >> 16) & 1, last = (d_cur.y >> 17) & 1;
-                const int n0 = cur.tt * Cfg::kBnT;
-                const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
-                const int ngrp = (nvalid + 127) >> 7;
-                if (first) {
-                    acc = item % kNAcc;
-                    const uint32_t aph = (item / kNAcc) & 1u;
-                    if (!mbar_wait(acce_bar(acc), aph ^ 1u, ctl, 12)) break;
-                    tc_fence_after_sync();
-                    d0 = tmem_base + acc * Cfg::kAccCols;
-                }
-                const int s = it % STAGES;
-                const uint32_t ph = (it / STAGES) & 1u;
-                if (!mbar_wait(full_bar(s), ph, ctl, 13)) break;
-                tc_fence_after_sync();
-                const uint32_t sb = smem_base + s * Cfg::kStageBytes;
-                const int nks = cnt / Cfg::kKStep;
-                for (int ks = 0; ks < nks; ++ks) {
-                    const uint64_t bdesc = make_smem_desc(sb + Cfg::kDenseBytes + ks * (kWH * 32), kWH * 16, 128, SWZ_NONE);
-                    const uint32_t accum = (!first || ks > 0) ? 1u : 0u;
-                    for (int g = 0; g < ngrp; ++g) {
-                        const uint64_t adesc = make_smem_desc(
-                            sb + g * Cfg::kAtomsPerGroup * Cfg::kAtomStride + ks * (Cfg::kKStep / 8) * 1024,
-                            Cfg::kAtomStride, ES == 2 ? 1024 : 512, ES == 2 ? SWZ_128B : SWZ_128B_BASE32B);
-                        umma_ss<FMT == 2>(d0 + g * kWH, adesc, bdesc, idesc, accum);
+        // The whole warp walks the fill list (descriptor windows via shuffles) and waits for
+        // stages and accumulators; one elected lane issues the MMAs and commits.
+        constexpr uint32_t idesc = make_idesc(FMT, 128, kWH, 1, 0);
+        const uint64_t adesc0 = make_smem_desc(0, Cfg::kAtomStride, ES == 2 ? 1024 : 512, ES == 2 ? SWZ_128B : SWZ_128B_BASE32B);
+        const uint64_t bdesc0 = make_smem_desc(0, kWH * 16, 128, SWZ_NONE);
+        TRACE_DECL(tr_full);
+        TRACE_DECL(tr_acce);
+        TRACE_DECL(tr_issue);
+        TRACE_DECL(tr_commit);
+        TRACE_T0(tr_start);
+        SegIter seg;
+        seg.init();
+        uint32_t it = 0, item = 0, d0 = 0, kstep_item = 0;
+        int acc = 0;
+        bool ok = true;
+        while (ok && seg.next(p)) {
+            const int f0 = __ldg(p.bin_fill + seg.b), f1 = __ldg(p.bin_fill + seg.b + 1);
+            const int n0 = seg.tt * Cfg::kBnT;
+            const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
+            const int ngrp = (nvalid + 127) >> 7;
+            int2 win = (f0 + lane < f1) ? __ldg(p.fills + f0 + lane) : kNoDesc;
+            for (int wbase = f0; wbase < f1 && ok; wbase += 32) {
+                const int2 nwin = (wbase + 32 + lane < f1) ? __ldg(p.fills + wbase + 32 + lane) : kNoDesc;
+                const int nj = min(32, f1 - wbase);
+                for (int j = 0; j < nj; ++j, ++it) {
+                    const int dy = __shfl_sync(0xffffffffu, win.y, j);
+                    const int cnt = dy & 0xFFFF;
+                    const bool first = (dy >> 16) & 1, last = (dy >> 17) & 1;
+                    // warp-uniform control flow: every lane waits and builds the (uniform)
+                    // descriptors, one elected lane issues the tcgen05 instructions
+                    if (first) {
+                        acc = item % Cfg::kNAcc;
+                        const uint32_t aph = (item / Cfg::kNAcc) & 1u;
+                        TRACE_T0(tr_a);
+                        ok = __all_sync(0xffffffffu, mbar_wait(acce_bar(acc), aph ^ 1u, ctl, 12));
+                        TRACE_ADD(tr_acce, tr_a);
+                        tc_fence_after_sync();
+                        d0 = tmem_base + acc * Cfg::kAccCols;
+                        kstep_item = 0;
                     }
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    TRACE_T0(tr_b);
+                    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(full_bar(s), ph, ctl, 13));
+                    TRACE_ADD(tr_full, tr_b);
+                    if (ok) {
+                        tc_fence_after_sync();
+                        TRACE_T0(tr_c);
+                        const uint32_t sb = smem_base + s * Cfg::kStageBytes;
+                        const int nks = cnt / Cfg::kKStep;
+                        if (elect_one()) {
+                            // descriptors differ only in their start-address field (bytes >> 4)
+                            const uint64_t a0 = adesc0 + (sb >> 4);
+                            const uint64_t b0 = bdesc0 + ((sb + Cfg::kDenseBytes) >> 4);
+                            uint32_t kk = kstep_item;
+                            for (int ks = 0; ks < nks; ++ks, ++kk) {
+                                const uint32_t dsub = d0 + (kk & (kNSub - 1)) * kWH;
+                                const uint32_t accum = kk >= kNSub ? 1u : 0u;    // first use overwrites
+#pragma unroll
+                                for (int g = 0; g < GROUPS; ++g)
+                                    if (g < ngrp)
+                                        umma_ss<FMT == 2>(dsub + g * kNSub * kWH,
+                                                          a0 + ((g * Cfg::kAtomsPerGroup * Cfg::kAtomStride + ks * (Cfg::kKStep / 8) * 1024) >> 4),
+                                                          b0 + ((ks * (kWH * 32)) >> 4), idesc, accum);
+                            }
+                            tc_commit(empty_bar(s));
+                            if (last) tc_commit(accf_bar(acc));
+                        }
+                        __syncwarp();
+                        kstep_item += nks;
+                        TRACE_ADD(tr_issue, tr_c);
+                    }
+                    if (last) ++item;
+                    if (!ok) break;
                 }
-                tc_commit(empty_bar(s));
-                if (last) {
-                    tc_commit(accf_bar(acc));
-                    ++item;
-                }
-                cur = nxt;
-                d_cur = d_nxt;
-                have = have_n;
-                ++it;
+                win = nwin;
             }
         }
+#ifdef SPMM_TRACE
+        if (lane == 0) {
+            TRACE_PUT(4, clock64() - tr_start);
+            TRACE_PUT(5, tr_full);
+            TRACE_PUT(6, tr_acce);
+            TRACE_PUT(7, (long long)it);
+            TRACE_PUT(12, tr_issue);
+            TRACE_PUT(13, tr_commit);
+        }
+#endif
     } else {
         // ------------------------------------------------------------------ epilogue warps
         const int qd = warp & 3;
+        TRACE_DECL(tr_accf);
+        TRACE_T0(tr_start);
+        SegIter seg;
+        seg.init();
         uint32_t item = 0;
         bool ok = true;
-        for (int sp = blockIdx.x; sp < p.n_bins && ok; sp += gridDim.x) {
-            const int t_begin = p.bin_ptr[sp], t_end = p.bin_ptr[sp + 1];
-            for (int tt = 0; tt < p.n_tt && ok; ++tt) {
-                const int n0 = tt * Cfg::kBnT;
-                for (int ti = t_begin; ti < t_end; ++ti, ++item) {
-                    const int t = __ldg(p.bin_tasks + ti);
-                    const WcsrDevTask task = p.tasks[t];
+        while (ok && seg.next(p)) {
+            const int i0 = __ldg(p.bin_ptr + seg.b), i1 = __ldg(p.bin_ptr + seg.b + 1);
+            const int n0 = seg.tt * Cfg::kBnT;
+            const int4 kNoItem = make_int4(0, 0, 0, 0);
+            int4 win = (i0 + lane < i1) ? __ldg(p.items + i0 + lane) : kNoItem;
+            for (int wbase = i0; wbase < i1 && ok; wbase += 32) {
+                const int4 nwin = (wbase + 32 + lane < i1) ? __ldg(p.items + wbase + 32 + lane) : kNoItem;
+                const int nj = min(32, i1 - wbase);
+                for (int j = 0; j < nj; ++j, ++item) {
+                    const int window = __shfl_sync(0xffffffffu, win.x, j);
+                    const int slot = __shfl_sync(0xffffffffu, win.y, j);
+                    const int nks = __shfl_sync(0xffffffffu, win.z, j) / Cfg::kKStep;
+                    const int nsub = nks < kNSub ? nks : kNSub;
                     float* out;
                     int rows;
-                    if (task.slot < 0) {
-                        const int64_t row0 = static_cast<int64_t>(task.window) * kWH;
+                    if (slot < 0) {
+                        const int64_t row0 = static_cast<int64_t>(window) * kWH;
                         out = p.C + row0 * N;
                         rows = static_cast<int>(min_i64(kWH, p.m - row0));
                     } else {
-                        out = p.partial + static_cast<int64_t>(task.slot) * kWH * N;
+                        out = p.partial + static_cast<int64_t>(slot) * kWH * N;
                         rows = kWH;
                     }
-                    const int acc = item % kNAcc;
-                    const uint32_t aph = (item / kNAcc) & 1u;
-                    if (!mbar_wait(accf_bar(acc), aph, ctl, 14)) { ok = false; break; }
+                    const int acc = item % Cfg::kNAcc;
+                    const uint32_t aph = (item / Cfg::kNAcc) & 1u;
+                    TRACE_T0(tr_a);
+                    if (!__all_sync(0xffffffffu, mbar_wait(accf_bar(acc), aph, ctl, 14))) { ok = false; break; }
+                    TRACE_ADD(tr_accf, tr_a);
                     tc_fence_after_sync();
-                    uint32_t v[GROUPS][16];
+                    float v[GROUPS][16];
+                    const uint32_t tbase = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + acc * Cfg::kAccCols;
 #pragma unroll
-                    for (int g = 0; g < GROUPS; ++g)
-                        tmem_ld_x16(tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + acc * Cfg::kAccCols + g * kWH, v[g]);
-                    tmem_ld_wait();
+                    for (int g = 0; g < GROUPS; ++g) {
+                        uint32_t u[16];
+                        tmem_ld_x16(tbase + (g * kNSub) * kWH, u);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int jr = 0; jr < kWH; ++jr) v[g][jr] = __uint_as_float(u[jr]);
+                        for (int sub = 1; sub < nsub; ++sub) {
+                            tmem_ld_x16(tbase + (g * kNSub + sub) * kWH, u);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int jr = 0; jr < kWH; ++jr) v[g][jr] += __uint_as_float(u[jr]);
+                        }
+                    }
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(acce_bar(acc));
@@ -329,13 +393,22 @@ wcsr_spmm_kernel(const WcsrParams p) {
                         const int n = n0 + g * 128 + qd * 32 + lane;
                         if (n < N) {
 #pragma unroll
-                            for (int j = 0; j < kWH; ++j)
-                                if (j < rows) out[static_cast<int64_t>(j) * N + n] = __uint_as_float(v[g][j]);
+                            for (int jr = 0; jr < kWH; ++jr)
+                                if (jr < rows) out[static_cast<int64_t>(jr) * N + n] = v[g][jr];
                         }
                     }
                 }
+                win = nwin;
             }
         }
+#ifdef SPMM_TRACE
+        if (warp == 5 && lane == 0) {
+            TRACE_PUT(8, clock64() - tr_start);
+            TRACE_PUT(9, tr_accf);
+            TRACE_PUT(10, (long long)item);
+            TRACE_PUT(11, (long long)globaltimer_ns());
+        }
+#endif
     }
 
     tc_fence_before_sync();
@@ -372,7 +445,7 @@ wcsr_merge_kernel(const MergeParams p) {
 }
 
 template <int ES, int FMT, int GROUPS, int KT, int STAGES>
-cudaError_t launch_one(const WcsrParams& p, int sms, cudaStream_t stream) {
+cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
     using Cfg = WcsrCfg<ES, GROUPS, KT, STAGES>;
     auto kfn = wcsr_spmm_kernel<ES, FMT, GROUPS, KT, STAGES>;
     static int occ = 0;
@@ -390,22 +463,22 @@ cudaError_t launch_one(const WcsrParams& p, int sms, cudaStream_t stream) {
     int grid = sms * occ;
     if (grid > p.n_bins) grid = p.n_bins;
     if (grid < 1) return cudaSuccess;
-    kfn<<<grid, 288, Cfg::kSmemBytes, stream>>>(p);
+    kfn<<<grid, 288, Cfg::kSmemBytes, stream>>>(tmB, p);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_wcsr(int dtype, int groups, const WcsrParams& p, int sms, cudaStream_t stream) {
+cudaError_t launch_wcsr(int dtype, int groups, const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
     if (dtype == 2) {
-        if (groups == 1) return launch_one<4, 2, 1, 32, 6>(p, sms, stream);
-        if (groups == 2) return launch_one<4, 2, 2, 32, 6>(p, sms, stream);
+        if (groups == 1) return launch_one<4, 2, 1, 32, 6>(tmB, p, sms, stream);
+        if (groups == 2) return launch_one<4, 2, 2, 32, 6>(tmB, p, sms, stream);
     } else if (dtype == 1) {
-        if (groups == 1) return launch_one<2, 0, 1, 64, 6>(p, sms, stream);
-        if (groups == 2) return launch_one<2, 0, 2, 64, 6>(p, sms, stream);
+        if (groups == 1) return launch_one<2, 0, 1, 64, 6>(tmB, p, sms, stream);
+        if (groups == 2) return launch_one<2, 0, 2, 64, 6>(tmB, p, sms, stream);
     } else if (dtype == 0) {
-        if (groups == 1) return launch_one<2, 1, 1, 64, 6>(p, sms, stream);
-        if (groups == 2) return launch_one<2, 1, 2, 64, 6>(p, sms, stream);
+        if (groups == 1) return launch_one<2, 1, 1, 64, 6>(tmB, p, sms, stream);
+        if (groups == 2) return launch_one<2, 1, 2, 64, 6>(tmB, p, sms, stream);
     }
     return cudaErrorInvalidValue;
 }
