@@ -95,6 +95,10 @@ typedef struct {
     double  bytes_gather;    /* B bytes that must enter shared memory (no reuse assumed)      */
     double  flops_stored;    /* 2 * stored_values * N                                         */
     int64_t workspace_bytes; /* device scratch spmm_run needs at this N (WCSR partial tiles)  */
+    /* BCSR tile schedule currently held (spmm_bcsr_plan or the last spmm_run); 0 if none:   */
+    int64_t plan_n;          /* dense width it was built for                                  */
+    int32_t plan_token_tile; /* columns of B per tile: 128, 256 or 512                        */
+    int32_t plan_slab_tiles; /* token tiles per L2 slab                                       */
 } spmm_info_t;
 
 /* Arrays spmm_export can return, in their canonical (paper) layout. */
@@ -103,6 +107,8 @@ typedef enum {
     SPMM_X_BCSR_BLOCK_COL_IDX = 1,  /* int32 [n_blocks], ascending inside a block-row         */
     SPMM_X_BCSR_BLOCKS = 2,         /* dtype [n_blocks][b][b] row-major, zero filled          */
     SPMM_X_BCSR_ROW_ORDER = 3,      /* int32 [block-rows]: schedule order, longest first      */
+    SPMM_X_BCSR_TILE_PTR = 4,       /* int32 [n_ctas+1]: per-CTA ranges of TILES (needs a plan) */
+    SPMM_X_BCSR_TILES = 5,          /* int32 [n_tiles][2]: block-row, token tile; CTA-major    */
     SPMM_X_WCSR_WINDOW_ROW_PTR = 10,/* int32 [ceil(m/h)+1], in columns                        */
     SPMM_X_WCSR_WINDOW_COL_IDX = 11,/* int32 [P], -1 on padding                               */
     SPMM_X_WCSR_VALUES = 12,        /* dtype [h][P] row-major                                 */
@@ -146,6 +152,17 @@ int spmm_wcsr_create_csr(spmm_handle_t *out, int64_t m, int64_t k, const int64_t
 int spmm_wcsr_create_coo(spmm_handle_t *out, int64_t m, int64_t k, int64_t nnz,
                          const int32_t *rows, const int32_t *cols, const void *vals, int dtype,
                          int window_height, const spmm_opts_t *opts);
+
+/*
+ * BCSR only: build (and keep) the static tile schedule for dense width N -- the one
+ * spmm_run(h, ., ., N, .) uses -- so that it can be inspected with spmm_export / spmm_get_info.
+ * The schedule answers the load imbalance Sec. 3.5 and Sec. 4.2 (opt6) report for a persistent
+ * kernel with a fixed tile order: tiles (block-row x token tile) are dealt to the CTAs ahead
+ * of time, longest block-row first, each to the least loaded CTA.  Works on host_only handles.
+ * spmm_run builds the same schedule on its first call with a new N (that call allocates and
+ * may synchronise the device).
+ */
+int spmm_bcsr_plan(spmm_handle_t h, int64_t N);
 
 /*
  * C = A x B (Sec. 2.3; kernels of Sec. 3).  Asynchronous on `stream` (a cudaStream_t passed

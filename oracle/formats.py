@@ -212,3 +212,35 @@ def task_bins(plan, n_bins, fixed_cost=32):
     bin_ptr[1:] = np.cumsum([len(x) for x in members])
     tasks = [t for x in members for t in sorted(x)]
     return bin_ptr.astype(np.int32), np.asarray(tasks, dtype=np.int32)
+
+
+def bcsr_tile_schedule(block_row_ptr, n_tt, slab_w, n_ctas, fixed_cost=2):
+    """Static schedule of BCSR tiles (block-row, token tile) over n_ctas CTAs.
+
+    Addresses the imbalance Sec. 3.5 / Sec. 4.2 (opt6) report for a fixed tile
+    order.  Tiles are taken slab by slab (slab_w consecutive token tiles), inside a
+    slab in bcsr_row_order (most stored blocks first), inside a block-row by
+    ascending token tile; each goes to the CTA whose load is smallest at that
+    moment (ties: lowest CTA), load = sum of (stored blocks + fixed_cost); loads
+    carry over between slabs.  Returns (cta_ptr int32 [n_ctas+1],
+    tiles int32 [n_tiles, 2]) with every CTA's tiles in the order it received them.
+    """
+    import heapq
+    brp = np.asarray(block_row_ptr, dtype=np.int64)
+    lens = np.diff(brp)
+    order = bcsr_row_order(brp)
+    heap = [(0, c) for c in range(n_ctas)]
+    heapq.heapify(heap)
+    lists = [[] for _ in range(n_ctas)]
+    for t0 in range(0, n_tt, slab_w):
+        t1 = min(n_tt, t0 + slab_w)
+        for I in order.tolist():
+            cost = int(lens[I]) + fixed_cost
+            for t in range(t0, t1):
+                load, c = heapq.heappop(heap)
+                lists[c].append((I, t))
+                heapq.heappush(heap, (load + cost, c))
+    cta_ptr = np.zeros(n_ctas + 1, dtype=np.int64)
+    cta_ptr[1:] = np.cumsum([len(x) for x in lists])
+    tiles = np.asarray([p for x in lists for p in x], dtype=np.int32).reshape(-1, 2)
+    return cta_ptr.astype(np.int32), tiles

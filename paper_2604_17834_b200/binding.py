@@ -37,12 +37,13 @@ SPMM_ERR_HOST_ONLY = -8
 SPMM_ERR_TOO_LARGE = -9
 
 X_BCSR_BLOCK_ROW_PTR, X_BCSR_BLOCK_COL_IDX, X_BCSR_BLOCKS, X_BCSR_ROW_ORDER = 0, 1, 2, 3
+X_BCSR_TILE_PTR, X_BCSR_TILES = 4, 5
 X_WCSR_WINDOW_ROW_PTR, X_WCSR_WINDOW_COL_IDX, X_WCSR_VALUES, X_WCSR_TASKS = 10, 11, 12, 13
 X_WCSR_BIN_PTR, X_WCSR_BIN_TASKS = 14, 15
 
 EXPORTED_SYMBOLS = (
     "spmm_bcsr_create_csr", "spmm_bcsr_create_coo", "spmm_wcsr_create_csr", "spmm_wcsr_create_coo",
-    "spmm_run", "spmm_wcsr_run_static", "spmm_run_host", "spmm_check", "spmm_get_info", "spmm_export", "spmm_destroy",
+    "spmm_bcsr_plan", "spmm_run", "spmm_wcsr_run_static", "spmm_run_host", "spmm_check", "spmm_get_info", "spmm_export", "spmm_destroy",
     "spmm_status_string", "spmm_set_wait_limit_ns",
 )
 
@@ -67,6 +68,7 @@ class SpmmInfo(ctypes.Structure):
         ("bytes_b_touched", ctypes.c_double), ("bytes_c", ctypes.c_double),
         ("bytes_gather", ctypes.c_double), ("flops_stored", ctypes.c_double),
         ("workspace_bytes", ctypes.c_int64),
+        ("plan_n", ctypes.c_int64), ("plan_token_tile", ctypes.c_int32), ("plan_slab_tiles", ctypes.c_int32),
     ]
 
     def as_dict(self):
@@ -79,6 +81,7 @@ _lib.spmm_wcsr_create_csr.argtypes = _lib.spmm_bcsr_create_csr.argtypes
 _lib.spmm_bcsr_create_coo.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _vp, _vp, _vp, _i32, _i32, ctypes.POINTER(SpmmOpts)]
 _lib.spmm_wcsr_create_coo.argtypes = _lib.spmm_bcsr_create_coo.argtypes
 _lib.spmm_run.argtypes = [_vp, _vp, _vp, _i64, _vp]
+_lib.spmm_bcsr_plan.argtypes = [_vp, _i64]
 _lib.spmm_run_host.argtypes = [_vp, _vp, _vp, _i64, _vp]
 _lib.spmm_wcsr_run_static.argtypes = [_vp, _vp, _vp, _i64, _vp]
 _lib.spmm_check.argtypes = [_vp]
@@ -165,6 +168,13 @@ def spmm_bcsr_create_coo(m, k, rows, cols, vals, dtype, block, **opt):
 def spmm_wcsr_create_coo(m, k, rows, cols, vals, dtype, window_height=16, **opt):
     return _create_coo(_lib.spmm_wcsr_create_coo, "spmm_wcsr_create_coo", m, k, rows, cols, vals, dtype,
                        window_height, _opts(**opt))
+
+
+def spmm_bcsr_plan(h, N):
+    """BCSR: build and keep the tile schedule spmm_run would use for dense width N."""
+    rc = _lib.spmm_bcsr_plan(h, N)
+    if rc != SPMM_OK:
+        raise SpmmError(rc, "spmm_bcsr_plan")
 
 
 def spmm_run(h, B_dev_ptr, C_dev_ptr, N, stream=0):

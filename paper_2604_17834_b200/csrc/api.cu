@@ -85,6 +85,9 @@ struct spmm_handle_s {
     int32_t* d_idx = nullptr;        // block_col_idx / window_col_idx
     uint8_t* d_vals = nullptr;       // blocks / packed values
     int32_t* d_order = nullptr;      // BCSR row order
+    BcsrSchedule sched;              // BCSR tile schedule of the most recent dense width
+    int32_t* d_tiles = nullptr;
+    int32_t* d_cta_ptr = nullptr;
     WcsrDevTask* d_tasks = nullptr;
     int32_t* d_bin_ptr = nullptr;
     int32_t* d_bin_tasks = nullptr;
@@ -121,6 +124,8 @@ void free_handle(spmm_handle_s* h) {
         cudaFree(h->d_idx);
         cudaFree(h->d_vals);
         cudaFree(h->d_order);
+        cudaFree(h->d_tiles);
+        cudaFree(h->d_cta_ptr);
         cudaFree(h->d_tasks);
         cudaFree(h->d_bin_ptr);
         cudaFree(h->d_bin_tasks);
@@ -313,9 +318,10 @@ int ensure_tmB(spmm_handle_s* h, const void* B, int64_t N, int groups) {
     return SPMM_OK;
 }
 
-int run_bcsr(spmm_handle_s* h, const void* B, float* C, int64_t N, cudaStream_t stream) {
+// Tile width, slab width and the tile schedule for dense width N (cached for the last N).
+int ensure_schedule(spmm_handle_s* h, int64_t N) {
+    if (h->sched.N == N) return SPMM_OK;
     const BcsrHost& f = h->bcsr;
-    if (N < 64) return SPMM_ERR_UNSUPPORTED;   // the B box is 64 tokens wide
     // token tile: the largest of 512 / 256 / 128 columns that divides N (Sec. 4.3: pick a tile
     // width that divides the dense width so that no padded columns are computed); otherwise
     // the largest tile, whose ragged last tile is predicated.
@@ -324,39 +330,69 @@ int run_bcsr(spmm_handle_s* h, const void* B, float* C, int64_t N, cudaStream_t 
     for (int g = gmax; g >= 1; g >>= 1)
         if (N % (128 * g) == 0) { groups = g; break; }
     if (!groups) groups = N >= 128 * gmax ? gmax : (N > 128 ? 2 : 1);
-    // keep at least ~4 tiles per CTA when the matrix is small
-    while (groups > 1 && f.nbr * ((N + 128 * groups - 1) / (128 * groups)) < 4 * h->n_ctas) groups >>= 1;
+    // keep at least ~8 tiles per CTA so that the schedule has something to balance
+    while (groups > 1 && f.nbr * ((N + 128 * groups - 1) / (128 * groups)) < 8 * h->n_ctas) groups >>= 1;
     const int bnt = 128 * groups;
-    BcsrParams p;
-    p.block_row_ptr = h->d_ptr;
-    p.block_col_idx = h->d_idx;
-    p.row_order = h->d_order;
-    p.C = C;
-    p.m = h->m;
-    p.N = N;
-    p.nbr = static_cast<int32_t>(f.nbr);
-    p.n_tt = static_cast<int32_t>((N + bnt - 1) / bnt);
+    const int n_tt = static_cast<int>((N + bnt - 1) / bnt);
     // slab: token tiles whose B rows (k x slab columns) stay within ~48 MB of L2
     const int64_t slab_cols = (int64_t{48} << 20) / (h->k * h->es > 0 ? h->k * h->es : 1);
     int64_t sw = slab_cols / bnt;
     if (sw < 1) sw = 1;
-    if (sw > p.n_tt) sw = p.n_tt;
-    p.slab_w = static_cast<int32_t>(sw);
-    p.total_tiles = static_cast<int64_t>(p.nbr) * p.n_tt;
+    if (sw > n_tt) sw = n_tt;
+    BcsrSchedule sc;
+    int rc;
+    try {
+        rc = build_bcsr_schedule(f, n_tt, static_cast<int>(sw), h->n_ctas, &sc);
+    } catch (const std::bad_alloc&) {
+        rc = SPMM_ERR_ALLOC;
+    }
+    if (rc) return rc;
+    sc.groups = groups;
+    sc.N = N;
+    if (!h->host_only) {
+        if (h->d_tiles) {   // a previous schedule may still be in use by a running kernel
+            if (cudaDeviceSynchronize() != cudaSuccess) return SPMM_ERR_CUDA;
+            cudaFree(h->d_tiles);
+            cudaFree(h->d_cta_ptr);
+            h->d_tiles = h->d_cta_ptr = nullptr;
+        }
+        rc = upload(&h->d_tiles, sc.tiles.data(), sc.tiles.size() * 4);
+        if (!rc) rc = upload(&h->d_cta_ptr, sc.cta_ptr.data(), sc.cta_ptr.size() * 4);
+        if (rc) return rc;
+    }
+    h->sched = std::move(sc);
+    return SPMM_OK;
+}
+
+int run_bcsr(spmm_handle_s* h, const void* B, float* C, int64_t N, cudaStream_t stream) {
+    const BcsrHost& f = h->bcsr;
+    if (N < 64) return SPMM_ERR_UNSUPPORTED;   // the B box is 64 tokens wide
+    if (f.nbr == 0) return SPMM_OK;
+    int rc = ensure_schedule(h, N);
+    if (rc) return rc;
+    BcsrParams p;
+    p.block_row_ptr = h->d_ptr;
+    p.block_col_idx = h->d_idx;
+    p.tiles = reinterpret_cast<const int2*>(h->d_tiles);
+    p.cta_ptr = h->d_cta_ptr;
+    p.C = C;
+    p.m = h->m;
+    p.N = N;
     p.status = h->d_status;
     p.wait_limit_ns = g_wait_limit_ns.load();
-    if (p.total_tiles == 0) return SPMM_OK;
+    p.trace = nullptr;
+#ifdef SPMM_TRACE
+    p.trace = g_trace;
+#endif
     CUtensorMap tmA = h->tmA;
     if (!h->tmA_ok) {
         // no stored block at all: the kernel never touches A, any valid map will do
-        int rc = encode_2d_16bit(&tmA, h->dtype, h->d_vals, 8, 8, 8, 8, CU_TENSOR_MAP_SWIZZLE_NONE);
+        rc = encode_2d_16bit(&tmA, h->dtype, h->d_vals, 8, 8, 8, 8, CU_TENSOR_MAP_SWIZZLE_NONE);
         if (rc) return rc;
     }
-    int rc = ensure_tmB(h, B, N, groups);
+    rc = ensure_tmB(h, B, N, h->sched.groups);
     if (rc) return rc;
-    int grid = h->n_ctas;
-    if (grid > p.total_tiles) grid = static_cast<int>(p.total_tiles);
-    cudaError_t e = launch_bcsr(h->dtype, f.b, groups, tmA, h->tmB, p, grid, stream);
+    cudaError_t e = launch_bcsr(h->dtype, f.b, h->sched.groups, tmA, h->tmB, p, h->n_ctas, stream);
     return e == cudaSuccess ? SPMM_OK : SPMM_ERR_CUDA;
 }
 
@@ -499,6 +535,13 @@ int spmm_run(spmm_handle_t h, const void* B_dev, void* C_dev, int64_t N, void* s
     return run_wcsr(h, B_dev, static_cast<float*>(C_dev), N, st);
 }
 
+int spmm_bcsr_plan(spmm_handle_t h, int64_t N) {
+    if (!h || N <= 0) return SPMM_ERR_INVALID_ARG;
+    if (h->format != 0) return SPMM_ERR_INVALID_ARG;
+    if (N < 64 || (N * h->es) % 16 != 0) return SPMM_ERR_UNSUPPORTED;
+    return ensure_schedule(h, N);
+}
+
 int spmm_wcsr_run_static(spmm_handle_t h, const void* B_dev, void* C_dev, int64_t N, void* stream) {
     int rc = check_run_args(h, B_dev, C_dev, N);
     if (rc) return rc;
@@ -573,6 +616,11 @@ int spmm_get_info(spmm_handle_t h, int64_t N, spmm_info_t* info) {
         info->bytes_a = static_cast<double>(info->stored_values) * s;
         info->bytes_idx = static_cast<double>(f.nbr + 1 + f.nnzb) * 4.0;
         info->bytes_gather = static_cast<double>(f.nnzb) * f.b * n * s;
+        if (h->sched.N >= 0) {
+            info->plan_n = h->sched.N;
+            info->plan_token_tile = 128 * h->sched.groups;
+            info->plan_slab_tiles = h->sched.slab_w;
+        }
     } else {
         const WcsrHost& f = h->wcsr;
         info->block = f.wh;
@@ -612,6 +660,12 @@ int spmm_export(spmm_handle_t h, int which, void* host_dst, size_t cap, size_t* 
             case SPMM_X_BCSR_BLOCK_COL_IDX: bytes = f.block_col_idx.size() * 4; dev_src = h->d_idx; host_src = f.block_col_idx.data(); break;
             case SPMM_X_BCSR_BLOCKS: bytes = static_cast<size_t>(f.nnzb) * f.b * f.b * h->es; dev_src = h->d_vals; host_src = f.blocks.data(); break;
             case SPMM_X_BCSR_ROW_ORDER: bytes = f.row_order.size() * 4; dev_src = h->d_order; host_src = f.row_order.data(); break;
+            case SPMM_X_BCSR_TILE_PTR:
+                if (h->sched.N < 0) return SPMM_ERR_INVALID_ARG;
+                bytes = h->sched.cta_ptr.size() * 4; dev_src = h->d_cta_ptr; host_src = h->sched.cta_ptr.data(); break;
+            case SPMM_X_BCSR_TILES:
+                if (h->sched.N < 0) return SPMM_ERR_INVALID_ARG;
+                bytes = h->sched.tiles.size() * 4; dev_src = h->d_tiles; host_src = h->sched.tiles.data(); break;
             default: return SPMM_ERR_INVALID_ARG;
         }
     } else {

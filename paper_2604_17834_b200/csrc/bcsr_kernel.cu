@@ -15,8 +15,8 @@
 //               buffers; tcgen05.commit frees the ring slot / publishes the accumulator.
 //   warps 2-5   epilogue: tcgen05.ld -> registers -> global C (zeros for empty block-rows),
 //               overlapping the next tile's MMAs thanks to the second TMEM buffer.
-// Tiles are enumerated slab-major (a slab = a group of token tiles whose B rows fit in L2)
-// and, inside a slab, block-rows longest first; CTA c takes tiles c, c + grid, ...
+// The host deals tiles to CTAs ahead of time: slab by slab (a slab = token tiles whose B rows
+// fit in L2), longest block-row first, each tile to the least loaded CTA; CTA c walks its list.
 #include "kernels.h"
 #include "ptx.cuh"
 
@@ -39,20 +39,6 @@ struct BcsrCfg {
     static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
     static_assert(2 * kAccCols <= 512, "accumulators exceed TMEM");
 };
-
-struct TileCoord { int I; int t; };
-
-__device__ __forceinline__ TileCoord tile_coord(int64_t L, const BcsrParams& p) {
-    const int64_t per_slab = static_cast<int64_t>(p.nbr) * p.slab_w;
-    const int s = static_cast<int>(L / per_slab);
-    const int64_t u = L - s * per_slab;
-    const int t0 = s * p.slab_w;
-    const int w = min(p.slab_w, p.n_tt - t0);
-    TileCoord c;
-    c.I = p.row_order[static_cast<int>(u / w)];
-    c.t = t0 + static_cast<int>(u % w);
-    return c;
-}
 
 template <int B, int GROUPS, int STAGES, int FMT>
 __global__ void __launch_bounds__(192, 1)
@@ -93,23 +79,29 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t tmem_base = *tmem_slot;
 
     const int64_t N = p.N;
+    const int tile_begin = __ldg(p.cta_ptr + blockIdx.x), tile_end = __ldg(p.cta_ptr + blockIdx.x + 1);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int64_t L = blockIdx.x; L < p.total_tiles && ok; L += gridDim.x) {
-                const TileCoord tc = tile_coord(L, p);
-                const int n0 = tc.t * Cfg::kBnT;
+            TRACE_DECL(tr_empty);
+            TRACE_T0(tr_start);
+            for (int ti = tile_begin; ti < tile_end && ok; ++ti) {
+                const int2 tcd = __ldg(p.tiles + ti);
+                const int tI = tcd.x;
+                const int n0 = tcd.y * Cfg::kBnT;
                 const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
                 const int nbox = (nvalid + 63) >> 6;
                 const uint32_t tx = Cfg::kABytes + nbox * Cfg::kBoxBytes;
-                const int pb = p.block_row_ptr[tc.I], pe = p.block_row_ptr[tc.I + 1];
+                const int pb = p.block_row_ptr[tI], pe = p.block_row_ptr[tI + 1];
                 for (int q = pb; q < pe; ++q, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
+                    TRACE_T0(tr_a);
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, ctl, 1)) { ok = false; break; }
+                    TRACE_ADD(tr_empty, tr_a);
                     const uint32_t sb = smem_base + s * Cfg::kStageBytes;
                     mbar_arrive_expect_tx(full_bar(s), tx);
                     const int J = p.block_col_idx[q];
@@ -123,6 +115,9 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         tma_load_2d(sb + x * Cfg::kBoxBytes, &tmB, full_bar(s), n0 + x * 64, J * B);
                 }
             }
+            TRACE_PUT(0, clock64() - tr_start);
+            TRACE_PUT(1, tr_empty);
+            TRACE_PUT(3, (long long)it);
             if (!ok) {
                 // leave no bulk copy in flight: wait (bounded) for the fills already issued
                 const uint32_t first = it > STAGES ? it - STAGES : 0;
@@ -141,22 +136,32 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint64_t bdesc0 = make_smem_desc(0, 16, 8 * Cfg::kARowBytes, Cfg::kASwizzle);
             uint32_t it = 0, tile_i = 0;
             bool ok = true;
-            for (int64_t L = blockIdx.x; L < p.total_tiles && ok; L += gridDim.x, ++tile_i) {
-                const TileCoord tc = tile_coord(L, p);
-                const int n0 = tc.t * Cfg::kBnT;
+            TRACE_DECL(tr_full);
+            TRACE_DECL(tr_acce);
+            TRACE_DECL(tr_issue);
+            TRACE_T0(tr_start);
+            for (int ti = tile_begin; ti < tile_end && ok; ++ti, ++tile_i) {
+                const int2 tcd = __ldg(p.tiles + ti);
+                const int tI = tcd.x;
+                const int n0 = tcd.y * Cfg::kBnT;
                 const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
                 const int ngrp = (nvalid + 127) >> 7;
                 const int acc = tile_i & 1;
                 const uint32_t aph = (tile_i >> 1) & 1u;
+                TRACE_T0(tr_a);
                 if (!mbar_wait(acce_bar(acc), aph ^ 1u, ctl, 2)) { ok = false; break; }
+                TRACE_ADD(tr_acce, tr_a);
                 tc_fence_after_sync();
                 const uint32_t d0 = tmem_base + acc * Cfg::kAccCols;
-                const int pb = p.block_row_ptr[tc.I], pe = p.block_row_ptr[tc.I + 1];
+                const int pb = p.block_row_ptr[tI], pe = p.block_row_ptr[tI + 1];
                 for (int q = pb; q < pe; ++q, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
+                    TRACE_T0(tr_b);
                     if (!mbar_wait(full_bar(s), ph, ctl, 3)) { ok = false; break; }
+                    TRACE_ADD(tr_full, tr_b);
                     tc_fence_after_sync();
+                    TRACE_T0(tr_c);
                     const uint32_t sb = smem_base + s * Cfg::kStageBytes;
                     // descriptors differ only in their start-address field (bytes >> 4)
                     const uint64_t a0 = adesc0 + (sb >> 4);
@@ -172,28 +177,39 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                                b0 + (boff >> 4), idesc, accum);
                     }
                     tc_commit(empty_bar(s));
+                    TRACE_ADD(tr_issue, tr_c);
                 }
                 if (!ok) break;
                 if (pe > pb) tc_commit(accf_bar(acc));
                 else mbar_arrive(accf_bar(acc));
             }
+            TRACE_PUT(4, clock64() - tr_start);
+            TRACE_PUT(5, tr_full);
+            TRACE_PUT(6, tr_acce);
+            TRACE_PUT(7, (long long)it);
+            TRACE_PUT(12, tr_issue);
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
         const int qd = warp & 3;                    // TMEM lane quarter this warp may read
         uint32_t tile_i = 0;
         bool ok = true;
-        for (int64_t L = blockIdx.x; L < p.total_tiles && ok; L += gridDim.x, ++tile_i) {
-            const TileCoord tc = tile_coord(L, p);
-            const int n0 = tc.t * Cfg::kBnT;
+        TRACE_DECL(tr_accf);
+        TRACE_T0(tr_start);
+        for (int ti = tile_begin; ti < tile_end && ok; ++ti, ++tile_i) {
+            const int2 tcd = __ldg(p.tiles + ti);
+            const int tI = tcd.x;
+            const int n0 = tcd.y * Cfg::kBnT;
             const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
             const int ngrp = (nvalid + 127) >> 7;
             const int acc = tile_i & 1;
             const uint32_t aph = (tile_i >> 1) & 1u;
-            const bool has_blocks = p.block_row_ptr[tc.I + 1] > p.block_row_ptr[tc.I];
+            const bool has_blocks = p.block_row_ptr[tI + 1] > p.block_row_ptr[tI];
+            TRACE_T0(tr_a);
             if (!__all_sync(0xffffffffu, mbar_wait(accf_bar(acc), aph, ctl, 4))) { ok = false; break; }
+            TRACE_ADD(tr_accf, tr_a);
             tc_fence_after_sync();
-            const int64_t row0 = static_cast<int64_t>(tc.I) * B;
+            const int64_t row0 = static_cast<int64_t>(tI) * B;
             const int rows = static_cast<int>(min_i64(B, p.m - row0));
             for (int g = 0; g < ngrp; ++g) {
                 const int n = n0 + g * 128 + qd * 32 + lane;
@@ -231,6 +247,14 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(acce_bar(acc));
         }
+#ifdef SPMM_TRACE
+        if (warp == 2 && lane == 0) {
+            TRACE_PUT(8, clock64() - tr_start);
+            TRACE_PUT(9, tr_accf);
+            TRACE_PUT(10, (long long)tile_i);
+            TRACE_PUT(11, (long long)globaltimer_ns());
+        }
+#endif
     }
 
     tc_fence_before_sync();

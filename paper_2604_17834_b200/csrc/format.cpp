@@ -127,6 +127,49 @@ int build_bcsr(const CsrView& a, int b, BcsrHost* out) {
     return SPMM_OK;
 }
 
+int build_bcsr_schedule(const BcsrHost& f, int n_tt, int slab_w, int n_ctas, BcsrSchedule* out) {
+    if (n_tt <= 0 || slab_w <= 0 || n_ctas <= 0) return SPMM_ERR_INVALID_ARG;
+    out->n_tt = n_tt;
+    out->slab_w = slab_w;
+    out->n_ctas = n_ctas;
+    const int64_t ntiles = f.nbr * n_tt;
+    if (ntiles >= (int64_t{1} << 30)) return SPMM_ERR_TOO_LARGE;
+    using Load = std::pair<int64_t, int32_t>;   // (load, CTA): smallest load, then lowest CTA, on top
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+    for (int32_t c = 0; c < n_ctas; ++c) heap.push(Load(0, c));
+    std::vector<int32_t> owner(static_cast<size_t>(ntiles));
+    std::vector<int32_t> seq_I(static_cast<size_t>(ntiles)), seq_t(static_cast<size_t>(ntiles));
+    std::vector<int32_t> count(static_cast<size_t>(n_ctas), 0);
+    int64_t n = 0;
+    for (int t0 = 0; t0 < n_tt; t0 += slab_w) {
+        const int t1 = std::min(n_tt, t0 + slab_w);
+        for (int64_t r = 0; r < f.nbr; ++r) {
+            const int32_t I = f.row_order[r];
+            const int64_t cost = (f.block_row_ptr[I + 1] - f.block_row_ptr[I]) + kTileFixedCost;
+            for (int t = t0; t < t1; ++t, ++n) {
+                Load top = heap.top();
+                heap.pop();
+                owner[n] = top.second;
+                seq_I[n] = I;
+                seq_t[n] = t;
+                count[top.second]++;
+                top.first += cost;
+                heap.push(top);
+            }
+        }
+    }
+    out->cta_ptr.assign(static_cast<size_t>(n_ctas) + 1, 0);
+    for (int c = 0; c < n_ctas; ++c) out->cta_ptr[c + 1] = out->cta_ptr[c] + count[c];
+    out->tiles.assign(static_cast<size_t>(2 * ntiles), 0);
+    std::vector<int32_t> pos(out->cta_ptr.begin(), out->cta_ptr.end() - 1);
+    for (int64_t i = 0; i < ntiles; ++i) {
+        const int32_t dst = pos[owner[i]]++;
+        out->tiles[2 * dst] = seq_I[i];
+        out->tiles[2 * dst + 1] = seq_t[i];
+    }
+    return SPMM_OK;
+}
+
 // ----------------------------------------------------------------------------- WCSR
 
 int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost* out) {

@@ -32,6 +32,19 @@ struct BcsrHost {
     std::vector<int32_t> row_order;       // [nbr] block-rows, most stored blocks first (stable)
 };
 
+// Static tile schedule of the BCSR kernel for one dense width: a tile is (block-row, token
+// tile).  Tiles are taken slab by slab (a slab = slab_w consecutive token tiles, sized so the
+// B rows it touches stay in L2) and, inside a slab, block-rows with the most stored blocks
+// first; each tile goes to the CTA whose load is smallest at that moment (ties: lowest CTA),
+// load = sum of (stored blocks + kTileFixedCost).  Loads carry over from slab to slab.
+struct BcsrSchedule {
+    int64_t N = -1;
+    int groups = 0, n_tt = 0, slab_w = 0, n_ctas = 0;
+    std::vector<int32_t> cta_ptr;    // [n_ctas+1]
+    std::vector<int32_t> tiles;      // 2 * n_tiles: {block-row, token tile}, CTA-major
+};
+constexpr int kTileFixedCost = 2;
+
 struct WcsrTask { int32_t window, q0, count, slot; };
 
 struct WcsrHost {
@@ -69,6 +82,7 @@ int validate_csr(const CsrView& a);
 int coo_to_csr(int64_t m, int64_t k, int64_t nnz, const int32_t* rows, const int32_t* cols,
                const uint8_t* vals, int es, CsrOwned* out);
 int build_bcsr(const CsrView& a, int b, BcsrHost* out);
+int build_bcsr_schedule(const BcsrHost& f, int n_tt, int slab_w, int n_ctas, BcsrSchedule* out);
 // T = 0 picks the sub-task size from the matrix: about a quarter of one bin's share of the
 // padded columns, rounded down to a multiple of 64 and clamped to [128, 4096].
 int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost* out);

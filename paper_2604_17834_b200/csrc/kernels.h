@@ -10,15 +10,13 @@ namespace spmm {
 struct BcsrParams {
     const int32_t* block_row_ptr;
     const int32_t* block_col_idx;
-    const int32_t* row_order;
+    const int2* tiles;        // {block-row, token tile}, CTA-major
+    const int32_t* cta_ptr;   // [grid+1] ranges of tiles
     float* C;
     int64_t m, N;
-    int32_t nbr;        // block-rows
-    int32_t n_tt;       // token tiles = ceil(N / (128 * groups))
-    int32_t slab_w;     // token tiles per L2 slab
-    int64_t total_tiles;
     int* status;
     uint64_t wait_limit_ns;
+    long long* trace;   // tuning builds only (SPMM_TRACE); nullptr otherwise
 };
 
 // dtype: 0 bf16, 1 fp16.  groups: token tile = 128 * groups columns of B (1, 2 or 4).

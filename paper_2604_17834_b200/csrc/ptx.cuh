@@ -10,6 +10,20 @@
 
 namespace spmm {
 
+// Optional per-CTA cycle accounting for kernel tuning (compiled out unless SPMM_TRACE is
+// defined; the buffer is the params' trace pointer, 16 counters per CTA).
+#ifdef SPMM_TRACE
+#define TRACE_DECL(name) long long name = 0
+#define TRACE_T0(t) const long long t = clock64()
+#define TRACE_ADD(acc, t) acc += clock64() - t
+#define TRACE_PUT(slot, val) do { if (p.trace) p.trace[blockIdx.x * 16 + (slot)] = (val); } while (0)
+#else
+#define TRACE_DECL(name)
+#define TRACE_T0(t)
+#define TRACE_ADD(acc, t)
+#define TRACE_PUT(slot, val)
+#endif
+
 // ----------------------------------------------------------------------------- misc
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

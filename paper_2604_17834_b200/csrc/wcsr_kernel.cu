@@ -30,20 +30,6 @@ namespace spmm {
 
 namespace {
 
-// Optional per-CTA cycle accounting for kernel tuning (compiled out unless SPMM_TRACE is
-// defined; the buffer is WcsrParams::trace, 16 counters per CTA).
-#ifdef SPMM_TRACE
-#define TRACE_DECL(name) long long name = 0
-#define TRACE_T0(t) const long long t = clock64()
-#define TRACE_ADD(acc, t) acc += clock64() - t
-#define TRACE_PUT(slot, val) do { if (p.trace) p.trace[blockIdx.x * 16 + (slot)] = (val); } while (0)
-#else
-#define TRACE_DECL(name)
-#define TRACE_T0(t)
-#define TRACE_ADD(acc, t)
-#define TRACE_PUT(slot, val)
-#endif
-
 constexpr int kWH = 16;
 constexpr int kProducerWarps = 4;
 // A 128 x 16 x K MMA is tiny, and MMAs that accumulate into the same TMEM tile serialise on

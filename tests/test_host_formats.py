@@ -91,6 +91,38 @@ def test_bcsr_workload_generators_round_trip(lib):
     lib.spmm_destroy(h)
 
 
+@pytest.mark.parametrize("b,N,n_ctas", [(64, 4096, 148), (16, 1024, 7), (128, 640, 5), (32, 200, 3)])
+def test_bcsr_tile_schedule_is_bit_exact_and_balanced(lib, b, N, n_ctas):
+    s = wl.bcsr_sweep(55 + b, m=4096, k=2048, b=b, density=0.1)
+    h = lib.spmm_bcsr_create_csr(4096, 2048, s["row_ptr"], s["col_idx"], s["vals"], "fp16", b, host_only=True,
+                                 n_ctas=n_ctas)
+    try:
+        with pytest.raises(lib.SpmmError):
+            lib.spmm_export(h, lib.X_BCSR_TILES, np.int32)          # no plan yet
+        lib.spmm_bcsr_plan(h, N)
+        info = lib.spmm_get_info(h, N)
+        assert info["plan_n"] == N and info["plan_token_tile"] in (128, 256, 512)
+        bnt = info["plan_token_tile"]
+        n_tt = -(-N // bnt)
+        f = F.bcsr_from_csr(4096, 2048, s["row_ptr"], s["col_idx"], s["vals"], b)
+        want_ptr, want_tiles = F.bcsr_tile_schedule(f["block_row_ptr"], n_tt, info["plan_slab_tiles"], n_ctas)
+        got_ptr = lib.spmm_export(h, lib.X_BCSR_TILE_PTR, np.int32)
+        got_tiles = lib.spmm_export(h, lib.X_BCSR_TILES, np.int32).reshape(-1, 2)
+        assert np.array_equal(got_ptr, want_ptr) and np.array_equal(got_tiles, want_tiles)
+        # every (block-row, token tile) exactly once
+        nbr = f["block_row_ptr"].shape[0] - 1
+        keys = got_tiles[:, 0].astype(np.int64) * n_tt + got_tiles[:, 1]
+        assert np.array_equal(np.sort(keys), np.arange(nbr * n_tt))
+        # greedy longest-first bound: no CTA exceeds the lightest by more than the heaviest tile
+        cost = np.diff(f["block_row_ptr"])[got_tiles[:, 0]].astype(np.int64) + 2
+        loads = np.array([cost[got_ptr[c]:got_ptr[c + 1]].sum() for c in range(n_ctas)])
+        assert loads.max() - loads.min() <= cost.max()
+        if N % 512 == 0 and b != 128 and nbr * (N // 512) >= 8 * n_ctas:
+            assert bnt == 512                                        # widest tile that divides N
+    finally:
+        lib.spmm_destroy(h)
+
+
 WCSR_CASES = [("tf32", 1000, 900, 0.01, 64), ("fp16", 333, 517, 0.05, 32), ("bf16", 160, 4000, 0.2, 128),
               ("fp16", 16, 40, 0.5, 16)]
 
