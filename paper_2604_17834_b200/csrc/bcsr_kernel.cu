@@ -83,7 +83,11 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        // A warp serialises the TMA requests of its lanes (~60 cycles each) but needs far
+        // longer for requests issued one after the other by a single thread, so the loads of
+        // a stage are spread over the lanes: lane x < nbox fetches B box x, lanes 8 / 9 the
+        // A block (two halves when b = 128).  Lane 0 posts the stage's byte count first.
+        {
             uint32_t it = 0;
             bool ok = true;
             TRACE_DECL(tr_empty);
@@ -95,30 +99,38 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
                 const int nbox = (nvalid + 63) >> 6;
                 const uint32_t tx = Cfg::kABytes + nbox * Cfg::kBoxBytes;
-                const int pb = p.block_row_ptr[tI], pe = p.block_row_ptr[tI + 1];
-                for (int q = pb; q < pe; ++q, ++it) {
-                    const int s = it % STAGES;
-                    const uint32_t ph = (it / STAGES) & 1u;
-                    TRACE_T0(tr_a);
-                    if (!mbar_wait(empty_bar(s), ph ^ 1u, ctl, 1)) { ok = false; break; }
-                    TRACE_ADD(tr_empty, tr_a);
-                    const uint32_t sb = smem_base + s * Cfg::kStageBytes;
-                    mbar_arrive_expect_tx(full_bar(s), tx);
-                    const int J = p.block_col_idx[q];
-                    if constexpr (B <= 64) {
-                        tma_load_2d(sb + Cfg::kDenseBytes, &tmA, full_bar(s), 0, q * B);
-                    } else {
-                        tma_load_2d(sb + Cfg::kDenseBytes, &tmA, full_bar(s), 0, q * B);
-                        tma_load_2d(sb + Cfg::kDenseBytes + B * 128, &tmA, full_bar(s), 64, q * B);
+                const int pb = __ldg(p.block_row_ptr + tI), pe = __ldg(p.block_row_ptr + tI + 1);
+                for (int q0 = pb; q0 < pe && ok; q0 += 32) {
+                    // block columns of up to 32 stored blocks with one coalesced load
+                    const int Jl = (q0 + lane < pe) ? __ldg(p.block_col_idx + q0 + lane) : 0;
+                    const int nq = min(32, pe - q0);
+                    for (int jq = 0; jq < nq; ++jq, ++it) {
+                        const int q = q0 + jq;
+                        const int J = __shfl_sync(0xffffffffu, Jl, jq);
+                        const int s = it % STAGES;
+                        const uint32_t ph = (it / STAGES) & 1u;
+                        TRACE_T0(tr_a);
+                        if (!__all_sync(0xffffffffu, mbar_wait(empty_bar(s), ph ^ 1u, ctl, 1))) { ok = false; break; }
+                        TRACE_ADD(tr_empty, tr_a);
+                        const uint32_t sb = smem_base + s * Cfg::kStageBytes;
+                        if (lane == 0) mbar_arrive_expect_tx(full_bar(s), tx);
+                        __syncwarp();
+                        if (lane < nbox) {
+                            tma_load_2d(sb + lane * Cfg::kBoxBytes, &tmB, full_bar(s), n0 + lane * 64, J * B);
+                        } else if (lane == 8) {
+                            tma_load_2d(sb + Cfg::kDenseBytes, &tmA, full_bar(s), 0, q * B);
+                        } else if (B > 64 && lane == 9) {
+                            tma_load_2d(sb + Cfg::kDenseBytes + B * 128, &tmA, full_bar(s), 64, q * B);
+                        }
                     }
-                    for (int x = 0; x < nbox; ++x)
-                        tma_load_2d(sb + x * Cfg::kBoxBytes, &tmB, full_bar(s), n0 + x * 64, J * B);
                 }
             }
-            TRACE_PUT(0, clock64() - tr_start);
-            TRACE_PUT(1, tr_empty);
-            TRACE_PUT(3, (long long)it);
-            if (!ok) {
+            if (lane == 0) {
+                TRACE_PUT(0, clock64() - tr_start);
+                TRACE_PUT(1, tr_empty);
+                TRACE_PUT(3, (long long)it);
+            }
+            if (!ok && lane == 0) {
                 // leave no bulk copy in flight: wait (bounded) for the fills already issued
                 const uint32_t first = it > STAGES ? it - STAGES : 0;
                 for (uint32_t j = first; j < it; ++j) {
@@ -130,10 +142,13 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // Warp-uniform control flow (all lanes wait and compute the uniform descriptors); one
+        // elected lane issues the tcgen05 instructions.
+        {
             constexpr uint32_t idesc = make_idesc(FMT, 128, B, 1, 0);
             const uint64_t adesc0 = make_smem_desc(0, Cfg::kBoxBytes, 1024, SWZ_128B);
             const uint64_t bdesc0 = make_smem_desc(0, 16, 8 * Cfg::kARowBytes, Cfg::kASwizzle);
+            const bool leader = elect_one();
             uint32_t it = 0, tile_i = 0;
             bool ok = true;
             TRACE_DECL(tr_full);
@@ -149,16 +164,16 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int acc = tile_i & 1;
                 const uint32_t aph = (tile_i >> 1) & 1u;
                 TRACE_T0(tr_a);
-                if (!mbar_wait(acce_bar(acc), aph ^ 1u, ctl, 2)) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(acce_bar(acc), aph ^ 1u, ctl, 2))) { ok = false; break; }
                 TRACE_ADD(tr_acce, tr_a);
                 tc_fence_after_sync();
                 const uint32_t d0 = tmem_base + acc * Cfg::kAccCols;
-                const int pb = p.block_row_ptr[tI], pe = p.block_row_ptr[tI + 1];
+                const int pb = __ldg(p.block_row_ptr + tI), pe = __ldg(p.block_row_ptr + tI + 1);
                 for (int q = pb; q < pe; ++q, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
                     TRACE_T0(tr_b);
-                    if (!mbar_wait(full_bar(s), ph, ctl, 3)) { ok = false; break; }
+                    if (!__all_sync(0xffffffffu, mbar_wait(full_bar(s), ph, ctl, 3))) { ok = false; break; }
                     TRACE_ADD(tr_full, tr_b);
                     tc_fence_after_sync();
                     TRACE_T0(tr_c);
@@ -166,28 +181,32 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     // descriptors differ only in their start-address field (bytes >> 4)
                     const uint64_t a0 = adesc0 + (sb >> 4);
                     const uint64_t b0 = bdesc0 + ((sb + Cfg::kDenseBytes) >> 4);
+                    const uint32_t accum0 = q > pb ? 1u : 0u;
 #pragma unroll
                     for (int ks = 0; ks < B / 16; ++ks) {
                         const uint32_t boff = B <= 64 ? ks * 32 : (ks >> 2) * (B * 128) + (ks & 3) * 32;
-                        const uint32_t accum = (q > pb || ks > 0) ? 1u : 0u;
 #pragma unroll
                         for (int g = 0; g < GROUPS; ++g)
-                            if (g < ngrp)
+                            if (leader && g < ngrp)
                                 umma_ss<false>(d0 + g * B, a0 + ((g * 2 * Cfg::kBoxBytes + ks * 2048) >> 4),
-                                               b0 + (boff >> 4), idesc, accum);
+                                               b0 + (boff >> 4), idesc, ks > 0 ? 1u : accum0);
                     }
-                    tc_commit(empty_bar(s));
+                    if (leader) tc_commit(empty_bar(s));
                     TRACE_ADD(tr_issue, tr_c);
                 }
                 if (!ok) break;
-                if (pe > pb) tc_commit(accf_bar(acc));
-                else mbar_arrive(accf_bar(acc));
+                if (leader) {
+                    if (pe > pb) tc_commit(accf_bar(acc));
+                    else mbar_arrive(accf_bar(acc));
+                }
             }
-            TRACE_PUT(4, clock64() - tr_start);
-            TRACE_PUT(5, tr_full);
-            TRACE_PUT(6, tr_acce);
-            TRACE_PUT(7, (long long)it);
-            TRACE_PUT(12, tr_issue);
+            if (lane == 0) {
+                TRACE_PUT(4, clock64() - tr_start);
+                TRACE_PUT(5, tr_full);
+                TRACE_PUT(6, tr_acce);
+                TRACE_PUT(7, (long long)it);
+                TRACE_PUT(12, tr_issue);
+            }
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps

@@ -39,7 +39,6 @@ constexpr int kNSub = 4;
 
 template <int ES, int GROUPS, int KT, int STAGES>
 struct WcsrCfg {
-    static constexpr int kE16 = 16 / ES;                    // elements per 16-byte chunk
     static constexpr int kKStep = 32 / ES;                  // columns per MMA (= b_col)
     static constexpr int kBnT = 128 * GROUPS;
     static constexpr int kRowBytes = kBnT * ES;
@@ -234,6 +233,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
         constexpr uint32_t idesc = make_idesc(FMT, 128, kWH, 1, 0);
         const uint64_t adesc0 = make_smem_desc(0, Cfg::kAtomStride, ES == 2 ? 1024 : 512, ES == 2 ? SWZ_128B : SWZ_128B_BASE32B);
         const uint64_t bdesc0 = make_smem_desc(0, kWH * 16, 128, SWZ_NONE);
+        const bool leader = elect_one();
         TRACE_DECL(tr_full);
         TRACE_DECL(tr_acce);
         TRACE_DECL(tr_issue);
@@ -279,21 +279,21 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                         TRACE_T0(tr_c);
                         const uint32_t sb = smem_base + s * Cfg::kStageBytes;
                         const int nks = cnt / Cfg::kKStep;
-                        if (elect_one()) {
-                            // descriptors differ only in their start-address field (bytes >> 4)
-                            const uint64_t a0 = adesc0 + (sb >> 4);
-                            const uint64_t b0 = bdesc0 + ((sb + Cfg::kDenseBytes) >> 4);
-                            uint32_t kk = kstep_item;
-                            for (int ks = 0; ks < nks; ++ks, ++kk) {
-                                const uint32_t dsub = d0 + (kk & (kNSub - 1)) * kWH;
-                                const uint32_t accum = kk >= kNSub ? 1u : 0u;    // first use overwrites
+                        // descriptors differ only in their start-address field (bytes >> 4)
+                        const uint64_t a0 = adesc0 + (sb >> 4);
+                        const uint64_t b0 = bdesc0 + ((sb + Cfg::kDenseBytes) >> 4);
+                        uint32_t kk = kstep_item;
+                        for (int ks = 0; ks < nks; ++ks, ++kk) {
+                            const uint32_t dsub = d0 + (kk & (kNSub - 1)) * kWH;
+                            const uint32_t accum = kk >= kNSub ? 1u : 0u;    // first use overwrites
 #pragma unroll
-                                for (int g = 0; g < GROUPS; ++g)
-                                    if (g < ngrp)
-                                        umma_ss<FMT == 2>(dsub + g * kNSub * kWH,
-                                                          a0 + ((g * Cfg::kAtomsPerGroup * Cfg::kAtomStride + ks * (Cfg::kKStep / 8) * 1024) >> 4),
-                                                          b0 + ((ks * (kWH * 32)) >> 4), idesc, accum);
-                            }
+                            for (int g = 0; g < GROUPS; ++g)
+                                if (leader && g < ngrp)
+                                    umma_ss<FMT == 2>(dsub + g * kNSub * kWH,
+                                                      a0 + ((g * Cfg::kAtomsPerGroup * Cfg::kAtomStride + ks * (Cfg::kKStep / 8) * 1024) >> 4),
+                                                      b0 + ((ks * (kWH * 32)) >> 4), idesc, accum);
+                        }
+                        if (leader) {
                             tc_commit(empty_bar(s));
                             if (last) tc_commit(accf_bar(acc));
                         }
