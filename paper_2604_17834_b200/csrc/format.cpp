@@ -7,6 +7,7 @@
 #include <queue>
 #include <utility>
 
+#include "kernels.h"
 #include "spmm_b200.h"
 
 namespace spmm {
@@ -292,7 +293,7 @@ int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost*
 
     // pipeline schedule: one fill per stage-sized run of columns (16 KB of gathered B rows at
     // 128 tokens: 64 columns of a 2-byte type, 32 of a 4-byte type), bin-major
-    out->kt = 128 / a.es;
+    out->kt = wcsr_stage_cols(a.es);
     out->fills.clear();
     out->bin_fill.assign(static_cast<size_t>(n_bins) + 1, 0);
     for (int j = 0; j < n_bins; ++j) {

@@ -24,6 +24,28 @@ cudaError_t launch_bcsr(int dtype, int b, int groups, const CUtensorMap& tmA, co
                         const BcsrParams& p, int grid, cudaStream_t stream);
 int bcsr_token_groups_max(int b);
 
+// WCSR pipeline shape, shared by the host schedule (fills are cut to the stage size) and the
+// kernel: columns per shared-memory stage, ring depth and producer warps for the one-group
+// (N <= 128, two CTAs per SM) and two-group (N > 128, one CTA per SM) variants.
+#ifndef WCSR_STAGE_ROW_BYTES
+#define WCSR_STAGE_ROW_BYTES 128
+#endif
+#ifndef WCSR_STAGES1
+#define WCSR_STAGES1 6
+#endif
+#ifndef WCSR_STAGES2
+#define WCSR_STAGES2 6
+#endif
+#ifndef WCSR_PW1
+#define WCSR_PW1 6
+#endif
+#ifndef WCSR_PW2
+#define WCSR_PW2 6
+#endif
+constexpr int wcsr_stage_cols(int es) { return WCSR_STAGE_ROW_BYTES / es; }
+constexpr int kWcsrStages1 = WCSR_STAGES1, kWcsrStages2 = WCSR_STAGES2;
+constexpr int kWcsrProducerWarps1 = WCSR_PW1, kWcsrProducerWarps2 = WCSR_PW2;
+
 // Device task descriptor of the WCSR kernel (one per sub-task of the split plan).
 struct WcsrDevTask {
     int32_t col_begin;   // absolute position of the task's first padded column

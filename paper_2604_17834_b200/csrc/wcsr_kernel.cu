@@ -7,7 +7,7 @@
 // shared memory in the MN-major 128-byte-swizzled layout tcgen05.mma reads) and the 16
 // window rows as the MMA N side (operand = the packed window tile, K-major, un-swizzled).
 //
-// Roles (288 threads, persistent CTAs):
+// Roles ((PW + 5) warps, persistent CTAs; PW producer warps):
 //   warps 0-3   gather producers: warp w owns the CTA's fills w, w + 4, ...; per fill every
 //               lane reads four column indices and issues one TMA row-gather (four B rows x
 //               128 bytes, hardware swizzle, zero fill for -1 pads) into a STAGES-deep ring;
@@ -31,7 +31,6 @@ namespace spmm {
 namespace {
 
 constexpr int kWH = 16;
-constexpr int kProducerWarps = 4;
 // A 128 x 16 x K MMA is tiny, and MMAs that accumulate into the same TMEM tile serialise on
 // it, so the K steps of an item rotate over kNSub independent partial accumulators that the
 // epilogue adds (in index order).
@@ -54,8 +53,8 @@ struct WcsrCfg {
     static constexpr int kAccCols = GROUPS * kNSub * kWH;   // TMEM columns of one item
     static constexpr int kTmemCols = kNAcc * kAccCols;      // 256
     static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 + 256;
-    static_assert(KT % 8 == 0 && KT % kKStep == 0 && KT <= 64, "stage shape");
-    static_assert(kGathers % 32 == 0, "gather instructions are dealt to whole warps");
+    static_assert(KT % 8 == 0 && KT % kKStep == 0 && KT <= 128, "stage shape");
+    static_assert(kGathers % 32 == 0 || kGathers == 16, "gather instructions are dealt to warps");
     static_assert(kStageBytes % 1024 == 0, "stage alignment");
 };
 
@@ -77,13 +76,20 @@ struct SegIter {
     }
 };
 
-template <int ES, int FMT, int GROUPS, int KT, int STAGES>
-__global__ void __launch_bounds__(288, (WcsrCfg<ES, GROUPS, KT, STAGES>::kSmemBytes + 1024) * 2 <= 227 * 1024 ? 2 : 1)
+template <int ES, int FMT, int GROUPS, int KT, int STAGES, int PW>
+__global__ void __launch_bounds__((PW + 5) * 32, (WcsrCfg<ES, GROUPS, KT, STAGES>::kSmemBytes + 1024) * 2 <= 227 * 1024 ? 2 : 1)
 wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
     using Cfg = WcsrCfg<ES, GROUPS, KT, STAGES>;
+    constexpr int kProducerWarps = PW;          // warps 0 .. PW-1; MMA warp PW; epilogue PW+1 .. PW+4
+    constexpr int kMmaWarp = PW;
+    // Fill i goes to stage i % STAGES and is produced by warp i % PW.  With STAGES a multiple
+    // of PW every stage is always refilled by the same warp, which therefore sees each of its
+    // releases in turn: the parity wait on the empty barrier is exact.
+    static_assert(STAGES % PW == 0, "every stage must belong to one producer warp");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
+    static_assert((2 * STAGES + 2 * Cfg::kNAcc + 2) * 8 <= 256, "barrier area is 256 bytes");
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * Cfg::kStageBytes);
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -103,7 +109,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
         fence_mbar_init();
         prefetch_tmap(&tmB);
     }
-    if (warp == 4) {
+    if (warp == kMmaWarp) {
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);
         tmem_relinquish();
     }
@@ -151,7 +157,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
             for (int wbase = f0; wbase < f1 && ok; wbase += 32) {
                 const int2 nwin = (wbase + 32 + lane < f1) ? __ldg(p.fills + wbase + 32 + lane) : kNoDesc;
                 const uint32_t itw = it0 + static_cast<uint32_t>(wbase - f0);   // counter of window slot 0
-                int j = static_cast<int>((static_cast<uint32_t>(warp) - itw) & 3u);
+                int j = static_cast<int>((static_cast<uint32_t>(warp) + kProducerWarps - itw % kProducerWarps) % kProducerWarps);
                 for (; j < 32 && wbase + j < f1; j += kProducerWarps) {
                     const uint32_t it = itw + j;
                     int2 d;
@@ -226,7 +232,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
             while (!mbar_try_wait(full_bar(last_it % STAGES), (last_it / STAGES) & 1u) &&
                    globaltimer_ns() - t0 < 2000000ull) {}
         }
-    } else if (warp == 4) {
+    } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issuer
         // The whole warp walks the fill list (descriptor windows via shuffles) and waits for
         // stages and accumulators; one elected lane issues the MMAs and commits.
@@ -388,7 +394,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
             }
         }
 #ifdef SPMM_TRACE
-        if (warp == 5 && lane == 0) {
+        if (warp == kMmaWarp + 1 && lane == 0) {
             TRACE_PUT(8, clock64() - tr_start);
             TRACE_PUT(9, tr_accf);
             TRACE_PUT(10, (long long)item);
@@ -399,7 +405,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
 
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == kMmaWarp) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, Cfg::kTmemCols);
     }
@@ -430,10 +436,10 @@ wcsr_merge_kernel(const MergeParams p) {
     }
 }
 
-template <int ES, int FMT, int GROUPS, int KT, int STAGES>
+template <int ES, int FMT, int GROUPS, int KT, int STAGES, int PW>
 cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
     using Cfg = WcsrCfg<ES, GROUPS, KT, STAGES>;
-    auto kfn = wcsr_spmm_kernel<ES, FMT, GROUPS, KT, STAGES>;
+    auto kfn = wcsr_spmm_kernel<ES, FMT, GROUPS, KT, STAGES, PW>;
     static int occ = 0;
     if (occ == 0) {
         cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
@@ -441,7 +447,7 @@ cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cud
         e = cudaFuncSetAttribute(kfn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         // resident CTAs per SM: 227 KB of shared memory (1 KB reserved per CTA), 512 TMEM
-        // columns, and the register file (__launch_bounds__ keeps two CTAs of 288 threads)
+        // columns, and the register file (__launch_bounds__ keeps two CTAs resident)
         int o = (227 * 1024) / (Cfg::kSmemBytes + 1024);
         o = o < 512 / Cfg::kTmemCols ? o : 512 / Cfg::kTmemCols;
         occ = o < 1 ? 1 : (o > 2 ? 2 : o);
@@ -449,22 +455,24 @@ cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cud
     int grid = sms * occ;
     if (grid > p.n_bins) grid = p.n_bins;
     if (grid < 1) return cudaSuccess;
-    kfn<<<grid, 288, Cfg::kSmemBytes, stream>>>(tmB, p);
+    kfn<<<grid, (PW + 5) * 32, Cfg::kSmemBytes, stream>>>(tmB, p);
     return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_wcsr(int dtype, int groups, const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
+    constexpr int K2 = wcsr_stage_cols(2), K4 = wcsr_stage_cols(4);
+    constexpr int S1 = kWcsrStages1, S2 = kWcsrStages2, P1 = kWcsrProducerWarps1, P2 = kWcsrProducerWarps2;
     if (dtype == 2) {
-        if (groups == 1) return launch_one<4, 2, 1, 32, 6>(tmB, p, sms, stream);
-        if (groups == 2) return launch_one<4, 2, 2, 32, 6>(tmB, p, sms, stream);
+        if (groups == 1) return launch_one<4, 2, 1, K4, S1, P1>(tmB, p, sms, stream);
+        if (groups == 2) return launch_one<4, 2, 2, K4, S2, P2>(tmB, p, sms, stream);
     } else if (dtype == 1) {
-        if (groups == 1) return launch_one<2, 0, 1, 64, 6>(tmB, p, sms, stream);
-        if (groups == 2) return launch_one<2, 0, 2, 64, 6>(tmB, p, sms, stream);
+        if (groups == 1) return launch_one<2, 0, 1, K2, S1, P1>(tmB, p, sms, stream);
+        if (groups == 2) return launch_one<2, 0, 2, K2, S2, P2>(tmB, p, sms, stream);
     } else if (dtype == 0) {
-        if (groups == 1) return launch_one<2, 1, 1, 64, 6>(tmB, p, sms, stream);
-        if (groups == 2) return launch_one<2, 1, 2, 64, 6>(tmB, p, sms, stream);
+        if (groups == 1) return launch_one<2, 1, 1, K2, S1, P1>(tmB, p, sms, stream);
+        if (groups == 2) return launch_one<2, 1, 2, K2, S2, P2>(tmB, p, sms, stream);
     }
     return cudaErrorInvalidValue;
 }
