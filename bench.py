@@ -2,7 +2,7 @@
 """Benchmark of the B200 SpMM hot path (BCSR and WCSR kernels behind the C ABI).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
-                    [--only NAME] [--skip-others] [--with-graph]
+                    [--only NAME [--dense-width N]] [--skip-others] [--others A,B] [--no-cpu]
 
 A step is one ``spmm_run`` (the SpMM kernel, plus the merge kernel for WCSR) on
 inputs already resident in HBM.  The headline workload is configs[1] (WCSR,
@@ -64,7 +64,9 @@ def workload_table():
 
     def cfg5(N):
         def f():
-            return dict(kind="wcsr", a=wl.rmat(), dtype="fp16", size=16, N=N, Bdist=("normal", 0.0, 1.0))
+            if "rmat" not in _CACHE:                 # ~30 s to draw: shared by the three widths
+                _CACHE["rmat"] = wl.rmat()
+            return dict(kind="wcsr", a=_CACHE["rmat"], dtype="fp16", size=16, N=N, Bdist=("normal", 0.0, 1.0))
         return f
 
     t = {
@@ -86,9 +88,18 @@ def workload_table():
     return t
 
 
+_CACHE = {}
 HEADLINE = "cfg2_wcsr_irregular"
-DEFAULT_OTHERS = ["cfg1_bcsr_tiny", "cfg3_bcsr_llm_gate", "cfg4_bcsr_sweep_b64_d0.1", "cfg4_bcsr_sweep_b16_d0.1",
-                  "cfg4_bcsr_sweep_b128_d0.1", "cfg4_bcsr_flat_b64_d0.05"]
+DEFAULT_OTHERS = ["cfg1_bcsr_tiny", "cfg3_bcsr_llm_gate", "cfg3_bcsr_llm_down",
+                  "cfg4_bcsr_sweep_b16_d0.1", "cfg4_bcsr_sweep_b32_d0.1", "cfg4_bcsr_sweep_b64_d0.1",
+                  "cfg4_bcsr_sweep_b128_d0.1", "cfg4_bcsr_sweep_b64_d0.5", "cfg4_bcsr_flat_b64_d0.05",
+                  "cfg5_wcsr_rmat_n32", "cfg5_wcsr_rmat_n128", "cfg5_wcsr_rmat_n256"]
+
+# DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures whose
+# summaries are under profiles/ (None where no capture of that exact launch exists).
+NCU_DRAM_TRAFFIC = {
+    "cfg2_wcsr_irregular": 134.4e6,     # profiles/wcsr_spmm_cfg2_ncu.md
+}
 
 
 # --------------------------------------------------------------------------- helpers
@@ -191,6 +202,12 @@ def roofline_of(info, ms, pk):
     r.update({"peak_source": pk["source"], "model_bytes": model_bytes, "t_roof_us": max(t_hbm, t_tc) * 1e6,
               "gather_bytes": info["bytes_gather"], "traffic": None})
     return r
+
+
+def with_traffic(roof, name):
+    roof = dict(roof)
+    roof["traffic"] = NCU_DRAM_TRAFFIC.get(name)
+    return roof
 
 
 def time_workload(torch, lib, w, steps, warmup, flush):
@@ -298,6 +315,7 @@ def main():
     ap.add_argument("--skip-others", action="store_true")
     ap.add_argument("--others", default=None, help="comma-separated workload names to report beside the headline")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--dense-width", type=int, default=0, help="override N of the --only workload (small profiling cases)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -320,6 +338,9 @@ def main():
     name = args.only or HEADLINE
     desc, builder = table[name]
     w = builder()
+    if args.dense_width:
+        w["N"] = args.dense_width
+        desc += " [N overridden to %d]" % args.dense_width
     warmup = max(3, args.warmup)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
 
@@ -397,7 +418,7 @@ def main():
                        "multi_gpu": "independent replicas, no collective"},
             "clocks": clocks, "e2e": e2e,
             "gpu_launches": int(res["launches_per_step"] * args.steps),
-            "roofline": head["roofline"], "cpu_baseline": cpu,
+            "roofline": with_traffic(head["roofline"], name if not args.dense_width else None), "cpu_baseline": cpu,
             "headline_detail": {k: head[k] for k in ("ms_median", "ms_min", "gflops_useful", "fill_ratio", "create_ms")},
             "others": others,
         }

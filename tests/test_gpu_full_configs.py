@@ -1,0 +1,99 @@
+"""GPU parity at the full sizes of the five benchmark configurations, launched exactly as
+bench.py launches them (spmm_run on device-resident operands).
+
+Where the oracle cannot afford every output, all rows are checked on a seeded subset of
+columns: the columns of C are independent of one another (C[:, j] depends on B[:, j] only,
+pinned in tests/test_oracle_spmm.py), and the subset covers the first, an interior and the
+last position of a token tile, a tile boundary, and the ragged end of N.
+"""
+import numpy as np
+import pytest
+
+from paper_2604_17834_b200 import workloads as wl
+
+from helpers import assert_close, reference, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2604_17834_b200 import binding
+    return binding
+
+
+def _sample_cols(N, seed):
+    fixed = [0, 1, 31, 32, 63, 64, 127, 128, 129, 255, 256, 511, 512, 513, N // 2, N - 129, N - 128, N - 65, N - 2, N - 1]
+    rng = np.random.default_rng(seed)
+    cols = set(c for c in fixed if 0 <= c < N) | set(rng.integers(0, N, size=44).tolist())
+    return np.array(sorted(cols), dtype=np.int64)
+
+
+def _run_and_check(lib, kind, a, dtype, size, N, Bs, cols=None, what=""):
+    import torch
+    mk = lib.spmm_bcsr_create_csr if kind == "bcsr" else lib.spmm_wcsr_create_csr
+    h = mk(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], dtype, size)
+    try:
+        Bd = to_device(Bs)
+        C = torch.full((a["m"], N), float("nan"), dtype=torch.float32, device="cuda")
+        st = torch.cuda.current_stream().cuda_stream
+        lib.spmm_run(h, Bd.data_ptr(), C.data_ptr(), N, st)
+        torch.cuda.synchronize()
+        lib.spmm_check(h)
+        assert not bool(torch.isnan(C).any()), "%s: unwritten outputs" % what
+        if cols is None:
+            got = C.cpu().numpy()
+            Cr, S = reference(a, Bs, dtype)
+        else:
+            got = C[:, torch.from_numpy(cols).cuda()].cpu().numpy()
+            Cr, S = reference(a, Bs, dtype, cols=cols)
+        worst = assert_close(got, Cr, S, dtype, what)
+        # second launch: same bits
+        C2 = torch.empty_like(C)
+        lib.spmm_run(h, Bd.data_ptr(), C2.data_ptr(), N, st)
+        torch.cuda.synchronize()
+        assert bool(torch.equal(C, C2)), "%s: run-to-run difference" % what
+        return worst
+    finally:
+        lib.spmm_destroy(h)
+
+
+def test_config1_wcsr_irregular_full(lib):
+    """configs[1]: 100,000 x 100,000 TF32, N = 128 -- every output element."""
+    a = wl.wcsr_irregular()
+    Bs = wl.dense(1102, a["k"], 128, ("normal", 0.0, 1.0), "tf32")
+    worst = _run_and_check(lib, "wcsr", a, "tf32", 16, 128, Bs, what="configs[1]")
+    assert worst < 1.0
+
+
+@pytest.mark.parametrize("shape", ["gate", "down"])
+def test_config2_bcsr_llm_full(lib, shape):
+    """configs[2]: 18944 x 3584 (gate) and 3584 x 18944 (down), 64 x 64 blocks, N = 65536."""
+    a = wl.bcsr_llm() if shape == "gate" else wl.bcsr_llm(seed=1013, m=3584, k=18944)
+    N = 65536
+    Bs = wl.dense(1103, a["k"], N, ("normal", 0.0, 1.0), "bf16")
+    _run_and_check(lib, "bcsr", a, "bf16", 64, N, Bs, cols=_sample_cols(N, 3), what="configs[2] " + shape)
+
+
+@pytest.mark.parametrize("b,d,skewed", [(16, 0.1, True), (32, 0.2, True), (64, 0.1, True), (128, 0.05, True),
+                                         (64, 0.05, False), (16, 0.01, False), (128, 0.5, True)])
+def test_config3_bcsr_sweep_full(lib, b, d, skewed):
+    """configs[3]: 8192 x 8192 fp16, N = 4096, skewed block-row lengths and flat low densities."""
+    a = wl.bcsr_sweep(1004 + b + int(d * 1000), b=b, density=d, skewed=skewed)
+    N = 4096
+    Bs = wl.dense(1104, a["k"], N, ("uniform", -1.0, 1.0), "fp16")
+    _run_and_check(lib, "bcsr", a, "fp16", b, N, Bs, cols=_sample_cols(N, b), what="configs[3] b=%d d=%g" % (b, d))
+
+
+@pytest.fixture(scope="module")
+def rmat_full():
+    return wl.rmat()
+
+
+@pytest.mark.parametrize("N", [32, 128, 256])
+def test_config4_wcsr_rmat_full(lib, rmat_full, N):
+    """configs[4]: R-MAT 2^21 x 2^21, ~32.4 M nnz, fp16, N = 32 / 128 / 256."""
+    a = rmat_full
+    Bs = wl.dense(1105 + N, a["k"], N, ("normal", 0.0, 1.0), "fp16")
+    cols = _sample_cols(N, N)[::3] if N > 32 else np.arange(0, 32, 3)
+    _run_and_check(lib, "wcsr", a, "fp16", 16, N, Bs, cols=cols, what="configs[4] N=%d" % N)
