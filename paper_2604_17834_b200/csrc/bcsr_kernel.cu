@@ -14,7 +14,8 @@
 //   warp 1      MMA issuer: one thread issues tcgen05.mma into one of two TMEM accumulator
 //               buffers; tcgen05.commit frees the ring slot / publishes the accumulator.
 //   warps 2-5   epilogue: tcgen05.ld -> registers -> global C (zeros for empty block-rows),
-//               overlapping the next tile's MMAs thanks to the second TMEM buffer.
+//               overlapping the next tile's MMAs thanks to the second TMEM buffer.  C is
+//               written with streaming stores so that it does not push the B slab out of L2.
 // The host deals tiles to CTAs ahead of time: slab by slab (a slab = token tiles whose B rows
 // fit in L2), longest block-row first, each tile to the least loaded CTA; CTA c walks its list.
 #include "kernels.h"
@@ -258,7 +259,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (nok) {
 #pragma unroll
                         for (int j = 0; j < W; ++j)
-                            if (c0 + j < rows) cp[static_cast<int64_t>(c0 + j) * N] = __uint_as_float(v[j]);
+                            if (c0 + j < rows) __stcs(cp + static_cast<int64_t>(c0 + j) * N, __uint_as_float(v[j]));
                     }
                 }
             }

@@ -116,6 +116,10 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // The merge kernel is launched as a programmatic dependent: let its CTAs be scheduled (and
+    // fetch their lists) while this grid runs; they block in griddepcontrol.wait until this
+    // grid has completed and its writes are visible.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
     const int64_t N = p.N;
     const int2 kNoDesc = make_int2(0, 0);
@@ -419,6 +423,9 @@ wcsr_merge_kernel(const MergeParams p) {
     const int w = p.window[i];
     const int first = p.first[i];
     const int nparts = p.nparts[i];
+    // everything above is creation-time data; the partial tiles and C belong to the SpMM
+    // kernel launched just before on the same stream: wait until it has completed
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t N = p.N;
     const int64_t row0 = static_cast<int64_t>(w) * kWH;
     const int rows = static_cast<int>(min_i64(kWH, p.m - row0));
@@ -507,8 +514,17 @@ cudaError_t wcsr_static_scratch(float** ptr, size_t* bytes) {
 
 cudaError_t launch_wcsr_merge(const MergeParams& p, cudaStream_t stream) {
     if (p.n <= 0) return cudaSuccess;
-    wcsr_merge_kernel<<<p.n, 256, 0, stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(p.n));
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel, p);
 }
 
 }  // namespace spmm
