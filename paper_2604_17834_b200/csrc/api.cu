@@ -105,6 +105,9 @@ struct spmm_handle_s {
     CUtensorMap tmA;
     bool tmA_ok = false;
     CUtensorMap tmB;
+    CUtensorMap tmB3;                // BCSR: B as [N / 64][k][64] for whole-tile loads
+    bool tmB3_ok = false;
+    int tmB_groups = 0;
     const void* tmB_ptr = nullptr;
     int64_t tmB_N = -1;
 
@@ -304,17 +307,34 @@ int encode_gather_map(CUtensorMap* map, int dtype, const void* base, uint64_t ro
 }
 
 int ensure_tmB(spmm_handle_s* h, const void* B, int64_t N, int groups) {
-    (void)groups;
-    if (h->tmB_ptr == B && h->tmB_N == N) return SPMM_OK;
+    if (h->tmB_ptr == B && h->tmB_N == N && h->tmB_groups == groups) return SPMM_OK;
     int rc;
-    if (h->format == 1)
+    if (h->format == 1) {
         rc = encode_gather_map(&h->tmB, h->dtype, B, static_cast<uint64_t>(h->k), static_cast<uint64_t>(N));
-    else
+    } else {
         rc = encode_2d_16bit(&h->tmB, h->dtype, B, static_cast<uint64_t>(h->k), static_cast<uint64_t>(N),
                              static_cast<uint32_t>(h->bcsr.b), 64, CU_TENSOR_MAP_SWIZZLE_128B);
+        // the same memory as [N / 64][k][64]: one request then brings a whole token tile
+        // (2 * groups boxes); only full 64-token groups are covered, a ragged tail uses tmB
+        h->tmB3_ok = false;
+        h->tmB3 = h->tmB;
+        EncodeTiledFn fn = get_encode_fn();
+        if (!rc && fn && N >= 64) {
+            const cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(h->k), static_cast<cuuint64_t>(N / 64)};
+            const cuuint64_t strides[2] = {static_cast<cuuint64_t>(N) * 2, 128};
+            const cuuint32_t box[3] = {64, static_cast<cuuint32_t>(h->bcsr.b), static_cast<cuuint32_t>(2 * groups)};
+            const cuuint32_t estr[3] = {1, 1, 1};
+            const CUtensorMapDataType dt = h->dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+            CUresult r = fn(&h->tmB3, dt, 3, const_cast<void*>(B), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            h->tmB3_ok = r == CUDA_SUCCESS;
+            if (!h->tmB3_ok) h->tmB3 = h->tmB;
+        }
+    }
     if (rc) return rc;
     h->tmB_ptr = B;
     h->tmB_N = N;
+    h->tmB_groups = groups;
     return SPMM_OK;
 }
 
@@ -392,7 +412,8 @@ int run_bcsr(spmm_handle_s* h, const void* B, float* C, int64_t N, cudaStream_t 
     }
     rc = ensure_tmB(h, B, N, h->sched.groups);
     if (rc) return rc;
-    cudaError_t e = launch_bcsr(h->dtype, f.b, h->sched.groups, tmA, h->tmB, p, h->n_ctas, stream);
+    p.use_3d = h->tmB3_ok ? 1 : 0;
+    cudaError_t e = launch_bcsr(h->dtype, f.b, h->sched.groups, tmA, h->tmB, h->tmB3, p, h->n_ctas, stream);
     return e == cudaSuccess ? SPMM_OK : SPMM_ERR_CUDA;
 }
 

@@ -44,7 +44,7 @@ struct BcsrCfg {
 template <int B, int GROUPS, int STAGES, int FMT>
 __global__ void __launch_bounds__(192, 1)
 bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                 const BcsrParams p) {
+                 const __grid_constant__ CUtensorMap tmB3, const BcsrParams p) {
     using Cfg = BcsrCfg<B, GROUPS, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -69,6 +69,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         fence_mbar_init();
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
+        prefetch_tmap(&tmB3);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);
@@ -100,6 +101,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
                 const int nbox = (nvalid + 63) >> 6;
                 const uint32_t tx = Cfg::kABytes + nbox * Cfg::kBoxBytes;
+                const bool whole_tile = p.use_3d && nvalid == Cfg::kBnT;
                 const int pb = __ldg(p.block_row_ptr + tI), pe = __ldg(p.block_row_ptr + tI + 1);
                 for (int q0 = pb; q0 < pe && ok; q0 += 32) {
                     // block columns of up to 32 stored blocks with one coalesced load
@@ -116,9 +118,14 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         const uint32_t sb = smem_base + s * Cfg::kStageBytes;
                         if (lane == 0) mbar_arrive_expect_tx(full_bar(s), tx);
                         __syncwarp();
-                        if (lane < nbox) {
+                        if (whole_tile) {
+                            // all 2 * GROUPS boxes of the stage with one request: B seen as
+                            // [64-token group][k][64 tokens], box = kNBox x b x 64
+                            if (lane == 0) tma_load_3d(sb, &tmB3, full_bar(s), 0, J * B, n0 >> 6);
+                        } else if (lane < nbox) {
                             tma_load_2d(sb + lane * Cfg::kBoxBytes, &tmB, full_bar(s), n0 + lane * 64, J * B);
-                        } else if (lane == 8) {
+                        }
+                        if (lane == 8) {
                             tma_load_2d(sb + Cfg::kDenseBytes, &tmA, full_bar(s), 0, q * B);
                         } else if (B > 64 && lane == 9) {
                             tma_load_2d(sb + Cfg::kDenseBytes + B * 128, &tmA, full_bar(s), 64, q * B);
@@ -286,8 +293,8 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 }
 
 template <int B, int GROUPS, int STAGES, int FMT>
-cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const BcsrParams& p, int grid,
-                       cudaStream_t stream) {
+cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3, const BcsrParams& p,
+                       int grid, cudaStream_t stream) {
     using Cfg = BcsrCfg<B, GROUPS, STAGES>;
     auto kfn = bcsr_spmm_kernel<B, GROUPS, STAGES, FMT>;
     static bool attr_done = false;
@@ -296,25 +303,25 @@ cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const Bcs
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    kfn<<<grid, 192, Cfg::kSmemBytes, stream>>>(tmA, tmB, p);
+    kfn<<<grid, 192, Cfg::kSmemBytes, stream>>>(tmA, tmB, tmB3, p);
     return cudaGetLastError();
 }
 
 template <int FMT>
-cudaError_t launch_fmt(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB,
+cudaError_t launch_fmt(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
                        const BcsrParams& p, int grid, cudaStream_t stream) {
     switch (b * 10 + groups) {
-        case 161: return launch_one<16, 1, 8, FMT>(tmA, tmB, p, grid, stream);
-        case 162: return launch_one<16, 2, 8, FMT>(tmA, tmB, p, grid, stream);
-        case 164: return launch_one<16, 4, 8, FMT>(tmA, tmB, p, grid, stream);
-        case 321: return launch_one<32, 1, 8, FMT>(tmA, tmB, p, grid, stream);
-        case 322: return launch_one<32, 2, 8, FMT>(tmA, tmB, p, grid, stream);
-        case 324: return launch_one<32, 4, 6, FMT>(tmA, tmB, p, grid, stream);
-        case 641: return launch_one<64, 1, 8, FMT>(tmA, tmB, p, grid, stream);
-        case 642: return launch_one<64, 2, 5, FMT>(tmA, tmB, p, grid, stream);
-        case 644: return launch_one<64, 4, 3, FMT>(tmA, tmB, p, grid, stream);
-        case 1281: return launch_one<128, 1, 3, FMT>(tmA, tmB, p, grid, stream);
-        case 1282: return launch_one<128, 2, 2, FMT>(tmA, tmB, p, grid, stream);
+        case 161: return launch_one<16, 1, 8, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 162: return launch_one<16, 2, 8, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 164: return launch_one<16, 4, 8, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 321: return launch_one<32, 1, 8, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 322: return launch_one<32, 2, 8, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 324: return launch_one<32, 4, 6, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 641: return launch_one<64, 1, 8, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 642: return launch_one<64, 2, 5, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 644: return launch_one<64, 4, 3, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 1281: return launch_one<128, 1, 3, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 1282: return launch_one<128, 2, 2, FMT>(tmA, tmB, tmB3, p, grid, stream);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -324,9 +331,9 @@ cudaError_t launch_fmt(int b, int groups, const CUtensorMap& tmA, const CUtensor
 int bcsr_token_groups_max(int b) { return b == 128 ? 2 : 4; }
 
 cudaError_t launch_bcsr(int dtype, int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                        const BcsrParams& p, int grid, cudaStream_t stream) {
-    if (dtype == 1) return launch_fmt<0>(b, groups, tmA, tmB, p, grid, stream);   // fp16
-    if (dtype == 0) return launch_fmt<1>(b, groups, tmA, tmB, p, grid, stream);   // bf16
+                        const CUtensorMap& tmB3, const BcsrParams& p, int grid, cudaStream_t stream) {
+    if (dtype == 1) return launch_fmt<0>(b, groups, tmA, tmB, tmB3, p, grid, stream);   // fp16
+    if (dtype == 0) return launch_fmt<1>(b, groups, tmA, tmB, tmB3, p, grid, stream);   // bf16
     return cudaErrorInvalidValue;
 }
 

@@ -17,11 +17,13 @@ struct BcsrParams {
     int* status;
     uint64_t wait_limit_ns;
     long long* trace;   // tuning builds only (SPMM_TRACE); nullptr otherwise
+    int32_t use_3d;     // tmB3 is valid: whole token tiles are fetched with one 3-D request
 };
 
 // dtype: 0 bf16, 1 fp16.  groups: token tile = 128 * groups columns of B (1, 2 or 4).
+// tmB: B as [k][N], box b x 64.  tmB3: B as [N / 64][k][64], box (2 * groups) x b x 64.
 cudaError_t launch_bcsr(int dtype, int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                        const BcsrParams& p, int grid, cudaStream_t stream);
+                        const CUtensorMap& tmB3, const BcsrParams& p, int grid, cudaStream_t stream);
 int bcsr_token_groups_max(int b);
 
 // WCSR pipeline shape, shared by the host schedule (fills are cut to the stage size) and the

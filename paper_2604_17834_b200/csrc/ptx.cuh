@@ -146,6 +146,16 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* m, 
         : "memory");
 }
 
+// 3-D tiled load, no multicast: box at element coordinates (x = innermost, y, z = outermost).
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* m, uint32_t bar,
+                                            int32_t x, int32_t y, int32_t z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+
 // Row gather (tile::gather4): four rows y0..y3 of a 2-D tensor, each starting at element x and
 // as wide as the tensor map's box (whose row extent is 1), land as four consecutive box rows
 // at dst.  Rows outside the tensor (e.g. index -1) are filled with zeros.  No multicast.
