@@ -92,6 +92,9 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         {
             uint32_t it = 0;
             bool ok = true;
+            // A blocks and the B slab are re-read by other CTAs while the slab lasts: ask L2 to
+            // keep them in preference to the C lines streaming through
+            const uint64_t keep = l2_policy_evict_last();
             TRACE_DECL(tr_empty);
             TRACE_T0(tr_start);
             for (int ti = tile_begin; ti < tile_end && ok; ++ti) {
@@ -121,14 +124,14 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         if (whole_tile) {
                             // all 2 * GROUPS boxes of the stage with one request: B seen as
                             // [64-token group][k][64 tokens], box = kNBox x b x 64
-                            if (lane == 0) tma_load_3d(sb, &tmB3, full_bar(s), 0, J * B, n0 >> 6);
+                            if (lane == 0) tma_load_3d_hint(sb, &tmB3, full_bar(s), 0, J * B, n0 >> 6, keep);
                         } else if (lane < nbox) {
-                            tma_load_2d(sb + lane * Cfg::kBoxBytes, &tmB, full_bar(s), n0 + lane * 64, J * B);
+                            tma_load_2d_hint(sb + lane * Cfg::kBoxBytes, &tmB, full_bar(s), n0 + lane * 64, J * B, keep);
                         }
                         if (lane == 8) {
-                            tma_load_2d(sb + Cfg::kDenseBytes, &tmA, full_bar(s), 0, q * B);
+                            tma_load_2d_hint(sb + Cfg::kDenseBytes, &tmA, full_bar(s), 0, q * B, keep);
                         } else if (B > 64 && lane == 9) {
-                            tma_load_2d(sb + Cfg::kDenseBytes + B * 128, &tmA, full_bar(s), 64, q * B);
+                            tma_load_2d_hint(sb + Cfg::kDenseBytes + B * 128, &tmA, full_bar(s), 64, q * B, keep);
                         }
                     }
                 }
