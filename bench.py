@@ -253,6 +253,18 @@ def summarize(name, desc, res, pk, N):
     }
 
 
+def aggregate_over_ranks(ms_local, flops_per_rank, world, dist=None, device="cpu"):
+    """Replicas-only aggregation: every rank ran the same workload on its own GPU.
+    -> (max step time over ranks in ms, whole-job GFLOP/s = world * flops / max time)."""
+    ms = float(ms_local)
+    if world > 1:
+        import torch
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms, world * flops_per_rank / (ms * 1e-3) / 1e9
+
+
 # --------------------------------------------------------------------------- CPU oracle legs
 
 
@@ -355,13 +367,8 @@ def main():
     res = time_workload(torch, lib, w, args.steps, warmup, flush)
     barrier()
     clocks = sampler.stop()
-    ms = res["ms_mean"]
-    if world > 1:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
     info = res["info"]
-    value = world * info["flops_stored"] / (ms * 1e-3) / 1e9
+    ms, value = aggregate_over_ranks(res["ms_mean"], info["flops_stored"], world, dist, "cuda")
     head = summarize(name, desc, res, pk, w["N"])
 
     # end to end through the C ABI with host buffers (pinned), copies inside the timed region
@@ -381,11 +388,8 @@ def main():
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
     lib.spmm_destroy(h)
-    if world > 1:
-        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e = {"value": world * info["flops_stored"] / e2e_s / 1e9, "unit": UNIT, "ms_per_step": e2e_s * 1e3,
+    e2e_ms, e2e_value = aggregate_over_ranks(e2e_s * 1e3, info["flops_stored"], world, dist, "cuda")
+    e2e = {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
            "h2d_bytes_per_step": int(Bh.numel() * Bh.element_size()), "d2h_bytes_per_step": int(Ch.numel() * 4)}
     del res["B"], res["C"]
 

@@ -235,7 +235,9 @@ const char *spmm_status_string(int code);
 
 /*
  * Upper bound, in nanoseconds, of any single wait inside a kernel (default 2e9).  Process
- * wide; meant for tests of the timeout path.  Values below 1000 are raised to 1000.
+ * wide.  0 makes every wait that is not satisfied on its first poll run out at once: a hook
+ * for testing the failure path (the kernel leaves early, spmm_check reports
+ * SPMM_ERR_DEV_TIMEOUT, the context stays usable).
  */
 int spmm_set_wait_limit_ns(uint64_t ns);
 

@@ -779,7 +779,7 @@ void spmm_debug_set_trace(long long* dev_buf) { g_trace = dev_buf; }
 #endif
 
 int spmm_set_wait_limit_ns(uint64_t ns) {
-    g_wait_limit_ns.store(ns < 1000 ? 1000 : ns);
+    g_wait_limit_ns.store(ns);
     return SPMM_OK;
 }
 

@@ -58,6 +58,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * STAGES + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * STAGES + 5);
+    const uint32_t drain_bar = bar0 + 8u * (2 * STAGES + 6);   // abort path: MMAs still in flight
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     WaitCtl ctl{abort_flag, p.status, p.wait_limit_ns};
@@ -65,6 +66,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(accf_bar(a), 1); mbar_init(acce_bar(a), 4); }
+        mbar_init(drain_bar, 1);
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tmap(&tmA);
@@ -210,6 +212,12 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (pe > pb) tc_commit(accf_bar(acc));
                     else mbar_arrive(accf_bar(acc));
                 }
+            }
+            if (!ok && leader) {
+                // abort path: let the MMAs already issued finish before TMEM is freed
+                tc_commit(drain_bar);
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < 2000000ull) {}
             }
             if (lane == 0) {
                 TRACE_PUT(4, clock64() - tr_start);

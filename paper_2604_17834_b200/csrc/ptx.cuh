@@ -88,6 +88,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
+// Non-blocking poll (try_wait may suspend the thread for a while before it answers).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
 // Shared by every role of a CTA: where a bounded wait reports that it ran out.
 struct WaitCtl {
     volatile int* abort_flag;   // shared memory: set once any wait of the CTA ran out
@@ -99,11 +114,16 @@ struct WaitCtl {
 // the caller then leaves its loop and walks to the kernel's common teardown.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtl& ctl,
                                           int site) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (ctl.limit_ns == 0) {
+        // test hook: one non-blocking poll, then the wait counts as run out
+        if (mbar_test_wait(bar, parity)) return true;
+    } else if (mbar_try_wait(bar, parity)) {
+        return true;
+    }
     const uint64_t t0 = globaltimer_ns();
     for (uint32_t spin = 1;; ++spin) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 63u) == 0u) {
+        if (ctl.limit_ns != 0 && mbar_try_wait(bar, parity)) return true;
+        if ((spin & 63u) == 0u || ctl.limit_ns == 0) {
             if (*ctl.abort_flag) return false;
             if (globaltimer_ns() - t0 > ctl.limit_ns) {
                 *ctl.abort_flag = 1;

@@ -89,7 +89,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
-    static_assert((2 * STAGES + 2 * Cfg::kNAcc + 2) * 8 <= 256, "barrier area is 256 bytes");
+    static_assert((2 * STAGES + 2 * Cfg::kNAcc + 3) * 8 <= 256, "barrier area is 256 bytes");
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * Cfg::kStageBytes);
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -98,6 +98,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
     auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + Cfg::kNAcc + a); };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * STAGES + 2 * Cfg::kNAcc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * STAGES + 2 * Cfg::kNAcc + 1);
+    const uint32_t drain_bar = bar0 + 8u * (2 * STAGES + 2 * Cfg::kNAcc + 2);   // abort path: MMAs still in flight
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     WaitCtl ctl{abort_flag, p.status, p.wait_limit_ns};
@@ -105,6 +106,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < Cfg::kNAcc; ++a) { mbar_init(accf_bar(a), 1); mbar_init(acce_bar(a), 4); }
+        mbar_init(drain_bar, 1);
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tmap(&tmB);
@@ -316,6 +318,12 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                 }
                 win = nwin;
             }
+        }
+        if (!ok && leader) {
+            // abort path: let the MMAs already issued finish before TMEM is freed
+            tc_commit(drain_bar);
+            const uint64_t t0 = globaltimer_ns();
+            while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < 2000000ull) {}
         }
 #ifdef SPMM_TRACE
         if (lane == 0) {

@@ -164,3 +164,33 @@ def test_bad_run_arguments(lib):
             lib.spmm_run(h, *args)
         assert e.value.code == code
     lib.spmm_destroy(h)
+
+
+@pytest.mark.parametrize("kind", ["bcsr", "wcsr"])
+def test_wait_that_runs_out_is_reported_and_the_context_survives(lib, kind):
+    """Every wait inside the kernels is bounded.  With the bound set to zero the first wait
+    for operands that are still on their way runs out: the kernel leaves early
+    through its normal teardown, spmm_check reports SPMM_ERR_DEV_TIMEOUT, and the same
+    handle then works again once the bound is restored."""
+    if kind == "bcsr":
+        a, dtype, size, N = wl.bcsr_sweep(404, m=2048, k=2048, b=64, density=0.3, dtype="fp16"), "fp16", 64, 1024
+        mk = lib.spmm_bcsr_create_csr
+    else:
+        a, dtype, size, N = wl.wcsr_irregular(seed=405, m=20000, dtype="tf32"), "tf32", 16, 128
+        mk = lib.spmm_wcsr_create_csr
+    Bs = wl.dense(41, a["k"], N, ("normal", 0.0, 1.0), dtype)
+    h = mk(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], dtype, size)
+    try:
+        lib.spmm_set_wait_limit_ns(0)
+        run_gpu(lib, h, Bs, a["m"], N, check=False)
+        with pytest.raises(lib.SpmmError) as e:
+            lib.spmm_check(h)
+        assert e.value.code == lib.SPMM_ERR_DEV_TIMEOUT
+        lib.spmm_set_wait_limit_ns(2_000_000_000)
+        lib.spmm_check(h)                                   # the status word was cleared
+        C = run_gpu(lib, h, Bs, a["m"], N)
+        Cr, S = reference(a, Bs, dtype)
+        assert_close(C, Cr, S, dtype, "after timeout")
+    finally:
+        lib.spmm_set_wait_limit_ns(2_000_000_000)
+        lib.spmm_destroy(h)
