@@ -226,7 +226,7 @@ int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const s
     rc = device_setup(h, opts);
     if (rc) { free_handle(h); return rc; }
     try {
-        rc = build_wcsr(a, wh, b_col, T, h->n_ctas * 2, &h->wcsr);
+        rc = build_wcsr(a, wh, b_col, T, h->n_ctas * kWcsrBinsPerSm, &h->wcsr);
     } catch (const std::bad_alloc&) {
         rc = SPMM_ERR_ALLOC;
     }

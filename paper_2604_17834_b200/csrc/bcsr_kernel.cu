@@ -213,12 +213,6 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     else mbar_arrive(accf_bar(acc));
                 }
             }
-            if (!ok && leader) {
-                // abort path: let the MMAs already issued finish before TMEM is freed
-                tc_commit(drain_bar);
-                const uint64_t t0 = globaltimer_ns();
-                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < 2000000ull) {}
-            }
             if (lane == 0) {
                 TRACE_PUT(4, clock64() - tr_start);
                 TRACE_PUT(5, tr_full);
@@ -298,6 +292,17 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
+        if (*abort_flag) {
+            // abort path: let the MMAs this warp's elected lane already issued finish before
+            // TMEM is freed (kept out of the role loop above on purpose: placed there it
+            // slowed the normal path measurably)
+            if (elect_one()) {
+                tc_commit(drain_bar);
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < 2000000ull) {}
+            }
+            __syncwarp();
+        }
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, Cfg::kTmemCols);
     }

@@ -44,6 +44,10 @@ int bcsr_token_groups_max(int b);
 #ifndef WCSR_PW2
 #define WCSR_PW2 6
 #endif
+// bins per SM of the static WCSR schedule = the largest CTAs-per-SM count of the kernel
+// variants: every resident CTA gets one bin (two when a variant fits one CTA per SM).  More,
+// smaller bins measured slower: each bin start pays a chain of cold index loads.
+constexpr int kWcsrBinsPerSm = 2;
 constexpr int wcsr_stage_cols(int es) { return WCSR_STAGE_ROW_BYTES / es; }
 constexpr int kWcsrStages1 = WCSR_STAGES1, kWcsrStages2 = WCSR_STAGES2;
 constexpr int kWcsrProducerWarps1 = WCSR_PW1, kWcsrProducerWarps2 = WCSR_PW2;

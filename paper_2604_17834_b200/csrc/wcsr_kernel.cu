@@ -49,9 +49,13 @@ struct WcsrCfg {
     static constexpr int kDenseBytes = KT * kRowBytes;
     static constexpr int kABytes = (KT / kKStep) * (kWH * 32);
     static constexpr int kStageBytes = kDenseBytes + kABytes;
-    static constexpr int kNAcc = GROUPS == 1 ? 4 : 2;       // items with live accumulators
+    // CTAs that fit one SM by shared memory (1 KB per CTA is reserved), at most kWcsrBinsPerSm
+    static constexpr int kCtasBySmem = (227 * 1024) / (STAGES * kStageBytes + 1024 + 256 + 1024);
+    static constexpr int kCtasPerSm = kCtasBySmem < 1 ? 1 : (kCtasBySmem > kWcsrBinsPerSm ? kWcsrBinsPerSm : kCtasBySmem);
+    // items with live accumulators: the SM's 512 TMEM columns are shared by its resident CTAs
+    static constexpr int kNAcc = (512 / kCtasPerSm) / (GROUPS * kNSub * kWH) >= 4 ? 4 : 2;
     static constexpr int kAccCols = GROUPS * kNSub * kWH;   // TMEM columns of one item
-    static constexpr int kTmemCols = kNAcc * kAccCols;      // 256
+    static constexpr int kTmemCols = kNAcc * kAccCols;      // 128 or 256
     static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 + 256;
     static_assert(KT % 8 == 0 && KT % kKStep == 0 && KT <= 128, "stage shape");
     static_assert(kGathers % 32 == 0 || kGathers == 16, "gather instructions are dealt to warps");
@@ -77,7 +81,7 @@ struct SegIter {
 };
 
 template <int ES, int FMT, int GROUPS, int KT, int STAGES, int PW>
-__global__ void __launch_bounds__((PW + 5) * 32, (WcsrCfg<ES, GROUPS, KT, STAGES>::kSmemBytes + 1024) * 2 <= 227 * 1024 ? 2 : 1)
+__global__ void __launch_bounds__((PW + 5) * 32, WcsrCfg<ES, GROUPS, KT, STAGES>::kCtasPerSm)
 wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
     using Cfg = WcsrCfg<ES, GROUPS, KT, STAGES>;
     constexpr int kProducerWarps = PW;          // warps 0 .. PW-1; MMA warp PW; epilogue PW+1 .. PW+4
@@ -294,8 +298,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                         // descriptors differ only in their start-address field (bytes >> 4)
                         const uint64_t a0 = adesc0 + (sb >> 4);
                         const uint64_t b0 = bdesc0 + ((sb + Cfg::kDenseBytes) >> 4);
-                        uint32_t kk = kstep_item;
-                        for (int ks = 0; ks < nks; ++ks, ++kk) {
+                        auto issue = [&](int ks, uint32_t kk) {
                             const uint32_t dsub = d0 + (kk & (kNSub - 1)) * kWH;
                             const uint32_t accum = kk >= kNSub ? 1u : 0u;    // first use overwrites
 #pragma unroll
@@ -304,6 +307,13 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                                     umma_ss<FMT == 2>(dsub + g * kNSub * kWH,
                                                       a0 + ((g * Cfg::kAtomsPerGroup * Cfg::kAtomStride + ks * (Cfg::kKStep / 8) * 1024) >> 4),
                                                       b0 + ((ks * (kWH * 32)) >> 4), idesc, accum);
+                        };
+                        constexpr int kFullSteps = KT / Cfg::kKStep;
+                        if (nks == kFullSteps) {                 // a full stage: straight-line code
+#pragma unroll
+                            for (int ks = 0; ks < kFullSteps; ++ks) issue(ks, kstep_item + ks);
+                        } else {
+                            for (int ks = 0; ks < nks; ++ks) issue(ks, kstep_item + ks);
                         }
                         if (leader) {
                             tc_commit(empty_bar(s));
@@ -318,12 +328,6 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                 }
                 win = nwin;
             }
-        }
-        if (!ok && leader) {
-            // abort path: let the MMAs already issued finish before TMEM is freed
-            tc_commit(drain_bar);
-            const uint64_t t0 = globaltimer_ns();
-            while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < 2000000ull) {}
         }
 #ifdef SPMM_TRACE
         if (lane == 0) {
@@ -418,6 +422,17 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
     tc_fence_before_sync();
     __syncthreads();
     if (warp == kMmaWarp) {
+        if (*abort_flag) {
+            // abort path: let the MMAs this warp's elected lane already issued finish before
+            // TMEM is freed (kept out of the role loop above on purpose: placed there it
+            // slowed the normal path measurably)
+            if (elect_one()) {
+                tc_commit(drain_bar);
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < 2000000ull) {}
+            }
+            __syncwarp();
+        }
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, Cfg::kTmemCols);
     }
@@ -461,11 +476,10 @@ cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cud
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(kfn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
-        // resident CTAs per SM: 227 KB of shared memory (1 KB reserved per CTA), 512 TMEM
-        // columns, and the register file (__launch_bounds__ keeps two CTAs resident)
-        int o = (227 * 1024) / (Cfg::kSmemBytes + 1024);
-        o = o < 512 / Cfg::kTmemCols ? o : 512 / Cfg::kTmemCols;
-        occ = o < 1 ? 1 : (o > 2 ? 2 : o);
+        // resident CTAs per SM: by shared memory and TMEM columns (see WcsrCfg); the register
+        // file follows from __launch_bounds__
+        static_assert(Cfg::kCtasPerSm * Cfg::kTmemCols <= 512, "TMEM over-subscribed");
+        occ = Cfg::kCtasPerSm;
     }
     int grid = sms * occ;
     if (grid > p.n_bins) grid = p.n_bins;
