@@ -195,7 +195,8 @@ int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, cons
             const int bw = f.b < 64 ? f.b : 64;
             const CUtensorMapSwizzle swz = bw == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
                                           : (bw == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
-            rc = encode_2d_16bit(&h->tmA, dtype, h->d_vals, static_cast<uint64_t>(f.nnzb) * f.b, f.b, f.b, bw, swz);
+            rc = encode_2d_16bit(&h->tmA, dtype, h->d_vals, static_cast<uint64_t>(f.nnzb) * f.b, f.b,
+                                 static_cast<uint32_t>(f.b * bcsr_blocks_per_stage(f.b)), bw, swz);
             h->tmA_ok = rc == SPMM_OK;
         }
         if (rc) { free_handle(h); return rc; }

@@ -28,17 +28,25 @@ namespace {
 template <int B, int GROUPS, int STAGES>
 struct BcsrCfg {
     static constexpr int kBnT = 128 * GROUPS;
-    static constexpr int kNBox = 2 * GROUPS;                 // 64-token boxes per stage
+    static constexpr int kNBox = 2 * GROUPS;                 // 64-token boxes per block
     static constexpr int kBoxBytes = B * 128;                // b k-rows x 128 B
-    static constexpr int kDenseBytes = kNBox * kBoxBytes;
+    static constexpr int kDenseBytes = kNBox * kBoxBytes;    // B tile of one block
     static constexpr int kABytes = B * B * 2;
-    static constexpr int kStageBytes = ((kDenseBytes + kABytes + 1023) / 1024) * 1024;
+    // Small blocks carry too little work for the fixed cost of a pipeline stage (barrier
+    // round trip, request issue, MMA hand-off): a stage holds several consecutive stored
+    // blocks of the block-row, their B tiles first, then their A blocks (one request).
+    static constexpr int kBps = bcsr_blocks_per_stage(B);
+    static constexpr int kStageBytes = ((kBps * (kDenseBytes + kABytes) + 1023) / 1024) * 1024;
+    static constexpr int kAOff = kBps * kDenseBytes;         // A blocks inside the stage
     static constexpr int kARowBytes = (B < 64 ? B : 64) * 2;
     static constexpr uint32_t kASwizzle = kARowBytes == 128 ? SWZ_128B : (kARowBytes == 64 ? SWZ_64B : SWZ_32B);
     static constexpr int kAccCols = GROUPS * B;
     static constexpr int kTmemCols = (2 * kAccCols <= 32) ? 32 : (2 * kAccCols <= 64 ? 64 : (2 * kAccCols <= 128 ? 128 : (2 * kAccCols <= 256 ? 256 : 512)));
     static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
     static_assert(2 * kAccCols <= 512, "accumulators exceed TMEM");
+    static_assert(kSmemBytes <= 227 * 1024, "stage ring exceeds shared memory");
+    static_assert((2 * STAGES + 7) * 8 <= 256, "barrier area is 256 bytes");
+    static_assert(kBps == 1 || B <= 32, "multi-block stages are for the small block sizes");
 };
 
 template <int B, int GROUPS, int STAGES, int FMT>
@@ -105,35 +113,41 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int n0 = tcd.y * Cfg::kBnT;
                 const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
                 const int nbox = (nvalid + 63) >> 6;
-                const uint32_t tx = Cfg::kABytes + nbox * Cfg::kBoxBytes;
                 const bool whole_tile = p.use_3d && nvalid == Cfg::kBnT;
                 const int pb = __ldg(p.block_row_ptr + tI), pe = __ldg(p.block_row_ptr + tI + 1);
                 for (int q0 = pb; q0 < pe && ok; q0 += 32) {
                     // block columns of up to 32 stored blocks with one coalesced load
                     const int Jl = (q0 + lane < pe) ? __ldg(p.block_col_idx + q0 + lane) : 0;
                     const int nq = min(32, pe - q0);
-                    for (int jq = 0; jq < nq; ++jq, ++it) {
+                    for (int jq = 0; jq < nq; jq += Cfg::kBps, ++it) {
                         const int q = q0 + jq;
-                        const int J = __shfl_sync(0xffffffffu, Jl, jq);
+                        const int nb = min(Cfg::kBps, nq - jq);          // stored blocks in this stage
                         const int s = it % STAGES;
                         const uint32_t ph = (it / STAGES) & 1u;
                         TRACE_T0(tr_a);
                         if (!__all_sync(0xffffffffu, mbar_wait(empty_bar(s), ph ^ 1u, ctl, 1))) { ok = false; break; }
                         TRACE_ADD(tr_empty, tr_a);
                         const uint32_t sb = smem_base + s * Cfg::kStageBytes;
-                        if (lane == 0) mbar_arrive_expect_tx(full_bar(s), tx);
+                        // the A request always brings kBps blocks (the box of the tensor map)
+                        if (lane == 0) mbar_arrive_expect_tx(full_bar(s), Cfg::kBps * Cfg::kABytes + nb * nbox * Cfg::kBoxBytes);
                         __syncwarp();
                         if (whole_tile) {
-                            // all 2 * GROUPS boxes of the stage with one request: B seen as
-                            // [64-token group][k][64 tokens], box = kNBox x b x 64
-                            if (lane == 0) tma_load_3d_hint(sb, &tmB3, full_bar(s), 0, J * B, n0 >> 6, keep);
-                        } else if (lane < nbox) {
-                            tma_load_2d_hint(sb + lane * Cfg::kBoxBytes, &tmB, full_bar(s), n0 + lane * 64, J * B, keep);
+                            // all 2 * GROUPS boxes of a block with one request: B seen as
+                            // [64-token group][k][64 tokens], box = kNBox x b x 64; lane i takes block i
+                            const int J = __shfl_sync(0xffffffffu, Jl, jq + (lane < nb ? lane : 0));
+                            if (lane < nb) tma_load_3d_hint(sb + lane * Cfg::kDenseBytes, &tmB3, full_bar(s), 0, J * B, n0 >> 6, keep);
+                        } else {
+                            for (int i = 0; i < nb; ++i) {
+                                const int J = __shfl_sync(0xffffffffu, Jl, jq + i);
+                                if (lane < nbox)
+                                    tma_load_2d_hint(sb + i * Cfg::kDenseBytes + lane * Cfg::kBoxBytes, &tmB, full_bar(s),
+                                                     n0 + lane * 64, J * B, keep);
+                            }
                         }
                         if (lane == 8) {
-                            tma_load_2d_hint(sb + Cfg::kDenseBytes, &tmA, full_bar(s), 0, q * B, keep);
+                            tma_load_2d_hint(sb + Cfg::kAOff, &tmA, full_bar(s), 0, q * B, keep);
                         } else if (B > 64 && lane == 9) {
-                            tma_load_2d_hint(sb + Cfg::kDenseBytes + B * 128, &tmA, full_bar(s), 64, q * B, keep);
+                            tma_load_2d_hint(sb + Cfg::kAOff + B * 128, &tmA, full_bar(s), 64, q * B, keep);
                         }
                     }
                 }
@@ -182,7 +196,9 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 tc_fence_after_sync();
                 const uint32_t d0 = tmem_base + acc * Cfg::kAccCols;
                 const int pb = __ldg(p.block_row_ptr + tI), pe = __ldg(p.block_row_ptr + tI + 1);
-                for (int q = pb; q < pe; ++q, ++it) {
+                for (int q = pb; q < pe; q += Cfg::kBps, ++it) {
+                    // stages never straddle the producer's 32-block windows (kBps divides 32)
+                    const int nb = min(Cfg::kBps, min(pe - q, 32 - ((q - pb) & 31)));
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
                     TRACE_T0(tr_b);
@@ -191,18 +207,23 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     tc_fence_after_sync();
                     TRACE_T0(tr_c);
                     const uint32_t sb = smem_base + s * Cfg::kStageBytes;
-                    // descriptors differ only in their start-address field (bytes >> 4)
-                    const uint64_t a0 = adesc0 + (sb >> 4);
-                    const uint64_t b0 = bdesc0 + ((sb + Cfg::kDenseBytes) >> 4);
-                    const uint32_t accum0 = q > pb ? 1u : 0u;
 #pragma unroll
-                    for (int ks = 0; ks < B / 16; ++ks) {
-                        const uint32_t boff = B <= 64 ? ks * 32 : (ks >> 2) * (B * 128) + (ks & 3) * 32;
+                    for (int i = 0; i < Cfg::kBps; ++i) {
+                        if (i < nb) {
+                            // descriptors differ only in their start-address field (bytes >> 4)
+                            const uint64_t a0 = adesc0 + ((sb + i * Cfg::kDenseBytes) >> 4);
+                            const uint64_t b0 = bdesc0 + ((sb + Cfg::kAOff + i * Cfg::kABytes) >> 4);
+                            const uint32_t accum0 = (q > pb || i > 0) ? 1u : 0u;
 #pragma unroll
-                        for (int g = 0; g < GROUPS; ++g)
-                            if (leader && g < ngrp)
-                                umma_ss<false>(d0 + g * B, a0 + ((g * 2 * Cfg::kBoxBytes + ks * 2048) >> 4),
-                                               b0 + (boff >> 4), idesc, ks > 0 ? 1u : accum0);
+                            for (int ks = 0; ks < B / 16; ++ks) {
+                                const uint32_t boff = B <= 64 ? ks * 32 : (ks >> 2) * (B * 128) + (ks & 3) * 32;
+#pragma unroll
+                                for (int g = 0; g < GROUPS; ++g)
+                                    if (leader && g < ngrp)
+                                        umma_ss<false>(d0 + g * B, a0 + ((g * 2 * Cfg::kBoxBytes + ks * 2048) >> 4),
+                                                       b0 + (boff >> 4), idesc, ks > 0 ? 1u : accum0);
+                            }
+                        }
                     }
                     if (leader) tc_commit(empty_bar(s));
                     TRACE_ADD(tr_issue, tr_c);
@@ -327,12 +348,12 @@ template <int FMT>
 cudaError_t launch_fmt(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
                        const BcsrParams& p, int grid, cudaStream_t stream) {
     switch (b * 10 + groups) {
-        case 161: return launch_one<16, 1, 8, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 162: return launch_one<16, 2, 8, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 164: return launch_one<16, 4, 8, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 321: return launch_one<32, 1, 8, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 322: return launch_one<32, 2, 8, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 324: return launch_one<32, 4, 6, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 161: return launch_one<16, 1, 10, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 162: return launch_one<16, 2, 5, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 164: return launch_one<16, 4, 3, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 321: return launch_one<32, 1, 10, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 322: return launch_one<32, 2, 5, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 324: return launch_one<32, 4, 3, FMT>(tmA, tmB, tmB3, p, grid, stream);
         case 641: return launch_one<64, 1, 8, FMT>(tmA, tmB, tmB3, p, grid, stream);
         case 642: return launch_one<64, 2, 5, FMT>(tmA, tmB, tmB3, p, grid, stream);
         case 644: return launch_one<64, 4, 3, FMT>(tmA, tmB, tmB3, p, grid, stream);

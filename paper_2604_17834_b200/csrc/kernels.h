@@ -25,6 +25,8 @@ struct BcsrParams {
 cudaError_t launch_bcsr(int dtype, int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB,
                         const CUtensorMap& tmB3, const BcsrParams& p, int grid, cudaStream_t stream);
 int bcsr_token_groups_max(int b);
+// stored blocks that share one pipeline stage (and one A request): 4 / 2 for b = 16 / 32
+constexpr int bcsr_blocks_per_stage(int b) { return b == 16 ? 4 : (b == 32 ? 2 : 1); }
 
 // WCSR pipeline shape, shared by the host schedule (fills are cut to the stage size) and the
 // kernel: columns per shared-memory stage, ring depth and producer warps for the one-group
