@@ -99,6 +99,9 @@ typedef struct {
     int64_t plan_n;          /* dense width it was built for                                  */
     int32_t plan_token_tile; /* columns of B per tile: 128, 256 or 512                        */
     int32_t plan_slab_tiles; /* token tiles per L2 slab                                       */
+    int32_t n_bins;          /* WCSR: bins of the static task schedule (0 for BCSR): n_ctas x
+                                the resident CTAs per SM of the kernel for this value type     */
+    int32_t reserved0;
 } spmm_info_t;
 
 /* Arrays spmm_export can return, in their canonical (paper) layout. */

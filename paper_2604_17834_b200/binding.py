@@ -69,6 +69,7 @@ class SpmmInfo(ctypes.Structure):
         ("bytes_gather", ctypes.c_double), ("flops_stored", ctypes.c_double),
         ("workspace_bytes", ctypes.c_int64),
         ("plan_n", ctypes.c_int64), ("plan_token_tile", ctypes.c_int32), ("plan_slab_tiles", ctypes.c_int32),
+        ("n_bins", ctypes.c_int32), ("reserved0", ctypes.c_int32),
     ]
 
     def as_dict(self):

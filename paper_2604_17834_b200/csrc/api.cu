@@ -227,7 +227,7 @@ int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const s
     rc = device_setup(h, opts);
     if (rc) { free_handle(h); return rc; }
     try {
-        rc = build_wcsr(a, wh, b_col, T, h->n_ctas * kWcsrBinsPerSm, &h->wcsr);
+        rc = build_wcsr(a, wh, b_col, T, h->n_ctas * wcsr_bins_per_sm(elem_size(dtype)), &h->wcsr);
     } catch (const std::bad_alloc&) {
         rc = SPMM_ERR_ALLOC;
     }
@@ -427,8 +427,7 @@ int64_t wcsr_workspace_bytes(const spmm_handle_s* h, int64_t N) {
 
 int launch_wcsr_all(spmm_handle_s* h, const void* B, float* C, float* partial, int64_t N, cudaStream_t stream) {
     const WcsrHost& f = h->wcsr;
-    const int groups = N > 128 ? 2 : 1;
-    const int bnt = 128 * groups;
+    const int bnt = 128;                    // tokens per tile; wider B takes one pass per tile
     WcsrParams p;
     p.bin_ptr = h->d_bin_ptr;
     p.items = reinterpret_cast<const int4*>(h->d_items);
@@ -450,9 +449,9 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, float* C, float* partial, i
     p.trace = g_trace;
 #endif
     if (!f.tasks.empty()) {
-        int rc = ensure_tmB(h, B, N, groups);
+        int rc = ensure_tmB(h, B, N, 1);
         if (rc) return rc;
-        cudaError_t e = launch_wcsr(h->dtype, groups, h->tmB, p, h->sms, stream);
+        cudaError_t e = launch_wcsr(h->dtype, h->tmB, p, h->sms, stream);
         if (e != cudaSuccess) return SPMM_ERR_CUDA;
     }
     MergeParams mp;
@@ -658,6 +657,7 @@ int spmm_get_info(spmm_handle_t h, int64_t N, spmm_info_t* info) {
         info->n_split = f.n_split;
         info->n_slots = f.n_slots;
         info->split_cols = f.T;
+        info->n_bins = static_cast<int32_t>(f.bin_ptr.size()) - 1;
         info->distinct_b_rows = f.distinct_cols;
         info->bytes_a = static_cast<double>(info->stored_values) * s;
         info->bytes_idx = static_cast<double>(f.nwin + 1 + f.P) * 4.0;

@@ -29,30 +29,37 @@ int bcsr_token_groups_max(int b);
 constexpr int bcsr_blocks_per_stage(int b) { return b == 16 ? 4 : (b == 32 ? 2 : 1); }
 
 // WCSR pipeline shape, shared by the host schedule (fills are cut to the stage size) and the
-// kernel: columns per shared-memory stage, ring depth and producer warps for the one-group
-// (N <= 128, two CTAs per SM) and two-group (N > 128, one CTA per SM) variants.
+// kernel.  A stage holds 128 / es columns (64 of a 2-byte type, 32 of TF32) of one 128-token
+// tile: 16 KB of gathered B rows + 2 KB of A.  Per value size: ring depth, producer warps
+// (each owns STAGES / PW stages) and resident CTAs per SM, which is also the number of bins
+// per SM of the static schedule (every resident CTA walks one bin).  Measured on B200:
+// 2-byte types run fastest as three small CTAs per SM (4 stages, 4 producer warps), TF32 as
+// two deeper ones (6 stages, 6 producer warps); both fill the SM's shared memory.
 #ifndef WCSR_STAGE_ROW_BYTES
 #define WCSR_STAGE_ROW_BYTES 128
 #endif
-#ifndef WCSR_STAGES1
-#define WCSR_STAGES1 6
+#ifndef WCSR_STAGES_16
+#define WCSR_STAGES_16 4
 #endif
-#ifndef WCSR_STAGES2
-#define WCSR_STAGES2 6
+#ifndef WCSR_PW_16
+#define WCSR_PW_16 4
 #endif
-#ifndef WCSR_PW1
-#define WCSR_PW1 6
+#ifndef WCSR_BINS_16
+#define WCSR_BINS_16 3
 #endif
-#ifndef WCSR_PW2
-#define WCSR_PW2 6
+#ifndef WCSR_STAGES_32
+#define WCSR_STAGES_32 6
 #endif
-// bins per SM of the static WCSR schedule = the largest CTAs-per-SM count of the kernel
-// variants: every resident CTA gets one bin (two when a variant fits one CTA per SM).  More,
-// smaller bins measured slower: each bin start pays a chain of cold index loads.
-constexpr int kWcsrBinsPerSm = 2;
+#ifndef WCSR_PW_32
+#define WCSR_PW_32 6
+#endif
+#ifndef WCSR_BINS_32
+#define WCSR_BINS_32 2
+#endif
 constexpr int wcsr_stage_cols(int es) { return WCSR_STAGE_ROW_BYTES / es; }
-constexpr int kWcsrStages1 = WCSR_STAGES1, kWcsrStages2 = WCSR_STAGES2;
-constexpr int kWcsrProducerWarps1 = WCSR_PW1, kWcsrProducerWarps2 = WCSR_PW2;
+constexpr int wcsr_stages(int es) { return es == 4 ? WCSR_STAGES_32 : WCSR_STAGES_16; }
+constexpr int wcsr_producer_warps(int es) { return es == 4 ? WCSR_PW_32 : WCSR_PW_16; }
+constexpr int wcsr_bins_per_sm(int es) { return es == 4 ? WCSR_BINS_32 : WCSR_BINS_16; }
 
 // Device task descriptor of the WCSR kernel (one per sub-task of the split plan).
 struct WcsrDevTask {
@@ -82,7 +89,7 @@ struct WcsrParams {
 
 // dtype: 0 bf16, 1 fp16, 2 tf32.  groups: 1 or 2.  tmB: 2-D map of B (k rows x N), box = 128
 // bytes x 1 row, 128-byte swizzle (32-byte atoms for tf32), used in row-gather mode.
-cudaError_t launch_wcsr(int dtype, int groups, const CUtensorMap& tmB, const WcsrParams& p, int sms,
+cudaError_t launch_wcsr(int dtype, const CUtensorMap& tmB, const WcsrParams& p, int sms,
                         cudaStream_t stream);
 
 struct MergeParams {

@@ -1,21 +1,21 @@
 // WCSR SpMM kernel for sm_100a (Sec. 3.2 - 3.3 of the paper, re-designed for Blackwell).
 //
 // Work item: one sub-task of the split plan (a run of `count` condensed columns of one
-// 16-row window) times BN_T = 128 * GROUPS columns of B ("tokens").  It accumulates
+// 16-row window) times one tile of 128 columns of B ("tokens"; wider B: one pass per tile).  It accumulates
 //     D[n, r] += sum_q  B[window_col_idx[q], n0 + n] * values[r, q]
 // with the tokens on the 128 TMEM lanes (MMA M side; the gathered B rows are written to
 // shared memory in the MN-major 128-byte-swizzled layout tcgen05.mma reads) and the 16
 // window rows as the MMA N side (operand = the packed window tile, K-major, un-swizzled).
 //
-// Roles ((PW + 5) warps, persistent CTAs; PW producer warps):
-//   warps 0-3   gather producers: warp w owns the CTA's fills w, w + 4, ...; per fill every
-//               lane reads four column indices and issues one TMA row-gather (four B rows x
-//               128 bytes, hardware swizzle, zero fill for -1 pads) into a STAGES-deep ring;
-//               lane 0 also bulk-copies the contiguous packed A tile.  Completion is counted
-//               in bytes on the stage's mbarrier, so producers never wait for data.
-//   warp 4      MMA issuer (one thread): count / b_col tcgen05.mma per group and stage.
-//   warps 5-8   epilogue: tcgen05.ld, release the TMEM buffer, store to C (unsplit window)
-//               or to the task's partial tile (split window).
+// Roles (PW + 5 warps, persistent CTAs, two or three resident per SM):
+//   warps 0..PW-1     gather producers: warp w owns the CTA's fills w, w + PW, ...; per fill
+//               every lane reads four column indices and issues one TMA row-gather (four B
+//               rows x 128 bytes, hardware swizzle, zero fill for -1 pads) into a STAGES-deep
+//               ring; lane 0 also bulk-copies the contiguous packed A tile.  Completion is
+//               counted in bytes on the stage's mbarrier, so producers never wait for data.
+//   warp PW           MMA issuer (one elected lane): count / b_col tcgen05.mma per stage.
+//   warps PW+1..PW+4  epilogue: tcgen05.ld, release the TMEM buffer, store to C (unsplit
+//               window) or to the task's partial tile (split window).
 // Tasks are dealt to bins by the longest-processing-time rule at creation; CTA c walks bins
 // c, c + grid, ...; inside a bin tasks ascend, so all CTAs sweep the matrix top to bottom
 // together and neighbouring windows (which share B rows in banded matrices) meet in L2.
@@ -36,25 +36,25 @@ constexpr int kWH = 16;
 // epilogue adds (in index order).
 constexpr int kNSub = 4;
 
-template <int ES, int GROUPS, int KT, int STAGES>
+template <int ES, int KT, int STAGES>
 struct WcsrCfg {
     static constexpr int kKStep = 32 / ES;                  // columns per MMA (= b_col)
-    static constexpr int kBnT = 128 * GROUPS;
+    static constexpr int kBnT = 128;                        // tokens per tile = TMEM lanes
     static constexpr int kRowBytes = kBnT * ES;
     static constexpr int kSegs = kRowBytes / 128;           // 128-byte segments per gathered row
     static constexpr int kGathers = (KT / 4) * kSegs;       // row-gather instructions per full fill
     static constexpr int kRounds = (kGathers + 31) / 32;    // per lane
     static constexpr int kAtomStride = KT * 128;            // bytes between MN atoms
-    static constexpr int kAtomsPerGroup = ES;               // 128 tokens * ES / 128 B
     static constexpr int kDenseBytes = KT * kRowBytes;
     static constexpr int kABytes = (KT / kKStep) * (kWH * 32);
     static constexpr int kStageBytes = kDenseBytes + kABytes;
-    // CTAs that fit one SM by shared memory (1 KB per CTA is reserved), at most kWcsrBinsPerSm
-    static constexpr int kCtasBySmem = (227 * 1024) / (STAGES * kStageBytes + 1024 + 256 + 1024);
-    static constexpr int kCtasPerSm = kCtasBySmem < 1 ? 1 : (kCtasBySmem > kWcsrBinsPerSm ? kWcsrBinsPerSm : kCtasBySmem);
-    // items with live accumulators: the SM's 512 TMEM columns are shared by its resident CTAs
-    static constexpr int kNAcc = (512 / kCtasPerSm) / (GROUPS * kNSub * kWH) >= 4 ? 4 : 2;
-    static constexpr int kAccCols = GROUPS * kNSub * kWH;   // TMEM columns of one item
+    // resident CTAs per SM = bins per SM of the schedule; they must fit the SM's shared memory
+    // (1 KB per CTA is reserved by the system) and share its 512 TMEM columns
+    static constexpr int kCtasPerSm = wcsr_bins_per_sm(ES);
+    static_assert(kCtasPerSm * (STAGES * kStageBytes + 1024 + 256 + 1024) <= 227 * 1024, "shared memory over-subscribed");
+    // items with live accumulators
+    static constexpr int kNAcc = (512 / kCtasPerSm) / (kNSub * kWH) >= 4 ? 4 : 2;
+    static constexpr int kAccCols = kNSub * kWH;            // TMEM columns of one item
     static constexpr int kTmemCols = kNAcc * kAccCols;      // 128 or 256
     static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 + 256;
     static_assert(KT % 8 == 0 && KT % kKStep == 0 && KT <= 128, "stage shape");
@@ -80,10 +80,10 @@ struct SegIter {
     }
 };
 
-template <int ES, int FMT, int GROUPS, int KT, int STAGES, int PW>
-__global__ void __launch_bounds__((PW + 5) * 32, WcsrCfg<ES, GROUPS, KT, STAGES>::kCtasPerSm)
+template <int ES, int FMT, int KT, int STAGES, int PW>
+__global__ void __launch_bounds__((PW + 5) * 32, WcsrCfg<ES, KT, STAGES>::kCtasPerSm)
 wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
-    using Cfg = WcsrCfg<ES, GROUPS, KT, STAGES>;
+    using Cfg = WcsrCfg<ES, KT, STAGES>;
     constexpr int kProducerWarps = PW;          // warps 0 .. PW-1; MMA warp PW; epilogue PW+1 .. PW+4
     constexpr int kMmaWarp = PW;
     // Fill i goes to stage i % STAGES and is produced by warp i % PW.  With STAGES a multiple
@@ -262,9 +262,6 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
         bool ok = true;
         while (ok && seg.next(p)) {
             const int f0 = __ldg(p.bin_fill + seg.b), f1 = __ldg(p.bin_fill + seg.b + 1);
-            const int n0 = seg.tt * Cfg::kBnT;
-            const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
-            const int ngrp = (nvalid + 127) >> 7;
             int2 win = (f0 + lane < f1) ? __ldg(p.fills + f0 + lane) : kNoDesc;
             for (int wbase = f0; wbase < f1 && ok; wbase += 32) {
                 const int2 nwin = (wbase + 32 + lane < f1) ? __ldg(p.fills + wbase + 32 + lane) : kNoDesc;
@@ -301,12 +298,9 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                         auto issue = [&](int ks, uint32_t kk) {
                             const uint32_t dsub = d0 + (kk & (kNSub - 1)) * kWH;
                             const uint32_t accum = kk >= kNSub ? 1u : 0u;    // first use overwrites
-#pragma unroll
-                            for (int g = 0; g < GROUPS; ++g)
-                                if (leader && g < ngrp)
-                                    umma_ss<FMT == 2>(dsub + g * kNSub * kWH,
-                                                      a0 + ((g * Cfg::kAtomsPerGroup * Cfg::kAtomStride + ks * (Cfg::kKStep / 8) * 1024) >> 4),
-                                                      b0 + ((ks * (kWH * 32)) >> 4), idesc, accum);
+                            if (leader)
+                                umma_ss<FMT == 2>(dsub, a0 + ((ks * (Cfg::kKStep / 8) * 1024) >> 4),
+                                                  b0 + ((ks * (kWH * 32)) >> 4), idesc, accum);
                         };
                         constexpr int kFullSteps = KT / Cfg::kKStep;
                         if (nks == kFullSteps) {                 // a full stage: straight-line code
@@ -377,33 +371,29 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     if (!__all_sync(0xffffffffu, mbar_wait(accf_bar(acc), aph, ctl, 14))) { ok = false; break; }
                     TRACE_ADD(tr_accf, tr_a);
                     tc_fence_after_sync();
-                    float v[GROUPS][16];
+                    float v[kWH];
                     const uint32_t tbase = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + acc * Cfg::kAccCols;
-#pragma unroll
-                    for (int g = 0; g < GROUPS; ++g) {
+                    {
                         uint32_t u[16];
-                        tmem_ld_x16(tbase + (g * kNSub) * kWH, u);
+                        tmem_ld_x16(tbase, u);
                         tmem_ld_wait();
 #pragma unroll
-                        for (int jr = 0; jr < kWH; ++jr) v[g][jr] = __uint_as_float(u[jr]);
+                        for (int jr = 0; jr < kWH; ++jr) v[jr] = __uint_as_float(u[jr]);
                         for (int sub = 1; sub < nsub; ++sub) {
-                            tmem_ld_x16(tbase + (g * kNSub + sub) * kWH, u);
+                            tmem_ld_x16(tbase + sub * kWH, u);
                             tmem_ld_wait();
 #pragma unroll
-                            for (int jr = 0; jr < kWH; ++jr) v[g][jr] += __uint_as_float(u[jr]);
+                            for (int jr = 0; jr < kWH; ++jr) v[jr] += __uint_as_float(u[jr]);
                         }
                     }
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(acce_bar(acc));
+                    const int n = n0 + qd * 32 + lane;
+                    if (n < N) {
 #pragma unroll
-                    for (int g = 0; g < GROUPS; ++g) {
-                        const int n = n0 + g * 128 + qd * 32 + lane;
-                        if (n < N) {
-#pragma unroll
-                            for (int jr = 0; jr < kWH; ++jr)
-                                if (jr < rows) out[static_cast<int64_t>(jr) * N + n] = v[g][jr];
-                        }
+                        for (int jr = 0; jr < kWH; ++jr)
+                            if (jr < rows) out[static_cast<int64_t>(jr) * N + n] = v[jr];
                     }
                 }
                 win = nwin;
@@ -466,18 +456,19 @@ wcsr_merge_kernel(const MergeParams p) {
     }
 }
 
-template <int ES, int FMT, int GROUPS, int KT, int STAGES, int PW>
+template <int ES, int FMT>
 cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
-    using Cfg = WcsrCfg<ES, GROUPS, KT, STAGES>;
-    auto kfn = wcsr_spmm_kernel<ES, FMT, GROUPS, KT, STAGES, PW>;
+    constexpr int KT = wcsr_stage_cols(ES), STAGES = wcsr_stages(ES), PW = wcsr_producer_warps(ES);
+    using Cfg = WcsrCfg<ES, KT, STAGES>;
+    auto kfn = wcsr_spmm_kernel<ES, FMT, KT, STAGES, PW>;
     static int occ = 0;
     if (occ == 0) {
         cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(kfn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
-        // resident CTAs per SM: by shared memory and TMEM columns (see WcsrCfg); the register
-        // file follows from __launch_bounds__
+        // resident CTAs per SM: shared memory and TMEM columns are checked in WcsrCfg; the
+        // register file follows from __launch_bounds__
         static_assert(Cfg::kCtasPerSm * Cfg::kTmemCols <= 512, "TMEM over-subscribed");
         occ = Cfg::kCtasPerSm;
     }
@@ -490,19 +481,10 @@ cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cud
 
 }  // namespace
 
-cudaError_t launch_wcsr(int dtype, int groups, const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
-    constexpr int K2 = wcsr_stage_cols(2), K4 = wcsr_stage_cols(4);
-    constexpr int S1 = kWcsrStages1, S2 = kWcsrStages2, P1 = kWcsrProducerWarps1, P2 = kWcsrProducerWarps2;
-    if (dtype == 2) {
-        if (groups == 1) return launch_one<4, 2, 1, K4, S1, P1>(tmB, p, sms, stream);
-        if (groups == 2) return launch_one<4, 2, 2, K4, S2, P2>(tmB, p, sms, stream);
-    } else if (dtype == 1) {
-        if (groups == 1) return launch_one<2, 0, 1, K2, S1, P1>(tmB, p, sms, stream);
-        if (groups == 2) return launch_one<2, 0, 2, K2, S2, P2>(tmB, p, sms, stream);
-    } else if (dtype == 0) {
-        if (groups == 1) return launch_one<2, 1, 1, K2, S1, P1>(tmB, p, sms, stream);
-        if (groups == 2) return launch_one<2, 1, 2, K2, S2, P2>(tmB, p, sms, stream);
-    }
+cudaError_t launch_wcsr(int dtype, const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
+    if (dtype == 2) return launch_one<4, 2>(tmB, p, sms, stream);
+    if (dtype == 1) return launch_one<2, 0>(tmB, p, sms, stream);
+    if (dtype == 0) return launch_one<2, 1>(tmB, p, sms, stream);
     return cudaErrorInvalidValue;
 }
 

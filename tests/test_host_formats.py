@@ -143,15 +143,17 @@ def test_wcsr_format_plan_and_bins_are_bit_exact(lib, dtype, m, k, dens, T):
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_TASKS, np.int32).reshape(-1, 4), plan)
         bin_ptr = lib.spmm_export(h, lib.X_WCSR_BIN_PTR, np.int32)
         bin_tasks = lib.spmm_export(h, lib.X_WCSR_BIN_TASKS, np.int32)
-        want_ptr, want_tasks = F.task_bins(plan, 5 * 2)
+        info = lib.spmm_get_info(h, 128)
+        n_bins = info["n_bins"]
+        assert n_bins == 5 * (2 if dtype == "tf32" else 3)     # one bin per resident CTA
+        want_ptr, want_tasks = F.task_bins(plan, n_bins)
         assert np.array_equal(bin_ptr, want_ptr) and np.array_equal(bin_tasks, want_tasks)
         assert sorted(bin_tasks.tolist()) == list(range(plan.shape[0]))      # every task exactly once
         cost = plan[:, 2].astype(np.int64) + 32
-        loads = np.array([cost[bin_tasks[bin_ptr[j]:bin_ptr[j + 1]]].sum() for j in range(10)])
+        loads = np.array([cost[bin_tasks[bin_ptr[j]:bin_ptr[j + 1]]].sum() for j in range(n_bins)])
         assert loads.max() - loads.min() <= cost.max()                       # LPT balance property
-        for j in range(10):
+        for j in range(n_bins):
             assert np.all(np.diff(bin_tasks[bin_ptr[j]:bin_ptr[j + 1]]) > 0)
-        info = lib.spmm_get_info(h, 128)
         P = f["window_col_idx"].shape[0]
         assert info["n_units"] == P and info["stored_values"] == 16 * P
         assert info["n_tasks"] == plan.shape[0]
@@ -169,7 +171,7 @@ def test_default_split_size(lib):
     a = wl.wcsr_irregular(seed=4, m=30000, dtype="fp16")
     h = lib.spmm_wcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "fp16", 16, host_only=True, n_ctas=3)
     info = lib.spmm_get_info(h)
-    assert info["split_cols"] == F.default_split_cols(info["n_units"], 6)
+    assert info["n_bins"] == 9 and info["split_cols"] == F.default_split_cols(info["n_units"], 9)
     assert 128 <= info["split_cols"] <= 4096 and info["split_cols"] % 64 == 0
     lib.spmm_destroy(h)
     assert F.default_split_cols(100, 8) == 128 and F.default_split_cols(10 ** 9, 8) == 4096
