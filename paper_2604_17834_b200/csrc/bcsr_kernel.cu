@@ -9,8 +9,10 @@
 // writes C rows with fully coalesced 128-byte warp stores.
 //
 // Roles (192 threads, one CTA per SM, persistent):
-//   warp 0      TMA producer: per stored block one A-block load plus 2*GROUPS B boxes into a
-//               STAGES-deep shared-memory ring, full/empty mbarriers with phase bits.
+//   warp 0      TMA producer: per pipeline stage (1, 2 or 4 stored blocks) one request for
+//               the A blocks and one 3-D request per block for its B tile (2*GROUPS boxes of
+//               b x 64 tokens), issued by different lanes of one warp-instruction, into a
+//               STAGES-deep shared-memory ring; full/empty mbarriers with phase bits.
 //   warp 1      MMA issuer: one thread issues tcgen05.mma into one of two TMEM accumulator
 //               buffers; tcgen05.commit frees the ring slot / publishes the accumulator.
 //   warps 2-5   epilogue: tcgen05.ld -> registers -> global C (zeros for empty block-rows),
