@@ -57,6 +57,24 @@ typedef enum {
     SPMM_TF32 = 2                /* 4-byte fp32 storage, TF32 tensor-core arithmetic          */
 } spmm_dtype_t;
 
+/* Element type of C (opts.c_type).  Accumulation is fp32 either way. */
+typedef enum {
+    SPMM_C_FP32 = 0,             /* fp32 (default; the type the paper's kernels write)        */
+    SPMM_C_SAME_AS_INPUT = 1     /* bf16 / fp16 handles: C in that type, rounded to nearest
+                                    even from the fp32 accumulator.  TF32 handles: fp32.      */
+} spmm_ctype_t;
+
+/* Operand layout (opts.layout), BCSR only. */
+typedef enum {
+    SPMM_ROWMAJOR = 0,           /* B is k x N, C is m x N, both row-major (default)          */
+    SPMM_COLMAJOR = 1            /* B and C column-major, i.e. the caller holds X = B^T as a
+                                    row-major N x k array and receives Y = C^T as a row-major
+                                    N x m array: the layout of the paper's BCSR kernel
+                                    (Sec. 3.2) and of a linear layer Y = X W^T with a sparse
+                                    weight W = A (Sec. 4.3).  Needs m % 8 == 0, k % 8 == 0 and
+                                    N >= 128; N itself is unconstrained.                      */
+} spmm_layout_t;
+
 /* Optional creation parameters; pass NULL for all defaults.  Zero = default. */
 typedef struct {
     int32_t b_col;       /* WCSR: pad every window to a multiple of this many columns.
@@ -70,7 +88,9 @@ typedef struct {
                             handle serves spmm_export / spmm_get_info, spmm_run fails.       */
     int32_t n_ctas;      /* persistent grid size the schedule is built for; default = the
                             device's SM count (148 when host_only).                          */
-    int32_t reserved[12];
+    int32_t c_type;      /* spmm_ctype_t                                                      */
+    int32_t layout;      /* spmm_layout_t; SPMM_COLMAJOR with a WCSR handle is UNSUPPORTED    */
+    int32_t reserved[10];
 } spmm_opts_t;
 
 typedef struct {
@@ -171,8 +191,11 @@ int spmm_bcsr_plan(spmm_handle_t h, int64_t N);
  * C = A x B (Sec. 2.3; kernels of Sec. 3).  Asynchronous on `stream` (a cudaStream_t passed
  * as void*; NULL = the default stream); never synchronises.
  *   B_dev  device, k x N row-major, elements of the handle's dtype, 16-byte aligned.
- *   C_dev  device, m x N row-major fp32, 16-byte aligned; every element is written.
+ *   C_dev  device, m x N row-major, fp32 (or the handle's 16-bit type with
+ *          SPMM_C_SAME_AS_INPUT), 16-byte aligned; every element is written.
  *   N      dense width; N * element size must be a multiple of 16 bytes.
+ * With SPMM_COLMAJOR (BCSR): B_dev is X, N x k row-major, and C_dev is Y, N x m row-major,
+ * Y[n][i] = sum_j A[i][j] * X[n][j]; any N >= 128.
  * WCSR keeps the partial tiles of split windows in a device workspace owned by the handle;
  * it is (re)allocated here the first time a given N needs more than it holds, so two runs
  * of one handle must not overlap on the GPU, and the first run at a new N may synchronise.
@@ -206,7 +229,8 @@ int spmm_wcsr_run_static(spmm_handle_t h, const void *B_dev, void *C_dev, int64_
 /*
  * Same result as spmm_run, for callers that hold HOST buffers: copies B to the device,
  * runs, copies C back and synchronises `stream` before returning.  B_host / C_host are
- * ordinary or pinned host memory of k*N elements / m*N floats; the device staging buffers
+ * ordinary or pinned host memory of k*N elements / m*N elements of C's type, in the
+ * handle's layout; the device staging buffers
  * belong to the handle and are reused between calls.
  */
 int spmm_run_host(spmm_handle_t h, const void *B_host, void *C_host, int64_t N, void *stream);

@@ -73,6 +73,9 @@ struct spmm_handle_s {
     int es = 2;
     int64_t m = 0, k = 0, nnz = 0;
     bool host_only = false;
+    bool c16 = false;        // C in the input's 16-bit type (never with TF32, whose input type is fp32)
+    bool col_major = false;  // BCSR: B given as X[N][k], C as Y[N][m]
+    int cs = 4;              // bytes per C element
     int n_ctas = 148;
     int sms = 148;
     int device = 0;
@@ -163,8 +166,16 @@ int device_setup(spmm_handle_s* h, const spmm_opts_t* opts) {
     return SPMM_OK;
 }
 
+int check_opts(const spmm_opts_t* opts) {
+    if (!opts) return SPMM_OK;
+    if (opts->c_type != SPMM_C_FP32 && opts->c_type != SPMM_C_SAME_AS_INPUT) return SPMM_ERR_INVALID_ARG;
+    if (opts->layout != SPMM_ROWMAJOR && opts->layout != SPMM_COLMAJOR) return SPMM_ERR_INVALID_ARG;
+    return SPMM_OK;
+}
+
 int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, const spmm_opts_t* opts) {
     if (dtype != SPMM_BF16 && dtype != SPMM_FP16) return SPMM_ERR_UNSUPPORTED;
+    if (int orc = check_opts(opts)) return orc;
     int rc = validate_csr(a);
     if (rc) return rc;
     spmm_handle_s* h = new (std::nothrow) spmm_handle_s;
@@ -176,6 +187,12 @@ int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, cons
     h->k = a.k;
     h->nnz = a.nnz;
     h->host_only = opts && opts->host_only;
+    h->c16 = opts && opts->c_type == SPMM_C_SAME_AS_INPUT;
+    h->cs = h->c16 ? 2 : 4;
+    h->col_major = opts && opts->layout == SPMM_COLMAJOR;
+    // column-major operands: rows of X (k elements) and of Y (m elements) must be multiples of
+    // 16 bytes for the tensor map and for the 16-byte pieces the epilogue writes
+    if (h->col_major && (a.m % 8 != 0 || a.k % 8 != 0)) { delete h; return SPMM_ERR_UNSUPPORTED; }
     rc = device_setup(h, opts);
     if (rc) { free_handle(h); return rc; }
     try {
@@ -208,6 +225,8 @@ int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, cons
 
 int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const spmm_opts_t* opts) {
     if (dtype != SPMM_BF16 && dtype != SPMM_FP16 && dtype != SPMM_TF32) return SPMM_ERR_UNSUPPORTED;
+    if (int orc = check_opts(opts)) return orc;
+    if (opts && opts->layout == SPMM_COLMAJOR) return SPMM_ERR_UNSUPPORTED;   // BCSR only
     int rc = validate_csr(a);
     if (rc) return rc;
     const int b_col_default = 32 / a.es;
@@ -224,6 +243,8 @@ int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const s
     h->k = a.k;
     h->nnz = a.nnz;
     h->host_only = opts && opts->host_only;
+    h->c16 = opts && opts->c_type == SPMM_C_SAME_AS_INPUT && dtype != SPMM_TF32;
+    h->cs = h->c16 ? 2 : 4;
     rc = device_setup(h, opts);
     if (rc) { free_handle(h); return rc; }
     try {
@@ -312,6 +333,28 @@ int ensure_tmB(spmm_handle_s* h, const void* B, int64_t N, int groups) {
     int rc;
     if (h->format == 1) {
         rc = encode_gather_map(&h->tmB, h->dtype, B, static_cast<uint64_t>(h->k), static_cast<uint64_t>(N));
+    } else if (h->col_major) {
+        // X as [N][k]: box = 128 tokens x min(b, 64) elements, swizzle = the box's row bytes;
+        // and the same memory as [N / 128][128][k] so that one request brings all token groups
+        // of a tile (whole groups only; a ragged last tile uses the 2-D map, zero filled)
+        const uint32_t bw = h->bcsr.b < 64 ? h->bcsr.b : 64;
+        const CUtensorMapSwizzle swz = bw == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                      : (bw == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+        rc = encode_2d_16bit(&h->tmB, h->dtype, B, static_cast<uint64_t>(N), static_cast<uint64_t>(h->k), 128, bw, swz);
+        h->tmB3_ok = false;
+        h->tmB3 = h->tmB;
+        EncodeTiledFn fn = get_encode_fn();
+        if (!rc && fn && N >= 128) {
+            const cuuint64_t dims[3] = {static_cast<cuuint64_t>(h->k), 128, static_cast<cuuint64_t>(N / 128)};
+            const cuuint64_t strides[2] = {static_cast<cuuint64_t>(h->k) * 2, static_cast<cuuint64_t>(h->k) * 256};
+            const cuuint32_t box[3] = {bw, 128, static_cast<cuuint32_t>(groups)};
+            const cuuint32_t estr[3] = {1, 1, 1};
+            const CUtensorMapDataType dt = h->dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+            CUresult r = fn(&h->tmB3, dt, 3, const_cast<void*>(B), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            h->tmB3_ok = r == CUDA_SUCCESS;
+            if (!h->tmB3_ok) h->tmB3 = h->tmB;
+        }
     } else {
         rc = encode_2d_16bit(&h->tmB, h->dtype, B, static_cast<uint64_t>(h->k), static_cast<uint64_t>(N),
                              static_cast<uint32_t>(h->bcsr.b), 64, CU_TENSOR_MAP_SWIZZLE_128B);
@@ -388,9 +431,9 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
     return SPMM_OK;
 }
 
-int run_bcsr(spmm_handle_s* h, const void* B, float* C, int64_t N, cudaStream_t stream) {
+int run_bcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t stream) {
     const BcsrHost& f = h->bcsr;
-    if (N < 64) return SPMM_ERR_UNSUPPORTED;   // the B box is 64 tokens wide
+    if (N < (h->col_major ? 128 : 64)) return SPMM_ERR_UNSUPPORTED;   // the box is 64 (128) tokens wide
     if (f.nbr == 0) return SPMM_OK;
     int rc = ensure_schedule(h, N);
     if (rc) return rc;
@@ -417,7 +460,7 @@ int run_bcsr(spmm_handle_s* h, const void* B, float* C, int64_t N, cudaStream_t 
     rc = ensure_tmB(h, B, N, h->sched.groups);
     if (rc) return rc;
     p.use_3d = h->tmB3_ok ? 1 : 0;
-    cudaError_t e = launch_bcsr(h->dtype, f.b, h->sched.groups, tmA, h->tmB, h->tmB3, p, h->n_ctas, stream);
+    cudaError_t e = launch_bcsr(h->dtype, f.b, h->sched.groups, h->c16, h->col_major, tmA, h->tmB, h->tmB3, p, h->n_ctas, stream);
     return e == cudaSuccess ? SPMM_OK : SPMM_ERR_CUDA;
 }
 
@@ -425,7 +468,7 @@ int64_t wcsr_workspace_bytes(const spmm_handle_s* h, int64_t N) {
     return h->wcsr.n_slots * int64_t{16} * N * 4;
 }
 
-int launch_wcsr_all(spmm_handle_s* h, const void* B, float* C, float* partial, int64_t N, cudaStream_t stream) {
+int launch_wcsr_all(spmm_handle_s* h, const void* B, void* C, float* partial, int64_t N, cudaStream_t stream) {
     const WcsrHost& f = h->wcsr;
     const int bnt = 128;                    // tokens per tile; wider B takes one pass per tile
     WcsrParams p;
@@ -451,7 +494,7 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, float* C, float* partial, i
     if (!f.tasks.empty()) {
         int rc = ensure_tmB(h, B, N, 1);
         if (rc) return rc;
-        cudaError_t e = launch_wcsr(h->dtype, h->tmB, p, h->sms, stream);
+        cudaError_t e = launch_wcsr(h->dtype, h->c16, h->tmB, p, h->sms, stream);
         if (e != cudaSuccess) return SPMM_ERR_CUDA;
     }
     MergeParams mp;
@@ -463,11 +506,11 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, float* C, float* partial, i
     mp.m = h->m;
     mp.N = N;
     mp.n = h->n_merge;
-    cudaError_t e = launch_wcsr_merge(mp, stream);
+    cudaError_t e = launch_wcsr_merge(mp, h->c16 ? (h->dtype == SPMM_FP16 ? 1 : 2) : 0, stream);
     return e == cudaSuccess ? SPMM_OK : SPMM_ERR_CUDA;
 }
 
-int run_wcsr(spmm_handle_s* h, const void* B, float* C, int64_t N, cudaStream_t stream) {
+int run_wcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t stream) {
     const size_t need = static_cast<size_t>(wcsr_workspace_bytes(h, N));
     if (need > h->partial_bytes) {
         if (h->d_partial) {
@@ -485,7 +528,9 @@ int run_wcsr(spmm_handle_s* h, const void* B, float* C, int64_t N, cudaStream_t 
 int check_run_args(spmm_handle_s* h, const void* B, const void* C, int64_t N) {
     if (!h || !B || !C || N <= 0) return SPMM_ERR_INVALID_ARG;
     if (h->host_only) return SPMM_ERR_HOST_ONLY;
-    if ((N * h->es) % 16 != 0) return SPMM_ERR_UNSUPPORTED;
+    // row-major B and C have N elements per row: rows must stay 16-byte aligned (column-major
+    // operands have k and m elements per row, checked at creation)
+    if (!h->col_major && (N * h->es) % 16 != 0) return SPMM_ERR_UNSUPPORTED;
     if ((reinterpret_cast<uintptr_t>(B) & 15) || (reinterpret_cast<uintptr_t>(C) & 15)) return SPMM_ERR_UNSUPPORTED;
     if (N >= (int64_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
     return SPMM_OK;
@@ -555,14 +600,14 @@ int spmm_run(spmm_handle_t h, const void* B_dev, void* C_dev, int64_t N, void* s
     int rc = check_run_args(h, B_dev, C_dev, N);
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (h->format == 0) return run_bcsr(h, B_dev, static_cast<float*>(C_dev), N, st);
-    return run_wcsr(h, B_dev, static_cast<float*>(C_dev), N, st);
+    if (h->format == 0) return run_bcsr(h, B_dev, C_dev, N, st);
+    return run_wcsr(h, B_dev, C_dev, N, st);
 }
 
 int spmm_bcsr_plan(spmm_handle_t h, int64_t N) {
     if (!h || N <= 0) return SPMM_ERR_INVALID_ARG;
     if (h->format != 0) return SPMM_ERR_INVALID_ARG;
-    if (N < 64 || (N * h->es) % 16 != 0) return SPMM_ERR_UNSUPPORTED;
+    if (N < (h->col_major ? 128 : 64) || (!h->col_major && (N * h->es) % 16 != 0)) return SPMM_ERR_UNSUPPORTED;
     return ensure_schedule(h, N);
 }
 
@@ -574,7 +619,7 @@ int spmm_wcsr_run_static(spmm_handle_t h, const void* B_dev, void* C_dev, int64_
     size_t cap = 0;
     if (wcsr_static_scratch(&scratch, &cap) != cudaSuccess) return SPMM_ERR_CUDA;
     if (static_cast<size_t>(wcsr_workspace_bytes(h, N)) > cap) return SPMM_ERR_TOO_LARGE;
-    return launch_wcsr_all(h, B_dev, static_cast<float*>(C_dev), scratch, N, static_cast<cudaStream_t>(stream));
+    return launch_wcsr_all(h, B_dev, C_dev, scratch, N, static_cast<cudaStream_t>(stream));
 }
 
 int spmm_run_host(spmm_handle_t h, const void* B_host, void* C_host, int64_t N, void* stream) {
@@ -582,7 +627,7 @@ int spmm_run_host(spmm_handle_t h, const void* B_host, void* C_host, int64_t N, 
     if (h->host_only) return SPMM_ERR_HOST_ONLY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t bbytes = static_cast<size_t>(h->k) * N * h->es;
-    const size_t cbytes = static_cast<size_t>(h->m) * N * 4;
+    const size_t cbytes = static_cast<size_t>(h->m) * N * h->cs;
     if (bbytes > h->Bstage_bytes) {
         cudaFree(h->d_Bstage);
         h->d_Bstage = nullptr;
@@ -666,7 +711,7 @@ int spmm_get_info(spmm_handle_t h, int64_t N, spmm_info_t* info) {
     }
     info->fill_ratio = info->stored_values ? static_cast<double>(h->nnz) / static_cast<double>(info->stored_values) : 0.0;
     info->bytes_b_touched = static_cast<double>(info->distinct_b_rows) * n * s;
-    info->bytes_c = static_cast<double>(h->m) * n * 4.0;
+    info->bytes_c = static_cast<double>(h->m) * n * h->cs;
     info->flops_stored = 2.0 * static_cast<double>(info->stored_values) * n;
     return SPMM_OK;
 }

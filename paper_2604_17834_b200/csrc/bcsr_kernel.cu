@@ -18,6 +18,14 @@
 //   warps 2-5   epilogue: tcgen05.ld -> registers -> global C (zeros for empty block-rows),
 //               overlapping the next tile's MMAs thanks to the second TMEM buffer.  C is
 //               written with streaming stores so that it does not push the B slab out of L2.
+// Two optional variants, both template parameters:
+//   CT = 1   C is written in the input's 16-bit type instead of fp32.
+//   CM = 1   "column-major" operands (the layout of the paper's BCSR kernel, Sec. 3.2, and of a
+//            linear layer Y = X W^T, Sec. 4.3): B is given as X[N][k] (one row per token, k
+//            contiguous) and C as Y[N][m].  The token tile is then a K-major MMA operand
+//            (rows of min(b, 64) elements, swizzle = row bytes; b = 128 as two K halves), and
+//            every epilogue thread owns one token: it writes its b accumulator columns as
+//            contiguous 16-byte pieces of that token's row of Y.
 // The host deals tiles to CTAs ahead of time: slab by slab (a slab = token tiles whose B rows
 // fit in L2), longest block-row first, each tile to the least loaded CTA; CTA c walks its list.
 #include "kernels.h"
@@ -26,6 +34,31 @@
 namespace spmm {
 
 namespace {
+
+// streaming (evict-first) stores of C: one element, or one 16-byte piece of consecutive elements
+template <typename T> __device__ __forceinline__ void store_elem(T* dst, float x) {
+    if constexpr (sizeof(T) == 4) {
+        __stcs(dst, x);
+    } else {
+        const T h = from_f32<T>(x);
+        __stcs(reinterpret_cast<unsigned short*>(dst), *reinterpret_cast<const unsigned short*>(&h));
+    }
+}
+template <typename T> __device__ __forceinline__ void store_piece(T* dst, const uint32_t* v) {
+    if constexpr (sizeof(T) == 4) {
+        __stcs(reinterpret_cast<float4*>(dst), make_float4(__uint_as_float(v[0]), __uint_as_float(v[1]),
+                                                           __uint_as_float(v[2]), __uint_as_float(v[3])));
+    } else {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const T lo = from_f32<T>(__uint_as_float(v[2 * i])), hi = from_f32<T>(__uint_as_float(v[2 * i + 1]));
+            w[i] = static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(&lo)) |
+                   (static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(&hi)) << 16);
+        }
+        __stcs(reinterpret_cast<uint4*>(dst), make_uint4(w[0], w[1], w[2], w[3]));
+    }
+}
 
 template <int B, int GROUPS, int STAGES>
 struct BcsrCfg {
@@ -42,6 +75,9 @@ struct BcsrCfg {
     static constexpr int kAOff = kBps * kDenseBytes;         // A blocks inside the stage
     static constexpr int kARowBytes = (B < 64 ? B : 64) * 2;
     static constexpr uint32_t kASwizzle = kARowBytes == 128 ? SWZ_128B : (kARowBytes == 64 ? SWZ_64B : SWZ_32B);
+    // column-major operands: a token group's tile is 128 rows x kXRowBytes, K-major
+    static constexpr int kXRowBytes = (B < 64 ? B : 64) * 2;
+    static constexpr int kXGroupBytes = 128 * kXRowBytes;    // one K half of one token group
     static constexpr int kAccCols = GROUPS * B;
     static constexpr int kTmemCols = (2 * kAccCols <= 32) ? 32 : (2 * kAccCols <= 64 ? 64 : (2 * kAccCols <= 128 ? 128 : (2 * kAccCols <= 256 ? 256 : 512)));
     static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
@@ -51,7 +87,7 @@ struct BcsrCfg {
     static_assert(kBps == 1 || B <= 32, "multi-block stages are for the small block sizes");
 };
 
-template <int B, int GROUPS, int STAGES, int FMT>
+template <int B, int GROUPS, int STAGES, int FMT, int CT, int CM>
 __global__ void __launch_bounds__(192, 1)
 bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmB3, const BcsrParams p) {
@@ -131,8 +167,29 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         TRACE_ADD(tr_empty, tr_a);
                         const uint32_t sb = smem_base + s * Cfg::kStageBytes;
                         // the A request always brings kBps blocks (the box of the tensor map)
-                        if (lane == 0) mbar_arrive_expect_tx(full_bar(s), Cfg::kBps * Cfg::kABytes + nb * nbox * Cfg::kBoxBytes);
+                        const uint32_t dense_tx = CM ? (whole_tile ? Cfg::kDenseBytes : ((nvalid + 127) >> 7) * (B * 256))
+                                                     : nbox * Cfg::kBoxBytes;
+                        if (lane == 0) mbar_arrive_expect_tx(full_bar(s), Cfg::kBps * Cfg::kABytes + nb * dense_tx);
                         __syncwarp();
+                        if constexpr (CM) {
+                            // X as [N / 128][128][k]: box = GROUPS x 128 tokens x min(b, 64) elements
+                            // of block column J (b = 128: lanes nb.. fetch the second K half)
+                            constexpr int kHalves = B > 64 ? 2 : 1;
+                            const int blk = lane % Cfg::kBps, hf = lane / Cfg::kBps;
+                            const int J = __shfl_sync(0xffffffffu, Jl, jq + (blk < nb ? blk : 0));
+                            if (whole_tile) {
+                                if (blk < nb && hf < kHalves)
+                                    tma_load_3d_hint(sb + blk * Cfg::kDenseBytes + hf * (GROUPS * Cfg::kXGroupBytes), &tmB3,
+                                                     full_bar(s), J * B + hf * 64, 0, n0 >> 7, keep);
+                            } else {
+                                // ragged tile: one request per 128-token group, rows >= N are zero filled
+                                const int ngrp = (nvalid + 127) >> 7;
+                                for (int g = 0; g < ngrp; ++g)
+                                    if (blk < nb && hf < kHalves)
+                                        tma_load_2d_hint(sb + blk * Cfg::kDenseBytes + hf * (GROUPS * Cfg::kXGroupBytes) + g * Cfg::kXGroupBytes,
+                                                         &tmB, full_bar(s), J * B + hf * 64, n0 + g * 128, keep);
+                            }
+                        } else
                         if (whole_tile) {
                             // all 2 * GROUPS boxes of a block with one request: B seen as
                             // [64-token group][k][64 tokens], box = kNBox x b x 64; lane i takes block i
@@ -174,8 +231,9 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // Warp-uniform control flow (all lanes wait and compute the uniform descriptors); one
         // elected lane issues the tcgen05 instructions.
         {
-            constexpr uint32_t idesc = make_idesc(FMT, 128, B, 1, 0);
-            const uint64_t adesc0 = make_smem_desc(0, Cfg::kBoxBytes, 1024, SWZ_128B);
+            constexpr uint32_t idesc = make_idesc(FMT, 128, B, CM ? 0 : 1, 0);
+            const uint64_t adesc0 = CM ? make_smem_desc(0, 16, 8 * Cfg::kXRowBytes, Cfg::kASwizzle)
+                                       : make_smem_desc(0, Cfg::kBoxBytes, 1024, SWZ_128B);
             const uint64_t bdesc0 = make_smem_desc(0, 16, 8 * Cfg::kARowBytes, Cfg::kASwizzle);
             const bool leader = elect_one();
             uint32_t it = 0, tile_i = 0;
@@ -222,7 +280,10 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                                 for (int g = 0; g < GROUPS; ++g)
                                     if (leader && g < ngrp)
-                                        umma_ss<false>(d0 + g * B, a0 + ((g * 2 * Cfg::kBoxBytes + ks * 2048) >> 4),
+                                        umma_ss<false>(d0 + g * B,
+                                                       a0 + ((CM ? (B <= 64 ? g * Cfg::kXGroupBytes + ks * 32
+                                                                            : (ks >> 2) * (GROUPS * Cfg::kXGroupBytes) + g * Cfg::kXGroupBytes + (ks & 3) * 32)
+                                                                 : g * 2 * Cfg::kBoxBytes + ks * 2048) >> 4),
                                                        b0 + (boff >> 4), idesc, ks > 0 ? 1u : accum0);
                             }
                         }
@@ -266,10 +327,14 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             tc_fence_after_sync();
             const int64_t row0 = static_cast<int64_t>(tI) * B;
             const int rows = static_cast<int>(min_i64(B, p.m - row0));
+            using CElem = typename CType<FMT, CT>::type;
+            CElem* const Cb = static_cast<CElem*>(p.C);
             for (int g = 0; g < ngrp; ++g) {
                 const int n = n0 + g * 128 + qd * 32 + lane;
                 const bool nok = n < N;
-                float* cp = p.C + row0 * N + n;
+                // row-major: C[row0 + j][n], one 4- or 2-byte element per lane and row;
+                // column-major: Y[n][row0 + j], this lane's token row
+                CElem* cp = CM ? Cb + static_cast<int64_t>(n) * p.m + row0 : Cb + row0 * N + n;
 #pragma unroll
                 for (int c0 = 0; c0 < B; c0 += 32) {
                     constexpr int W = B < 32 ? B : 32;
@@ -292,9 +357,17 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         for (int j = 0; j < W; ++j) v[j] = 0u;
                     }
                     if (nok) {
+                        if constexpr (CM) {
+                            // rows is a multiple of 8 (m % 8 == 0 is required): whole 16-byte pieces
+                            constexpr int kPer = 16 / static_cast<int>(sizeof(CElem));   // elements per piece
 #pragma unroll
-                        for (int j = 0; j < W; ++j)
-                            if (c0 + j < rows) __stcs(cp + static_cast<int64_t>(c0 + j) * N, __uint_as_float(v[j]));
+                            for (int j = 0; j < W; j += kPer)
+                                if (c0 + j < rows) store_piece<CElem>(cp + c0 + j, v + j);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < W; ++j)
+                                if (c0 + j < rows) store_elem<CElem>(cp + static_cast<int64_t>(c0 + j) * N, __uint_as_float(v[j]));
+                        }
                     }
                 }
             }
@@ -331,11 +404,11 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
 }
 
-template <int B, int GROUPS, int STAGES, int FMT>
+template <int B, int GROUPS, int STAGES, int FMT, int CT, int CM>
 cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3, const BcsrParams& p,
                        int grid, cudaStream_t stream) {
     using Cfg = BcsrCfg<B, GROUPS, STAGES>;
-    auto kfn = bcsr_spmm_kernel<B, GROUPS, STAGES, FMT>;
+    auto kfn = bcsr_spmm_kernel<B, GROUPS, STAGES, FMT, CT, CM>;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
@@ -346,33 +419,42 @@ cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUt
     return cudaGetLastError();
 }
 
-template <int FMT>
-cudaError_t launch_fmt(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
-                       const BcsrParams& p, int grid, cudaStream_t stream) {
+template <int FMT, int CT, int CM>
+cudaError_t launch_shape(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
+                         const BcsrParams& p, int grid, cudaStream_t stream) {
     switch (b * 10 + groups) {
-        case 161: return launch_one<16, 1, 10, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 162: return launch_one<16, 2, 5, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 164: return launch_one<16, 4, 3, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 321: return launch_one<32, 1, 10, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 322: return launch_one<32, 2, 5, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 324: return launch_one<32, 4, 3, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 641: return launch_one<64, 1, 8, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 642: return launch_one<64, 2, 5, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 644: return launch_one<64, 4, 3, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 1281: return launch_one<128, 1, 3, FMT>(tmA, tmB, tmB3, p, grid, stream);
-        case 1282: return launch_one<128, 2, 2, FMT>(tmA, tmB, tmB3, p, grid, stream);
+        case 161: return launch_one<16, 1, 10, FMT, CT, CM>(tmA, tmB, tmB3, p, grid, stream);
+        case 162: return launch_one<16, 2, 5, FMT, CT, CM>(tmA, tmB, tmB3, p, grid, stream);
+        case 164: return launch_one<16, 4, 3, FMT, CT, CM>(tmA, tmB, tmB3, p, grid, stream);
+        case 321: return launch_one<32, 1, 10, FMT, CT, CM>(tmA, tmB, tmB3, p, grid, stream);
+        case 322: return launch_one<32, 2, 5, FMT, CT, CM>(tmA, tmB, tmB3, p, grid, stream);
+        case 324: return launch_one<32, 4, 3, FMT, CT, CM>(tmA, tmB, tmB3, p, grid, stream);
+        case 641: return launch_one<64, 1, 8, FMT, CT, CM>(tmA, tmB, tmB3, p, grid, stream);
+        case 642: return launch_one<64, 2, 5, FMT, CT, CM>(tmA, tmB, tmB3, p, grid, stream);
+        case 644: return launch_one<64, 4, 3, FMT, CT, CM>(tmA, tmB, tmB3, p, grid, stream);
+        case 1281: return launch_one<128, 1, 3, FMT, CT, CM>(tmA, tmB, tmB3, p, grid, stream);
+        case 1282: return launch_one<128, 2, 2, FMT, CT, CM>(tmA, tmB, tmB3, p, grid, stream);
         default: return cudaErrorInvalidValue;
     }
+}
+
+template <int FMT>
+cudaError_t launch_fmt(int b, int groups, int c16, int cm, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                       const CUtensorMap& tmB3, const BcsrParams& p, int grid, cudaStream_t stream) {
+    if (cm) return c16 ? launch_shape<FMT, 1, 1>(b, groups, tmA, tmB, tmB3, p, grid, stream)
+                       : launch_shape<FMT, 0, 1>(b, groups, tmA, tmB, tmB3, p, grid, stream);
+    return c16 ? launch_shape<FMT, 1, 0>(b, groups, tmA, tmB, tmB3, p, grid, stream)
+               : launch_shape<FMT, 0, 0>(b, groups, tmA, tmB, tmB3, p, grid, stream);
 }
 
 }  // namespace
 
 int bcsr_token_groups_max(int b) { return b == 128 ? 2 : 4; }
 
-cudaError_t launch_bcsr(int dtype, int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB,
+cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, const CUtensorMap& tmA, const CUtensorMap& tmB,
                         const CUtensorMap& tmB3, const BcsrParams& p, int grid, cudaStream_t stream) {
-    if (dtype == 1) return launch_fmt<0>(b, groups, tmA, tmB, tmB3, p, grid, stream);   // fp16
-    if (dtype == 0) return launch_fmt<1>(b, groups, tmA, tmB, tmB3, p, grid, stream);   // bf16
+    if (dtype == 1) return launch_fmt<0>(b, groups, c16, col_major, tmA, tmB, tmB3, p, grid, stream);   // fp16
+    if (dtype == 0) return launch_fmt<1>(b, groups, c16, col_major, tmA, tmB, tmB3, p, grid, stream);   // bf16
     return cudaErrorInvalidValue;
 }
 

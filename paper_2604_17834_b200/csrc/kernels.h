@@ -12,7 +12,7 @@ struct BcsrParams {
     const int32_t* block_col_idx;
     const int2* tiles;        // {block-row, token tile}, CTA-major
     const int32_t* cta_ptr;   // [grid+1] ranges of tiles
-    float* C;
+    void* C;            // fp32 or the input's 16-bit type; [m][N], or [N][m] with column-major operands
     int64_t m, N;
     int* status;
     uint64_t wait_limit_ns;
@@ -21,9 +21,13 @@ struct BcsrParams {
 };
 
 // dtype: 0 bf16, 1 fp16.  groups: token tile = 128 * groups columns of B (1, 2 or 4).
-// tmB: B as [k][N], box b x 64.  tmB3: B as [N / 64][k][64], box (2 * groups) x b x 64.
-cudaError_t launch_bcsr(int dtype, int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                        const CUtensorMap& tmB3, const BcsrParams& p, int grid, cudaStream_t stream);
+// c16: C in the input's 16-bit type.  Row-major operands: tmB = B as [k][N], box b x 64;
+// tmB3 = B as [N / 64][k][64], box (2 * groups) x b x 64.  Column-major operands (col_major):
+// tmB = X as [N][k], box 128 tokens x min(b, 64); tmB3 = X as [N / 128][128][k], box
+// groups x 128 x min(b, 64); both with the swizzle of min(b, 64) * 2 bytes.
+cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, const CUtensorMap& tmA,
+                        const CUtensorMap& tmB, const CUtensorMap& tmB3, const BcsrParams& p, int grid,
+                        cudaStream_t stream);
 int bcsr_token_groups_max(int b);
 // stored blocks that share one pipeline stage (and one A request): 4 / 2 for b = 16 / 32
 constexpr int bcsr_blocks_per_stage(int b) { return b == 16 ? 4 : (b == 32 ? 2 : 1); }
@@ -77,7 +81,7 @@ struct WcsrParams {
     const int32_t* col_idx;      // window_col_idx [P]
     const uint8_t* packed;       // packed A values
     const void* B;               // k x N row-major
-    float* C;
+    void* C;                     // [m][N] fp32, or the input's 16-bit type
     float* partial;              // [n_slots][16][N]
     int64_t m, N;
     int32_t n_bins;
@@ -89,7 +93,7 @@ struct WcsrParams {
 
 // dtype: 0 bf16, 1 fp16, 2 tf32.  groups: 1 or 2.  tmB: 2-D map of B (k rows x N), box = 128
 // bytes x 1 row, 128-byte swizzle (32-byte atoms for tf32), used in row-gather mode.
-cudaError_t launch_wcsr(int dtype, const CUtensorMap& tmB, const WcsrParams& p, int sms,
+cudaError_t launch_wcsr(int dtype, int c16, const CUtensorMap& tmB, const WcsrParams& p, int sms,
                         cudaStream_t stream);
 
 struct MergeParams {
@@ -97,11 +101,11 @@ struct MergeParams {
     const int32_t* first;    // first slot or -1
     const int32_t* nparts;   // slots to add (0 = zero fill)
     const float* partial;
-    float* C;
+    void* C;
     int64_t m, N;
     int32_t n;
 };
-cudaError_t launch_wcsr_merge(const MergeParams& p, cudaStream_t stream);
+cudaError_t launch_wcsr_merge(const MergeParams& p, int ctype, cudaStream_t stream);   // ctype: 0 fp32, 1 fp16, 2 bf16
 
 // Device address and size in bytes of the library's built-in partial-tile scratch on the
 // current device (resolved on the first call per device).

@@ -5,6 +5,8 @@
 #pragma once
 
 #include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -344,5 +346,17 @@ __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64
             : "memory");
     }
 }
+
+// ----------------------------------------------------------------------------- output element
+
+// Element type of C: fp32, or the input's 16-bit type when CT = 1 (FMT 0 = fp16, 1 = bf16;
+// TF32 inputs are fp32 values, so their "same as input" output is fp32 as well).
+template <int FMT, int CT> struct CType { using type = float; };
+template <> struct CType<0, 1> { using type = __half; };
+template <> struct CType<1, 1> { using type = __nv_bfloat16; };
+
+template <typename T> __device__ __forceinline__ T from_f32(float x) { return x; }
+template <> __device__ __forceinline__ __half from_f32<__half>(float x) { return __float2half_rn(x); }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
 
 }  // namespace spmm

@@ -80,7 +80,7 @@ struct SegIter {
     }
 };
 
-template <int ES, int FMT, int KT, int STAGES, int PW>
+template <int ES, int FMT, int KT, int STAGES, int PW, int CT>
 __global__ void __launch_bounds__((PW + 5) * 32, WcsrCfg<ES, KT, STAGES>::kCtasPerSm)
 wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
     using Cfg = WcsrCfg<ES, KT, STAGES>;
@@ -355,16 +355,8 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     const int slot = __shfl_sync(0xffffffffu, win.y, j);
                     const int nks = __shfl_sync(0xffffffffu, win.z, j) / Cfg::kKStep;
                     const int nsub = nks < kNSub ? nks : kNSub;
-                    float* out;
-                    int rows;
-                    if (slot < 0) {
-                        const int64_t row0 = static_cast<int64_t>(window) * kWH;
-                        out = p.C + row0 * N;
-                        rows = static_cast<int>(min_i64(kWH, p.m - row0));
-                    } else {
-                        out = p.partial + static_cast<int64_t>(slot) * kWH * N;
-                        rows = kWH;
-                    }
+                    const int64_t row0 = static_cast<int64_t>(window) * kWH;
+                    const int rows = slot < 0 ? static_cast<int>(min_i64(kWH, p.m - row0)) : kWH;
                     const int acc = item % Cfg::kNAcc;
                     const uint32_t aph = (item / Cfg::kNAcc) & 1u;
                     TRACE_T0(tr_a);
@@ -391,9 +383,19 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     if (lane == 0) mbar_arrive(acce_bar(acc));
                     const int n = n0 + qd * 32 + lane;
                     if (n < N) {
+                        if (slot < 0) {
+                            // unsplit window: straight to C, fp32 or the input's 16-bit type
+                            using CElem = typename CType<FMT, CT>::type;
+                            CElem* out = static_cast<CElem*>(p.C) + row0 * N + n;
 #pragma unroll
-                        for (int jr = 0; jr < kWH; ++jr)
-                            if (jr < rows) out[static_cast<int64_t>(jr) * N + n] = v[jr];
+                            for (int jr = 0; jr < kWH; ++jr)
+                                if (jr < rows) out[static_cast<int64_t>(jr) * N] = from_f32<CElem>(v[jr]);
+                        } else {
+                            // split window: fp32 partial tile, summed by the merge kernel
+                            float* out = p.partial + static_cast<int64_t>(slot) * kWH * N + n;
+#pragma unroll
+                            for (int jr = 0; jr < kWH; ++jr) out[static_cast<int64_t>(jr) * N] = v[jr];
+                        }
                     }
                 }
                 win = nwin;
@@ -430,6 +432,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
 
 // C rows of split windows = sum of their partial tiles in slot order; C rows of empty
 // windows = 0.  One CTA per listed window.
+template <typename CElem>
 __global__ void __launch_bounds__(256)
 wcsr_merge_kernel(const MergeParams p) {
     const int i = blockIdx.x;
@@ -445,22 +448,27 @@ wcsr_merge_kernel(const MergeParams p) {
     const int64_t n4 = N >> 2;     // N is a multiple of 4
     const int64_t total = static_cast<int64_t>(rows) * n4;
     const float4* part = reinterpret_cast<const float4*>(p.partial);
-    float4* out = reinterpret_cast<float4*>(p.C + row0 * N);
+    CElem* out = static_cast<CElem*>(p.C) + row0 * N;
     for (int64_t e = threadIdx.x; e < total; e += blockDim.x) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int s = 0; s < nparts; ++s) {
             const float4 v = part[static_cast<int64_t>(first + s) * kWH * n4 + e];
             acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
         }
-        out[e] = acc;
+        if constexpr (sizeof(CElem) == 4) {
+            reinterpret_cast<float4*>(out)[e] = acc;
+        } else {
+            alignas(8) CElem q[4] = {from_f32<CElem>(acc.x), from_f32<CElem>(acc.y), from_f32<CElem>(acc.z), from_f32<CElem>(acc.w)};
+            reinterpret_cast<uint2*>(out)[e] = *reinterpret_cast<const uint2*>(q);
+        }
     }
 }
 
-template <int ES, int FMT>
+template <int ES, int FMT, int CT>
 cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
     constexpr int KT = wcsr_stage_cols(ES), STAGES = wcsr_stages(ES), PW = wcsr_producer_warps(ES);
     using Cfg = WcsrCfg<ES, KT, STAGES>;
-    auto kfn = wcsr_spmm_kernel<ES, FMT, KT, STAGES, PW>;
+    auto kfn = wcsr_spmm_kernel<ES, FMT, KT, STAGES, PW, CT>;
     static int occ = 0;
     if (occ == 0) {
         cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
@@ -481,10 +489,10 @@ cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cud
 
 }  // namespace
 
-cudaError_t launch_wcsr(int dtype, const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
-    if (dtype == 2) return launch_one<4, 2>(tmB, p, sms, stream);
-    if (dtype == 1) return launch_one<2, 0>(tmB, p, sms, stream);
-    if (dtype == 0) return launch_one<2, 1>(tmB, p, sms, stream);
+cudaError_t launch_wcsr(int dtype, int c16, const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
+    if (dtype == 2) return launch_one<4, 2, 0>(tmB, p, sms, stream);
+    if (dtype == 1) return c16 ? launch_one<2, 0, 1>(tmB, p, sms, stream) : launch_one<2, 0, 0>(tmB, p, sms, stream);
+    if (dtype == 0) return c16 ? launch_one<2, 1, 1>(tmB, p, sms, stream) : launch_one<2, 1, 0>(tmB, p, sms, stream);
     return cudaErrorInvalidValue;
 }
 
@@ -516,7 +524,8 @@ cudaError_t wcsr_static_scratch(float** ptr, size_t* bytes) {
     return cudaSuccess;
 }
 
-cudaError_t launch_wcsr_merge(const MergeParams& p, cudaStream_t stream) {
+// ctype: 0 = fp32 C, 1 = fp16, 2 = bf16
+cudaError_t launch_wcsr_merge(const MergeParams& p, int ctype, cudaStream_t stream) {
     if (p.n <= 0) return cudaSuccess;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(p.n));
@@ -528,7 +537,9 @@ cudaError_t launch_wcsr_merge(const MergeParams& p, cudaStream_t stream) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel, p);
+    if (ctype == 1) return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel<__half>, p);
+    if (ctype == 2) return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel<__nv_bfloat16>, p);
+    return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel<float>, p);
 }
 
 }  // namespace spmm

@@ -34,6 +34,24 @@ def run_gpu(lib, h, B_storage, m, N, fill=float("nan"), check=True):
     return C.cpu().numpy()
 
 
+def run_gpu_variant(lib, h, B_storage, m, N, dtype, c16=False, col_major=False, check=True):
+    """spmm_run for a handle created with c_type / layout options.  B_storage is always the
+    k x N operand; with col_major the device gets X = B^T (N x k) and returns Y = C^T (N x m).
+    The result comes back as an m x N float32 array either way."""
+    import torch
+    Bs = np.ascontiguousarray(B_storage.T) if col_major else B_storage
+    Bd = to_device(Bs)
+    tdt = torch.float32 if not c16 else (torch.bfloat16 if dtype == "bf16" else torch.float16)
+    shape = (N, m) if col_major else (m, N)
+    C = torch.full(shape, float("nan"), dtype=tdt, device="cuda")
+    lib.spmm_run(h, Bd.data_ptr(), C.data_ptr(), N, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    if check:
+        lib.spmm_check(h)
+    out = C.float().cpu().numpy()
+    return np.ascontiguousarray(out.T) if col_major else out
+
+
 def reference(a, B_storage, dtype, cols=None, rows=None):
     v64 = wl.widen(a["vals"], dtype)
     B64 = wl.widen(B_storage if cols is None else B_storage[:, cols], dtype)

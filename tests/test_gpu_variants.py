@@ -1,0 +1,133 @@
+"""GPU parity of the output-type and operand-layout variants: C in the input's 16-bit type
+(BCSR and WCSR) and column-major operands (BCSR: X = B^T in, Y = C^T out, the layout of the
+paper's BCSR kernel, Sec. 3.2, and of a sparse linear layer, Sec. 4.3).  Same oracle, same
+bound as the default path: a 16-bit C adds at most 2^-9 |C| <= 2^-9 sum|a b| of rounding.
+"""
+import numpy as np
+import pytest
+
+from paper_2604_17834_b200 import workloads as wl
+
+from helpers import assert_close, reference, run_gpu, run_gpu_variant
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2604_17834_b200 import binding
+    return binding
+
+
+def _bcsr_variant(lib, a, dtype, b, N, c16, col_major, seed=29):
+    Bs = wl.dense(seed, a["k"], N, ("uniform", -1.0, 1.0), dtype)
+    h = lib.spmm_bcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], dtype, b,
+                                 c_type=lib.C_SAME_AS_INPUT if c16 else lib.C_FP32,
+                                 layout=lib.COLMAJOR if col_major else lib.ROWMAJOR)
+    try:
+        C = run_gpu_variant(lib, h, Bs, a["m"], N, dtype, c16=c16, col_major=col_major)
+        Cr, S = reference(a, Bs, dtype)
+        worst = assert_close(C, Cr, S, dtype, "bcsr b=%d N=%d c16=%d cm=%d" % (b, N, c16, col_major))
+        C2 = run_gpu_variant(lib, h, Bs, a["m"], N, dtype, c16=c16, col_major=col_major)
+        assert np.array_equal(C, C2)
+        return worst
+    finally:
+        lib.spmm_destroy(h)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp16"])
+@pytest.mark.parametrize("b", [16, 32, 64, 128])
+@pytest.mark.parametrize("c16,col_major", [(True, False), (False, True), (True, True)])
+def test_bcsr_variants_block_sizes(lib, dtype, b, c16, col_major):
+    a = wl.bcsr_sweep(500 + b, m=1024, k=768, b=b, density=0.2, dtype=dtype)
+    _bcsr_variant(lib, a, dtype, b, 640, c16, col_major)      # 640 = 512 + 128: several token tiles
+
+
+@pytest.mark.parametrize("m,k,b,N", [(504, 304, 64, 200), (136, 72, 32, 136), (1000, 1000, 16, 1030),
+                                      (264, 640, 128, 333), (64, 64, 64, 128)])
+@pytest.mark.parametrize("c16", [False, True])
+def test_bcsr_colmajor_ragged_shapes(lib, m, k, b, N, c16):
+    """m, k multiples of 8 only; N arbitrary (not a multiple of 128, 64 or even 8); scattered
+    entries, empty block-rows."""
+    a = wl.random_csr(17 + m, m, k, 0.02, "bf16", empty_rows=tuple(range(min(b, m // 2))))
+    _bcsr_variant(lib, a, "bf16", b, N, c16, True)
+
+
+def test_bcsr_colmajor_matches_rowmajor_bitwise(lib):
+    """Same products in the same order: the two layouts differ only in how operands are read and
+    results written, so fp32 results are identical."""
+    a = wl.bcsr_sweep(77, m=512, k=1024, b=64, density=0.3, dtype="fp16")
+    Bs = wl.dense(5, 1024, 512, ("normal", 0.0, 1.0), "fp16")
+    h0 = lib.spmm_bcsr_create_csr(512, 1024, a["row_ptr"], a["col_idx"], a["vals"], "fp16", 64)
+    h1 = lib.spmm_bcsr_create_csr(512, 1024, a["row_ptr"], a["col_idx"], a["vals"], "fp16", 64, layout=lib.COLMAJOR)
+    C0 = run_gpu(lib, h0, Bs, 512, 512)
+    C1 = run_gpu_variant(lib, h1, Bs, 512, 512, "fp16", col_major=True)
+    lib.spmm_destroy(h0)
+    lib.spmm_destroy(h1)
+    assert np.array_equal(C0, C1)
+
+
+def test_bcsr_c16_is_the_rounded_fp32_result(lib):
+    a = wl.bcsr_tiny()
+    Bs = wl.dense(3, 512, 256, ("uniform", -1.0, 1.0), "bf16")
+    h0 = lib.spmm_bcsr_create_csr(512, 512, a["row_ptr"], a["col_idx"], a["vals"], "bf16", 64)
+    h1 = lib.spmm_bcsr_create_csr(512, 512, a["row_ptr"], a["col_idx"], a["vals"], "bf16", 64, c_type=lib.C_SAME_AS_INPUT)
+    C0 = run_gpu(lib, h0, Bs, 512, 256)
+    C1 = run_gpu_variant(lib, h1, Bs, 512, 256, "bf16", c16=True)
+    lib.spmm_destroy(h0)
+    lib.spmm_destroy(h1)
+    import torch
+    want = torch.from_numpy(C0).to(torch.bfloat16).float().numpy()     # round to nearest even
+    assert np.array_equal(C1, want)
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("N", [128, 72, 328])
+def test_wcsr_c16(lib, dtype, N):
+    a = wl.random_csr(53, 1000, 900, 0.02, dtype, empty_rows=tuple(range(32, 64)))
+    Bs = wl.dense(19, 900, N, ("normal", 0.0, 1.0), dtype)
+    h = lib.spmm_wcsr_create_csr(1000, 900, a["row_ptr"], a["col_idx"], a["vals"], dtype, 16, split_cols=64,
+                                 c_type=lib.C_SAME_AS_INPUT)
+    try:
+        info = lib.spmm_get_info(h, N)
+        assert info["n_split"] > 0 and info["n_empty"] >= 2        # direct, merged and zero-filled rows
+        assert info["bytes_c"] == 1000 * N * 2
+        C = run_gpu_variant(lib, h, Bs, 1000, N, dtype, c16=True)
+        Cr, S = reference(a, Bs, dtype)
+        assert_close(C, Cr, S, dtype, "wcsr c16 %s N=%d" % (dtype, N))
+        assert np.array_equal(C, run_gpu_variant(lib, h, Bs, 1000, N, dtype, c16=True))
+    finally:
+        lib.spmm_destroy(h)
+
+
+def test_wcsr_tf32_same_as_input_is_fp32(lib):
+    a = wl.wcsr_irregular(seed=6, m=3000, dtype="tf32")
+    Bs = wl.dense(2, a["k"], 128, ("normal", 0.0, 1.0), "tf32")
+    h0 = lib.spmm_wcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "tf32", 16)
+    h1 = lib.spmm_wcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "tf32", 16, c_type=lib.C_SAME_AS_INPUT)
+    C0, C1 = run_gpu(lib, h0, Bs, a["m"], 128), run_gpu(lib, h1, Bs, a["m"], 128)
+    lib.spmm_destroy(h0)
+    lib.spmm_destroy(h1)
+    assert np.array_equal(C0, C1)
+
+
+def test_variant_argument_errors(lib):
+    a = wl.bcsr_tiny()
+    args = (512, 512, a["row_ptr"], a["col_idx"], a["vals"], "bf16")
+    with pytest.raises(lib.SpmmError) as e:
+        lib.spmm_wcsr_create_csr(*args, 16, layout=lib.COLMAJOR)            # BCSR only
+    assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
+    with pytest.raises(lib.SpmmError) as e:
+        lib.spmm_bcsr_create_csr(*args, 64, c_type=7)
+    assert e.value.code == lib.SPMM_ERR_INVALID_ARG
+    b = wl.random_csr(3, 100, 64, 0.1, "bf16")                             # m = 100: not a multiple of 8
+    with pytest.raises(lib.SpmmError) as e:
+        lib.spmm_bcsr_create_csr(100, 64, b["row_ptr"], b["col_idx"], b["vals"], "bf16", 32, layout=lib.COLMAJOR)
+    assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
+    import torch
+    h = lib.spmm_bcsr_create_csr(*args, 64, layout=lib.COLMAJOR)
+    buf = torch.zeros(1 << 20, dtype=torch.float32, device="cuda")
+    with pytest.raises(lib.SpmmError) as e:
+        lib.spmm_run(h, buf.data_ptr(), buf.data_ptr(), 64)                 # fewer than 128 tokens
+    assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
+    lib.spmm_destroy(h)
