@@ -56,6 +56,15 @@ def workload_table():
         return dict(kind="bcsr", a=wl.bcsr_llm(seed=1013, m=3584, k=18944), dtype="bf16", size=64, N=65536,
                     Bdist=("normal", 0.0, 1.0))
 
+    def variant(base, c16=False, cm=False):
+        """Same matrix and dense operand; C in the input's 16-bit type and / or column-major
+        operands (X = B^T in, Y = C^T out: the linear-layer shape of Sec. 4.3)."""
+        def f():
+            w = base()
+            w["opts"] = dict(c_type=1 if c16 else 0, layout=1 if cm else 0)
+            return w
+        return f
+
     def cfg4(b, d, skewed=True):
         def f():
             return dict(kind="bcsr", a=wl.bcsr_sweep(1004 + b + int(d * 1000), b=b, density=d, skewed=skewed),
@@ -74,6 +83,14 @@ def workload_table():
         "cfg2_wcsr_irregular": ("configs[1] WCSR 100000x100000 tf32 zipf(2) rows, 50% band, wh=16, N=128", cfg2),
         "cfg3_bcsr_llm_gate": ("configs[2] BCSR 18944x3584 bf16 b=64 90% blocks zero, N=65536", cfg3_gate),
         "cfg3_bcsr_llm_down": ("configs[2] BCSR 3584x18944 bf16 b=64 90% blocks zero, N=65536", cfg3_down),
+        "cfg3_bcsr_llm_gate_c16": ("configs[2] gate, C written as bf16", variant(cfg3_gate, c16=True)),
+        "cfg3_bcsr_llm_gate_cm": ("configs[2] gate, column-major operands (X [N][k] in, Y [N][m] out), fp32 Y",
+                                  variant(cfg3_gate, cm=True)),
+        "cfg3_bcsr_llm_gate_cm_c16": ("configs[2] gate as a linear layer: X [N][k] bf16 in, Y [N][m] bf16 out",
+                                      variant(cfg3_gate, c16=True, cm=True)),
+        "cfg3_bcsr_llm_down_cm_c16": ("configs[2] down as a linear layer: X [N][k] bf16 in, Y [N][m] bf16 out",
+                                      variant(cfg3_down, c16=True, cm=True)),
+        "cfg5_wcsr_rmat_n128_c16": ("configs[4] N=128, C written as fp16", variant(cfg5(128), c16=True)),
         "cfg5_wcsr_rmat_n32": ("configs[4] WCSR R-MAT 2^21 deg 16 fp16 wh=16, N=32", cfg5(32)),
         "cfg5_wcsr_rmat_n128": ("configs[4] WCSR R-MAT 2^21 deg 16 fp16 wh=16, N=128", cfg5(128)),
         "cfg5_wcsr_rmat_n256": ("configs[4] WCSR R-MAT 2^21 deg 16 fp16 wh=16, N=256", cfg5(256)),
@@ -93,7 +110,9 @@ HEADLINE = "cfg2_wcsr_irregular"
 DEFAULT_OTHERS = ["cfg1_bcsr_tiny", "cfg3_bcsr_llm_gate", "cfg3_bcsr_llm_down",
                   "cfg4_bcsr_sweep_b16_d0.1", "cfg4_bcsr_sweep_b32_d0.1", "cfg4_bcsr_sweep_b64_d0.1",
                   "cfg4_bcsr_sweep_b128_d0.1", "cfg4_bcsr_sweep_b64_d0.5", "cfg4_bcsr_flat_b64_d0.05",
-                  "cfg5_wcsr_rmat_n32", "cfg5_wcsr_rmat_n128", "cfg5_wcsr_rmat_n256"]
+                  "cfg5_wcsr_rmat_n32", "cfg5_wcsr_rmat_n128", "cfg5_wcsr_rmat_n256",
+                  "cfg3_bcsr_llm_gate_c16", "cfg3_bcsr_llm_gate_cm", "cfg3_bcsr_llm_gate_cm_c16",
+                  "cfg3_bcsr_llm_down_cm_c16", "cfg5_wcsr_rmat_n128_c16"]
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures whose
 # summaries are under profiles/ (None where no capture of that exact launch exists).
@@ -164,6 +183,7 @@ class ClockSampler:
 
 def create_handle(lib, w, **opt):
     a = w["a"]
+    opt = dict(w.get("opts", {}), **opt)
     t0 = time.perf_counter()
     if w["kind"] == "bcsr":
         h = lib.spmm_bcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], w["dtype"], w["size"], **opt)
@@ -221,7 +241,13 @@ def time_workload(torch, lib, w, steps, warmup, flush):
         N = w["N"]
         info = lib.spmm_get_info(h, N)
         B = device_B(torch, w)
-        C = torch.empty((w["a"]["m"], N), dtype=torch.float32, device="cuda")
+        o = w.get("opts", {})
+        cdt = B.dtype if (o.get("c_type") and w["dtype"] != "tf32") else torch.float32
+        if o.get("layout"):
+            B = B.t().contiguous()              # X = B^T, N x k
+            C = torch.empty((N, w["a"]["m"]), dtype=cdt, device="cuda")
+        else:
+            C = torch.empty((w["a"]["m"], N), dtype=cdt, device="cuda")
         st = torch.cuda.current_stream().cuda_stream
         for _ in range(max(3, warmup)):
             lib.spmm_run(h, B.data_ptr(), C.data_ptr(), N, st)
@@ -243,6 +269,29 @@ def time_workload(torch, lib, w, steps, warmup, flush):
                     create_ms=create_ms, launches_per_step=launches, B=B, C=C)
     finally:
         lib.spmm_destroy(h)
+
+
+def dense_context(torch, flush, m=18944, k=3584, N=65536, steps=5):
+    """Context only (Sec. 4.3 compares against the dense layer): the dense bf16 product of the
+    configs[2] gate shape, Y[N][m] = X[N][k] W[m][k]^T, by torch.matmul (cuBLAS)."""
+    X = torch.randn((N, k), device="cuda", dtype=torch.bfloat16)
+    W = torch.randn((m, k), device="cuda", dtype=torch.bfloat16) * 0.02
+    for _ in range(2):
+        Y = X @ W.t()
+    torch.cuda.synchronize()
+    evs = []
+    for _ in range(steps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        Y = X @ W.t()
+        e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    del X, W, Y
+    return {"what": "dense bf16 torch.matmul of the configs[2] gate shape (library GEMM, context only)",
+            "ms_per_step": ms, "tflops_dense": 2.0 * m * k * N / (ms * 1e-3) / 1e12}
 
 
 def summarize(name, desc, res, pk, N):
@@ -377,9 +426,9 @@ def main():
 
     # end to end through the C ABI with host buffers (pinned), copies inside the timed region
     a, N = w["a"], w["N"]
-    Bh = torch.empty((a["k"], N), dtype=res["B"].dtype).pin_memory()
+    Bh = torch.empty(tuple(res["B"].shape), dtype=res["B"].dtype).pin_memory()
     Bh.copy_(res["B"])
-    Ch = torch.empty((a["m"], N), dtype=torch.float32).pin_memory()
+    Ch = torch.empty(tuple(res["C"].shape), dtype=res["C"].dtype).pin_memory()
     h, _ = create_handle(lib, w)
     st = torch.cuda.current_stream().cuda_stream
     e2e_steps = max(3, min(args.steps, 10))
@@ -394,10 +443,10 @@ def main():
     lib.spmm_destroy(h)
     e2e_ms, e2e_value = aggregate_over_ranks(e2e_s * 1e3, info["flops_stored"], world, dist, "cuda")
     e2e = {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
-           "h2d_bytes_per_step": int(Bh.numel() * Bh.element_size()), "d2h_bytes_per_step": int(Ch.numel() * 4)}
+           "h2d_bytes_per_step": int(Bh.numel() * Bh.element_size()), "d2h_bytes_per_step": int(Ch.numel() * Ch.element_size())}
     del res["B"], res["C"]
 
-    others = []
+    others, context = [], None
     if rank == 0 and not args.skip_others and args.only is None:
         names = args.others.split(",") if args.others else DEFAULT_OTHERS
         for nm in names:
@@ -408,6 +457,8 @@ def main():
             others.append(summarize(nm, d2, r2, pk, w2["N"]))
             del w2
             torch.cuda.empty_cache()
+        context = dense_context(torch, flush)
+        torch.cuda.empty_cache()
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -428,7 +479,7 @@ def main():
             "gpu_launches": int(res["launches_per_step"] * args.steps),
             "roofline": with_traffic(head["roofline"], name if not args.dense_width else None), "cpu_baseline": cpu,
             "headline_detail": {k: head[k] for k in ("ms_median", "ms_min", "gflops_useful", "fill_ratio", "create_ms")},
-            "others": others,
+            "others": others, "context": context,
         }
         print(json.dumps(line))
     if world > 1:
