@@ -113,6 +113,9 @@ struct spmm_handle_s {
     int tmB_groups = 0;
     const void* tmB_ptr = nullptr;
     int64_t tmB_N = -1;
+    CUtensorMap tmC;                 // BCSR: the store map of C (or of Y, column-major)
+    const void* tmC_ptr = nullptr;
+    int64_t tmC_N = -1;
 
     // staging for spmm_run_host
     void* d_Bstage = nullptr;
@@ -382,6 +385,36 @@ int ensure_tmB(spmm_handle_s* h, const void* B, int64_t N, int groups) {
     return SPMM_OK;
 }
 
+// Store map of C for the BCSR epilogue (shared-memory staging tile -> TMA store).
+int ensure_tmC(spmm_handle_s* h, void* C, int64_t N) {
+    if (h->tmC_ptr == C && h->tmC_N == N) return SPMM_OK;
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return SPMM_ERR_CUDA;
+    const uint32_t w = static_cast<uint32_t>(bcsr_epi_cols(h->bcsr.b, h->c16, h->col_major));
+    const CUtensorMapDataType dt = !h->c16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                 : (h->dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r;
+    if (h->col_major) {
+        const cuuint64_t dims[2] = {static_cast<cuuint64_t>(h->m), static_cast<cuuint64_t>(N)};
+        const cuuint64_t strides[1] = {static_cast<cuuint64_t>(h->m) * h->cs};
+        const cuuint32_t box[2] = {w, 32};
+        const CUtensorMapSwizzle swz = w * h->cs == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE;
+        r = fn(&h->tmC, dt, 2, C, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+               CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        const cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(h->m)};
+        const cuuint64_t strides[1] = {static_cast<cuuint64_t>(N) * h->cs};
+        const cuuint32_t box[2] = {32, w};
+        r = fn(&h->tmC, dt, 2, C, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+               CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
+    if (r != CUDA_SUCCESS) return SPMM_ERR_CUDA;
+    h->tmC_ptr = C;
+    h->tmC_N = N;
+    return SPMM_OK;
+}
+
 // Tile width, slab width and the tile schedule for dense width N (cached for the last N).
 int ensure_schedule(spmm_handle_s* h, int64_t N) {
     if (h->sched.N == N) return SPMM_OK;
@@ -460,7 +493,10 @@ int run_bcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t s
     rc = ensure_tmB(h, B, N, h->sched.groups);
     if (rc) return rc;
     p.use_3d = h->tmB3_ok ? 1 : 0;
-    cudaError_t e = launch_bcsr(h->dtype, f.b, h->sched.groups, h->c16, h->col_major, tmA, h->tmB, h->tmB3, p, h->n_ctas, stream);
+    rc = ensure_tmC(h, C, N);
+    if (rc) return rc;
+    cudaError_t e = launch_bcsr(h->dtype, f.b, h->sched.groups, h->c16, h->col_major, tmA, h->tmB, h->tmB3,
+                                h->tmC, p, h->n_ctas, stream);
     return e == cudaSuccess ? SPMM_OK : SPMM_ERR_CUDA;
 }
 

@@ -25,10 +25,16 @@ struct BcsrParams {
 // tmB3 = B as [N / 64][k][64], box (2 * groups) x b x 64.  Column-major operands (col_major):
 // tmB = X as [N][k], box 128 tokens x min(b, 64); tmB3 = X as [N / 128][128][k], box
 // groups x 128 x min(b, 64); both with the swizzle of min(b, 64) * 2 bytes.
+// tmC: C as [m][N], box 32 x bcsr_epi_cols, no swizzle; or Y as [N][m], box bcsr_epi_cols x 32,
+// 64-byte swizzle when a box row is 64 bytes.
 cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, const CUtensorMap& tmA,
-                        const CUtensorMap& tmB, const CUtensorMap& tmB3, const BcsrParams& p, int grid,
-                        cudaStream_t stream);
+                        const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p,
+                        int grid, cudaStream_t stream);
 int bcsr_token_groups_max(int b);
+// Accumulator columns (= rows of A's block) an epilogue warp handles at a time: it stages them
+// in a 2 KB shared-memory tile and stores the tile with one TMA request whose box is 32 tokens x
+// this many rows (row-major C) or this many columns x 32 tokens (column-major Y).
+constexpr int bcsr_epi_cols(int b, bool c16, bool col_major) { return (b < 32 || !c16) ? 16 : 32; }
 // stored blocks that share one pipeline stage (and one A request): 4 / 2 for b = 16 / 32
 constexpr int bcsr_blocks_per_stage(int b) { return b == 16 ? 4 : (b == 32 ? 2 : 1); }
 
