@@ -29,23 +29,31 @@ def _sample_cols(N, seed):
     return np.array(sorted(cols), dtype=np.int64)
 
 
-def _run_and_check(lib, kind, a, dtype, size, N, Bs, cols=None, what=""):
+def _run_and_check(lib, kind, a, dtype, size, N, Bs, cols=None, what="", c16=False, col_major=False):
+    """Bs is the k x N operand.  c16: C in the input's 16-bit type; col_major: the device gets
+    X = B^T (N x k) and returns Y = C^T (N x m)."""
     import torch
     mk = lib.spmm_bcsr_create_csr if kind == "bcsr" else lib.spmm_wcsr_create_csr
-    h = mk(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], dtype, size)
+    h = mk(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], dtype, size,
+           c_type=lib.C_SAME_AS_INPUT if c16 else lib.C_FP32, layout=lib.COLMAJOR if col_major else lib.ROWMAJOR)
     try:
         Bd = to_device(Bs)
-        C = torch.full((a["m"], N), float("nan"), dtype=torch.float32, device="cuda")
+        if col_major:
+            Bd = Bd.t().contiguous()
+        cdt = torch.float32 if not c16 else (torch.bfloat16 if dtype == "bf16" else torch.float16)
+        shape = (N, a["m"]) if col_major else (a["m"], N)
+        C = torch.full(shape, float("nan"), dtype=cdt, device="cuda")
         st = torch.cuda.current_stream().cuda_stream
         lib.spmm_run(h, Bd.data_ptr(), C.data_ptr(), N, st)
         torch.cuda.synchronize()
         lib.spmm_check(h)
         assert not bool(torch.isnan(C).any()), "%s: unwritten outputs" % what
         if cols is None:
-            got = C.cpu().numpy()
+            got = (C.t() if col_major else C).float().cpu().numpy()
             Cr, S = reference(a, Bs, dtype)
         else:
-            got = C[:, torch.from_numpy(cols).cuda()].cpu().numpy()
+            ci = torch.from_numpy(cols).cuda()
+            got = (C[ci, :].t() if col_major else C[:, ci]).float().cpu().numpy()
             Cr, S = reference(a, Bs, dtype, cols=cols)
         worst = assert_close(got, Cr, S, dtype, what)
         # second launch: same bits
@@ -75,6 +83,18 @@ def test_config2_bcsr_llm_full(lib, shape):
     _run_and_check(lib, "bcsr", a, "bf16", 64, N, Bs, cols=_sample_cols(N, 3), what="configs[2] " + shape)
 
 
+@pytest.mark.parametrize("shape,c16,col_major", [("gate", True, False), ("gate", False, True), ("gate", True, True),
+                                                  ("down", True, True)])
+def test_config2_bcsr_llm_variants_full(lib, shape, c16, col_major):
+    """configs[2] with C in bf16 and / or column-major operands (the linear-layer shape of
+    Sec. 4.3: X [65536][k] in, Y [65536][m] out), as bench.py launches them."""
+    a = wl.bcsr_llm() if shape == "gate" else wl.bcsr_llm(seed=1013, m=3584, k=18944)
+    N = 65536
+    Bs = wl.dense(1103, a["k"], N, ("normal", 0.0, 1.0), "bf16")
+    _run_and_check(lib, "bcsr", a, "bf16", 64, N, Bs, cols=_sample_cols(N, 3), c16=c16, col_major=col_major,
+                   what="configs[2] %s c16=%d cm=%d" % (shape, c16, col_major))
+
+
 @pytest.mark.parametrize("b,d,skewed", [(16, 0.1, True), (32, 0.2, True), (64, 0.1, True), (128, 0.05, True),
                                          (64, 0.05, False), (16, 0.01, False), (128, 0.5, True)])
 def test_config3_bcsr_sweep_full(lib, b, d, skewed):
@@ -97,3 +117,10 @@ def test_config4_wcsr_rmat_full(lib, rmat_full, N):
     Bs = wl.dense(1105 + N, a["k"], N, ("normal", 0.0, 1.0), "fp16")
     cols = _sample_cols(N, N)[::3] if N > 32 else np.arange(0, 32, 3)
     _run_and_check(lib, "wcsr", a, "fp16", 16, N, Bs, cols=cols, what="configs[4] N=%d" % N)
+
+
+def test_config4_wcsr_rmat_fp16_output_full(lib, rmat_full):
+    """configs[4] at N = 128 with C written as fp16."""
+    a = rmat_full
+    Bs = wl.dense(1105 + 128, a["k"], 128, ("normal", 0.0, 1.0), "fp16")
+    _run_and_check(lib, "wcsr", a, "fp16", 16, 128, Bs, cols=_sample_cols(128, 128)[::3], c16=True, what="configs[4] N=128 fp16 C")
