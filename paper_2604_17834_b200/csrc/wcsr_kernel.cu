@@ -355,8 +355,22 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     const int slot = __shfl_sync(0xffffffffu, win.y, j);
                     const int nks = __shfl_sync(0xffffffffu, win.z, j) / Cfg::kKStep;
                     const int nsub = nks < kNSub ? nks : kNSub;
-                    const int64_t row0 = static_cast<int64_t>(window) * kWH;
-                    const int rows = slot < 0 ? static_cast<int>(min_i64(kWH, p.m - row0)) : kWH;
+                    // unsplit window: straight to C (fp32 or the input's 16-bit type); split
+                    // window: fp32 partial tile, summed by the merge kernel
+                    using CElem = typename CType<FMT, CT>::type;
+                    float* out;         // fp32 destination (C when it is fp32, or the partial tile)
+                    CElem* outc;        // C in its own type
+                    int rows;
+                    if (slot < 0) {
+                        const int64_t row0 = static_cast<int64_t>(window) * kWH;
+                        outc = static_cast<CElem*>(p.C) + row0 * N;
+                        out = reinterpret_cast<float*>(outc);
+                        rows = static_cast<int>(min_i64(kWH, p.m - row0));
+                    } else {
+                        out = p.partial + static_cast<int64_t>(slot) * kWH * N;
+                        outc = nullptr;
+                        rows = kWH;
+                    }
                     const int acc = item % Cfg::kNAcc;
                     const uint32_t aph = (item / Cfg::kNAcc) & 1u;
                     TRACE_T0(tr_a);
@@ -383,18 +397,14 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     if (lane == 0) mbar_arrive(acce_bar(acc));
                     const int n = n0 + qd * 32 + lane;
                     if (n < N) {
-                        if (slot < 0) {
-                            // unsplit window: straight to C, fp32 or the input's 16-bit type
-                            using CElem = typename CType<FMT, CT>::type;
-                            CElem* out = static_cast<CElem*>(p.C) + row0 * N + n;
+                        if (sizeof(CElem) == 4 || slot >= 0) {
 #pragma unroll
                             for (int jr = 0; jr < kWH; ++jr)
-                                if (jr < rows) out[static_cast<int64_t>(jr) * N] = from_f32<CElem>(v[jr]);
+                                if (jr < rows) out[static_cast<int64_t>(jr) * N + n] = v[jr];
                         } else {
-                            // split window: fp32 partial tile, summed by the merge kernel
-                            float* out = p.partial + static_cast<int64_t>(slot) * kWH * N + n;
 #pragma unroll
-                            for (int jr = 0; jr < kWH; ++jr) out[static_cast<int64_t>(jr) * N] = v[jr];
+                            for (int jr = 0; jr < kWH; ++jr)
+                                if (jr < rows) outc[static_cast<int64_t>(jr) * N + n] = from_f32<CElem>(v[jr]);
                         }
                     }
                 }
