@@ -31,10 +31,10 @@ namespace spmm {
 namespace {
 
 constexpr int kWH = 16;
-// A 128 x 16 x K MMA is tiny, and MMAs that accumulate into the same TMEM tile serialise on
-// it, so the K steps of an item rotate over kNSub independent partial accumulators that the
-// epilogue adds (in index order).
-constexpr int kNSub = 4;
+// All K steps of an item accumulate into one 128 x 16 TMEM tile.  (Rotating them over several
+// partial accumulators that the epilogue adds was built and measured 4 - 7 % slower: the
+// tensor pipe takes a 128 x 16 MMA every 39 cycles whether or not it depends on the previous
+// one, and the extra TMEM loads lengthen the epilogue.)
 
 template <int ES, int KT, int STAGES>
 struct WcsrCfg {
@@ -53,9 +53,9 @@ struct WcsrCfg {
     static constexpr int kCtasPerSm = wcsr_bins_per_sm(ES);
     static_assert(kCtasPerSm * (STAGES * kStageBytes + 1024 + 256 + 1024) <= 227 * 1024, "shared memory over-subscribed");
     // items with live accumulators
-    static constexpr int kNAcc = (512 / kCtasPerSm) / (kNSub * kWH) >= 4 ? 4 : 2;
-    static constexpr int kAccCols = kNSub * kWH;            // TMEM columns of one item
-    static constexpr int kTmemCols = kNAcc * kAccCols;      // 128 or 256
+    static constexpr int kNAcc = 4;                         // items with live accumulators
+    static constexpr int kAccCols = kWH;                    // TMEM columns of one item
+    static constexpr int kTmemCols = kNAcc * kAccCols;      // 64
     static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 + 256;
     static_assert(KT % 8 == 0 && KT % kKStep == 0 && KT <= 128, "stage shape");
     static_assert(kGathers % 32 == 0 || kGathers == 16, "gather instructions are dealt to warps");
@@ -257,7 +257,8 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
         TRACE_T0(tr_start);
         SegIter seg;
         seg.init();
-        uint32_t it = 0, item = 0, d0 = 0, kstep_item = 0;
+        uint32_t it = 0, item = 0, d0 = 0;
+        bool fresh = true;                           // the item's accumulator has not been written yet
         int acc = 0;
         bool ok = true;
         while (ok && seg.next(p)) {
@@ -280,7 +281,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                         TRACE_ADD(tr_acce, tr_a);
                         tc_fence_after_sync();
                         d0 = tmem_base + acc * Cfg::kAccCols;
-                        kstep_item = 0;
+                        fresh = true;
                     }
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
@@ -295,26 +296,25 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                         // descriptors differ only in their start-address field (bytes >> 4)
                         const uint64_t a0 = adesc0 + (sb >> 4);
                         const uint64_t b0 = bdesc0 + ((sb + Cfg::kDenseBytes) >> 4);
-                        auto issue = [&](int ks, uint32_t kk) {
-                            const uint32_t dsub = d0 + (kk & (kNSub - 1)) * kWH;
-                            const uint32_t accum = kk >= kNSub ? 1u : 0u;    // first use overwrites
+                        auto issue = [&](int ks) {
+                            // the item's first MMA overwrites the accumulator: no zeroing pass
                             if (leader)
-                                umma_ss<FMT == 2>(dsub, a0 + ((ks * (Cfg::kKStep / 8) * 1024) >> 4),
-                                                  b0 + ((ks * (kWH * 32)) >> 4), idesc, accum);
+                                umma_ss<FMT == 2>(d0, a0 + ((ks * (Cfg::kKStep / 8) * 1024) >> 4),
+                                                  b0 + ((ks * (kWH * 32)) >> 4), idesc, (ks > 0 || !fresh) ? 1u : 0u);
                         };
                         constexpr int kFullSteps = KT / Cfg::kKStep;
                         if (nks == kFullSteps) {                 // a full stage: straight-line code
 #pragma unroll
-                            for (int ks = 0; ks < kFullSteps; ++ks) issue(ks, kstep_item + ks);
+                            for (int ks = 0; ks < kFullSteps; ++ks) issue(ks);
                         } else {
-                            for (int ks = 0; ks < nks; ++ks) issue(ks, kstep_item + ks);
+                            for (int ks = 0; ks < nks; ++ks) issue(ks);
                         }
+                        fresh = false;
                         if (leader) {
                             tc_commit(empty_bar(s));
                             if (last) tc_commit(accf_bar(acc));
                         }
                         __syncwarp();
-                        kstep_item += nks;
                         TRACE_ADD(tr_issue, tr_c);
                     }
                     if (last) ++item;
@@ -353,8 +353,6 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                 for (int j = 0; j < nj; ++j, ++item) {
                     const int window = __shfl_sync(0xffffffffu, win.x, j);
                     const int slot = __shfl_sync(0xffffffffu, win.y, j);
-                    const int nks = __shfl_sync(0xffffffffu, win.z, j) / Cfg::kKStep;
-                    const int nsub = nks < kNSub ? nks : kNSub;
                     // unsplit window: straight to C (fp32 or the input's 16-bit type); split
                     // window: fp32 partial tile, summed by the merge kernel
                     using CElem = typename CType<FMT, CT>::type;
@@ -385,12 +383,6 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                         tmem_ld_wait();
 #pragma unroll
                         for (int jr = 0; jr < kWH; ++jr) v[jr] = __uint_as_float(u[jr]);
-                        for (int sub = 1; sub < nsub; ++sub) {
-                            tmem_ld_x16(tbase + sub * kWH, u);
-                            tmem_ld_wait();
-#pragma unroll
-                            for (int jr = 0; jr < kWH; ++jr) v[jr] += __uint_as_float(u[jr]);
-                        }
                     }
                     tc_fence_before_sync();
                     __syncwarp();
