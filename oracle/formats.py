@@ -214,7 +214,7 @@ def task_bins(plan, n_bins, fixed_cost=32):
     return bin_ptr.astype(np.int32), np.asarray(tasks, dtype=np.int32)
 
 
-def bcsr_tile_schedule(block_row_ptr, n_tt, slab_w, n_ctas, fixed_cost=2):
+def bcsr_tile_schedule(block_row_ptr, n_tt, slab_w, n_ctas, fixed_cost=4):
     """Static schedule of BCSR tiles (block-row, token tile) over n_ctas CTAs.
 
     Addresses the imbalance Sec. 3.5 / Sec. 4.2 (opt6) report for a fixed tile

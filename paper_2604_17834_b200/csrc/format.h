@@ -43,7 +43,9 @@ struct BcsrSchedule {
     std::vector<int32_t> cta_ptr;    // [n_ctas+1]
     std::vector<int32_t> tiles;      // 2 * n_tiles: {block-row, token tile}, CTA-major
 };
-constexpr int kTileFixedCost = 2;
+// a tile's fixed cost in stored-block units: its epilogue writes b x BN x 4 bytes of C, a stored
+// block brings b x BN x 2 bytes of B (measured best of 2 / 4 / 6 / 10 on the skewed sweep)
+constexpr int kTileFixedCost = 4;
 
 struct WcsrTask { int32_t window, q0, count, slot; };
 
