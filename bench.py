@@ -56,12 +56,13 @@ def workload_table():
         return dict(kind="bcsr", a=wl.bcsr_llm(seed=1013, m=3584, k=18944), dtype="bf16", size=64, N=65536,
                     Bdist=("normal", 0.0, 1.0))
 
-    def variant(base, c16=False, cm=False):
+    def variant(base, c16=False, cm=False, dyn=False):
         """Same matrix and dense operand; C in the input's 16-bit type and / or column-major
-        operands (X = B^T in, Y = C^T out: the linear-layer shape of Sec. 4.3)."""
+        operands (X = B^T in, Y = C^T out: the linear-layer shape of Sec. 4.3), or tiles
+        scheduled at run time through Cluster Launch Control instead of the static plan."""
         def f():
             w = base()
-            w["opts"] = dict(c_type=1 if c16 else 0, layout=1 if cm else 0)
+            w["opts"] = dict(c_type=1 if c16 else 0, layout=1 if cm else 0, schedule=1 if dyn else 0)
             return w
         return f
 
@@ -95,10 +96,14 @@ def workload_table():
         "cfg5_wcsr_rmat_n128": ("configs[4] WCSR R-MAT 2^21 deg 16 fp16 wh=16, N=128", cfg5(128)),
         "cfg5_wcsr_rmat_n256": ("configs[4] WCSR R-MAT 2^21 deg 16 fp16 wh=16, N=256", cfg5(256)),
     }
+    t["cfg3_bcsr_llm_gate_dyn"] = ("configs[2] gate, dynamic tile scheduling", variant(cfg3_gate, dyn=True))
+    t["cfg3_bcsr_llm_down_dyn"] = ("configs[2] down, dynamic tile scheduling", variant(cfg3_down, dyn=True))
     for b in (16, 32, 64, 128):
         for d in (0.5, 0.2, 0.1, 0.05, 0.01):
             t["cfg4_bcsr_sweep_b%d_d%g" % (b, d)] = (
                 "configs[3] BCSR 8192x8192 fp16 b=%d skewed rows, keep %g in the rest, N=4096" % (b, d), cfg4(b, d))
+            t["cfg4_bcsr_sweep_b%d_d%g_dyn" % (b, d)] = (
+                "configs[3] b=%d skewed rows, keep %g, dynamic tile scheduling" % (b, d), variant(cfg4(b, d), dyn=True))
         for d in (0.05, 0.01):
             t["cfg4_bcsr_flat_b%d_d%g" % (b, d)] = (
                 "configs[3] BCSR 8192x8192 fp16 b=%d flat Bernoulli(%g), N=4096" % (b, d), cfg4(b, d, False))

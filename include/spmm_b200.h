@@ -75,6 +75,17 @@ typedef enum {
                                     N >= 128; N itself is unconstrained.                      */
 } spmm_layout_t;
 
+/* How the BCSR kernel's tiles (block-row x token tile) reach the CTAs (opts.schedule). */
+typedef enum {
+    SPMM_SCHED_STATIC = 0,       /* dealt to the persistent CTAs ahead of time (default)     */
+    SPMM_SCHED_DYNAMIC = 1       /* one CTA per tile in the grid; running CTAs take over the
+                                    tiles of CTAs that have not started yet (Cluster Launch
+                                    Control), in the schedule's global order.  BCSR, fp32
+                                    row-major C only.  Sec. 3.5 / Sec. 5: the paper's dynamic
+                                    scheduler used an atomic counter and lost to the hardware
+                                    block scheduler; this is the hardware queue itself.       */
+} spmm_sched_t;
+
 /* Optional creation parameters; pass NULL for all defaults.  Zero = default. */
 typedef struct {
     int32_t b_col;       /* WCSR: pad every window to a multiple of this many columns.
@@ -90,7 +101,9 @@ typedef struct {
                             device's SM count (148 when host_only).                          */
     int32_t c_type;      /* spmm_ctype_t                                                      */
     int32_t layout;      /* spmm_layout_t; SPMM_COLMAJOR with a WCSR handle is UNSUPPORTED    */
-    int32_t reserved[10];
+    int32_t schedule;    /* spmm_sched_t; with SPMM_SCHED_DYNAMIC the exported tile list is a
+                            single range (TILE_PTR = {0, n_tiles}) in the global order       */
+    int32_t reserved[9];
 } spmm_opts_t;
 
 typedef struct {

@@ -51,7 +51,7 @@ EXPORTED_SYMBOLS = (
 class SpmmOpts(ctypes.Structure):
     _fields_ = [("b_col", ctypes.c_int32), ("split_cols", ctypes.c_int32), ("host_only", ctypes.c_int32),
                 ("n_ctas", ctypes.c_int32), ("c_type", ctypes.c_int32), ("layout", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 10)]
+                ("schedule", ctypes.c_int32), ("reserved", ctypes.c_int32 * 9)]
 
 
 class SpmmInfo(ctypes.Structure):
@@ -112,10 +112,13 @@ C_FP32, C_SAME_AS_INPUT = 0, 1
 ROWMAJOR, COLMAJOR = 0, 1
 
 
-def _opts(b_col=0, split_cols=0, host_only=False, n_ctas=0, c_type=C_FP32, layout=ROWMAJOR):
+SCHED_STATIC, SCHED_DYNAMIC = 0, 1
+
+
+def _opts(b_col=0, split_cols=0, host_only=False, n_ctas=0, c_type=C_FP32, layout=ROWMAJOR, schedule=SCHED_STATIC):
     o = SpmmOpts()
     o.b_col, o.split_cols, o.host_only, o.n_ctas = b_col, split_cols, int(bool(host_only)), n_ctas
-    o.c_type, o.layout = int(c_type), int(layout)
+    o.c_type, o.layout, o.schedule = int(c_type), int(layout), int(schedule)
     return o
 
 

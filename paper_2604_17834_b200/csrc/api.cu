@@ -75,6 +75,7 @@ struct spmm_handle_s {
     bool host_only = false;
     bool c16 = false;        // C in the input's 16-bit type (never with TF32, whose input type is fp32)
     bool col_major = false;  // BCSR: B given as X[N][k], C as Y[N][m]
+    bool dynamic = false;    // BCSR: tiles handed out at run time through Cluster Launch Control
     int cs = 4;              // bytes per C element
     int n_ctas = 148;
     int sms = 148;
@@ -173,6 +174,7 @@ int check_opts(const spmm_opts_t* opts) {
     if (!opts) return SPMM_OK;
     if (opts->c_type != SPMM_C_FP32 && opts->c_type != SPMM_C_SAME_AS_INPUT) return SPMM_ERR_INVALID_ARG;
     if (opts->layout != SPMM_ROWMAJOR && opts->layout != SPMM_COLMAJOR) return SPMM_ERR_INVALID_ARG;
+    if (opts->schedule != SPMM_SCHED_STATIC && opts->schedule != SPMM_SCHED_DYNAMIC) return SPMM_ERR_INVALID_ARG;
     return SPMM_OK;
 }
 
@@ -193,6 +195,8 @@ int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, cons
     h->c16 = opts && opts->c_type == SPMM_C_SAME_AS_INPUT;
     h->cs = h->c16 ? 2 : 4;
     h->col_major = opts && opts->layout == SPMM_COLMAJOR;
+    h->dynamic = opts && opts->schedule == SPMM_SCHED_DYNAMIC;
+    if (h->dynamic && (h->c16 || h->col_major)) { delete h; return SPMM_ERR_UNSUPPORTED; }
     // column-major operands: rows of X (k elements) and of Y (m elements) must be multiples of
     // 16 bytes for the tensor map and for the 16-byte pieces the epilogue writes
     if (h->col_major && (a.m % 8 != 0 || a.k % 8 != 0)) { delete h; return SPMM_ERR_UNSUPPORTED; }
@@ -230,6 +234,7 @@ int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const s
     if (dtype != SPMM_BF16 && dtype != SPMM_FP16 && dtype != SPMM_TF32) return SPMM_ERR_UNSUPPORTED;
     if (int orc = check_opts(opts)) return orc;
     if (opts && opts->layout == SPMM_COLMAJOR) return SPMM_ERR_UNSUPPORTED;   // BCSR only
+    if (opts && opts->schedule == SPMM_SCHED_DYNAMIC) return SPMM_ERR_UNSUPPORTED;
     int rc = validate_csr(a);
     if (rc) return rc;
     const int b_col_default = 32 / a.es;
@@ -442,7 +447,8 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
     BcsrSchedule sc;
     int rc;
     try {
-        rc = build_bcsr_schedule(f, n_tt, static_cast<int>(sw), h->n_ctas, &sc);
+        // dynamic scheduling: one list in the global order (slab by slab, longest block-row first)
+        rc = build_bcsr_schedule(f, n_tt, static_cast<int>(sw), h->dynamic ? 1 : h->n_ctas, &sc);
     } catch (const std::bad_alloc&) {
         rc = SPMM_ERR_ALLOC;
     }
@@ -495,8 +501,11 @@ int run_bcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t s
     p.use_3d = h->tmB3_ok ? 1 : 0;
     rc = ensure_tmC(h, C, N);
     if (rc) return rc;
-    cudaError_t e = launch_bcsr(h->dtype, f.b, h->sched.groups, h->c16, h->col_major, tmA, h->tmB, h->tmB3,
-                                h->tmC, p, h->n_ctas, stream);
+    // dynamic: one CTA per tile, the schedule was built as a single list in the global order
+    const int grid = h->dynamic ? static_cast<int>(h->sched.tiles.size() / 2) : h->n_ctas;
+    if (grid <= 0) return SPMM_OK;
+    cudaError_t e = launch_bcsr(h->dtype, f.b, h->sched.groups, h->c16, h->col_major, h->dynamic, tmA, h->tmB, h->tmB3,
+                                h->tmC, p, grid, stream);
     return e == cudaSuccess ? SPMM_OK : SPMM_ERR_CUDA;
 }
 

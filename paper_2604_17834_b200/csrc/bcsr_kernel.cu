@@ -27,6 +27,13 @@
 //            contiguous) and C as Y[N][m].  The token tile is then a K-major MMA operand
 //            (rows of min(b, 64) elements, swizzle = row bytes; b = 128 as two K halves), and
 //            the staging tile is [32 tokens][16 or 32 columns of Y].
+//   DYN = 1  dynamic tile scheduling with Cluster Launch Control (the direction Sec. 5 points
+//            to after the paper's atomic-counter scheduler lost to the hardware block
+//            scheduler, Sec. 3.5): the grid has one CTA per tile, in the schedule's global order
+//            (slab by slab, longest block-row first); a CTA runs tile blockIdx.x and then
+//            keeps cancelling the launch of not-yet-started CTAs and running their tiles.  A
+//            seventh warp fetches the tile indices ahead of time into a four-deep ring that
+//            the six working warps read.
 // The host deals tiles to CTAs ahead of time: slab by slab (a slab = token tiles whose B rows
 // fit in L2), longest block-row first, each tile to the least loaded CTA; CTA c walks its list.
 #include "kernels.h"
@@ -60,15 +67,18 @@ struct BcsrCfg {
     static constexpr int kAccCols = GROUPS * B;
     static constexpr int kTmemCols = (2 * kAccCols <= 32) ? 32 : (2 * kAccCols <= 64 ? 64 : (2 * kAccCols <= 128 ? 128 : (2 * kAccCols <= 256 ? 256 : 512)));
     static constexpr int kStagingBytes = 4 * 2048;           // one 2 KB tile per epilogue warp
-    static constexpr int kSmemBytes = STAGES * kStageBytes + kStagingBytes + 1024 /*align*/ + 256 /*barriers*/;
+    static constexpr int kBarrierBytes = 512;                // mbarriers, TMEM slot, flags, tile-index ring
+    static constexpr int kSmemBytes = STAGES * kStageBytes + kStagingBytes + 1024 /*align*/ + kBarrierBytes;
     static_assert(2 * kAccCols <= 512, "accumulators exceed TMEM");
     static_assert(kSmemBytes <= 227 * 1024, "stage ring exceeds shared memory");
-    static_assert((2 * STAGES + 7) * 8 <= 256, "barrier area is 256 bytes");
+    static_assert((2 * STAGES + 7 + 8) * 8 + 64 <= kBarrierBytes, "barrier area");
     static_assert(kBps == 1 || B <= 32, "multi-block stages are for the small block sizes");
 };
 
-template <int B, int GROUPS, int STAGES, int FMT, int CT, int CM>
-__global__ void __launch_bounds__(192, 1)
+constexpr int kSchedDepth = 4;      // tile indices fetched ahead by the dynamic scheduler
+
+template <int B, int GROUPS, int STAGES, int FMT, int CT, int CM, int DYN>
+__global__ void __launch_bounds__(DYN ? 224 : 192, 1)
 bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ CUtensorMap tmC, const BcsrParams p) {
     using Cfg = BcsrCfg<B, GROUPS, STAGES>;
@@ -86,6 +96,10 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * STAGES + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * STAGES + 5);
     const uint32_t drain_bar = bar0 + 8u * (2 * STAGES + 6);   // abort path: MMAs still in flight
+    // dynamic scheduling: ring of fetched tile indices (16-byte answers) with full / empty barriers
+    auto schf_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 7 + s); };
+    auto sche_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 7 + kSchedDepth + s); };
+    const uint32_t sched_resp = (bar0 + 8u * (2 * STAGES + 7 + 2 * kSchedDepth) + 15u) & ~15u;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     WaitCtl ctl{abort_flag, p.status, p.wait_limit_ns};
@@ -94,6 +108,9 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(accf_bar(a), 1); mbar_init(acce_bar(a), 4); }
         mbar_init(drain_bar, 1);
+        if constexpr (DYN) {
+            for (int s = 0; s < kSchedDepth; ++s) { mbar_init(schf_bar(s), 1); mbar_init(sche_bar(s), 6); }
+        }
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tmap(&tmA);
@@ -111,7 +128,39 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t tmem_base = *tmem_slot;
 
     const int64_t N = p.N;
-    const int tile_begin = __ldg(p.cta_ptr + blockIdx.x), tile_end = __ldg(p.cta_ptr + blockIdx.x + 1);
+    // Static schedule: this CTA's range of the tile list.  Dynamic: tile blockIdx.x, then the
+    // indices the scheduler warp obtains; every working warp walks the same sequence.
+    int tile_begin = 0, tile_end = 0;
+    if constexpr (!DYN) {
+        tile_begin = __ldg(p.cta_ptr + blockIdx.x);
+        tile_end = __ldg(p.cta_ptr + blockIdx.x + 1);
+    }
+    // next tile of this warp's walk; nth = number of tiles it has taken so far
+    auto next_tile = [&](uint32_t nth, int* ti, bool* ok) -> bool {
+        if constexpr (!DYN) {
+            *ti = tile_begin + static_cast<int>(nth);
+            return *ti < tile_end;
+        } else {
+            if (nth == 0) { *ti = static_cast<int>(blockIdx.x); return true; }
+            // fetched tile nth is entry nth - 1 of the ring
+            const int slot = (nth - 1u) % kSchedDepth;
+            const uint32_t use = (nth - 1u) / kSchedDepth;
+            if (!__all_sync(0xffffffffu, mbar_wait(schf_bar(slot), use & 1u, ctl, 5))) { *ok = false; return false; }
+            uint32_t x;
+            const bool valid = clc_query(sched_resp + 16u * slot, &x);
+            fence_proxy_async_smem();           // the slot is rewritten by the asynchronous proxy later
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sche_bar(slot));
+            if (valid && x >= gridDim.x) {
+                // cannot happen with a well-formed answer; recorded instead of trusted
+                if (lane == 0 && atomicCAS(p.status, 0, 2) == 0) { p.status[1] = 8; p.status[2] = static_cast<int>(x); }
+                *ok = false;
+                return false;
+            }
+            *ti = static_cast<int>(x);
+            return valid;
+        }
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -127,7 +176,8 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint64_t keep = l2_policy_evict_last();
             TRACE_DECL(tr_empty);
             TRACE_T0(tr_start);
-            for (int ti = tile_begin; ti < tile_end && ok; ++ti) {
+            int ti;
+            for (uint32_t nth = 0; ok && next_tile(nth, &ti, &ok); ++nth) {
                 const int2 tcd = __ldg(p.tiles + ti);
                 const int tI = tcd.x;
                 const int n0 = tcd.y * Cfg::kBnT;
@@ -224,7 +274,8 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             TRACE_DECL(tr_acce);
             TRACE_DECL(tr_issue);
             TRACE_T0(tr_start);
-            for (int ti = tile_begin; ti < tile_end && ok; ++ti, ++tile_i) {
+            int ti;
+            for (; ok && next_tile(tile_i, &ti, &ok); ++tile_i) {
                 const int2 tcd = __ldg(p.tiles + ti);
                 const int tI = tcd.x;
                 const int n0 = tcd.y * Cfg::kBnT;
@@ -287,14 +338,15 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 TRACE_PUT(12, tr_issue);
             }
         }
-    } else {
+    } else if (warp < 6) {
         // ------------------------------------------------------------------ epilogue warps
         const int qd = warp & 3;                    // TMEM lane quarter this warp may read
         uint32_t tile_i = 0;
         bool ok = true;
         TRACE_DECL(tr_accf);
         TRACE_T0(tr_start);
-        for (int ti = tile_begin; ti < tile_end && ok; ++ti, ++tile_i) {
+        int ti;
+        for (; ok && next_tile(tile_i, &ti, &ok); ++tile_i) {
             const int2 tcd = __ldg(p.tiles + ti);
             const int tI = tcd.x;
             const int n0 = tcd.y * Cfg::kBnT;
@@ -396,6 +448,24 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #endif
     }
 
+    if constexpr (DYN) {
+        if (warp == 6 && lane == 0) {
+            // -------------------------------------------------------------- tile scheduler
+            // One request at a time (a request after a failed one is not allowed), up to
+            // kSchedDepth tiles ahead of the slowest working warp.
+            for (uint32_t r = 0;; ++r) {             // ring entry r = the CTA's tile r + 1
+                const int slot = r % kSchedDepth;
+                const uint32_t use = r / kSchedDepth;
+                if (use > 0 && !mbar_wait(sche_bar(slot), (use - 1u) & 1u, ctl, 6)) break;
+                mbar_arrive_expect_tx(schf_bar(slot), 16);
+                clc_try_cancel(sched_resp + 16u * slot, schf_bar(slot));
+                if (!mbar_wait(schf_bar(slot), use & 1u, ctl, 7)) break;
+                uint32_t x;
+                if (!clc_query(sched_resp + 16u * slot, &x)) break;      // no CTA left to cancel: the walk ends
+            }
+        }
+    }
+
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
@@ -415,57 +485,60 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
 }
 
-template <int B, int GROUPS, int STAGES, int FMT, int CT, int CM>
+template <int B, int GROUPS, int STAGES, int FMT, int CT, int CM, int DYN>
 cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p,
                        int grid, cudaStream_t stream) {
     using Cfg = BcsrCfg<B, GROUPS, STAGES>;
-    auto kfn = bcsr_spmm_kernel<B, GROUPS, STAGES, FMT, CT, CM>;
+    auto kfn = bcsr_spmm_kernel<B, GROUPS, STAGES, FMT, CT, CM, DYN>;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    kfn<<<grid, 192, Cfg::kSmemBytes, stream>>>(tmA, tmB, tmB3, tmC, p);
+    kfn<<<grid, DYN ? 224 : 192, Cfg::kSmemBytes, stream>>>(tmA, tmB, tmB3, tmC, p);
     return cudaGetLastError();
 }
 
-template <int FMT, int CT, int CM>
+template <int FMT, int CT, int CM, int DYN>
 cudaError_t launch_shape(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
                          const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
     switch (b * 10 + groups) {
-        case 161: return launch_one<16, 1, 10, FMT, CT, CM>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 162: return launch_one<16, 2, 5, FMT, CT, CM>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 164: return launch_one<16, 4, 3, FMT, CT, CM>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 321: return launch_one<32, 1, 10, FMT, CT, CM>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 322: return launch_one<32, 2, 5, FMT, CT, CM>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 324: return launch_one<32, 4, 3, FMT, CT, CM>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 641: return launch_one<64, 1, 8, FMT, CT, CM>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 642: return launch_one<64, 2, 5, FMT, CT, CM>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 644: return launch_one<64, 4, 3, FMT, CT, CM>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 1281: return launch_one<128, 1, 3, FMT, CT, CM>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 1282: return launch_one<128, 2, 2, FMT, CT, CM>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 161: return launch_one<16, 1, 10, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 162: return launch_one<16, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 164: return launch_one<16, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 321: return launch_one<32, 1, 10, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 322: return launch_one<32, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 324: return launch_one<32, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 641: return launch_one<64, 1, 8, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 642: return launch_one<64, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 644: return launch_one<64, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 1281: return launch_one<128, 1, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 1282: return launch_one<128, 2, 2, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
         default: return cudaErrorInvalidValue;
     }
 }
 
 template <int FMT>
-cudaError_t launch_fmt(int b, int groups, int c16, int cm, const CUtensorMap& tmA, const CUtensorMap& tmB,
+cudaError_t launch_fmt(int b, int groups, int c16, int cm, int dyn, const CUtensorMap& tmA, const CUtensorMap& tmB,
                        const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
-    if (cm) return c16 ? launch_shape<FMT, 1, 1>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream)
-                       : launch_shape<FMT, 0, 1>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
-    return c16 ? launch_shape<FMT, 1, 0>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream)
-               : launch_shape<FMT, 0, 0>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
+    // dynamic scheduling is built for the default output (fp32, row-major) only
+    if (dyn) return (c16 || cm) ? cudaErrorInvalidValue : launch_shape<FMT, 0, 0, 1>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
+    if (cm) return c16 ? launch_shape<FMT, 1, 1, 0>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream)
+                       : launch_shape<FMT, 0, 1, 0>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
+    return c16 ? launch_shape<FMT, 1, 0, 0>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream)
+               : launch_shape<FMT, 0, 0, 0>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
 }
 
 }  // namespace
 
 int bcsr_token_groups_max(int b) { return b == 128 ? 2 : 4; }
 
-cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                        const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
-    if (dtype == 1) return launch_fmt<0>(b, groups, c16, col_major, tmA, tmB, tmB3, tmC, p, grid, stream);   // fp16
-    if (dtype == 0) return launch_fmt<1>(b, groups, c16, col_major, tmA, tmB, tmB3, tmC, p, grid, stream);   // bf16
+cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, int dynamic, const CUtensorMap& tmA,
+                        const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p,
+                        int grid, cudaStream_t stream) {
+    if (dtype == 1) return launch_fmt<0>(b, groups, c16, col_major, dynamic, tmA, tmB, tmB3, tmC, p, grid, stream);   // fp16
+    if (dtype == 0) return launch_fmt<1>(b, groups, c16, col_major, dynamic, tmA, tmB, tmB3, tmC, p, grid, stream);   // bf16
     return cudaErrorInvalidValue;
 }
 

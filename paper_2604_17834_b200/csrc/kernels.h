@@ -27,7 +27,9 @@ struct BcsrParams {
 // groups x 128 x min(b, 64); both with the swizzle of min(b, 64) * 2 bytes.
 // tmC: C as [m][N], box 32 x bcsr_epi_cols, no swizzle; or Y as [N][m], box bcsr_epi_cols x 32,
 // 64-byte swizzle when a box row is 64 bytes.
-cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, const CUtensorMap& tmA,
+// dynamic: the grid is one CTA per tile (grid = number of tiles, p.tiles in the schedule's global
+// order, p.cta_ptr unused) and CTAs steal tiles through Cluster Launch Control; fp32 row-major only.
+cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, int dynamic, const CUtensorMap& tmA,
                         const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p,
                         int grid, cudaStream_t stream);
 int bcsr_token_groups_max(int b);

@@ -361,6 +361,34 @@ __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64
     }
 }
 
+// ----------------------------------------------------------------------------- cluster launch control
+
+// Ask the hardware to cancel the launch of a CTA of this grid that has not started yet and to
+// hand its index to the caller instead (work stealing from the grid's own launch queue).  The
+// 16-byte answer is written to shared memory at `resp`; completion is counted on `bar` (16 bytes).
+__device__ __forceinline__ void clc_try_cancel(uint32_t resp, uint32_t bar) {
+    asm volatile("clusterlaunchcontrol.try_cancel.async.shared::cta.mbarrier::complete_tx::bytes.b128 [%0], [%1];"
+                 ::"r"(resp), "r"(bar) : "memory");
+}
+// Decode an answer: true and the cancelled CTA's blockIdx.x, or false (nothing left to cancel).
+__device__ __forceinline__ bool clc_query(uint32_t resp, uint32_t* ctaid_x) {
+    uint32_t valid, x = 0;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b128 r;\n\t"
+        "ld.shared.b128 r, [%2];\n\t"
+        "clusterlaunchcontrol.query_cancel.is_canceled.pred.b128 p, r;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "@p clusterlaunchcontrol.query_cancel.get_first_ctaid::x.b32.b128 %1, r;\n\t"
+        "}\n"
+        : "=r"(valid), "+r"(x)
+        : "r"(resp)
+        : "memory");
+    *ctaid_x = x;
+    return valid != 0;
+}
+
 // ----------------------------------------------------------------------------- shared-memory stores
 
 __device__ __forceinline__ void st_shared_u16(uint32_t addr, unsigned short x) {

@@ -111,6 +111,38 @@ def test_wcsr_tf32_same_as_input_is_fp32(lib):
     assert np.array_equal(C0, C1)
 
 
+@pytest.mark.parametrize("b,N", [(16, 1024), (32, 2048), (64, 640), (128, 1032), (64, 4096)])
+def test_bcsr_dynamic_schedule_matches_static_bitwise(lib, b, N):
+    """Tiles handed out at run time through Cluster Launch Control (more tiles than SMs, so
+    running CTAs do take over tiles of CTAs that never start): every tile is computed exactly
+    once and exactly as in the static plan, whichever CTA runs it."""
+    a = wl.bcsr_sweep(700 + b, m=2048, k=1024, b=b, density=0.15, dtype="fp16")
+    Bs = wl.dense(31, a["k"], N, ("uniform", -1.0, 1.0), "fp16")
+    args = (a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "fp16", b)
+    h0 = lib.spmm_bcsr_create_csr(*args)
+    h1 = lib.spmm_bcsr_create_csr(*args, schedule=lib.SCHED_DYNAMIC)
+    try:
+        C0 = run_gpu(lib, h0, Bs, a["m"], N)
+        C1 = run_gpu(lib, h1, Bs, a["m"], N)
+        assert np.array_equal(C0, C1)
+        assert np.array_equal(C1, run_gpu(lib, h1, Bs, a["m"], N))
+        Cr, S = reference(a, Bs, "fp16")
+        assert_close(C1, Cr, S, "fp16", "bcsr dynamic b=%d N=%d" % (b, N))
+        # the dynamic plan is one list: every (block-row, token tile) once, slab by slab, longest first
+        tp = lib.spmm_export(h1, lib.X_BCSR_TILE_PTR, np.int32)
+        tiles = lib.spmm_export(h1, lib.X_BCSR_TILES, np.int32).reshape(-1, 2)
+        info = lib.spmm_get_info(h1, N)
+        n_tt = -(-N // info["plan_token_tile"])
+        assert tp.tolist() == [0, tiles.shape[0]] and tiles.shape[0] == (2048 // b) * n_tt
+        from oracle import formats as F
+        f = F.bcsr_from_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], b)
+        want_ptr, want_tiles = F.bcsr_tile_schedule(f["block_row_ptr"], n_tt, info["plan_slab_tiles"], 1)
+        assert np.array_equal(tiles, want_tiles)
+    finally:
+        lib.spmm_destroy(h0)
+        lib.spmm_destroy(h1)
+
+
 def test_variant_argument_errors(lib):
     a = wl.bcsr_tiny()
     args = (512, 512, a["row_ptr"], a["col_idx"], a["vals"], "bf16")
@@ -120,6 +152,12 @@ def test_variant_argument_errors(lib):
     with pytest.raises(lib.SpmmError) as e:
         lib.spmm_bcsr_create_csr(*args, 64, c_type=7)
     assert e.value.code == lib.SPMM_ERR_INVALID_ARG
+    with pytest.raises(lib.SpmmError) as e:
+        lib.spmm_bcsr_create_csr(*args, 64, schedule=lib.SCHED_DYNAMIC, c_type=lib.C_SAME_AS_INPUT)   # fp32 row-major only
+    assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
+    with pytest.raises(lib.SpmmError) as e:
+        lib.spmm_wcsr_create_csr(*args, 16, schedule=lib.SCHED_DYNAMIC)
+    assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
     b = wl.random_csr(3, 100, 64, 0.1, "bf16")                             # m = 100: not a multiple of 8
     with pytest.raises(lib.SpmmError) as e:
         lib.spmm_bcsr_create_csr(100, 64, b["row_ptr"], b["col_idx"], b["vals"], "bf16", 32, layout=lib.COLMAJOR)
