@@ -96,6 +96,15 @@ def workload_table():
         "cfg5_wcsr_rmat_n128": ("configs[4] WCSR R-MAT 2^21 deg 16 fp16 wh=16, N=128", cfg5(128)),
         "cfg5_wcsr_rmat_n256": ("configs[4] WCSR R-MAT 2^21 deg 16 fp16 wh=16, N=256", cfg5(256)),
     }
+    def tall(base):
+        """Same matrix with the paper's own 64-row WCSR windows (Sec. 4.1) instead of 16."""
+        def f():
+            w = base()
+            w["size"] = 64
+            return w
+        return f
+    t["cfg2_wcsr_irregular_wh64"] = ("configs[1] with 64-row windows", tall(cfg2))
+    t["cfg5_wcsr_rmat_n128_wh64"] = ("configs[4] N=128 with 64-row windows", tall(cfg5(128)))
     t["cfg3_bcsr_llm_gate_dyn"] = ("configs[2] gate, dynamic tile scheduling", variant(cfg3_gate, dyn=True))
     t["cfg3_bcsr_llm_down_dyn"] = ("configs[2] down, dynamic tile scheduling", variant(cfg3_down, dyn=True))
     for b in (16, 32, 64, 128):

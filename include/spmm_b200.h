@@ -177,8 +177,9 @@ int spmm_bcsr_create_coo(spmm_handle_t *out, int64_t m, int64_t k, int64_t nnz,
 
 /*
  * Create a WCSR handle (Sec. 2.3, WCSR paragraph; task split of Sec. 3.3).
- * Arguments as above; window_height is 16 (the only supported value; Sec. 5
- * names finer-than-64 windows as the redesign this library performs).
+ * Arguments as above; window_height is 16 (the benchmark configurations; Sec. 5 names
+ * finer-than-64 windows as the redesign this library performs) or 64 (the paper's own
+ * window, Sec. 4.1).
  * Per window the kept columns are ascending, then -1 pads up to a multiple of b_col.
  */
 int spmm_wcsr_create_csr(spmm_handle_t *out, int64_t m, int64_t k, const int64_t *row_ptr,

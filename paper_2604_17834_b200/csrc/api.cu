@@ -256,7 +256,7 @@ int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const s
     rc = device_setup(h, opts);
     if (rc) { free_handle(h); return rc; }
     try {
-        rc = build_wcsr(a, wh, b_col, T, h->n_ctas * wcsr_bins_per_sm(elem_size(dtype)), &h->wcsr);
+        rc = build_wcsr(a, wh, b_col, T, h->n_ctas * wcsr_bins_per_sm(elem_size(dtype), wh), &h->wcsr);
     } catch (const std::bad_alloc&) {
         rc = SPMM_ERR_ALLOC;
     }
@@ -510,7 +510,7 @@ int run_bcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t s
 }
 
 int64_t wcsr_workspace_bytes(const spmm_handle_s* h, int64_t N) {
-    return h->wcsr.n_slots * int64_t{16} * N * 4;
+    return h->wcsr.n_slots * int64_t{h->wcsr.wh} * N * 4;
 }
 
 int launch_wcsr_all(spmm_handle_s* h, const void* B, void* C, float* partial, int64_t N, cudaStream_t stream) {
@@ -539,7 +539,7 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, void* C, float* partial, in
     if (!f.tasks.empty()) {
         int rc = ensure_tmB(h, B, N, 1);
         if (rc) return rc;
-        cudaError_t e = launch_wcsr(h->dtype, h->c16, h->tmB, p, h->sms, stream);
+        cudaError_t e = launch_wcsr(h->dtype, f.wh, h->c16, h->tmB, p, h->sms, stream);
         if (e != cudaSuccess) return SPMM_ERR_CUDA;
     }
     MergeParams mp;
@@ -551,7 +551,7 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, void* C, float* partial, in
     mp.m = h->m;
     mp.N = N;
     mp.n = h->n_merge;
-    cudaError_t e = launch_wcsr_merge(mp, h->c16 ? (h->dtype == SPMM_FP16 ? 1 : 2) : 0, stream);
+    cudaError_t e = launch_wcsr_merge(mp, f.wh, h->c16 ? (h->dtype == SPMM_FP16 ? 1 : 2) : 0, stream);
     return e == cudaSuccess ? SPMM_OK : SPMM_ERR_CUDA;
 }
 

@@ -174,7 +174,7 @@ int build_bcsr_schedule(const BcsrHost& f, int n_tt, int slab_w, int n_ctas, Bcs
 // ----------------------------------------------------------------------------- WCSR
 
 int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost* out) {
-    if (wh != 16) return SPMM_ERR_UNSUPPORTED;
+    if (wh != 16 && wh != 64) return SPMM_ERR_UNSUPPORTED;
     if (b_col * a.es != 32) return SPMM_ERR_UNSUPPORTED;
     if (T < 0 || T % b_col != 0 || n_bins <= 0) return SPMM_ERR_INVALID_ARG;
     out->wh = wh;

@@ -42,36 +42,20 @@ constexpr int bcsr_blocks_per_stage(int b) { return b == 16 ? 4 : (b == 32 ? 2 :
 
 // WCSR pipeline shape, shared by the host schedule (fills are cut to the stage size) and the
 // kernel.  A stage holds 128 / es columns (64 of a 2-byte type, 32 of TF32) of one 128-token
-// tile: 16 KB of gathered B rows + 2 KB of A.  Per value size: ring depth, producer warps
-// (each owns STAGES / PW stages) and resident CTAs per SM, which is also the number of bins
-// per SM of the static schedule (every resident CTA walks one bin).  Measured on B200:
-// 2-byte types run fastest as three small CTAs per SM (4 stages, 4 producer warps), TF32 as
-// two deeper ones (6 stages, 6 producer warps); both fill the SM's shared memory.
+// tile: 16 KB of gathered B rows + the A tile (2 KB at window height 16, 8 KB at 64).  Per value
+// size and window height: ring depth, producer warps (each owns STAGES / PW stages) and resident
+// CTAs per SM, which is also the number of bins per SM of the static schedule (every resident
+// CTA walks one bin).  Measured on B200 at height 16: 2-byte types run fastest as three small
+// CTAs per SM (4 stages, 4 producer warps), TF32 as two deeper ones (6 stages, 6 producer warps);
+// both fill the SM's shared memory.  Height 64: two CTAs per SM, 4 stages of 24 KB, 4 producer
+// warps (the accumulators of two CTAs fill the 512 TMEM columns).
 #ifndef WCSR_STAGE_ROW_BYTES
 #define WCSR_STAGE_ROW_BYTES 128
 #endif
-#ifndef WCSR_STAGES_16
-#define WCSR_STAGES_16 4
-#endif
-#ifndef WCSR_PW_16
-#define WCSR_PW_16 4
-#endif
-#ifndef WCSR_BINS_16
-#define WCSR_BINS_16 3
-#endif
-#ifndef WCSR_STAGES_32
-#define WCSR_STAGES_32 6
-#endif
-#ifndef WCSR_PW_32
-#define WCSR_PW_32 6
-#endif
-#ifndef WCSR_BINS_32
-#define WCSR_BINS_32 2
-#endif
 constexpr int wcsr_stage_cols(int es) { return WCSR_STAGE_ROW_BYTES / es; }
-constexpr int wcsr_stages(int es) { return es == 4 ? WCSR_STAGES_32 : WCSR_STAGES_16; }
-constexpr int wcsr_producer_warps(int es) { return es == 4 ? WCSR_PW_32 : WCSR_PW_16; }
-constexpr int wcsr_bins_per_sm(int es) { return es == 4 ? WCSR_BINS_32 : WCSR_BINS_16; }
+constexpr int wcsr_stages(int es, int wh) { return wh == 64 ? 4 : (es == 4 ? 6 : 4); }
+constexpr int wcsr_producer_warps(int es, int wh) { return wh == 64 ? 4 : (es == 4 ? 6 : 4); }
+constexpr int wcsr_bins_per_sm(int es, int wh) { return wh == 64 ? 2 : (es == 4 ? 2 : 3); }
 
 // Device task descriptor of the WCSR kernel (one per sub-task of the split plan).
 struct WcsrDevTask {
@@ -90,7 +74,7 @@ struct WcsrParams {
     const uint8_t* packed;       // packed A values
     const void* B;               // k x N row-major
     void* C;                     // [m][N] fp32, or the input's 16-bit type
-    float* partial;              // [n_slots][16][N]
+    float* partial;              // [n_slots][window height][N]
     int64_t m, N;
     int32_t n_bins;
     int32_t n_tt;                // token tiles = ceil(N / (128 * groups))
@@ -101,7 +85,7 @@ struct WcsrParams {
 
 // dtype: 0 bf16, 1 fp16, 2 tf32.  groups: 1 or 2.  tmB: 2-D map of B (k rows x N), box = 128
 // bytes x 1 row, 128-byte swizzle (32-byte atoms for tf32), used in row-gather mode.
-cudaError_t launch_wcsr(int dtype, int c16, const CUtensorMap& tmB, const WcsrParams& p, int sms,
+cudaError_t launch_wcsr(int dtype, int wh, int c16, const CUtensorMap& tmB, const WcsrParams& p, int sms,
                         cudaStream_t stream);
 
 struct MergeParams {
@@ -113,7 +97,7 @@ struct MergeParams {
     int64_t m, N;
     int32_t n;
 };
-cudaError_t launch_wcsr_merge(const MergeParams& p, int ctype, cudaStream_t stream);   // ctype: 0 fp32, 1 fp16, 2 bf16
+cudaError_t launch_wcsr_merge(const MergeParams& p, int wh, int ctype, cudaStream_t stream);   // ctype: 0 fp32, 1 fp16, 2 bf16
 
 // Device address and size in bytes of the library's built-in partial-tile scratch on the
 // current device (resolved on the first call per device).

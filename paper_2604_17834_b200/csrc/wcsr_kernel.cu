@@ -30,14 +30,14 @@ namespace spmm {
 
 namespace {
 
-constexpr int kWH = 16;
 // All K steps of an item accumulate into one 128 x 16 TMEM tile.  (Rotating them over several
 // partial accumulators that the epilogue adds was built and measured 4 - 7 % slower: the
 // tensor pipe takes a 128 x 16 MMA every 39 cycles whether or not it depends on the previous
 // one, and the extra TMEM loads lengthen the epilogue.)
 
-template <int ES, int KT, int STAGES>
+template <int ES, int WH, int KT, int STAGES>
 struct WcsrCfg {
+    static constexpr int kWH = WH;                          // window height = MMA N
     static constexpr int kKStep = 32 / ES;                  // columns per MMA (= b_col)
     static constexpr int kBnT = 128;                        // tokens per tile = TMEM lanes
     static constexpr int kRowBytes = kBnT * ES;
@@ -50,12 +50,12 @@ struct WcsrCfg {
     static constexpr int kStageBytes = kDenseBytes + kABytes;
     // resident CTAs per SM = bins per SM of the schedule; they must fit the SM's shared memory
     // (1 KB per CTA is reserved by the system) and share its 512 TMEM columns
-    static constexpr int kCtasPerSm = wcsr_bins_per_sm(ES);
+    static constexpr int kCtasPerSm = wcsr_bins_per_sm(ES, WH);
     static_assert(kCtasPerSm * (STAGES * kStageBytes + 1024 + 256 + 1024) <= 227 * 1024, "shared memory over-subscribed");
     // items with live accumulators
     static constexpr int kNAcc = 4;                         // items with live accumulators
     static constexpr int kAccCols = kWH;                    // TMEM columns of one item
-    static constexpr int kTmemCols = kNAcc * kAccCols;      // 64
+    static constexpr int kTmemCols = kNAcc * kAccCols;      // 64 or 256
     static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 + 256;
     static_assert(KT % 8 == 0 && KT % kKStep == 0 && KT <= 128, "stage shape");
     static_assert(kGathers % 32 == 0 || kGathers == 16, "gather instructions are dealt to warps");
@@ -80,10 +80,11 @@ struct SegIter {
     }
 };
 
-template <int ES, int FMT, int KT, int STAGES, int PW, int CT>
-__global__ void __launch_bounds__((PW + 5) * 32, WcsrCfg<ES, KT, STAGES>::kCtasPerSm)
+template <int ES, int FMT, int WH, int KT, int STAGES, int PW, int CT>
+__global__ void __launch_bounds__((PW + 5) * 32, WcsrCfg<ES, WH, KT, STAGES>::kCtasPerSm)
 wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
-    using Cfg = WcsrCfg<ES, KT, STAGES>;
+    using Cfg = WcsrCfg<ES, WH, KT, STAGES>;
+    constexpr int kWH = WH;
     constexpr int kProducerWarps = PW;          // warps 0 .. PW-1; MMA warp PW; epilogue PW+1 .. PW+4
     constexpr int kMmaWarp = PW;
     // Fill i goes to stage i % STAGES and is produced by warp i % PW.  With STAGES a multiple
@@ -377,12 +378,13 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     tc_fence_after_sync();
                     float v[kWH];
                     const uint32_t tbase = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + acc * Cfg::kAccCols;
-                    {
+#pragma unroll
+                    for (int c = 0; c < kWH; c += 16) {
                         uint32_t u[16];
-                        tmem_ld_x16(tbase, u);
+                        tmem_ld_x16(tbase + c, u);
                         tmem_ld_wait();
 #pragma unroll
-                        for (int jr = 0; jr < kWH; ++jr) v[jr] = __uint_as_float(u[jr]);
+                        for (int jr = 0; jr < 16; ++jr) v[c + jr] = __uint_as_float(u[jr]);
                     }
                     tc_fence_before_sync();
                     __syncwarp();
@@ -434,9 +436,10 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
 
 // C rows of split windows = sum of their partial tiles in slot order; C rows of empty
 // windows = 0.  One CTA per listed window.
-template <typename CElem>
+template <typename CElem, int WH>
 __global__ void __launch_bounds__(256)
 wcsr_merge_kernel(const MergeParams p) {
+    constexpr int kWH = WH;
     const int i = blockIdx.x;
     const int w = p.window[i];
     const int first = p.first[i];
@@ -466,11 +469,11 @@ wcsr_merge_kernel(const MergeParams p) {
     }
 }
 
-template <int ES, int FMT, int CT>
+template <int ES, int FMT, int WH, int CT>
 cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
-    constexpr int KT = wcsr_stage_cols(ES), STAGES = wcsr_stages(ES), PW = wcsr_producer_warps(ES);
-    using Cfg = WcsrCfg<ES, KT, STAGES>;
-    auto kfn = wcsr_spmm_kernel<ES, FMT, KT, STAGES, PW, CT>;
+    constexpr int KT = wcsr_stage_cols(ES), STAGES = wcsr_stages(ES, WH), PW = wcsr_producer_warps(ES, WH);
+    using Cfg = WcsrCfg<ES, WH, KT, STAGES>;
+    auto kfn = wcsr_spmm_kernel<ES, FMT, WH, KT, STAGES, PW, CT>;
     static int occ = 0;
     if (occ == 0) {
         cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
@@ -489,12 +492,19 @@ cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cud
     return cudaGetLastError();
 }
 
+template <int WH>
+cudaError_t launch_wh(int dtype, int c16, const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
+    if (dtype == 2) return launch_one<4, 2, WH, 0>(tmB, p, sms, stream);
+    if (dtype == 1) return c16 ? launch_one<2, 0, WH, 1>(tmB, p, sms, stream) : launch_one<2, 0, WH, 0>(tmB, p, sms, stream);
+    if (dtype == 0) return c16 ? launch_one<2, 1, WH, 1>(tmB, p, sms, stream) : launch_one<2, 1, WH, 0>(tmB, p, sms, stream);
+    return cudaErrorInvalidValue;
+}
+
 }  // namespace
 
-cudaError_t launch_wcsr(int dtype, int c16, const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
-    if (dtype == 2) return launch_one<4, 2, 0>(tmB, p, sms, stream);
-    if (dtype == 1) return c16 ? launch_one<2, 0, 1>(tmB, p, sms, stream) : launch_one<2, 0, 0>(tmB, p, sms, stream);
-    if (dtype == 0) return c16 ? launch_one<2, 1, 1>(tmB, p, sms, stream) : launch_one<2, 1, 0>(tmB, p, sms, stream);
+cudaError_t launch_wcsr(int dtype, int wh, int c16, const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
+    if (wh == 16) return launch_wh<16>(dtype, c16, tmB, p, sms, stream);
+    if (wh == 64) return launch_wh<64>(dtype, c16, tmB, p, sms, stream);
     return cudaErrorInvalidValue;
 }
 
@@ -527,7 +537,7 @@ cudaError_t wcsr_static_scratch(float** ptr, size_t* bytes) {
 }
 
 // ctype: 0 = fp32 C, 1 = fp16, 2 = bf16
-cudaError_t launch_wcsr_merge(const MergeParams& p, int ctype, cudaStream_t stream) {
+cudaError_t launch_wcsr_merge(const MergeParams& p, int wh, int ctype, cudaStream_t stream) {
     if (p.n <= 0) return cudaSuccess;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(p.n));
@@ -539,9 +549,14 @@ cudaError_t launch_wcsr_merge(const MergeParams& p, int ctype, cudaStream_t stre
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (ctype == 1) return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel<__half>, p);
-    if (ctype == 2) return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel<__nv_bfloat16>, p);
-    return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel<float>, p);
+    if (wh == 64) {
+        if (ctype == 1) return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel<__half, 64>, p);
+        if (ctype == 2) return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel<__nv_bfloat16, 64>, p);
+        return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel<float, 64>, p);
+    }
+    if (ctype == 1) return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel<__half, 16>, p);
+    if (ctype == 2) return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel<__nv_bfloat16, 16>, p);
+    return cudaLaunchKernelEx(&cfg, wcsr_merge_kernel<float, 16>, p);
 }
 
 }  // namespace spmm

@@ -100,6 +100,37 @@ def test_wcsr_c16(lib, dtype, N):
         lib.spmm_destroy(h)
 
 
+@pytest.mark.parametrize("dtype", ["tf32", "fp16", "bf16"])
+@pytest.mark.parametrize("N", [128, 72, 328])
+def test_wcsr_window_height_64(lib, dtype, N):
+    """The paper's own window height (Sec. 4.1): 64-row windows, MMA N = 64.  Format arrays
+    bit-exact against the format oracle, result against the SpMM oracle, split + empty windows."""
+    from oracle import formats as F
+    a = wl.random_csr(57, 1000, 900, 0.02, dtype, empty_rows=tuple(range(64, 192)))
+    Bs = wl.dense(19, 900, N, ("normal", 0.0, 1.0), dtype)
+    h = lib.spmm_wcsr_create_csr(1000, 900, a["row_ptr"], a["col_idx"], a["vals"], dtype, 64, split_cols=128)
+    try:
+        b_col = 8 if dtype == "tf32" else 16
+        f = F.wcsr_from_csr(1000, 900, a["row_ptr"], a["col_idx"], a["vals"], 64, b_col)
+        bits = np.uint32 if dtype == "tf32" else np.uint16
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_ROW_PTR, np.int32), f["window_row_ptr"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_COL_IDX, np.int32), f["window_col_idx"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_VALUES, wl.storage_np_dtype(dtype)).view(bits),
+                              f["values"].view(bits).ravel())
+        info = lib.spmm_get_info(h, N)
+        assert info["block"] == 64 and info["n_split"] > 0 and info["n_empty"] >= 2
+        assert info["stored_values"] == 64 * f["window_col_idx"].shape[0]
+        assert info["workspace_bytes"] == info["n_slots"] * 64 * N * 4
+        plan = F.split_plan(f["window_row_ptr"], 128)
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_TASKS, np.int32).reshape(-1, 4), plan)
+        C = run_gpu(lib, h, Bs, 1000, N)
+        Cr, S = reference(a, Bs, dtype)
+        assert_close(C, Cr, S, dtype, "wcsr wh=64 %s N=%d" % (dtype, N))
+        assert np.array_equal(C, run_gpu(lib, h, Bs, 1000, N))
+    finally:
+        lib.spmm_destroy(h)
+
+
 def test_wcsr_tf32_same_as_input_is_fp32(lib):
     a = wl.wcsr_irregular(seed=6, m=3000, dtype="tf32")
     Bs = wl.dense(2, a["k"], 128, ("normal", 0.0, 1.0), "tf32")

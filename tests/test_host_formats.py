@@ -127,14 +127,15 @@ WCSR_CASES = [("tf32", 1000, 900, 0.01, 64), ("fp16", 333, 517, 0.05, 32), ("bf1
               ("fp16", 16, 40, 0.5, 16)]
 
 
+@pytest.mark.parametrize("wh", [16, 64])
 @pytest.mark.parametrize("dtype,m,k,dens,T", WCSR_CASES)
-def test_wcsr_format_plan_and_bins_are_bit_exact(lib, dtype, m, k, dens, T):
+def test_wcsr_format_plan_and_bins_are_bit_exact(lib, dtype, m, k, dens, T, wh):
     a = wl.random_csr(41 + m, m, k, dens, dtype, empty_rows=tuple(range(16, min(32, m))))
     b_col = 8 if dtype == "tf32" else 16
-    h = lib.spmm_wcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, 16, split_cols=T,
+    h = lib.spmm_wcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, wh, split_cols=T,
                                  host_only=True, n_ctas=5)
     try:
-        f = F.wcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], 16, b_col)
+        f = F.wcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], wh, b_col)
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_ROW_PTR, np.int32), f["window_row_ptr"])
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_COL_IDX, np.int32), f["window_col_idx"])
         got = lib.spmm_export(h, lib.X_WCSR_VALUES, wl.storage_np_dtype(dtype))
@@ -145,7 +146,7 @@ def test_wcsr_format_plan_and_bins_are_bit_exact(lib, dtype, m, k, dens, T):
         bin_tasks = lib.spmm_export(h, lib.X_WCSR_BIN_TASKS, np.int32)
         info = lib.spmm_get_info(h, 128)
         n_bins = info["n_bins"]
-        assert n_bins == 5 * (2 if dtype == "tf32" else 3)     # one bin per resident CTA
+        assert n_bins == 5 * (2 if (dtype == "tf32" or wh == 64) else 3)     # one bin per resident CTA
         want_ptr, want_tasks = F.task_bins(plan, n_bins)
         assert np.array_equal(bin_ptr, want_ptr) and np.array_equal(bin_tasks, want_tasks)
         assert sorted(bin_tasks.tolist()) == list(range(plan.shape[0]))      # every task exactly once
@@ -155,14 +156,14 @@ def test_wcsr_format_plan_and_bins_are_bit_exact(lib, dtype, m, k, dens, T):
         for j in range(n_bins):
             assert np.all(np.diff(bin_tasks[bin_ptr[j]:bin_ptr[j + 1]]) > 0)
         P = f["window_col_idx"].shape[0]
-        assert info["n_units"] == P and info["stored_values"] == 16 * P
+        assert info["n_units"] == P and info["stored_values"] == wh * P
         assert info["n_tasks"] == plan.shape[0]
         assert info["n_slots"] == int((plan[:, 3] >= 0).sum())
         assert info["n_split"] == np.unique(plan[plan[:, 3] >= 0, 0]).shape[0]
         assert info["n_empty"] == int((np.diff(f["window_row_ptr"]) == 0).sum())
         assert info["distinct_b_rows"] == np.unique(a["col_idx"]).shape[0]
-        assert info["workspace_bytes"] == info["n_slots"] * 16 * 128 * 4
-        assert info["fill_ratio"] == pytest.approx(F.fill_ratio_wcsr(info["nnz"], P, 16))
+        assert info["workspace_bytes"] == info["n_slots"] * wh * 128 * 4
+        assert info["fill_ratio"] == pytest.approx(F.fill_ratio_wcsr(info["nnz"], P, wh))
     finally:
         lib.spmm_destroy(h)
 
