@@ -103,6 +103,15 @@ def workload_table():
             w["size"] = 64
             return w
         return f
+    def fp8_linear(m, k, seed):
+        def f():
+            return dict(kind="bcsr", a=wl.bcsr_llm(seed=seed, m=m, k=k, dtype="fp8", std=0.5), dtype="fp8", size=64, N=65536,
+                        Bdist=("normal", 0.0, 1.0), opts=dict(layout=1))
+        return f
+    t["cfg3_bcsr_llm_gate_cm_fp8"] = ("configs[2] gate shape with E4M3 weights and activations, X [N][k] in, fp32 Y [N][m] out",
+                                      fp8_linear(18944, 3584, 1003))
+    t["cfg3_bcsr_llm_down_cm_fp8"] = ("configs[2] down shape with E4M3 weights and activations, X [N][k] in, fp32 Y [N][m] out",
+                                      fp8_linear(3584, 18944, 1013))
     t["cfg2_wcsr_irregular_wh64"] = ("configs[1] with 64-row windows", tall(cfg2))
     t["cfg5_wcsr_rmat_n128_wh64"] = ("configs[4] N=128 with 64-row windows", tall(cfg5(128)))
     t["cfg3_bcsr_llm_gate_dyn"] = ("configs[2] gate, dynamic tile scheduling", variant(cfg3_gate, dyn=True))
@@ -211,7 +220,7 @@ def device_B(torch, w, seed=7):
     g = torch.Generator(device="cuda")
     g.manual_seed(seed)
     k, N = w["a"]["k"], w["N"]
-    tdt = {"bf16": torch.bfloat16, "fp16": torch.float16, "tf32": torch.float32}[w["dtype"]]
+    tdt = {"bf16": torch.bfloat16, "fp16": torch.float16, "tf32": torch.float32, "fp8": torch.float8_e4m3fn}[w["dtype"]]
     B = torch.empty((k, N), dtype=tdt, device="cuda")
     rows = max(1, (1 << 26) // N)
     for r0 in range(0, k, rows):
@@ -227,7 +236,8 @@ def device_B(torch, w, seed=7):
 def roofline_of(info, ms, pk):
     """Roofline of one spmm_run: slower of tensor time for the stored flops and HBM time for the model bytes."""
     model_bytes = info["bytes_a"] + info["bytes_idx"] + info["bytes_b_touched"] + info["bytes_c"]
-    tc_peak = pk["bf16_tflops"] * (0.5 if info["dtype"] == 2 else 1.0)       # TF32 = half the bf16 rate (nominal ratio)
+    # TF32 = half, 8-bit = twice the measured bf16 rate (nominal ratios)
+    tc_peak = pk["bf16_tflops"] * {2: 0.5, 3: 2.0}.get(info["dtype"], 1.0)
     t_hbm = model_bytes / (pk["hbm_gbs"] * 1e9)
     t_tc = info["flops_stored"] / (tc_peak * 1e12)
     t = ms * 1e-3

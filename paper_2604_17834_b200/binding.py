@@ -22,8 +22,8 @@ if not os.path.exists(LIB_PATH):
         "(there is no CPU fallback)" % LIB_PATH)
 _lib = ctypes.CDLL(LIB_PATH)
 
-SPMM_BF16, SPMM_FP16, SPMM_TF32 = 0, 1, 2
-DTYPE_CODE = {"bf16": SPMM_BF16, "fp16": SPMM_FP16, "tf32": SPMM_TF32}
+SPMM_BF16, SPMM_FP16, SPMM_TF32, SPMM_FP8_E4M3 = 0, 1, 2, 3
+DTYPE_CODE = {"bf16": SPMM_BF16, "fp16": SPMM_FP16, "tf32": SPMM_TF32, "fp8": SPMM_FP8_E4M3}
 
 SPMM_OK = 0
 SPMM_ERR_INVALID_ARG = -1
@@ -123,7 +123,7 @@ def _opts(b_col=0, split_cols=0, host_only=False, n_ctas=0, c_type=C_FP32, layou
 
 
 def _vals_buffer(vals, dtype):
-    want = {"bf16": np.uint16, "fp16": np.float16, "tf32": np.float32}[dtype]
+    want = {"bf16": np.uint16, "fp16": np.float16, "tf32": np.float32, "fp8": np.uint8}[dtype]
     v = np.ascontiguousarray(vals)
     if v.dtype != want:
         raise TypeError("vals for %s must be %s (raw storage), got %s" % (dtype, want.__name__, v.dtype))

@@ -21,7 +21,7 @@ std::atomic<uint64_t> g_wait_limit_ns{2000000000ull};
 long long* g_trace = nullptr;
 #endif
 
-inline int elem_size(int dtype) { return dtype == SPMM_TF32 ? 4 : 2; }
+inline int elem_size(int dtype) { return dtype == SPMM_TF32 ? 4 : (dtype == SPMM_FP8_E4M3 ? 1 : 2); }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -41,16 +41,18 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-// 2-D row-major tensor [rows][cols] of 16-bit elements, box [box_rows][box_cols].
+// 2-D row-major tensor [rows][cols] of 16-bit (or, for E4M3, 8-bit) elements, box [box_rows][box_cols].
 int encode_2d_16bit(CUtensorMap* map, int dtype, const void* base, uint64_t rows, uint64_t cols,
                     uint32_t box_rows, uint32_t box_cols, CUtensorMapSwizzle swz) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return SPMM_ERR_CUDA;
+    const uint64_t es = dtype == SPMM_FP8_E4M3 ? 1 : 2;
     const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint64_t strides[1] = {cols * es};
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    const CUtensorMapDataType dt = dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+    const CUtensorMapDataType dt = dtype == SPMM_FP8_E4M3 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                 : (dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
     CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? SPMM_OK : SPMM_ERR_CUDA;
@@ -179,8 +181,15 @@ int check_opts(const spmm_opts_t* opts) {
 }
 
 int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, const spmm_opts_t* opts) {
-    if (dtype != SPMM_BF16 && dtype != SPMM_FP16) return SPMM_ERR_UNSUPPORTED;
+    if (dtype != SPMM_BF16 && dtype != SPMM_FP16 && dtype != SPMM_FP8_E4M3) return SPMM_ERR_UNSUPPORTED;
     if (int orc = check_opts(opts)) return orc;
+    if (dtype == SPMM_FP8_E4M3) {
+        // 8-bit inputs: the K-major (column-major operand) path only, fp32 C, static schedule; a block
+        // row must hold a whole 32-element K step; rows of X are k bytes and must be multiples of 16
+        if (!opts || opts->layout != SPMM_COLMAJOR || opts->c_type != SPMM_C_FP32 || opts->schedule != SPMM_SCHED_STATIC)
+            return SPMM_ERR_UNSUPPORTED;
+        if (block < 32 || a.k % 16 != 0) return SPMM_ERR_UNSUPPORTED;
+    }
     int rc = validate_csr(a);
     if (rc) return rc;
     spmm_handle_s* h = new (std::nothrow) spmm_handle_s;
@@ -216,9 +225,11 @@ int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, cons
         if (!rc) rc = upload(&h->d_vals, f.blocks.data(), f.blocks.size());
         if (!rc) rc = upload(&h->d_order, f.row_order.data(), f.row_order.size() * 4);
         if (!rc && f.nnzb > 0) {
-            const int bw = f.b < 64 ? f.b : 64;
-            const CUtensorMapSwizzle swz = bw == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
-                                          : (bw == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+            // box rows of min(b * es, 128) bytes, swizzle = the row bytes
+            const int row_bytes = f.b * h->es < 128 ? f.b * h->es : 128;
+            const int bw = row_bytes / h->es;
+            const CUtensorMapSwizzle swz = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                          : (row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
             rc = encode_2d_16bit(&h->tmA, dtype, h->d_vals, static_cast<uint64_t>(f.nnzb) * f.b, f.b,
                                  static_cast<uint32_t>(f.b * bcsr_blocks_per_stage(f.b)), bw, swz);
             h->tmA_ok = rc == SPMM_OK;
@@ -305,7 +316,7 @@ int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const s
 
 int make_view(CsrView* v, int64_t m, int64_t k, const int64_t* row_ptr, const int32_t* col_idx, const void* vals,
               int dtype) {
-    if (dtype < 0 || dtype > 2) return SPMM_ERR_INVALID_ARG;
+    if (dtype < 0 || dtype > 3) return SPMM_ERR_INVALID_ARG;
     if (m < 0 || k < 0 || !row_ptr) return SPMM_ERR_INVALID_ARG;
     if (m >= (int64_t{1} << 31) || k >= (int64_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
     v->m = m;
@@ -345,19 +356,21 @@ int ensure_tmB(spmm_handle_s* h, const void* B, int64_t N, int groups) {
         // X as [N][k]: box = 128 tokens x min(b, 64) elements, swizzle = the box's row bytes;
         // and the same memory as [N / 128][128][k] so that one request brings all token groups
         // of a tile (whole groups only; a ragged last tile uses the 2-D map, zero filled)
-        const uint32_t bw = h->bcsr.b < 64 ? h->bcsr.b : 64;
-        const CUtensorMapSwizzle swz = bw == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
-                                      : (bw == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+        const uint32_t row_bytes = h->bcsr.b * h->es < 128 ? h->bcsr.b * h->es : 128;
+        const uint32_t bw = row_bytes / h->es;
+        const CUtensorMapSwizzle swz = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                      : (row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
         rc = encode_2d_16bit(&h->tmB, h->dtype, B, static_cast<uint64_t>(N), static_cast<uint64_t>(h->k), 128, bw, swz);
         h->tmB3_ok = false;
         h->tmB3 = h->tmB;
         EncodeTiledFn fn = get_encode_fn();
         if (!rc && fn && N >= 128) {
             const cuuint64_t dims[3] = {static_cast<cuuint64_t>(h->k), 128, static_cast<cuuint64_t>(N / 128)};
-            const cuuint64_t strides[2] = {static_cast<cuuint64_t>(h->k) * 2, static_cast<cuuint64_t>(h->k) * 256};
+            const cuuint64_t strides[2] = {static_cast<cuuint64_t>(h->k) * h->es, static_cast<cuuint64_t>(h->k) * 128 * h->es};
             const cuuint32_t box[3] = {bw, 128, static_cast<cuuint32_t>(groups)};
             const cuuint32_t estr[3] = {1, 1, 1};
-            const CUtensorMapDataType dt = h->dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+            const CUtensorMapDataType dt = h->dtype == SPMM_FP8_E4M3 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                         : (h->dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
             CUresult r = fn(&h->tmB3, dt, 3, const_cast<void*>(B), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                             swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             h->tmB3_ok = r == CUDA_SUCCESS;
@@ -601,7 +614,7 @@ int spmm_bcsr_create_coo(spmm_handle_t* out, int64_t m, int64_t k, int64_t nnz, 
                          const int32_t* cols, const void* vals, int dtype, int block, const spmm_opts_t* opts) {
     if (!out) return SPMM_ERR_INVALID_ARG;
     *out = nullptr;
-    if (dtype < 0 || dtype > 2) return SPMM_ERR_INVALID_ARG;
+    if (dtype < 0 || dtype > 3) return SPMM_ERR_INVALID_ARG;
     CsrOwned o;
     int rc;
     try {
@@ -628,7 +641,7 @@ int spmm_wcsr_create_coo(spmm_handle_t* out, int64_t m, int64_t k, int64_t nnz, 
                          const spmm_opts_t* opts) {
     if (!out) return SPMM_ERR_INVALID_ARG;
     *out = nullptr;
-    if (dtype < 0 || dtype > 2) return SPMM_ERR_INVALID_ARG;
+    if (dtype < 0 || dtype > 3) return SPMM_ERR_INVALID_ARG;
     CsrOwned o;
     int rc;
     try {

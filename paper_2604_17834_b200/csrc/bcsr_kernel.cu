@@ -46,23 +46,26 @@ namespace {
 template <int B, int CT, int CM>
 struct EpiCols { static constexpr int value = bcsr_epi_cols(B, CT != 0, CM != 0); };
 
-template <int B, int GROUPS, int STAGES>
+// ES = bytes per input element: 2 (fp16 / bf16), or 1 (E4M3, column-major operands only).
+template <int B, int GROUPS, int STAGES, int ES>
 struct BcsrCfg {
+    static constexpr int kBB = B * ES;                       // bytes of one block row (its K extent)
+    static constexpr int kKSteps = kBB / 32;                 // MMAs per block and token group (32 bytes of K each)
     static constexpr int kBnT = 128 * GROUPS;
-    static constexpr int kNBox = 2 * GROUPS;                 // 64-token boxes per block
-    static constexpr int kBoxBytes = B * 128;                // b k-rows x 128 B
-    static constexpr int kDenseBytes = kNBox * kBoxBytes;    // B tile of one block
-    static constexpr int kABytes = B * B * 2;
+    static constexpr int kNBox = 2 * GROUPS;                 // 64-token boxes per block (row-major B)
+    static constexpr int kBoxBytes = B * 128;                // b k-rows x 128 B (row-major B, 2-byte elements)
+    static constexpr int kDenseBytes = kBnT * kBB;           // B tile of one block
+    static constexpr int kABytes = B * kBB;
     // Small blocks carry too little work for the fixed cost of a pipeline stage (barrier
     // round trip, request issue, MMA hand-off): a stage holds several consecutive stored
     // blocks of the block-row, their B tiles first, then their A blocks (one request).
     static constexpr int kBps = bcsr_blocks_per_stage(B);
     static constexpr int kStageBytes = ((kBps * (kDenseBytes + kABytes) + 1023) / 1024) * 1024;
     static constexpr int kAOff = kBps * kDenseBytes;         // A blocks inside the stage
-    static constexpr int kARowBytes = (B < 64 ? B : 64) * 2;
+    static constexpr int kARowBytes = kBB < 128 ? kBB : 128;
     static constexpr uint32_t kASwizzle = kARowBytes == 128 ? SWZ_128B : (kARowBytes == 64 ? SWZ_64B : SWZ_32B);
     // column-major operands: a token group's tile is 128 rows x kXRowBytes, K-major
-    static constexpr int kXRowBytes = (B < 64 ? B : 64) * 2;
+    static constexpr int kXRowBytes = kARowBytes;
     static constexpr int kXGroupBytes = 128 * kXRowBytes;    // one K half of one token group
     static constexpr int kAccCols = GROUPS * B;
     static constexpr int kTmemCols = (2 * kAccCols <= 32) ? 32 : (2 * kAccCols <= 64 ? 64 : (2 * kAccCols <= 128 ? 128 : (2 * kAccCols <= 256 ? 256 : 512)));
@@ -73,6 +76,7 @@ struct BcsrCfg {
     static_assert(kSmemBytes <= 227 * 1024, "stage ring exceeds shared memory");
     static_assert((2 * STAGES + 7 + 8) * 8 + 64 <= kBarrierBytes, "barrier area");
     static_assert(kBps == 1 || B <= 32, "multi-block stages are for the small block sizes");
+    static_assert(kBB % 32 == 0, "a block row must hold whole K steps");
 };
 
 constexpr int kSchedDepth = 4;      // tile indices fetched ahead by the dynamic scheduler
@@ -81,7 +85,9 @@ template <int B, int GROUPS, int STAGES, int FMT, int CT, int CM, int DYN>
 __global__ void __launch_bounds__(DYN ? 224 : 192, 1)
 bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ CUtensorMap tmC, const BcsrParams p) {
-    using Cfg = BcsrCfg<B, GROUPS, STAGES>;
+    constexpr int ES = FMT == 3 ? 1 : 2;
+    static_assert(ES == 2 || CM, "8-bit inputs: column-major operands only");
+    using Cfg = BcsrCfg<B, GROUPS, STAGES, ES>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -199,27 +205,27 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         TRACE_ADD(tr_empty, tr_a);
                         const uint32_t sb = smem_base + s * Cfg::kStageBytes;
                         // the A request always brings kBps blocks (the box of the tensor map)
-                        const uint32_t dense_tx = CM ? (whole_tile ? Cfg::kDenseBytes : ((nvalid + 127) >> 7) * (B * 256))
+                        const uint32_t dense_tx = CM ? (whole_tile ? Cfg::kDenseBytes : ((nvalid + 127) >> 7) * (128 * Cfg::kBB))
                                                      : nbox * Cfg::kBoxBytes;
                         if (lane == 0) mbar_arrive_expect_tx(full_bar(s), Cfg::kBps * Cfg::kABytes + nb * dense_tx);
                         __syncwarp();
                         if constexpr (CM) {
                             // X as [N / 128][128][k]: box = GROUPS x 128 tokens x min(b, 64) elements
                             // of block column J (b = 128: lanes nb.. fetch the second K half)
-                            constexpr int kHalves = B > 64 ? 2 : 1;
+                            constexpr int kHalves = Cfg::kBB > 128 ? 2 : 1;
                             const int blk = lane % Cfg::kBps, hf = lane / Cfg::kBps;
                             const int J = __shfl_sync(0xffffffffu, Jl, jq + (blk < nb ? blk : 0));
                             if (whole_tile) {
                                 if (blk < nb && hf < kHalves)
                                     tma_load_3d_hint(sb + blk * Cfg::kDenseBytes + hf * (GROUPS * Cfg::kXGroupBytes), &tmB3,
-                                                     full_bar(s), J * B + hf * 64, 0, n0 >> 7, keep);
+                                                     full_bar(s), J * B + hf * (128 / ES), 0, n0 >> 7, keep);
                             } else {
                                 // ragged tile: one request per 128-token group, rows >= N are zero filled
                                 const int ngrp = (nvalid + 127) >> 7;
                                 for (int g = 0; g < ngrp; ++g)
                                     if (blk < nb && hf < kHalves)
                                         tma_load_2d_hint(sb + blk * Cfg::kDenseBytes + hf * (GROUPS * Cfg::kXGroupBytes) + g * Cfg::kXGroupBytes,
-                                                         &tmB, full_bar(s), J * B + hf * 64, n0 + g * 128, keep);
+                                                         &tmB, full_bar(s), J * B + hf * (128 / ES), n0 + g * 128, keep);
                             }
                         } else
                         if (whole_tile) {
@@ -237,8 +243,8 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         }
                         if (lane == 8) {
                             tma_load_2d_hint(sb + Cfg::kAOff, &tmA, full_bar(s), 0, q * B, keep);
-                        } else if (B > 64 && lane == 9) {
-                            tma_load_2d_hint(sb + Cfg::kAOff + B * 128, &tmA, full_bar(s), 64, q * B, keep);
+                        } else if (Cfg::kBB > 128 && lane == 9) {
+                            tma_load_2d_hint(sb + Cfg::kAOff + B * 128, &tmA, full_bar(s), 128 / ES, q * B, keep);
                         }
                     }
                 }
@@ -263,7 +269,8 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // Warp-uniform control flow (all lanes wait and compute the uniform descriptors); one
         // elected lane issues the tcgen05 instructions.
         {
-            constexpr uint32_t idesc = make_idesc(FMT, 128, B, CM ? 0 : 1, 0);
+            // 8-bit floats: format code 0 = E4M3 in both operand fields
+            constexpr uint32_t idesc = make_idesc(FMT == 3 ? 0 : FMT, 128, B, CM ? 0 : 1, 0);
             const uint64_t adesc0 = CM ? make_smem_desc(0, 16, 8 * Cfg::kXRowBytes, Cfg::kASwizzle)
                                        : make_smem_desc(0, Cfg::kBoxBytes, 1024, SWZ_128B);
             const uint64_t bdesc0 = make_smem_desc(0, 16, 8 * Cfg::kARowBytes, Cfg::kASwizzle);
@@ -308,13 +315,13 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             const uint64_t b0 = bdesc0 + ((sb + Cfg::kAOff + i * Cfg::kABytes) >> 4);
                             const uint32_t accum0 = (q > pb || i > 0) ? 1u : 0u;
 #pragma unroll
-                            for (int ks = 0; ks < B / 16; ++ks) {
-                                const uint32_t boff = B <= 64 ? ks * 32 : (ks >> 2) * (B * 128) + (ks & 3) * 32;
+                            for (int ks = 0; ks < Cfg::kKSteps; ++ks) {
+                                const uint32_t boff = Cfg::kBB <= 128 ? ks * 32 : (ks >> 2) * (B * 128) + (ks & 3) * 32;
 #pragma unroll
                                 for (int g = 0; g < GROUPS; ++g)
                                     if (leader && g < ngrp)
-                                        umma_ss<false>(d0 + g * B,
-                                                       a0 + ((CM ? (B <= 64 ? g * Cfg::kXGroupBytes + ks * 32
+                                        umma_kind<FMT == 3 ? 2 : 0>(d0 + g * B,
+                                                       a0 + ((CM ? (Cfg::kBB <= 128 ? g * Cfg::kXGroupBytes + ks * 32
                                                                             : (ks >> 2) * (GROUPS * Cfg::kXGroupBytes) + g * Cfg::kXGroupBytes + (ks & 3) * 32)
                                                                  : g * 2 * Cfg::kBoxBytes + ks * 2048) >> 4),
                                                        b0 + (boff >> 4), idesc, ks > 0 ? 1u : accum0);
@@ -488,7 +495,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 template <int B, int GROUPS, int STAGES, int FMT, int CT, int CM, int DYN>
 cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p,
                        int grid, cudaStream_t stream) {
-    using Cfg = BcsrCfg<B, GROUPS, STAGES>;
+    using Cfg = BcsrCfg<B, GROUPS, STAGES, FMT == 3 ? 1 : 2>;
     auto kfn = bcsr_spmm_kernel<B, GROUPS, STAGES, FMT, CT, CM, DYN>;
     static bool attr_done = false;
     if (!attr_done) {
@@ -519,6 +526,23 @@ cudaError_t launch_shape(int b, int groups, const CUtensorMap& tmA, const CUtens
     }
 }
 
+// E4M3 inputs: column-major operands, fp32 C, static schedule; b = 32, 64 or 128 (a block row
+// must hold at least one 32-element K step).  Stages are half the bytes of the 16-bit ones.
+cudaError_t launch_fp8(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
+                       const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
+    switch (b * 10 + groups) {
+        case 321: return launch_one<32, 1, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 322: return launch_one<32, 2, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 324: return launch_one<32, 4, 6, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 641: return launch_one<64, 1, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 642: return launch_one<64, 2, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 644: return launch_one<64, 4, 5, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 1281: return launch_one<128, 1, 6, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 1282: return launch_one<128, 2, 4, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
 template <int FMT>
 cudaError_t launch_fmt(int b, int groups, int c16, int cm, int dyn, const CUtensorMap& tmA, const CUtensorMap& tmB,
                        const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
@@ -539,6 +563,8 @@ cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, in
                         int grid, cudaStream_t stream) {
     if (dtype == 1) return launch_fmt<0>(b, groups, c16, col_major, dynamic, tmA, tmB, tmB3, tmC, p, grid, stream);   // fp16
     if (dtype == 0) return launch_fmt<1>(b, groups, c16, col_major, dynamic, tmA, tmB, tmB3, tmC, p, grid, stream);   // bf16
+    if (dtype == 3) return (c16 || !col_major || dynamic) ? cudaErrorInvalidValue
+                                                           : launch_fp8(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
     return cudaErrorInvalidValue;
 }
 

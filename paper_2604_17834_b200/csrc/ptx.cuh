@@ -336,16 +336,27 @@ __host__ __device__ constexpr uint32_t make_idesc(uint32_t fmt, uint32_t m, uint
            ((n >> 3) << 17) | ((m >> 4) << 24);
 }
 
-// D[tmem] (+)= A[smem] * B[smem]; one thread issues.  kTf32 selects kind::tf32, else kind::f16.
-template <bool kTf32>
-__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
-                                        uint32_t idesc, uint32_t accumulate) {
-    if constexpr (kTf32) {
+// D[tmem] (+)= A[smem] * B[smem]; one thread issues.  kKind selects the instruction kind:
+// 0 = kind::f16 (fp16 / bf16, K = 16), 1 = kind::tf32 (K = 8), 2 = kind::f8f6f4 (8-bit floats,
+// K = 32; the element formats are in the instruction descriptor, 0 = E4M3).
+template <int kKind>
+__device__ __forceinline__ void umma_kind(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate) {
+    if constexpr (kKind == 1) {
         asm volatile(
             "{\n\t"
             ".reg .pred p;\n\t"
             "setp.ne.b32 p, %4, 0;\n\t"
             "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t"
+            "}\n"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else if constexpr (kKind == 2) {
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t"
             "}\n"
             ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
             : "memory");
@@ -359,6 +370,11 @@ __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64
             ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
             : "memory");
     }
+}
+template <bool kTf32>
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                        uint32_t idesc, uint32_t accumulate) {
+    umma_kind<kTf32 ? 1 : 0>(d_tmem, a_desc, b_desc, idesc, accumulate);
 }
 
 // ----------------------------------------------------------------------------- cluster launch control

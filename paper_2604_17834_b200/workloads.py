@@ -20,13 +20,15 @@ Stand-ins (the paper's own data is not available here):
 
 Storage dtypes: "bf16" travels as uint16 bit patterns (numpy has no
 bfloat16), "fp16" as numpy.float16, "tf32" as numpy.float32 (fp32 storage,
-TF32 tensor-core arithmetic).
+TF32 tensor-core arithmetic), "fp8" as uint8 bit patterns of E4M3 (1 sign,
+4 exponent bits with bias 7, 3 mantissa bits; no infinities, largest finite
+value 448; the all-ones exponent-and-mantissa code is NaN and never drawn).
 """
 from __future__ import annotations
 
 import numpy as np
 
-DTYPES = ("bf16", "fp16", "tf32")
+DTYPES = ("bf16", "fp16", "tf32", "fp8")
 
 
 # --------------------------------------------------------------------------- dtype helpers
@@ -43,7 +45,23 @@ def to_storage(x, dtype):
         u = x32.view(np.uint32)
         rounded = u + (np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1)))
         return (rounded >> np.uint32(16)).astype(np.uint16)
+    if dtype == "fp8":
+        # nearest E4M3 value, ties to the even code, saturating at +-448
+        mag = _e4m3_magnitudes()                              # codes 0..126, ascending
+        ax = np.minimum(np.abs(x32.astype(np.float64)), mag[-1])
+        hi = np.clip(np.searchsorted(mag, ax, side="left"), 1, mag.shape[0] - 1)
+        lo = hi - 1
+        dlo, dhi = ax - mag[lo], mag[hi] - ax
+        code = np.where(dlo < dhi, lo, np.where(dhi < dlo, hi, np.where(lo % 2 == 0, lo, hi)))
+        return (code.astype(np.uint8) | (np.signbit(x32).astype(np.uint8) << np.uint8(7))).astype(np.uint8)
     raise ValueError(dtype)
+
+
+def _e4m3_magnitudes():
+    """Values of the E4M3 codes 0 .. 126 (sign bit clear, NaN code 127 left out)."""
+    code = np.arange(127)
+    e, m = code >> 3, code & 7
+    return np.where(e == 0, m / 8.0 * 2.0 ** -6, (1.0 + m / 8.0) * 2.0 ** (e.astype(np.float64) - 7.0))
 
 
 def widen(s, dtype):
@@ -51,15 +69,18 @@ def widen(s, dtype):
     s = np.asarray(s)
     if dtype == "bf16":
         return (s.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    if dtype == "fp8":
+        mag = np.append(_e4m3_magnitudes(), np.nan)
+        return np.where(s >> 7 == 1, -1.0, 1.0) * mag[s & 0x7F]
     return s.astype(np.float64)
 
 
 def elem_size(dtype):
-    return 4 if dtype == "tf32" else 2
+    return {"tf32": 4, "fp8": 1}.get(dtype, 2)
 
 
 def storage_np_dtype(dtype):
-    return {"bf16": np.uint16, "fp16": np.float16, "tf32": np.float32}[dtype]
+    return {"bf16": np.uint16, "fp16": np.float16, "tf32": np.float32, "fp8": np.uint8}[dtype]
 
 
 def dense(seed, rows, cols, dist, dtype, chunk_rows=4096):

@@ -3,14 +3,14 @@ compare it element by element with the fp64 oracle under the stated bound
 
     |C_gpu - C_ref| <= tau * sum_k |a_ik b_kj| + 1e-6,
 
-tau = 8e-3 for bf16 / fp16 inputs, 2e-3 for the TF32 path (fp32 accumulation).
+tau = 8e-3 for bf16 / fp16 (and E4M3) inputs, 2e-3 for the TF32 path (fp32 accumulation).
 """
 import numpy as np
 
 from oracle import spmm_ref
 from paper_2604_17834_b200 import workloads as wl
 
-TAU = {"bf16": 8e-3, "fp16": 8e-3, "tf32": 2e-3}
+TAU = {"bf16": 8e-3, "fp16": 8e-3, "tf32": 2e-3, "fp8": 8e-3}
 
 
 def to_device(arr):

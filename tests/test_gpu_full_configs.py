@@ -95,6 +95,14 @@ def test_config2_bcsr_llm_variants_full(lib, shape, c16, col_major):
                    what="configs[2] %s c16=%d cm=%d" % (shape, c16, col_major))
 
 
+def test_config2_bcsr_llm_fp8_full(lib):
+    """configs[2] gate shape with E4M3 weights and activations (column-major operands, fp32 Y)."""
+    a = wl.bcsr_llm(dtype="fp8", std=0.5)
+    N = 65536
+    Bs = wl.dense(1103, a["k"], N, ("normal", 0.0, 1.0), "fp8", chunk_rows=256)
+    _run_and_check(lib, "bcsr", a, "fp8", 64, N, Bs, cols=_sample_cols(N, 3), col_major=True, what="configs[2] gate fp8")
+
+
 @pytest.mark.parametrize("b,d,skewed", [(16, 0.1, True), (32, 0.2, True), (64, 0.1, True), (128, 0.05, True),
                                          (64, 0.05, False), (16, 0.01, False), (128, 0.5, True)])
 def test_config3_bcsr_sweep_full(lib, b, d, skewed):

@@ -174,6 +174,28 @@ def test_bcsr_dynamic_schedule_matches_static_bitwise(lib, b, N):
         lib.spmm_destroy(h1)
 
 
+@pytest.mark.parametrize("b", [32, 64, 128])
+@pytest.mark.parametrize("N", [640, 333, 128])
+def test_bcsr_fp8_e4m3_colmajor(lib, b, N):
+    """8-bit E4M3 inputs (the next step Sec. 5 names), K-major operands: X [N][k] and the stored
+    blocks as E4M3, fp32 accumulation and output.  Products of two E4M3 values are exact in
+    fp32, so the 16-bit bound applies unchanged."""
+    a = wl.bcsr_sweep(900 + b, m=1024, k=768, b=b, density=0.2, dtype="fp8")
+    Bs = wl.dense(37, a["k"], N, ("uniform", -1.0, 1.0), "fp8")
+    h = lib.spmm_bcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "fp8", b, layout=lib.COLMAJOR)
+    try:
+        from oracle import formats as F
+        f = F.bcsr_from_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], b)
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCK_COL_IDX, np.int32), f["block_col_idx"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCKS, np.uint8), f["blocks"].ravel())
+        C = run_gpu_variant(lib, h, Bs, a["m"], N, "fp8", col_major=True)
+        Cr, S = reference(a, Bs, "fp8")
+        assert_close(C, Cr, S, "fp8", "bcsr fp8 b=%d N=%d" % (b, N))
+        assert np.array_equal(C, run_gpu_variant(lib, h, Bs, a["m"], N, "fp8", col_major=True))
+    finally:
+        lib.spmm_destroy(h)
+
+
 def test_variant_argument_errors(lib):
     a = wl.bcsr_tiny()
     args = (512, 512, a["row_ptr"], a["col_idx"], a["vals"], "bf16")
@@ -188,6 +210,14 @@ def test_variant_argument_errors(lib):
     assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
     with pytest.raises(lib.SpmmError) as e:
         lib.spmm_wcsr_create_csr(*args, 16, schedule=lib.SCHED_DYNAMIC)
+    assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
+    a8 = wl.bcsr_sweep(5, m=256, k=256, b=32, density=0.3, dtype="fp8")
+    for kw in (dict(), dict(layout=lib.COLMAJOR, c_type=lib.C_SAME_AS_INPUT)):    # E4M3: column-major, fp32 C only
+        with pytest.raises(lib.SpmmError) as e:
+            lib.spmm_bcsr_create_csr(256, 256, a8["row_ptr"], a8["col_idx"], a8["vals"], "fp8", 32, **kw)
+        assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
+    with pytest.raises(lib.SpmmError) as e:
+        lib.spmm_bcsr_create_csr(256, 256, a8["row_ptr"], a8["col_idx"], a8["vals"], "fp8", 16, layout=lib.COLMAJOR)
     assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
     b = wl.random_csr(3, 100, 64, 0.1, "bf16")                             # m = 100: not a multiple of 8
     with pytest.raises(lib.SpmmError) as e:

@@ -130,3 +130,21 @@ def test_matches_scipy_on_a_medium_matrix():
 def test_rejects_out_of_range_column():
     with pytest.raises(ValueError):
         spmm_ref(np.array([0, 1], np.int64), np.array([3], np.int32), np.ones(1), np.ones((3, 2)))
+
+
+def test_e4m3_storage_matches_an_independent_conversion():
+    """The E4M3 quantiser of the input generators (nearest, ties to even) against torch's
+    float8_e4m3fn cast, and its decoder against torch's widening, on values inside the finite
+    range; saturation and the sign of zero separately."""
+    import torch
+    rng = np.random.default_rng(12)
+    x = np.concatenate([rng.standard_normal(50000).astype(np.float32) * 3.0,
+                        rng.standard_normal(50000).astype(np.float32) * 0.01,
+                        np.array([0.0, 448.0, -448.0, 2.0 ** -9, 2.0 ** -10, 1.0625, 1.1875, 0.4375 + 2.0 ** -5], np.float32)])
+    code = wl.to_storage(x, "fp8")
+    t = torch.from_numpy(x).to(torch.float8_e4m3fn)
+    assert np.array_equal(code, t.view(torch.uint8).numpy())
+    assert np.array_equal(wl.widen(code, "fp8"), t.float().numpy().astype(np.float64))
+    assert wl.widen(wl.to_storage(np.array([1e6, -1e6], np.float32), "fp8"), "fp8").tolist() == [448.0, -448.0]
+    z = wl.to_storage(np.array([-0.0], np.float32), "fp8")
+    assert z[0] == 0x80 and np.signbit(wl.widen(z, "fp8"))[0]
