@@ -173,6 +173,18 @@ int spmm_bcsr_create_csr(spmm_handle_t *out, int64_t m, int64_t k, const int64_t
                          const int32_t *col_idx, const void *vals, int dtype, int block,
                          const spmm_opts_t *opts);
 
+/*
+ * Same handle, built on the GPU from a CSR matrix that already lives in DEVICE memory
+ * (block mask, index and value packing of Sec. 2.3 as kernels; the paper builds its formats
+ * offline).  row_ptr_dev / col_idx_dev / vals_dev are device pointers with the layout of
+ * spmm_bcsr_create_csr; the caller keeps them.  The CSR is validated on the device (same
+ * error codes).  The call runs on `stream` (a cudaStream_t as void*, NULL = default) and
+ * synchronises it; opts.host_only is not allowed.  Limit: ceil(k / block) <= 819,200.
+ */
+int spmm_bcsr_create_csr_device(spmm_handle_t *out, int64_t m, int64_t k, const int64_t *row_ptr_dev,
+                                const int32_t *col_idx_dev, const void *vals_dev, int dtype, int block,
+                                const spmm_opts_t *opts, void *stream);
+
 /* Same from COO: host int32 rows[nnz], cols[nnz] in any order, no duplicate (row, col). */
 int spmm_bcsr_create_coo(spmm_handle_t *out, int64_t m, int64_t k, int64_t nnz,
                          const int32_t *rows, const int32_t *cols, const void *vals, int dtype,

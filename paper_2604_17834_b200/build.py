@@ -16,7 +16,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 OUT = os.path.join(HERE, "libspmm_b200.so")
 OBJDIR = os.path.join(CSRC, "build")
-SOURCES = ["api.cu", "bcsr_kernel.cu", "wcsr_kernel.cu", "format.cpp"]
+SOURCES = ["api.cu", "bcsr_kernel.cu", "wcsr_kernel.cu", "format_gpu.cu", "format.cpp"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -180,7 +180,8 @@ int check_opts(const spmm_opts_t* opts) {
     return SPMM_OK;
 }
 
-int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, const spmm_opts_t* opts) {
+// Option checks shared by the host and the device builder; on success *hp is a fresh handle.
+int new_bcsr_handle(spmm_handle_s** hp, int64_t m, int64_t k, int dtype, int block, const spmm_opts_t* opts) {
     if (dtype != SPMM_BF16 && dtype != SPMM_FP16 && dtype != SPMM_FP8_E4M3) return SPMM_ERR_UNSUPPORTED;
     if (int orc = check_opts(opts)) return orc;
     if (dtype == SPMM_FP8_E4M3) {
@@ -188,18 +189,15 @@ int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, cons
         // row must hold a whole 32-element K step; rows of X are k bytes and must be multiples of 16
         if (!opts || opts->layout != SPMM_COLMAJOR || opts->c_type != SPMM_C_FP32 || opts->schedule != SPMM_SCHED_STATIC)
             return SPMM_ERR_UNSUPPORTED;
-        if (block < 32 || a.k % 16 != 0) return SPMM_ERR_UNSUPPORTED;
+        if (block < 32 || k % 16 != 0) return SPMM_ERR_UNSUPPORTED;
     }
-    int rc = validate_csr(a);
-    if (rc) return rc;
     spmm_handle_s* h = new (std::nothrow) spmm_handle_s;
     if (!h) return SPMM_ERR_ALLOC;
     h->format = 0;
     h->dtype = dtype;
-    h->es = a.es;
-    h->m = a.m;
-    h->k = a.k;
-    h->nnz = a.nnz;
+    h->es = elem_size(dtype);
+    h->m = m;
+    h->k = k;
     h->host_only = opts && opts->host_only;
     h->c16 = opts && opts->c_type == SPMM_C_SAME_AS_INPUT;
     h->cs = h->c16 ? 2 : 4;
@@ -208,7 +206,33 @@ int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, cons
     if (h->dynamic && (h->c16 || h->col_major)) { delete h; return SPMM_ERR_UNSUPPORTED; }
     // column-major operands: rows of X (k elements) and of Y (m elements) must be multiples of
     // 16 bytes for the tensor map and for the 16-byte pieces the epilogue writes
-    if (h->col_major && (a.m % 8 != 0 || a.k % 8 != 0)) { delete h; return SPMM_ERR_UNSUPPORTED; }
+    if (h->col_major && (m % 8 != 0 || k % 8 != 0)) { delete h; return SPMM_ERR_UNSUPPORTED; }
+    *hp = h;
+    return SPMM_OK;
+}
+
+// Tensor map of the stored blocks: box rows of min(b * es, 128) bytes, swizzle = the row bytes.
+int encode_tmA(spmm_handle_s* h) {
+    const BcsrHost& f = h->bcsr;
+    if (f.nnzb <= 0) return SPMM_OK;
+    if (static_cast<int64_t>(f.nnzb) * f.b >= (int64_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
+    const int row_bytes = f.b * h->es < 128 ? f.b * h->es : 128;
+    const int bw = row_bytes / h->es;
+    const CUtensorMapSwizzle swz = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                  : (row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+    int rc = encode_2d_16bit(&h->tmA, h->dtype, h->d_vals, static_cast<uint64_t>(f.nnzb) * f.b, f.b,
+                             static_cast<uint32_t>(f.b * bcsr_blocks_per_stage(f.b)), bw, swz);
+    h->tmA_ok = rc == SPMM_OK;
+    return rc;
+}
+
+int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, const spmm_opts_t* opts) {
+    spmm_handle_s* h = nullptr;
+    int rc = new_bcsr_handle(&h, a.m, a.k, dtype, block, opts);
+    if (rc) return rc;
+    rc = validate_csr(a);
+    if (rc) { delete h; return rc; }
+    h->nnz = a.nnz;
     rc = device_setup(h, opts);
     if (rc) { free_handle(h); return rc; }
     try {
@@ -224,19 +248,32 @@ int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, cons
         if (!rc) rc = upload(&h->d_idx, f.block_col_idx.data(), f.block_col_idx.size() * 4);
         if (!rc) rc = upload(&h->d_vals, f.blocks.data(), f.blocks.size());
         if (!rc) rc = upload(&h->d_order, f.row_order.data(), f.row_order.size() * 4);
-        if (!rc && f.nnzb > 0) {
-            // box rows of min(b * es, 128) bytes, swizzle = the row bytes
-            const int row_bytes = f.b * h->es < 128 ? f.b * h->es : 128;
-            const int bw = row_bytes / h->es;
-            const CUtensorMapSwizzle swz = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
-                                          : (row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
-            rc = encode_2d_16bit(&h->tmA, dtype, h->d_vals, static_cast<uint64_t>(f.nnzb) * f.b, f.b,
-                                 static_cast<uint32_t>(f.b * bcsr_blocks_per_stage(f.b)), bw, swz);
-            h->tmA_ok = rc == SPMM_OK;
-        }
+        if (!rc) rc = encode_tmA(h);
         if (rc) { free_handle(h); return rc; }
         std::vector<uint8_t>().swap(h->bcsr.blocks);   // the device copy is the one that counts
     }
+    *out = h;
+    return SPMM_OK;
+}
+
+// The same handle from a CSR matrix in device memory: the format is built by GPU kernels.
+int create_bcsr_device(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* d_row_ptr, const int32_t* d_col_idx,
+                       const void* d_vals, int dtype, int block, const spmm_opts_t* opts, cudaStream_t stream) {
+    if (opts && opts->host_only) return SPMM_ERR_INVALID_ARG;
+    spmm_handle_s* h = nullptr;
+    int rc = new_bcsr_handle(&h, m, k, dtype, block, opts);
+    if (rc) return rc;
+    rc = device_setup(h, opts);
+    if (rc) { free_handle(h); return rc; }
+    try {
+        rc = build_bcsr_device(m, k, d_row_ptr, d_col_idx, static_cast<const uint8_t*>(d_vals), h->es, block, stream,
+                               &h->bcsr, &h->nnz, &h->d_ptr, &h->d_idx, &h->d_vals);
+    } catch (const std::bad_alloc&) {
+        rc = SPMM_ERR_ALLOC;
+    }
+    if (!rc) rc = upload(&h->d_order, h->bcsr.row_order.data(), h->bcsr.row_order.size() * 4);
+    if (!rc) rc = encode_tmA(h);
+    if (rc) { free_handle(h); return rc; }
     *out = h;
     return SPMM_OK;
 }
@@ -608,6 +645,16 @@ int spmm_bcsr_create_csr(spmm_handle_t* out, int64_t m, int64_t k, const int64_t
     int rc = make_view(&v, m, k, row_ptr, col_idx, vals, dtype);
     if (rc) return rc;
     return create_bcsr(out, v, dtype, block, opts);
+}
+
+int spmm_bcsr_create_csr_device(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* row_ptr_dev,
+                                const int32_t* col_idx_dev, const void* vals_dev, int dtype, int block,
+                                const spmm_opts_t* opts, void* stream) {
+    if (!out) return SPMM_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (dtype < 0 || dtype > 3 || m < 0 || k < 0 || !row_ptr_dev) return SPMM_ERR_INVALID_ARG;
+    if (m >= (int64_t{1} << 31) || k >= (int64_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
+    return create_bcsr_device(out, m, k, row_ptr_dev, col_idx_dev, vals_dev, dtype, block, opts, static_cast<cudaStream_t>(stream));
 }
 
 int spmm_bcsr_create_coo(spmm_handle_t* out, int64_t m, int64_t k, int64_t nnz, const int32_t* rows,

@@ -74,7 +74,6 @@ int build_bcsr(const CsrView& a, int b, BcsrHost* out) {
 
     // pass 1: which block columns each block-row touches (structural: any stored entry)
     std::vector<int64_t> stamp(static_cast<size_t>(nbc), -1);
-    std::vector<uint8_t> col_used(static_cast<size_t>(nbc), 0);
     std::vector<int32_t> found;
     for (int64_t I = 0; I < nbr; ++I) {
         found.clear();
@@ -88,14 +87,12 @@ int build_bcsr(const CsrView& a, int b, BcsrHost* out) {
                 }
             }
         std::sort(found.begin(), found.end());
-        for (int32_t J : found) col_used[J] = 1;
         out->block_col_idx.insert(out->block_col_idx.end(), found.begin(), found.end());
         if (out->block_col_idx.size() >= (size_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
         out->block_row_ptr[I + 1] = static_cast<int32_t>(out->block_col_idx.size());
     }
     const int64_t nnzb = static_cast<int64_t>(out->block_col_idx.size());
     out->nnzb = nnzb;
-    out->distinct_bcols = std::count(col_used.begin(), col_used.end(), uint8_t{1});
 
     // pass 2: scatter the values into their dense tiles
     const size_t tile_bytes = static_cast<size_t>(b) * b * a.es;
@@ -114,17 +111,7 @@ int build_bcsr(const CsrView& a, int b, BcsrHost* out) {
             }
     }
 
-    // schedule: block-rows with the most stored blocks first, ties by index
-    out->row_order.resize(static_cast<size_t>(nbr));
-    std::iota(out->row_order.begin(), out->row_order.end(), 0);
-    std::stable_sort(out->row_order.begin(), out->row_order.end(), [&](int32_t x, int32_t y) {
-        const int32_t lx = out->block_row_ptr[x + 1] - out->block_row_ptr[x];
-        const int32_t ly = out->block_row_ptr[y + 1] - out->block_row_ptr[y];
-        return lx > ly;
-    });
-    out->n_empty = 0;
-    for (int64_t I = 0; I < nbr; ++I)
-        if (out->block_row_ptr[I + 1] == out->block_row_ptr[I]) out->n_empty++;
+    finish_bcsr_host(out);      // row order (most stored blocks first, ties by index), empty rows, distinct columns
     return SPMM_OK;
 }
 

@@ -3,6 +3,8 @@
 // the static schedules (Sec. 2.3 formats; Sec. 3.3 task decomposition).
 #pragma once
 
+#include <cuda_runtime.h>
+
 #include <cstdint>
 #include <vector>
 
@@ -84,6 +86,14 @@ int validate_csr(const CsrView& a);
 int coo_to_csr(int64_t m, int64_t k, int64_t nnz, const int32_t* rows, const int32_t* cols,
                const uint8_t* vals, int es, CsrOwned* out);
 int build_bcsr(const CsrView& a, int b, BcsrHost* out);
+// Fills row_order, n_empty and distinct_bcols from the index arrays.
+void finish_bcsr_host(BcsrHost* out);
+// The same format built on the GPU from a CSR matrix in device memory (format_gpu.cu): validates the
+// CSR, allocates and fills the three device arrays (owned by the caller afterwards), and leaves the
+// index arrays and counts in *out (out->blocks stays empty).  Synchronises `stream`.
+int build_bcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int32_t* d_col_idx, const uint8_t* d_vals,
+                      int es, int b, cudaStream_t stream, BcsrHost* out, int64_t* nnz_out, int32_t** d_block_row_ptr,
+                      int32_t** d_block_col_idx, uint8_t** d_blocks);
 int build_bcsr_schedule(const BcsrHost& f, int n_tt, int slab_w, int n_ctas, BcsrSchedule* out);
 // T = 0 picks the sub-task size from the matrix: about a quarter of one bin's share of the
 // padded columns, rounded down to a multiple of 64 and clamped to [128, 4096].

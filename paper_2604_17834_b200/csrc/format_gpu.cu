@@ -1,0 +1,299 @@
+// GPU-side construction of the BCSR format (Sec. 2.3) from a CSR matrix that already lives in
+// device memory: block mask and index (which (I, J) blocks hold a stored entry, block columns
+// ascending inside a block-row) and value packing into zero-filled b x b tiles.  Same arrays,
+// bit for bit, as the host builder in format.cpp.
+//
+// One CTA per block-row.  The entries of a block-row are one contiguous range of the CSR
+// arrays (rows I*b .. I*b + b - 1), and its block columns are collected in a shared-memory
+// bitmap of ceil(k / b) bits:
+//   count pass   bitmap -> number of stored blocks of the block-row
+//   scan         exclusive prefix sum over block-rows -> block_row_ptr
+//   fill pass    bitmap again, prefix popcounts over its words -> block_col_idx (ascending by
+//                construction) and the slot of every entry's block; values scattered into
+//                blocks[slot][row in block][column in block]
+// A bitmap needs 2 * ceil(k / b) / 8 bytes of shared memory (bits + word prefix), at most 200 KB:
+// k / b <= 819,200.
+#include <cstring>
+#include <numeric>
+#include <algorithm>
+
+#include "format.h"
+#include "kernels.h"
+#include "spmm_b200.h"
+
+namespace spmm {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// Validation in two passes, so that the second one never reads past the arrays: once row_ptr is
+// known to start at 0 and to be monotone, every position below row_ptr[m] lies inside col_idx.
+__global__ void csr_check_rows_kernel(int64_t m, const int64_t* row_ptr, int* err) {
+    if (blockIdx.x == 0 && threadIdx.x == 0 && row_ptr[0] != 0) atomicMin(err, SPMM_ERR_INVALID_ARG);
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < m;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x)
+        if (row_ptr[i + 1] < row_ptr[i]) atomicMin(err, SPMM_ERR_INVALID_ARG);
+}
+
+__global__ void csr_check_cols_kernel(int64_t m, int64_t k, const int64_t* row_ptr, const int32_t* col_idx, int* err) {
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < m;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        int64_t prev = -1;
+        for (int64_t p = row_ptr[i]; p < row_ptr[i + 1]; ++p) {
+            const int64_t c = col_idx[p];
+            if (c < 0 || c >= k) { atomicMin(err, SPMM_ERR_OUT_OF_RANGE); break; }
+            if (c <= prev) { atomicMin(err, SPMM_ERR_UNSORTED); break; }
+            prev = c;
+        }
+    }
+}
+
+// Shared-memory bitmap of the block columns of block-row I.
+__device__ __forceinline__ void mark_block_columns(uint32_t* bits, int words, int64_t I, int64_t m, int b,
+                                                   const int64_t* row_ptr, const int32_t* col_idx) {
+    for (int w = threadIdx.x; w < words; w += blockDim.x) bits[w] = 0u;
+    __syncthreads();
+    const int64_t r1 = (I + 1) * b < m ? (I + 1) * b : m;
+    const int64_t p0 = row_ptr[I * b], p1 = row_ptr[r1];
+    for (int64_t p = p0 + threadIdx.x; p < p1; p += blockDim.x) {
+        const int J = col_idx[p] / b;
+        atomicOr(&bits[J >> 5], 1u << (J & 31));
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kThreads)
+bcsr_count_kernel(int64_t m, int b, int words, const int64_t* row_ptr, const int32_t* col_idx, int32_t* counts) {
+    extern __shared__ uint32_t smem[];
+    __shared__ int total;
+    if (threadIdx.x == 0) total = 0;
+    mark_block_columns(smem, words, blockIdx.x, m, b, row_ptr, col_idx);
+    int n = 0;
+    for (int w = threadIdx.x; w < words; w += blockDim.x) n += __popc(smem[w]);
+    for (int o = 16; o > 0; o >>= 1) n += __shfl_down_sync(0xffffffffu, n, o);
+    if ((threadIdx.x & 31) == 0 && n) atomicAdd(&total, n);
+    __syncthreads();
+    if (threadIdx.x == 0) counts[blockIdx.x] = total;
+}
+
+// out[0] = 0, out[i + 1] = counts[0] + ... + counts[i]; *overflow set if the total passes int32.
+__global__ void __launch_bounds__(1024)
+exclusive_scan_kernel(const int32_t* counts, int64_t n, int32_t* out, int* overflow) {
+    __shared__ long long warp_sum[32];
+    __shared__ long long carry;
+    if (threadIdx.x == 0) { carry = 0; out[0] = 0; }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int64_t base = 0; base < n; base += blockDim.x) {
+        const int64_t i = base + threadIdx.x;
+        long long v = i < n ? counts[i] : 0;
+        long long x = v;
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+        }
+        if (lane == 31) warp_sum[warp] = x;
+        __syncthreads();
+        if (warp == 0) {
+            long long s = warp_sum[lane];
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long y = __shfl_up_sync(0xffffffffu, s, o);
+                if (lane >= o) s += y;
+            }
+            warp_sum[lane] = s;
+        }
+        __syncthreads();
+        const long long incl = carry + (warp ? warp_sum[warp - 1] : 0) + x;
+        if (i < n) {
+            if (incl >= (1ll << 31)) *overflow = 1;
+            out[i + 1] = static_cast<int32_t>(incl);
+        }
+        __syncthreads();
+        if (threadIdx.x == blockDim.x - 1) carry = incl;
+        __syncthreads();
+    }
+}
+
+template <int ES>
+__global__ void __launch_bounds__(kThreads)
+bcsr_fill_kernel(int64_t m, int b, int words, const int64_t* row_ptr, const int32_t* col_idx, const uint8_t* vals,
+                 const int32_t* block_row_ptr, int32_t* block_col_idx, uint8_t* blocks) {
+    extern __shared__ uint32_t smem[];
+    uint32_t* bits = smem;
+    uint32_t* prefix = smem + words;         // set bits in the words before this one
+    __shared__ int warp_sum[kThreads / 32];
+    __shared__ int carry;
+    const int64_t I = blockIdx.x;
+    mark_block_columns(bits, words, I, m, b, row_ptr, col_idx);
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int base = 0; base < words; base += blockDim.x) {
+        const int w = base + threadIdx.x;
+        const int v = w < words ? __popc(bits[w]) : 0;
+        int x = v;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+        }
+        if (lane == 31) warp_sum[warp] = x;
+        __syncthreads();
+        if (warp == 0 && lane < kThreads / 32) {
+            int s = warp_sum[lane];
+            for (int o = 1; o < kThreads / 32; o <<= 1) {
+                const int y = __shfl_up_sync(0xffu, s, o);
+                if (lane >= o) s += y;
+            }
+            warp_sum[lane] = s;
+        }
+        __syncthreads();
+        const int incl = carry + (warp ? warp_sum[warp - 1] : 0) + x;
+        if (w < words) prefix[w] = static_cast<uint32_t>(incl - v);
+        __syncthreads();
+        if (threadIdx.x == blockDim.x - 1) carry = incl;
+        __syncthreads();
+    }
+    const int32_t slot0 = block_row_ptr[I];
+    // block columns, ascending: word by word, bit by bit
+    for (int w = threadIdx.x; w < words; w += blockDim.x) {
+        uint32_t x = bits[w];
+        int32_t pos = slot0 + static_cast<int32_t>(prefix[w]);
+        while (x) {
+            const int bit = __ffs(x) - 1;
+            block_col_idx[pos++] = w * 32 + bit;
+            x &= x - 1;
+        }
+    }
+    // values: one warp per row of the block-row
+    const int64_t r1 = (I + 1) * b < m ? (I + 1) * b : m;
+    const size_t tile_bytes = static_cast<size_t>(b) * b * ES;
+    for (int64_t i = I * b + warp; i < r1; i += kThreads / 32) {
+        const int64_t p0 = row_ptr[i], p1 = row_ptr[i + 1];
+        for (int64_t p = p0 + lane; p < p1; p += 32) {
+            const int c = col_idx[p];
+            const int J = c / b;
+            const uint32_t below = bits[J >> 5] & ((1u << (J & 31)) - 1u);
+            const size_t slot = static_cast<size_t>(slot0) + prefix[J >> 5] + __popc(below);
+            uint8_t* dst = blocks + slot * tile_bytes + (static_cast<size_t>(i - I * b) * b + (c - J * b)) * ES;
+            const uint8_t* src = vals + static_cast<size_t>(p) * ES;
+            if constexpr (ES == 1) *dst = *src;
+            else *reinterpret_cast<uint16_t*>(dst) = *reinterpret_cast<const uint16_t*>(src);
+        }
+    }
+}
+
+}  // namespace
+
+void finish_bcsr_host(BcsrHost* out) {
+    const int64_t nbr = out->nbr;
+    std::vector<uint8_t> col_used(static_cast<size_t>(out->nbc), 0);
+    for (int32_t J : out->block_col_idx) col_used[J] = 1;
+    out->distinct_bcols = std::count(col_used.begin(), col_used.end(), uint8_t{1});
+    out->row_order.resize(static_cast<size_t>(nbr));
+    std::iota(out->row_order.begin(), out->row_order.end(), 0);
+    std::stable_sort(out->row_order.begin(), out->row_order.end(), [&](int32_t x, int32_t y) {
+        const int32_t lx = out->block_row_ptr[x + 1] - out->block_row_ptr[x];
+        const int32_t ly = out->block_row_ptr[y + 1] - out->block_row_ptr[y];
+        return lx > ly;
+    });
+    out->n_empty = 0;
+    for (int64_t I = 0; I < nbr; ++I)
+        if (out->block_row_ptr[I + 1] == out->block_row_ptr[I]) out->n_empty++;
+}
+
+int build_bcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int32_t* d_col_idx, const uint8_t* d_vals,
+                      int es, int b, cudaStream_t st, BcsrHost* out, int64_t* nnz_out, int32_t** d_block_row_ptr,
+                      int32_t** d_block_col_idx, uint8_t** d_blocks) {
+    if (b != 16 && b != 32 && b != 64 && b != 128) return SPMM_ERR_UNSUPPORTED;
+    if (es != 1 && es != 2) return SPMM_ERR_UNSUPPORTED;
+    if (m < 0 || k < 0 || !d_row_ptr) return SPMM_ERR_INVALID_ARG;
+    const int64_t nbr = (m + b - 1) / b, nbc = (k + b - 1) / b;
+    const int words = static_cast<int>((nbc + 31) / 32);
+    const size_t smem = static_cast<size_t>(2) * (words > 0 ? words : 1) * 4;
+    if (smem > 200 * 1024) return SPMM_ERR_TOO_LARGE;
+    *d_block_row_ptr = nullptr;
+    *d_block_col_idx = nullptr;
+    *d_blocks = nullptr;
+    out->b = b;
+    out->nbr = nbr;
+    out->nbc = nbc;
+
+    int* d_flags = nullptr;                     // [0] CSR error code (min), [1] scan overflow
+    int32_t* d_counts = nullptr;
+    auto fail = [&](int code) {
+        cudaFree(d_flags);
+        cudaFree(d_counts);
+        cudaFree(*d_block_row_ptr);
+        cudaFree(*d_block_col_idx);
+        cudaFree(*d_blocks);
+        *d_block_row_ptr = nullptr;
+        *d_block_col_idx = nullptr;
+        *d_blocks = nullptr;
+        return code;
+    };
+    if (cudaMalloc(reinterpret_cast<void**>(&d_flags), 2 * sizeof(int)) != cudaSuccess) return fail(SPMM_ERR_ALLOC);
+    if (cudaMemsetAsync(d_flags, 0, 2 * sizeof(int), st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    if (cudaMalloc(reinterpret_cast<void**>(&d_counts), static_cast<size_t>(nbr + 1) * 4) != cudaSuccess) return fail(SPMM_ERR_ALLOC);
+    if (cudaMalloc(reinterpret_cast<void**>(d_block_row_ptr), static_cast<size_t>(nbr + 1) * 4) != cudaSuccess) return fail(SPMM_ERR_ALLOC);
+
+    // 1. the CSR must be canonical (the count and fill passes rely on in-range columns)
+    int64_t nnz = 0;
+    int flags[2] = {0, 0};
+    const unsigned check_grid = static_cast<unsigned>(std::min<int64_t>((m + 255) / 256, 2048));
+    if (m > 0) {
+        csr_check_rows_kernel<<<check_grid, 256, 0, st>>>(m, d_row_ptr, d_flags);
+        if (cudaMemcpyAsync(&nnz, d_row_ptr + m, sizeof(int64_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    }
+    if (cudaMemcpyAsync(flags, d_flags, sizeof(flags), cudaMemcpyDeviceToHost, st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    if (flags[0] != 0) return fail(flags[0]);
+    if (nnz < 0 || (nnz > 0 && (!d_col_idx || !d_vals))) return fail(SPMM_ERR_INVALID_ARG);
+    if (nnz > 0) {
+        csr_check_cols_kernel<<<check_grid, 256, 0, st>>>(m, k, d_row_ptr, d_col_idx, d_flags);
+        if (cudaMemcpyAsync(flags, d_flags, sizeof(flags), cudaMemcpyDeviceToHost, st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+        if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+        if (flags[0] != 0) return fail(flags[0]);
+    }
+    *nnz_out = nnz;
+
+    // 2. stored blocks per block-row, 3. block_row_ptr
+    if (smem > 48 * 1024) {
+        cudaFuncSetAttribute(bcsr_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        cudaFuncSetAttribute(bcsr_fill_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        cudaFuncSetAttribute(bcsr_fill_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    }
+    if (nbr > 0) bcsr_count_kernel<<<static_cast<unsigned>(nbr), kThreads, smem, st>>>(m, b, words, d_row_ptr, d_col_idx, d_counts);
+    exclusive_scan_kernel<<<1, 1024, 0, st>>>(d_counts, nbr, *d_block_row_ptr, d_flags + 1);
+    out->block_row_ptr.assign(static_cast<size_t>(nbr) + 1, 0);
+    if (cudaMemcpyAsync(out->block_row_ptr.data(), *d_block_row_ptr, static_cast<size_t>(nbr + 1) * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return fail(SPMM_ERR_CUDA);
+    if (cudaMemcpyAsync(flags, d_flags, sizeof(flags), cudaMemcpyDeviceToHost, st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    if (flags[1]) return fail(SPMM_ERR_TOO_LARGE);
+    const int64_t nnzb = out->block_row_ptr[static_cast<size_t>(nbr)];
+    out->nnzb = nnzb;
+
+    // 4. block columns and values
+    const size_t tile_bytes = static_cast<size_t>(b) * b * es;
+    const size_t idx_bytes = static_cast<size_t>(nnzb) * 4, val_bytes = static_cast<size_t>(nnzb) * tile_bytes;
+    if (cudaMalloc(reinterpret_cast<void**>(d_block_col_idx), idx_bytes ? idx_bytes : 16) != cudaSuccess) return fail(SPMM_ERR_ALLOC);
+    if (cudaMalloc(reinterpret_cast<void**>(d_blocks), val_bytes ? val_bytes : 16) != cudaSuccess) return fail(SPMM_ERR_ALLOC);
+    if (val_bytes && cudaMemsetAsync(*d_blocks, 0, val_bytes, st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    if (nbr > 0 && nnzb > 0) {
+        if (es == 1)
+            bcsr_fill_kernel<1><<<static_cast<unsigned>(nbr), kThreads, smem, st>>>(m, b, words, d_row_ptr, d_col_idx, d_vals, *d_block_row_ptr, *d_block_col_idx, *d_blocks);
+        else
+            bcsr_fill_kernel<2><<<static_cast<unsigned>(nbr), kThreads, smem, st>>>(m, b, words, d_row_ptr, d_col_idx, d_vals, *d_block_row_ptr, *d_block_col_idx, *d_blocks);
+    }
+    out->block_col_idx.assign(static_cast<size_t>(nnzb), 0);
+    if (nnzb && cudaMemcpyAsync(out->block_col_idx.data(), *d_block_col_idx, idx_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return fail(SPMM_ERR_CUDA);
+    if (cudaStreamSynchronize(st) != cudaSuccess || cudaGetLastError() != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    cudaFree(d_flags);
+    cudaFree(d_counts);
+    finish_bcsr_host(out);       // row order, empty block-rows, distinct block columns: host, from the index arrays
+    return SPMM_OK;
+}
+
+}  // namespace spmm

@@ -8,7 +8,7 @@ import pytest
 
 from paper_2604_17834_b200 import workloads as wl
 
-from helpers import assert_close, reference, run_gpu, run_gpu_variant
+from helpers import assert_close, reference, run_gpu, run_gpu_variant, to_device
 
 pytestmark = pytest.mark.gpu
 
@@ -194,6 +194,52 @@ def test_bcsr_fp8_e4m3_colmajor(lib, b, N):
         assert np.array_equal(C, run_gpu_variant(lib, h, Bs, a["m"], N, "fp8", col_major=True))
     finally:
         lib.spmm_destroy(h)
+
+
+@pytest.mark.parametrize("dtype,b,m,k", [("fp16", 64, 1024, 768), ("bf16", 16, 1000, 1000), ("fp16", 32, 130, 70),
+                                          ("bf16", 128, 257, 640), ("fp16", 16, 4096, 70000)])
+def test_bcsr_built_on_the_gpu_is_bit_exact(lib, dtype, b, m, k):
+    """Format construction as GPU kernels from a CSR matrix in device memory: every exported
+    array equals the format oracle's, and the handle runs like a host-built one."""
+    import torch
+    from oracle import formats as F
+    a = wl.random_csr(23 + m, m, k, 0.02 if k < 5000 else 0.0005, dtype, empty_rows=tuple(range(min(b, m // 2))))
+    rp = torch.from_numpy(a["row_ptr"].astype(np.int64)).cuda()
+    ci = torch.from_numpy(a["col_idx"].astype(np.int32)).cuda()
+    va = to_device(a["vals"])
+    h = lib.spmm_bcsr_create_csr_device(m, k, rp.data_ptr(), ci.data_ptr(), va.data_ptr(), dtype, b)
+    try:
+        f = F.bcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], b)
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCK_ROW_PTR, np.int32), f["block_row_ptr"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCK_COL_IDX, np.int32), f["block_col_idx"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCKS, np.uint16), f["blocks"].view(np.uint16).ravel())
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_ROW_ORDER, np.int32), F.bcsr_row_order(f["block_row_ptr"]))
+        info = lib.spmm_get_info(h, 128)
+        assert info["nnz"] == a["col_idx"].shape[0] and info["n_units"] == f["block_col_idx"].shape[0]
+        assert info["n_empty"] == int((np.diff(f["block_row_ptr"]) == 0).sum())
+        N = 200
+        Bs = wl.dense(3, k, N, ("uniform", -1.0, 1.0), dtype)
+        C = run_gpu(lib, h, Bs, m, N)
+        Cr, S = reference(a, Bs, dtype)
+        assert_close(C, Cr, S, dtype, "bcsr built on the GPU b=%d" % b)
+    finally:
+        lib.spmm_destroy(h)
+
+
+def test_bcsr_gpu_builder_rejects_malformed_csr(lib):
+    import torch
+    vals = to_device(wl.to_storage(np.ones(4), "fp16"))
+    cases = [(np.array([0, 2, 4]), np.array([1, 0, 2, 3]), lib.SPMM_ERR_UNSORTED),         # descending columns
+             (np.array([0, 2, 4]), np.array([0, 0, 2, 3]), lib.SPMM_ERR_UNSORTED),         # duplicate
+             (np.array([0, 2, 4]), np.array([0, 1, 2, 9]), lib.SPMM_ERR_OUT_OF_RANGE),     # column >= k
+             (np.array([0, 3, 2]), np.array([0, 1, 2, 3]), lib.SPMM_ERR_INVALID_ARG),      # row_ptr not monotone
+             (np.array([1, 2, 4]), np.array([0, 1, 2, 3]), lib.SPMM_ERR_INVALID_ARG)]      # row_ptr[0] != 0
+    for rp, ci, code in cases:
+        rpd = torch.from_numpy(rp.astype(np.int64)).cuda()
+        cid = torch.from_numpy(ci.astype(np.int32)).cuda()
+        with pytest.raises(lib.SpmmError) as e:
+            lib.spmm_bcsr_create_csr_device(2, 8, rpd.data_ptr(), cid.data_ptr(), vals.data_ptr(), "fp16", 16)
+        assert e.value.code == code
 
 
 def test_variant_argument_errors(lib):
