@@ -185,6 +185,15 @@ int spmm_bcsr_create_csr_device(spmm_handle_t *out, int64_t m, int64_t k, const 
                                 const int32_t *col_idx_dev, const void *vals_dev, int dtype, int block,
                                 const spmm_opts_t *opts, void *stream);
 
+/*
+ * The WCSR counterpart: window condensation and value packing on the GPU from a device-resident
+ * CSR (sort / unique of (window, column) keys); arguments as spmm_bcsr_create_csr_device with
+ * window_height in place of block.  nnz must be below 2^31.
+ */
+int spmm_wcsr_create_csr_device(spmm_handle_t *out, int64_t m, int64_t k, const int64_t *row_ptr_dev,
+                                const int32_t *col_idx_dev, const void *vals_dev, int dtype,
+                                int window_height, const spmm_opts_t *opts, void *stream);
+
 /* Same from COO: host int32 rows[nnz], cols[nnz] in any order, no duplicate (row, col). */
 int spmm_bcsr_create_coo(spmm_handle_t *out, int64_t m, int64_t k, int64_t nnz,
                          const int32_t *rows, const int32_t *cols, const void *vals, int dtype,

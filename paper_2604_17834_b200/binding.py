@@ -42,7 +42,8 @@ X_WCSR_WINDOW_ROW_PTR, X_WCSR_WINDOW_COL_IDX, X_WCSR_VALUES, X_WCSR_TASKS = 10, 
 X_WCSR_BIN_PTR, X_WCSR_BIN_TASKS = 14, 15
 
 EXPORTED_SYMBOLS = (
-    "spmm_bcsr_create_csr", "spmm_bcsr_create_csr_device", "spmm_bcsr_create_coo", "spmm_wcsr_create_csr", "spmm_wcsr_create_coo",
+    "spmm_bcsr_create_csr", "spmm_bcsr_create_csr_device", "spmm_bcsr_create_coo", "spmm_wcsr_create_csr",
+    "spmm_wcsr_create_csr_device", "spmm_wcsr_create_coo",
     "spmm_bcsr_plan", "spmm_run", "spmm_wcsr_run_static", "spmm_run_host", "spmm_check", "spmm_get_info", "spmm_export", "spmm_destroy",
     "spmm_status_string", "spmm_set_wait_limit_ns",
 )
@@ -81,6 +82,7 @@ _vp, _i64, _i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
 _lib.spmm_bcsr_create_csr.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _vp, _vp, _vp, _i32, _i32, ctypes.POINTER(SpmmOpts)]
 _lib.spmm_wcsr_create_csr.argtypes = _lib.spmm_bcsr_create_csr.argtypes
 _lib.spmm_bcsr_create_csr_device.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _vp, _vp, _vp, _i32, _i32, ctypes.POINTER(SpmmOpts), _vp]
+_lib.spmm_wcsr_create_csr_device.argtypes = _lib.spmm_bcsr_create_csr_device.argtypes
 _lib.spmm_bcsr_create_coo.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _vp, _vp, _vp, _i32, _i32, ctypes.POINTER(SpmmOpts)]
 _lib.spmm_wcsr_create_coo.argtypes = _lib.spmm_bcsr_create_coo.argtypes
 _lib.spmm_run.argtypes = [_vp, _vp, _vp, _i64, _vp]
@@ -160,6 +162,17 @@ def spmm_bcsr_create_csr_device(m, k, row_ptr_dev, col_idx_dev, vals_dev, dtype,
                                           _vp(int(vals_dev)), DTYPE_CODE[dtype], block, ctypes.byref(o), _vp(stream))
     if rc != SPMM_OK:
         raise SpmmError(rc, "spmm_bcsr_create_csr_device")
+    return h
+
+
+def spmm_wcsr_create_csr_device(m, k, row_ptr_dev, col_idx_dev, vals_dev, dtype, window_height=16, stream=0, **opt):
+    """-> handle.  CSR arrays in device memory -> WCSR built by GPU kernels."""
+    h = _vp()
+    o = _opts(**opt)
+    rc = _lib.spmm_wcsr_create_csr_device(ctypes.byref(h), m, k, _vp(int(row_ptr_dev)), _vp(int(col_idx_dev)),
+                                          _vp(int(vals_dev)), DTYPE_CODE[dtype], window_height, ctypes.byref(o), _vp(stream))
+    if rc != SPMM_OK:
+        raise SpmmError(rc, "spmm_wcsr_create_csr_device")
     return h
 
 

@@ -278,14 +278,50 @@ int create_bcsr_device(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* 
     return SPMM_OK;
 }
 
-int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const spmm_opts_t* opts) {
+// Uploads the schedule arrays of a WCSR handle (everything but the three format arrays).
+int upload_wcsr_plan(spmm_handle_s* h) {
+    const WcsrHost& f = h->wcsr;
+    std::vector<WcsrDevTask> dt(f.tasks.size());
+    for (size_t i = 0; i < f.tasks.size(); ++i) {
+        dt[i].col_begin = f.window_row_ptr[f.tasks[i].window] + f.tasks[i].q0;
+        dt[i].count = f.tasks[i].count;
+        dt[i].window = f.tasks[i].window;
+        dt[i].slot = f.tasks[i].slot;
+    }
+    const size_t nm = f.merge_window.size();
+    std::vector<int32_t> mg(3 * nm);
+    for (size_t i = 0; i < nm; ++i) {
+        mg[i] = f.merge_window[i];
+        mg[nm + i] = f.merge_first[i];
+        mg[2 * nm + i] = f.merge_nparts[i];
+    }
+    h->n_merge = static_cast<int>(nm);
+    int rc = upload(&h->d_tasks, dt.data(), dt.size() * sizeof(WcsrDevTask));
+    if (!rc) rc = upload(&h->d_bin_ptr, f.bin_ptr.data(), f.bin_ptr.size() * 4);
+    if (!rc) rc = upload(&h->d_bin_tasks, f.bin_tasks.data(), f.bin_tasks.size() * 4);
+    if (!rc) {
+        std::vector<int32_t> items(4 * f.bin_tasks.size(), 0);
+        for (size_t i = 0; i < f.bin_tasks.size(); ++i) {
+            items[4 * i] = f.tasks[f.bin_tasks[i]].window;
+            items[4 * i + 1] = f.tasks[f.bin_tasks[i]].slot;
+            items[4 * i + 2] = f.tasks[f.bin_tasks[i]].count;
+        }
+        rc = upload(&h->d_items, items.data(), items.size() * 4);
+    }
+    if (!rc) rc = upload(&h->d_fills, f.fills.data(), f.fills.size() * 4);
+    if (!rc) rc = upload(&h->d_bin_fill, f.bin_fill.data(), f.bin_fill.size() * 4);
+    if (!rc) rc = upload(&h->d_merge, mg.data(), mg.size() * 4);
+    return rc;
+}
+
+// Option and size checks shared by the host and the device builder; on success *hp is a fresh handle.
+int new_wcsr_handle(spmm_handle_s** hp, int64_t m, int64_t k, int dtype, const spmm_opts_t* opts, int* b_col_out, int* T_out) {
     if (dtype != SPMM_BF16 && dtype != SPMM_FP16 && dtype != SPMM_TF32) return SPMM_ERR_UNSUPPORTED;
     if (int orc = check_opts(opts)) return orc;
     if (opts && opts->layout == SPMM_COLMAJOR) return SPMM_ERR_UNSUPPORTED;   // BCSR only
     if (opts && opts->schedule == SPMM_SCHED_DYNAMIC) return SPMM_ERR_UNSUPPORTED;
-    int rc = validate_csr(a);
-    if (rc) return rc;
-    const int b_col_default = 32 / a.es;
+    const int es = elem_size(dtype);
+    const int b_col_default = 32 / es;
     const int b_col = (opts && opts->b_col > 0) ? opts->b_col : b_col_default;
     if (b_col != b_col_default) return SPMM_ERR_UNSUPPORTED;
     const int T = (opts && opts->split_cols > 0) ? opts->split_cols : 0;   // 0: chosen from the matrix
@@ -294,59 +330,66 @@ int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const s
     if (!h) return SPMM_ERR_ALLOC;
     h->format = 1;
     h->dtype = dtype;
-    h->es = a.es;
-    h->m = a.m;
-    h->k = a.k;
-    h->nnz = a.nnz;
+    h->es = es;
+    h->m = m;
+    h->k = k;
     h->host_only = opts && opts->host_only;
     h->c16 = opts && opts->c_type == SPMM_C_SAME_AS_INPUT && dtype != SPMM_TF32;
     h->cs = h->c16 ? 2 : 4;
+    *hp = h;
+    *b_col_out = b_col;
+    *T_out = T;
+    return SPMM_OK;
+}
+
+int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const spmm_opts_t* opts) {
+    spmm_handle_s* h = nullptr;
+    int b_col = 0, T = 0;
+    int rc = new_wcsr_handle(&h, a.m, a.k, dtype, opts, &b_col, &T);
+    if (rc) return rc;
+    rc = validate_csr(a);
+    if (rc) { delete h; return rc; }
+    h->nnz = a.nnz;
     rc = device_setup(h, opts);
     if (rc) { free_handle(h); return rc; }
     try {
-        rc = build_wcsr(a, wh, b_col, T, h->n_ctas * wcsr_bins_per_sm(elem_size(dtype), wh), &h->wcsr);
+        rc = build_wcsr(a, wh, b_col, T, h->n_ctas * wcsr_bins_per_sm(h->es, wh), &h->wcsr);
     } catch (const std::bad_alloc&) {
         rc = SPMM_ERR_ALLOC;
     }
     if (rc) { free_handle(h); return rc; }
     if (!h->host_only) {
         const WcsrHost& f = h->wcsr;
-        std::vector<WcsrDevTask> dt(f.tasks.size());
-        for (size_t i = 0; i < f.tasks.size(); ++i) {
-            dt[i].col_begin = f.window_row_ptr[f.tasks[i].window] + f.tasks[i].q0;
-            dt[i].count = f.tasks[i].count;
-            dt[i].window = f.tasks[i].window;
-            dt[i].slot = f.tasks[i].slot;
-        }
-        const size_t nm = f.merge_window.size();
-        std::vector<int32_t> mg(3 * nm);
-        for (size_t i = 0; i < nm; ++i) {
-            mg[i] = f.merge_window[i];
-            mg[nm + i] = f.merge_first[i];
-            mg[2 * nm + i] = f.merge_nparts[i];
-        }
-        h->n_merge = static_cast<int>(nm);
         rc = upload(&h->d_ptr, f.window_row_ptr.data(), f.window_row_ptr.size() * 4);
         if (!rc) rc = upload(&h->d_idx, f.window_col_idx.data(), f.window_col_idx.size() * 4);
         if (!rc) rc = upload(&h->d_vals, f.packed.data(), f.packed.size());
-        if (!rc) rc = upload(&h->d_tasks, dt.data(), dt.size() * sizeof(WcsrDevTask));
-        if (!rc) rc = upload(&h->d_bin_ptr, f.bin_ptr.data(), f.bin_ptr.size() * 4);
-        if (!rc) rc = upload(&h->d_bin_tasks, f.bin_tasks.data(), f.bin_tasks.size() * 4);
-        if (!rc) {
-            std::vector<int32_t> items(4 * f.bin_tasks.size(), 0);
-            for (size_t i = 0; i < f.bin_tasks.size(); ++i) {
-                items[4 * i] = f.tasks[f.bin_tasks[i]].window;
-                items[4 * i + 1] = f.tasks[f.bin_tasks[i]].slot;
-                items[4 * i + 2] = f.tasks[f.bin_tasks[i]].count;
-            }
-            rc = upload(&h->d_items, items.data(), items.size() * 4);
-        }
-        if (!rc) rc = upload(&h->d_fills, f.fills.data(), f.fills.size() * 4);
-        if (!rc) rc = upload(&h->d_bin_fill, f.bin_fill.data(), f.bin_fill.size() * 4);
-        if (!rc) rc = upload(&h->d_merge, mg.data(), mg.size() * 4);
+        if (!rc) rc = upload_wcsr_plan(h);
         if (rc) { free_handle(h); return rc; }
         std::vector<uint8_t>().swap(h->wcsr.packed);
     }
+    *out = h;
+    return SPMM_OK;
+}
+
+// The same handle from a CSR matrix in device memory: the format arrays are built by GPU kernels.
+int create_wcsr_device(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* d_row_ptr, const int32_t* d_col_idx,
+                       const void* d_vals, int dtype, int wh, const spmm_opts_t* opts, cudaStream_t stream) {
+    if (opts && opts->host_only) return SPMM_ERR_INVALID_ARG;
+    spmm_handle_s* h = nullptr;
+    int b_col = 0, T = 0;
+    int rc = new_wcsr_handle(&h, m, k, dtype, opts, &b_col, &T);
+    if (rc) return rc;
+    rc = device_setup(h, opts);
+    if (rc) { free_handle(h); return rc; }
+    try {
+        rc = build_wcsr_device(m, k, d_row_ptr, d_col_idx, static_cast<const uint8_t*>(d_vals), h->es, wh, b_col, T,
+                               h->n_ctas * wcsr_bins_per_sm(h->es, wh), stream, &h->wcsr, &h->nnz, &h->d_ptr, &h->d_idx,
+                               &h->d_vals);
+        if (!rc) rc = upload_wcsr_plan(h);
+    } catch (const std::bad_alloc&) {
+        rc = SPMM_ERR_ALLOC;
+    }
+    if (rc) { free_handle(h); return rc; }
     *out = h;
     return SPMM_OK;
 }
@@ -657,6 +700,16 @@ int spmm_bcsr_create_csr_device(spmm_handle_t* out, int64_t m, int64_t k, const 
     return create_bcsr_device(out, m, k, row_ptr_dev, col_idx_dev, vals_dev, dtype, block, opts, static_cast<cudaStream_t>(stream));
 }
 
+int spmm_wcsr_create_csr_device(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* row_ptr_dev,
+                                const int32_t* col_idx_dev, const void* vals_dev, int dtype, int window_height,
+                                const spmm_opts_t* opts, void* stream) {
+    if (!out) return SPMM_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (dtype < 0 || dtype > 3 || m < 0 || k < 0 || !row_ptr_dev) return SPMM_ERR_INVALID_ARG;
+    if (m >= (int64_t{1} << 31) || k >= (int64_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
+    return create_wcsr_device(out, m, k, row_ptr_dev, col_idx_dev, vals_dev, dtype, window_height, opts, static_cast<cudaStream_t>(stream));
+}
+
 int spmm_bcsr_create_coo(spmm_handle_t* out, int64_t m, int64_t k, int64_t nnz, const int32_t* rows,
                          const int32_t* cols, const void* vals, int dtype, int block, const spmm_opts_t* opts) {
     if (!out) return SPMM_ERR_INVALID_ARG;
@@ -847,7 +900,7 @@ int spmm_export(spmm_handle_t h, int which, void* host_dst, size_t cap, size_t* 
         const WcsrHost& f = h->wcsr;
         switch (which) {
             case SPMM_X_WCSR_WINDOW_ROW_PTR: bytes = f.window_row_ptr.size() * 4; dev_src = h->d_ptr; host_src = f.window_row_ptr.data(); break;
-            case SPMM_X_WCSR_WINDOW_COL_IDX: bytes = f.window_col_idx.size() * 4; dev_src = h->d_idx; host_src = f.window_col_idx.data(); break;
+            case SPMM_X_WCSR_WINDOW_COL_IDX: bytes = static_cast<size_t>(f.P) * 4; dev_src = h->d_idx; host_src = f.window_col_idx.data(); break;
             case SPMM_X_WCSR_VALUES: bytes = static_cast<size_t>(f.P) * f.wh * h->es; unpack_wcsr = true; break;
             case SPMM_X_WCSR_TASKS: bytes = f.tasks.size() * 16; break;
             case SPMM_X_WCSR_BIN_PTR: bytes = f.bin_ptr.size() * 4; dev_src = h->d_bin_ptr; host_src = f.bin_ptr.data(); break;

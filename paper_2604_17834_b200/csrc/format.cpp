@@ -208,6 +208,11 @@ int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost*
         }
     }
 
+    return plan_wcsr(out, T, n_bins, a.es);
+}
+
+int plan_wcsr(WcsrHost* out, int T, int n_bins, int es) {
+    const int64_t nwin = out->nwin, P = out->P;
     if (T == 0) {
         int64_t t = P / (static_cast<int64_t>(n_bins) * 4);
         t = (t / 64) * 64;
@@ -280,7 +285,7 @@ int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost*
 
     // pipeline schedule: one fill per stage-sized run of columns (16 KB of gathered B rows at
     // 128 tokens: 64 columns of a 2-byte type, 32 of a 4-byte type), bin-major
-    out->kt = wcsr_stage_cols(a.es);
+    out->kt = wcsr_stage_cols(es);
     out->fills.clear();
     out->bin_fill.assign(static_cast<size_t>(n_bins) + 1, 0);
     for (int j = 0; j < n_bins; ++j) {

@@ -98,8 +98,20 @@ int build_bcsr_schedule(const BcsrHost& f, int n_tt, int slab_w, int n_ctas, Bcs
 // T = 0 picks the sub-task size from the matrix: about a quarter of one bin's share of the
 // padded columns, rounded down to a multiple of 64 and clamped to [128, 4096].
 int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost* out);
+// Second half of build_wcsr: split plan, bins, fills and merge lists from out->window_row_ptr / out->P.
+int plan_wcsr(WcsrHost* out, int T, int n_bins, int es);
+// The WCSR format arrays built on the GPU from a CSR matrix in device memory (format_gpu.cu):
+// validates the CSR, allocates and fills window_row_ptr, window_col_idx and the packed values on
+// the device (owned by the caller afterwards), leaves window_row_ptr, P and distinct_cols in *out
+// (out->window_col_idx and out->packed stay empty) and runs plan_wcsr.  Synchronises `stream`.
+int build_wcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int32_t* d_col_idx, const uint8_t* d_vals,
+                      int es, int wh, int b_col, int T, int n_bins, cudaStream_t stream, WcsrHost* out, int64_t* nnz_out,
+                      int32_t** d_window_row_ptr, int32_t** d_window_col_idx, uint8_t** d_packed);
 
 // Byte offset of element (row r, padded column q) inside the packed WCSR value array.
+#ifdef __CUDACC__
+__host__ __device__
+#endif
 inline size_t wcsr_packed_offset(int wh, int b_col, int es, int r, int64_t q) {
     const int64_t chunk = q / b_col;
     const int c = static_cast<int>(q % b_col);

@@ -13,6 +13,15 @@
 //                blocks[slot][row in block][column in block]
 // A bitmap needs 2 * ceil(k / b) / 8 bytes of shared memory (bits + word prefix), at most 200 KB:
 // k / b <= 819,200.
+//
+// WCSR (window condensation of Sec. 2.3): every stored entry becomes the 64-bit key
+// (window << 32 | column); a radix sort and a unique pass (CUB primitives) leave, window after
+// window, the ascending union of each window's columns; counting keys per window and two prefix
+// sums give window_row_ptr (lengths padded to b_col) and each window's place in the key list;
+// window_col_idx is those columns over a -1 fill, and every value finds its condensed column by
+// binary search in its window's list and goes straight into the packed tile layout.
+#include <cub/cub.cuh>
+
 #include <cstring>
 #include <numeric>
 #include <algorithm>
@@ -294,6 +303,212 @@ int build_bcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int3
     cudaFree(d_counts);
     finish_bcsr_host(out);       // row order, empty block-rows, distinct block columns: host, from the index arrays
     return SPMM_OK;
+}
+
+namespace {
+
+__global__ void wcsr_keys_kernel(int64_t m, int wh, const int64_t* row_ptr, const int32_t* col_idx, uint64_t* keys) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = (blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x) >> 5;
+    const int64_t nwarps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+    for (int64_t i = warp0; i < m; i += nwarps) {
+        const uint64_t hi = static_cast<uint64_t>(i / wh) << 32;
+        for (int64_t p = row_ptr[i] + lane; p < row_ptr[i + 1]; p += 32) keys[p] = hi | static_cast<uint32_t>(col_idx[p]);
+    }
+}
+
+// per window: how many distinct columns; per column: is it referenced at all
+__global__ void wcsr_count_kernel(const uint64_t* ukeys, const int* n_unique, int32_t* cnt, uint8_t* used) {
+    const int64_t n = *n_unique;
+    for (int64_t j = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; j < n;
+         j += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const uint64_t key = ukeys[j];
+        atomicAdd(&cnt[key >> 32], 1);
+        used[static_cast<uint32_t>(key)] = 1;
+    }
+}
+
+__global__ void wcsr_pad_kernel(const int32_t* cnt, int64_t nwin, int b_col, int32_t* len) {
+    for (int64_t w = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; w < nwin;
+         w += static_cast<int64_t>(gridDim.x) * blockDim.x)
+        len[w] = (cnt[w] + b_col - 1) / b_col * b_col;
+}
+
+__global__ void wcsr_sum_used_kernel(const uint8_t* used, int64_t k, unsigned long long* total) {
+    unsigned long long n = 0;
+    for (int64_t c = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; c < k;
+         c += static_cast<int64_t>(gridDim.x) * blockDim.x)
+        n += used[c];
+    for (int o = 16; o > 0; o >>= 1) n += __shfl_down_sync(0xffffffffu, n, o);
+    if ((threadIdx.x & 31) == 0 && n) atomicAdd(total, n);
+}
+
+__global__ void wcsr_cols_kernel(const uint64_t* ukeys, const int* n_unique, const int32_t* ustart,
+                                 const int32_t* window_row_ptr, int32_t* window_col_idx) {
+    const int64_t n = *n_unique;
+    for (int64_t j = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; j < n;
+         j += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const uint64_t key = ukeys[j];
+        const int64_t w = static_cast<int64_t>(key >> 32);
+        window_col_idx[window_row_ptr[w] + (j - ustart[w])] = static_cast<int32_t>(static_cast<uint32_t>(key));
+    }
+}
+
+template <int ES>
+__global__ void wcsr_values_kernel(int64_t m, int wh, int b_col, const int64_t* row_ptr, const int32_t* col_idx,
+                                   const uint8_t* vals, const int32_t* cnt, const int32_t* window_row_ptr,
+                                   const int32_t* window_col_idx, uint8_t* packed) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = (blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x) >> 5;
+    const int64_t nwarps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+    for (int64_t i = warp0; i < m; i += nwarps) {
+        const int64_t w = i / wh;
+        const int r = static_cast<int>(i - w * wh);
+        const int64_t base = window_row_ptr[w];
+        const int32_t* seg = window_col_idx + base;
+        const int n = cnt[w];
+        for (int64_t p = row_ptr[i] + lane; p < row_ptr[i + 1]; p += 32) {
+            const int32_t c = col_idx[p];
+            int lo = 0, hi = n;                      // first position with seg[pos] >= c; c is in the list
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (seg[mid] < c) lo = mid + 1; else hi = mid;
+            }
+            uint8_t* dst = packed + wcsr_packed_offset(wh, b_col, ES, r, base + lo);
+            const uint8_t* src = vals + static_cast<size_t>(p) * ES;
+            if constexpr (ES == 2) *reinterpret_cast<uint16_t*>(dst) = *reinterpret_cast<const uint16_t*>(src);
+            else *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(src);
+        }
+    }
+}
+
+}  // namespace
+
+int build_wcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int32_t* d_col_idx, const uint8_t* d_vals,
+                      int es, int wh, int b_col, int T, int n_bins, cudaStream_t st, WcsrHost* out, int64_t* nnz_out,
+                      int32_t** d_window_row_ptr, int32_t** d_window_col_idx, uint8_t** d_packed) {
+    if (wh != 16 && wh != 64) return SPMM_ERR_UNSUPPORTED;
+    if ((es != 2 && es != 4) || b_col * es != 32) return SPMM_ERR_UNSUPPORTED;
+    if (T < 0 || T % b_col != 0 || n_bins <= 0) return SPMM_ERR_INVALID_ARG;
+    if (m < 0 || k < 0 || !d_row_ptr) return SPMM_ERR_INVALID_ARG;
+    const int64_t nwin = (m + wh - 1) / wh;
+    out->wh = wh;
+    out->b_col = b_col;
+    out->nwin = nwin;
+    *d_window_row_ptr = nullptr;
+    *d_window_col_idx = nullptr;
+    *d_packed = nullptr;
+
+    int* d_flags = nullptr;                   // [0] CSR error code, [1] scan overflow, [2] number of unique keys
+    uint64_t *d_keys = nullptr, *d_keys2 = nullptr;
+    int32_t *d_cnt = nullptr, *d_len = nullptr, *d_ustart = nullptr;
+    uint8_t* d_used = nullptr;
+    unsigned long long* d_total = nullptr;
+    void* d_temp = nullptr;
+    auto release = [&]() {
+        cudaFree(d_flags); cudaFree(d_keys); cudaFree(d_keys2); cudaFree(d_cnt); cudaFree(d_len);
+        cudaFree(d_ustart); cudaFree(d_used); cudaFree(d_total); cudaFree(d_temp);
+    };
+    auto fail = [&](int code) {
+        release();
+        cudaFree(*d_window_row_ptr); cudaFree(*d_window_col_idx); cudaFree(*d_packed);
+        *d_window_row_ptr = nullptr; *d_window_col_idx = nullptr; *d_packed = nullptr;
+        return code;
+    };
+    auto alloc = [&](void** ptr, size_t bytes) { return cudaMalloc(ptr, bytes ? bytes : 16) == cudaSuccess; };
+
+    if (!alloc(reinterpret_cast<void**>(&d_flags), 4 * sizeof(int))) return fail(SPMM_ERR_ALLOC);
+    if (cudaMemsetAsync(d_flags, 0, 4 * sizeof(int), st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    int64_t nnz = 0;
+    int flags[4] = {0, 0, 0, 0};
+    const unsigned check_grid = static_cast<unsigned>(std::min<int64_t>((m + 255) / 256, 2048));
+    if (m > 0) {
+        csr_check_rows_kernel<<<check_grid, 256, 0, st>>>(m, d_row_ptr, d_flags);
+        if (cudaMemcpyAsync(&nnz, d_row_ptr + m, sizeof(int64_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    }
+    if (cudaMemcpyAsync(flags, d_flags, sizeof(flags), cudaMemcpyDeviceToHost, st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    if (flags[0] != 0) return fail(flags[0]);
+    if (nnz < 0 || (nnz > 0 && (!d_col_idx || !d_vals))) return fail(SPMM_ERR_INVALID_ARG);
+    if (nnz >= (int64_t{1} << 31)) return fail(SPMM_ERR_TOO_LARGE);
+    if (nnz > 0) {
+        csr_check_cols_kernel<<<check_grid, 256, 0, st>>>(m, k, d_row_ptr, d_col_idx, d_flags);
+        if (cudaMemcpyAsync(flags, d_flags, sizeof(flags), cudaMemcpyDeviceToHost, st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+        if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+        if (flags[0] != 0) return fail(flags[0]);
+    }
+    *nnz_out = nnz;
+
+    // keys -> sorted -> unique
+    if (!alloc(reinterpret_cast<void**>(&d_keys), static_cast<size_t>(nnz) * 8) ||
+        !alloc(reinterpret_cast<void**>(&d_keys2), static_cast<size_t>(nnz) * 8) ||
+        !alloc(reinterpret_cast<void**>(&d_cnt), static_cast<size_t>(nwin + 1) * 4) ||
+        !alloc(reinterpret_cast<void**>(&d_len), static_cast<size_t>(nwin + 1) * 4) ||
+        !alloc(reinterpret_cast<void**>(&d_ustart), static_cast<size_t>(nwin + 1) * 4) ||
+        !alloc(reinterpret_cast<void**>(&d_used), static_cast<size_t>(k)) ||
+        !alloc(reinterpret_cast<void**>(&d_total), 8) ||
+        !alloc(reinterpret_cast<void**>(d_window_row_ptr), static_cast<size_t>(nwin + 1) * 4))
+        return fail(SPMM_ERR_ALLOC);
+    cudaMemsetAsync(d_cnt, 0, static_cast<size_t>(nwin + 1) * 4, st);
+    cudaMemsetAsync(d_used, 0, static_cast<size_t>(k ? k : 1), st);
+    cudaMemsetAsync(d_total, 0, 8, st);
+    const int n = static_cast<int>(nnz);
+    int end_bit = 32;
+    while (end_bit < 64 && (int64_t{1} << (end_bit - 32)) < nwin) ++end_bit;
+    if (n > 0) {
+        wcsr_keys_kernel<<<static_cast<unsigned>(std::min<int64_t>((m + 7) / 8, 4096)), 256, 0, st>>>(m, wh, d_row_ptr, d_col_idx, d_keys);
+        size_t t1 = 0, t2 = 0;
+        cub::DeviceRadixSort::SortKeys(nullptr, t1, d_keys, d_keys2, n, 0, end_bit, st);
+        cub::DeviceSelect::Unique(nullptr, t2, d_keys2, d_keys, d_flags + 2, n, st);
+        if (!alloc(&d_temp, std::max(t1, t2))) return fail(SPMM_ERR_ALLOC);
+        size_t tb = std::max(t1, t2);
+        if (cub::DeviceRadixSort::SortKeys(d_temp, tb, d_keys, d_keys2, n, 0, end_bit, st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+        tb = std::max(t1, t2);
+        if (cub::DeviceSelect::Unique(d_temp, tb, d_keys2, d_keys, d_flags + 2, n, st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+        // d_keys now holds the unique keys, d_flags[2] their number
+        wcsr_count_kernel<<<2048, 256, 0, st>>>(d_keys, d_flags + 2, d_cnt, d_used);
+    }
+    wcsr_pad_kernel<<<static_cast<unsigned>(std::min<int64_t>((nwin + 255) / 256 + 1, 2048)), 256, 0, st>>>(d_cnt, nwin, b_col, d_len);
+    exclusive_scan_kernel<<<1, 1024, 0, st>>>(d_len, nwin, *d_window_row_ptr, d_flags + 1);
+    exclusive_scan_kernel<<<1, 1024, 0, st>>>(d_cnt, nwin, d_ustart, d_flags + 3);
+    if (k > 0) wcsr_sum_used_kernel<<<static_cast<unsigned>(std::min<int64_t>((k + 255) / 256, 1024)), 256, 0, st>>>(d_used, k, d_total);
+    out->window_row_ptr.assign(static_cast<size_t>(nwin) + 1, 0);
+    unsigned long long distinct = 0;
+    if (cudaMemcpyAsync(out->window_row_ptr.data(), *d_window_row_ptr, static_cast<size_t>(nwin + 1) * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(flags, d_flags, sizeof(flags), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(&distinct, d_total, 8, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return fail(SPMM_ERR_CUDA);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    if (flags[1]) return fail(SPMM_ERR_TOO_LARGE);
+    const int64_t P = out->window_row_ptr[static_cast<size_t>(nwin)];
+    out->P = P;
+    out->distinct_cols = static_cast<int64_t>(distinct);
+
+    // window_col_idx over a -1 fill, values into the zero-filled packed tiles
+    const size_t packed_bytes = static_cast<size_t>(P) * wh * es;
+    if (!alloc(reinterpret_cast<void**>(d_window_col_idx), static_cast<size_t>(P) * 4) ||
+        !alloc(reinterpret_cast<void**>(d_packed), packed_bytes))
+        return fail(SPMM_ERR_ALLOC);
+    if (P > 0) {
+        cudaMemsetAsync(*d_window_col_idx, 0xFF, static_cast<size_t>(P) * 4, st);
+        cudaMemsetAsync(*d_packed, 0, packed_bytes, st);
+    }
+    if (n > 0) {
+        wcsr_cols_kernel<<<2048, 256, 0, st>>>(d_keys, d_flags + 2, d_ustart, *d_window_row_ptr, *d_window_col_idx);
+        const unsigned vgrid = static_cast<unsigned>(std::min<int64_t>((m + 7) / 8, 8192));
+        if (es == 2)
+            wcsr_values_kernel<2><<<vgrid, 256, 0, st>>>(m, wh, b_col, d_row_ptr, d_col_idx, d_vals, d_cnt, *d_window_row_ptr, *d_window_col_idx, *d_packed);
+        else
+            wcsr_values_kernel<4><<<vgrid, 256, 0, st>>>(m, wh, b_col, d_row_ptr, d_col_idx, d_vals, d_cnt, *d_window_row_ptr, *d_window_col_idx, *d_packed);
+    }
+    if (cudaStreamSynchronize(st) != cudaSuccess || cudaGetLastError() != cudaSuccess) return fail(SPMM_ERR_CUDA);
+    release();
+    const int rc = plan_wcsr(out, T, n_bins, es);
+    if (rc) {
+        cudaFree(*d_window_row_ptr); cudaFree(*d_window_col_idx); cudaFree(*d_packed);
+        *d_window_row_ptr = nullptr; *d_window_col_idx = nullptr; *d_packed = nullptr;
+    }
+    return rc;
 }
 
 }  // namespace spmm

@@ -226,6 +226,44 @@ def test_bcsr_built_on_the_gpu_is_bit_exact(lib, dtype, b, m, k):
         lib.spmm_destroy(h)
 
 
+@pytest.mark.parametrize("dtype,wh,m,k,dens", [("tf32", 16, 1000, 900, 0.02), ("fp16", 16, 333, 517, 0.05),
+                                                ("bf16", 64, 1000, 4000, 0.01), ("fp16", 16, 5000, 70000, 0.0005),
+                                                ("tf32", 64, 130, 70, 0.2)])
+def test_wcsr_built_on_the_gpu_is_bit_exact(lib, dtype, wh, m, k, dens):
+    """Window condensation and value packing as GPU kernels (sort / unique of (window, column)
+    keys): every exported array equals the format oracle's, plan and bins included, and the
+    handle runs like a host-built one."""
+    import torch
+    from oracle import formats as F
+    a = wl.random_csr(29 + m, m, k, dens, dtype, empty_rows=tuple(range(wh, min(3 * wh, m))))
+    rp = torch.from_numpy(a["row_ptr"].astype(np.int64)).cuda()
+    ci = torch.from_numpy(a["col_idx"].astype(np.int32)).cuda()
+    va = to_device(a["vals"])
+    h = lib.spmm_wcsr_create_csr_device(m, k, rp.data_ptr(), ci.data_ptr(), va.data_ptr(), dtype, wh, split_cols=64)
+    h0 = lib.spmm_wcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, wh, split_cols=64)
+    try:
+        b_col = 8 if dtype == "tf32" else 16
+        f = F.wcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], wh, b_col)
+        bits = np.uint32 if dtype == "tf32" else np.uint16
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_ROW_PTR, np.int32), f["window_row_ptr"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_COL_IDX, np.int32), f["window_col_idx"])
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_VALUES, wl.storage_np_dtype(dtype)).view(bits),
+                              f["values"].view(bits).ravel())
+        for which in (lib.X_WCSR_TASKS, lib.X_WCSR_BIN_PTR, lib.X_WCSR_BIN_TASKS):
+            assert np.array_equal(lib.spmm_export(h, which, np.int32), lib.spmm_export(h0, which, np.int32))
+        i1, i0 = lib.spmm_get_info(h, 128), lib.spmm_get_info(h0, 128)
+        assert i1 == i0
+        N = 136
+        Bs = wl.dense(3, k, N, ("normal", 0.0, 1.0), dtype)
+        C = run_gpu(lib, h, Bs, m, N)
+        assert np.array_equal(C, run_gpu(lib, h0, Bs, m, N))
+        Cr, S = reference(a, Bs, dtype)
+        assert_close(C, Cr, S, dtype, "wcsr built on the GPU wh=%d" % wh)
+    finally:
+        lib.spmm_destroy(h)
+        lib.spmm_destroy(h0)
+
+
 def test_bcsr_gpu_builder_rejects_malformed_csr(lib):
     import torch
     vals = to_device(wl.to_storage(np.ones(4), "fp16"))
@@ -239,6 +277,9 @@ def test_bcsr_gpu_builder_rejects_malformed_csr(lib):
         cid = torch.from_numpy(ci.astype(np.int32)).cuda()
         with pytest.raises(lib.SpmmError) as e:
             lib.spmm_bcsr_create_csr_device(2, 8, rpd.data_ptr(), cid.data_ptr(), vals.data_ptr(), "fp16", 16)
+        assert e.value.code == code
+        with pytest.raises(lib.SpmmError) as e:
+            lib.spmm_wcsr_create_csr_device(2, 8, rpd.data_ptr(), cid.data_ptr(), vals.data_ptr(), "fp16", 16)
         assert e.value.code == code
 
 
