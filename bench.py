@@ -135,7 +135,9 @@ DEFAULT_OTHERS = ["cfg1_bcsr_tiny", "cfg3_bcsr_llm_gate", "cfg3_bcsr_llm_down",
                   "cfg4_bcsr_sweep_b128_d0.1", "cfg4_bcsr_sweep_b64_d0.5", "cfg4_bcsr_flat_b64_d0.05",
                   "cfg5_wcsr_rmat_n32", "cfg5_wcsr_rmat_n128", "cfg5_wcsr_rmat_n256",
                   "cfg3_bcsr_llm_gate_c16", "cfg3_bcsr_llm_gate_cm", "cfg3_bcsr_llm_gate_cm_c16",
-                  "cfg3_bcsr_llm_down_cm_c16", "cfg5_wcsr_rmat_n128_c16"]
+                  "cfg3_bcsr_llm_down_cm_c16", "cfg5_wcsr_rmat_n128_c16",
+                  "cfg3_bcsr_llm_gate_cm_fp8", "cfg3_bcsr_llm_down_cm_fp8", "cfg2_wcsr_irregular_wh64",
+                  "cfg4_bcsr_sweep_b64_d0.1_dyn"]
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures whose
 # summaries are under profiles/ (None where no capture of that exact launch exists).
