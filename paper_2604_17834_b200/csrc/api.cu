@@ -92,7 +92,8 @@ struct spmm_handle_s {
     uint8_t* d_vals = nullptr;       // blocks / packed values
     int32_t* d_order = nullptr;      // BCSR row order
     BcsrSchedule sched;              // BCSR tile schedule of the most recent dense width
-    int32_t* d_tiles = nullptr;
+    int32_t* d_tiles = nullptr;      // {block-row, token tile} pairs (the exported schedule)
+    int32_t* d_tile_recs = nullptr;  // the kernel's records: {block-row, token tile, first block, end block}
     int32_t* d_cta_ptr = nullptr;
     WcsrDevTask* d_tasks = nullptr;
     int32_t* d_bin_ptr = nullptr;
@@ -137,6 +138,7 @@ void free_handle(spmm_handle_s* h) {
         cudaFree(h->d_vals);
         cudaFree(h->d_order);
         cudaFree(h->d_tiles);
+        cudaFree(h->d_tile_recs);
         cudaFree(h->d_cta_ptr);
         cudaFree(h->d_tasks);
         cudaFree(h->d_bin_ptr);
@@ -552,10 +554,24 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
         if (h->d_tiles) {   // a previous schedule may still be in use by a running kernel
             if (cudaDeviceSynchronize() != cudaSuccess) return SPMM_ERR_CUDA;
             cudaFree(h->d_tiles);
+            cudaFree(h->d_tile_recs);
             cudaFree(h->d_cta_ptr);
-            h->d_tiles = h->d_cta_ptr = nullptr;
+            h->d_tiles = h->d_tile_recs = h->d_cta_ptr = nullptr;
         }
         rc = upload(&h->d_tiles, sc.tiles.data(), sc.tiles.size() * 4);
+        if (!rc) {
+            // self-contained records, so that a role needs one load per tile (and can fetch it a tile ahead)
+            const size_t nt = sc.tiles.size() / 2;
+            std::vector<int32_t> recs(4 * nt);
+            for (size_t i = 0; i < nt; ++i) {
+                const int32_t I = sc.tiles[2 * i];
+                recs[4 * i] = I;
+                recs[4 * i + 1] = sc.tiles[2 * i + 1];
+                recs[4 * i + 2] = f.block_row_ptr[I];
+                recs[4 * i + 3] = f.block_row_ptr[I + 1];
+            }
+            rc = upload(&h->d_tile_recs, recs.data(), recs.size() * 4);
+        }
         if (!rc) rc = upload(&h->d_cta_ptr, sc.cta_ptr.data(), sc.cta_ptr.size() * 4);
         if (rc) return rc;
     }
@@ -572,7 +588,7 @@ int run_bcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t s
     BcsrParams p;
     p.block_row_ptr = h->d_ptr;
     p.block_col_idx = h->d_idx;
-    p.tiles = reinterpret_cast<const int2*>(h->d_tiles);
+    p.tiles = reinterpret_cast<const int4*>(h->d_tile_recs);
     p.cta_ptr = h->d_cta_ptr;
     p.C = C;
     p.m = h->m;

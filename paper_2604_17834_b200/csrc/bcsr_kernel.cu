@@ -141,13 +141,21 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         tile_begin = __ldg(p.cta_ptr + blockIdx.x);
         tile_end = __ldg(p.cta_ptr + blockIdx.x + 1);
     }
-    // next tile of this warp's walk; nth = number of tiles it has taken so far
-    auto next_tile = [&](uint32_t nth, int* ti, bool* ok) -> bool {
+    // Next tile of this warp's walk; nth = number of tiles it has taken so far.  A tile's record
+    // {block-row, token tile, first stored block, end block} is all a role needs to know about
+    // it; with the static schedule the following tile's record is requested one tile ahead
+    // (*rec_next), so that its latency is not paid between tiles.
+    auto next_tile = [&](uint32_t nth, int4* rec, int4* rec_next, bool* ok) -> bool {
         if constexpr (!DYN) {
-            *ti = tile_begin + static_cast<int>(nth);
-            return *ti < tile_end;
+            const int ti = tile_begin + static_cast<int>(nth);
+            if (ti >= tile_end) return false;
+            *rec = nth == 0 ? __ldg(p.tiles + ti) : *rec_next;
+            if (ti + 1 < tile_end) *rec_next = __ldg(p.tiles + ti + 1);
+            return true;
         } else {
-            if (nth == 0) { *ti = static_cast<int>(blockIdx.x); return true; }
+            int ti_dyn;
+            int* ti = &ti_dyn;
+            if (nth == 0) { *rec = __ldg(p.tiles + blockIdx.x); return true; }
             // fetched tile nth is entry nth - 1 of the ring
             const int slot = (nth - 1u) % kSchedDepth;
             const uint32_t use = (nth - 1u) / kSchedDepth;
@@ -164,6 +172,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 return false;
             }
             *ti = static_cast<int>(x);
+            if (valid) *rec = __ldg(p.tiles + *ti);
             return valid;
         }
     };
@@ -182,18 +191,24 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint64_t keep = l2_policy_evict_last();
             TRACE_DECL(tr_empty);
             TRACE_T0(tr_start);
-            int ti;
-            for (uint32_t nth = 0; ok && next_tile(nth, &ti, &ok); ++nth) {
-                const int2 tcd = __ldg(p.tiles + ti);
-                const int tI = tcd.x;
+            int4 tcd, tcd_next;
+            int Jl_next = 0;                 // block columns of the next tile's first 32 blocks, fetched a tile ahead
+            bool have_next = false;
+            for (uint32_t nth = 0; ok && next_tile(nth, &tcd, &tcd_next, &ok); ++nth) {
                 const int n0 = tcd.y * Cfg::kBnT;
                 const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
                 const int nbox = (nvalid + 63) >> 6;
                 const bool whole_tile = p.use_3d && nvalid == Cfg::kBnT;
-                const int pb = __ldg(p.block_row_ptr + tI), pe = __ldg(p.block_row_ptr + tI + 1);
+                const int pb = tcd.z, pe = tcd.w;
+                const int Jl_first = have_next ? Jl_next : ((pb + lane < pe) ? __ldg(p.block_col_idx + pb + lane) : 0);
+                if constexpr (!DYN) {
+                    // the record of the following tile was requested when this one was taken
+                    have_next = tile_begin + static_cast<int>(nth) + 1 < tile_end;
+                    if (have_next) Jl_next = (tcd_next.z + lane < tcd_next.w) ? __ldg(p.block_col_idx + tcd_next.z + lane) : 0;
+                }
                 for (int q0 = pb; q0 < pe && ok; q0 += 32) {
                     // block columns of up to 32 stored blocks with one coalesced load
-                    const int Jl = (q0 + lane < pe) ? __ldg(p.block_col_idx + q0 + lane) : 0;
+                    const int Jl = q0 == pb ? Jl_first : ((q0 + lane < pe) ? __ldg(p.block_col_idx + q0 + lane) : 0);
                     const int nq = min(32, pe - q0);
                     for (int jq = 0; jq < nq; jq += Cfg::kBps, ++it) {
                         const int q = q0 + jq;
@@ -281,10 +296,8 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             TRACE_DECL(tr_acce);
             TRACE_DECL(tr_issue);
             TRACE_T0(tr_start);
-            int ti;
-            for (; ok && next_tile(tile_i, &ti, &ok); ++tile_i) {
-                const int2 tcd = __ldg(p.tiles + ti);
-                const int tI = tcd.x;
+            int4 tcd, tcd_next;
+            for (; ok && next_tile(tile_i, &tcd, &tcd_next, &ok); ++tile_i) {
                 const int n0 = tcd.y * Cfg::kBnT;
                 const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
                 const int ngrp = (nvalid + 127) >> 7;
@@ -295,7 +308,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 TRACE_ADD(tr_acce, tr_a);
                 tc_fence_after_sync();
                 const uint32_t d0 = tmem_base + acc * Cfg::kAccCols;
-                const int pb = __ldg(p.block_row_ptr + tI), pe = __ldg(p.block_row_ptr + tI + 1);
+                const int pb = tcd.z, pe = tcd.w;
                 for (int q = pb; q < pe; q += Cfg::kBps, ++it) {
                     // stages never straddle the producer's 32-block windows (kBps divides 32)
                     const int nb = min(Cfg::kBps, min(pe - q, 32 - ((q - pb) & 31)));
@@ -352,16 +365,15 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         bool ok = true;
         TRACE_DECL(tr_accf);
         TRACE_T0(tr_start);
-        int ti;
-        for (; ok && next_tile(tile_i, &ti, &ok); ++tile_i) {
-            const int2 tcd = __ldg(p.tiles + ti);
+        int4 tcd, tcd_next;
+        for (; ok && next_tile(tile_i, &tcd, &tcd_next, &ok); ++tile_i) {
             const int tI = tcd.x;
             const int n0 = tcd.y * Cfg::kBnT;
             const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
             const int ngrp = (nvalid + 127) >> 7;
             const int acc = tile_i & 1;
             const uint32_t aph = (tile_i >> 1) & 1u;
-            const bool has_blocks = p.block_row_ptr[tI + 1] > p.block_row_ptr[tI];
+            const bool has_blocks = tcd.w > tcd.z;
             TRACE_T0(tr_a);
             if (!__all_sync(0xffffffffu, mbar_wait(accf_bar(acc), aph, ctl, 4))) { ok = false; break; }
             TRACE_ADD(tr_accf, tr_a);

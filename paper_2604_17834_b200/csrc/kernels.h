@@ -10,7 +10,7 @@ namespace spmm {
 struct BcsrParams {
     const int32_t* block_row_ptr;
     const int32_t* block_col_idx;
-    const int2* tiles;        // {block-row, token tile}, CTA-major
+    const int4* tiles;        // {block-row, token tile, first stored block, end block}, CTA-major
     const int32_t* cta_ptr;   // [grid+1] ranges of tiles
     void* C;            // fp32 or the input's 16-bit type; [m][N], or [N][m] with column-major operands
     int64_t m, N;
