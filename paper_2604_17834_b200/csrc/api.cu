@@ -529,9 +529,6 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
     if (!groups) groups = N >= 128 * gmax ? gmax : (N > 128 ? 2 : 1);
     // keep at least ~8 tiles per CTA so that the schedule has something to balance
     while (groups > 1 && f.nbr * ((N + 128 * groups - 1) / (128 * groups)) < 8 * h->n_ctas) groups >>= 1;
-#ifdef SPMM_FORCE_GROUPS
-    groups = SPMM_FORCE_GROUPS;
-#endif
     const int bnt = 128 * groups;
     const int n_tt = static_cast<int>((N + bnt - 1) / bnt);
     // slab: token tiles whose B rows (k x slab columns) stay within ~16 MB of L2 (C streams through the same cache)

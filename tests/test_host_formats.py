@@ -249,3 +249,17 @@ def test_empty_matrix(lib):
     h = lib.spmm_bcsr_create_csr(32, 10, rp, np.zeros(0, np.int32), np.zeros(0, np.uint16), "bf16", 16, host_only=True)
     assert lib.spmm_get_info(h)["n_units"] == 0
     lib.spmm_destroy(h)
+
+
+def test_binding_structs_match_the_header(lib, tmp_path):
+    """The ctypes mirrors of spmm_opts_t / spmm_info_t have the sizes a C compiler gives the
+    header's structs (the header must also compile as plain C)."""
+    import ctypes, os, subprocess
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "sizes.c"
+    src.write_text('#include <stdio.h>\n#include "spmm_b200.h"\n'
+                   'int main(void){printf("%zu %zu\\n", sizeof(spmm_opts_t), sizeof(spmm_info_t));return 0;}\n')
+    exe = tmp_path / "sizes"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(root, "include"), str(src), "-o", str(exe)], check=True)
+    so, si = (int(x) for x in subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split())
+    assert so == ctypes.sizeof(lib.SpmmOpts) and si == ctypes.sizeof(lib.SpmmInfo)
