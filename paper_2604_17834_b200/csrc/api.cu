@@ -101,6 +101,8 @@ struct spmm_handle_s {
     int32_t* d_items = nullptr;
     int32_t* d_fills = nullptr;
     int32_t* d_bin_fill = nullptr;
+    int32_t* d_fills_narrow = nullptr;    // WCSR narrow-operand variant (2-byte types, height 16)
+    int32_t* d_bin_fill_narrow = nullptr;
     int32_t* d_merge = nullptr;      // window | first | nparts, each [n_merge]
     int n_merge = 0;
     int* d_status = nullptr;
@@ -146,6 +148,8 @@ void free_handle(spmm_handle_s* h) {
         cudaFree(h->d_items);
         cudaFree(h->d_fills);
         cudaFree(h->d_bin_fill);
+        cudaFree(h->d_fills_narrow);
+        cudaFree(h->d_bin_fill_narrow);
         cudaFree(h->d_merge);
         cudaFree(h->d_status);
         cudaFree(h->d_partial);
@@ -312,6 +316,10 @@ int upload_wcsr_plan(spmm_handle_s* h) {
     }
     if (!rc) rc = upload(&h->d_fills, f.fills.data(), f.fills.size() * 4);
     if (!rc) rc = upload(&h->d_bin_fill, f.bin_fill.data(), f.bin_fill.size() * 4);
+    if (!rc && !f.bin_fill_narrow.empty()) {
+        rc = upload(&h->d_fills_narrow, f.fills_narrow.data(), f.fills_narrow.size() * 4);
+        if (!rc) rc = upload(&h->d_bin_fill_narrow, f.bin_fill_narrow.data(), f.bin_fill_narrow.size() * 4);
+    }
     if (!rc) rc = upload(&h->d_merge, mg.data(), mg.size() * 4);
     return rc;
 }
@@ -625,8 +633,10 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, void* C, float* partial, in
     WcsrParams p;
     p.bin_ptr = h->d_bin_ptr;
     p.items = reinterpret_cast<const int4*>(h->d_items);
-    p.fills = reinterpret_cast<const int2*>(h->d_fills);
-    p.bin_fill = h->d_bin_fill;
+    // narrow dense operand: the variant whose stages hold more columns
+    const bool narrow = h->d_bin_fill_narrow != nullptr && N <= kWcsrNarrowMaxN;
+    p.fills = reinterpret_cast<const int2*>(narrow ? h->d_fills_narrow : h->d_fills);
+    p.bin_fill = narrow ? h->d_bin_fill_narrow : h->d_bin_fill;
     p.col_idx = h->d_idx;
     p.packed = h->d_vals;
     p.B = B;
@@ -645,7 +655,7 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, void* C, float* partial, in
     if (!f.tasks.empty()) {
         int rc = ensure_tmB(h, B, N, 1);
         if (rc) return rc;
-        cudaError_t e = launch_wcsr(h->dtype, f.wh, h->c16, h->tmB, p, h->sms, stream);
+        cudaError_t e = launch_wcsr(h->dtype, f.wh, h->c16, narrow ? 1 : 0, h->tmB, p, h->sms, stream);
         if (e != cudaSuccess) return SPMM_ERR_CUDA;
     }
     MergeParams mp;

@@ -286,22 +286,30 @@ int plan_wcsr(WcsrHost* out, int T, int n_bins, int es) {
     // pipeline schedule: one fill per stage-sized run of columns (16 KB of gathered B rows at
     // 128 tokens: 64 columns of a 2-byte type, 32 of a 4-byte type), bin-major
     out->kt = wcsr_stage_cols(es);
-    out->fills.clear();
-    out->bin_fill.assign(static_cast<size_t>(n_bins) + 1, 0);
-    for (int j = 0; j < n_bins; ++j) {
-        for (int32_t i = out->bin_ptr[j]; i < out->bin_ptr[j + 1]; ++i) {
-            const WcsrTask& tk = out->tasks[out->bin_tasks[i]];
-            const int32_t base = out->window_row_ptr[tk.window] + tk.q0;
-            for (int32_t done = 0; done < tk.count; done += out->kt) {
-                const int32_t cnt = std::min(out->kt, tk.count - done);
-                const int32_t first = done == 0, last = done + out->kt >= tk.count;
-                out->fills.push_back(base + done);
-                out->fills.push_back(cnt | (first << 16) | (last << 17));
+    auto cut = [&](int kt, std::vector<int32_t>* fills, std::vector<int32_t>* bin_fill) -> int {
+        fills->clear();
+        bin_fill->assign(static_cast<size_t>(n_bins) + 1, 0);
+        for (int j = 0; j < n_bins; ++j) {
+            for (int32_t i = out->bin_ptr[j]; i < out->bin_ptr[j + 1]; ++i) {
+                const WcsrTask& tk = out->tasks[out->bin_tasks[i]];
+                const int32_t base = out->window_row_ptr[tk.window] + tk.q0;
+                for (int32_t done = 0; done < tk.count; done += kt) {
+                    const int32_t cnt = std::min(kt, tk.count - done);
+                    const int32_t first = done == 0, last = done + kt >= tk.count;
+                    fills->push_back(base + done);
+                    fills->push_back(cnt | (first << 16) | (last << 17));
+                }
             }
+            if (fills->size() / 2 >= (size_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
+            (*bin_fill)[j + 1] = static_cast<int32_t>(fills->size() / 2);
         }
-        if (out->fills.size() / 2 >= (size_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
-        out->bin_fill[j + 1] = static_cast<int32_t>(out->fills.size() / 2);
-    }
+        return SPMM_OK;
+    };
+    int rc = cut(out->kt, &out->fills, &out->bin_fill);
+    out->fills_narrow.clear();
+    out->bin_fill_narrow.clear();
+    if (!rc && es == 2 && out->wh == 16) rc = cut(kWcsrNarrowCols, &out->fills_narrow, &out->bin_fill_narrow);
+    if (rc) return rc;
     return SPMM_OK;
 }
 

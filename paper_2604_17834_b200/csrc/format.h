@@ -75,6 +75,9 @@ struct WcsrHost {
     int kt = 0;
     std::vector<int32_t> fills;           // 2 * n_fills
     std::vector<int32_t> bin_fill;        // [n_bins+1]
+    // the same for the narrow-operand kernel variant (stages of kWcsrNarrowCols columns); empty
+    // unless the value type is 2 bytes wide and the window height 16
+    std::vector<int32_t> fills_narrow, bin_fill_narrow;
     // finalisation lists: windows whose C rows the merge kernel writes
     std::vector<int32_t> merge_window;    // split windows then empty windows
     std::vector<int32_t> merge_first;     // first slot (split) or -1 (empty)

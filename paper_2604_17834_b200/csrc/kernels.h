@@ -53,6 +53,11 @@ constexpr int bcsr_blocks_per_stage(int b) { return b == 16 ? 4 : (b == 32 ? 2 :
 #define WCSR_STAGE_ROW_BYTES 128
 #endif
 constexpr int wcsr_stage_cols(int es) { return WCSR_STAGE_ROW_BYTES / es; }
+// Narrow dense operands (2-byte types, window height 16, N <= 64): a gathered row is one 128-byte
+// segment instead of two, so a stage of the same size class holds 96 columns (12 KB of rows +
+// 3 KB of A): a third fewer stage hand-shakes per column, which is what bounds the narrow case.
+constexpr int kWcsrNarrowCols = 96;
+constexpr int kWcsrNarrowMaxN = 64;
 constexpr int wcsr_stages(int es, int wh) { return wh == 64 ? 4 : (es == 4 ? 6 : 4); }
 constexpr int wcsr_producer_warps(int es, int wh) { return wh == 64 ? 4 : (es == 4 ? 6 : 4); }
 constexpr int wcsr_bins_per_sm(int es, int wh) { return wh == 64 ? 2 : (es == 4 ? 2 : 3); }
@@ -68,7 +73,7 @@ struct WcsrDevTask {
 struct WcsrParams {
     const int32_t* bin_ptr;      // [n_bins+1] ranges of items
     const int4* items;           // {window, partial slot or -1, columns, 0} of every task, bin-major
-    const int2* fills;           // {first padded column, count | first<<16 | last<<17}, bin-major
+    const int2* fills;           // {first padded column, count | first<<16 | last<<17}, bin-major (cut to the launch's stage size)
     const int32_t* bin_fill;     // [n_bins+1] fill ranges
     const int32_t* col_idx;      // window_col_idx [P]
     const uint8_t* packed;       // packed A values
@@ -85,7 +90,8 @@ struct WcsrParams {
 
 // dtype: 0 bf16, 1 fp16, 2 tf32.  groups: 1 or 2.  tmB: 2-D map of B (k rows x N), box = 128
 // bytes x 1 row, 128-byte swizzle (32-byte atoms for tf32), used in row-gather mode.
-cudaError_t launch_wcsr(int dtype, int wh, int c16, const CUtensorMap& tmB, const WcsrParams& p, int sms,
+// narrow: the N <= 64 variant for 2-byte types at window height 16 (p.fills / p.bin_fill cut to kWcsrNarrowCols).
+cudaError_t launch_wcsr(int dtype, int wh, int c16, int narrow, const CUtensorMap& tmB, const WcsrParams& p, int sms,
                         cudaStream_t stream);
 
 struct MergeParams {

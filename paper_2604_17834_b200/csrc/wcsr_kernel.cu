@@ -35,13 +35,14 @@ namespace {
 // tensor pipe takes a 128 x 16 MMA every 39 cycles whether or not it depends on the previous
 // one, and the extra TMEM loads lengthen the epilogue.)
 
-template <int ES, int WH, int KT, int STAGES>
+template <int ES, int WH, int KT, int STAGES, bool NARROW = false>
 struct WcsrCfg {
     static constexpr int kWH = WH;                          // window height = MMA N
     static constexpr int kKStep = 32 / ES;                  // columns per MMA (= b_col)
     static constexpr int kBnT = 128;                        // tokens per tile = TMEM lanes
-    static constexpr int kRowBytes = kBnT * ES;
-    static constexpr int kSegs = kRowBytes / 128;           // 128-byte segments per gathered row
+    // 128-byte segments per gathered row: all 128 tokens, or (narrow: N <= 64, 2-byte types) one
+    static constexpr int kSegs = NARROW ? 1 : kBnT * ES / 128;
+    static constexpr int kRowBytes = kSegs * 128;
     static constexpr int kGathers = (KT / 4) * kSegs;       // row-gather instructions per full fill
     static constexpr int kRounds = (kGathers + 31) / 32;    // per lane
     static constexpr int kAtomStride = KT * 128;            // bytes between MN atoms
@@ -58,7 +59,8 @@ struct WcsrCfg {
     static constexpr int kTmemCols = kNAcc * kAccCols;      // 64 or 256
     static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 + 256;
     static_assert(KT % 8 == 0 && KT % kKStep == 0 && KT <= 128, "stage shape");
-    static_assert(kGathers % 32 == 0 || kGathers == 16, "gather instructions are dealt to warps");
+    static_assert(kGathers <= 32, "one gather instruction per lane and fill");
+    static_assert(!NARROW || (ES == 2 && WH == 16), "narrow variant: 2-byte types, window height 16");
     static_assert(kStageBytes % 1024 == 0, "stage alignment");
 };
 
@@ -80,10 +82,10 @@ struct SegIter {
     }
 };
 
-template <int ES, int FMT, int WH, int KT, int STAGES, int PW, int CT>
-__global__ void __launch_bounds__((PW + 5) * 32, WcsrCfg<ES, WH, KT, STAGES>::kCtasPerSm)
+template <int ES, int FMT, int WH, int KT, int STAGES, int PW, int CT, bool NARROW>
+__global__ void __launch_bounds__((PW + 5) * 32, WcsrCfg<ES, WH, KT, STAGES, NARROW>::kCtasPerSm)
 wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
-    using Cfg = WcsrCfg<ES, WH, KT, STAGES>;
+    using Cfg = WcsrCfg<ES, WH, KT, STAGES, NARROW>;
     constexpr int kWH = WH;
     constexpr int kProducerWarps = PW;          // warps 0 .. PW-1; MMA warp PW; epilogue PW+1 .. PW+4
     constexpr int kMmaWarp = PW;
@@ -248,7 +250,10 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
         // The whole warp walks the fill list (descriptor windows via shuffles) and waits for
         // stages and accumulators; one elected lane issues the MMAs and commits.
         constexpr uint32_t idesc = make_idesc(FMT, 128, kWH, 1, 0);
-        const uint64_t adesc0 = make_smem_desc(0, Cfg::kAtomStride, ES == 2 ? 1024 : 512, ES == 2 ? SWZ_128B : SWZ_128B_BASE32B);
+        // narrow variant: only the first 64-token atom is staged; the MMA's second atom is made to
+        // alias it (atom stride 0) so that no address outside the stage is read; its TMEM lanes
+        // (tokens 64..127) are never stored
+        const uint64_t adesc0 = make_smem_desc(0, NARROW ? 0 : Cfg::kAtomStride, ES == 2 ? 1024 : 512, ES == 2 ? SWZ_128B : SWZ_128B_BASE32B);
         const uint64_t bdesc0 = make_smem_desc(0, kWH * 16, 128, SWZ_NONE);
         const bool leader = elect_one();
         TRACE_DECL(tr_full);
@@ -469,11 +474,12 @@ wcsr_merge_kernel(const MergeParams p) {
     }
 }
 
-template <int ES, int FMT, int WH, int CT>
+template <int ES, int FMT, int WH, int CT, bool NARROW = false>
 cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
-    constexpr int KT = wcsr_stage_cols(ES), STAGES = wcsr_stages(ES, WH), PW = wcsr_producer_warps(ES, WH);
-    using Cfg = WcsrCfg<ES, WH, KT, STAGES>;
-    auto kfn = wcsr_spmm_kernel<ES, FMT, WH, KT, STAGES, PW, CT>;
+    constexpr int KT = NARROW ? kWcsrNarrowCols : wcsr_stage_cols(ES);
+    constexpr int STAGES = wcsr_stages(ES, WH), PW = wcsr_producer_warps(ES, WH);
+    using Cfg = WcsrCfg<ES, WH, KT, STAGES, NARROW>;
+    auto kfn = wcsr_spmm_kernel<ES, FMT, WH, KT, STAGES, PW, CT, NARROW>;
     static int occ = 0;
     if (occ == 0) {
         cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
@@ -502,7 +508,12 @@ cudaError_t launch_wh(int dtype, int c16, const CUtensorMap& tmB, const WcsrPara
 
 }  // namespace
 
-cudaError_t launch_wcsr(int dtype, int wh, int c16, const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
+cudaError_t launch_wcsr(int dtype, int wh, int c16, int narrow, const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
+    if (narrow) {
+        if (wh != 16 || (dtype != 0 && dtype != 1)) return cudaErrorInvalidValue;
+        if (dtype == 1) return c16 ? launch_one<2, 0, 16, 1, true>(tmB, p, sms, stream) : launch_one<2, 0, 16, 0, true>(tmB, p, sms, stream);
+        return c16 ? launch_one<2, 1, 16, 1, true>(tmB, p, sms, stream) : launch_one<2, 1, 16, 0, true>(tmB, p, sms, stream);
+    }
     if (wh == 16) return launch_wh<16>(dtype, c16, tmB, p, sms, stream);
     if (wh == 64) return launch_wh<64>(dtype, c16, tmB, p, sms, stream);
     return cudaErrorInvalidValue;
