@@ -112,6 +112,8 @@ def workload_table():
                                       fp8_linear(18944, 3584, 1003))
     t["cfg3_bcsr_llm_down_cm_fp8"] = ("configs[2] down shape with E4M3 weights and activations, X [N][k] in, fp32 Y [N][m] out",
                                       fp8_linear(3584, 18944, 1013))
+    t["cfg5_wcsr_rmat_s19_n128"] = ("configs[4] recipe at 2^19 rows (a profiling-sized case: B 134 MB), N=128",
+                                    lambda: dict(kind="wcsr", a=wl.rmat(scale=19), dtype="fp16", size=16, N=128, Bdist=("normal", 0.0, 1.0)))
     t["cfg2_wcsr_irregular_wh64"] = ("configs[1] with 64-row windows", tall(cfg2))
     t["cfg5_wcsr_rmat_n128_wh64"] = ("configs[4] N=128 with 64-row windows", tall(cfg5(128)))
     t["cfg3_bcsr_llm_gate_dyn"] = ("configs[2] gate, dynamic tile scheduling", variant(cfg3_gate, dyn=True))
