@@ -244,3 +244,10 @@ def bcsr_tile_schedule(block_row_ptr, n_tt, slab_w, n_ctas, fixed_cost=4):
     cta_ptr[1:] = np.cumsum([len(x) for x in lists])
     tiles = np.asarray([p for x in lists for p in x], dtype=np.int32).reshape(-1, 2)
     return cta_ptr.astype(np.int32), tiles
+
+
+def padded_width(N, BN):
+    """Dense width after padding to a whole number of N-tiles of BN columns, and the share of
+    the padded width that is padding (the cost Sec. 4.3 discusses for its N-tile sweep)."""
+    padded = -(-N // BN) * BN
+    return padded, (padded - N) / N

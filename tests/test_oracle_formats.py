@@ -216,3 +216,16 @@ def test_generators_are_deterministic_and_shaped():
     keys = np.repeat(np.arange(2000), np.diff(w["row_ptr"])) * 2000 + w["col_idx"]
     assert np.all(np.diff(keys) > 0)
     assert np.diff(w["row_ptr"]).min() >= 1
+
+
+def test_tile_padding_numbers_of_the_paper():
+    """tests/golden/sec4_3_tile_padding.txt: the padded widths and waste percentages Sec. 4.3
+    prints for its N-tile sweep (waste relative to the unpadded width, rounded as printed)."""
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "sec4_3_tile_padding.txt")
+    rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    assert len(rows) >= 5
+    for N, BN, padded, pct in ((int(a), int(b), int(c), int(d)) for a, b, c, d in rows):
+        got_padded, waste = F.padded_width(N, BN)
+        assert got_padded == padded
+        assert round(100.0 * waste) == pct
