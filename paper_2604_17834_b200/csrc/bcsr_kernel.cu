@@ -478,7 +478,13 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (use > 0 && !mbar_wait(sche_bar(slot), (use - 1u) & 1u, ctl, 6)) break;
                 mbar_arrive_expect_tx(schf_bar(slot), 16);
                 clc_try_cancel(sched_resp + 16u * slot, schf_bar(slot));
-                if (!mbar_wait(schf_bar(slot), use & 1u, ctl, 7)) break;
+                if (!mbar_wait(schf_bar(slot), use & 1u, ctl, 7)) {
+                    // leaving early: the answer of the request just issued must still land in
+                    // this CTA's shared memory before the CTA may exit (bounded)
+                    const uint64_t t0 = globaltimer_ns();
+                    while (!mbar_try_wait(schf_bar(slot), use & 1u) && globaltimer_ns() - t0 < 2000000ull) {}
+                    break;
+                }
                 uint32_t x;
                 if (!clc_query(sched_resp + 16u * slot, &x)) break;      // no CTA left to cancel: the walk ends
             }

@@ -166,15 +166,18 @@ def test_bad_run_arguments(lib):
     lib.spmm_destroy(h)
 
 
-@pytest.mark.parametrize("kind", ["bcsr", "wcsr"])
+@pytest.mark.parametrize("kind", ["bcsr", "wcsr", "bcsr_dynamic"])
 def test_wait_that_runs_out_is_reported_and_the_context_survives(lib, kind):
     """Every wait inside the kernels is bounded.  With the bound set to zero the first wait
     for operands that are still on their way runs out: the kernel leaves early
     through its normal teardown, spmm_check reports SPMM_ERR_DEV_TIMEOUT, and the same
     handle then works again once the bound is restored."""
-    if kind == "bcsr":
+    if kind.startswith("bcsr"):
         a, dtype, size, N = wl.bcsr_sweep(404, m=2048, k=2048, b=64, density=0.3, dtype="fp16"), "fp16", 64, 1024
         mk = lib.spmm_bcsr_create_csr
+        if kind == "bcsr_dynamic":       # tiles handed out at run time: the scheduler warp's waits are bounded too
+            def mk(*args):
+                return lib.spmm_bcsr_create_csr(*args, schedule=lib.SCHED_DYNAMIC)
     else:
         a, dtype, size, N = wl.wcsr_irregular(seed=405, m=20000, dtype="tf32"), "tf32", 16, 128
         mk = lib.spmm_wcsr_create_csr
