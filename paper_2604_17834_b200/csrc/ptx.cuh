@@ -157,7 +157,7 @@ __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
 }
 
-// 2-D tiled load, no multicast: box at element coordinates (x = inner, y = outer).
+// 2-D tiled load into this CTA only: box at element coordinates (x = inner, y = outer).
 // x * element size must be a multiple of 16 bytes.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* m, uint32_t bar,
                                             int32_t x, int32_t y) {
@@ -193,7 +193,7 @@ __device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap
         : "memory");
 }
 
-// 3-D tiled load, no multicast: box at element coordinates (x = innermost, y, z = outermost).
+// 3-D tiled load into this CTA only: box at element coordinates (x = innermost, y, z = outermost).
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* m, uint32_t bar,
                                             int32_t x, int32_t y, int32_t z) {
     asm volatile(
@@ -205,7 +205,7 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* m, 
 
 // Row gather (tile::gather4): four rows y0..y3 of a 2-D tensor, each starting at element x and
 // as wide as the tensor map's box (whose row extent is 1), land as four consecutive box rows
-// at dst.  Rows outside the tensor (e.g. index -1) are filled with zeros.  No multicast.
+// at dst.  Rows outside the tensor (e.g. index -1) are filled with zeros.
 __device__ __forceinline__ void tma_gather4_2d(uint32_t dst, const CUtensorMap* m, uint32_t bar,
                                                int32_t x, int32_t y0, int32_t y1, int32_t y2, int32_t y3) {
     asm volatile(
