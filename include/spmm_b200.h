@@ -47,7 +47,10 @@ typedef enum {
     SPMM_ERR_CUDA = -6,          /* a CUDA call or a launch failed (no device, bad context)   */
     SPMM_ERR_DEV_TIMEOUT = -7,   /* a bounded wait inside a kernel ran out (see spmm_check)   */
     SPMM_ERR_HOST_ONLY = -8,     /* the handle was created host_only and cannot run           */
-    SPMM_ERR_TOO_LARGE = -9      /* a size exceeds a fixed capacity (int32 index, scratch)    */
+    SPMM_ERR_TOO_LARGE = -9,     /* a size exceeds a fixed capacity (int32 index, scratch)    */
+    SPMM_ERR_DEV_BOUNDS = -10    /* a kernel met an index outside its range and stopped using
+                                    it (reported by spmm_check; cannot happen with a handle
+                                    this library built)                                       */
 } spmm_status_t;
 
 /* Value type of A and B.  Accumulation and C are always fp32. */

@@ -838,7 +838,7 @@ int spmm_check(spmm_handle_t h) {
     if (cudaMemcpy(st, h->d_status, sizeof(st), cudaMemcpyDeviceToHost) != cudaSuccess) return SPMM_ERR_CUDA;
     if (st[0] != 0) {
         cudaMemset(h->d_status, 0, sizeof(st));
-        return SPMM_ERR_DEV_TIMEOUT;
+        return st[0] == 2 ? SPMM_ERR_DEV_BOUNDS : SPMM_ERR_DEV_TIMEOUT;
     }
     return SPMM_OK;
 }
@@ -997,6 +997,7 @@ const char* spmm_status_string(int code) {
         case SPMM_ERR_DEV_TIMEOUT: return "a bounded wait inside a kernel ran out";
         case SPMM_ERR_HOST_ONLY: return "handle was created host_only";
         case SPMM_ERR_TOO_LARGE: return "size exceeds a fixed capacity";
+        case SPMM_ERR_DEV_BOUNDS: return "a kernel met an index outside its range";
         default: return "unknown status";
     }
 }
