@@ -141,6 +141,8 @@ DEFAULT_OTHERS = ["cfg1_bcsr_tiny", "cfg3_bcsr_llm_gate", "cfg3_bcsr_llm_down",
                   "cfg3_bcsr_llm_gate_cm_fp8", "cfg3_bcsr_llm_down_cm_fp8", "cfg2_wcsr_irregular_wh64",
                   "cfg4_bcsr_sweep_b64_d0.1_dyn"]
 
+L2_TO_SM_GBS = 19800.0      # measured aggregate L2 -> shared-memory TMA rate (148 SMs x 70 B/cycle at 1.9 GHz)
+
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures whose
 # summaries are under profiles/ (None where no capture of that exact launch exists).
 NCU_DRAM_TRAFFIC = {
@@ -253,6 +255,19 @@ def roofline_of(info, ms, pk):
         r = {"bound": "tensor", "achieved": ach, "peak": tc_peak, "unit": "TFLOP/s", "frac": ach / tc_peak}
     r.update({"peak_source": pk["source"], "model_bytes": model_bytes, "t_roof_us": max(t_hbm, t_tc) * 1e6,
               "gather_bytes": info["bytes_gather"], "traffic": None})
+    # Second ceiling, context only: every staged operand byte crosses L2 -> shared memory once; the
+    # aggregate TMA rate measured on this GPU type with an L2-resident source is 19.8 TB/s
+    # (microbenchmark described in the design doc section 5).
+    # the stored values of A are fetched once per token tile (BCSR: the plan's tile width; WCSR: 128)
+    tile = info["plan_token_tile"] if info["format"] == 0 and info["plan_token_tile"] else 128
+    n_tt = -(-int(info["plan_n"] if info["format"] == 0 and info["plan_n"] else 0) // tile) if info["format"] == 0 else None
+    if info["format"] == 0:
+        a_passes = max(1, n_tt)
+    else:
+        a_passes = max(1, -(-int(round(info["flops_stored"] / (2.0 * max(1, info["stored_values"])))) // 128))
+    l2_bytes = info["bytes_gather"] + info["bytes_a"] * a_passes
+    r["l2_to_sm"] = {"bytes": l2_bytes, "rate_gbs": L2_TO_SM_GBS, "achieved_gbs": l2_bytes / t / 1e9,
+                     "frac": l2_bytes / t / 1e9 / L2_TO_SM_GBS}
     return r
 
 
@@ -281,6 +296,7 @@ def time_workload(torch, lib, w, steps, warmup, flush):
             lib.spmm_run(h, B.data_ptr(), C.data_ptr(), N, st)
         torch.cuda.synchronize()
         lib.spmm_check(h)
+        info = lib.spmm_get_info(h, N)          # again: the BCSR plan fields are filled by the first run
         evs = []
         for _ in range(steps):
             flush.zero_()
