@@ -109,7 +109,18 @@ typedef struct {
     int32_t layout;      /* spmm_layout_t; SPMM_COLMAJOR with a WCSR handle is UNSUPPORTED    */
     int32_t schedule;    /* spmm_sched_t; with SPMM_SCHED_DYNAMIC the exported tile list is a
                             single range (TILE_PTR = {0, n_tiles}) in the global order       */
-    int32_t reserved[9];
+    int32_t stack_min_fill; /* BCSR row groups (no counterpart in the paper): where 128 / b
+                            block-rows store blocks in mostly the same block columns, the
+                            kernel computes them together from 128-row stacked blocks (absent
+                            sub-blocks zero), so that each slice of the dense operand is staged
+                            once for all of them.  Candidates are runs of 128 / b consecutive
+                            non-empty block-rows in ROW_ORDER; one is taken when at least this
+                            percentage of its sub-blocks is stored.  0 = default (30 / 45 / 75
+                            for b = 16 / 32 / 64), -1 = off, 1..100 = threshold.  A private
+                            second copy of the grouped rows' values is kept on the device; the
+                            exported format arrays and nnz_stored are unaffected.  Ignored for
+                            b = 128, E4M3 inputs and the dynamic schedule.                    */
+    int32_t reserved[8];
 } spmm_opts_t;
 
 typedef struct {
@@ -140,7 +151,8 @@ typedef struct {
     int32_t plan_slab_tiles; /* token tiles per L2 slab                                       */
     int32_t n_bins;          /* WCSR: bins of the static task schedule (0 for BCSR): n_ctas x
                                 the resident CTAs per SM of the kernel for this value type     */
-    int32_t reserved0;
+    int32_t n_stacked_rows;  /* BCSR: block-rows computed as members of row groups            */
+    int64_t n_stack_blocks;  /* BCSR: 128-row stacked blocks those groups hold                 */
 } spmm_info_t;
 
 /* Arrays spmm_export can return, in their canonical (paper) layout. */
@@ -150,7 +162,15 @@ typedef enum {
     SPMM_X_BCSR_BLOCKS = 2,         /* dtype [n_blocks][b][b] row-major, zero filled          */
     SPMM_X_BCSR_ROW_ORDER = 3,      /* int32 [block-rows]: schedule order, longest first      */
     SPMM_X_BCSR_TILE_PTR = 4,       /* int32 [n_ctas+1]: per-CTA ranges of TILES (needs a plan) */
-    SPMM_X_BCSR_TILES = 5,          /* int32 [n_tiles][2]: block-row, token tile; CTA-major    */
+    SPMM_X_BCSR_TILES = 5,          /* int32 [n_tiles][2]: block-row, token tile; CTA-major
+                                       (block-rows outside the row groups only)               */
+    SPMM_X_BCSR_STACK_ROWS = 6,     /* int32 [groups][128/b]: block-rows of every row group     */
+    SPMM_X_BCSR_STACK_PTR = 7,      /* int32 [groups+1]: ranges of STACK_COL_IDX                */
+    SPMM_X_BCSR_STACK_COL_IDX = 8,  /* int32 [n_stack_blocks]: block columns of a group's union,
+                                       ascending                                              */
+    SPMM_X_BCSR_STACK_TILE_PTR = 9, /* int32 [n_ctas+1]: per-CTA ranges of STACK_TILES (needs a
+                                       plan)                                                  */
+    SPMM_X_BCSR_STACK_TILES = 20,   /* int32 [n][2]: row group, 256-column token tile; CTA-major */
     SPMM_X_WCSR_WINDOW_ROW_PTR = 10,/* int32 [ceil(m/h)+1], in columns                        */
     SPMM_X_WCSR_WINDOW_COL_IDX = 11,/* int32 [P], -1 on padding                               */
     SPMM_X_WCSR_VALUES = 12,        /* dtype [h][P] row-major                                 */

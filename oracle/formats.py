@@ -214,28 +214,38 @@ def task_bins(plan, n_bins, fixed_cost=32):
     return bin_ptr.astype(np.int32), np.asarray(tasks, dtype=np.int32)
 
 
-def bcsr_tile_schedule(block_row_ptr, n_tt, slab_w, n_ctas, fixed_cost=4):
+def bcsr_tile_schedule(block_row_ptr, n_tt, slab_w, n_ctas, fixed_cost=4, units=None, lens=None,
+                       unit_cost=1, initial=None, return_loads=False):
     """Static schedule of BCSR tiles (block-row, token tile) over n_ctas CTAs.
 
     Addresses the imbalance Sec. 3.5 / Sec. 4.2 (opt6) report for a fixed tile
     order.  Tiles are taken slab by slab (slab_w consecutive token tiles), inside a
     slab in bcsr_row_order (most stored blocks first), inside a block-row by
     ascending token tile; each goes to the CTA whose load is smallest at that
-    moment (ties: lowest CTA), load = sum of (stored blocks + fixed_cost); loads
-    carry over between slabs.  Returns (cta_ptr int32 [n_ctas+1],
-    tiles int32 [n_tiles, 2]) with every CTA's tiles in the order it received them.
+    moment (ties: lowest CTA), load = sum of (stored blocks + fixed_cost) * unit_cost
+    on top of the CTA's initial load (0 unless given); loads carry over between
+    slabs.  Returns (cta_ptr int32 [n_ctas+1], tiles int32 [n_tiles, 2]) with every
+    CTA's tiles in the order it received them (and the CTAs' final loads when
+    return_loads).
+
+    ``units`` / ``lens`` replace the block-rows and their lengths by any list of
+    units given in schedule order (a subset of the block-rows, or row groups).
     """
     import heapq
-    brp = np.asarray(block_row_ptr, dtype=np.int64)
-    lens = np.diff(brp)
-    order = bcsr_row_order(brp)
-    heap = [(0, c) for c in range(n_ctas)]
+    if units is None:
+        brp = np.asarray(block_row_ptr, dtype=np.int64)
+        all_lens = np.diff(brp)
+        units = bcsr_row_order(brp)
+        lens = all_lens[units]
+    units = [int(u) for u in units]
+    lens = [int(x) for x in lens]
+    heap = [(0 if initial is None else int(initial[c]), c) for c in range(n_ctas)]
     heapq.heapify(heap)
     lists = [[] for _ in range(n_ctas)]
     for t0 in range(0, n_tt, slab_w):
         t1 = min(n_tt, t0 + slab_w)
-        for I in order.tolist():
-            cost = int(lens[I]) + fixed_cost
+        for I, ln in zip(units, lens):
+            cost = (ln + fixed_cost) * unit_cost
             for t in range(t0, t1):
                 load, c = heapq.heappop(heap)
                 lists[c].append((I, t))
@@ -243,7 +253,43 @@ def bcsr_tile_schedule(block_row_ptr, n_tt, slab_w, n_ctas, fixed_cost=4):
     cta_ptr = np.zeros(n_ctas + 1, dtype=np.int64)
     cta_ptr[1:] = np.cumsum([len(x) for x in lists])
     tiles = np.asarray([p for x in lists for p in x], dtype=np.int32).reshape(-1, 2)
+    if return_loads:
+        loads = np.zeros(n_ctas, dtype=np.int64)
+        for load, c in heap:
+            loads[c] = load
+        return cta_ptr.astype(np.int32), tiles, loads
     return cta_ptr.astype(np.int32), tiles
+
+
+def bcsr_row_groups(block_row_ptr, block_col_idx, b, min_fill_pct):
+    """Row groups of the BCSR kernel (a device-side regrouping with no counterpart in the
+    paper, whose BCSR blocks are all b x b, Sec. 2.3): R = 128 // b block-rows that store
+    blocks in mostly the same block columns are computed together, one 128-row stacked block
+    per block column of their union.
+
+    Rule: walk bcsr_row_order (most stored blocks first, stable); every run of R consecutive
+    block-rows in that order is a candidate while its last row is non-empty; a candidate is
+    accepted when 100 * (stored blocks of its rows) >= min_fill_pct * R * |union of their
+    block columns|.  Returns (rows int32 [ng, R], ptr int32 [ng+1], col_idx int32 [ns]):
+    member rows in row order, and per group the ascending union of block columns.
+    """
+    brp = np.asarray(block_row_ptr, dtype=np.int64)
+    bci = np.asarray(block_col_idx, dtype=np.int64)
+    R = 128 // b
+    order = bcsr_row_order(brp)
+    rows, ptr, cols = [], [0], []
+    for r0 in range(0, len(order) - R + 1, R):
+        cand = order[r0:r0 + R]
+        if brp[cand[-1] + 1] == brp[cand[-1]]:
+            break
+        stored = int(sum(brp[I + 1] - brp[I] for I in cand))
+        union = np.unique(np.concatenate([bci[brp[I]:brp[I + 1]] for I in cand]))
+        if 100 * stored >= min_fill_pct * R * len(union):
+            rows.append([int(I) for I in cand])
+            cols.extend(union.tolist())
+            ptr.append(len(cols))
+    return (np.asarray(rows, dtype=np.int32).reshape(-1, R), np.asarray(ptr, dtype=np.int32),
+            np.asarray(cols, dtype=np.int32))
 
 
 def padded_width(N, BN):

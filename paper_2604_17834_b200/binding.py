@@ -39,6 +39,7 @@ SPMM_ERR_DEV_BOUNDS = -10
 
 X_BCSR_BLOCK_ROW_PTR, X_BCSR_BLOCK_COL_IDX, X_BCSR_BLOCKS, X_BCSR_ROW_ORDER = 0, 1, 2, 3
 X_BCSR_TILE_PTR, X_BCSR_TILES = 4, 5
+X_BCSR_STACK_ROWS, X_BCSR_STACK_PTR, X_BCSR_STACK_COL_IDX, X_BCSR_STACK_TILE_PTR, X_BCSR_STACK_TILES = 6, 7, 8, 9, 20
 X_WCSR_WINDOW_ROW_PTR, X_WCSR_WINDOW_COL_IDX, X_WCSR_VALUES, X_WCSR_TASKS = 10, 11, 12, 13
 X_WCSR_BIN_PTR, X_WCSR_BIN_TASKS = 14, 15
 
@@ -53,7 +54,7 @@ EXPORTED_SYMBOLS = (
 class SpmmOpts(ctypes.Structure):
     _fields_ = [("b_col", ctypes.c_int32), ("split_cols", ctypes.c_int32), ("host_only", ctypes.c_int32),
                 ("n_ctas", ctypes.c_int32), ("c_type", ctypes.c_int32), ("layout", ctypes.c_int32),
-                ("schedule", ctypes.c_int32), ("reserved", ctypes.c_int32 * 9)]
+                ("schedule", ctypes.c_int32), ("stack_min_fill", ctypes.c_int32), ("reserved", ctypes.c_int32 * 8)]
 
 
 class SpmmInfo(ctypes.Structure):
@@ -72,7 +73,7 @@ class SpmmInfo(ctypes.Structure):
         ("bytes_gather", ctypes.c_double), ("flops_stored", ctypes.c_double),
         ("workspace_bytes", ctypes.c_int64),
         ("plan_n", ctypes.c_int64), ("plan_token_tile", ctypes.c_int32), ("plan_slab_tiles", ctypes.c_int32),
-        ("n_bins", ctypes.c_int32), ("reserved0", ctypes.c_int32),
+        ("n_bins", ctypes.c_int32), ("n_stacked_rows", ctypes.c_int32), ("n_stack_blocks", ctypes.c_int64),
     ]
 
     def as_dict(self):
@@ -119,8 +120,10 @@ ROWMAJOR, COLMAJOR = 0, 1
 SCHED_STATIC, SCHED_DYNAMIC = 0, 1
 
 
-def _opts(b_col=0, split_cols=0, host_only=False, n_ctas=0, c_type=C_FP32, layout=ROWMAJOR, schedule=SCHED_STATIC):
+def _opts(b_col=0, split_cols=0, host_only=False, n_ctas=0, c_type=C_FP32, layout=ROWMAJOR, schedule=SCHED_STATIC,
+          stack_min_fill=0):
     o = SpmmOpts()
+    o.stack_min_fill = int(stack_min_fill)
     o.b_col, o.split_cols, o.host_only, o.n_ctas = b_col, split_cols, int(bool(host_only)), n_ctas
     o.c_type, o.layout, o.schedule = int(c_type), int(layout), int(schedule)
     return o

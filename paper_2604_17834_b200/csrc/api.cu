@@ -2,6 +2,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cstdio>
 #include <cstring>
@@ -92,6 +93,18 @@ struct spmm_handle_s {
     uint8_t* d_vals = nullptr;       // blocks / packed values
     int32_t* d_order = nullptr;      // BCSR row order
     BcsrSchedule sched;              // BCSR tile schedule of the most recent dense width
+    // BCSR row groups (stacked 128-row blocks): plan, device arrays and their own tile schedule
+    BcsrStack stack;
+    int stack_min_fill = 0;          // opts.stack_min_fill
+    BcsrSchedule sched_stack;
+    int32_t* d_sidx = nullptr;       // block columns of the stacked blocks
+    int32_t* d_srows = nullptr;      // [groups][R] member block-rows
+    uint8_t* d_svals = nullptr;      // [stacked blocks][128][b]
+    int32_t* d_stile_recs = nullptr; // {group, token tile, first stacked block, end}
+    int32_t* d_scta_ptr = nullptr;
+    CUtensorMap tmAs;                // map of d_svals
+    CUtensorMap tmB3s;               // whole-tile map of B for the stacked launch's 256-token tile
+    bool tmB3s_ok = false;
     int32_t* d_tiles = nullptr;      // {block-row, token tile} pairs (the exported schedule)
     int32_t* d_tile_recs = nullptr;  // the kernel's records: {block-row, token tile, first block, end block}
     int32_t* d_cta_ptr = nullptr;
@@ -142,6 +155,11 @@ void free_handle(spmm_handle_s* h) {
         cudaFree(h->d_tiles);
         cudaFree(h->d_tile_recs);
         cudaFree(h->d_cta_ptr);
+        cudaFree(h->d_sidx);
+        cudaFree(h->d_srows);
+        cudaFree(h->d_svals);
+        cudaFree(h->d_stile_recs);
+        cudaFree(h->d_scta_ptr);
         cudaFree(h->d_tasks);
         cudaFree(h->d_bin_ptr);
         cudaFree(h->d_bin_tasks);
@@ -209,6 +227,8 @@ int new_bcsr_handle(spmm_handle_s** hp, int64_t m, int64_t k, int dtype, int blo
     h->cs = h->c16 ? 2 : 4;
     h->col_major = opts && opts->layout == SPMM_COLMAJOR;
     h->dynamic = opts && opts->schedule == SPMM_SCHED_DYNAMIC;
+    h->stack_min_fill = opts ? opts->stack_min_fill : 0;
+    if (h->stack_min_fill > 100) { delete h; return SPMM_ERR_INVALID_ARG; }
     if (h->dynamic && (h->c16 || h->col_major)) { delete h; return SPMM_ERR_UNSUPPORTED; }
     // column-major operands: rows of X (k elements) and of Y (m elements) must be multiples of
     // 16 bytes for the tensor map and for the 16-byte pieces the epilogue writes
@@ -230,6 +250,26 @@ int encode_tmA(spmm_handle_s* h) {
                              static_cast<uint32_t>(f.b * bcsr_blocks_per_stage(f.b)), bw, swz);
     h->tmA_ok = rc == SPMM_OK;
     return rc;
+}
+
+// Row groups: the plan from the index arrays, then (unless host_only) the stacked values built on
+// the device from the uploaded blocks, the groups' index arrays and the map of the stacked values.
+int setup_stack(spmm_handle_s* h) {
+    const BcsrHost& f = h->bcsr;
+    // 16-bit types with the static schedule; b = 128 blocks already are 128 rows high
+    const bool eligible = h->es == 2 && !h->dynamic && f.b < 128 && h->stack_min_fill >= 0;
+    int rc = build_bcsr_stack(f, eligible ? h->stack_min_fill : -1, &h->stack);
+    if (rc || h->host_only || h->stack.ng == 0) return rc;
+    const BcsrStack& st = h->stack;
+    rc = stack_bcsr_device(h->d_vals, st, f.b, h->es, &h->d_svals);
+    if (!rc) rc = upload(&h->d_sidx, st.col_idx.data(), st.col_idx.size() * 4);
+    if (!rc) rc = upload(&h->d_srows, st.rows.data(), st.rows.size() * 4);
+    if (rc) return rc;
+    std::vector<int32_t>().swap(h->stack.src);        // only needed to build the values
+    const int row_bytes = f.b * h->es;                // <= 128 for b <= 64
+    const CUtensorMapSwizzle swz = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                  : (row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+    return encode_2d_16bit(&h->tmAs, h->dtype, h->d_svals, static_cast<uint64_t>(st.ns) * kStackRows, f.b, kStackRows, f.b, swz);
 }
 
 int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, const spmm_opts_t* opts) {
@@ -258,6 +298,12 @@ int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, cons
         if (rc) { free_handle(h); return rc; }
         std::vector<uint8_t>().swap(h->bcsr.blocks);   // the device copy is the one that counts
     }
+    try {
+        rc = setup_stack(h);
+    } catch (const std::bad_alloc&) {
+        rc = SPMM_ERR_ALLOC;
+    }
+    if (rc) { free_handle(h); return rc; }
     *out = h;
     return SPMM_OK;
 }
@@ -279,6 +325,13 @@ int create_bcsr_device(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* 
     }
     if (!rc) rc = upload(&h->d_order, h->bcsr.row_order.data(), h->bcsr.row_order.size() * 4);
     if (!rc) rc = encode_tmA(h);
+    if (!rc) {
+        try {
+            rc = setup_stack(h);
+        } catch (const std::bad_alloc&) {
+            rc = SPMM_ERR_ALLOC;
+        }
+    }
     if (rc) { free_handle(h); return rc; }
     *out = h;
     return SPMM_OK;
@@ -451,40 +504,46 @@ int ensure_tmB(spmm_handle_s* h, const void* B, int64_t N, int groups) {
         const CUtensorMapSwizzle swz = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                       : (row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
         rc = encode_2d_16bit(&h->tmB, h->dtype, B, static_cast<uint64_t>(N), static_cast<uint64_t>(h->k), 128, bw, swz);
-        h->tmB3_ok = false;
-        h->tmB3 = h->tmB;
         EncodeTiledFn fn = get_encode_fn();
-        if (!rc && fn && N >= 128) {
+        auto whole_tile_map = [&](int g, CUtensorMap* out, bool* ok) {
+            *ok = false;
+            *out = h->tmB;
+            if (rc || !fn || N < 128) return;
             const cuuint64_t dims[3] = {static_cast<cuuint64_t>(h->k), 128, static_cast<cuuint64_t>(N / 128)};
             const cuuint64_t strides[2] = {static_cast<cuuint64_t>(h->k) * h->es, static_cast<cuuint64_t>(h->k) * 128 * h->es};
-            const cuuint32_t box[3] = {bw, 128, static_cast<cuuint32_t>(groups)};
+            const cuuint32_t box[3] = {bw, 128, static_cast<cuuint32_t>(g)};
             const cuuint32_t estr[3] = {1, 1, 1};
             const CUtensorMapDataType dt = h->dtype == SPMM_FP8_E4M3 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
                                          : (h->dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
-            CUresult r = fn(&h->tmB3, dt, 3, const_cast<void*>(B), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CUresult r = fn(out, dt, 3, const_cast<void*>(B), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                             swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-            h->tmB3_ok = r == CUDA_SUCCESS;
-            if (!h->tmB3_ok) h->tmB3 = h->tmB;
-        }
+            *ok = r == CUDA_SUCCESS;
+            if (!*ok) *out = h->tmB;
+        };
+        whole_tile_map(groups, &h->tmB3, &h->tmB3_ok);
+        if (h->stack.ng > 0) whole_tile_map(kStackGroups, &h->tmB3s, &h->tmB3s_ok);
     } else {
         rc = encode_2d_16bit(&h->tmB, h->dtype, B, static_cast<uint64_t>(h->k), static_cast<uint64_t>(N),
                              static_cast<uint32_t>(h->bcsr.b), 64, CU_TENSOR_MAP_SWIZZLE_128B);
         // the same memory as [N / 64][k][64]: one request then brings a whole token tile
         // (2 * groups boxes); only full 64-token groups are covered, a ragged tail uses tmB
-        h->tmB3_ok = false;
-        h->tmB3 = h->tmB;
         EncodeTiledFn fn = get_encode_fn();
-        if (!rc && fn && N >= 64) {
+        auto whole_tile_map = [&](int g, CUtensorMap* out, bool* ok) {
+            *ok = false;
+            *out = h->tmB;
+            if (rc || !fn || N < 64) return;
             const cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(h->k), static_cast<cuuint64_t>(N / 64)};
             const cuuint64_t strides[2] = {static_cast<cuuint64_t>(N) * 2, 128};
-            const cuuint32_t box[3] = {64, static_cast<cuuint32_t>(h->bcsr.b), static_cast<cuuint32_t>(2 * groups)};
+            const cuuint32_t box[3] = {64, static_cast<cuuint32_t>(h->bcsr.b), static_cast<cuuint32_t>(2 * g)};
             const cuuint32_t estr[3] = {1, 1, 1};
             const CUtensorMapDataType dt = h->dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
-            CUresult r = fn(&h->tmB3, dt, 3, const_cast<void*>(B), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CUresult r = fn(out, dt, 3, const_cast<void*>(B), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-            h->tmB3_ok = r == CUDA_SUCCESS;
-            if (!h->tmB3_ok) h->tmB3 = h->tmB;
-        }
+            *ok = r == CUDA_SUCCESS;
+            if (!*ok) *out = h->tmB;
+        };
+        whole_tile_map(groups, &h->tmB3, &h->tmB3_ok);
+        if (h->stack.ng > 0) whole_tile_map(kStackGroups, &h->tmB3s, &h->tmB3s_ok);
     }
     if (rc) return rc;
     h->tmB_ptr = B;
@@ -544,11 +603,51 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
     int64_t sw = slab_cols / bnt;
     if (sw < 1) sw = 1;
     if (sw > n_tt) sw = n_tt;
-    BcsrSchedule sc;
+    BcsrSchedule sc, ss;
+    const BcsrStack& st = h->stack;
     int rc;
     try {
         // dynamic scheduling: one list in the global order (slab by slab, longest block-row first)
-        rc = build_bcsr_schedule(f, n_tt, static_cast<int>(sw), h->dynamic ? 1 : h->n_ctas, &sc);
+        // b = 64 gains little per stacked block (its MMAs, not the operand traffic, bound it), so
+        // its row groups are used only when they make at least one tile per CTA
+        const int64_t n_tt_groups = (N + 128 * kStackGroups - 1) / (128 * kStackGroups);
+        const bool use_groups = st.ng > 0 && (f.b <= 32 || st.ng * n_tt_groups >= h->n_ctas);
+        if (!use_groups) {
+            rc = build_bcsr_schedule(f, n_tt, static_cast<int>(sw), h->dynamic ? 1 : h->n_ctas, &sc);
+        } else {
+            // The row groups get a launch and a schedule of their own; the launch of the remaining
+            // block-rows starts on the SMs the first one leaves idle, CTA after CTA as they free up.
+            // CTAs are dispatched in index order, so CTA j of the second launch starts when the
+            // j-th lightest CTA of the first one is done: its list is dealt with that head start.
+            const int bnt_s = 128 * kStackGroups;
+            const int n_tt_s = static_cast<int>((N + bnt_s - 1) / bnt_s);
+            int64_t sws = slab_cols / bnt_s;
+            if (sws < 1) sws = 1;
+            if (sws > n_tt_s) sws = n_tt_s;
+            std::vector<int32_t> units, lens;
+            for (int64_t g = 0; g < st.ng; ++g) {
+                units.push_back(static_cast<int32_t>(g));
+                lens.push_back(st.ptr[g + 1] - st.ptr[g]);
+            }
+            std::vector<int64_t> loads;
+            rc = build_tile_schedule(units, lens, kStackTileFixedCost, n_tt_s, static_cast<int>(sws), h->n_ctas, &ss,
+                                     bcsr_stack_block_cost(), nullptr, &loads);
+            ss.groups = kStackGroups;
+            ss.N = N;
+            if (!rc) {
+                std::sort(loads.begin(), loads.end());
+                units.clear();
+                lens.clear();
+                for (int64_t r = 0; r < f.nbr; ++r) {
+                    const int32_t I = f.row_order[r];
+                    if (st.stacked[I]) continue;
+                    units.push_back(I);
+                    lens.push_back(f.block_row_ptr[I + 1] - f.block_row_ptr[I]);
+                }
+                rc = build_tile_schedule(units, lens, kTileFixedCost, n_tt, static_cast<int>(sw), h->n_ctas, &sc,
+                                         bcsr_block_cost(f.b, groups), &loads);
+            }
+        }
     } catch (const std::bad_alloc&) {
         rc = SPMM_ERR_ALLOC;
     }
@@ -561,7 +660,9 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
             cudaFree(h->d_tiles);
             cudaFree(h->d_tile_recs);
             cudaFree(h->d_cta_ptr);
-            h->d_tiles = h->d_tile_recs = h->d_cta_ptr = nullptr;
+            cudaFree(h->d_stile_recs);
+            cudaFree(h->d_scta_ptr);
+            h->d_tiles = h->d_tile_recs = h->d_cta_ptr = h->d_stile_recs = h->d_scta_ptr = nullptr;
         }
         rc = upload(&h->d_tiles, sc.tiles.data(), sc.tiles.size() * 4);
         if (!rc) {
@@ -578,8 +679,22 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
             rc = upload(&h->d_tile_recs, recs.data(), recs.size() * 4);
         }
         if (!rc) rc = upload(&h->d_cta_ptr, sc.cta_ptr.data(), sc.cta_ptr.size() * 4);
+        if (!rc && !ss.tiles.empty()) {
+            const size_t nt = ss.tiles.size() / 2;
+            std::vector<int32_t> recs(4 * nt);
+            for (size_t i = 0; i < nt; ++i) {
+                const int32_t g = ss.tiles[2 * i];
+                recs[4 * i] = g;
+                recs[4 * i + 1] = ss.tiles[2 * i + 1];
+                recs[4 * i + 2] = st.ptr[g];
+                recs[4 * i + 3] = st.ptr[g + 1];
+            }
+            rc = upload(&h->d_stile_recs, recs.data(), recs.size() * 4);
+            if (!rc) rc = upload(&h->d_scta_ptr, ss.cta_ptr.data(), ss.cta_ptr.size() * 4);
+        }
         if (rc) return rc;
     }
+    h->sched_stack = std::move(ss);
     h->sched = std::move(sc);
     return SPMM_OK;
 }
@@ -601,6 +716,8 @@ int run_bcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t s
     p.status = h->d_status;
     p.wait_limit_ns = g_wait_limit_ns.load();
     p.trace = nullptr;
+    p.stack_rows = nullptr;
+    p.overlap = 0;
 #ifdef SPMM_TRACE
     p.trace = g_trace;
 #endif
@@ -615,6 +732,21 @@ int run_bcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t s
     p.use_3d = h->tmB3_ok ? 1 : 0;
     rc = ensure_tmC(h, C, N);
     if (rc) return rc;
+    if (!h->sched_stack.tiles.empty()) {
+        // the row groups first (the longest block-rows are among them), then everything else
+        BcsrParams ps = p;
+        ps.block_col_idx = h->d_sidx;
+        ps.tiles = reinterpret_cast<const int4*>(h->d_stile_recs);
+        ps.cta_ptr = h->d_scta_ptr;
+        ps.stack_rows = h->d_srows;
+        ps.use_3d = h->tmB3s_ok ? 1 : 0;
+        ps.overlap = 1;
+        p.overlap = 2;
+        cudaError_t es = launch_bcsr_stacked(h->dtype, f.b, h->c16, h->col_major, h->tmAs, h->tmB, h->tmB3s, h->tmC, ps,
+                                             h->n_ctas, stream);
+        if (es != cudaSuccess) return SPMM_ERR_CUDA;
+        if (h->sched.tiles.empty()) return SPMM_OK;
+    }
     // dynamic: one CTA per tile, the schedule was built as a single list in the global order
     const int grid = h->dynamic ? static_cast<int>(h->sched.tiles.size() / 2) : h->n_ctas;
     if (grid <= 0) return SPMM_OK;
@@ -866,6 +998,8 @@ int spmm_get_info(spmm_handle_t h, int64_t N, spmm_info_t* info) {
         info->bytes_a = static_cast<double>(info->stored_values) * s;
         info->bytes_idx = static_cast<double>(f.nbr + 1 + f.nnzb) * 4.0;
         info->bytes_gather = static_cast<double>(f.nnzb) * f.b * n * s;
+        info->n_stacked_rows = static_cast<int32_t>(h->stack.rows.size());
+        info->n_stack_blocks = h->stack.ns;
         if (h->sched.N >= 0) {
             info->plan_n = h->sched.N;
             info->plan_token_tile = 128 * h->sched.groups;
@@ -903,6 +1037,7 @@ int spmm_export(spmm_handle_t h, int which, void* host_dst, size_t cap, size_t* 
     const void* host_src = nullptr;   // host array in canonical layout
     size_t bytes = 0;
     bool unpack_wcsr = false;
+    bool host_copy = false;           // the array is kept on the host even when the handle is on the device
     std::vector<int32_t> tmp;
     if (h->format == 0) {
         const BcsrHost& f = h->bcsr;
@@ -917,6 +1052,16 @@ int spmm_export(spmm_handle_t h, int which, void* host_dst, size_t cap, size_t* 
             case SPMM_X_BCSR_TILES:
                 if (h->sched.N < 0) return SPMM_ERR_INVALID_ARG;
                 bytes = h->sched.tiles.size() * 4; dev_src = h->d_tiles; host_src = h->sched.tiles.data(); break;
+            // the row-group plan lives on the host in every mode
+            case SPMM_X_BCSR_STACK_ROWS: bytes = h->stack.rows.size() * 4; host_src = h->stack.rows.data(); host_copy = true; break;
+            case SPMM_X_BCSR_STACK_PTR: bytes = h->stack.ptr.size() * 4; host_src = h->stack.ptr.data(); host_copy = true; break;
+            case SPMM_X_BCSR_STACK_COL_IDX: bytes = h->stack.col_idx.size() * 4; host_src = h->stack.col_idx.data(); host_copy = true; break;
+            case SPMM_X_BCSR_STACK_TILE_PTR:
+                if (h->sched.N < 0) return SPMM_ERR_INVALID_ARG;
+                bytes = h->sched_stack.cta_ptr.size() * 4; host_src = h->sched_stack.cta_ptr.data(); host_copy = true; break;
+            case SPMM_X_BCSR_STACK_TILES:
+                if (h->sched.N < 0) return SPMM_ERR_INVALID_ARG;
+                bytes = h->sched_stack.tiles.size() * 4; host_src = h->sched_stack.tiles.data(); host_copy = true; break;
             default: return SPMM_ERR_INVALID_ARG;
         }
     } else {
@@ -973,7 +1118,7 @@ int spmm_export(spmm_handle_t h, int which, void* host_dst, size_t cap, size_t* 
         }
         return SPMM_OK;
     }
-    if (h->host_only) {
+    if (h->host_only || host_copy) {
         std::memcpy(host_dst, host_src, bytes);
         return SPMM_OK;
     }

@@ -47,7 +47,9 @@ template <int B, int CT, int CM>
 struct EpiCols { static constexpr int value = bcsr_epi_cols(B, CT != 0, CM != 0); };
 
 // ES = bytes per input element: 2 (fp16 / bf16), or 1 (E4M3, column-major operands only).
-template <int B, int GROUPS, int STAGES, int ES>
+// H = rows of one stored block = the MMA's N extent: B for the format's own b x b blocks, 128 for
+// the stacked blocks of a row group (128 / b block-rows on top of one another, see format.h).
+template <int B, int H, int GROUPS, int STAGES, int ES>
 struct BcsrCfg {
     static constexpr int kBB = B * ES;                       // bytes of one block row (its K extent)
     static constexpr int kKSteps = kBB / 32;                 // MMAs per block and token group (32 bytes of K each)
@@ -55,7 +57,7 @@ struct BcsrCfg {
     static constexpr int kNBox = 2 * GROUPS;                 // 64-token boxes per block (row-major B)
     static constexpr int kBoxBytes = B * 128;                // b k-rows x 128 B (row-major B, 2-byte elements)
     static constexpr int kDenseBytes = kBnT * kBB;           // B tile of one block
-    static constexpr int kABytes = B * kBB;
+    static constexpr int kABytes = H * kBB;
     // Small blocks carry too little work for the fixed cost of a pipeline stage (barrier
     // round trip, request issue, MMA hand-off): a stage holds several consecutive stored
     // blocks of the block-row, their B tiles first, then their A blocks (one request).
@@ -67,7 +69,7 @@ struct BcsrCfg {
     // column-major operands: a token group's tile is 128 rows x kXRowBytes, K-major
     static constexpr int kXRowBytes = kARowBytes;
     static constexpr int kXGroupBytes = 128 * kXRowBytes;    // one K half of one token group
-    static constexpr int kAccCols = GROUPS * B;
+    static constexpr int kAccCols = GROUPS * H;
     static constexpr int kTmemCols = (2 * kAccCols <= 32) ? 32 : (2 * kAccCols <= 64 ? 64 : (2 * kAccCols <= 128 ? 128 : (2 * kAccCols <= 256 ? 256 : 512)));
     static constexpr int kStagingBytes = 4 * 2048;           // one 2 KB tile per epilogue warp
     static constexpr int kBarrierBytes = 512;                // mbarriers, TMEM slot, flags, tile-index ring
@@ -77,17 +79,19 @@ struct BcsrCfg {
     static_assert((2 * STAGES + 7 + 8) * 8 + 64 <= kBarrierBytes, "barrier area");
     static_assert(kBps == 1 || B <= 32, "multi-block stages are for the small block sizes");
     static_assert(kBB % 32 == 0, "a block row must hold whole K steps");
+    static_assert(H == B || (H == 128 && B < 128 && ES == 2), "stacked blocks: 128 rows of a 16-bit type");
 };
 
 constexpr int kSchedDepth = 4;      // tile indices fetched ahead by the dynamic scheduler
 
-template <int B, int GROUPS, int STAGES, int FMT, int CT, int CM, int DYN>
+template <int B, int H, int GROUPS, int STAGES, int FMT, int CT, int CM, int DYN>
 __global__ void __launch_bounds__(DYN ? 224 : 192, 1)
 bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ CUtensorMap tmC, const BcsrParams p) {
     constexpr int ES = FMT == 3 ? 1 : 2;
     static_assert(ES == 2 || CM, "8-bit inputs: column-major operands only");
-    using Cfg = BcsrCfg<B, GROUPS, STAGES, ES>;
+    static_assert(H == B || !DYN, "stacked blocks: static schedule only");
+    using Cfg = BcsrCfg<B, H, GROUPS, STAGES, ES>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -132,6 +136,9 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // the row groups' launch: the launch of the remaining block-rows may begin on the SMs this
+    // grid leaves idle (the two write disjoint rows of C)
+    if (p.overlap == 1) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     const int64_t N = p.N;
     // Static schedule: this CTA's range of the tile list.  Dynamic: tile blockIdx.x, then the
@@ -222,7 +229,8 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         // the A request always brings kBps blocks (the box of the tensor map)
                         const uint32_t dense_tx = CM ? (whole_tile ? Cfg::kDenseBytes : ((nvalid + 127) >> 7) * (128 * Cfg::kBB))
                                                      : nbox * Cfg::kBoxBytes;
-                        if (lane == 0) mbar_arrive_expect_tx(full_bar(s), Cfg::kBps * Cfg::kABytes + nb * dense_tx);
+                        // (stacked blocks: one request per block, a box holds at most 256 rows)
+                        if (lane == 0) mbar_arrive_expect_tx(full_bar(s), (H == B ? Cfg::kBps : nb) * Cfg::kABytes + nb * dense_tx);
                         __syncwarp();
                         if constexpr (CM) {
                             // X as [N / 128][128][k]: box = GROUPS x 128 tokens x min(b, 64) elements
@@ -256,10 +264,15 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                                      n0 + lane * 64, J * B, keep);
                             }
                         }
-                        if (lane == 8) {
-                            tma_load_2d_hint(sb + Cfg::kAOff, &tmA, full_bar(s), 0, q * B, keep);
-                        } else if (Cfg::kBB > 128 && lane == 9) {
-                            tma_load_2d_hint(sb + Cfg::kAOff + B * 128, &tmA, full_bar(s), 128 / ES, q * B, keep);
+                        if constexpr (H == B) {
+                            if (lane == 8) {
+                                tma_load_2d_hint(sb + Cfg::kAOff, &tmA, full_bar(s), 0, q * B, keep);
+                            } else if (Cfg::kBB > 128 && lane == 9) {
+                                tma_load_2d_hint(sb + Cfg::kAOff + B * 128, &tmA, full_bar(s), 128 / ES, q * B, keep);
+                            }
+                        } else {
+                            if (lane >= 8 && lane < 8 + nb)
+                                tma_load_2d_hint(sb + Cfg::kAOff + (lane - 8) * Cfg::kABytes, &tmA, full_bar(s), 0, (q + lane - 8) * H, keep);
                         }
                     }
                 }
@@ -285,7 +298,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // elected lane issues the tcgen05 instructions.
         {
             // 8-bit floats: format code 0 = E4M3 in both operand fields
-            constexpr uint32_t idesc = make_idesc(FMT == 3 ? 0 : FMT, 128, B, CM ? 0 : 1, 0);
+            constexpr uint32_t idesc = make_idesc(FMT == 3 ? 0 : FMT, 128, H, CM ? 0 : 1, 0);
             const uint64_t adesc0 = CM ? make_smem_desc(0, 16, 8 * Cfg::kXRowBytes, Cfg::kASwizzle)
                                        : make_smem_desc(0, Cfg::kBoxBytes, 1024, SWZ_128B);
             const uint64_t bdesc0 = make_smem_desc(0, 16, 8 * Cfg::kARowBytes, Cfg::kASwizzle);
@@ -333,7 +346,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                                 for (int g = 0; g < GROUPS; ++g)
                                     if (leader && g < ngrp)
-                                        umma_kind<FMT == 3 ? 2 : 0>(d0 + g * B,
+                                        umma_kind<FMT == 3 ? 2 : 0>(d0 + g * H,
                                                        a0 + ((CM ? (Cfg::kBB <= 128 ? g * Cfg::kXGroupBytes + ks * 32
                                                                             : (ks >> 2) * (GROUPS * Cfg::kXGroupBytes) + g * Cfg::kXGroupBytes + (ks & 3) * 32)
                                                                  : g * 2 * Cfg::kBoxBytes + ks * 2048) >> 4),
@@ -374,6 +387,9 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const int acc = tile_i & 1;
             const uint32_t aph = (tile_i >> 1) & 1u;
             const bool has_blocks = tcd.w > tcd.z;
+            // stacked blocks: the block-rows the group's 128 accumulator columns belong to
+            int member = 0;
+            if constexpr (H != B) member = lane < H / B ? __ldg(p.stack_rows + tI * (H / B) + lane) : 0;
             TRACE_T0(tr_a);
             if (!__all_sync(0xffffffffu, mbar_wait(accf_bar(acc), aph, ctl, 4))) { ok = false; break; }
             TRACE_ADD(tr_accf, tr_a);
@@ -386,11 +402,11 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int nw = n0 + g * 128 + qd * 32;          // first token of this warp
                 if (nw >= N) break;                             // the whole warp is beyond the last token
 #pragma unroll
-                for (int c0 = 0; c0 < B; c0 += W) {
+                for (int c0 = 0; c0 < H; c0 += W) {
                     uint32_t v[W];
                     if (has_blocks) {
                         const uint32_t ta = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) +
-                                            acc * Cfg::kAccCols + g * B + c0;
+                                            acc * Cfg::kAccCols + g * H + c0;
                         if constexpr (W == 16) tmem_ld_x16(ta, v);
                         else tmem_ld_x32(ta, v);
                         tmem_ld_wait();
@@ -442,11 +458,13 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         }
                         fence_proxy_async_smem();
                         __syncwarp();
+                        int32_t crow = static_cast<int32_t>(row0) + c0;
+                        if constexpr (H != B) crow = __shfl_sync(0xffffffffu, member, c0 / B) * B + (c0 % B);
                         if (lane == 0) {
                             // row-major: box = 32 tokens x W rows at (token, row); column-major: box =
                             // W columns x 32 tokens at (column, token).  Out-of-range parts are clipped.
-                            if constexpr (!CM) tma_store_2d(&tmC, stg, nw, static_cast<int32_t>(row0) + c0);
-                            else tma_store_2d(&tmC, stg, static_cast<int32_t>(row0) + c0, nw);
+                            if constexpr (!CM) tma_store_2d(&tmC, stg, nw, crow);
+                            else tma_store_2d(&tmC, stg, crow, nw);
                             bulk_commit_group();
                         }
                     }
@@ -493,6 +511,8 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     tc_fence_before_sync();
     __syncthreads();
+    // launched while the previous grid of the stream was still running: do not finish before it
+    if (p.overlap == 2) asm volatile("griddepcontrol.wait;" ::: "memory");
     if (warp == 1) {
         if (*abort_flag) {
             // abort path: let the MMAs this warp's elected lane already issued finish before
@@ -510,16 +530,29 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
 }
 
-template <int B, int GROUPS, int STAGES, int FMT, int CT, int CM, int DYN>
+template <int B, int H, int GROUPS, int STAGES, int FMT, int CT, int CM, int DYN>
 cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p,
                        int grid, cudaStream_t stream) {
-    using Cfg = BcsrCfg<B, GROUPS, STAGES, FMT == 3 ? 1 : 2>;
-    auto kfn = bcsr_spmm_kernel<B, GROUPS, STAGES, FMT, CT, CM, DYN>;
+    using Cfg = BcsrCfg<B, H, GROUPS, STAGES, FMT == 3 ? 1 : 2>;
+    auto kfn = bcsr_spmm_kernel<B, H, GROUPS, STAGES, FMT, CT, CM, DYN>;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
         if (e != cudaSuccess) return e;
         attr_done = true;
+    }
+    if (p.overlap == 2) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(grid));
+        cfg.blockDim = dim3(DYN ? 224 : 192);
+        cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, kfn, tmA, tmB, tmB3, tmC, p);
     }
     kfn<<<grid, DYN ? 224 : 192, Cfg::kSmemBytes, stream>>>(tmA, tmB, tmB3, tmC, p);
     return cudaGetLastError();
@@ -529,19 +562,40 @@ template <int FMT, int CT, int CM, int DYN>
 cudaError_t launch_shape(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
                          const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
     switch (b * 10 + groups) {
-        case 161: return launch_one<16, 1, 10, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 162: return launch_one<16, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 164: return launch_one<16, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 321: return launch_one<32, 1, 10, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 322: return launch_one<32, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 324: return launch_one<32, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 641: return launch_one<64, 1, 8, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 642: return launch_one<64, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 644: return launch_one<64, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 1281: return launch_one<128, 1, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 1282: return launch_one<128, 2, 2, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 161: return launch_one<16, 16, 1, 10, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 162: return launch_one<16, 16, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 164: return launch_one<16, 16, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 321: return launch_one<32, 32, 1, 10, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 322: return launch_one<32, 32, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 324: return launch_one<32, 32, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 641: return launch_one<64, 64, 1, 8, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 642: return launch_one<64, 64, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 644: return launch_one<64, 64, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 1281: return launch_one<128, 128, 1, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 1282: return launch_one<128, 128, 2, 2, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
         default: return cudaErrorInvalidValue;
     }
+}
+
+// Stacked blocks (row groups): 128 rows x b, token tile 256, four stages of 48 KB.
+template <int FMT, int CT, int CM>
+cudaError_t launch_stack_shape(int b, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
+                               const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
+    switch (b) {
+        case 16: return launch_one<16, 128, 2, 4, FMT, CT, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 32: return launch_one<32, 128, 2, 4, FMT, CT, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 64: return launch_one<64, 128, 2, 4, FMT, CT, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+template <int FMT>
+cudaError_t launch_stack_fmt(int b, int c16, int cm, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
+                             const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
+    if (cm) return c16 ? launch_stack_shape<FMT, 1, 1>(b, tmA, tmB, tmB3, tmC, p, grid, stream)
+                       : launch_stack_shape<FMT, 0, 1>(b, tmA, tmB, tmB3, tmC, p, grid, stream);
+    return c16 ? launch_stack_shape<FMT, 1, 0>(b, tmA, tmB, tmB3, tmC, p, grid, stream)
+               : launch_stack_shape<FMT, 0, 0>(b, tmA, tmB, tmB3, tmC, p, grid, stream);
 }
 
 // E4M3 inputs: column-major operands, fp32 C, static schedule; b = 32, 64 or 128 (a block row
@@ -549,14 +603,14 @@ cudaError_t launch_shape(int b, int groups, const CUtensorMap& tmA, const CUtens
 cudaError_t launch_fp8(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
                        const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
     switch (b * 10 + groups) {
-        case 321: return launch_one<32, 1, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 322: return launch_one<32, 2, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 324: return launch_one<32, 4, 6, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 641: return launch_one<64, 1, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 642: return launch_one<64, 2, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 644: return launch_one<64, 4, 5, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 1281: return launch_one<128, 1, 6, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 1282: return launch_one<128, 2, 4, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 321: return launch_one<32, 32, 1, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 322: return launch_one<32, 32, 2, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 324: return launch_one<32, 32, 4, 6, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 641: return launch_one<64, 64, 1, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 642: return launch_one<64, 64, 2, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 644: return launch_one<64, 64, 4, 5, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 1281: return launch_one<128, 128, 1, 6, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 1282: return launch_one<128, 128, 2, 4, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -583,6 +637,14 @@ cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, in
     if (dtype == 0) return launch_fmt<1>(b, groups, c16, col_major, dynamic, tmA, tmB, tmB3, tmC, p, grid, stream);   // bf16
     if (dtype == 3) return (c16 || !col_major || dynamic) ? cudaErrorInvalidValue
                                                            : launch_fp8(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_bcsr_stacked(int dtype, int b, int c16, int col_major, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                                const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p, int grid,
+                                cudaStream_t stream) {
+    if (dtype == 1) return launch_stack_fmt<0>(b, c16, col_major, tmA, tmB, tmB3, tmC, p, grid, stream);   // fp16
+    if (dtype == 0) return launch_stack_fmt<1>(b, c16, col_major, tmA, tmB, tmB3, tmC, p, grid, stream);   // bf16
     return cudaErrorInvalidValue;
 }
 

@@ -115,25 +115,29 @@ int build_bcsr(const CsrView& a, int b, BcsrHost* out) {
     return SPMM_OK;
 }
 
-int build_bcsr_schedule(const BcsrHost& f, int n_tt, int slab_w, int n_ctas, BcsrSchedule* out) {
-    if (n_tt <= 0 || slab_w <= 0 || n_ctas <= 0) return SPMM_ERR_INVALID_ARG;
+int build_tile_schedule(const std::vector<int32_t>& units, const std::vector<int32_t>& lens, int fixed_cost, int n_tt,
+                        int slab_w, int n_ctas, BcsrSchedule* out, int64_t unit_cost, const std::vector<int64_t>* initial,
+                        std::vector<int64_t>* final_loads) {
+    if (n_tt <= 0 || slab_w <= 0 || n_ctas <= 0 || units.size() != lens.size()) return SPMM_ERR_INVALID_ARG;
+    if (initial && initial->size() != static_cast<size_t>(n_ctas)) return SPMM_ERR_INVALID_ARG;
     out->n_tt = n_tt;
     out->slab_w = slab_w;
     out->n_ctas = n_ctas;
-    const int64_t ntiles = f.nbr * n_tt;
+    const int64_t nu = static_cast<int64_t>(units.size());
+    const int64_t ntiles = nu * n_tt;
     if (ntiles >= (int64_t{1} << 30)) return SPMM_ERR_TOO_LARGE;
     using Load = std::pair<int64_t, int32_t>;   // (load, CTA): smallest load, then lowest CTA, on top
     std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
-    for (int32_t c = 0; c < n_ctas; ++c) heap.push(Load(0, c));
+    for (int32_t c = 0; c < n_ctas; ++c) heap.push(Load(initial ? (*initial)[c] : 0, c));
     std::vector<int32_t> owner(static_cast<size_t>(ntiles));
     std::vector<int32_t> seq_I(static_cast<size_t>(ntiles)), seq_t(static_cast<size_t>(ntiles));
     std::vector<int32_t> count(static_cast<size_t>(n_ctas), 0);
     int64_t n = 0;
     for (int t0 = 0; t0 < n_tt; t0 += slab_w) {
         const int t1 = std::min(n_tt, t0 + slab_w);
-        for (int64_t r = 0; r < f.nbr; ++r) {
-            const int32_t I = f.row_order[r];
-            const int64_t cost = (f.block_row_ptr[I + 1] - f.block_row_ptr[I]) + kTileFixedCost;
+        for (int64_t r = 0; r < nu; ++r) {
+            const int32_t I = units[r];
+            const int64_t cost = (lens[r] + fixed_cost) * unit_cost;
             for (int t = t0; t < t1; ++t, ++n) {
                 Load top = heap.top();
                 heap.pop();
@@ -154,6 +158,79 @@ int build_bcsr_schedule(const BcsrHost& f, int n_tt, int slab_w, int n_ctas, Bcs
         const int32_t dst = pos[owner[i]]++;
         out->tiles[2 * dst] = seq_I[i];
         out->tiles[2 * dst + 1] = seq_t[i];
+    }
+    if (final_loads) {
+        final_loads->assign(static_cast<size_t>(n_ctas), 0);
+        while (!heap.empty()) {
+            (*final_loads)[heap.top().second] = heap.top().first;
+            heap.pop();
+        }
+    }
+    return SPMM_OK;
+}
+
+int build_bcsr_schedule(const BcsrHost& f, int n_tt, int slab_w, int n_ctas, BcsrSchedule* out) {
+    std::vector<int32_t> lens(static_cast<size_t>(f.nbr));
+    for (int64_t r = 0; r < f.nbr; ++r) {
+        const int32_t I = f.row_order[r];
+        lens[r] = f.block_row_ptr[I + 1] - f.block_row_ptr[I];
+    }
+    return build_tile_schedule(f.row_order, lens, kTileFixedCost, n_tt, slab_w, n_ctas, out);
+}
+
+int build_bcsr_stack(const BcsrHost& f, int min_fill_pct, BcsrStack* out) {
+    *out = BcsrStack();
+    out->stacked.assign(static_cast<size_t>(f.nbr), 0);
+    if (f.b >= 128 || min_fill_pct < 0) return SPMM_OK;
+    const int R = 128 / f.b;
+    out->R = R;
+    out->min_fill_pct = min_fill_pct > 0 ? min_fill_pct : bcsr_stack_default_fill(f.b);
+    out->ptr.push_back(0);
+    std::vector<int32_t> cursor(static_cast<size_t>(R));
+    for (int64_t r0 = 0; r0 + R <= f.nbr; r0 += R) {
+        // the candidate's rows; row_order lists empty block-rows last, so the walk can stop there
+        const int32_t* rows = f.row_order.data() + r0;
+        const int32_t last = rows[R - 1];
+        if (f.block_row_ptr[last + 1] == f.block_row_ptr[last]) break;
+        int64_t stored = 0;
+        for (int i = 0; i < R; ++i) {
+            cursor[i] = f.block_row_ptr[rows[i]];
+            stored += f.block_row_ptr[rows[i] + 1] - f.block_row_ptr[rows[i]];
+        }
+        // merge of the R ascending column lists
+        const size_t col0 = out->col_idx.size();
+        for (;;) {
+            int32_t J = INT32_MAX;
+            for (int i = 0; i < R; ++i)
+                if (cursor[i] < f.block_row_ptr[rows[i] + 1]) J = std::min(J, f.block_col_idx[cursor[i]]);
+            if (J == INT32_MAX) break;
+            out->col_idx.push_back(J);
+            for (int i = 0; i < R; ++i) {
+                if (cursor[i] < f.block_row_ptr[rows[i] + 1] && f.block_col_idx[cursor[i]] == J) out->src.push_back(cursor[i]++);
+                else out->src.push_back(-1);
+            }
+        }
+        const int64_t U = static_cast<int64_t>(out->col_idx.size() - col0);
+        if (100 * stored >= static_cast<int64_t>(out->min_fill_pct) * R * U) {
+            for (int i = 0; i < R; ++i) {
+                out->rows.push_back(rows[i]);
+                out->stacked[rows[i]] = 1;
+            }
+            out->ptr.push_back(static_cast<int32_t>(out->col_idx.size()));
+        } else {
+            out->col_idx.resize(col0);
+            out->src.resize(col0 * R);
+        }
+    }
+    out->ng = static_cast<int64_t>(out->ptr.size()) - 1;
+    out->ns = static_cast<int64_t>(out->col_idx.size());
+    if (out->ns * 128 >= (int64_t{1} << 31)) {     // row coordinate of the stacked values' tensor map
+        const int keepR = out->R, keepF = out->min_fill_pct;
+        *out = BcsrStack();
+        out->R = keepR;
+        out->min_fill_pct = keepF;
+        out->stacked.assign(static_cast<size_t>(f.nbr), 0);
+        out->ptr.push_back(0);
     }
     return SPMM_OK;
 }

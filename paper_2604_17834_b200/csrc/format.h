@@ -34,6 +34,31 @@ struct BcsrHost {
     std::vector<int32_t> row_order;       // [nbr] block-rows, most stored blocks first (stable)
 };
 
+// Row stacking (device-private; no counterpart in the paper, whose blocks are all b x b).  A
+// stored block costs the kernel one b-row slice of the token tile however few rows of A it has,
+// so with small blocks the operand traffic into shared memory, not the arithmetic, bounds it.
+// Where R = 128 / b block-rows store blocks in mostly the same block columns, they are computed
+// as one "row group": for every block column of the union one stacked block of 128 rows x b
+// (absent sub-blocks zero), so that the slice of the token tile is fetched once for all R rows
+// and one MMA with N = 128 replaces R MMAs with N = b.
+// Rule (a pure function of the index arrays): walk row_order (most stored blocks first); every
+// run of R consecutive non-empty block-rows in that order is a candidate, accepted when
+// 100 * (stored blocks of the R rows) >= min_fill_pct * R * (block columns in their union).
+struct BcsrStack {
+    int R = 0;                          // block-rows per group; 0: no stacking for this handle
+    int min_fill_pct = 0;
+    int64_t ng = 0, ns = 0;             // row groups, stacked blocks
+    std::vector<int32_t> rows;          // [ng][R] member block-rows, in row_order order
+    std::vector<int32_t> ptr;           // [ng+1] ranges of stacked blocks
+    std::vector<int32_t> col_idx;       // [ns] block columns of the union, ascending inside a group
+    std::vector<int32_t> src;           // [ns][R] stored block behind each sub-block, or -1
+    std::vector<uint8_t> stacked;       // [nbr] 1: the block-row belongs to a group
+};
+// default acceptance threshold per block size, from the bytes a stacked and an unstacked block
+// bring into shared memory per unit of work (and measured on the Bernoulli sweep)
+constexpr int bcsr_stack_default_fill(int b) { return b == 16 ? 30 : (b == 32 ? 45 : 75); }
+int build_bcsr_stack(const BcsrHost& f, int min_fill_pct, BcsrStack* out);
+
 // Static tile schedule of the BCSR kernel for one dense width: a tile is (block-row, token
 // tile).  Tiles are taken slab by slab (a slab = slab_w consecutive token tiles, sized so the
 // B rows it touches stay in L2) and, inside a slab, block-rows with the most stored blocks
@@ -97,7 +122,24 @@ void finish_bcsr_host(BcsrHost* out);
 int build_bcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int32_t* d_col_idx, const uint8_t* d_vals,
                       int es, int b, cudaStream_t stream, BcsrHost* out, int64_t* nnz_out, int32_t** d_block_row_ptr,
                       int32_t** d_block_col_idx, uint8_t** d_blocks);
+// Allocates and fills the stacked values [ns][128][b] on the device from the stored blocks and
+// st.src (format_gpu.cu); *d_stacked is owned by the caller afterwards.  Synchronises the device.
+int stack_bcsr_device(const uint8_t* d_blocks, const BcsrStack& st, int b, int es, uint8_t** d_stacked);
 int build_bcsr_schedule(const BcsrHost& f, int n_tt, int slab_w, int n_ctas, BcsrSchedule* out);
+// The same rule over any list of units (block-rows or row groups) given in schedule order with
+// their lengths in stored blocks; tiles = {unit, token tile}.
+// A tile's load is (length + fixed_cost) * unit_cost; CTA c starts with load initial[c] (all zero
+// when initial is null); *final_loads (optional) receives the CTAs' loads at the end.
+int build_tile_schedule(const std::vector<int32_t>& units, const std::vector<int32_t>& lens, int fixed_cost, int n_tt,
+                        int slab_w, int n_ctas, BcsrSchedule* out, int64_t unit_cost = 1,
+                        const std::vector<int64_t>* initial = nullptr, std::vector<int64_t>* final_loads = nullptr);
+// Relative cost of one stored block in the two launches of a handle with row groups, in bytes
+// staged per block divided by b: a stacked block brings 256 tokens x b and 128 x b of A, a b x b
+// block 128 * groups tokens x b and b x b of A (both launches are bound by that traffic).
+constexpr int64_t bcsr_stack_block_cost() { return 2 * (256 + 128); }
+constexpr int64_t bcsr_block_cost(int b, int groups) { return 2 * (128 * groups + b); }
+// a row group's tile writes 128 rows of C whatever its length
+constexpr int kStackTileFixedCost = 8;
 // T = 0 picks the sub-task size from the matrix: about a quarter of one bin's share of the
 // padded columns, rounded down to a multiple of 64 and clamped to [128, 4096].
 int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost* out);

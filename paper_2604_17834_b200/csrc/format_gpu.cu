@@ -211,6 +211,44 @@ void finish_bcsr_host(BcsrHost* out) {
         if (out->block_row_ptr[I + 1] == out->block_row_ptr[I]) out->n_empty++;
 }
 
+// One thread per 16-byte piece of the stacked values: sub-block r of stacked block s is stored
+// block src[s][r] (b x b, row-major) or zeros.
+__global__ void bcsr_stack_kernel(const uint4* __restrict__ blocks, const int32_t* __restrict__ src, uint4* __restrict__ out,
+                                  int R, int pieces_per_block, int64_t n_pieces) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n_pieces) return;
+    const int64_t sub = i / pieces_per_block;          // = s * R + r
+    const int piece = static_cast<int>(i % pieces_per_block);
+    const int32_t p = __ldg(src + sub);
+    out[i] = p >= 0 ? __ldg(blocks + static_cast<int64_t>(p) * pieces_per_block + piece) : make_uint4(0u, 0u, 0u, 0u);
+    (void)R;
+}
+
+int stack_bcsr_device(const uint8_t* d_blocks, const BcsrStack& st, int b, int es, uint8_t** d_stacked) {
+    *d_stacked = nullptr;
+    if (st.ns == 0) return SPMM_OK;
+    const int pieces = b * b * es / 16;
+    const int64_t n_pieces = st.ns * st.R * pieces;
+    int32_t* d_src = nullptr;
+    if (cudaMalloc(reinterpret_cast<void**>(&d_src), st.src.size() * 4) != cudaSuccess) return SPMM_ERR_ALLOC;
+    if (cudaMalloc(reinterpret_cast<void**>(d_stacked), static_cast<size_t>(n_pieces) * 16) != cudaSuccess) {
+        cudaFree(d_src);
+        return SPMM_ERR_ALLOC;
+    }
+    int rc = SPMM_OK;
+    if (cudaMemcpy(d_src, st.src.data(), st.src.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) rc = SPMM_ERR_CUDA;
+    if (!rc) {
+        const int threads = 256;
+        const int64_t grid = (n_pieces + threads - 1) / threads;
+        bcsr_stack_kernel<<<static_cast<unsigned>(grid), threads>>>(reinterpret_cast<const uint4*>(d_blocks), d_src,
+                                                                   reinterpret_cast<uint4*>(*d_stacked), st.R, pieces, n_pieces);
+        if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) rc = SPMM_ERR_CUDA;
+    }
+    cudaFree(d_src);
+    if (rc) { cudaFree(*d_stacked); *d_stacked = nullptr; }
+    return rc;
+}
+
 int build_bcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int32_t* d_col_idx, const uint8_t* d_vals,
                       int es, int b, cudaStream_t st, BcsrHost* out, int64_t* nnz_out, int32_t** d_block_row_ptr,
                       int32_t** d_block_col_idx, uint8_t** d_blocks) {

@@ -18,6 +18,14 @@ struct BcsrParams {
     uint64_t wait_limit_ns;
     long long* trace;   // tuning builds only (SPMM_TRACE); nullptr otherwise
     int32_t use_3d;     // tmB3 is valid: whole token tiles are fetched with one 3-D request
+    // stacked launch only: [groups][128 / b] block-rows of every row group (see BcsrStack); the
+    // tile records then name {group, token tile, first stacked block, end stacked block} and
+    // block_col_idx is the stacked blocks' column index
+    const int32_t* stack_rows;
+    // 1: this grid lets the next launch of the stream start while it runs (its first
+    // instruction after set-up is griddepcontrol.launch_dependents); 2: this grid was launched
+    // that way behind another one and waits for it (griddepcontrol.wait) before its CTAs exit
+    int32_t overlap;
 };
 
 // dtype: 0 bf16, 1 fp16.  groups: token tile = 128 * groups columns of B (1, 2 or 4).
@@ -32,6 +40,13 @@ struct BcsrParams {
 cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, int dynamic, const CUtensorMap& tmA,
                         const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p,
                         int grid, cudaStream_t stream);
+// Row groups: the same kernel with 128 x b stacked blocks (MMA N = 128) and a 256-token tile.
+// tmA: the stacked values as [blocks * 128][b], box 128 x b; tmB3 built for groups = 2; b = 16, 32, 64.
+constexpr int kStackRows = 128;
+constexpr int kStackGroups = 2;
+cudaError_t launch_bcsr_stacked(int dtype, int b, int c16, int col_major, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                                const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p, int grid,
+                                cudaStream_t stream);
 int bcsr_token_groups_max(int b);
 // Accumulator columns (= rows of A's block) an epilogue warp handles at a time: it stages them
 // in a 2 KB shared-memory tile and stores the tile with one TMA request whose box is 32 tokens x

@@ -74,6 +74,17 @@ def test_config1_wcsr_irregular_full(lib):
     assert worst < 1.0
 
 
+def test_config1_second_reading_zipf_1_8_full(lib):
+    """configs[1] quotes a mean row length of 12, which Zipf(2) clipped at 5000 cannot give
+    (its mean is near 6); an exponent of 1.8 does.  Same check on that second reading."""
+    a = wl.wcsr_irregular(seed=1012, alpha=1.8)
+    mean_len = float(a["row_ptr"][-1]) / a["m"]
+    assert 10.0 < mean_len < 16.0
+    Bs = wl.dense(1112, a["k"], 128, ("normal", 0.0, 1.0), "tf32")
+    worst = _run_and_check(lib, "wcsr", a, "tf32", 16, 128, Bs, what="configs[1] zipf(1.8)")
+    assert worst < 1.0
+
+
 @pytest.mark.parametrize("shape", ["gate", "down"])
 def test_config2_bcsr_llm_full(lib, shape):
     """configs[2]: 18944 x 3584 (gate) and 3584 x 18944 (down), 64 x 64 blocks, N = 65536."""

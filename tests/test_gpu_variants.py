@@ -317,3 +317,95 @@ def test_variant_argument_errors(lib):
         lib.spmm_run(h, buf.data_ptr(), buf.data_ptr(), 64)                 # fewer than 128 tokens
     assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
     lib.spmm_destroy(h)
+
+
+# --------------------------------------------------------------------------- row groups (stacked 128-row blocks)
+
+
+def _grouped_matrix(seed, m, k, b, dtype):
+    """Block pattern with what the grouping looks for: a band of dense block-rows, block-rows
+    that share most of their columns, sparse ones and empty ones, in scattered positions."""
+    rng = np.random.default_rng(seed)
+    nbr, nbc = -(-m // b), -(-k // b)
+    kind = rng.choice(4, size=nbr, p=[0.3, 0.3, 0.25, 0.15])
+    shared = rng.random(nbc) < 0.5
+    mask = np.zeros((nbr, nbc), dtype=bool)
+    for i in range(nbr):
+        if kind[i] == 0:
+            mask[i] = True
+        elif kind[i] == 1:
+            mask[i] = shared & (rng.random(nbc) < 0.9)
+        elif kind[i] == 2:
+            mask[i] = rng.random(nbc) < 0.08
+    D = np.zeros((nbr * b, nbc * b), dtype=np.float32)
+    for i, j in zip(*np.nonzero(mask)):
+        blk = rng.uniform(-1.0, 1.0, size=(b, b)).astype(np.float32)
+        blk[rng.random((b, b)) < 0.3] = 0.0                           # blocks are not full either
+        D[i * b:(i + 1) * b, j * b:(j + 1) * b] = blk
+    D = D[:m, :k]
+    rows, cols = np.nonzero(D)
+    row_ptr = np.concatenate(([0], np.cumsum(np.bincount(rows, minlength=m)))).astype(np.int64)
+    return dict(m=m, k=k, row_ptr=row_ptr, col_idx=cols.astype(np.int32), vals=wl.to_storage(D[rows, cols], dtype))
+
+
+@pytest.mark.parametrize("b,dtype,m,k,N,c16,cm,fill", [
+    (16, "fp16", 1024, 640, 384, False, False, 0),
+    (16, "bf16", 1000, 520, 328, True, False, 0),        # ragged m, k and N
+    (32, "fp16", 1024, 768, 256, False, True, 0),
+    (32, "bf16", 1096, 512, 200, True, True, 0),         # N below one 256-token tile, Y rows of 1096 elements
+    (64, "fp16", 2048, 512, 1184, False, False, 0),      # (b = 64 groups are used when they make a tile per CTA: 24 CTAs)
+    (64, "bf16", 2048, 512, 1184, True, True, 0),
+    (16, "fp16", 512, 512, 128, False, False, 1),        # forced: groups of sparse rows, mostly absent sub-blocks
+    (32, "fp16", 640, 384, 512, False, False, 1),
+    (64, "fp16", 4096, 256, 608, False, False, 1),
+])
+def test_bcsr_row_groups_match_the_oracle(lib, b, dtype, m, k, N, c16, cm, fill):
+    from oracle import formats as F
+    a = _grouped_matrix(7 * b + N, m, k, b, dtype)
+    Bs = wl.dense(300 + b, k, N, ("uniform", -1.0, 1.0), dtype)
+    Cr, S = reference(a, Bs, dtype)
+    outs = {}
+    for mode in (fill, -1):
+        h = lib.spmm_bcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, b,
+                                     c_type=lib.C_SAME_AS_INPUT if c16 else lib.C_FP32,
+                                     layout=lib.COLMAJOR if cm else lib.ROWMAJOR, stack_min_fill=mode,
+                                     n_ctas=24 if b == 64 else 0)
+        try:
+            info = lib.spmm_get_info(h, N)
+            if mode >= 0:
+                assert info["n_stacked_rows"] >= 128 // b, "the test matrix must produce row groups"
+            else:
+                assert info["n_stacked_rows"] == 0
+            got = run_gpu_variant(lib, h, Bs, m, N, dtype, c16=c16, col_major=cm)
+            assert_close(got, Cr, S, dtype, "b=%d %s groups %s" % (b, dtype, "on" if mode >= 0 else "off"))
+            if mode >= 0:
+                used = lib.spmm_export(h, lib.X_BCSR_STACK_TILES, np.int32).size > 0
+                assert used, "the plan must use the row groups in this case"
+                # the exported format stays the canonical one
+                f = F.bcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], b)
+                assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCK_COL_IDX, np.int32), f["block_col_idx"])
+                again = run_gpu_variant(lib, h, Bs, m, N, dtype, c16=c16, col_major=cm)
+                assert np.array_equal(got, again), "run-to-run difference"
+            outs[mode] = got
+        finally:
+            lib.spmm_destroy(h)
+    # absent sub-blocks add exact zeros: the grouped and the plain launch agree to the last bit
+    assert np.array_equal(outs[fill], outs[-1])
+
+
+def test_bcsr_row_groups_from_the_gpu_builder(lib):
+    """Same handle from a device-resident CSR: the stacked values are built from the blocks the GPU builder wrote."""
+    import torch
+    b, dtype, m, k, N = 16, "fp16", 768, 512, 256
+    a = _grouped_matrix(5, m, k, b, dtype)
+    Bs = wl.dense(77, k, N, ("uniform", -1.0, 1.0), dtype)
+    Cr, S = reference(a, Bs, dtype)
+    rp, ci, v = to_device(a["row_ptr"]), to_device(a["col_idx"]), to_device(a["vals"])
+    h = lib.spmm_bcsr_create_csr_device(m, k, rp.data_ptr(), ci.data_ptr(), v.data_ptr(), dtype, b,
+                                        stream=torch.cuda.current_stream().cuda_stream)
+    try:
+        assert lib.spmm_get_info(h, N)["n_stacked_rows"] > 0
+        got = run_gpu_variant(lib, h, Bs, m, N, dtype)
+        assert_close(got, Cr, S, dtype, "gpu-built, row groups")
+    finally:
+        lib.spmm_destroy(h)

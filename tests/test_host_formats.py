@@ -95,7 +95,7 @@ def test_bcsr_workload_generators_round_trip(lib):
 def test_bcsr_tile_schedule_is_bit_exact_and_balanced(lib, b, N, n_ctas):
     s = wl.bcsr_sweep(55 + b, m=4096, k=2048, b=b, density=0.1)
     h = lib.spmm_bcsr_create_csr(4096, 2048, s["row_ptr"], s["col_idx"], s["vals"], "fp16", b, host_only=True,
-                                 n_ctas=n_ctas)
+                                 n_ctas=n_ctas, stack_min_fill=-1)
     try:
         with pytest.raises(lib.SpmmError):
             lib.spmm_export(h, lib.X_BCSR_TILES, np.int32)          # no plan yet
@@ -119,6 +119,72 @@ def test_bcsr_tile_schedule_is_bit_exact_and_balanced(lib, b, N, n_ctas):
         assert loads.max() - loads.min() <= cost.max()
         if N % 512 == 0 and b != 128 and nbr * (N // 512) >= 8 * n_ctas:
             assert bnt == 512                                        # widest tile that divides N
+    finally:
+        lib.spmm_destroy(h)
+
+
+@pytest.mark.parametrize("b,N,n_ctas,fill", [(16, 4096, 148, 0), (32, 1000, 13, 0), (64, 8192, 8, 0), (16, 512, 5, 1),
+                                             (32, 4096, 148, 100), (64, 256, 148, 0), (128, 512, 4, 0)])
+def test_bcsr_row_groups_and_their_schedules_are_bit_exact(lib, b, N, n_ctas, fill):
+    """Row groups (128 / b block-rows computed from 128-row stacked blocks): the grouping, and the two
+    tile schedules of a handle that has groups, against the definitions in oracle/formats.py."""
+    m, k = 4096, 2048
+    s = wl.bcsr_sweep(91 + b, m=m, k=k, b=b, density=0.3)            # 10 % full block-rows, 20 % empty, rest 0.3
+    h = lib.spmm_bcsr_create_csr(m, k, s["row_ptr"], s["col_idx"], s["vals"], "fp16", b, host_only=True, n_ctas=n_ctas,
+                                 stack_min_fill=fill)
+    try:
+        f = F.bcsr_from_csr(m, k, s["row_ptr"], s["col_idx"], s["vals"], b)
+        brp = f["block_row_ptr"]
+        info = lib.spmm_get_info(h, N)
+        if b == 128:                                                  # blocks already are 128 rows high
+            assert info["n_stacked_rows"] == 0 and lib.spmm_export(h, lib.X_BCSR_STACK_ROWS, np.int32).size == 0
+            return
+        R = 128 // b
+        default = {16: 30, 32: 45, 64: 75}[b]
+        rows, ptr, cols = F.bcsr_row_groups(brp, f["block_col_idx"], b, fill or default)
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_STACK_ROWS, np.int32).reshape(-1, R), rows)
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_STACK_PTR, np.int32), ptr)
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_STACK_COL_IDX, np.int32), cols)
+        assert info["n_stacked_rows"] == rows.size and info["n_stack_blocks"] == cols.size
+        assert rows.shape[0] >= (m // b) // (10 * R)                  # the full block-rows are grouped
+        # the plan: groups first (tiles of 256 tokens), the other block-rows dealt with the head start
+        # the j-th lightest CTA of the first launch leaves to CTA j of the second
+        lib.spmm_bcsr_plan(h, N)
+        info = lib.spmm_get_info(h, N)
+        ng = rows.shape[0]
+        n_tt_g = -(-N // 256)
+        got_gtiles = lib.spmm_export(h, lib.X_BCSR_STACK_TILES, np.int32).reshape(-1, 2)
+        groups_used = b <= 32 or ng * n_tt_g >= n_ctas
+        bnt = info["plan_token_tile"]
+        n_tt = -(-N // bnt)
+        got_ptr = lib.spmm_export(h, lib.X_BCSR_TILE_PTR, np.int32)
+        got_tiles = lib.spmm_export(h, lib.X_BCSR_TILES, np.int32).reshape(-1, 2)
+        if not groups_used:
+            assert got_gtiles.size == 0
+            want_ptr, want_tiles = F.bcsr_tile_schedule(brp, n_tt, info["plan_slab_tiles"], n_ctas)
+            assert np.array_equal(got_ptr, want_ptr) and np.array_equal(got_tiles, want_tiles)
+            return
+        slab_cols = (16 << 20) // (k * 2)
+        slab_g = max(1, min(n_tt_g, slab_cols // 256))
+        gp, gt, loads = F.bcsr_tile_schedule(None, n_tt_g, slab_g, n_ctas, fixed_cost=8, units=np.arange(ng),
+                                             lens=np.diff(ptr), unit_cost=2 * (256 + 128), return_loads=True)
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_STACK_TILE_PTR, np.int32), gp)
+        assert np.array_equal(got_gtiles, gt)
+        order = F.bcsr_row_order(brp)
+        rest = order[~np.isin(order, rows.reshape(-1))]
+        want_ptr, want_tiles = F.bcsr_tile_schedule(None, n_tt, info["plan_slab_tiles"], n_ctas, units=rest,
+                                                    lens=np.diff(brp)[rest], unit_cost=2 * (128 * (bnt // 128) + b),
+                                                    initial=np.sort(loads))
+        assert np.array_equal(got_ptr, want_ptr) and np.array_equal(got_tiles, want_tiles)
+        # together: every (block-row, 128-token group) exactly once
+        n128 = -(-N // 128)
+        seen = np.zeros((m // b, n128), dtype=np.int32)
+        for I, t in got_tiles:
+            seen[I, t * (bnt // 128):min(n128, (t + 1) * (bnt // 128))] += 1
+        for g, t in got_gtiles:
+            for I in rows[g]:
+                seen[I, 2 * t:min(n128, 2 * t + 2)] += 1
+        assert np.all(seen == 1)
     finally:
         lib.spmm_destroy(h)
 

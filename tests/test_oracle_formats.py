@@ -229,3 +229,94 @@ def test_tile_padding_numbers_of_the_paper():
         got_padded, waste = F.padded_width(N, BN)
         assert got_padded == padded
         assert round(100.0 * waste) == pct
+
+
+# --------------------------------------------------------------------------- schedules and row groups
+
+
+def _brute_schedule(units, lens, n_tt, slab_w, n_ctas, fixed, unit_cost, initial):
+    """The longest-first dealing rule with a plain argmin instead of a heap."""
+    loads = [0] * n_ctas if initial is None else [int(x) for x in initial]
+    lists = [[] for _ in range(n_ctas)]
+    for t0 in range(0, n_tt, slab_w):
+        for I, ln in zip(units, lens):
+            for t in range(t0, min(n_tt, t0 + slab_w)):
+                c = min(range(n_ctas), key=lambda j: (loads[j], j))
+                lists[c].append((int(I), t))
+                loads[c] += (int(ln) + fixed) * unit_cost
+    return lists, loads
+
+
+@pytest.mark.parametrize("seed,n_ctas,n_tt,slab_w", [(0, 3, 5, 2), (1, 7, 4, 4), (2, 1, 3, 1), (3, 5, 1, 1)])
+def test_tile_schedule_matches_brute_force(seed, n_ctas, n_tt, slab_w):
+    rng = np.random.default_rng(seed)
+    lens_all = rng.integers(0, 9, size=11)
+    brp = np.concatenate(([0], np.cumsum(lens_all)))
+    order = F.bcsr_row_order(brp)
+    assert np.all(np.diff(lens_all[order]) <= 0)                                   # longest first
+    assert all(order[i] < order[i + 1] for i in range(10) if lens_all[order[i]] == lens_all[order[i + 1]])   # stable
+    ptr, tiles = F.bcsr_tile_schedule(brp, n_tt, slab_w, n_ctas)
+    lists, _ = _brute_schedule(order, lens_all[order], n_tt, slab_w, n_ctas, 4, 1, None)
+    assert [tuple(x) for x in tiles.tolist()] == [p for l in lists for p in l]
+    assert ptr.tolist() == np.concatenate(([0], np.cumsum([len(l) for l in lists]))).tolist()
+    # a subset of the units, weighted costs and a head start per CTA
+    units = order[1::2]
+    initial = rng.integers(0, 400, size=n_ctas)
+    ptr2, tiles2, loads2 = F.bcsr_tile_schedule(None, n_tt, slab_w, n_ctas, fixed_cost=3, units=units, lens=lens_all[units],
+                                                unit_cost=17, initial=initial, return_loads=True)
+    lists2, bl = _brute_schedule(units, lens_all[units], n_tt, slab_w, n_ctas, 3, 17, initial)
+    assert [tuple(x) for x in tiles2.tolist()] == [p for l in lists2 for p in l]
+    assert loads2.tolist() == bl
+    assert loads2.sum() == initial.sum() + 17 * n_tt * int((lens_all[units] + 3).sum())
+
+
+def _brute_groups(rows_cols, R, min_fill_pct):
+    """rows_cols: list of sets of block columns per block-row."""
+    order = sorted(range(len(rows_cols)), key=lambda i: (-len(rows_cols[i]), i))
+    out = []
+    for r0 in range(0, len(order) - R + 1, R):
+        cand = order[r0:r0 + R]
+        if not rows_cols[cand[-1]]:
+            break
+        union = set().union(*[rows_cols[i] for i in cand])
+        stored = sum(len(rows_cols[i]) for i in cand)
+        if 100 * stored >= min_fill_pct * R * len(union):
+            out.append((cand, sorted(union)))
+    return out
+
+
+@pytest.mark.parametrize("b,seed,fill", [(16, 0, 30), (32, 1, 45), (64, 2, 75), (16, 3, 1), (32, 4, 100), (64, 5, 50)])
+def test_row_groups_match_brute_force(b, seed, fill):
+    rng = np.random.default_rng(seed)
+    R = 128 // b
+    nbr, nbc = 4 * R + 3, 12
+    dens = rng.choice([0.0, 0.2, 0.6, 1.0], size=nbr)
+    mask = rng.random((nbr, nbc)) < dens[:, None]
+    brp = np.concatenate(([0], np.cumsum(mask.sum(axis=1)))).astype(np.int32)
+    bci = np.concatenate([np.flatnonzero(mask[i]) for i in range(nbr)]).astype(np.int32)
+    rows, ptr, cols = F.bcsr_row_groups(brp, bci, b, fill)
+    want = _brute_groups([set(np.flatnonzero(mask[i]).tolist()) for i in range(nbr)], R, fill)
+    assert rows.tolist() == [c for c, _ in want]
+    assert ptr.tolist() == np.concatenate(([0], np.cumsum([len(u) for _, u in want]))).astype(int).tolist()
+    assert cols.tolist() == [j for _, u in want for j in u]
+    assert len(set(rows.reshape(-1).tolist())) == rows.size                          # a block-row is in at most one group
+    assert all(mask[i].any() for i in rows.reshape(-1))                              # and never empty
+
+
+def test_row_groups_special_cases():
+    b, R = 32, 4
+    # identical block-rows: the union is every row's own column set, fill 100 %
+    cols = np.array([1, 4, 5, 9], dtype=np.int32)
+    brp = np.arange(0, 4 * 9, 4, dtype=np.int32)                                     # 8 block-rows of 4 blocks
+    bci = np.tile(cols, 8)
+    rows, ptr, gcols = F.bcsr_row_groups(brp, bci, b, 100)
+    assert rows.tolist() == [[0, 1, 2, 3], [4, 5, 6, 7]] and ptr.tolist() == [0, 4, 8] and gcols.tolist() == cols.tolist() * 2
+    # block-diagonal: the union of R rows has R columns for R stored blocks, fill 100 / R %
+    brp = np.arange(9, dtype=np.int32)
+    bci = np.arange(8, dtype=np.int32)
+    assert F.bcsr_row_groups(brp, bci, b, 100 // R)[0].shape[0] == 2
+    assert F.bcsr_row_groups(brp, bci, b, 100 // R + 1)[0].shape[0] == 0
+    # fewer non-empty block-rows than a group needs: nothing to group
+    brp = np.array([0, 3, 3, 3, 6, 6, 6, 6, 6], dtype=np.int32)
+    bci = np.array([0, 1, 2, 0, 1, 2], dtype=np.int32)
+    assert F.bcsr_row_groups(brp, bci, b, 1)[0].shape[0] == 0
