@@ -110,6 +110,13 @@ def workload_table():
             w["size"] = 64
             return w
         return f
+    def plain(base):
+        """Same workload with the BCSR row groups (stacked 128-row blocks) switched off."""
+        def f():
+            w = base()
+            w["opts"] = dict(w.get("opts", {}), stack_min_fill=-1)
+            return w
+        return f
     def fp8_linear(m, k, seed):
         def f():
             return dict(kind="bcsr", a=wl.bcsr_llm(seed=seed, m=m, k=k, dtype="fp8", std=0.5), dtype="fp8", size=64, N=65536,
@@ -131,6 +138,8 @@ def workload_table():
                 "configs[3] BCSR 8192x8192 fp16 b=%d skewed rows, keep %g in the rest, N=4096" % (b, d), cfg4(b, d))
             t["cfg4_bcsr_sweep_b%d_d%g_dyn" % (b, d)] = (
                 "configs[3] b=%d skewed rows, keep %g, dynamic tile scheduling" % (b, d), variant(cfg4(b, d), dyn=True))
+        t["cfg4_bcsr_sweep_b%d_d0.1_plain" % b] = ("configs[3] b=%d skewed rows, keep 0.1, row groups switched off" % b,
+                                                    plain(cfg4(b, 0.1)))
         for d in (0.05, 0.01):
             t["cfg4_bcsr_flat_b%d_d%g" % (b, d)] = (
                 "configs[3] BCSR 8192x8192 fp16 b=%d flat Bernoulli(%g), N=4096" % (b, d), cfg4(b, d, False))
@@ -147,7 +156,7 @@ DEFAULT_OTHERS = ["cfg1_bcsr_tiny", "cfg2_wcsr_irregular_alpha1.8", "cfg3_bcsr_l
                   "cfg3_bcsr_llm_gate_c16", "cfg3_bcsr_llm_gate_cm", "cfg3_bcsr_llm_gate_cm_c16",
                   "cfg3_bcsr_llm_down_cm_c16", "cfg5_wcsr_rmat_n128_c16",
                   "cfg3_bcsr_llm_gate_cm_fp8", "cfg3_bcsr_llm_down_cm_fp8", "cfg2_wcsr_irregular_wh64",
-                  "cfg4_bcsr_sweep_b64_d0.1_dyn"]
+                  "cfg4_bcsr_sweep_b64_d0.1_dyn", "cfg4_bcsr_sweep_b16_d0.1_plain", "cfg4_bcsr_sweep_b32_d0.1_plain"]
 
 L2_TO_SM_GBS = 19800.0      # measured aggregate L2 -> shared-memory TMA rate (148 SMs x 70 B/cycle at 1.9 GHz)
 
@@ -247,7 +256,7 @@ def device_B(torch, w, seed=7):
     return B
 
 
-def roofline_of(info, ms, pk):
+def roofline_of(info, ms, pk, groups=None):
     """Roofline of one spmm_run: slower of tensor time for the stored flops and HBM time for the model bytes."""
     model_bytes = info["bytes_a"] + info["bytes_idx"] + info["bytes_b_touched"] + info["bytes_c"]
     # TF32 = half, 8-bit = twice the measured bf16 rate (nominal ratios)
@@ -274,6 +283,15 @@ def roofline_of(info, ms, pk):
     else:
         a_passes = max(1, -(-int(round(info["flops_stored"] / (2.0 * max(1, info["stored_values"])))) // 128))
     l2_bytes = info["bytes_gather"] + info["bytes_a"] * a_passes
+    if groups and groups["used"]:
+        # row groups: the grouped block-rows stage one slice of the dense operand per stacked block
+        # (not per stored block) and 128 x b of A per 256-token tile
+        es, b, n = 2, info["block"], info["flops_stored"] / (2.0 * max(1, info["stored_values"]))
+        plain = info["n_units"] - groups["grouped_blocks"]
+        l2_bytes = (plain * (b * n * es + b * b * es * a_passes) +
+                    info["n_stack_blocks"] * (b * n * es + 128 * b * es * max(1, -(-int(round(n)) // 256))))
+        r["row_groups"] = {"block_rows": info["n_stacked_rows"], "stored_blocks": groups["grouped_blocks"],
+                           "stacked_blocks": info["n_stack_blocks"]}
     r["l2_to_sm"] = {"bytes": l2_bytes, "rate_gbs": L2_TO_SM_GBS, "achieved_gbs": l2_bytes / t / 1e9,
                      "frac": l2_bytes / t / 1e9 / L2_TO_SM_GBS}
     return r
@@ -328,7 +346,15 @@ def time_workload(torch, lib, w, steps, warmup, flush):
         torch.cuda.synchronize()
         ms_warm = float(np.mean([a.elapsed_time(b) for a, b in wevs]))
         launches = 1 + (1 if (w["kind"] == "wcsr" and (info["n_split"] + info["n_empty"]) > 0) else 0)
-        return dict(h=None, info=info, ms_mean=float(ms.mean()), ms_median=float(np.median(ms)), ms_min=float(ms.min()), ms_warm=ms_warm,
+        groups = None
+        if w["kind"] == "bcsr" and info["n_stacked_rows"] > 0:
+            used = lib.spmm_export(h, lib.X_BCSR_STACK_TILES, np.int32).size > 0
+            rows = lib.spmm_export(h, lib.X_BCSR_STACK_ROWS, np.int32)
+            brp = lib.spmm_export(h, lib.X_BCSR_BLOCK_ROW_PTR, np.int32)
+            groups = {"used": bool(used), "grouped_blocks": int(np.diff(brp)[rows].sum())}
+            if used and lib.spmm_export(h, lib.X_BCSR_TILES, np.int32).size > 0:
+                launches = 2
+        return dict(h=None, info=info, groups=groups, ms_mean=float(ms.mean()), ms_median=float(np.median(ms)), ms_min=float(ms.min()), ms_warm=ms_warm,
                     create_ms=create_ms, launches_per_step=launches, B=B, C=C)
     finally:
         lib.spmm_destroy(h)
@@ -387,7 +413,7 @@ def summarize(name, desc, res, pk, N):
         "ms_warm_l2": res["ms_warm"],
         "gflops_stored": gf, "gflops_useful": 2.0 * info["nnz"] * N / (ms * 1e-3) / 1e9,
         "fill_ratio": info["fill_ratio"], "stored_values": info["stored_values"], "n_units": info["n_units"],
-        "create_ms": res["create_ms"], "roofline": roofline_of(info, ms, pk),
+        "create_ms": res["create_ms"], "roofline": roofline_of(info, ms, pk, res.get("groups")),
     }
 
 
