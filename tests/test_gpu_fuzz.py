@@ -63,6 +63,52 @@ def test_bcsr_random_case(lib, seed):
         lib.spmm_destroy(h)
 
 
+@pytest.mark.parametrize("seed", range(40))
+def test_bcsr_row_groups_random_case(lib, seed):
+    """Row groups forced on (every run of 128 / b non-empty block-rows is stacked, however few of its
+    sub-blocks are stored) or left to the default threshold, over ragged shapes and all output options."""
+    import torch
+    rng = np.random.default_rng(11000 + seed)
+    dtype = ["bf16", "fp16"][int(rng.integers(0, 2))]
+    b = int([16, 32, 64][int(rng.integers(0, 3))])
+    col_major = bool(rng.integers(0, 2))
+    c16 = bool(rng.integers(0, 2))
+    on_gpu = bool(rng.integers(0, 2))
+    fill = int([1, 1, 0, 20][int(rng.integers(0, 4))])
+    n_ctas = int([0, 0, 5, 37][int(rng.integers(0, 4))])
+    m, k = int(rng.integers(130, 2500)), int(rng.integers(1, 1200))
+    if col_major:
+        m, k = _round_up(m, 8), _round_up(k, 8)
+    N = int(rng.integers(128 if col_major else 64, 1100))
+    if not col_major:
+        N = _round_up(N, 8)
+    dens = float(10.0 ** rng.uniform(-2.5, -0.3))
+    a = wl.random_csr(int(rng.integers(0, 1 << 30)), m, k, dens, dtype, empty_rows=tuple(range(min(b, m // 3))))
+    Bs = wl.dense(int(rng.integers(0, 1 << 30)), k, N, ("uniform", -1.0, 1.0), dtype)
+    opt = dict(c_type=lib.C_SAME_AS_INPUT if c16 else lib.C_FP32, layout=lib.COLMAJOR if col_major else lib.ROWMAJOR,
+               stack_min_fill=fill, n_ctas=n_ctas)
+    what = "seed %d: %s b=%d m=%d k=%d N=%d dens=%.4f cm=%d c16=%d fill=%d ctas=%d gpu-built=%d" % (
+        seed, dtype, b, m, k, N, dens, col_major, c16, fill, n_ctas, on_gpu)
+    if on_gpu:
+        rp = torch.from_numpy(a["row_ptr"].astype(np.int64)).cuda()
+        ci = torch.from_numpy(a["col_idx"].astype(np.int32)).cuda()
+        va = to_device(a["vals"])
+        h = lib.spmm_bcsr_create_csr_device(m, k, rp.data_ptr(), ci.data_ptr(), va.data_ptr(), dtype, b, **opt)
+    else:
+        h = lib.spmm_bcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, b, **opt)
+    try:
+        from oracle import formats as F
+        f = F.bcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], b)
+        rows, _, cols = F.bcsr_row_groups(f["block_row_ptr"], f["block_col_idx"], b, fill or {16: 30, 32: 45, 64: 75}[b])
+        info = lib.spmm_get_info(h, N)
+        assert info["n_stacked_rows"] == rows.size and info["n_stack_blocks"] == cols.size, what
+        C = run_gpu_variant(lib, h, Bs, m, N, dtype, c16=c16, col_major=col_major)
+        Cr, S = reference(a, Bs, dtype)
+        assert_close(C, Cr, S, dtype, what)
+    finally:
+        lib.spmm_destroy(h)
+
+
 @pytest.mark.parametrize("seed", range(60))
 def test_wcsr_random_case(lib, seed):
     import torch
