@@ -122,6 +122,9 @@ SCHED_STATIC, SCHED_DYNAMIC = 0, 1
 
 def _opts(b_col=0, split_cols=0, host_only=False, n_ctas=0, c_type=C_FP32, layout=ROWMAJOR, schedule=SCHED_STATIC,
           stack_min_fill=0):
+    """Keyword options of the create functions -> spmm_opts_t (zero = the library's default; the
+    header documents every field).  stack_min_fill: BCSR row groups, 0 = default threshold,
+    -1 = off, 1..100 = minimum percentage of stored sub-blocks for a group to be formed."""
     o = SpmmOpts()
     o.stack_min_fill = int(stack_min_fill)
     o.b_col, o.split_cols, o.host_only, o.n_ctas = b_col, split_cols, int(bool(host_only)), n_ctas
