@@ -119,7 +119,7 @@ typedef struct {
                             for b = 16 / 32 / 64), -1 = off, 1..100 = threshold.  A private
                             second copy of the grouped rows' values is kept on the device; the
                             exported format arrays and nnz_stored are unaffected.  Ignored for
-                            b = 128, E4M3 inputs and the dynamic schedule.                    */
+                            b = 128 and the dynamic schedule.                                 */
     int32_t reserved[8];
 } spmm_opts_t;
 

@@ -256,8 +256,8 @@ int encode_tmA(spmm_handle_s* h) {
 // the device from the uploaded blocks, the groups' index arrays and the map of the stacked values.
 int setup_stack(spmm_handle_s* h) {
     const BcsrHost& f = h->bcsr;
-    // 16-bit types with the static schedule; b = 128 blocks already are 128 rows high
-    const bool eligible = h->es == 2 && !h->dynamic && f.b < 128 && h->stack_min_fill >= 0;
+    // static schedule only; b = 128 blocks already are 128 rows high
+    const bool eligible = !h->dynamic && f.b < 128 && h->stack_min_fill >= 0;
     int rc = build_bcsr_stack(f, eligible ? h->stack_min_fill : -1, &h->stack);
     if (rc || h->host_only || h->stack.ng == 0) return rc;
     const BcsrStack& st = h->stack;

@@ -79,7 +79,7 @@ struct BcsrCfg {
     static_assert((2 * STAGES + 7 + 8) * 8 + 64 <= kBarrierBytes, "barrier area");
     static_assert(kBps == 1 || B <= 32, "multi-block stages are for the small block sizes");
     static_assert(kBB % 32 == 0, "a block row must hold whole K steps");
-    static_assert(H == B || (H == 128 && B < 128 && ES == 2), "stacked blocks: 128 rows of a 16-bit type");
+    static_assert(H == B || (H == 128 && B < 128), "stacked blocks are 128 rows high");
 };
 
 constexpr int kSchedDepth = 4;      // tile indices fetched ahead by the dynamic scheduler
@@ -645,6 +645,11 @@ cudaError_t launch_bcsr_stacked(int dtype, int b, int c16, int col_major, const 
                                 cudaStream_t stream) {
     if (dtype == 1) return launch_stack_fmt<0>(b, c16, col_major, tmA, tmB, tmB3, tmC, p, grid, stream);   // fp16
     if (dtype == 0) return launch_stack_fmt<1>(b, c16, col_major, tmA, tmB, tmB3, tmC, p, grid, stream);   // bf16
+    if (dtype == 3 && !c16 && col_major) {
+        // E4M3: half the bytes per stage, twice the ring depth
+        if (b == 32) return launch_one<32, 128, 2, 8, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        if (b == 64) return launch_one<64, 128, 2, 8, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+    }
     return cudaErrorInvalidValue;
 }
 

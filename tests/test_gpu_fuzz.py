@@ -69,16 +69,18 @@ def test_bcsr_row_groups_random_case(lib, seed):
     sub-blocks are stored) or left to the default threshold, over ragged shapes and all output options."""
     import torch
     rng = np.random.default_rng(11000 + seed)
-    dtype = ["bf16", "fp16"][int(rng.integers(0, 2))]
+    dtype = ["bf16", "fp16", "fp8"][seed % 3]
     b = int([16, 32, 64][int(rng.integers(0, 3))])
-    col_major = bool(rng.integers(0, 2))
-    c16 = bool(rng.integers(0, 2))
+    col_major = bool(rng.integers(0, 2)) or dtype == "fp8"
+    c16 = bool(rng.integers(0, 2)) and dtype != "fp8"
+    if dtype == "fp8" and b == 16:
+        b = 32
     on_gpu = bool(rng.integers(0, 2))
     fill = int([1, 1, 0, 20][int(rng.integers(0, 4))])
     n_ctas = int([0, 0, 5, 37][int(rng.integers(0, 4))])
     m, k = int(rng.integers(130, 2500)), int(rng.integers(1, 1200))
     if col_major:
-        m, k = _round_up(m, 8), _round_up(k, 8)
+        m, k = _round_up(m, 8), _round_up(k, 16 if dtype == "fp8" else 8)
     N = int(rng.integers(128 if col_major else 64, 1100))
     if not col_major:
         N = _round_up(N, 8)

@@ -358,6 +358,9 @@ def _grouped_matrix(seed, m, k, b, dtype):
     (16, "fp16", 512, 512, 128, False, False, 1),        # forced: groups of sparse rows, mostly absent sub-blocks
     (32, "fp16", 640, 384, 512, False, False, 1),
     (64, "fp16", 4096, 256, 608, False, False, 1),
+    (32, "fp8", 1024, 768, 328, False, True, 0),         # E4M3: column-major operands, fp32 Y
+    (64, "fp8", 2048, 512, 1184, False, True, 0),
+    (32, "fp8", 640, 384, 512, False, True, 1),
 ])
 def test_bcsr_row_groups_match_the_oracle(lib, b, dtype, m, k, N, c16, cm, fill):
     from oracle import formats as F
