@@ -166,13 +166,18 @@ def test_bad_run_arguments(lib):
     lib.spmm_destroy(h)
 
 
-@pytest.mark.parametrize("kind", ["bcsr", "wcsr", "bcsr_dynamic"])
+@pytest.mark.parametrize("kind", ["bcsr", "wcsr", "bcsr_dynamic", "bcsr_row_groups"])
 def test_wait_that_runs_out_is_reported_and_the_context_survives(lib, kind):
     """Every wait inside the kernels is bounded.  With the bound set to zero the first wait
     for operands that are still on their way runs out: the kernel leaves early
     through its normal teardown, spmm_check reports SPMM_ERR_DEV_TIMEOUT, and the same
     handle then works again once the bound is restored."""
-    if kind.startswith("bcsr"):
+    if kind == "bcsr_row_groups":
+        # 10 % of the block-rows are full: they form row groups, so the step is two overlapping
+        # launches (the second waits for the first before its CTAs exit) and both leave early
+        a, dtype, size, N = wl.bcsr_sweep(406, m=2048, k=2048, b=16, density=0.1, dtype="fp16"), "fp16", 16, 1024
+        mk = lib.spmm_bcsr_create_csr
+    elif kind.startswith("bcsr"):
         a, dtype, size, N = wl.bcsr_sweep(404, m=2048, k=2048, b=64, density=0.3, dtype="fp16"), "fp16", 64, 1024
         mk = lib.spmm_bcsr_create_csr
         if kind == "bcsr_dynamic":       # tiles handed out at run time: the scheduler warp's waits are bounded too
@@ -184,6 +189,8 @@ def test_wait_that_runs_out_is_reported_and_the_context_survives(lib, kind):
     Bs = wl.dense(41, a["k"], N, ("normal", 0.0, 1.0), dtype)
     h = mk(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], dtype, size)
     try:
+        if kind == "bcsr_row_groups":
+            assert lib.spmm_get_info(h, N)["n_stacked_rows"] > 0
         lib.spmm_set_wait_limit_ns(0)
         run_gpu(lib, h, Bs, a["m"], N, check=False)
         with pytest.raises(lib.SpmmError) as e:
