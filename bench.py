@@ -273,8 +273,8 @@ def roofline_of(info, ms, pk, groups=None):
     r.update({"peak_source": pk["source"], "model_bytes": model_bytes, "t_roof_us": max(t_hbm, t_tc) * 1e6,
               "gather_bytes": info["bytes_gather"], "traffic": None})
     # Second ceiling, context only: every staged operand byte crosses L2 -> shared memory once; the
-    # aggregate TMA rate measured on this GPU type with an L2-resident source is 19.8 TB/s
-    # (microbenchmark described in the design doc section 5).
+    # aggregate TMA rate measured on this GPU type with an L2-resident source is 19.8 TB/s (a
+    # microbenchmark in which every SM streams 128-byte-wide boxes from a 32 MB array).
     # the stored values of A are fetched once per token tile (BCSR: the plan's tile width; WCSR: 128)
     tile = info["plan_token_tile"] if info["format"] == 0 and info["plan_token_tile"] else 128
     n_tt = -(-int(info["plan_n"] if info["format"] == 0 and info["plan_n"] else 0) // tile) if info["format"] == 0 else None
