@@ -293,6 +293,13 @@ int spmm_wcsr_run_static(spmm_handle_t h, const void *B_dev, void *C_dev, int64_
  * ordinary or pinned host memory of k*N elements / m*N elements of C's type, in the
  * handle's layout; the device staging buffers
  * belong to the handle and are reused between calls.
+ * Operands of 8 MB and more travel in up to eight equal chunks of N (column ranges of
+ * row-major operands, moved with 2-D copies of at least 256 bytes per row; token ranges of
+ * column-major ones), each computed by its own kernel launch on `stream`, so that a
+ * chunk's result goes back to the host while the next chunk's operand comes in: two
+ * copy streams owned by the handle carry the transfers, ordered against `stream` with
+ * events.  The result does not depend on the chunking.  Pinned host memory is needed for
+ * the copies to overlap.
  */
 int spmm_run_host(spmm_handle_t h, const void *B_host, void *C_host, int64_t N, void *stream);
 

@@ -141,6 +141,10 @@ struct spmm_handle_s {
     size_t Bstage_bytes = 0;
     float* d_Cstage = nullptr;
     size_t Cstage_bytes = 0;
+    // spmm_run_host in column chunks: the copy streams and the events that order them
+    static constexpr int kMaxHostChunks = 8;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_in[kMaxHostChunks] = {}, ev_run[kMaxHostChunks] = {};
 };
 
 namespace {
@@ -173,6 +177,13 @@ void free_handle(spmm_handle_s* h) {
         cudaFree(h->d_partial);
         cudaFree(h->d_Bstage);
         cudaFree(h->d_Cstage);
+        if (h->s_in) cudaStreamDestroy(h->s_in);
+        if (h->s_out) cudaStreamDestroy(h->s_out);
+        if (h->ev_start) cudaEventDestroy(h->ev_start);
+        for (int i = 0; i < spmm_handle_s::kMaxHostChunks; ++i) {
+            if (h->ev_in[i]) cudaEventDestroy(h->ev_in[i]);
+            if (h->ev_run[i]) cudaEventDestroy(h->ev_run[i]);
+        }
     }
     delete h;
 }
@@ -955,12 +966,79 @@ int spmm_run_host(spmm_handle_t h, const void* B_host, void* C_host, int64_t N, 
         if (cudaMalloc(reinterpret_cast<void**>(&h->d_Cstage), cbytes ? cbytes : 16) != cudaSuccess) return SPMM_ERR_ALLOC;
         h->Cstage_bytes = cbytes;
     }
-    if (cudaMemcpyAsync(h->d_Bstage, B_host, bbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SPMM_ERR_CUDA;
-    int rc = spmm_run(h, h->d_Bstage, h->d_Cstage, N, stream);
+    // Large operands go in column chunks (token chunks), so that the copy of one chunk's result to
+    // the host overlaps the copy of the next chunk's operand to the device (the two directions of
+    // the link are independent) and the kernels in between.  Chunks are whole slices of N that the
+    // kernels accept by themselves; each is staged as its own contiguous array, so the kernels
+    // run unchanged on it.  Row-major operands: a chunk is a column range, copied with 2-D
+    // copies whose rows are at least 256 bytes; column-major: a contiguous range of tokens.
+    int nchunks = 1;
+    if (bbytes + cbytes >= (size_t{8} << 20)) {
+        for (int c = spmm_handle_s::kMaxHostChunks; c >= 2; c >>= 1) {
+            if (N % c != 0) continue;
+            const int64_t nc = N / c;
+            const bool ok = h->col_major ? (nc >= 128)
+                                         : (nc * h->es >= 256 && (nc * h->es) % 16 == 0 && (nc * h->cs) % 16 == 0 &&
+                                            (h->format == 1 || nc >= 64));
+            if (ok) { nchunks = c; break; }
+        }
+    }
+    if (nchunks == 1) {
+        if (cudaMemcpyAsync(h->d_Bstage, B_host, bbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SPMM_ERR_CUDA;
+        int rc = spmm_run(h, h->d_Bstage, h->d_Cstage, N, stream);
+        if (rc) return rc;
+        if (cudaMemcpyAsync(C_host, h->d_Cstage, cbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SPMM_ERR_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return SPMM_ERR_CUDA;
+        return SPMM_OK;
+    }
+    if (!h->s_in) {
+        if (cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&h->ev_start, cudaEventDisableTiming) != cudaSuccess)
+            return SPMM_ERR_CUDA;
+        for (int i = 0; i < spmm_handle_s::kMaxHostChunks; ++i)
+            if (cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&h->ev_run[i], cudaEventDisableTiming) != cudaSuccess)
+                return SPMM_ERR_CUDA;
+    }
+    const int64_t nc = N / nchunks;
+    const size_t bchunk = bbytes / nchunks, cchunk = cbytes / nchunks;
+    const uint8_t* Bh = static_cast<const uint8_t*>(B_host);
+    uint8_t* Chost = static_cast<uint8_t*>(C_host);
+    uint8_t* dB = static_cast<uint8_t*>(h->d_Bstage);
+    uint8_t* dC = reinterpret_cast<uint8_t*>(h->d_Cstage);
+    bool bad = false;
+    // the staging buffers may still be read by work queued on `stream` earlier
+    bad |= cudaEventRecord(h->ev_start, st) != cudaSuccess;
+    bad |= cudaStreamWaitEvent(h->s_in, h->ev_start, 0) != cudaSuccess;
+    for (int c = 0; c < nchunks && !bad; ++c) {
+        if (h->col_major)
+            bad |= cudaMemcpyAsync(dB + c * bchunk, Bh + c * bchunk, bchunk, cudaMemcpyHostToDevice, h->s_in) != cudaSuccess;
+        else
+            bad |= cudaMemcpy2DAsync(dB + c * bchunk, nc * h->es, Bh + static_cast<size_t>(c) * nc * h->es, N * h->es, nc * h->es,
+                                     static_cast<size_t>(h->k), cudaMemcpyHostToDevice, h->s_in) != cudaSuccess;
+        bad |= cudaEventRecord(h->ev_in[c], h->s_in) != cudaSuccess;
+    }
+    int rc = SPMM_OK;
+    for (int c = 0; c < nchunks && !bad && !rc; ++c) {
+        bad |= cudaStreamWaitEvent(st, h->ev_in[c], 0) != cudaSuccess;
+        if (bad) break;
+        rc = spmm_run(h, dB + c * bchunk, dC + c * cchunk, nc, stream);
+        if (rc) break;
+        bad |= cudaEventRecord(h->ev_run[c], st) != cudaSuccess;
+        bad |= cudaStreamWaitEvent(h->s_out, h->ev_run[c], 0) != cudaSuccess;
+        if (h->col_major)
+            bad |= cudaMemcpyAsync(Chost + c * cchunk, dC + c * cchunk, cchunk, cudaMemcpyDeviceToHost, h->s_out) != cudaSuccess;
+        else
+            bad |= cudaMemcpy2DAsync(Chost + static_cast<size_t>(c) * nc * h->cs, N * h->cs, dC + c * cchunk, nc * h->cs, nc * h->cs,
+                                     static_cast<size_t>(h->m), cudaMemcpyDeviceToHost, h->s_out) != cudaSuccess;
+    }
+    // nothing of this call may still be in flight when it returns, whatever happened above
+    const bool s1 = cudaStreamSynchronize(h->s_in) == cudaSuccess;
+    const bool s2 = cudaStreamSynchronize(st) == cudaSuccess;
+    const bool s3 = cudaStreamSynchronize(h->s_out) == cudaSuccess;
     if (rc) return rc;
-    if (cudaMemcpyAsync(C_host, h->d_Cstage, cbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SPMM_ERR_CUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return SPMM_ERR_CUDA;
-    return SPMM_OK;
+    return (bad || !s1 || !s2 || !s3) ? SPMM_ERR_CUDA : SPMM_OK;
 }
 
 int spmm_check(spmm_handle_t h) {

@@ -9,7 +9,7 @@ import pytest
 from oracle import formats as F
 from paper_2604_17834_b200 import workloads as wl
 
-from helpers import assert_close, reference, run_gpu
+from helpers import assert_close, reference, run_gpu, run_gpu_variant
 
 pytestmark = pytest.mark.gpu
 
@@ -150,6 +150,56 @@ def test_run_host_matches_device_run(lib):
     lib.spmm_run_host(h, Bs, Ch, 256)
     assert np.array_equal(C, Ch)
     lib.spmm_destroy(h)
+
+
+@pytest.mark.parametrize("case", ["wcsr_tf32", "bcsr_fp16", "bcsr_bf16_colmajor_c16", "wcsr_fp16_c16"])
+def test_run_host_in_chunks_matches_device_run(lib, case):
+    """Operands of 8 MB and more go through spmm_run_host in column chunks whose transfers overlap;
+    the result is the one spmm_run gives on the whole operand, bit for bit, with pinned and with
+    ordinary host memory, and the same again on the second call."""
+    import torch
+    c16 = case.endswith("c16")
+    cm = "colmajor" in case
+    if case.startswith("wcsr"):
+        dtype = "tf32" if "tf32" in case else "fp16"
+        a = wl.wcsr_irregular(seed=77, m=24000, dtype=dtype)
+        N = 128 if dtype == "tf32" else 256
+        h = lib.spmm_wcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], dtype, 16,
+                                     c_type=lib.C_SAME_AS_INPUT if c16 else lib.C_FP32)
+    else:
+        dtype = "bf16" if "bf16" in case else "fp16"
+        a = wl.bcsr_sweep(78, m=4096, k=4096, b=32, density=0.1, dtype=dtype)
+        N = 1024
+        h = lib.spmm_bcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], dtype, 32,
+                                     c_type=lib.C_SAME_AS_INPUT if c16 else lib.C_FP32,
+                                     layout=lib.COLMAJOR if cm else lib.ROWMAJOR)
+    try:
+        m, k = a["m"], a["k"]
+        Bs = wl.dense(79, k, N, ("uniform", -1.0, 1.0), dtype)
+        want = run_gpu_variant(lib, h, Bs, m, N, dtype, c16=c16, col_major=cm)       # m x N float32
+        Bh = np.ascontiguousarray(Bs.T) if cm else np.ascontiguousarray(Bs)
+        cdt = np.float32 if not c16 else np.uint16
+        shape = (N, m) if cm else (m, N)
+        assert Bh.nbytes + int(np.prod(shape)) * np.dtype(cdt).itemsize >= 8 << 20
+        for pinned in (False, True, True):
+            if pinned:
+                Bt = torch.from_numpy(Bh.view(np.int16) if Bh.dtype == np.uint16 else Bh).pin_memory()
+                Ct = torch.zeros(shape, dtype=torch.float32 if not c16 else torch.int16).pin_memory()
+                lib.spmm_run_host(h, Bt.data_ptr(), Ct.data_ptr(), N)
+                got_raw = Ct.numpy().view(cdt)
+            else:
+                got_raw = np.zeros(shape, dtype=cdt)
+                lib.spmm_run_host(h, Bh, got_raw, N)
+            lib.spmm_check(h)
+            if c16:
+                t16 = torch.from_numpy(got_raw.view(np.int16).copy()).view(torch.bfloat16 if dtype == "bf16" else torch.float16)
+                got = t16.float().numpy()
+            else:
+                got = got_raw
+            got = np.ascontiguousarray(got.T) if cm else got
+            assert np.array_equal(got, want), "%s pinned=%s" % (case, pinned)
+    finally:
+        lib.spmm_destroy(h)
 
 
 def test_bad_run_arguments(lib):
