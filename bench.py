@@ -156,7 +156,8 @@ DEFAULT_OTHERS = ["cfg1_bcsr_tiny", "cfg2_wcsr_irregular_alpha1.8", "cfg3_bcsr_l
                   "cfg3_bcsr_llm_gate_c16", "cfg3_bcsr_llm_gate_cm", "cfg3_bcsr_llm_gate_cm_c16",
                   "cfg3_bcsr_llm_down_cm_c16", "cfg5_wcsr_rmat_n128_c16",
                   "cfg3_bcsr_llm_gate_cm_fp8", "cfg3_bcsr_llm_down_cm_fp8", "cfg2_wcsr_irregular_wh64", "cfg5_wcsr_rmat_n128_wh64",
-                  "cfg4_bcsr_sweep_b64_d0.1_dyn", "cfg4_bcsr_sweep_b16_d0.1_plain", "cfg4_bcsr_sweep_b32_d0.1_plain"]
+                  "cfg4_bcsr_sweep_b64_d0.1_dyn", "cfg4_bcsr_sweep_b16_d0.1_plain", "cfg4_bcsr_sweep_b32_d0.1_plain",
+                  "cfg4_bcsr_sweep_b16_d0.5", "cfg4_bcsr_sweep_b32_d0.5"]
 
 L2_TO_SM_GBS = 19800.0      # measured aggregate L2 -> shared-memory TMA rate (148 SMs x 70 B/cycle at 1.9 GHz)
 
