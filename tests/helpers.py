@@ -22,15 +22,39 @@ def to_device(arr):
     return torch.from_numpy(a).cuda()
 
 
+GUARD = 8192          # elements of canary on either side of C
+CANARY = 24576.0      # exact in fp32, fp16 and bf16
+
+
+def guarded_c(shape, tdt, fill):
+    """C inside a larger allocation whose margins hold a canary value: a store that lands outside C
+    (a tile clipped wrongly, a row index off by one block) shows up in check_guards.
+    -> (whole buffer, view of C with the requested shape)."""
+    import torch
+    n = int(np.prod(shape))
+    buf = torch.full((n + 2 * GUARD,), CANARY, dtype=tdt, device="cuda")
+    C = buf[GUARD:GUARD + n].view(*shape)
+    C.fill_(fill)
+    return buf, C
+
+
+def check_guards(buf, what=""):
+    import torch
+    lo, hi = buf[:GUARD].float(), buf[-GUARD:].float()
+    assert bool(torch.all(lo == CANARY)) and bool(torch.all(hi == CANARY)), "%s: a store landed outside C" % what
+
+
 def run_gpu(lib, h, B_storage, m, N, fill=float("nan"), check=True):
-    """One spmm_run on device buffers; C is pre-filled with NaN so unwritten elements show."""
+    """One spmm_run on device buffers; C is pre-filled with NaN so unwritten elements show, and
+    sits between two canary margins so that stores outside it show as well."""
     import torch
     Bd = to_device(B_storage)
-    C = torch.full((m, N), fill, dtype=torch.float32, device="cuda")
+    buf, C = guarded_c((m, N), torch.float32, fill)
     lib.spmm_run(h, Bd.data_ptr(), C.data_ptr(), N, torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
     if check:
         lib.spmm_check(h)
+    check_guards(buf, "spmm_run")
     return C.cpu().numpy()
 
 
@@ -43,11 +67,12 @@ def run_gpu_variant(lib, h, B_storage, m, N, dtype, c16=False, col_major=False, 
     Bd = to_device(Bs)
     tdt = torch.float32 if not c16 else (torch.bfloat16 if dtype == "bf16" else torch.float16)
     shape = (N, m) if col_major else (m, N)
-    C = torch.full(shape, float("nan"), dtype=tdt, device="cuda")
+    buf, C = guarded_c(shape, tdt, float("nan"))
     lib.spmm_run(h, Bd.data_ptr(), C.data_ptr(), N, torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
     if check:
         lib.spmm_check(h)
+    check_guards(buf, "spmm_run")
     out = C.float().cpu().numpy()
     return np.ascontiguousarray(out.T) if col_major else out
 
