@@ -128,6 +128,16 @@ def workload_table():
                                       fp8_linear(3584, 18944, 1013))
     t["cfg5_wcsr_rmat_s19_n128"] = ("configs[4] recipe at 2^19 rows (a profiling-sized case: B 134 MB), N=128",
                                     lambda: dict(kind="wcsr", a=wl.rmat(scale=19), dtype="fp16", size=16, N=128, Bdist=("normal", 0.0, 1.0)))
+    def lsu(base):
+        """Same workload with the paper's own gather (Sec. 3.2: 128-bit loads through the load/store
+        units) instead of the TMA row gather."""
+        def f():
+            w = base()
+            w["opts"] = dict(w.get("opts", {}), gather=1)
+            return w
+        return f
+    t["cfg2_wcsr_irregular_lsu_gather"] = ("configs[1], B rows gathered with 16-byte cp.async instead of TMA", lsu(cfg2))
+    t["cfg5_wcsr_rmat_n128_lsu_gather"] = ("configs[4] N=128, B rows gathered with 16-byte cp.async instead of TMA", lsu(cfg5(128)))
     t["cfg2_wcsr_irregular_wh64"] = ("configs[1] with 64-row windows", tall(cfg2))
     t["cfg5_wcsr_rmat_n128_wh64"] = ("configs[4] N=128 with 64-row windows", tall(cfg5(128)))
     t["cfg3_bcsr_llm_gate_dyn"] = ("configs[2] gate, dynamic tile scheduling", variant(cfg3_gate, dyn=True))
@@ -156,6 +166,7 @@ DEFAULT_OTHERS = ["cfg1_bcsr_tiny", "cfg2_wcsr_irregular_alpha1.8", "cfg3_bcsr_l
                   "cfg3_bcsr_llm_gate_c16", "cfg3_bcsr_llm_gate_cm", "cfg3_bcsr_llm_gate_cm_c16",
                   "cfg3_bcsr_llm_down_cm_c16", "cfg5_wcsr_rmat_n128_c16",
                   "cfg3_bcsr_llm_gate_cm_fp8", "cfg3_bcsr_llm_down_cm_fp8", "cfg2_wcsr_irregular_wh64", "cfg5_wcsr_rmat_n128_wh64",
+                  "cfg2_wcsr_irregular_lsu_gather", "cfg5_wcsr_rmat_n128_lsu_gather",
                   "cfg4_bcsr_sweep_b64_d0.1_dyn", "cfg4_bcsr_sweep_b16_d0.1_plain", "cfg4_bcsr_sweep_b32_d0.1_plain",
                   "cfg4_bcsr_sweep_b16_d0.5", "cfg4_bcsr_sweep_b32_d0.5"]
 

@@ -92,6 +92,19 @@ typedef enum {
                                     block scheduler; this is the hardware queue itself.       */
 } spmm_sched_t;
 
+/* How the WCSR kernel brings the gathered rows of B into shared memory (opts.gather). */
+typedef enum {
+    SPMM_GATHER_TMA = 0,         /* TMA row gather (four rows x 128 bytes per request), the
+                                    default: the indirect load Sec. 3.2 says TMA cannot do is
+                                    available on this architecture                            */
+    SPMM_GATHER_LSU = 1          /* the paper's own scheme (Sec. 3.2): the producer warps copy
+                                    the rows with 128-bit loads through the load/store units
+                                    (16-byte cp.async) to the swizzled positions the MMA reads.
+                                    Kept for the side-by-side measurement; window height 16,
+                                    fp32 C; measured 1.12x (configs[1]) and 1.43x (configs[4],
+                                    N = 128) slower than the TMA gather.                      */
+} spmm_gather_t;
+
 /* Optional creation parameters; pass NULL for all defaults.  Zero = default. */
 typedef struct {
     int32_t b_col;       /* WCSR: pad every window to a multiple of this many columns.
@@ -120,7 +133,8 @@ typedef struct {
                             second copy of the grouped rows' values is kept on the device; the
                             exported format arrays and nnz_stored are unaffected.  Ignored for
                             b = 128 and the dynamic schedule.                                 */
-    int32_t reserved[8];
+    int32_t gather;      /* spmm_gather_t; WCSR only (a BCSR handle ignores it)              */
+    int32_t reserved[7];
 } spmm_opts_t;
 
 typedef struct {

@@ -54,7 +54,7 @@ EXPORTED_SYMBOLS = (
 class SpmmOpts(ctypes.Structure):
     _fields_ = [("b_col", ctypes.c_int32), ("split_cols", ctypes.c_int32), ("host_only", ctypes.c_int32),
                 ("n_ctas", ctypes.c_int32), ("c_type", ctypes.c_int32), ("layout", ctypes.c_int32),
-                ("schedule", ctypes.c_int32), ("stack_min_fill", ctypes.c_int32), ("reserved", ctypes.c_int32 * 8)]
+                ("schedule", ctypes.c_int32), ("stack_min_fill", ctypes.c_int32), ("gather", ctypes.c_int32), ("reserved", ctypes.c_int32 * 7)]
 
 
 class SpmmInfo(ctypes.Structure):
@@ -118,15 +118,17 @@ ROWMAJOR, COLMAJOR = 0, 1
 
 
 SCHED_STATIC, SCHED_DYNAMIC = 0, 1
+GATHER_TMA, GATHER_LSU = 0, 1
 
 
 def _opts(b_col=0, split_cols=0, host_only=False, n_ctas=0, c_type=C_FP32, layout=ROWMAJOR, schedule=SCHED_STATIC,
-          stack_min_fill=0):
+          stack_min_fill=0, gather=GATHER_TMA):
     """Keyword options of the create functions -> spmm_opts_t (zero = the library's default; the
     header documents every field).  stack_min_fill: BCSR row groups, 0 = default threshold,
     -1 = off, 1..100 = minimum percentage of stored sub-blocks for a group to be formed."""
     o = SpmmOpts()
     o.stack_min_fill = int(stack_min_fill)
+    o.gather = int(gather)
     o.b_col, o.split_cols, o.host_only, o.n_ctas = b_col, split_cols, int(bool(host_only)), n_ctas
     o.c_type, o.layout, o.schedule = int(c_type), int(layout), int(schedule)
     return o

@@ -79,6 +79,7 @@ struct spmm_handle_s {
     bool c16 = false;        // C in the input's 16-bit type (never with TF32, whose input type is fp32)
     bool col_major = false;  // BCSR: B given as X[N][k], C as Y[N][m]
     bool dynamic = false;    // BCSR: tiles handed out at run time through Cluster Launch Control
+    bool lsu_gather = false; // WCSR: B rows gathered by the load/store units (comparison variant) instead of TMA
     int cs = 4;              // bytes per C element
     int n_ctas = 148;
     int sms = 148;
@@ -212,6 +213,7 @@ int check_opts(const spmm_opts_t* opts) {
     if (opts->c_type != SPMM_C_FP32 && opts->c_type != SPMM_C_SAME_AS_INPUT) return SPMM_ERR_INVALID_ARG;
     if (opts->layout != SPMM_ROWMAJOR && opts->layout != SPMM_COLMAJOR) return SPMM_ERR_INVALID_ARG;
     if (opts->schedule != SPMM_SCHED_STATIC && opts->schedule != SPMM_SCHED_DYNAMIC) return SPMM_ERR_INVALID_ARG;
+    if (opts->gather != SPMM_GATHER_TMA && opts->gather != SPMM_GATHER_LSU) return SPMM_ERR_INVALID_ARG;
     return SPMM_OK;
 }
 
@@ -410,6 +412,8 @@ int new_wcsr_handle(spmm_handle_s** hp, int64_t m, int64_t k, int dtype, const s
     h->host_only = opts && opts->host_only;
     h->c16 = opts && opts->c_type == SPMM_C_SAME_AS_INPUT && dtype != SPMM_TF32;
     h->cs = h->c16 ? 2 : 4;
+    h->lsu_gather = opts && opts->gather == SPMM_GATHER_LSU;
+    if (h->lsu_gather && h->c16) { delete h; return SPMM_ERR_UNSUPPORTED; }   // the comparison variant writes fp32 C
     *hp = h;
     *b_col_out = b_col;
     *T_out = T;
@@ -421,6 +425,7 @@ int create_wcsr(spmm_handle_t* out, const CsrView& a, int dtype, int wh, const s
     int b_col = 0, T = 0;
     int rc = new_wcsr_handle(&h, a.m, a.k, dtype, opts, &b_col, &T);
     if (rc) return rc;
+    if (h->lsu_gather && wh != 16) { delete h; return SPMM_ERR_UNSUPPORTED; }
     rc = validate_csr(a);
     if (rc) { delete h; return rc; }
     h->nnz = a.nnz;
@@ -453,6 +458,7 @@ int create_wcsr_device(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* 
     int b_col = 0, T = 0;
     int rc = new_wcsr_handle(&h, m, k, dtype, opts, &b_col, &T);
     if (rc) return rc;
+    if (h->lsu_gather && wh != 16) { delete h; return SPMM_ERR_UNSUPPORTED; }
     rc = device_setup(h, opts);
     if (rc) { free_handle(h); return rc; }
     try {
@@ -777,7 +783,7 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, void* C, float* partial, in
     p.bin_ptr = h->d_bin_ptr;
     p.items = reinterpret_cast<const int4*>(h->d_items);
     // narrow dense operand: the variant whose stages hold more columns
-    const bool narrow = h->d_bin_fill_narrow != nullptr && N <= kWcsrNarrowMaxN;
+    const bool narrow = h->d_bin_fill_narrow != nullptr && N <= kWcsrNarrowMaxN && !h->lsu_gather;
     p.fills = reinterpret_cast<const int2*>(narrow ? h->d_fills_narrow : h->d_fills);
     p.bin_fill = narrow ? h->d_bin_fill_narrow : h->d_bin_fill;
     p.col_idx = h->d_idx;
@@ -798,7 +804,7 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, void* C, float* partial, in
     if (!f.tasks.empty()) {
         int rc = ensure_tmB(h, B, N, 1);
         if (rc) return rc;
-        cudaError_t e = launch_wcsr(h->dtype, f.wh, h->c16, narrow ? 1 : 0, h->tmB, p, h->sms, stream);
+        cudaError_t e = launch_wcsr(h->dtype, f.wh, h->c16, narrow ? 1 : 0, h->lsu_gather ? 1 : 0, h->tmB, p, h->sms, stream);
         if (e != cudaSuccess) return SPMM_ERR_CUDA;
     }
     MergeParams mp;

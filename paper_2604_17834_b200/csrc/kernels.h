@@ -106,8 +106,10 @@ struct WcsrParams {
 // dtype: 0 bf16, 1 fp16, 2 tf32.  groups: 1 or 2.  tmB: 2-D map of B (k rows x N), box = 128
 // bytes x 1 row, 128-byte swizzle (32-byte atoms for tf32), used in row-gather mode.
 // narrow: the N <= 64 variant for 2-byte types at window height 16 (p.fills / p.bin_fill cut to kWcsrNarrowCols).
-cudaError_t launch_wcsr(int dtype, int wh, int c16, int narrow, const CUtensorMap& tmB, const WcsrParams& p, int sms,
-                        cudaStream_t stream);
+// lsu_gather: the comparison variant whose producers gather B rows with 16-byte cp.async copies through the
+// load/store units instead of TMA (window height 16, fp32 C, not narrow); tmB is then unused.
+cudaError_t launch_wcsr(int dtype, int wh, int c16, int narrow, int lsu_gather, const CUtensorMap& tmB, const WcsrParams& p,
+                        int sms, cudaStream_t stream);
 
 struct MergeParams {
     const int32_t* window;   // [n] windows the merge writes

@@ -82,7 +82,11 @@ struct SegIter {
     }
 };
 
-template <int ES, int FMT, int WH, int KT, int STAGES, int PW, int CT, bool NARROW>
+// LSU = true: the gathered rows reach shared memory through the load/store units instead of
+// TMA -- the cooperative gather with 128-bit loads that Sec. 3.2 describes, here as 16-byte
+// cp.async copies that every lane of the producer warp places at the swizzled position the MMA
+// expects.  Kept as a selectable variant so that the two gathers can be measured side by side.
+template <int ES, int FMT, int WH, int KT, int STAGES, int PW, int CT, bool NARROW, bool LSU = false>
 __global__ void __launch_bounds__((PW + 5) * 32, WcsrCfg<ES, WH, KT, STAGES, NARROW>::kCtasPerSm)
 wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
     using Cfg = WcsrCfg<ES, WH, KT, STAGES, NARROW>;
@@ -133,7 +137,110 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
     const int64_t N = p.N;
     const int2 kNoDesc = make_int2(0, 0);
 
-    if (warp < kProducerWarps) {
+    if (LSU && warp < kProducerWarps) {
+        // ------------------------------------------------------------------ gather producers, load/store-unit variant
+        // Same ownership of fills and stages as below.  A gathered row is kCh 16-byte chunks;
+        // one warp-wide issue copies 32 chunks (32 / kCh rows), lane -> (row, chunk) fixed.  The
+        // A tile still arrives by bulk copy (its bytes are the barrier's transaction count); the
+        // warp's own arrival follows the completion of its cp.async copies.
+        if constexpr (LSU) {
+            constexpr int kCh = Cfg::kRowBytes / 16;              // 16 (2-byte types) or 32 (TF32)
+            constexpr int kE16 = 16 / ES;                         // elements per chunk
+            constexpr int kRowsPerIssue = 32 / kCh;
+            constexpr int kIssues = KT / kRowsPerIssue;
+            constexpr int kIdxRegs = (KT + 31) / 32;
+            static_assert(kCh <= 32 && 32 % kCh == 0 && !NARROW, "row of at most 512 bytes");
+            const int c = lane % kCh;                             // my chunk inside a gathered row
+            const int rsub = lane / kCh;                          // my row inside one issue
+            const uint8_t* Bp = static_cast<const uint8_t*>(p.B);
+            const size_t row_pitch = static_cast<size_t>(N) * ES;
+            auto load_idx = [&](const int2 d, int (&idx)[kIdxRegs]) {
+                const int cnt = d.y & 0xFFFF;
+#pragma unroll
+                for (int j = 0; j < kIdxRegs; ++j)
+                    idx[j] = (j * 32 + lane < cnt) ? __ldg(p.col_idx + d.x + j * 32 + lane) : -1;
+            };
+            SegIter seg;
+            seg.init();
+            uint32_t it0 = 0, last_it = 0;
+            bool issued_any = false, ok = true;
+            int idx_cur[kIdxRegs], idx_nxt[kIdxRegs];
+            bool idx_ready = false;
+            while (ok && seg.next(p)) {
+                const int f0 = __ldg(p.bin_fill + seg.b), f1 = __ldg(p.bin_fill + seg.b + 1);
+                const int n0 = seg.tt * Cfg::kBnT;
+                int2 win = (f0 + lane < f1) ? __ldg(p.fills + f0 + lane) : kNoDesc;
+                for (int wbase = f0; wbase < f1 && ok; wbase += 32) {
+                    const int2 nwin = (wbase + 32 + lane < f1) ? __ldg(p.fills + wbase + 32 + lane) : kNoDesc;
+                    const uint32_t itw = it0 + static_cast<uint32_t>(wbase - f0);
+                    int j = static_cast<int>((static_cast<uint32_t>(warp) + kProducerWarps - itw % kProducerWarps) % kProducerWarps);
+                    for (; j < 32 && wbase + j < f1; j += kProducerWarps) {
+                        const uint32_t it = itw + j;
+                        int2 d;
+                        d.x = __shfl_sync(0xffffffffu, win.x, j);
+                        d.y = __shfl_sync(0xffffffffu, win.y, j);
+                        if (!idx_ready) load_idx(d, idx_cur);
+                        const int jn = j + kProducerWarps;        // this warp's next fill, if it is in this segment
+                        const bool have_n = wbase + jn < f1;
+                        int2 dn;
+                        dn.x = __shfl_sync(0xffffffffu, jn < 32 ? win.x : nwin.x, jn & 31);
+                        dn.y = __shfl_sync(0xffffffffu, jn < 32 ? win.y : nwin.y, jn & 31);
+                        const int s = it % STAGES;
+                        const uint32_t ph = (it / STAGES) & 1u;
+                        const int q = d.x;
+                        const int cnt = d.y & 0xFFFF;
+                        if (!__all_sync(0xffffffffu, mbar_wait(empty_bar(s), ph ^ 1u, ctl, 11))) { ok = false; break; }
+                        const uint32_t sb = smem_base + s * Cfg::kStageBytes;
+                        if (lane == 0) {
+                            const uint32_t abytes = (cnt / Cfg::kKStep) * (kWH * 32);
+                            mbar_expect_tx(full_bar(s), abytes);
+                            bulk_load_1d(sb + Cfg::kDenseBytes,
+                                         p.packed + static_cast<size_t>(q / Cfg::kKStep) * (kWH * 32), abytes, full_bar(s));
+                        }
+                        issued_any = true;
+                        last_it = it;
+#pragma unroll
+                        for (int i = 0; i < kIssues; ++i) {
+                            const int r = i * kRowsPerIssue + rsub;          // column of the fill = row of the stage
+                            // (the register that holds row r's index is known at compile time)
+                            const int idx = __shfl_sync(0xffffffffu, idx_cur[(i * kRowsPerIssue) >> 5], r & 31);
+                            if (r < cnt && n0 + c * kE16 < N) {
+                                uint32_t dst = sb + (c >> 3) * Cfg::kAtomStride + r * 128;
+                                if constexpr (ES == 2) {
+                                    dst += ((c & 7) ^ (r & 7)) << 4;         // 128-byte swizzle: chunk ^= row % 8
+                                } else {
+                                    // 128-byte swizzle with 32-byte atoms: 32-byte piece ^= row % 4
+                                    dst += ((((c & 7) >> 1) ^ (r & 3)) << 5) + ((c & 1) << 4);
+                                }
+                                const bool valid = idx >= 0;                  // -1 pads: 16 zero bytes, B is not read
+                                const uint8_t* src = Bp + (valid ? static_cast<size_t>(idx) * row_pitch +
+                                                                       (static_cast<size_t>(n0) + c * kE16) * ES
+                                                                 : 0);
+                                cp_async_16(dst, src, valid);
+                            }
+                        }
+                        cp_async_commit();
+                        if (have_n) load_idx(dn, idx_nxt);
+                        cp_async_wait<0>();
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(full_bar(s));
+#pragma unroll
+                        for (int jj = 0; jj < kIdxRegs; ++jj) idx_cur[jj] = idx_nxt[jj];
+                        idx_ready = have_n;
+                    }
+                    win = nwin;
+                }
+                it0 += static_cast<uint32_t>(f1 - f0);
+            }
+            cp_async_wait<0>();
+            if (!ok && lane == 0 && issued_any) {
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(full_bar(last_it % STAGES), (last_it / STAGES) & 1u) &&
+                       globaltimer_ns() - t0 < 2000000ull) {}
+            }
+        }
+    } else if (warp < kProducerWarps) {
         // ------------------------------------------------------------------ gather producers
         // Lane l of the owning warp issues gather u = l (+32 per round): row group u / kSegs
         // (rows 4*rg .. 4*rg+3 of the fill), 128-byte segment u % kSegs of those rows.
@@ -474,12 +581,12 @@ wcsr_merge_kernel(const MergeParams p) {
     }
 }
 
-template <int ES, int FMT, int WH, int CT, bool NARROW = false>
+template <int ES, int FMT, int WH, int CT, bool NARROW = false, bool LSU = false>
 cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
     constexpr int KT = NARROW ? kWcsrNarrowCols : wcsr_stage_cols(ES);
     constexpr int STAGES = wcsr_stages(ES, WH), PW = wcsr_producer_warps(ES, WH);
     using Cfg = WcsrCfg<ES, WH, KT, STAGES, NARROW>;
-    auto kfn = wcsr_spmm_kernel<ES, FMT, WH, KT, STAGES, PW, CT, NARROW>;
+    auto kfn = wcsr_spmm_kernel<ES, FMT, WH, KT, STAGES, PW, CT, NARROW, LSU>;
     static int occ = 0;
     if (occ == 0) {
         cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
@@ -508,7 +615,16 @@ cudaError_t launch_wh(int dtype, int c16, const CUtensorMap& tmB, const WcsrPara
 
 }  // namespace
 
-cudaError_t launch_wcsr(int dtype, int wh, int c16, int narrow, const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
+cudaError_t launch_wcsr(int dtype, int wh, int c16, int narrow, int lsu_gather, const CUtensorMap& tmB, const WcsrParams& p, int sms,
+                        cudaStream_t stream) {
+    if (lsu_gather) {
+        // the comparison variant: window height 16, fp32 C, 128-token stages
+        if (wh != 16 || c16 || narrow) return cudaErrorInvalidValue;
+        if (dtype == 2) return launch_one<4, 2, 16, 0, false, true>(tmB, p, sms, stream);
+        if (dtype == 1) return launch_one<2, 0, 16, 0, false, true>(tmB, p, sms, stream);
+        if (dtype == 0) return launch_one<2, 1, 16, 0, false, true>(tmB, p, sms, stream);
+        return cudaErrorInvalidValue;
+    }
     if (narrow) {
         if (wh != 16 || (dtype != 0 && dtype != 1)) return cudaErrorInvalidValue;
         if (dtype == 1) return c16 ? launch_one<2, 0, 16, 1, true>(tmB, p, sms, stream) : launch_one<2, 0, 16, 0, true>(tmB, p, sms, stream);

@@ -412,3 +412,42 @@ def test_bcsr_row_groups_from_the_gpu_builder(lib):
         assert_close(got, Cr, S, dtype, "gpu-built, row groups")
     finally:
         lib.spmm_destroy(h)
+
+
+# --------------------------------------------------------------------------- the paper's own gather (load/store units)
+
+
+@pytest.mark.parametrize("dtype,m,k,N,T", [("tf32", 3000, 2500, 128, 0), ("tf32", 1000, 900, 328, 64), ("fp16", 4000, 3000, 256, 0),
+                                           ("bf16", 777, 1300, 72, 32), ("fp16", 2048, 2048, 1000, 128)])
+def test_wcsr_lsu_gather_matches_the_oracle_and_the_tma_gather(lib, dtype, m, k, N, T):
+    """opts.gather = GATHER_LSU: B rows copied by the producer warps with 16-byte cp.async (the
+    cooperative 128-bit gather of Sec. 3.2) to the swizzled positions the MMA reads.  Same MMAs in the
+    same order as the default TMA gather, so the two results agree to the last bit."""
+    a = wl.wcsr_irregular(seed=500 + N, m=m, k=k, dtype=dtype, max_len=700)
+    Bs = wl.dense(501, k, N, ("normal", 0.0, 1.0), dtype)
+    Cr, S = reference(a, Bs, dtype)
+    outs = []
+    for gather in (lib.GATHER_LSU, lib.GATHER_TMA):
+        h = lib.spmm_wcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, 16, split_cols=T, gather=gather)
+        try:
+            info = lib.spmm_get_info(h, N)
+            if T:
+                assert info["n_split"] > 0, "the case must exercise split windows"
+            C = run_gpu(lib, h, Bs, m, N)
+            assert_close(C, Cr, S, dtype, "wcsr %s gather=%d" % (dtype, gather))
+            assert np.array_equal(C, run_gpu(lib, h, Bs, m, N))
+            outs.append(C)
+        finally:
+            lib.spmm_destroy(h)
+    assert np.array_equal(outs[0], outs[1])
+
+
+def test_wcsr_lsu_gather_argument_errors(lib):
+    a = wl.wcsr_irregular(seed=9, m=256, k=256, dtype="fp16")
+    for kw, wh in ((dict(gather=lib.GATHER_LSU), 64), (dict(gather=lib.GATHER_LSU, c_type=lib.C_SAME_AS_INPUT), 16)):
+        with pytest.raises(lib.SpmmError) as e:
+            lib.spmm_wcsr_create_csr(256, 256, a["row_ptr"], a["col_idx"], a["vals"], "fp16", wh, **kw)
+        assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
+    with pytest.raises(lib.SpmmError) as e:
+        lib.spmm_wcsr_create_csr(256, 256, a["row_ptr"], a["col_idx"], a["vals"], "fp16", 16, gather=7)
+    assert e.value.code == lib.SPMM_ERR_INVALID_ARG
