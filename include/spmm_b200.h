@@ -15,8 +15,10 @@
  *
  * Conventions
  *   - A is m x k, B is k x N row-major (B[r*N + c]), C is m x N row-major,
- *     fp32.  C is overwritten completely (no alpha / beta; Sec. 2.3 states
- *     the problem as C = A x B).
+ *     fp32 -- unless the handle was created with opts.layout (both operands
+ *     column-major, BCSR) or opts.c_type (C in the input's 16-bit type).  C is
+ *     overwritten completely (no alpha / beta; Sec. 2.3 states the problem as
+ *     C = A x B).
  *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA
  *     device memory of the current device.  The library never frees or keeps
  *     a caller's pointer beyond the call that receives it.
@@ -53,7 +55,7 @@ typedef enum {
                                     this library built)                                       */
 } spmm_status_t;
 
-/* Value type of A and B.  Accumulation and C are always fp32. */
+/* Value type of A and B.  Accumulation is always fp32 (C: see spmm_ctype_t). */
 typedef enum {
     SPMM_BF16 = 0,               /* 2-byte bfloat16 storage                                   */
     SPMM_FP16 = 1,               /* 2-byte IEEE half storage                                  */
@@ -256,7 +258,11 @@ int spmm_wcsr_create_coo(spmm_handle_t *out, int64_t m, int64_t k, int64_t nnz,
  * spmm_run(h, ., ., N, .) uses -- so that it can be inspected with spmm_export / spmm_get_info.
  * The schedule answers the load imbalance Sec. 3.5 and Sec. 4.2 (opt6) report for a persistent
  * kernel with a fixed tile order: tiles (block-row x token tile) are dealt to the CTAs ahead
- * of time, longest block-row first, each to the least loaded CTA.  Works on host_only handles.
+ * of time, longest block-row first, each to the least loaded CTA.  A handle with row groups
+ * (opts.stack_min_fill) gets two such lists: STACK_TILES for the groups (256-token tiles), whose
+ * launch goes first, and TILES for the other block-rows, dealt with the head start that the
+ * j-th lightest CTA of the first launch leaves to CTA j of the second (loads counted in bytes
+ * staged per block).  Works on host_only handles.
  * spmm_run builds the same schedule on its first call with a new N (that call allocates and
  * may synchronise the device).
  */
@@ -275,6 +281,8 @@ int spmm_bcsr_plan(spmm_handle_t h, int64_t N);
  * it is (re)allocated here the first time a given N needs more than it holds, so two runs
  * of one handle must not overlap on the GPU, and the first run at a new N may synchronise.
  * Split windows are merged by a fixed-order sum, so results are run-to-run identical.
+ * A BCSR handle with row groups launches its kernel twice (groups, then the other block-rows;
+ * the second launch starts on the SMs the first leaves idle and does not finish before it).
  */
 int spmm_run(spmm_handle_t h, const void *B_dev, void *C_dev, int64_t N, void *stream);
 
