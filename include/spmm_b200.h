@@ -114,8 +114,11 @@ typedef struct {
                             TF32 -- the K extent of one tensor-core instruction (Sec. 2.3,
                             Sec. 4.1 uses 8 with TF32).                                      */
     int32_t split_cols;  /* WCSR: sub-task size T in columns (Sec. 3.3); multiple of b_col.
-                            Default: about a quarter of one bin's share of the padded columns,
-                            rounded down to a multiple of 64 and clamped to [128, 4096].      */
+                            Default: the largest of one bin's share of the padded columns, its
+                            half, quarter and eighth (rounded down to a multiple of 64, clamped
+                            to [128, 65536]) whose longest-first assignment of the sub-tasks to
+                            the bins ends within 2 % of the best of the four: as few split
+                            windows as the balance allows.                                    */
     int32_t host_only;   /* 1: build the format on the host only (no CUDA call at all); the
                             handle serves spmm_export / spmm_get_info, spmm_run fails.       */
     int32_t n_ctas;      /* persistent grid size the schedule is built for; default = the

@@ -182,11 +182,39 @@ def bcsr_row_order(block_row_ptr):
     return np.argsort(-lens, kind="stable").astype(np.int32)
 
 
-def default_split_cols(P, n_bins):
-    """Sub-task size used when the caller gives none: a quarter of one bin's share of the
-    padded columns, rounded down to a multiple of 64, clamped to [128, 4096]."""
-    t = (P // (n_bins * 4)) // 64 * 64
-    return int(min(4096, max(128, t)))
+def default_split_cols(window_row_ptr, n_bins, fixed_cost=32):
+    """Sub-task size used when the caller gives none (the paper only says "fixed-size sub-tasks",
+    Sec. 3.3): candidates are one bin's share of the padded columns and its half, quarter and
+    eighth, each rounded down to a multiple of 64 and clamped to [128, 65536]; for each, the
+    windows are cut into chunks of T and dealt longest first to the lightest bin (cost = columns
+    + fixed_cost); the largest candidate whose heaviest bin is within 2 % of the best of the four
+    is taken -- as few split windows as the balance allows."""
+    import heapq
+    wptr = np.asarray(window_row_ptr, dtype=np.int64)
+    lens = np.diff(wptr)
+    P = int(wptr[-1])
+
+    def max_load(T):
+        full, rem = lens // T, lens % T
+        full = np.where((rem == 0) & (full > 0), full - 1, full)      # the last chunk of a multiple of T is a chunk of T
+        rem = np.where((rem == 0) & (lens > 0), T, rem)
+        counts = np.concatenate([np.full(int(full.sum()), T, dtype=np.int64), rem[rem > 0]])
+        counts = np.sort(counts)[::-1]
+        heap = [0] * n_bins
+        mx = 0
+        for c in counts.tolist():
+            l = heapq.heappop(heap) + c + fixed_cost
+            heapq.heappush(heap, l)
+            mx = max(mx, l)
+        return mx
+
+    cands = [int(min(65536, max(128, ((P // n_bins) >> i) // 64 * 64))) for i in range(4)]
+    loads = [max_load(T) for T in cands]
+    best = min(loads)
+    for T, l in zip(cands, loads):
+        if l * 100 <= best * 102:
+            return T
+    return cands[3]
 
 
 def task_bins(plan, n_bins, fixed_cost=32):

@@ -288,13 +288,45 @@ int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost*
     return plan_wcsr(out, T, n_bins, a.es);
 }
 
+// Largest bin load of the longest-processing-time assignment when windows are cut into chunks of T.
+static int64_t lpt_max_load(const std::vector<int32_t>& window_row_ptr, int64_t nwin, int T, int n_bins) {
+    std::vector<int32_t> counts;
+    for (int64_t w = 0; w < nwin; ++w) {
+        int32_t len = window_row_ptr[w + 1] - window_row_ptr[w];
+        for (; len > T; len -= T) counts.push_back(T);
+        if (len > 0) counts.push_back(len);
+    }
+    std::sort(counts.begin(), counts.end(), std::greater<int32_t>());
+    std::priority_queue<int64_t, std::vector<int64_t>, std::greater<int64_t>> heap;
+    for (int j = 0; j < n_bins; ++j) heap.push(0);
+    int64_t mx = 0;
+    for (int32_t c : counts) {
+        const int64_t l = heap.top() + c + kTaskFixedCost;
+        heap.pop();
+        heap.push(l);
+        mx = std::max(mx, l);
+    }
+    return mx;
+}
+
+int default_split_cols(const std::vector<int32_t>& window_row_ptr, int64_t nwin, int64_t P, int n_bins) {
+    // candidates: one bin's share of the padded columns and its half, quarter and eighth
+    int cand[4];
+    int64_t load[4], best = INT64_MAX;
+    for (int i = 0; i < 4; ++i) {
+        const int64_t t = ((P / n_bins) >> i) / 64 * 64;
+        cand[i] = static_cast<int>(std::min<int64_t>(65536, std::max<int64_t>(128, t)));
+        load[i] = (i > 0 && cand[i] == cand[i - 1]) ? load[i - 1] : lpt_max_load(window_row_ptr, nwin, cand[i], n_bins);
+        best = std::min(best, load[i]);
+    }
+    for (int i = 0; i < 4; ++i)
+        if (load[i] * 100 <= best * 102) return cand[i];
+    return cand[3];
+}
+
 int plan_wcsr(WcsrHost* out, int T, int n_bins, int es) {
     const int64_t nwin = out->nwin, P = out->P;
-    if (T == 0) {
-        int64_t t = P / (static_cast<int64_t>(n_bins) * 4);
-        t = (t / 64) * 64;
-        T = static_cast<int>(std::min<int64_t>(4096, std::max<int64_t>(128, t)));
-    }
+    if (T == 0) T = default_split_cols(out->window_row_ptr, nwin, P, n_bins);
     out->T = T;
 
     // split plan: consecutive chunks of T columns; a window with one chunk writes C itself

@@ -140,8 +140,11 @@ constexpr int64_t bcsr_stack_block_cost() { return 2 * (256 + 128); }
 constexpr int64_t bcsr_block_cost(int b, int groups) { return 2 * (128 * groups + b); }
 // a row group's tile writes 128 rows of C whatever its length
 constexpr int kStackTileFixedCost = 8;
-// T = 0 picks the sub-task size from the matrix: about a quarter of one bin's share of the
-// padded columns, rounded down to a multiple of 64 and clamped to [128, 4096].
+// T = 0 picks the sub-task size from the matrix (default_split_cols): the largest of one bin's
+// share of the padded columns, its half, quarter and eighth (each rounded down to a multiple of 64
+// and clamped to [128, 65536]) whose longest-processing-time assignment ends within 2 % of the
+// best of the four: as few split windows as the balance allows.
+int default_split_cols(const std::vector<int32_t>& window_row_ptr, int64_t nwin, int64_t P, int n_bins);
 int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost* out);
 // Second half of build_wcsr: split plan, bins, fills and merge lists from out->window_row_ptr / out->P.
 int plan_wcsr(WcsrHost* out, int T, int n_bins, int es);

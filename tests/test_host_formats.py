@@ -234,14 +234,41 @@ def test_wcsr_format_plan_and_bins_are_bit_exact(lib, dtype, m, k, dens, T, wh):
         lib.spmm_destroy(h)
 
 
+def _split_size_by_plan_and_bins(wptr, n_bins):
+    """The default sub-task size recomputed through the (separately pinned) split plan and bins."""
+    P = int(wptr[-1])
+    cands = [int(min(65536, max(128, ((P // n_bins) >> i) // 64 * 64))) for i in range(4)]
+    loads = []
+    for T in cands:
+        plan = F.split_plan(wptr, T)
+        bin_ptr, bin_tasks = F.task_bins(plan, n_bins)
+        cost = plan[:, 2].astype(np.int64) + 32
+        loads.append(max(int(cost[bin_tasks[bin_ptr[j]:bin_ptr[j + 1]]].sum()) for j in range(n_bins)))
+    best = min(loads)
+    return next(T for T, l in zip(cands, loads) if l * 100 <= best * 102), cands, loads
+
+
 def test_default_split_size(lib):
+    """No split_cols given: the largest of a bin's share of the columns and its half, quarter and eighth
+    whose longest-first assignment ends within 2 % of the best of the four."""
     a = wl.wcsr_irregular(seed=4, m=30000, dtype="fp16")
     h = lib.spmm_wcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "fp16", 16, host_only=True, n_ctas=3)
     info = lib.spmm_get_info(h)
-    assert info["n_bins"] == 9 and info["split_cols"] == F.default_split_cols(info["n_units"], 9)
-    assert 128 <= info["split_cols"] <= 4096 and info["split_cols"] % 64 == 0
+    wptr = lib.spmm_export(h, lib.X_WCSR_WINDOW_ROW_PTR, np.int32)
     lib.spmm_destroy(h)
-    assert F.default_split_cols(100, 8) == 128 and F.default_split_cols(10 ** 9, 8) == 4096
+    want, cands, loads = _split_size_by_plan_and_bins(wptr, 9)
+    assert info["n_bins"] == 9 and info["split_cols"] == want == F.default_split_cols(wptr, 9)
+    assert 128 <= info["split_cols"] <= 65536 and info["split_cols"] % 64 == 0
+    # few heavy windows among many light ones: the whole share balances, so nothing smaller is taken
+    wp = np.concatenate(([0], np.cumsum([10000] + [64] * 1000)))
+    assert F.default_split_cols(wp, 8) == _split_size_by_plan_and_bins(wp, 8)[0] == (74000 // 8) // 64 * 64
+    # nine equal heavy windows on eight bins: chunks of a whole share would leave one bin with two of them
+    wp = np.concatenate(([0], np.cumsum([4096] * 9)))
+    got = F.default_split_cols(wp, 8)
+    assert got == _split_size_by_plan_and_bins(wp, 8)[0] and got < 4608
+    # clamps
+    assert F.default_split_cols(np.array([0, 64, 128]), 8) == 128
+    assert F.default_split_cols(np.array([0, 10 ** 8]), 2) == 65536
 
 
 def test_wcsr_irregular_workload(lib):
