@@ -175,7 +175,7 @@ L2_TO_SM_GBS = 19800.0      # measured aggregate L2 -> shared-memory TMA rate (1
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures whose
 # summaries are under profiles/ (None where no capture of that exact launch exists).
 NCU_DRAM_TRAFFIC = {
-    "cfg2_wcsr_irregular": 138.6e6,     # profiles/wcsr_spmm_cfg2_ncu.md
+    "cfg2_wcsr_irregular": 131.8e6,     # profiles/wcsr_spmm_cfg2_ncu.md
     "cfg5_wcsr_rmat_n128": 3.80e9,      # profiles/wcsr_spmm_cfg5_n128_dram.md
     # captured at N = 16,384 (1.383 GB) and scaled by 4 to N = 65,536: one L2 slab is 2048
     # tokens, so traffic grows in proportion to N (profiles/bcsr_spmm_cfg3_n8192_ncu.md)
