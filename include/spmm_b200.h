@@ -103,7 +103,7 @@ typedef enum {
                                     the rows with 128-bit loads through the load/store units
                                     (16-byte cp.async) to the swizzled positions the MMA reads.
                                     Kept for the side-by-side measurement; window height 16,
-                                    fp32 C; measured 1.12x (configs[1]) and 1.43x (configs[4],
+                                    fp32 C; measured 1.16x (configs[1]) and 1.45x (configs[4],
                                     N = 128) slower than the TMA gather.                      */
 } spmm_gather_t;
 
