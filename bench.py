@@ -2,16 +2,23 @@
 """Benchmark of the B200 SpMM hot path (BCSR and WCSR kernels behind the C ABI).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
-                    [--only NAME [--dense-width N]] [--skip-others] [--others A,B] [--no-cpu]
+                    [--only NAME [--dense-width N]] [--skip-others] [--others A,B | all] [--no-cpu]
+                    [--no-e2e] [--ubench]
 
 A step is one ``spmm_run`` (the SpMM kernel, plus the merge kernel for WCSR) on
-inputs already resident in HBM.  The headline workload is configs[1] (WCSR,
-100,000 x 100,000 TF32, N = 128); the other configurations are measured the same
-way and reported under "others".  Throughput is GFLOP/s over stored nonzeros,
-2 * nnz_stored * N / t.  L2 is flushed (a 512 MB write) before every timed
-launch and each launch is timed with its own pair of CUDA events on the
-launching stream.  With N > 1 GPUs every rank runs an independent replica of the
-same workload (the path has no exchange step); value = total flops / max time.
+inputs already resident in HBM.  The headline workload is the largest single-GPU
+configuration, configs[2] gate (BCSR, 18944 x 3584 bf16, 64 x 64 blocks, 90 % of
+the blocks zero, N = 65,536, fp32 C); the other configurations are measured the
+same way.  Throughput is GFLOP/s over stored nonzeros, 2 * nnz_stored * N / t.
+L2 is flushed (a 512 MB write) before every timed launch and each launch is
+timed with its own pair of CUDA events on the launching stream.  With N > 1 GPUs
+every rank runs an independent replica of the same workload (the path has no
+exchange step); value = total flops / max time.
+
+Output: every other workload is printed as ONE short JSON line of its own
+({"other": ...}) as soon as it is measured; the LAST line of stdout is the
+compact result line (metric, value, roofline, cpu_baseline, e2e, clocks and a
+five-field summary of the others).
 
 ``--impl reference`` times the fp64 CPU oracle (oracle/) on the host cores on a
 bounded sample of the same workload and prints the same line with
@@ -36,6 +43,7 @@ from paper_2604_17834_b200 import workloads as wl  # noqa: E402
 
 METRIC = "SpMM GFLOP/s over stored nonzeros (2*nnz_stored*N/time)"
 UNIT = "GFLOP/s"
+MAX_LINE_BYTES = 1450      # the result line (last line of stdout)
 
 
 # --------------------------------------------------------------------------- workloads
@@ -64,7 +72,7 @@ def workload_table():
 
     def variant(base, c16=False, cm=False, dyn=False):
         """Same matrix and dense operand; C in the input's 16-bit type and / or column-major
-        operands (X = B^T in, Y = C^T out: the linear-layer shape of Sec. 4.3), or tiles
+        operands (X = B^T in, Y = C^T out: the linear-layer shape of Sec. 4.4), or tiles
         scheduled at run time through Cluster Launch Control instead of the static plan."""
         def f():
             w = base()
@@ -157,23 +165,26 @@ def workload_table():
 
 
 _CACHE = {}
-HEADLINE = "cfg2_wcsr_irregular"
-DEFAULT_OTHERS = ["cfg1_bcsr_tiny", "cfg2_wcsr_irregular_alpha1.8", "cfg3_bcsr_llm_gate", "cfg3_bcsr_llm_down",
+# the largest single-GPU configuration: the line's value, roofline, e2e and cpu_baseline are its
+HEADLINE = "cfg3_bcsr_llm_gate"
+# measured by default beside the headline: one or more cases of every other configuration
+DEFAULT_OTHERS = ["cfg1_bcsr_tiny", "cfg2_wcsr_irregular", "cfg3_bcsr_llm_down",
                   "cfg4_bcsr_sweep_b16_d0.1", "cfg4_bcsr_sweep_b32_d0.1", "cfg4_bcsr_sweep_b64_d0.1",
-                  "cfg4_bcsr_sweep_b128_d0.1", "cfg4_bcsr_sweep_b64_d0.5", "cfg4_bcsr_sweep_b64_d0.2",
-                  "cfg4_bcsr_sweep_b64_d0.05", "cfg4_bcsr_sweep_b64_d0.01", "cfg4_bcsr_flat_b64_d0.05", "cfg4_bcsr_flat_b64_d0.01",
-                  "cfg5_wcsr_rmat_n32", "cfg5_wcsr_rmat_n128", "cfg5_wcsr_rmat_n256",
-                  "cfg3_bcsr_llm_gate_c16", "cfg3_bcsr_llm_gate_cm", "cfg3_bcsr_llm_gate_cm_c16",
-                  "cfg3_bcsr_llm_down_cm_c16", "cfg5_wcsr_rmat_n128_c16",
-                  "cfg3_bcsr_llm_gate_cm_fp8", "cfg3_bcsr_llm_down_cm_fp8", "cfg2_wcsr_irregular_wh64", "cfg5_wcsr_rmat_n128_wh64",
-                  "cfg2_wcsr_irregular_lsu_gather", "cfg5_wcsr_rmat_n128_lsu_gather",
-                  "cfg4_bcsr_sweep_b64_d0.1_dyn", "cfg4_bcsr_sweep_b16_d0.1_plain", "cfg4_bcsr_sweep_b32_d0.1_plain",
-                  "cfg4_bcsr_sweep_b16_d0.5", "cfg4_bcsr_sweep_b32_d0.5"]
-
-L2_TO_SM_GBS = 19800.0      # measured aggregate L2 -> shared-memory TMA rate (148 SMs x 70 B/cycle at 1.9 GHz)
+                  "cfg4_bcsr_sweep_b128_d0.1", "cfg5_wcsr_rmat_n32", "cfg5_wcsr_rmat_n128", "cfg5_wcsr_rmat_n256"]
+# --others all: the variants (output type, operand layout, 8-bit inputs, 64-row windows, the
+# paper's own gather, dynamic scheduling, row groups off) and more sweep points
+ALL_OTHERS = DEFAULT_OTHERS + [
+    "cfg2_wcsr_irregular_alpha1.8", "cfg4_bcsr_sweep_b64_d0.5", "cfg4_bcsr_sweep_b64_d0.2",
+    "cfg4_bcsr_sweep_b64_d0.05", "cfg4_bcsr_sweep_b64_d0.01", "cfg4_bcsr_flat_b64_d0.05", "cfg4_bcsr_flat_b64_d0.01",
+    "cfg3_bcsr_llm_gate_c16", "cfg3_bcsr_llm_gate_cm", "cfg3_bcsr_llm_gate_cm_c16",
+    "cfg3_bcsr_llm_down_cm_c16", "cfg5_wcsr_rmat_n128_c16",
+    "cfg3_bcsr_llm_gate_cm_fp8", "cfg3_bcsr_llm_down_cm_fp8", "cfg2_wcsr_irregular_wh64", "cfg5_wcsr_rmat_n128_wh64",
+    "cfg2_wcsr_irregular_lsu_gather", "cfg5_wcsr_rmat_n128_lsu_gather",
+    "cfg4_bcsr_sweep_b64_d0.1_dyn", "cfg4_bcsr_sweep_b16_d0.1_plain", "cfg4_bcsr_sweep_b32_d0.1_plain",
+    "cfg4_bcsr_sweep_b16_d0.5", "cfg4_bcsr_sweep_b32_d0.5"]
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures whose
-# summaries are under profiles/ (None where no capture of that exact launch exists).
+# summaries are under profiles/ (absent where no capture of that exact launch exists).
 NCU_DRAM_TRAFFIC = {
     "cfg2_wcsr_irregular": 131.8e6,     # profiles/wcsr_spmm_cfg2_ncu.md
     "cfg5_wcsr_rmat_n128": 3.80e9,      # profiles/wcsr_spmm_cfg5_n128_dram.md
@@ -268,8 +279,10 @@ def device_B(torch, w, seed=7):
     return B
 
 
-def roofline_of(info, ms, pk, groups=None):
-    """Roofline of one spmm_run: slower of tensor time for the stored flops and HBM time for the model bytes."""
+def roofline_of(info, ms, pk, name=None):
+    """Roofline of one spmm_run: slower of tensor time for the stored flops and HBM time for the
+    model bytes (A values + indices + distinct B rows touched + C).  `traffic` is the DRAM
+    traffic ncu measured for the same launch, where a capture exists."""
     model_bytes = info["bytes_a"] + info["bytes_idx"] + info["bytes_b_touched"] + info["bytes_c"]
     # TF32 = half, 8-bit = twice the measured bf16 rate (nominal ratios)
     tc_peak = pk["bf16_tflops"] * {2: 0.5, 3: 2.0}.get(info["dtype"], 1.0)
@@ -282,37 +295,9 @@ def roofline_of(info, ms, pk, groups=None):
     else:
         ach = info["flops_stored"] / t / 1e12
         r = {"bound": "tensor", "achieved": ach, "peak": tc_peak, "unit": "TFLOP/s", "frac": ach / tc_peak}
-    r.update({"peak_source": pk["source"], "model_bytes": model_bytes, "t_roof_us": max(t_hbm, t_tc) * 1e6,
-              "gather_bytes": info["bytes_gather"], "traffic": None})
-    # Second ceiling, context only: every staged operand byte crosses L2 -> shared memory once; the
-    # aggregate TMA rate measured on this GPU type with an L2-resident source is 19.8 TB/s (a
-    # microbenchmark in which every SM streams 128-byte-wide boxes from a 32 MB array).
-    # the stored values of A are fetched once per token tile (BCSR: the plan's tile width; WCSR: 128)
-    tile = info["plan_token_tile"] if info["format"] == 0 and info["plan_token_tile"] else 128
-    n_tt = -(-int(info["plan_n"] if info["format"] == 0 and info["plan_n"] else 0) // tile) if info["format"] == 0 else None
-    if info["format"] == 0:
-        a_passes = max(1, n_tt)
-    else:
-        a_passes = max(1, -(-int(round(info["flops_stored"] / (2.0 * max(1, info["stored_values"])))) // 128))
-    l2_bytes = info["bytes_gather"] + info["bytes_a"] * a_passes
-    if groups and groups["used"]:
-        # row groups: the grouped block-rows stage one slice of the dense operand per stacked block
-        # (not per stored block) and 128 x b of A per 256-token tile
-        es, b, n = 2, info["block"], info["flops_stored"] / (2.0 * max(1, info["stored_values"]))
-        plain = info["n_units"] - groups["grouped_blocks"]
-        l2_bytes = (plain * (b * n * es + b * b * es * a_passes) +
-                    info["n_stack_blocks"] * (b * n * es + 128 * b * es * max(1, -(-int(round(n)) // 256))))
-        r["row_groups"] = {"block_rows": info["n_stacked_rows"], "stored_blocks": groups["grouped_blocks"],
-                           "stacked_blocks": info["n_stack_blocks"]}
-    r["l2_to_sm"] = {"bytes": l2_bytes, "rate_gbs": L2_TO_SM_GBS, "achieved_gbs": l2_bytes / t / 1e9,
-                     "frac": l2_bytes / t / 1e9 / L2_TO_SM_GBS}
+    r.update({"traffic": NCU_DRAM_TRAFFIC.get(name), "peak_source": pk["source"], "model_bytes": model_bytes,
+              "t_roof_us": max(t_hbm, t_tc) * 1e6})
     return r
-
-
-def with_traffic(roof, name):
-    roof = dict(roof)
-    roof["traffic"] = NCU_DRAM_TRAFFIC.get(name)
-    return roof
 
 
 def time_workload(torch, lib, w, steps, warmup, flush):
@@ -358,22 +343,18 @@ def time_workload(torch, lib, w, steps, warmup, flush):
         torch.cuda.synchronize()
         ms_warm = float(np.mean([a.elapsed_time(b) for a, b in wevs]))
         launches = 1 + (1 if (w["kind"] == "wcsr" and (info["n_split"] + info["n_empty"]) > 0) else 0)
-        groups = None
         if w["kind"] == "bcsr" and info["n_stacked_rows"] > 0:
-            used = lib.spmm_export(h, lib.X_BCSR_STACK_TILES, np.int32).size > 0
-            rows = lib.spmm_export(h, lib.X_BCSR_STACK_ROWS, np.int32)
-            brp = lib.spmm_export(h, lib.X_BCSR_BLOCK_ROW_PTR, np.int32)
-            groups = {"used": bool(used), "grouped_blocks": int(np.diff(brp)[rows].sum())}
-            if used and lib.spmm_export(h, lib.X_BCSR_TILES, np.int32).size > 0:
-                launches = 2
-        return dict(h=None, info=info, groups=groups, ms_mean=float(ms.mean()), ms_median=float(np.median(ms)), ms_min=float(ms.min()), ms_warm=ms_warm,
+            # row groups: their own launch, then the remaining block-rows (if any)
+            if lib.spmm_export(h, lib.X_BCSR_STACK_TILES, np.int32).size > 0:
+                launches = 2 if lib.spmm_export(h, lib.X_BCSR_TILES, np.int32).size > 0 else 1
+        return dict(info=info, ms_mean=float(ms.mean()), ms_median=float(np.median(ms)), ms_min=float(ms.min()), ms_warm=ms_warm,
                     create_ms=create_ms, launches_per_step=launches, B=B, C=C)
     finally:
         lib.spmm_destroy(h)
 
 
 def dense_context(torch, flush, m=18944, k=3584, N=65536, steps=5):
-    """Context only (Sec. 4.3 compares against the dense layer): the dense bf16 product of the
+    """Context only (Sec. 4.4 compares against the dense layer): the dense bf16 product of the
     configs[2] gate shape, Y[N][m] = X[N][k] W[m][k]^T, by torch.matmul (cuBLAS)."""
     X = torch.randn((N, k), device="cuda", dtype=torch.bfloat16)
     W = torch.randn((m, k), device="cuda", dtype=torch.bfloat16) * 0.02
@@ -425,8 +406,14 @@ def summarize(name, desc, res, pk, N):
         "ms_warm_l2": res["ms_warm"],
         "gflops_stored": gf, "gflops_useful": 2.0 * info["nnz"] * N / (ms * 1e-3) / 1e9,
         "fill_ratio": info["fill_ratio"], "stored_values": info["stored_values"], "n_units": info["n_units"],
-        "create_ms": res["create_ms"], "roofline": roofline_of(info, ms, pk, res.get("groups")),
+        "create_ms": res["create_ms"], "launches_per_step": res["launches_per_step"],
+        "roofline": roofline_of(info, ms, pk, name),
     }
+
+
+def r4(x):
+    """Four significant digits: keeps the result line short."""
+    return None if x is None else float("%.4g" % x)
 
 
 def aggregate_over_ranks(ms_local, flops_per_rank, world, dist=None, device="cpu"):
@@ -493,26 +480,35 @@ def cpu_oracle_time_all_cores(w, cores, budget_s=15.0, min_s=3.0):
     return dt * (N / cols), cols, dt * len(times), len(parts)
 
 
+def stored_values_by_oracle(w):
+    """nnz_stored of the workload's format, from the oracle's own format definitions (key pass
+    only: no value array is built): BCSR stored blocks * b * b, WCSR window height * padded columns."""
+    from oracle import formats
+    a = w["a"]
+    if w["kind"] == "bcsr":
+        return formats.bcsr_block_count(a["m"], a["k"], a["row_ptr"], a["col_idx"], w["size"]) * w["size"] ** 2
+    b_col = 32 // wl.elem_size(w["dtype"])
+    return formats.wcsr_padded_cols(a["m"], a["k"], a["row_ptr"], a["col_idx"], w["size"], b_col) * w["size"]
+
+
 def run_reference(args):
+    """The oracle as it stands on the host cores; nothing of the CUDA library is imported or loaded."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     name = args.only or HEADLINE
     desc, builder = workload_table()[name]
     w = builder()
-    from paper_2604_17834_b200 import build
-    build.build()
-    from paper_2604_17834_b200 import binding as lib
-    h, _ = create_handle(lib, w, host_only=True)
-    info = lib.spmm_get_info(h, w["N"])
-    lib.spmm_destroy(h)
+    if args.dense_width:
+        w["N"] = args.dense_width
+    flops_stored = 2.0 * stored_values_by_oracle(w) * w["N"]
     times = []
     for i in range(args.warmup + args.steps):
         t_full, cols, dt = cpu_oracle_time(w, budget_s=max(1.0, 60.0 / (args.warmup + args.steps)))
         if i >= args.warmup:
             times.append(t_full)
     t = float(np.mean(times))
-    val = info["flops_stored"] / t / 1e9
+    val = flops_stored / t / 1e9
     sample = "all %d rows x %d of %d columns per step, scaled linearly in N" % (w["a"]["m"], cols, w["N"])
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
@@ -535,12 +531,22 @@ def main():
     ap.add_argument("--impl", default="b200")
     ap.add_argument("--only", default=None, help="time just this workload as the headline (see workload_table)")
     ap.add_argument("--skip-others", action="store_true")
-    ap.add_argument("--others", default=None, help="comma-separated workload names to report beside the headline")
+    ap.add_argument("--others", default=None, help="comma-separated workload names to measure beside the headline, or 'all'")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end leg (profiling runs)")
     ap.add_argument("--dense-width", type=int, default=0, help="override N of the --only workload (small profiling cases)")
+    ap.add_argument("--ubench", action="store_true",
+                    help="run the machine-constant microbenchmarks (tcgen05.mma interval, TMA load and store rates alone "
+                         "and together) instead of the workloads; one JSON line per case")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.ubench:
+        from paper_2604_17834_b200 import build
+        exe = build.UBENCH_OUT
+        if not os.path.exists(exe):
+            raise SystemExit("%s is missing: build it with `python -m paper_2604_17834_b200.build`" % exe)
+        raise SystemExit(subprocess.call([exe]))
 
     import torch
     import torch.distributed as dist
@@ -579,72 +585,93 @@ def main():
     clocks = sampler.stop()
     info = res["info"]
     ms, value = aggregate_over_ranks(res["ms_mean"], info["flops_stored"], world, dist, "cuda")
-    head = summarize(name, desc, res, pk, w["N"])
+    head = summarize(name if not args.dense_width else None, desc, res, pk, w["N"])
 
     # end to end through the C ABI with host buffers (pinned), copies inside the timed region
     a, N = w["a"], w["N"]
-    Bh = torch.empty(tuple(res["B"].shape), dtype=res["B"].dtype).pin_memory()
-    Bh.copy_(res["B"])
-    Ch = torch.empty(tuple(res["C"].shape), dtype=res["C"].dtype).pin_memory()
-    h, _ = create_handle(lib, w)
-    st = torch.cuda.current_stream().cuda_stream
-    e2e_steps = max(3, min(args.steps, 10))
-    for _ in range(2):
-        lib.spmm_run_host(h, Bh.data_ptr(), Ch.data_ptr(), N, st)
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        lib.spmm_run_host(h, Bh.data_ptr(), Ch.data_ptr(), N, st)
-    torch.cuda.synchronize()
-    e2e_s = (time.perf_counter() - t0) / e2e_steps
-    lib.spmm_destroy(h)
-    e2e_ms, e2e_value = aggregate_over_ranks(e2e_s * 1e3, info["flops_stored"], world, dist, "cuda")
-    e2e = {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
-           "h2d_bytes_per_step": int(Bh.numel() * Bh.element_size()), "d2h_bytes_per_step": int(Ch.numel() * Ch.element_size())}
-    del res["B"], res["C"]
-
-    others, context = [], None
-    if rank == 0 and not args.skip_others and args.only is None:
-        names = args.others.split(",") if args.others else DEFAULT_OTHERS
-        for nm in names:
-            d2, b2 = table[nm]
-            w2 = b2()
-            r2 = time_workload(torch, lib, w2, max(5, args.steps // 3), 3, flush)
-            r2.pop("B"), r2.pop("C")
-            others.append(summarize(nm, d2, r2, pk, w2["N"]))
-            del w2
-            torch.cuda.empty_cache()
-        context = dense_context(torch, flush)
+    e2e = None
+    if not args.no_e2e:
+        Bh = torch.empty(tuple(res["B"].shape), dtype=res["B"].dtype, pin_memory=True)
+        Bh.copy_(res["B"])
+        Ch = torch.empty(tuple(res["C"].shape), dtype=res["C"].dtype, pin_memory=True)
+        del res["B"], res["C"]
         torch.cuda.empty_cache()
+        h, _ = create_handle(lib, w)
+        st = torch.cuda.current_stream().cuda_stream
+        e2e_steps = max(3, min(args.steps, 10))
+        for _ in range(2):
+            lib.spmm_run_host(h, Bh.data_ptr(), Ch.data_ptr(), N, st)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            lib.spmm_run_host(h, Bh.data_ptr(), Ch.data_ptr(), N, st)
+        torch.cuda.synchronize()
+        e2e_s = (time.perf_counter() - t0) / e2e_steps
+        lib.spmm_destroy(h)
+        e2e_ms, e2e_value = aggregate_over_ranks(e2e_s * 1e3, info["flops_stored"], world, dist, "cuda")
+        e2e = {"value": r4(e2e_value), "unit": UNIT, "ms_per_step": r4(e2e_ms), "steps": e2e_steps,
+               "h2d_bytes_per_step": int(Bh.numel() * Bh.element_size()), "d2h_bytes_per_step": int(Ch.numel() * Ch.element_size())}
+        del Bh, Ch
+    res.pop("B", None), res.pop("C", None)
+    torch.cuda.empty_cache()
+
+    # the other configurations: one short line each, printed as soon as it is measured
+    others = []
+    if rank == 0 and not args.skip_others and args.only is None:
+        names = ALL_OTHERS if args.others == "all" else (args.others.split(",") if args.others else DEFAULT_OTHERS)
+        for nm in names:
+            try:
+                d2, b2 = table[nm]
+                w2 = b2()
+                r2 = time_workload(torch, lib, w2, max(5, args.steps // 3), 3, flush)
+                r2.pop("B"), r2.pop("C")
+                o = summarize(nm, d2, r2, pk, w2["N"])
+                del w2
+            except Exception as exc:                    # the result line must come out whatever happens here
+                o = {"workload": nm, "error": "%s: %s" % (type(exc).__name__, exc)}
+            torch.cuda.empty_cache()
+            print(json.dumps({"other": o}), flush=True)
+            others.append(o)
+        if args.others == "all":
+            print(json.dumps({"context": dense_context(torch, flush)}), flush=True)
+            torch.cuda.empty_cache()
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         t_full, cols, dt = cpu_oracle_time(w)
-        cpu = {"value": info["flops_stored"] / t_full / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": "all %d rows x %d of %d columns (%.1f s), scaled linearly in N" % (a["m"], cols, N, dt),
-               "useful_gflops": 2.0 * info["nnz"] * N / t_full / 1e9}
+        cpu = {"value": r4(info["flops_stored"] / t_full / 1e9), "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": "all %d rows x %d of %d columns (%.1f s), scaled in N" % (a["m"], cols, N, dt)}
         cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
         if cores > 1:
             tp, pcols, pdt, nparts = cpu_oracle_time_all_cores(w, cores)
-            cpu["all_cores"] = {"value": info["flops_stored"] / tp / 1e9, "unit": UNIT, "cores": nparts,
-                                "sample": "the same routine on %d disjoint row ranges, one thread each; all rows x %d of %d "
-                                          "columns (%.1f s)" % (nparts, pcols, N, pdt)}
+            cpu["all_cores"] = {"value": r4(info["flops_stored"] / tp / 1e9), "cores": nparts,
+                                "sample": "same routine, %d disjoint row ranges, %d columns (%.1f s)" % (nparts, pcols, pdt)}
 
     if rank == 0:
+        roof = head["roofline"]
+        # everything that does not fit the result line: a line of its own, before it
+        print(json.dumps({"detail": {"headline": head, "cpu_baseline": cpu, "peaks": pk}}), flush=True)
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
-            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "metric": METRIC, "value": r4(value), "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+            "ms_per_step": r4(ms), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": w["dtype"], "data": "synthetic",
-            "config": {"workload": name, "description": desc, "l2": "flushed before every timed launch (512 MB write)",
-                       "timing": "one CUDA-event pair per launch on the launching stream; mean over steps",
-                       "multi_gpu": "independent replicas, no collective"},
+            "config": {"workload": name, "description": desc, "l2": "flushed (512 MB write) before every timed launch"},
             "clocks": clocks, "e2e": e2e,
             "gpu_launches": int(res["launches_per_step"] * args.steps),
-            "roofline": with_traffic(head["roofline"], name if not args.dense_width else None), "cpu_baseline": cpu,
-            "headline_detail": {k: head[k] for k in ("ms_median", "ms_min", "ms_warm_l2", "gflops_useful", "fill_ratio", "create_ms")},
-            "others": others, "context": context,
+            "roofline": {"bound": roof["bound"], "achieved": r4(roof["achieved"]), "peak": roof["peak"], "unit": roof["unit"],
+                         "frac": r4(roof["frac"]), "traffic": roof["traffic"], "peak_source": roof["peak_source"]},
+            "cpu_baseline": None if cpu is None else {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            # per other workload: [name, ms_per_step, roofline frac]; their own lines above have the rest
+            "others": [([o["workload"], "error"] if "error" in o else
+                        [o["workload"], r4(o["ms_per_step"]), float("%.3g" % o["roofline"]["frac"])]) for o in others],
         }
-        print(json.dumps(line))
+        # the result line stays short enough to survive a tail of the output whole: the other
+        # workloads' own lines above carry everything that is dropped here
+        text = json.dumps(line, separators=(",", ":"))
+        while len(text) > MAX_LINE_BYTES and line["others"]:
+            line["others"].pop()
+            text = json.dumps(line, separators=(",", ":"))
+        print(text, flush=True)
     if world > 1:
         dist.destroy_process_group()
 

@@ -50,9 +50,14 @@ typedef enum {
     SPMM_ERR_DEV_TIMEOUT = -7,   /* a bounded wait inside a kernel ran out (see spmm_check)   */
     SPMM_ERR_HOST_ONLY = -8,     /* the handle was created host_only and cannot run           */
     SPMM_ERR_TOO_LARGE = -9,     /* a size exceeds a fixed capacity (int32 index, scratch)    */
-    SPMM_ERR_DEV_BOUNDS = -10    /* a kernel met an index outside its range and stopped using
+    SPMM_ERR_DEV_BOUNDS = -10,   /* a kernel met an index outside its range and stopped using
                                     it (reported by spmm_check; cannot happen with a handle
                                     this library built)                                       */
+    SPMM_ERR_DEV_UNDRAINED = -11 /* as SPMM_ERR_DEV_TIMEOUT, and the wait for the copies or
+                                    tensor-core work the kernel had in flight when it gave up
+                                    ran out as well: it left while they may still have been
+                                    writing shared or tensor memory, so kernels that ran on the
+                                    device afterwards may be affected too (spmm_check)        */
 } spmm_status_t;
 
 /* Value type of A and B.  Accumulation is always fp32 (C: see spmm_ctype_t). */
@@ -79,7 +84,7 @@ typedef enum {
                                     row-major N x k array and receives Y = C^T as a row-major
                                     N x m array: the layout of the paper's BCSR kernel
                                     (Sec. 3.2) and of a linear layer Y = X W^T with a sparse
-                                    weight W = A (Sec. 4.3).  Needs m % 8 == 0, k % 8 == 0 and
+                                    weight W = A (Sec. 4.4).  Needs m % 8 == 0, k % 8 == 0 and
                                     N >= 128; N itself is unconstrained.                      */
 } spmm_layout_t;
 
@@ -89,7 +94,7 @@ typedef enum {
     SPMM_SCHED_DYNAMIC = 1       /* one CTA per tile in the grid; running CTAs take over the
                                     tiles of CTAs that have not started yet (Cluster Launch
                                     Control), in the schedule's global order.  BCSR, fp32
-                                    row-major C only.  Sec. 3.5 / Sec. 5: the paper's dynamic
+                                    row-major C only.  Sec. 3.6 / Sec. 5: the paper's dynamic
                                     scheduler used an atomic counter and lost to the hardware
                                     block scheduler; this is the hardware queue itself.       */
 } spmm_sched_t;
@@ -103,8 +108,7 @@ typedef enum {
                                     the rows with 128-bit loads through the load/store units
                                     (16-byte cp.async) to the swizzled positions the MMA reads.
                                     Kept for the side-by-side measurement; window height 16,
-                                    fp32 C; measured 1.16x (configs[1]) and 1.45x (configs[4],
-                                    N = 128) slower than the TMA gather.                      */
+                                    fp32 C.                                                   */
 } spmm_gather_t;
 
 /* Optional creation parameters; pass NULL for all defaults.  Zero = default. */
@@ -277,9 +281,13 @@ int spmm_bcsr_plan(spmm_handle_t h, int64_t N);
  *   B_dev  device, k x N row-major, elements of the handle's dtype, 16-byte aligned.
  *   C_dev  device, m x N row-major, fp32 (or the handle's 16-bit type with
  *          SPMM_C_SAME_AS_INPUT), 16-byte aligned; every element is written.
- *   N      dense width; N * element size must be a multiple of 16 bytes.
+ *   N      dense width; N * element size must be a multiple of 16 bytes.  A BCSR handle
+ *          with row-major operands also needs N >= 64 (SPMM_ERR_UNSUPPORTED below that; the
+ *          same holds for spmm_bcsr_plan); WCSR accepts any such N.
  * With SPMM_COLMAJOR (BCSR): B_dev is X, N x k row-major, and C_dev is Y, N x m row-major,
  * Y[n][i] = sum_j A[i][j] * X[n][j]; any N >= 128.
+ * The handle must be run with the device it was created on current (SPMM_ERR_INVALID_ARG
+ * otherwise, nothing is launched).
  * WCSR keeps the partial tiles of split windows in a device workspace owned by the handle;
  * it is (re)allocated here the first time a given N needs more than it holds, so two runs
  * of one handle must not overlap on the GPU, and the first run at a new N may synchronise.
@@ -298,11 +306,15 @@ int spmm_run(spmm_handle_t h, const void *B_dev, void *C_dev, int64_t N, void *s
  * call: code that runs inside a framework whose memory pool already owns the device, or a
  * latency-critical loop that cannot afford the device-wide synchronisation an allocation
  * or a free can cause.
- *   - The partial tiles need n_slots * 16 * N * 4 bytes (spmm_get_info: workspace_bytes).
- *     More than 8 MiB returns SPMM_ERR_TOO_LARGE and nothing is launched; choose a larger
- *     split_cols at creation, a smaller N, or use spmm_run.
- *   - The first call on each device looks up the scratch array's device address; make that
- *     first call outside any stream capture.  Later calls only launch kernels.
+ *   - The partial tiles need n_slots * window_height * N * 4 bytes (spmm_get_info:
+ *     workspace_bytes; a 64-row handle needs four times what a 16-row one does).  More than
+ *     8 MiB returns SPMM_ERR_TOO_LARGE and nothing is launched; choose a larger split_cols at
+ *     creation, a smaller N, or use spmm_run.
+ *   - The first call on each device looks up the scratch array's device address, and the
+ *     first launch of each kernel variant (value type, window height, C type, N <= 64 or
+ *     wider) on a device sets that kernel's attributes and may load its code.  Make one
+ *     warm-up call per handle type and N class outside any stream capture and outside the
+ *     loop that must not stall.  Later calls only launch kernels.
  *   - The array is shared by all handles and all calls and keeps the previous call's
  *     contents; every partial tile a call reads is first written by that same call, so
  *     nothing needs clearing.  Two calls that overlap on the GPU (different streams, or

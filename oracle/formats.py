@@ -84,6 +84,14 @@ def bcsr_to_dense(m, k, b, block_row_ptr, block_col_idx, blocks):
     return D[:m, :k]
 
 
+def bcsr_block_count(m, k, row_ptr, col_idx, b):
+    """Number of stored blocks of the BCSR form (Sec. 2.3) without building it: the count of
+    distinct (row // b, column // b) pairs over the stored entries."""
+    col = np.asarray(col_idx, dtype=np.int64)
+    rows = _csr_rows(row_ptr)
+    return int(np.unique((rows // b) * _cdiv(k, b) + (col // b)).shape[0])
+
+
 def fill_ratio_bcsr(nnz, nnzb, b):
     """nnz / (nnz_blocks * b_row * b_col)  (Sec. 2.3)."""
     return nnz / float(nnzb * b * b) if nnzb else 0.0
@@ -133,6 +141,16 @@ def wcsr_to_dense(m, k, wh, window_row_ptr, window_col_idx, values):
             if c >= 0:
                 D[w * wh:(w + 1) * wh, c] = values[:, q]
     return D[:m]
+
+
+def wcsr_padded_cols(m, k, row_ptr, col_idx, wh, b_col):
+    """Padded column count P of the WCSR form (Sec. 2.3) without building it: per window the
+    number of distinct columns, rounded up to a multiple of b_col, summed."""
+    col = np.asarray(col_idx, dtype=np.int64)
+    rows = _csr_rows(row_ptr)
+    ukeys = np.unique((rows // wh) * k + col)
+    cnt = np.bincount(ukeys // k, minlength=_cdiv(m, wh)).astype(np.int64)
+    return int((_cdiv(cnt, b_col) * b_col).sum())
 
 
 def fill_ratio_wcsr(nnz, P, wh):

@@ -36,6 +36,7 @@ SPMM_ERR_DEV_TIMEOUT = -7
 SPMM_ERR_HOST_ONLY = -8
 SPMM_ERR_TOO_LARGE = -9
 SPMM_ERR_DEV_BOUNDS = -10
+SPMM_ERR_DEV_UNDRAINED = -11
 
 X_BCSR_BLOCK_ROW_PTR, X_BCSR_BLOCK_COL_IDX, X_BCSR_BLOCKS, X_BCSR_ROW_ORDER = 0, 1, 2, 3
 X_BCSR_TILE_PTR, X_BCSR_TILES = 4, 5

@@ -67,5 +67,22 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return OUT
 
 
+UBENCH_OUT = os.path.join(HERE, "spmm_ubench")
+
+
+def build_ubench(force: bool = False) -> str:
+    """The machine-constant microbenchmarks (csrc/ubench.cu), a stand-alone program."""
+    src = os.path.join(CSRC, "ubench.cu")
+    if (force or not os.path.exists(UBENCH_OUT)
+            or os.path.getmtime(UBENCH_OUT) < max(os.path.getmtime(src), _newest_header())):
+        tmp = UBENCH_OUT + ".tmp%d" % os.getpid()
+        r = subprocess.run([NVCC] + FLAGS + [src, "-o", tmp], capture_output=True, text=True)
+        if r.returncode != 0:
+            raise RuntimeError("nvcc failed for ubench.cu:\n%s\n%s" % (r.stdout, r.stderr))
+        os.replace(tmp, UBENCH_OUT)
+    return UBENCH_OUT
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build_ubench(force="--force" in sys.argv))

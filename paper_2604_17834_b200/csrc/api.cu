@@ -9,6 +9,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "format.h"
 #include "kernels.h"
 #include "spmm_b200.h"
@@ -17,10 +19,15 @@ using namespace spmm;
 
 namespace {
 
+// NVTX range around an entry point (a no-op unless a profiler is attached).
+struct NvtxRange {
+    explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+    NvtxRange(const NvtxRange&) = delete;
+    NvtxRange& operator=(const NvtxRange&) = delete;
+};
+
 std::atomic<uint64_t> g_wait_limit_ns{2000000000ull};
-#ifdef SPMM_TRACE
-long long* g_trace = nullptr;
-#endif
 
 inline int elem_size(int dtype) { return dtype == SPMM_TF32 ? 4 : (dtype == SPMM_FP8_E4M3 ? 1 : 2); }
 
@@ -606,7 +613,7 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
     // token tile: the largest of 512 / 256 / 128 columns that divides N (Sec. 4.3: pick a tile
     // width that divides the dense width so that no padded columns are computed); otherwise
     // the largest tile, whose ragged last tile is predicated.
-    const int gmax = bcsr_token_groups_max(f.b);
+    const int gmax = bcsr_token_groups_max(f.b, h->c16 ? 1 : 0, h->col_major ? 1 : 0);
     int groups = 0;
     for (int g = gmax; g >= 1; g >>= 1)
         if (N % (128 * g) == 0) { groups = g; break; }
@@ -732,12 +739,8 @@ int run_bcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t s
     p.N = N;
     p.status = h->d_status;
     p.wait_limit_ns = g_wait_limit_ns.load();
-    p.trace = nullptr;
     p.stack_rows = nullptr;
     p.overlap = 0;
-#ifdef SPMM_TRACE
-    p.trace = g_trace;
-#endif
     CUtensorMap tmA = h->tmA;
     if (!h->tmA_ok) {
         // no stored block at all: the kernel never touches A, any valid map will do
@@ -797,10 +800,6 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, void* C, float* partial, in
     p.n_tt = static_cast<int32_t>((N + bnt - 1) / bnt);
     p.status = h->d_status;
     p.wait_limit_ns = g_wait_limit_ns.load();
-    p.trace = nullptr;
-#ifdef SPMM_TRACE
-    p.trace = g_trace;
-#endif
     if (!f.tasks.empty()) {
         int rc = ensure_tmB(h, B, N, 1);
         if (rc) return rc;
@@ -838,6 +837,10 @@ int run_wcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t s
 int check_run_args(spmm_handle_s* h, const void* B, const void* C, int64_t N) {
     if (!h || !B || !C || N <= 0) return SPMM_ERR_INVALID_ARG;
     if (h->host_only) return SPMM_ERR_HOST_ONLY;
+    // the handle's arrays, tensor maps and kernel attributes belong to the device it was created on
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SPMM_ERR_CUDA;
+    if (dev != h->device) return SPMM_ERR_INVALID_ARG;
     // row-major B and C have N elements per row: rows must stay 16-byte aligned (column-major
     // operands have k and m elements per row, checked at creation)
     if (!h->col_major && (N * h->es) % 16 != 0) return SPMM_ERR_UNSUPPORTED;
@@ -854,6 +857,7 @@ extern "C" {
 
 int spmm_bcsr_create_csr(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* row_ptr, const int32_t* col_idx,
                          const void* vals, int dtype, int block, const spmm_opts_t* opts) {
+    NvtxRange nvtx_range("spmm_bcsr_create_csr");
     if (!out) return SPMM_ERR_INVALID_ARG;
     *out = nullptr;
     CsrView v;
@@ -865,6 +869,7 @@ int spmm_bcsr_create_csr(spmm_handle_t* out, int64_t m, int64_t k, const int64_t
 int spmm_bcsr_create_csr_device(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* row_ptr_dev,
                                 const int32_t* col_idx_dev, const void* vals_dev, int dtype, int block,
                                 const spmm_opts_t* opts, void* stream) {
+    NvtxRange nvtx_range("spmm_bcsr_create_csr_device");
     if (!out) return SPMM_ERR_INVALID_ARG;
     *out = nullptr;
     if (dtype < 0 || dtype > 3 || m < 0 || k < 0 || !row_ptr_dev) return SPMM_ERR_INVALID_ARG;
@@ -875,6 +880,7 @@ int spmm_bcsr_create_csr_device(spmm_handle_t* out, int64_t m, int64_t k, const 
 int spmm_wcsr_create_csr_device(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* row_ptr_dev,
                                 const int32_t* col_idx_dev, const void* vals_dev, int dtype, int window_height,
                                 const spmm_opts_t* opts, void* stream) {
+    NvtxRange nvtx_range("spmm_wcsr_create_csr_device");
     if (!out) return SPMM_ERR_INVALID_ARG;
     *out = nullptr;
     if (dtype < 0 || dtype > 3 || m < 0 || k < 0 || !row_ptr_dev) return SPMM_ERR_INVALID_ARG;
@@ -884,6 +890,7 @@ int spmm_wcsr_create_csr_device(spmm_handle_t* out, int64_t m, int64_t k, const 
 
 int spmm_bcsr_create_coo(spmm_handle_t* out, int64_t m, int64_t k, int64_t nnz, const int32_t* rows,
                          const int32_t* cols, const void* vals, int dtype, int block, const spmm_opts_t* opts) {
+    NvtxRange nvtx_range("spmm_bcsr_create_coo");
     if (!out) return SPMM_ERR_INVALID_ARG;
     *out = nullptr;
     if (dtype < 0 || dtype > 3) return SPMM_ERR_INVALID_ARG;
@@ -900,6 +907,7 @@ int spmm_bcsr_create_coo(spmm_handle_t* out, int64_t m, int64_t k, int64_t nnz, 
 
 int spmm_wcsr_create_csr(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* row_ptr, const int32_t* col_idx,
                          const void* vals, int dtype, int window_height, const spmm_opts_t* opts) {
+    NvtxRange nvtx_range("spmm_wcsr_create_csr");
     if (!out) return SPMM_ERR_INVALID_ARG;
     *out = nullptr;
     CsrView v;
@@ -911,6 +919,7 @@ int spmm_wcsr_create_csr(spmm_handle_t* out, int64_t m, int64_t k, const int64_t
 int spmm_wcsr_create_coo(spmm_handle_t* out, int64_t m, int64_t k, int64_t nnz, const int32_t* rows,
                          const int32_t* cols, const void* vals, int dtype, int window_height,
                          const spmm_opts_t* opts) {
+    NvtxRange nvtx_range("spmm_wcsr_create_coo");
     if (!out) return SPMM_ERR_INVALID_ARG;
     *out = nullptr;
     if (dtype < 0 || dtype > 3) return SPMM_ERR_INVALID_ARG;
@@ -927,6 +936,7 @@ int spmm_wcsr_create_coo(spmm_handle_t* out, int64_t m, int64_t k, int64_t nnz, 
 }
 
 int spmm_run(spmm_handle_t h, const void* B_dev, void* C_dev, int64_t N, void* stream) {
+    NvtxRange nvtx_range("spmm_run");
     int rc = check_run_args(h, B_dev, C_dev, N);
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -935,6 +945,7 @@ int spmm_run(spmm_handle_t h, const void* B_dev, void* C_dev, int64_t N, void* s
 }
 
 int spmm_bcsr_plan(spmm_handle_t h, int64_t N) {
+    NvtxRange nvtx_range("spmm_bcsr_plan");
     if (!h || N <= 0) return SPMM_ERR_INVALID_ARG;
     if (h->format != 0) return SPMM_ERR_INVALID_ARG;
     if (N < (h->col_major ? 128 : 64) || (!h->col_major && (N * h->es) % 16 != 0)) return SPMM_ERR_UNSUPPORTED;
@@ -942,6 +953,7 @@ int spmm_bcsr_plan(spmm_handle_t h, int64_t N) {
 }
 
 int spmm_wcsr_run_static(spmm_handle_t h, const void* B_dev, void* C_dev, int64_t N, void* stream) {
+    NvtxRange nvtx_range("spmm_wcsr_run_static");
     int rc = check_run_args(h, B_dev, C_dev, N);
     if (rc) return rc;
     if (h->format != 1) return SPMM_ERR_INVALID_ARG;
@@ -953,8 +965,14 @@ int spmm_wcsr_run_static(spmm_handle_t h, const void* B_dev, void* C_dev, int64_
 }
 
 int spmm_run_host(spmm_handle_t h, const void* B_host, void* C_host, int64_t N, void* stream) {
+    NvtxRange nvtx_range("spmm_run_host");
     if (!h || !B_host || !C_host || N <= 0) return SPMM_ERR_INVALID_ARG;
     if (h->host_only) return SPMM_ERR_HOST_ONLY;
+    {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess) return SPMM_ERR_CUDA;
+        if (dev != h->device) return SPMM_ERR_INVALID_ARG;
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t bbytes = static_cast<size_t>(h->k) * N * h->es;
     const size_t cbytes = static_cast<size_t>(h->m) * N * h->cs;
@@ -1054,7 +1072,8 @@ int spmm_check(spmm_handle_t h) {
     if (cudaMemcpy(st, h->d_status, sizeof(st), cudaMemcpyDeviceToHost) != cudaSuccess) return SPMM_ERR_CUDA;
     if (st[0] != 0) {
         cudaMemset(h->d_status, 0, sizeof(st));
-        return st[0] == 2 ? SPMM_ERR_DEV_BOUNDS : SPMM_ERR_DEV_TIMEOUT;
+        if (st[0] == 2) return SPMM_ERR_DEV_BOUNDS;
+        return st[3] != 0 ? SPMM_ERR_DEV_UNDRAINED : SPMM_ERR_DEV_TIMEOUT;
     }
     return SPMM_OK;
 }
@@ -1227,13 +1246,11 @@ const char* spmm_status_string(int code) {
         case SPMM_ERR_HOST_ONLY: return "handle was created host_only";
         case SPMM_ERR_TOO_LARGE: return "size exceeds a fixed capacity";
         case SPMM_ERR_DEV_BOUNDS: return "a kernel met an index outside its range";
+        case SPMM_ERR_DEV_UNDRAINED: return "a bounded wait inside a kernel ran out and so did the wait for its work in flight";
         default: return "unknown status";
     }
 }
 
-#ifdef SPMM_TRACE
-void spmm_debug_set_trace(long long* dev_buf) { g_trace = dev_buf; }
-#endif
 
 int spmm_set_wait_limit_ns(uint64_t ns) {
     g_wait_limit_ns.store(ns);

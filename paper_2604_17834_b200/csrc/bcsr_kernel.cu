@@ -15,27 +15,30 @@
 //               STAGES-deep shared-memory ring; full/empty mbarriers with phase bits.
 //   warp 1      MMA issuer: one thread issues tcgen05.mma into one of two TMEM accumulator
 //               buffers; tcgen05.commit frees the ring slot / publishes the accumulator.
-//   warps 2-5   epilogue: tcgen05.ld -> registers -> the warp's 2 KB staging tile in shared
-//               memory -> one TMA store per 16 (fp32) or 32 (16-bit) C rows x 32 tokens, which
-//               also clips at the edges of C (zeros for empty block-rows); overlaps the next
-//               tile's MMAs thanks to the second TMEM buffer.  Measured 2 - 6 % faster than
-//               st.global from registers, and far faster for 16-bit or column-major C.
+//   warps 2-5   epilogue: tcgen05.ld -> registers -> one of the warp's staging tiles in shared
+//               memory (up to 64 C rows x 32 tokens = 8 KB of fp32; a ring of 2 or more tiles
+//               per warp, so that the warp fills the next tile while earlier TMA stores are
+//               still reading theirs) -> one TMA store per tile, which also clips at the edges
+//               of C (zeros for empty block-rows); overlaps the next tile's MMAs thanks to the
+//               second TMEM buffer.
 // Two optional variants, both template parameters:
 //   CT = 1   C is written in the input's 16-bit type instead of fp32.
 //   CM = 1   "column-major" operands (the layout of the paper's BCSR kernel, Sec. 3.2, and of a
-//            linear layer Y = X W^T, Sec. 4.3): B is given as X[N][k] (one row per token, k
+//            linear layer Y = X W^T, Sec. 4.4): B is given as X[N][k] (one row per token, k
 //            contiguous) and C as Y[N][m].  The token tile is then a K-major MMA operand
 //            (rows of min(b, 64) elements, swizzle = row bytes; b = 128 as two K halves), and
 //            the staging tile is [32 tokens][16 or 32 columns of Y].
 //   DYN = 1  dynamic tile scheduling with Cluster Launch Control (the direction Sec. 5 points
 //            to after the paper's atomic-counter scheduler lost to the hardware block
-//            scheduler, Sec. 3.5): the grid has one CTA per tile, in the schedule's global order
+//            scheduler, Sec. 3.6): the grid has one CTA per tile, in the schedule's global order
 //            (slab by slab, longest block-row first); a CTA runs tile blockIdx.x and then
 //            keeps cancelling the launch of not-yet-started CTAs and running their tiles.  A
 //            seventh warp fetches the tile indices ahead of time into a four-deep ring that
 //            the six working warps read.
 // The host deals tiles to CTAs ahead of time: slab by slab (a slab = token tiles whose B rows
 // fit in L2), longest block-row first, each tile to the least loaded CTA; CTA c walks its list.
+#include <mutex>
+
 #include "kernels.h"
 #include "ptx.cuh"
 
@@ -43,13 +46,11 @@ namespace spmm {
 
 namespace {
 
-template <int B, int CT, int CM>
-struct EpiCols { static constexpr int value = bcsr_epi_cols(B, CT != 0, CM != 0); };
-
 // ES = bytes per input element: 2 (fp16 / bf16), or 1 (E4M3, column-major operands only).
 // H = rows of one stored block = the MMA's N extent: B for the format's own b x b blocks, 128 for
 // the stacked blocks of a row group (128 / b block-rows on top of one another, see format.h).
-template <int B, int H, int GROUPS, int STAGES, int ES>
+// CS = bytes per element of C, CM = column-major operands: they fix the epilogue's staging tile.
+template <int B, int H, int GROUPS, int STAGES, int ES, int CS, int CM>
 struct BcsrCfg {
     static constexpr int kBB = B * ES;                       // bytes of one block row (its K extent)
     static constexpr int kKSteps = kBB / 32;                 // MMAs per block and token group (32 bytes of K each)
@@ -71,9 +72,20 @@ struct BcsrCfg {
     static constexpr int kXGroupBytes = 128 * kXRowBytes;    // one K half of one token group
     static constexpr int kAccCols = GROUPS * H;
     static constexpr int kTmemCols = (2 * kAccCols <= 32) ? 32 : (2 * kAccCols <= 64 ? 64 : (2 * kAccCols <= 128 ? 128 : (2 * kAccCols <= 256 ? 256 : 512)));
-    static constexpr int kStagingBytes = 4 * 2048;           // one 2 KB tile per epilogue warp
     static constexpr int kBarrierBytes = 512;                // mbarriers, TMEM slot, flags, tile-index ring
+    // Epilogue staging: a tile is kEpiCols accumulator columns (rows of C) x 32 tokens.  Every
+    // epilogue warp owns a ring of kEpiBufs tiles: as many as fit beside the stage ring (the
+    // operand stream comes first: a deeper stage ring gains more than more staging), at most
+    // eight.  With more than one tile a warp fills the next tile while earlier TMA stores are
+    // still reading theirs.
+    static constexpr int kEpiCols = bcsr_epi_cols(B, CS == 2, CM != 0);
+    static constexpr int kEpiTileBytes = kEpiCols * 32 * CS;
+    static constexpr int kEpiRoom = (227 * 1024 - 1024 /*align*/ - kBarrierBytes - STAGES * kStageBytes) / (4 * kEpiTileBytes);
+    static constexpr int kEpiBufs = kEpiRoom < 8 ? kEpiRoom : 8;
+    static constexpr int kStagingBytes = 4 * kEpiBufs * kEpiTileBytes;
     static constexpr int kSmemBytes = STAGES * kStageBytes + kStagingBytes + 1024 /*align*/ + kBarrierBytes;
+    static_assert(kEpiBufs >= 1 && kEpiBufs <= 8, "no room for the epilogue's staging tiles");
+    static_assert(kEpiCols <= B && H % kEpiCols == 0, "a staging tile never straddles two block-rows");
     static_assert(2 * kAccCols <= 512, "accumulators exceed TMEM");
     static_assert(kSmemBytes <= 227 * 1024, "stage ring exceeds shared memory");
     static_assert((2 * STAGES + 7 + 8) * 8 + 64 <= kBarrierBytes, "barrier area");
@@ -81,6 +93,15 @@ struct BcsrCfg {
     static_assert(kBB % 32 == 0, "a block row must hold whole K steps");
     static_assert(H == B || (H == 128 && B < 128), "stacked blocks are 128 rows high");
 };
+
+// Ring depth for a shape: CAP stages, fewer where they would leave no room for one staging tile
+// per epilogue warp.
+template <int B, int H, int GROUPS, int CAP, int ES, int CS, int CM>
+constexpr int bcsr_fit_stages() {
+    using C1 = BcsrCfg<B, H, GROUPS, 1, ES, CS, CM>;
+    const int s = (227 * 1024 - 1024 - C1::kBarrierBytes - 4 * C1::kEpiTileBytes) / C1::kStageBytes;
+    return s > CAP ? CAP : (s < 2 ? 2 : s);
+}
 
 constexpr int kSchedDepth = 4;      // tile indices fetched ahead by the dynamic scheduler
 
@@ -91,7 +112,8 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     constexpr int ES = FMT == 3 ? 1 : 2;
     static_assert(ES == 2 || CM, "8-bit inputs: column-major operands only");
     static_assert(H == B || !DYN, "stacked blocks: static schedule only");
-    using Cfg = BcsrCfg<B, H, GROUPS, STAGES, ES>;
+    using CElem = typename CType<FMT, CT>::type;
+    using Cfg = BcsrCfg<B, H, GROUPS, STAGES, ES, static_cast<int>(sizeof(CElem)), CM>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -196,8 +218,6 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // A blocks and the B slab are re-read by other CTAs while the slab lasts: ask L2 to
             // keep them in preference to the C lines streaming through
             const uint64_t keep = l2_policy_evict_last();
-            TRACE_DECL(tr_empty);
-            TRACE_T0(tr_start);
             int4 tcd, tcd_next;
             int Jl_next = 0;                 // block columns of the next tile's first 32 blocks, fetched a tile ahead
             bool have_next = false;
@@ -222,9 +242,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         const int nb = min(Cfg::kBps, nq - jq);          // stored blocks in this stage
                         const int s = it % STAGES;
                         const uint32_t ph = (it / STAGES) & 1u;
-                        TRACE_T0(tr_a);
                         if (!__all_sync(0xffffffffu, mbar_wait(empty_bar(s), ph ^ 1u, ctl, 1))) { ok = false; break; }
-                        TRACE_ADD(tr_empty, tr_a);
                         const uint32_t sb = smem_base + s * Cfg::kStageBytes;
                         // the A request always brings kBps blocks (the box of the tensor map)
                         const uint32_t dense_tx = CM ? (whole_tile ? Cfg::kDenseBytes : ((nvalid + 127) >> 7) * (128 * Cfg::kBB))
@@ -278,18 +296,12 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
             }
             if (lane == 0) {
-                TRACE_PUT(0, clock64() - tr_start);
-                TRACE_PUT(1, tr_empty);
-                TRACE_PUT(3, (long long)it);
             }
             if (!ok && lane == 0) {
                 // leave no bulk copy in flight: wait (bounded) for the fills already issued
                 const uint32_t first = it > STAGES ? it - STAGES : 0;
-                for (uint32_t j = first; j < it; ++j) {
-                    const uint64_t t0 = globaltimer_ns();
-                    while (!mbar_try_wait(full_bar(j % STAGES), (j / STAGES) & 1u) &&
-                           globaltimer_ns() - t0 < 2000000ull) {}
-                }
+                for (uint32_t j = first; j < it; ++j)
+                    if (!mbar_drain_wait(full_bar(j % STAGES), (j / STAGES) & 1u, ctl, 21)) break;
             }
         }
     } else if (warp == 1) {
@@ -305,10 +317,6 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const bool leader = elect_one();
             uint32_t it = 0, tile_i = 0;
             bool ok = true;
-            TRACE_DECL(tr_full);
-            TRACE_DECL(tr_acce);
-            TRACE_DECL(tr_issue);
-            TRACE_T0(tr_start);
             int4 tcd, tcd_next;
             for (; ok && next_tile(tile_i, &tcd, &tcd_next, &ok); ++tile_i) {
                 const int n0 = tcd.y * Cfg::kBnT;
@@ -316,9 +324,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int ngrp = (nvalid + 127) >> 7;
                 const int acc = tile_i & 1;
                 const uint32_t aph = (tile_i >> 1) & 1u;
-                TRACE_T0(tr_a);
                 if (!__all_sync(0xffffffffu, mbar_wait(acce_bar(acc), aph ^ 1u, ctl, 2))) { ok = false; break; }
-                TRACE_ADD(tr_acce, tr_a);
                 tc_fence_after_sync();
                 const uint32_t d0 = tmem_base + acc * Cfg::kAccCols;
                 const int pb = tcd.z, pe = tcd.w;
@@ -327,11 +333,8 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const int nb = min(Cfg::kBps, min(pe - q, 32 - ((q - pb) & 31)));
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
-                    TRACE_T0(tr_b);
                     if (!__all_sync(0xffffffffu, mbar_wait(full_bar(s), ph, ctl, 3))) { ok = false; break; }
-                    TRACE_ADD(tr_full, tr_b);
                     tc_fence_after_sync();
-                    TRACE_T0(tr_c);
                     const uint32_t sb = smem_base + s * Cfg::kStageBytes;
 #pragma unroll
                     for (int i = 0; i < Cfg::kBps; ++i) {
@@ -355,7 +358,6 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         }
                     }
                     if (leader) tc_commit(empty_bar(s));
-                    TRACE_ADD(tr_issue, tr_c);
                 }
                 if (!ok) break;
                 if (leader) {
@@ -364,20 +366,15 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
             }
             if (lane == 0) {
-                TRACE_PUT(4, clock64() - tr_start);
-                TRACE_PUT(5, tr_full);
-                TRACE_PUT(6, tr_acce);
-                TRACE_PUT(7, (long long)it);
-                TRACE_PUT(12, tr_issue);
             }
         }
     } else if (warp < 6) {
         // ------------------------------------------------------------------ epilogue warps
         const int qd = warp & 3;                    // TMEM lane quarter this warp may read
         uint32_t tile_i = 0;
+        uint32_t chunk = 0;                         // staging tiles this warp has filled so far
+        const uint32_t stg0 = smem_base + STAGES * Cfg::kStageBytes + (warp - 2) * (Cfg::kEpiBufs * Cfg::kEpiTileBytes);
         bool ok = true;
-        TRACE_DECL(tr_accf);
-        TRACE_T0(tr_start);
         int4 tcd, tcd_next;
         for (; ok && next_tile(tile_i, &tcd, &tcd_next, &ok); ++tile_i) {
             const int tI = tcd.x;
@@ -390,83 +387,78 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // stacked blocks: the block-rows the group's 128 accumulator columns belong to
             int member = 0;
             if constexpr (H != B) member = lane < H / B ? __ldg(p.stack_rows + tI * (H / B) + lane) : 0;
-            TRACE_T0(tr_a);
             if (!__all_sync(0xffffffffu, mbar_wait(accf_bar(acc), aph, ctl, 4))) { ok = false; break; }
-            TRACE_ADD(tr_accf, tr_a);
             tc_fence_after_sync();
             const int64_t row0 = static_cast<int64_t>(tI) * B;
-            using CElem = typename CType<FMT, CT>::type;
-            constexpr int W = EpiCols<B, CT, CM>::value;    // accumulator columns per chunk
-            const uint32_t stg = smem_base + STAGES * Cfg::kStageBytes + (warp - 2) * 2048;
+            constexpr int W = Cfg::kEpiCols;                // accumulator columns per staging tile
             for (int g = 0; g < ngrp; ++g) {
                 const int nw = n0 + g * 128 + qd * 32;          // first token of this warp
                 if (nw >= N) break;                             // the whole warp is beyond the last token
-#pragma unroll
+#pragma unroll 1
                 for (int c0 = 0; c0 < H; c0 += W) {
                     uint32_t v[W];
                     if (has_blocks) {
                         const uint32_t ta = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) +
                                             acc * Cfg::kAccCols + g * H + c0;
-                        if constexpr (W == 16) tmem_ld_x16(ta, v);
-                        else tmem_ld_x32(ta, v);
+                        tmem_ld_cols<W>(ta, v);
                         tmem_ld_wait();
                     } else {
 #pragma unroll
                         for (int j = 0; j < W; ++j) v[j] = 0u;
                     }
-                    {
-                        // registers -> this warp's staging tile -> one TMA store.  The previous store
-                        // of this warp must have read the tile first.
-                        if (lane == 0) bulk_wait_all<true>();
-                        __syncwarp();
-                        if constexpr (!CM) {
-                            // tile [W rows][32 tokens], no swizzle: 64-byte rows of 2-byte elements
-                            // (or 128-byte rows of fp32)
+                    // registers -> the next tile of this warp's staging ring -> one TMA store.  The
+                    // store that used this tile kEpiBufs chunks ago must have read it first.
+                    const uint32_t stg = stg0 + (chunk % Cfg::kEpiBufs) * Cfg::kEpiTileBytes;
+                    ++chunk;
+                    if (lane == 0) bulk_wait_read<Cfg::kEpiBufs - 1>();
+                    __syncwarp();
+                    if constexpr (!CM) {
+                        // tile [W rows][32 tokens], no swizzle: 128-byte rows of fp32 (64-byte rows
+                        // of 2-byte elements); a warp's store covers one row, so no bank is hit twice
 #pragma unroll
-                            for (int j = 0; j < W; ++j) {
-                                if constexpr (sizeof(CElem) == 4) {
-                                    st_shared_u32(stg + j * 128 + lane * 4, v[j]);
-                                } else {
-                                    const CElem h = from_f32<CElem>(__uint_as_float(v[j]));
-                                    st_shared_u16(stg + j * 64 + lane * 2, *reinterpret_cast<const unsigned short*>(&h));
-                                }
-                            }
-                        } else {
-                            // tile [32 tokens][W elements]: this lane's row, in 16-byte chunks; 64-byte
-                            // rows are stored with the tensor map's 64-byte swizzle (chunk index XOR
-                            // (row / 2) % 4), which also keeps the warp's stores off each other's banks
-                            constexpr int kChunks = W * static_cast<int>(sizeof(CElem)) / 16;     // 2 or 4
-                            constexpr int kPer = 16 / static_cast<int>(sizeof(CElem));            // elements per chunk
-#pragma unroll
-                            for (int c = 0; c < kChunks; ++c) {
-                                uint32_t w4[4];
-                                if constexpr (sizeof(CElem) == 4) {
-#pragma unroll
-                                    for (int i = 0; i < 4; ++i) w4[i] = v[c * kPer + i];
-                                } else {
-#pragma unroll
-                                    for (int i = 0; i < 4; ++i) {
-                                        const CElem lo = from_f32<CElem>(__uint_as_float(v[c * kPer + 2 * i]));
-                                        const CElem hi = from_f32<CElem>(__uint_as_float(v[c * kPer + 2 * i + 1]));
-                                        w4[i] = static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(&lo)) |
-                                                (static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(&hi)) << 16);
-                                    }
-                                }
-                                const int cs = kChunks == 4 ? (c ^ ((lane >> 1) & 3)) : c;
-                                st_shared_v4(stg + lane * (kChunks * 16) + (cs << 4), w4[0], w4[1], w4[2], w4[3]);
+                        for (int j = 0; j < W; ++j) {
+                            if constexpr (sizeof(CElem) == 4) {
+                                st_shared_u32(stg + j * 128 + lane * 4, v[j]);
+                            } else {
+                                const CElem h = from_f32<CElem>(__uint_as_float(v[j]));
+                                st_shared_u16(stg + j * 64 + lane * 2, *reinterpret_cast<const unsigned short*>(&h));
                             }
                         }
-                        fence_proxy_async_smem();
-                        __syncwarp();
-                        int32_t crow = static_cast<int32_t>(row0) + c0;
-                        if constexpr (H != B) crow = __shfl_sync(0xffffffffu, member, c0 / B) * B + (c0 % B);
-                        if (lane == 0) {
-                            // row-major: box = 32 tokens x W rows at (token, row); column-major: box =
-                            // W columns x 32 tokens at (column, token).  Out-of-range parts are clipped.
-                            if constexpr (!CM) tma_store_2d(&tmC, stg, nw, crow);
-                            else tma_store_2d(&tmC, stg, crow, nw);
-                            bulk_commit_group();
+                    } else {
+                        // tile [32 tokens][W elements]: this lane's row, in 16-byte chunks; 64-byte
+                        // rows are stored with the tensor map's 64-byte swizzle (chunk index XOR
+                        // (row / 2) % 4), which also keeps the warp's stores off each other's banks
+                        constexpr int kChunks = W * static_cast<int>(sizeof(CElem)) / 16;     // 2 or 4
+                        constexpr int kPer = 16 / static_cast<int>(sizeof(CElem));            // elements per chunk
+#pragma unroll
+                        for (int c = 0; c < kChunks; ++c) {
+                            uint32_t w4[4];
+                            if constexpr (sizeof(CElem) == 4) {
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) w4[i] = v[c * kPer + i];
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    const CElem lo = from_f32<CElem>(__uint_as_float(v[c * kPer + 2 * i]));
+                                    const CElem hi = from_f32<CElem>(__uint_as_float(v[c * kPer + 2 * i + 1]));
+                                    w4[i] = static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(&lo)) |
+                                            (static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(&hi)) << 16);
+                                }
+                            }
+                            const int cs = kChunks == 4 ? (c ^ ((lane >> 1) & 3)) : c;
+                            st_shared_v4(stg + lane * (kChunks * 16) + (cs << 4), w4[0], w4[1], w4[2], w4[3]);
                         }
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    int32_t crow = static_cast<int32_t>(row0) + c0;
+                    if constexpr (H != B) crow = __shfl_sync(0xffffffffu, member, c0 / B) * B + (c0 % B);
+                    if (lane == 0) {
+                        // row-major: box = 32 tokens x W rows at (token, row); column-major: box =
+                        // W columns x 32 tokens at (column, token).  Out-of-range parts are clipped.
+                        if constexpr (!CM) tma_store_2d(&tmC, stg, nw, crow);
+                        else tma_store_2d(&tmC, stg, crow, nw);
+                        bulk_commit_group();
                     }
                 }
             }
@@ -475,14 +467,6 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (lane == 0) mbar_arrive(acce_bar(acc));
         }
         if (lane == 0) bulk_wait_all<false>();          // this warp's last stores have landed
-#ifdef SPMM_TRACE
-        if (warp == 2 && lane == 0) {
-            TRACE_PUT(8, clock64() - tr_start);
-            TRACE_PUT(9, tr_accf);
-            TRACE_PUT(10, (long long)tile_i);
-            TRACE_PUT(11, (long long)globaltimer_ns());
-        }
-#endif
     }
 
     if constexpr (DYN) {
@@ -499,8 +483,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (!mbar_wait(schf_bar(slot), use & 1u, ctl, 7)) {
                     // leaving early: the answer of the request just issued must still land in
                     // this CTA's shared memory before the CTA may exit (bounded)
-                    const uint64_t t0 = globaltimer_ns();
-                    while (!mbar_try_wait(schf_bar(slot), use & 1u) && globaltimer_ns() - t0 < 2000000ull) {}
+                    mbar_drain_wait(schf_bar(slot), use & 1u, ctl, 22);
                     break;
                 }
                 uint32_t x;
@@ -520,8 +503,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // slowed the normal path measurably)
             if (elect_one()) {
                 tc_commit(drain_bar);
-                const uint64_t t0 = globaltimer_ns();
-                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < 2000000ull) {}
+                mbar_drain_wait(drain_bar, 0, ctl, 23);
             }
             __syncwarp();
         }
@@ -530,16 +512,30 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
 }
 
-template <int B, int H, int GROUPS, int STAGES, int FMT, int CT, int CM, int DYN>
+// CAP = the deepest ring the shape is given; the ring actually used also leaves room for the
+// epilogue's staging tiles (bcsr_fit_stages).
+template <int B, int H, int GROUPS, int CAP, int FMT, int CT, int CM, int DYN>
 cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p,
                        int grid, cudaStream_t stream) {
-    using Cfg = BcsrCfg<B, H, GROUPS, STAGES, FMT == 3 ? 1 : 2>;
+    constexpr int ES = FMT == 3 ? 1 : 2;
+    constexpr int CS = static_cast<int>(sizeof(typename CType<FMT, CT>::type));
+    constexpr int STAGES = bcsr_fit_stages<B, H, GROUPS, CAP, ES, CS, CM>();
+    using Cfg = BcsrCfg<B, H, GROUPS, STAGES, ES, CS, CM>;
     auto kfn = bcsr_spmm_kernel<B, H, GROUPS, STAGES, FMT, CT, CM, DYN>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+    // the attribute belongs to the (function, device) pair: set it once per device
+    static std::mutex mu;
+    static bool attr_done[kMaxDevices] = {};
+    {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> lock(mu);
+        if (!attr_done[dev]) {
+            e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+            if (e != cudaSuccess) return e;
+            attr_done[dev] = true;
+        }
     }
     if (p.overlap == 2) {
         cudaLaunchConfig_t cfg = {};
@@ -628,7 +624,14 @@ cudaError_t launch_fmt(int b, int groups, int c16, int cm, int dyn, const CUtens
 
 }  // namespace
 
-int bcsr_token_groups_max(int b) { return b == 128 ? 2 : 4; }
+// Widest token tile per block size, in 128-token groups.  b = 64 with row-major fp32 C writes
+// the most bytes of C per staged operand byte: there a 256-token tile with five 40 KB stages and
+// three staging tiles per epilogue warp measured 3 % faster than 512 tokens with three 72 KB
+// stages and one staging tile; every other combination measured equal or slower with 256.
+int bcsr_token_groups_max(int b, int c16, int col_major) {
+    if (b == 128) return 2;
+    return (b == 64 && !c16 && !col_major) ? 2 : 4;
+}
 
 cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, int dynamic, const CUtensorMap& tmA,
                         const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p,

@@ -7,6 +7,9 @@
 
 namespace spmm {
 
+// per-device caches (kernel attributes, the built-in scratch address) are arrays of this length
+constexpr int kMaxDevices = 64;
+
 struct BcsrParams {
     const int32_t* block_row_ptr;
     const int32_t* block_col_idx;
@@ -16,7 +19,6 @@ struct BcsrParams {
     int64_t m, N;
     int* status;
     uint64_t wait_limit_ns;
-    long long* trace;   // tuning builds only (SPMM_TRACE); nullptr otherwise
     int32_t use_3d;     // tmB3 is valid: whole token tiles are fetched with one 3-D request
     // stacked launch only: [groups][128 / b] block-rows of every row group (see BcsrStack); the
     // tile records then name {group, token tile, first stacked block, end stacked block} and
@@ -47,10 +49,11 @@ constexpr int kStackGroups = 2;
 cudaError_t launch_bcsr_stacked(int dtype, int b, int c16, int col_major, const CUtensorMap& tmA, const CUtensorMap& tmB,
                                 const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p, int grid,
                                 cudaStream_t stream);
-int bcsr_token_groups_max(int b);
+int bcsr_token_groups_max(int b, int c16, int col_major);
 // Accumulator columns (= rows of A's block) an epilogue warp handles at a time: it stages them
-// in a 2 KB shared-memory tile and stores the tile with one TMA request whose box is 32 tokens x
-// this many rows (row-major C) or this many columns x 32 tokens (column-major Y).
+// in a 2 KB (1 KB for b = 16 with 16-bit C) shared-memory tile and stores the tile with one TMA
+// request whose box is 32 tokens x this many rows (row-major C) or this many columns x 32 tokens
+// (column-major Y).  Larger tiles (up to 64 rows) were measured slower: the stage ring needs the room.
 constexpr int bcsr_epi_cols(int b, bool c16, bool col_major) { return (b < 32 || !c16) ? 16 : 32; }
 // stored blocks that share one pipeline stage (and one A request): 4 / 2 for b = 16 / 32
 constexpr int bcsr_blocks_per_stage(int b) { return b == 16 ? 4 : (b == 32 ? 2 : 1); }
@@ -100,7 +103,6 @@ struct WcsrParams {
     int32_t n_tt;                // token tiles = ceil(N / (128 * groups))
     int* status;
     uint64_t wait_limit_ns;
-    long long* trace;            // tuning builds only (SPMM_TRACE); nullptr otherwise
 };
 
 // dtype: 0 bf16, 1 fp16, 2 tf32.  groups: 1 or 2.  tmB: 2-D map of B (k rows x N), box = 128

@@ -12,20 +12,6 @@
 
 namespace spmm {
 
-// Optional per-CTA cycle accounting for kernel tuning (compiled out unless SPMM_TRACE is
-// defined; the buffer is the params' trace pointer, 16 counters per CTA).
-#ifdef SPMM_TRACE
-#define TRACE_DECL(name) long long name = 0
-#define TRACE_T0(t) const long long t = clock64()
-#define TRACE_ADD(acc, t) acc += clock64() - t
-#define TRACE_PUT(slot, val) do { if (p.trace) p.trace[blockIdx.x * 16 + (slot)] = (val); } while (0)
-#else
-#define TRACE_DECL(name)
-#define TRACE_T0(t)
-#define TRACE_ADD(acc, t)
-#define TRACE_PUT(slot, val)
-#endif
-
 // ----------------------------------------------------------------------------- misc
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -108,7 +94,8 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // Shared by every role of a CTA: where a bounded wait reports that it ran out.
 struct WaitCtl {
     volatile int* abort_flag;   // shared memory: set once any wait of the CTA ran out
-    int* status;                // global: [0] = code (0 ok, 1 timeout), [1] = site, [2] = block
+    int* status;                // global: [0] = code (0 ok, 1 timeout, 2 bounds), [1] = site, [2] = block,
+                                // [3] = site of a teardown wait that ran out as well (0: none)
     uint64_t limit_ns;
 };
 
@@ -137,6 +124,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
             }
         }
     }
+}
+
+// Teardown wait of the abort path, for copies or MMAs the CTA has already issued: they must land
+// before the CTA gives up its shared memory and TMEM.  Bounded by the configured limit (2 ms at
+// least, so that the zero-limit test hook still lets work in flight finish); if even that runs
+// out, status[3] records where: the CTA then leaves with work possibly still in flight.
+__device__ __forceinline__ bool mbar_drain_wait(uint32_t bar, uint32_t parity, const WaitCtl& ctl, int site) {
+    const uint64_t limit = ctl.limit_ns > 2000000ull ? ctl.limit_ns : 2000000ull;
+    const uint64_t t0 = globaltimer_ns();
+    while (!mbar_try_wait(bar, parity)) {
+        if (globaltimer_ns() - t0 > limit) {
+            atomicExch(ctl.status + 3, site);
+            return false;
+        }
+    }
+    return true;
 }
 
 // ----------------------------------------------------------------------------- fences
@@ -221,12 +224,27 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, uint32_t src,
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                  ::"l"(reinterpret_cast<uint64_t>(m)), "r"(src), "r"(x), "r"(y) : "memory");
 }
+// the same with an L2 cache-policy operand
+__device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* m, uint32_t src, int32_t x, int32_t y, uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(src), "r"(x), "r"(y), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // wait until the issuing thread's bulk groups have read their source (kRead) / completed
 template <bool kRead>
 __device__ __forceinline__ void bulk_wait_all() {
     if constexpr (kRead) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
     else asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+// wait until all but the kPending most recent bulk groups of the issuing thread have read their source
+template <int kPending>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kPending) : "memory");
 }
 
 // 1-D bulk copy global -> shared; both addresses 16-byte aligned, bytes % 16 == 0.
@@ -305,6 +323,20 @@ __device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr)
         : "memory");
+}
+
+// kCols = 16, 32 or 64 consecutive columns (64: two loads of 32, one wait by the caller).
+template <int kCols>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[kCols]) {
+    static_assert(kCols == 16 || kCols == 32 || kCols == 64, "16, 32 or 64 columns");
+    if constexpr (kCols == 16) {
+        tmem_ld_x16(taddr, r);
+    } else if constexpr (kCols == 32) {
+        tmem_ld_x32(taddr, r);
+    } else {
+        tmem_ld_x32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+        tmem_ld_x32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+    }
 }
 
 // ----------------------------------------------------------------------------- tcgen05.mma

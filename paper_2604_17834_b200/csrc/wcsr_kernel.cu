@@ -163,7 +163,8 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
             SegIter seg;
             seg.init();
             uint32_t it0 = 0, last_it = 0;
-            bool issued_any = false, ok = true;
+            uint32_t n_issued = 0;                       // fills this warp has issued
+            bool ok = true;
             int idx_cur[kIdxRegs], idx_nxt[kIdxRegs];
             bool idx_ready = false;
             while (ok && seg.next(p)) {
@@ -197,7 +198,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                             bulk_load_1d(sb + Cfg::kDenseBytes,
                                          p.packed + static_cast<size_t>(q / Cfg::kKStep) * (kWH * 32), abytes, full_bar(s));
                         }
-                        issued_any = true;
+                        ++n_issued;
                         last_it = it;
 #pragma unroll
                         for (int i = 0; i < kIssues; ++i) {
@@ -234,10 +235,13 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                 it0 += static_cast<uint32_t>(f1 - f0);
             }
             cp_async_wait<0>();
-            if (!ok && lane == 0 && issued_any) {
-                const uint64_t t0 = globaltimer_ns();
-                while (!mbar_try_wait(full_bar(last_it % STAGES), (last_it / STAGES) & 1u) &&
-                       globaltimer_ns() - t0 < 2000000ull) {}
+            if (!ok && lane == 0) {
+                // abort path: the bulk copies of the fills this warp issued last (one per stage it
+                // owns) may still be in flight
+                for (uint32_t k = 0; k < static_cast<uint32_t>(STAGES / PW) && k < n_issued; ++k) {
+                    const uint32_t j = last_it - k * kProducerWarps;
+                    if (!mbar_drain_wait(full_bar(j % STAGES), (j / STAGES) & 1u, ctl, 31)) break;
+                }
             }
         }
     } else if (warp < kProducerWarps) {
@@ -254,16 +258,12 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
             }
         };
 
-        TRACE_DECL(tr_empty);
-        TRACE_DECL(tr_copy);
-        TRACE_DECL(tr_issue_p);
-        TRACE_DECL(tr_fills);
-        TRACE_T0(tr_start);
         SegIter seg;
         seg.init();
         uint32_t it0 = 0;                            // CTA-wide number of fills before this segment
         uint32_t last_it = 0;
-        bool issued_any = false, ok = true;
+        uint32_t n_issued = 0;                       // fills this warp has issued
+        bool ok = true;
         // column indices of this warp's current fill and of its next two fills (requested two
         // fills ahead, so their latency never sits in the issue loop)
         int4 idx_cur[Cfg::kRounds], idx_n1[Cfg::kRounds], idx_n2[Cfg::kRounds];
@@ -299,11 +299,8 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     const uint32_t ph = (it / STAGES) & 1u;
                     const int q = d.x;
                     const int cnt = d.y & 0xFFFF;
-                    TRACE_T0(tr_a);
                     if (!__all_sync(0xffffffffu, mbar_wait(empty_bar(s), ph ^ 1u, ctl, 11))) { ok = false; break; }
-                    TRACE_ADD(tr_empty, tr_a);
                     const uint32_t sb = smem_base + s * Cfg::kStageBytes;
-                    TRACE_T0(tr_e);
                     if (lane == 0) {
                         const uint32_t abytes = (cnt / Cfg::kKStep) * (kWH * 32);
                         mbar_arrive_expect_tx(full_bar(s), abytes + (cnt / 4) * nseg * 512);
@@ -311,7 +308,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                                      p.packed + static_cast<size_t>(q / Cfg::kKStep) * (kWH * 32), abytes, full_bar(s));
                     }
                     __syncwarp();
-                    issued_any = true;
+                    ++n_issued;
                     last_it = it;
 #pragma unroll
                     for (int r = 0; r < Cfg::kRounds; ++r) {
@@ -321,10 +318,6 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                             tma_gather4_2d(sb + sg * Cfg::kAtomStride + rg * 512, &tmB, full_bar(s),
                                            n0 + sg * (128 / ES), idx_cur[r].x, idx_cur[r].y, idx_cur[r].z, idx_cur[r].w);
                     }
-                    TRACE_ADD(tr_issue_p, tr_e);
-#ifdef SPMM_TRACE
-                    ++tr_fills;
-#endif
 #pragma unroll
                     for (int r = 0; r < Cfg::kRounds; ++r) {
                         idx_cur[r] = idx_n1[r];
@@ -337,20 +330,12 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
             }
             it0 += static_cast<uint32_t>(f1 - f0);
         }
-#ifdef SPMM_TRACE
-        if (warp == 0 && lane == 0) {
-            TRACE_PUT(0, clock64() - tr_start);
-            TRACE_PUT(1, tr_empty);
-            TRACE_PUT(2, tr_copy);
-            TRACE_PUT(3, tr_fills);
-            TRACE_PUT(14, tr_issue_p);
-        }
-#endif
-        if (!ok && lane == 0 && issued_any) {
-            // abort path: this warp's last fill may still be in flight
-            const uint64_t t0 = globaltimer_ns();
-            while (!mbar_try_wait(full_bar(last_it % STAGES), (last_it / STAGES) & 1u) &&
-                   globaltimer_ns() - t0 < 2000000ull) {}
+        if (!ok && lane == 0) {
+            // abort path: the fills this warp issued last (one per stage it owns) may still be in flight
+            for (uint32_t k = 0; k < static_cast<uint32_t>(STAGES / PW) && k < n_issued; ++k) {
+                const uint32_t j = last_it - k * kProducerWarps;
+                if (!mbar_drain_wait(full_bar(j % STAGES), (j / STAGES) & 1u, ctl, 32)) break;
+            }
         }
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issuer
@@ -363,11 +348,6 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
         const uint64_t adesc0 = make_smem_desc(0, NARROW ? 0 : Cfg::kAtomStride, ES == 2 ? 1024 : 512, ES == 2 ? SWZ_128B : SWZ_128B_BASE32B);
         const uint64_t bdesc0 = make_smem_desc(0, kWH * 16, 128, SWZ_NONE);
         const bool leader = elect_one();
-        TRACE_DECL(tr_full);
-        TRACE_DECL(tr_acce);
-        TRACE_DECL(tr_issue);
-        TRACE_DECL(tr_commit);
-        TRACE_T0(tr_start);
         SegIter seg;
         seg.init();
         uint32_t it = 0, item = 0, d0 = 0;
@@ -389,21 +369,16 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     if (first) {
                         acc = item % Cfg::kNAcc;
                         const uint32_t aph = (item / Cfg::kNAcc) & 1u;
-                        TRACE_T0(tr_a);
                         ok = __all_sync(0xffffffffu, mbar_wait(acce_bar(acc), aph ^ 1u, ctl, 12));
-                        TRACE_ADD(tr_acce, tr_a);
                         tc_fence_after_sync();
                         d0 = tmem_base + acc * Cfg::kAccCols;
                         fresh = true;
                     }
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
-                    TRACE_T0(tr_b);
                     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(full_bar(s), ph, ctl, 13));
-                    TRACE_ADD(tr_full, tr_b);
                     if (ok) {
                         tc_fence_after_sync();
-                        TRACE_T0(tr_c);
                         const uint32_t sb = smem_base + s * Cfg::kStageBytes;
                         const int nks = cnt / Cfg::kKStep;
                         // descriptors differ only in their start-address field (bytes >> 4)
@@ -428,7 +403,6 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                             if (last) tc_commit(accf_bar(acc));
                         }
                         __syncwarp();
-                        TRACE_ADD(tr_issue, tr_c);
                     }
                     if (last) ++item;
                     if (!ok) break;
@@ -436,21 +410,9 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                 win = nwin;
             }
         }
-#ifdef SPMM_TRACE
-        if (lane == 0) {
-            TRACE_PUT(4, clock64() - tr_start);
-            TRACE_PUT(5, tr_full);
-            TRACE_PUT(6, tr_acce);
-            TRACE_PUT(7, (long long)it);
-            TRACE_PUT(12, tr_issue);
-            TRACE_PUT(13, tr_commit);
-        }
-#endif
     } else {
         // ------------------------------------------------------------------ epilogue warps
         const int qd = warp & 3;
-        TRACE_DECL(tr_accf);
-        TRACE_T0(tr_start);
         SegIter seg;
         seg.init();
         uint32_t item = 0;
@@ -484,9 +446,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     }
                     const int acc = item % Cfg::kNAcc;
                     const uint32_t aph = (item / Cfg::kNAcc) & 1u;
-                    TRACE_T0(tr_a);
                     if (!__all_sync(0xffffffffu, mbar_wait(accf_bar(acc), aph, ctl, 14))) { ok = false; break; }
-                    TRACE_ADD(tr_accf, tr_a);
                     tc_fence_after_sync();
                     float v[kWH];
                     const uint32_t tbase = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + acc * Cfg::kAccCols;
@@ -517,14 +477,6 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                 win = nwin;
             }
         }
-#ifdef SPMM_TRACE
-        if (warp == kMmaWarp + 1 && lane == 0) {
-            TRACE_PUT(8, clock64() - tr_start);
-            TRACE_PUT(9, tr_accf);
-            TRACE_PUT(10, (long long)item);
-            TRACE_PUT(11, (long long)globaltimer_ns());
-        }
-#endif
     }
 
     tc_fence_before_sync();
@@ -536,8 +488,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
             // slowed the normal path measurably)
             if (elect_one()) {
                 tc_commit(drain_bar);
-                const uint64_t t0 = globaltimer_ns();
-                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < 2000000ull) {}
+                mbar_drain_wait(drain_bar, 0, ctl, 33);
             }
             __syncwarp();
         }
@@ -587,18 +538,27 @@ cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cud
     constexpr int STAGES = wcsr_stages(ES, WH), PW = wcsr_producer_warps(ES, WH);
     using Cfg = WcsrCfg<ES, WH, KT, STAGES, NARROW>;
     auto kfn = wcsr_spmm_kernel<ES, FMT, WH, KT, STAGES, PW, CT, NARROW, LSU>;
-    static int occ = 0;
-    if (occ == 0) {
-        cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+    // resident CTAs per SM: shared memory and TMEM columns are checked in WcsrCfg; the
+    // register file follows from __launch_bounds__
+    static_assert(Cfg::kCtasPerSm * Cfg::kTmemCols <= 512, "TMEM over-subscribed");
+    // the attributes belong to the (function, device) pair: set them once per device
+    static std::mutex mu;
+    static bool attr_done[kMaxDevices] = {};
+    {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(kfn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return e;
-        // resident CTAs per SM: shared memory and TMEM columns are checked in WcsrCfg; the
-        // register file follows from __launch_bounds__
-        static_assert(Cfg::kCtasPerSm * Cfg::kTmemCols <= 512, "TMEM over-subscribed");
-        occ = Cfg::kCtasPerSm;
+        if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> lock(mu);
+        if (!attr_done[dev]) {
+            e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+            if (e != cudaSuccess) return e;
+            e = cudaFuncSetAttribute(kfn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+            if (e != cudaSuccess) return e;
+            attr_done[dev] = true;
+        }
     }
-    int grid = sms * occ;
+    int grid = sms * Cfg::kCtasPerSm;
     if (grid > p.n_bins) grid = p.n_bins;
     if (grid < 1) return cudaSuccess;
     kfn<<<grid, (PW + 5) * 32, Cfg::kSmemBytes, stream>>>(tmB, p);
@@ -644,7 +604,6 @@ static __device__ __align__(256) float g_static_scratch[kStaticScratchBytes / si
 cudaError_t wcsr_static_scratch(float** ptr, size_t* bytes) {
     // In host code the array's name is only a stand-in for the device symbol, never a
     // device address: resolve it once per device, with that device current.
-    constexpr int kMaxDevices = 64;
     static float* resolved[kMaxDevices] = {};
     static std::mutex mu;
     int dev = 0;

@@ -4,7 +4,8 @@ bench.py launches them (spmm_run on device-resident operands).
 Where the oracle cannot afford every output, all rows are checked on a seeded subset of
 columns: the columns of C are independent of one another (C[:, j] depends on B[:, j] only,
 pinned in tests/test_oracle_spmm.py), and the subset covers the first, an interior and the
-last position of a token tile, a tile boundary, and the ragged end of N.
+last position of a token tile, a tile boundary, the ragged end of N, and at least one column
+of every 128-column group, hence of every token tile the launch computes.
 """
 import numpy as np
 import pytest
@@ -23,9 +24,14 @@ def lib():
 
 
 def _sample_cols(N, seed):
+    """Fixed positions (tile edges, the ragged end) plus one seeded column inside EVERY group of
+    128 columns: whatever the kernel's token tile (128, 256 or 512 columns) and L2 slab, each
+    tile of the launch holds at least one column the oracle checks."""
     fixed = [0, 1, 31, 32, 63, 64, 127, 128, 129, 255, 256, 511, 512, 513, N // 2, N - 129, N - 128, N - 65, N - 2, N - 1]
     rng = np.random.default_rng(seed)
-    cols = set(c for c in fixed if 0 <= c < N) | set(rng.integers(0, N, size=44).tolist())
+    groups = np.arange(0, N, 128, dtype=np.int64)
+    per_group = np.minimum(groups + rng.integers(0, 128, size=groups.shape[0]), N - 1)
+    cols = set(c for c in fixed if 0 <= c < N) | set(per_group.tolist())
     return np.array(sorted(cols), dtype=np.int64)
 
 
@@ -98,7 +104,7 @@ def test_config2_bcsr_llm_full(lib, shape):
                                                   ("down", True, True)])
 def test_config2_bcsr_llm_variants_full(lib, shape, c16, col_major):
     """configs[2] with C in bf16 and / or column-major operands (the linear-layer shape of
-    Sec. 4.3: X [65536][k] in, Y [65536][m] out), as bench.py launches them."""
+    Sec. 4.4: X [65536][k] in, Y [65536][m] out), as bench.py launches them."""
     a = wl.bcsr_llm() if shape == "gate" else wl.bcsr_llm(seed=1013, m=3584, k=18944)
     N = 65536
     Bs = wl.dense(1103, a["k"], N, ("normal", 0.0, 1.0), "bf16")
@@ -134,7 +140,8 @@ def test_config4_wcsr_rmat_full(lib, rmat_full, N):
     """configs[4]: R-MAT 2^21 x 2^21, ~32.4 M nnz, fp16, N = 32 / 128 / 256."""
     a = rmat_full
     Bs = wl.dense(1105 + N, a["k"], N, ("normal", 0.0, 1.0), "fp16")
-    cols = _sample_cols(N, N)[::3] if N > 32 else np.arange(0, 32, 3)
+    # a third of the sampled positions, and in any case one column of every 128-column token tile
+    cols = np.unique(np.concatenate([_sample_cols(N, N)[::3], np.arange(5, N, 128)])) if N > 32 else np.arange(0, 32, 3)
     _run_and_check(lib, "wcsr", a, "fp16", 16, N, Bs, cols=cols, what="configs[4] N=%d" % N)
 
 

@@ -1,6 +1,6 @@
 """GPU parity of the output-type and operand-layout variants: C in the input's 16-bit type
 (BCSR and WCSR) and column-major operands (BCSR: X = B^T in, Y = C^T out, the layout of the
-paper's BCSR kernel, Sec. 3.2, and of a sparse linear layer, Sec. 4.3).  Same oracle, same
+paper's BCSR kernel, Sec. 3.2, and of a sparse linear layer, Sec. 4.4).  Same oracle, same
 bound as the default path: a 16-bit C adds at most 2^-9 |C| <= 2^-9 sum|a b| of rounding.
 """
 import numpy as np

@@ -356,3 +356,18 @@ def test_binding_structs_match_the_header(lib, tmp_path):
     subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(root, "include"), str(src), "-o", str(exe)], check=True)
     so, si = (int(x) for x in subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split())
     assert so == ctypes.sizeof(lib.SpmmOpts) and si == ctypes.sizeof(lib.SpmmInfo)
+
+
+def test_bcsr_row_major_needs_at_least_64_columns(lib):
+    """The documented minimum: a BCSR handle with row-major operands refuses N < 64 (the plan
+    call tells without a GPU); N = 64 is planned."""
+    a = wl.bcsr_tiny()
+    h = lib.spmm_bcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "bf16", 64, host_only=True)
+    try:
+        with pytest.raises(lib.SpmmError) as e:
+            lib.spmm_bcsr_plan(h, 32)
+        assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
+        lib.spmm_bcsr_plan(h, 64)
+        assert lib.spmm_get_info(h, 64)["plan_n"] == 64
+    finally:
+        lib.spmm_destroy(h)

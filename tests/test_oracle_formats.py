@@ -86,6 +86,8 @@ def test_bcsr_matches_brute_force_and_round_trips(m, k, dens, b):
         mask[I * b:(I + 1) * b, J * b:(J + 1) * b].any()
         for I in range(-(-m // b)) for J in range(-(-k // b)))
     assert len(idx) <= nb
+    # the count-only helper agrees with the bitmap brute force
+    assert F.bcsr_block_count(m, k, a["row_ptr"], a["col_idx"], b) == len(idx)
 
 
 def test_bcsr_structural_zero_keeps_block():
@@ -136,6 +138,8 @@ def test_wcsr_matches_brute_force_and_round_trips(m, k, dens, wh, b_col):
         assert np.all(np.diff(c) > 0)                         # strictly ascending
     back = F.wcsr_to_dense(m, k, wh, f["window_row_ptr"], f["window_col_idx"], f["values"])
     assert np.array_equal(back.view(np.uint16), D.view(np.uint16))
+    # the count-only helper agrees with the per-element construction
+    assert F.wcsr_padded_cols(m, k, a["row_ptr"], a["col_idx"], wh, b_col) == len(idx)
 
 
 def test_wcsr_height_one_is_padded_csr():
@@ -196,6 +200,77 @@ def test_split_plan(T):
         assert rows[0, 1] == 0
         assert np.all(rows[1:, 1] == rows[:-1, 1] + rows[:-1, 2])
         assert rows[-1, 1] + rows[-1, 2] == lens[w]
+
+
+def _brute_bins(plan, n_bins, fixed_cost=32):
+    """The longest-processing-time rule with plain loops: heaviest task first (ties: lower task
+    index), each into the bin with the smallest load so far (ties: lowest bin index)."""
+    order = sorted(range(len(plan)), key=lambda t: (-int(plan[t][2]), t))
+    loads = [0] * n_bins
+    members = [[] for _ in range(n_bins)]
+    for t in order:
+        b = min(range(n_bins), key=lambda j: (loads[j], j))
+        members[b].append(t)
+        loads[b] += int(plan[t][2]) + fixed_cost
+    return members, loads
+
+
+@pytest.mark.parametrize("seed,n_bins", [(1, 1), (2, 3), (3, 7), (4, 16), (5, 5)])
+def test_task_bins_match_brute_force(seed, n_bins):
+    rng = np.random.default_rng(seed)
+    # many equal lengths on purpose: the tie rules decide most placements
+    lens = rng.choice([0, 8, 8, 16, 16, 16, 64, 72, 200, 1000], size=80)
+    wptr = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    plan = F.split_plan(wptr, 64)
+    bin_ptr, bin_tasks = F.task_bins(plan, n_bins)
+    members, loads = _brute_bins(plan.tolist(), n_bins)
+    assert bin_ptr.tolist() == np.concatenate([[0], np.cumsum([len(x) for x in members])]).tolist()
+    assert bin_tasks.tolist() == [t for x in members for t in sorted(x)]
+    # every task once; the classical bound of the rule: no bin exceeds the mean by more than one task
+    assert sorted(bin_tasks.tolist()) == list(range(plan.shape[0]))
+    cost = plan[:, 2].astype(np.int64) + 32
+    assert max(loads) <= cost.sum() / n_bins + cost.max()
+
+
+def _brute_split_size(wptr, n_bins, fixed_cost=32):
+    """Default sub-task size written out with plain loops only (no call into the oracle's plan or
+    bins): the four candidates, each window cut into chunks, chunks dealt heaviest first."""
+    lens = [int(wptr[i + 1] - wptr[i]) for i in range(len(wptr) - 1)]
+    P = sum(lens)
+    cands = [min(65536, max(128, ((P // n_bins) >> i) // 64 * 64)) for i in range(4)]
+    worst = []
+    for T in cands:
+        chunks = []
+        for L in lens:
+            q = 0
+            while q < L:
+                chunks.append(min(T, L - q))
+                q += T
+        chunks.sort(reverse=True)
+        loads = [0] * n_bins
+        for c in chunks:
+            j = min(range(n_bins), key=lambda b: (loads[b], b))
+            loads[j] += c + fixed_cost
+        worst.append(max(loads))
+    best = min(worst)
+    for T, l in zip(cands, worst):
+        if l * 100 <= best * 102:
+            return T
+    return cands[3]
+
+
+@pytest.mark.parametrize("seed,n_bins", [(11, 4), (12, 9), (13, 16)])
+def test_default_split_cols_matches_plain_loops(seed, n_bins):
+    rng = np.random.default_rng(seed)
+    lens = rng.choice([0, 16, 32, 48, 64, 320, 2048, 9000], size=300, p=[.1, .3, .2, .15, .1, .1, .04, .01])
+    wptr = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    assert F.default_split_cols(wptr, n_bins) == _brute_split_size(wptr, n_bins)
+    # closed-form cases: one heavy window among light ones balances at a whole share; equal heavy
+    # windows, one more than bins, need a smaller size than the share
+    wp = np.concatenate(([0], np.cumsum([10000] + [64] * 1000)))
+    assert F.default_split_cols(wp, 8) == _brute_split_size(wp, 8) == (74000 // 8) // 64 * 64
+    wp = np.concatenate(([0], np.cumsum([4096] * 9)))
+    assert F.default_split_cols(wp, 8) == _brute_split_size(wp, 8) < 4608
 
 
 def test_generators_are_deterministic_and_shaped():

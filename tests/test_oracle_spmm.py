@@ -148,3 +148,27 @@ def test_e4m3_storage_matches_an_independent_conversion():
     assert wl.widen(wl.to_storage(np.array([1e6, -1e6], np.float32), "fp8"), "fp8").tolist() == [448.0, -448.0]
     z = wl.to_storage(np.array([-0.0], np.float32), "fp8")
     assert z[0] == 0x80 and np.signbit(wl.widen(z, "fp8"))[0]
+
+
+def test_bf16_and_fp16_storage_match_independent_conversions():
+    """The 16-bit quantisers of the input generators (round to nearest, ties to even) and their
+    exact widening against torch's casts: normal values, ties, subnormals of bf16, large values."""
+    import torch
+    rng = np.random.default_rng(13)
+    x = np.concatenate([rng.standard_normal(100000).astype(np.float32) * 2.0,
+                        rng.standard_normal(20000).astype(np.float32) * 1e-3,
+                        rng.standard_normal(2000).astype(np.float32) * 1e-40,       # subnormal in bf16 and fp32
+                        np.array([0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.0e38, -3.0e38, 65504.0, 2.0 ** -24], np.float32)])
+    t = torch.from_numpy(x)
+    b = wl.to_storage(x, "bf16")
+    assert b.dtype == np.uint16
+    assert np.array_equal(b, t.to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16))
+    assert np.array_equal(wl.widen(b, "bf16"), t.to(torch.bfloat16).to(torch.float64).numpy())
+    xh = x[np.abs(x) < 60000.0]
+    h = wl.to_storage(xh, "fp16")
+    th = torch.from_numpy(xh).to(torch.float16)
+    assert np.array_equal(h.view(np.uint16), th.view(torch.int16).numpy().view(np.uint16))
+    assert np.array_equal(wl.widen(h, "fp16"), th.to(torch.float64).numpy())
+    # the tie cases by hand: 1 + 2^-8 is halfway between two bf16 values -> the even one (1.0);
+    # 1 + 3 * 2^-8 is halfway as well -> the even one above (1 + 2^-6)
+    assert wl.widen(wl.to_storage(np.array([1.00390625, 1.01171875], np.float32), "bf16"), "bf16").tolist() == [1.0, 1.015625]
