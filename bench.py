@@ -144,6 +144,15 @@ def workload_table():
             w["opts"] = dict(w.get("opts", {}), gather=1)
             return w
         return f
+    def tf32_sweep(b, d):
+        """configs[3] shape in the value type of the paper's own BCSR evaluation (Sec. 4.1: TF32)."""
+        def f():
+            return dict(kind="bcsr", a=wl.bcsr_sweep(1004 + b + int(d * 1000), b=b, density=d, dtype="tf32"), dtype="tf32",
+                        size=b, N=4096, Bdist=("uniform", -1.0, 1.0))
+        return f
+    for b in (16, 32, 64, 128):
+        t["cfg4_bcsr_sweep_b%d_d0.1_tf32" % b] = ("configs[3] shape, b=%d skewed rows, keep 0.1, fp32 storage / TF32 arithmetic" % b,
+                                                   tf32_sweep(b, 0.1))
     t["cfg2_wcsr_irregular_lsu_gather"] = ("configs[1], B rows gathered with 16-byte cp.async instead of TMA", lsu(cfg2))
     t["cfg5_wcsr_rmat_n128_lsu_gather"] = ("configs[4] N=128, B rows gathered with 16-byte cp.async instead of TMA", lsu(cfg5(128)))
     t["cfg2_wcsr_irregular_wh64"] = ("configs[1] with 64-row windows", tall(cfg2))
@@ -181,7 +190,8 @@ ALL_OTHERS = DEFAULT_OTHERS + [
     "cfg3_bcsr_llm_gate_cm_fp8", "cfg3_bcsr_llm_down_cm_fp8", "cfg2_wcsr_irregular_wh64", "cfg5_wcsr_rmat_n128_wh64",
     "cfg2_wcsr_irregular_lsu_gather", "cfg5_wcsr_rmat_n128_lsu_gather",
     "cfg4_bcsr_sweep_b64_d0.1_dyn", "cfg4_bcsr_sweep_b16_d0.1_plain", "cfg4_bcsr_sweep_b32_d0.1_plain",
-    "cfg4_bcsr_sweep_b16_d0.5", "cfg4_bcsr_sweep_b32_d0.5"]
+    "cfg4_bcsr_sweep_b16_d0.5", "cfg4_bcsr_sweep_b32_d0.5",
+    "cfg4_bcsr_sweep_b16_d0.1_tf32", "cfg4_bcsr_sweep_b32_d0.1_tf32", "cfg4_bcsr_sweep_b64_d0.1_tf32", "cfg4_bcsr_sweep_b128_d0.1_tf32"]
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures whose
 # summaries are under profiles/ (absent where no capture of that exact launch exists).

@@ -64,7 +64,11 @@ typedef enum {
 typedef enum {
     SPMM_BF16 = 0,               /* 2-byte bfloat16 storage                                   */
     SPMM_FP16 = 1,               /* 2-byte IEEE half storage                                  */
-    SPMM_TF32 = 2,               /* 4-byte fp32 storage, TF32 tensor-core arithmetic          */
+    SPMM_TF32 = 2,               /* 4-byte fp32 storage, TF32 tensor-core arithmetic (the
+                                    k8 instruction shape of Sec. 3.1; Sec. 4.1 evaluates both
+                                    formats in it).  WCSR, and BCSR with every block size and
+                                    both layouts; C is fp32, the BCSR schedule static, and
+                                    BCSR row groups are not formed.                           */
     SPMM_FP8_E4M3 = 3            /* 1-byte E4M3 storage (Sec. 5 names 8-bit inputs as the next
                                     step).  BCSR with SPMM_COLMAJOR only, fp32 C, block 32,
                                     64 or 128, k % 16 == 0.                                   */

@@ -49,18 +49,23 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-// 2-D row-major tensor [rows][cols] of 16-bit (or, for E4M3, 8-bit) elements, box [box_rows][box_cols].
-int encode_2d_16bit(CUtensorMap* map, int dtype, const void* base, uint64_t rows, uint64_t cols,
+inline CUtensorMapDataType tmap_dtype(int dtype) {
+    return dtype == SPMM_FP8_E4M3 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+         : (dtype == SPMM_TF32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+         : (dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16));
+}
+
+// 2-D row-major tensor [rows][cols] of the handle's value type, box [box_rows][box_cols].
+int encode_2d(CUtensorMap* map, int dtype, const void* base, uint64_t rows, uint64_t cols,
                     uint32_t box_rows, uint32_t box_cols, CUtensorMapSwizzle swz) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return SPMM_ERR_CUDA;
-    const uint64_t es = dtype == SPMM_FP8_E4M3 ? 1 : 2;
+    const uint64_t es = static_cast<uint64_t>(elem_size(dtype));
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {cols * es};
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    const CUtensorMapDataType dt = dtype == SPMM_FP8_E4M3 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
-                                 : (dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
+    const CUtensorMapDataType dt = tmap_dtype(dtype);
     CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? SPMM_OK : SPMM_ERR_CUDA;
@@ -226,8 +231,10 @@ int check_opts(const spmm_opts_t* opts) {
 
 // Option checks shared by the host and the device builder; on success *hp is a fresh handle.
 int new_bcsr_handle(spmm_handle_s** hp, int64_t m, int64_t k, int dtype, int block, const spmm_opts_t* opts) {
-    if (dtype != SPMM_BF16 && dtype != SPMM_FP16 && dtype != SPMM_FP8_E4M3) return SPMM_ERR_UNSUPPORTED;
+    if (dtype != SPMM_BF16 && dtype != SPMM_FP16 && dtype != SPMM_FP8_E4M3 && dtype != SPMM_TF32) return SPMM_ERR_UNSUPPORTED;
     if (int orc = check_opts(opts)) return orc;
+    // TF32 (Sec. 3.1's k8 shape, the type of Sec. 4.1's BCSR evaluation): static schedule only
+    if (dtype == SPMM_TF32 && opts && opts->schedule != SPMM_SCHED_STATIC) return SPMM_ERR_UNSUPPORTED;
     if (dtype == SPMM_FP8_E4M3) {
         // 8-bit inputs: the K-major (column-major operand) path only, fp32 C, static schedule; a block
         // row must hold a whole 32-element K step; rows of X are k bytes and must be multiples of 16
@@ -243,7 +250,7 @@ int new_bcsr_handle(spmm_handle_s** hp, int64_t m, int64_t k, int dtype, int blo
     h->m = m;
     h->k = k;
     h->host_only = opts && opts->host_only;
-    h->c16 = opts && opts->c_type == SPMM_C_SAME_AS_INPUT;
+    h->c16 = opts && opts->c_type == SPMM_C_SAME_AS_INPUT && dtype != SPMM_TF32;   // TF32's own type is fp32
     h->cs = h->c16 ? 2 : 4;
     h->col_major = opts && opts->layout == SPMM_COLMAJOR;
     h->dynamic = opts && opts->schedule == SPMM_SCHED_DYNAMIC;
@@ -252,7 +259,7 @@ int new_bcsr_handle(spmm_handle_s** hp, int64_t m, int64_t k, int dtype, int blo
     if (h->dynamic && (h->c16 || h->col_major)) { delete h; return SPMM_ERR_UNSUPPORTED; }
     // column-major operands: rows of X (k elements) and of Y (m elements) must be multiples of
     // 16 bytes for the tensor map and for the 16-byte pieces the epilogue writes
-    if (h->col_major && (m % 8 != 0 || k % 8 != 0)) { delete h; return SPMM_ERR_UNSUPPORTED; }
+    if (h->col_major && (m % 8 != 0 || (k * h->es) % 16 != 0)) { delete h; return SPMM_ERR_UNSUPPORTED; }
     *hp = h;
     return SPMM_OK;
 }
@@ -262,11 +269,13 @@ int encode_tmA(spmm_handle_s* h) {
     const BcsrHost& f = h->bcsr;
     if (f.nnzb <= 0) return SPMM_OK;
     if (static_cast<int64_t>(f.nnzb) * f.b >= (int64_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
-    const int row_bytes = f.b * h->es < 128 ? f.b * h->es : 128;
+    // (a stage unit's rows: the whole block row, or one column slice of it, at most 128 bytes per piece)
+    const int unit_bytes = f.b / bcsr_k_split(f.b, h->es) * h->es;
+    const int row_bytes = unit_bytes < 128 ? unit_bytes : 128;
     const int bw = row_bytes / h->es;
     const CUtensorMapSwizzle swz = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                   : (row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
-    int rc = encode_2d_16bit(&h->tmA, h->dtype, h->d_vals, static_cast<uint64_t>(f.nnzb) * f.b, f.b,
+    int rc = encode_2d(&h->tmA, h->dtype, h->d_vals, static_cast<uint64_t>(f.nnzb) * f.b, f.b,
                              static_cast<uint32_t>(f.b * bcsr_blocks_per_stage(f.b)), bw, swz);
     h->tmA_ok = rc == SPMM_OK;
     return rc;
@@ -277,7 +286,7 @@ int encode_tmA(spmm_handle_s* h) {
 int setup_stack(spmm_handle_s* h) {
     const BcsrHost& f = h->bcsr;
     // static schedule only; b = 128 blocks already are 128 rows high
-    const bool eligible = !h->dynamic && f.b < 128 && h->stack_min_fill >= 0;
+    const bool eligible = !h->dynamic && f.b < 128 && h->stack_min_fill >= 0 && h->dtype != SPMM_TF32;
     int rc = build_bcsr_stack(f, eligible ? h->stack_min_fill : -1, &h->stack);
     if (rc || h->host_only || h->stack.ng == 0) return rc;
     const BcsrStack& st = h->stack;
@@ -289,7 +298,7 @@ int setup_stack(spmm_handle_s* h) {
     const int row_bytes = f.b * h->es;                // <= 128 for b <= 64
     const CUtensorMapSwizzle swz = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                   : (row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
-    return encode_2d_16bit(&h->tmAs, h->dtype, h->d_svals, static_cast<uint64_t>(st.ns) * kStackRows, f.b, kStackRows, f.b, swz);
+    return encode_2d(&h->tmAs, h->dtype, h->d_svals, static_cast<uint64_t>(st.ns) * kStackRows, f.b, kStackRows, f.b, swz);
 }
 
 int create_bcsr(spmm_handle_t* out, const CsrView& a, int dtype, int block, const spmm_opts_t* opts) {
@@ -523,11 +532,13 @@ int ensure_tmB(spmm_handle_s* h, const void* B, int64_t N, int groups) {
         // X as [N][k]: box = 128 tokens x min(b, 64) elements, swizzle = the box's row bytes;
         // and the same memory as [N / 128][128][k] so that one request brings all token groups
         // of a tile (whole groups only; a ragged last tile uses the 2-D map, zero filled)
-        const uint32_t row_bytes = h->bcsr.b * h->es < 128 ? h->bcsr.b * h->es : 128;
+        // (per stage unit: the block's k extent, or one column slice of it -- bcsr_k_split)
+        const uint32_t unit_bytes = h->bcsr.b / bcsr_k_split(h->bcsr.b, h->es) * h->es;
+        const uint32_t row_bytes = unit_bytes < 128 ? unit_bytes : 128;
         const uint32_t bw = row_bytes / h->es;
         const CUtensorMapSwizzle swz = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                       : (row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
-        rc = encode_2d_16bit(&h->tmB, h->dtype, B, static_cast<uint64_t>(N), static_cast<uint64_t>(h->k), 128, bw, swz);
+        rc = encode_2d(&h->tmB, h->dtype, B, static_cast<uint64_t>(N), static_cast<uint64_t>(h->k), 128, bw, swz);
         EncodeTiledFn fn = get_encode_fn();
         auto whole_tile_map = [&](int g, CUtensorMap* out, bool* ok) {
             *ok = false;
@@ -537,8 +548,7 @@ int ensure_tmB(spmm_handle_s* h, const void* B, int64_t N, int groups) {
             const cuuint64_t strides[2] = {static_cast<cuuint64_t>(h->k) * h->es, static_cast<cuuint64_t>(h->k) * 128 * h->es};
             const cuuint32_t box[3] = {bw, 128, static_cast<cuuint32_t>(g)};
             const cuuint32_t estr[3] = {1, 1, 1};
-            const CUtensorMapDataType dt = h->dtype == SPMM_FP8_E4M3 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
-                                         : (h->dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
+            const CUtensorMapDataType dt = tmap_dtype(h->dtype);
             CUresult r = fn(out, dt, 3, const_cast<void*>(B), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                             swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             *ok = r == CUDA_SUCCESS;
@@ -547,22 +557,27 @@ int ensure_tmB(spmm_handle_s* h, const void* B, int64_t N, int groups) {
         whole_tile_map(groups, &h->tmB3, &h->tmB3_ok);
         if (h->stack.ng > 0) whole_tile_map(kStackGroups, &h->tmB3s, &h->tmB3s_ok);
     } else {
-        rc = encode_2d_16bit(&h->tmB, h->dtype, B, static_cast<uint64_t>(h->k), static_cast<uint64_t>(N),
-                             static_cast<uint32_t>(h->bcsr.b), 64, CU_TENSOR_MAP_SWIZZLE_128B);
-        // the same memory as [N / 64][k][64]: one request then brings a whole token tile
-        // (2 * groups boxes); only full 64-token groups are covered, a ragged tail uses tmB
+        // B as [k][N]: box = kb rows (the block's k extent, or one column slice of A's block:
+        // bcsr_k_split) x 128 bytes of tokens; 4-byte elements take the 128-byte swizzle with
+        // 32-byte atoms, which is what a token-major (MN-major) tensor-core operand of that
+        // width reads
+        const uint32_t tok = 128u / static_cast<uint32_t>(h->es);          // tokens per box row
+        const uint32_t kb = static_cast<uint32_t>(h->bcsr.b / bcsr_k_split(h->bcsr.b, h->es));
+        const CUtensorMapSwizzle swz = h->es == 4 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B;
+        rc = encode_2d(&h->tmB, h->dtype, B, static_cast<uint64_t>(h->k), static_cast<uint64_t>(N), kb, tok, swz);
+        // the same memory as [N / tok][k][tok]: one request then brings a whole token tile
+        // (es * groups boxes); only full groups of tok tokens are covered, a ragged tail uses tmB
         EncodeTiledFn fn = get_encode_fn();
         auto whole_tile_map = [&](int g, CUtensorMap* out, bool* ok) {
             *ok = false;
             *out = h->tmB;
-            if (rc || !fn || N < 64) return;
-            const cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(h->k), static_cast<cuuint64_t>(N / 64)};
-            const cuuint64_t strides[2] = {static_cast<cuuint64_t>(N) * 2, 128};
-            const cuuint32_t box[3] = {64, static_cast<cuuint32_t>(h->bcsr.b), static_cast<cuuint32_t>(2 * g)};
+            if (rc || !fn || N < static_cast<int64_t>(tok)) return;
+            const cuuint64_t dims[3] = {tok, static_cast<cuuint64_t>(h->k), static_cast<cuuint64_t>(N / tok)};
+            const cuuint64_t strides[2] = {static_cast<cuuint64_t>(N) * h->es, 128};
+            const cuuint32_t box[3] = {tok, kb, static_cast<cuuint32_t>(h->es * g)};
             const cuuint32_t estr[3] = {1, 1, 1};
-            const CUtensorMapDataType dt = h->dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
-            CUresult r = fn(out, dt, 3, const_cast<void*>(B), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            CUresult r = fn(out, tmap_dtype(h->dtype), 3, const_cast<void*>(B), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             *ok = r == CUDA_SUCCESS;
             if (!*ok) *out = h->tmB;
         };
@@ -613,7 +628,7 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
     // token tile: the largest of 512 / 256 / 128 columns that divides N (Sec. 4.3: pick a tile
     // width that divides the dense width so that no padded columns are computed); otherwise
     // the largest tile, whose ragged last tile is predicated.
-    const int gmax = bcsr_token_groups_max(f.b, h->c16 ? 1 : 0, h->col_major ? 1 : 0);
+    const int gmax = bcsr_token_groups_max(h->dtype, f.b, h->c16 ? 1 : 0, h->col_major ? 1 : 0);
     int groups = 0;
     for (int g = gmax; g >= 1; g >>= 1)
         if (N % (128 * g) == 0) { groups = g; break; }
@@ -744,7 +759,7 @@ int run_bcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t s
     CUtensorMap tmA = h->tmA;
     if (!h->tmA_ok) {
         // no stored block at all: the kernel never touches A, any valid map will do
-        rc = encode_2d_16bit(&tmA, h->dtype, h->d_vals, 8, 8, 8, 8, CU_TENSOR_MAP_SWIZZLE_NONE);
+        rc = encode_2d(&tmA, h->dtype, h->d_vals, 8, 8, 8, 8, CU_TENSOR_MAP_SWIZZLE_NONE);
         if (rc) return rc;
     }
     rc = ensure_tmB(h, B, N, h->sched.groups);

@@ -46,18 +46,25 @@ namespace spmm {
 
 namespace {
 
-// ES = bytes per input element: 2 (fp16 / bf16), or 1 (E4M3, column-major operands only).
+// ES = bytes per input element: 2 (fp16 / bf16), 4 (fp32 storage, TF32 arithmetic), or 1 (E4M3,
+// column-major operands only).
 // H = rows of one stored block = the MMA's N extent: B for the format's own b x b blocks, 128 for
 // the stacked blocks of a row group (128 / b block-rows on top of one another, see format.h).
 // CS = bytes per element of C, CM = column-major operands: they fix the epilogue's staging tile.
+// A pipeline stage holds one "unit": kBps whole blocks (small b), or one of the kKS column
+// slices a block is cut into where its rows are longer than 128 bytes of 4-byte elements
+// (b = 64 / 128 with TF32: units of 32 columns, so that a stage stays a fraction of shared memory).
 template <int B, int H, int GROUPS, int STAGES, int ES, int CS, int CM>
 struct BcsrCfg {
-    static constexpr int kBB = B * ES;                       // bytes of one block row (its K extent)
-    static constexpr int kKSteps = kBB / 32;                 // MMAs per block and token group (32 bytes of K each)
+    static constexpr int kKS = (H == B) ? bcsr_k_split(B, ES) : 1;     // stage units per block
+    static constexpr int kKB = B / kKS;                      // columns of A (= rows of B) per unit
+    static constexpr int kBB = kKB * ES;                     // bytes of one unit row (its K extent)
+    static constexpr int kKSteps = kBB / 32;                 // MMAs per unit and token group (32 bytes of K each)
     static constexpr int kBnT = 128 * GROUPS;
-    static constexpr int kNBox = 2 * GROUPS;                 // 64-token boxes per block (row-major B)
-    static constexpr int kBoxBytes = B * 128;                // b k-rows x 128 B (row-major B, 2-byte elements)
-    static constexpr int kDenseBytes = kBnT * kBB;           // B tile of one block
+    static constexpr int kTokBox = 128 / ES;                 // tokens per 128-byte box row (row-major B)
+    static constexpr int kNBox = GROUPS * (128 / kTokBox);   // boxes per unit (row-major B)
+    static constexpr int kBoxBytes = kKB * 128;              // kKB k-rows x 128 B (row-major B)
+    static constexpr int kDenseBytes = kBnT * kBB;           // B tile of one unit
     static constexpr int kABytes = H * kBB;
     // Small blocks carry too little work for the fixed cost of a pipeline stage (barrier
     // round trip, request issue, MMA hand-off): a stage holds several consecutive stored
@@ -89,7 +96,8 @@ struct BcsrCfg {
     static_assert(2 * kAccCols <= 512, "accumulators exceed TMEM");
     static_assert(kSmemBytes <= 227 * 1024, "stage ring exceeds shared memory");
     static_assert((2 * STAGES + 7 + 8) * 8 + 64 <= kBarrierBytes, "barrier area");
-    static_assert(kBps == 1 || B <= 32, "multi-block stages are for the small block sizes");
+    static_assert(kBps == 1 || (B <= 32 && kKS == 1), "multi-block stages are for the small block sizes");
+    static_assert(kKS == 1 || kBB <= 128, "a column slice is at most one 128-byte row piece");
     static_assert(kBB % 32 == 0, "a block row must hold whole K steps");
     static_assert(H == B || (H == 128 && B < 128), "stacked blocks are 128 rows high");
 };
@@ -109,8 +117,9 @@ template <int B, int H, int GROUPS, int STAGES, int FMT, int CT, int CM, int DYN
 __global__ void __launch_bounds__(DYN ? 224 : 192, 1)
 bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ CUtensorMap tmC, const BcsrParams p) {
-    constexpr int ES = FMT == 3 ? 1 : 2;
-    static_assert(ES == 2 || CM, "8-bit inputs: column-major operands only");
+    constexpr int ES = FMT == 3 ? 1 : (FMT == 2 ? 4 : 2);
+    static_assert(ES != 1 || CM, "8-bit inputs: column-major operands only");
+    static_assert(FMT != 2 || (!CT && !DYN && H == B), "TF32: fp32 C, static schedule, no row groups");
     static_assert(H == B || !DYN, "stacked blocks: static schedule only");
     using CElem = typename CType<FMT, CT>::type;
     using Cfg = BcsrCfg<B, H, GROUPS, STAGES, ES, static_cast<int>(sizeof(CElem)), CM>;
@@ -224,7 +233,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             for (uint32_t nth = 0; ok && next_tile(nth, &tcd, &tcd_next, &ok); ++nth) {
                 const int n0 = tcd.y * Cfg::kBnT;
                 const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
-                const int nbox = (nvalid + 63) >> 6;
+                const int nbox = (nvalid + Cfg::kTokBox - 1) / Cfg::kTokBox;
                 const bool whole_tile = p.use_3d && nvalid == Cfg::kBnT;
                 const int pb = tcd.z, pe = tcd.w;
                 const int Jl_first = have_next ? Jl_next : ((pb + lane < pe) ? __ldg(p.block_col_idx + pb + lane) : 0);
@@ -237,8 +246,11 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     // block columns of up to 32 stored blocks with one coalesced load
                     const int Jl = q0 == pb ? Jl_first : ((q0 + lane < pe) ? __ldg(p.block_col_idx + q0 + lane) : 0);
                     const int nq = min(32, pe - q0);
-                    for (int jq = 0; jq < nq; jq += Cfg::kBps, ++it) {
+                    for (int jq = 0; jq < nq && ok; jq += Cfg::kBps)
+#pragma unroll 1
+                    for (int kp = 0; kp < Cfg::kKS; ++kp, ++it) {       // column slices of the block (1 unless TF32, b >= 64)
                         const int q = q0 + jq;
+                        const int kx = kp * Cfg::kKB;                    // first column of A / first row of B of this unit
                         const int nb = min(Cfg::kBps, nq - jq);          // stored blocks in this stage
                         const int s = it % STAGES;
                         const uint32_t ph = (it / STAGES) & 1u;
@@ -259,32 +271,32 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             if (whole_tile) {
                                 if (blk < nb && hf < kHalves)
                                     tma_load_3d_hint(sb + blk * Cfg::kDenseBytes + hf * (GROUPS * Cfg::kXGroupBytes), &tmB3,
-                                                     full_bar(s), J * B + hf * (128 / ES), 0, n0 >> 7, keep);
+                                                     full_bar(s), J * B + kx + hf * (128 / ES), 0, n0 >> 7, keep);
                             } else {
                                 // ragged tile: one request per 128-token group, rows >= N are zero filled
                                 const int ngrp = (nvalid + 127) >> 7;
                                 for (int g = 0; g < ngrp; ++g)
                                     if (blk < nb && hf < kHalves)
                                         tma_load_2d_hint(sb + blk * Cfg::kDenseBytes + hf * (GROUPS * Cfg::kXGroupBytes) + g * Cfg::kXGroupBytes,
-                                                         &tmB, full_bar(s), J * B + hf * (128 / ES), n0 + g * 128, keep);
+                                                         &tmB, full_bar(s), J * B + kx + hf * (128 / ES), n0 + g * 128, keep);
                             }
                         } else
                         if (whole_tile) {
-                            // all 2 * GROUPS boxes of a block with one request: B seen as
-                            // [64-token group][k][64 tokens], box = kNBox x b x 64; lane i takes block i
+                            // all boxes of a unit with one request: B seen as [token box][k][128 bytes of
+                            // tokens], box = kNBox x kKB x 128 bytes; lane i takes block i
                             const int J = __shfl_sync(0xffffffffu, Jl, jq + (lane < nb ? lane : 0));
-                            if (lane < nb) tma_load_3d_hint(sb + lane * Cfg::kDenseBytes, &tmB3, full_bar(s), 0, J * B, n0 >> 6, keep);
+                            if (lane < nb) tma_load_3d_hint(sb + lane * Cfg::kDenseBytes, &tmB3, full_bar(s), 0, J * B + kx, n0 / Cfg::kTokBox, keep);
                         } else {
                             for (int i = 0; i < nb; ++i) {
                                 const int J = __shfl_sync(0xffffffffu, Jl, jq + i);
                                 if (lane < nbox)
                                     tma_load_2d_hint(sb + i * Cfg::kDenseBytes + lane * Cfg::kBoxBytes, &tmB, full_bar(s),
-                                                     n0 + lane * 64, J * B, keep);
+                                                     n0 + lane * Cfg::kTokBox, J * B + kx, keep);
                             }
                         }
                         if constexpr (H == B) {
                             if (lane == 8) {
-                                tma_load_2d_hint(sb + Cfg::kAOff, &tmA, full_bar(s), 0, q * B, keep);
+                                tma_load_2d_hint(sb + Cfg::kAOff, &tmA, full_bar(s), kx, q * B, keep);
                             } else if (Cfg::kBB > 128 && lane == 9) {
                                 tma_load_2d_hint(sb + Cfg::kAOff + B * 128, &tmA, full_bar(s), 128 / ES, q * B, keep);
                             }
@@ -311,8 +323,11 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         {
             // 8-bit floats: format code 0 = E4M3 in both operand fields
             constexpr uint32_t idesc = make_idesc(FMT == 3 ? 0 : FMT, 128, H, CM ? 0 : 1, 0);
+            // row-major B: the token tile is MN-major; 4-byte elements need the 128-byte swizzle with
+            // 32-byte atoms (a pattern of 4 k-rows), 2-byte elements the plain one (8 k-rows)
             const uint64_t adesc0 = CM ? make_smem_desc(0, 16, 8 * Cfg::kXRowBytes, Cfg::kASwizzle)
-                                       : make_smem_desc(0, Cfg::kBoxBytes, 1024, SWZ_128B);
+                                       : make_smem_desc(0, Cfg::kBoxBytes, ES == 4 ? 512 : 1024, ES == 4 ? SWZ_128B_BASE32B : SWZ_128B);
+            constexpr int kStepBytes = (32 / ES) * 128;     // k-rows of one MMA x 128 bytes (row-major token tile)
             const uint64_t bdesc0 = make_smem_desc(0, 16, 8 * Cfg::kARowBytes, Cfg::kASwizzle);
             const bool leader = elect_one();
             uint32_t it = 0, tile_i = 0;
@@ -328,7 +343,9 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 tc_fence_after_sync();
                 const uint32_t d0 = tmem_base + acc * Cfg::kAccCols;
                 const int pb = tcd.z, pe = tcd.w;
-                for (int q = pb; q < pe; q += Cfg::kBps, ++it) {
+                for (int q = pb; q < pe && ok; q += Cfg::kBps)
+#pragma unroll 1
+                for (int kp = 0; kp < Cfg::kKS; ++kp, ++it) {
                     // stages never straddle the producer's 32-block windows (kBps divides 32)
                     const int nb = min(Cfg::kBps, min(pe - q, 32 - ((q - pb) & 31)));
                     const int s = it % STAGES;
@@ -342,17 +359,17 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             // descriptors differ only in their start-address field (bytes >> 4)
                             const uint64_t a0 = adesc0 + ((sb + i * Cfg::kDenseBytes) >> 4);
                             const uint64_t b0 = bdesc0 + ((sb + Cfg::kAOff + i * Cfg::kABytes) >> 4);
-                            const uint32_t accum0 = (q > pb || i > 0) ? 1u : 0u;
+                            const uint32_t accum0 = (q > pb || i > 0 || kp > 0) ? 1u : 0u;
 #pragma unroll
                             for (int ks = 0; ks < Cfg::kKSteps; ++ks) {
                                 const uint32_t boff = Cfg::kBB <= 128 ? ks * 32 : (ks >> 2) * (B * 128) + (ks & 3) * 32;
 #pragma unroll
                                 for (int g = 0; g < GROUPS; ++g)
                                     if (leader && g < ngrp)
-                                        umma_kind<FMT == 3 ? 2 : 0>(d0 + g * H,
+                                        umma_kind<FMT == 3 ? 2 : (FMT == 2 ? 1 : 0)>(d0 + g * H,
                                                        a0 + ((CM ? (Cfg::kBB <= 128 ? g * Cfg::kXGroupBytes + ks * 32
                                                                             : (ks >> 2) * (GROUPS * Cfg::kXGroupBytes) + g * Cfg::kXGroupBytes + (ks & 3) * 32)
-                                                                 : g * 2 * Cfg::kBoxBytes + ks * 2048) >> 4),
+                                                                 : g * (Cfg::kNBox / GROUPS) * Cfg::kBoxBytes + ks * kStepBytes) >> 4),
                                                        b0 + (boff >> 4), idesc, ks > 0 ? 1u : accum0);
                             }
                         }
@@ -517,7 +534,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 template <int B, int H, int GROUPS, int CAP, int FMT, int CT, int CM, int DYN>
 cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p,
                        int grid, cudaStream_t stream) {
-    constexpr int ES = FMT == 3 ? 1 : 2;
+    constexpr int ES = FMT == 3 ? 1 : (FMT == 2 ? 4 : 2);
     constexpr int CS = static_cast<int>(sizeof(typename CType<FMT, CT>::type));
     constexpr int STAGES = bcsr_fit_stages<B, H, GROUPS, CAP, ES, CS, CM>();
     using Cfg = BcsrCfg<B, H, GROUPS, STAGES, ES, CS, CM>;
@@ -611,6 +628,24 @@ cudaError_t launch_fp8(int b, int groups, const CUtensorMap& tmA, const CUtensor
     }
 }
 
+// TF32 (fp32 storage): fp32 C, static schedule; the deepest rings the stage sizes allow.
+template <int CM>
+cudaError_t launch_tf32(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
+                        const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
+    switch (b * 10 + groups) {
+        case 161: return launch_one<16, 16, 1, 5, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 162: return launch_one<16, 16, 2, 3, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 321: return launch_one<32, 32, 1, 5, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 322: return launch_one<32, 32, 2, 3, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 641: return launch_one<64, 64, 1, 8, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 642: return launch_one<64, 64, 2, 5, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 644: return launch_one<64, 64, 4, 3, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 1281: return launch_one<128, 128, 1, 6, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 1282: return launch_one<128, 128, 2, 4, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
 template <int FMT>
 cudaError_t launch_fmt(int b, int groups, int c16, int cm, int dyn, const CUtensorMap& tmA, const CUtensorMap& tmB,
                        const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
@@ -628,8 +663,11 @@ cudaError_t launch_fmt(int b, int groups, int c16, int cm, int dyn, const CUtens
 // the most bytes of C per staged operand byte: there a 256-token tile with five 40 KB stages and
 // three staging tiles per epilogue warp measured 3 % faster than 512 tokens with three 72 KB
 // stages and one staging tile; every other combination measured equal or slower with 256.
-int bcsr_token_groups_max(int b, int c16, int col_major) {
+// TF32: elements are twice as wide, so b = 16 / 32 stop at 256 tokens (a 512-token stage of
+// several blocks would not fit twice).
+int bcsr_token_groups_max(int dtype, int b, int c16, int col_major) {
     if (b == 128) return 2;
+    if (dtype == 2 && b <= 32) return 2;
     return (b == 64 && !c16 && !col_major) ? 2 : 4;
 }
 
@@ -640,6 +678,11 @@ cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, in
     if (dtype == 0) return launch_fmt<1>(b, groups, c16, col_major, dynamic, tmA, tmB, tmB3, tmC, p, grid, stream);   // bf16
     if (dtype == 3) return (c16 || !col_major || dynamic) ? cudaErrorInvalidValue
                                                            : launch_fp8(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
+    if (dtype == 2) {
+        if (c16 || dynamic) return cudaErrorInvalidValue;
+        return col_major ? launch_tf32<1>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream)
+                         : launch_tf32<0>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
+    }
     return cudaErrorInvalidValue;
 }
 

@@ -187,7 +187,8 @@ bcsr_fill_kernel(int64_t m, int b, int words, const int64_t* row_ptr, const int3
             uint8_t* dst = blocks + slot * tile_bytes + (static_cast<size_t>(i - I * b) * b + (c - J * b)) * ES;
             const uint8_t* src = vals + static_cast<size_t>(p) * ES;
             if constexpr (ES == 1) *dst = *src;
-            else *reinterpret_cast<uint16_t*>(dst) = *reinterpret_cast<const uint16_t*>(src);
+            else if constexpr (ES == 2) *reinterpret_cast<uint16_t*>(dst) = *reinterpret_cast<const uint16_t*>(src);
+            else *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(src);
         }
     }
 }
@@ -253,7 +254,7 @@ int build_bcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int3
                       int es, int b, cudaStream_t st, BcsrHost* out, int64_t* nnz_out, int32_t** d_block_row_ptr,
                       int32_t** d_block_col_idx, uint8_t** d_blocks) {
     if (b != 16 && b != 32 && b != 64 && b != 128) return SPMM_ERR_UNSUPPORTED;
-    if (es != 1 && es != 2) return SPMM_ERR_UNSUPPORTED;
+    if (es != 1 && es != 2 && es != 4) return SPMM_ERR_UNSUPPORTED;
     if (m < 0 || k < 0 || !d_row_ptr) return SPMM_ERR_INVALID_ARG;
     const int64_t nbr = (m + b - 1) / b, nbc = (k + b - 1) / b;
     const int words = static_cast<int>((nbc + 31) / 32);
@@ -330,6 +331,8 @@ int build_bcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int3
     if (nbr > 0 && nnzb > 0) {
         if (es == 1)
             bcsr_fill_kernel<1><<<static_cast<unsigned>(nbr), kThreads, smem, st>>>(m, b, words, d_row_ptr, d_col_idx, d_vals, *d_block_row_ptr, *d_block_col_idx, *d_blocks);
+        else if (es == 4)
+            bcsr_fill_kernel<4><<<static_cast<unsigned>(nbr), kThreads, smem, st>>>(m, b, words, d_row_ptr, d_col_idx, d_vals, *d_block_row_ptr, *d_block_col_idx, *d_blocks);
         else
             bcsr_fill_kernel<2><<<static_cast<unsigned>(nbr), kThreads, smem, st>>>(m, b, words, d_row_ptr, d_col_idx, d_vals, *d_block_row_ptr, *d_block_col_idx, *d_blocks);
     }

@@ -30,11 +30,15 @@ struct BcsrParams {
     int32_t overlap;
 };
 
-// dtype: 0 bf16, 1 fp16.  groups: token tile = 128 * groups columns of B (1, 2 or 4).
-// c16: C in the input's 16-bit type.  Row-major operands: tmB = B as [k][N], box b x 64;
-// tmB3 = B as [N / 64][k][64], box (2 * groups) x b x 64.  Column-major operands (col_major):
-// tmB = X as [N][k], box 128 tokens x min(b, 64); tmB3 = X as [N / 128][128][k], box
-// groups x 128 x min(b, 64); both with the swizzle of min(b, 64) * 2 bytes.
+// dtype: 0 bf16, 1 fp16, 2 tf32 (fp32 storage; fp32 C, static schedule), 3 E4M3 (column-major
+// operands, fp32 C).  groups: token tile = 128 * groups columns of B (1, 2 or 4).
+// c16: C in the input's 16-bit type.  With es = bytes per element, t = 128 / es tokens per
+// 128-byte box row and kb = b / bcsr_k_split(b, es) rows of B per stage unit --
+// row-major operands: tmB = B as [k][N], box kb x t; tmB3 = B as [N / t][k][t], box
+// (es * groups) x kb x t; 128-byte swizzle (with 32-byte atoms for es = 4).  Column-major operands
+// (col_major): tmB = X as [N][k], box 128 tokens x min(kb * es, 128) bytes; tmB3 = X as
+// [N / 128][128][k], box groups x 128 x the same; both with the swizzle of that row length.
+// tmA: the stored blocks as [blocks * b][b], box (b * blocks per stage) rows x min(kb * es, 128) bytes.
 // tmC: C as [m][N], box 32 x bcsr_epi_cols, no swizzle; or Y as [N][m], box bcsr_epi_cols x 32,
 // 64-byte swizzle when a box row is 64 bytes.
 // dynamic: the grid is one CTA per tile (grid = number of tiles, p.tiles in the schedule's global
@@ -49,7 +53,7 @@ constexpr int kStackGroups = 2;
 cudaError_t launch_bcsr_stacked(int dtype, int b, int c16, int col_major, const CUtensorMap& tmA, const CUtensorMap& tmB,
                                 const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p, int grid,
                                 cudaStream_t stream);
-int bcsr_token_groups_max(int b, int c16, int col_major);
+int bcsr_token_groups_max(int dtype, int b, int c16, int col_major);
 // Accumulator columns (= rows of A's block) an epilogue warp handles at a time: it stages them
 // in a 2 KB (1 KB for b = 16 with 16-bit C) shared-memory tile and stores the tile with one TMA
 // request whose box is 32 tokens x this many rows (row-major C) or this many columns x 32 tokens
@@ -57,6 +61,10 @@ int bcsr_token_groups_max(int b, int c16, int col_major);
 constexpr int bcsr_epi_cols(int b, bool c16, bool col_major) { return (b < 32 || !c16) ? 16 : 32; }
 // stored blocks that share one pipeline stage (and one A request): 4 / 2 for b = 16 / 32
 constexpr int bcsr_blocks_per_stage(int b) { return b == 16 ? 4 : (b == 32 ? 2 : 1); }
+// Column slices a stored block is cut into, one pipeline stage each: blocks of 4-byte elements
+// with rows longer than 128 bytes (TF32, b = 64 / 128) go through the ring 32 columns at a time;
+// every other block is one unit.
+constexpr int bcsr_k_split(int b, int es) { return (es == 4 && b > 32) ? b / 32 : 1; }
 
 // WCSR pipeline shape, shared by the host schedule (fills are cut to the stage size) and the
 // kernel.  A stage holds 128 / es columns (64 of a 2-byte type, 32 of TF32) of one 128-token

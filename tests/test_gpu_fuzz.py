@@ -63,6 +63,45 @@ def test_bcsr_random_case(lib, seed):
         lib.spmm_destroy(h)
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_bcsr_tf32_random_case(lib, seed):
+    """fp32 storage / TF32 arithmetic: block sizes, both operand layouts, both builders, ragged shapes."""
+    import torch
+    rng = np.random.default_rng(13000 + seed)
+    b = int([16, 32, 64, 128][seed % 4])
+    col_major = bool(rng.integers(0, 2))
+    on_gpu = bool(rng.integers(0, 2))
+    m, k = int(rng.integers(1, 1500)), int(rng.integers(1, 1500))
+    if col_major:
+        m, k = _round_up(m, 8), _round_up(k, 4)
+    N = int(rng.integers(128 if col_major else 64, 1400))
+    if not col_major:
+        N = _round_up(N, 4)
+    dens = float(10.0 ** rng.uniform(-3.0, -0.7))
+    a = wl.random_csr(int(rng.integers(0, 1 << 30)), m, k, dens, "tf32", empty_rows=tuple(range(min(b, m // 3))))
+    Bs = wl.dense(int(rng.integers(0, 1 << 30)), k, N, ("normal", 0.0, 1.0), "tf32")
+    opt = dict(layout=lib.COLMAJOR if col_major else lib.ROWMAJOR)
+    what = "seed %d: tf32 b=%d m=%d k=%d N=%d dens=%.4f cm=%d gpu-built=%d" % (seed, b, m, k, N, dens, col_major, on_gpu)
+    if on_gpu:
+        rp = torch.from_numpy(a["row_ptr"].astype(np.int64)).cuda()
+        ci = torch.from_numpy(a["col_idx"].astype(np.int32)).cuda()
+        va = to_device(a["vals"])
+        h = lib.spmm_bcsr_create_csr_device(m, k, rp.data_ptr(), ci.data_ptr(), va.data_ptr(), "tf32", b, **opt)
+    else:
+        h = lib.spmm_bcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], "tf32", b, **opt)
+    try:
+        if on_gpu:
+            from oracle import formats as F
+            f = F.bcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], b)
+            assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCK_COL_IDX, np.int32), f["block_col_idx"]), what
+            assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCKS, np.uint32), f["blocks"].view(np.uint32).ravel()), what
+        C = run_gpu_variant(lib, h, Bs, m, N, "tf32", col_major=col_major)
+        Cr, S = reference(a, Bs, "tf32")
+        assert_close(C, Cr, S, "tf32", what)
+    finally:
+        lib.spmm_destroy(h)
+
+
 @pytest.mark.parametrize("seed", range(40))
 def test_bcsr_row_groups_random_case(lib, seed):
     """Row groups forced on (every run of 128 / b non-empty block-rows is stacked, however few of its

@@ -27,10 +27,11 @@ def _bcsr_case(lib, a, dtype, b, N, Bdist=("uniform", -1.0, 1.0), seed=9):
         f = F.bcsr_from_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], b)
         assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCK_ROW_PTR, np.int32), f["block_row_ptr"])
         assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCK_COL_IDX, np.int32), f["block_col_idx"])
-        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCKS, np.uint16), f["blocks"].view(np.uint16).ravel())
+        bits = np.uint32 if dtype == "tf32" else np.uint16
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_BLOCKS, bits), f["blocks"].view(bits).ravel())
         C = run_gpu(lib, h, Bs, a["m"], N)
         Cr, S = reference(a, Bs, dtype)
-        worst = assert_close(C, Cr, S, dtype, "bcsr b=%d N=%d" % (b, N))
+        worst = assert_close(C, Cr, S, dtype, "bcsr %s b=%d N=%d" % (dtype, b, N))
         C2 = run_gpu(lib, h, Bs, a["m"], N)
         assert np.array_equal(C, C2)                   # run-to-run identical
         return worst
@@ -57,6 +58,42 @@ def test_bcsr_ragged_shapes(lib, m, k, b, N):
     """m, k not multiples of b; N not a multiple of the token tile; scattered entries."""
     a = wl.random_csr(7 + m, m, k, 0.02, "fp16", empty_rows=tuple(range(min(b, m // 2))))
     _bcsr_case(lib, a, "fp16", b, N)
+
+
+@pytest.mark.parametrize("b", [16, 32, 64, 128])
+def test_bcsr_tf32_block_sizes(lib, b):
+    """fp32 storage, TF32 tensor-core arithmetic (the type of Sec. 4.1's BCSR evaluation; Sec. 3.1's
+    k8 instruction shape): every block size, several token tiles, bound 2e-3."""
+    a = wl.bcsr_sweep(400 + b, m=1024, k=768, b=b, density=0.2, dtype="tf32")
+    worst = _bcsr_case(lib, a, "tf32", b, 640, Bdist=("normal", 0.0, 1.0))
+    assert worst < 1.0
+
+
+@pytest.mark.parametrize("m,k,b,N", [(500, 300, 64, 200), (130, 70, 32, 72), (1000, 1000, 16, 1032),
+                                      (257, 640, 128, 328), (64, 64, 64, 64), (300, 200, 128, 2052)])
+def test_bcsr_tf32_ragged_shapes(lib, m, k, b, N):
+    """m, k not multiples of b; N not a multiple of the token tile (nor of the 32-token box)."""
+    a = wl.random_csr(9 + m, m, k, 0.02, "tf32", empty_rows=tuple(range(min(b, m // 2))))
+    _bcsr_case(lib, a, "tf32", b, N)
+
+
+@pytest.mark.parametrize("b,N", [(16, 384), (32, 200), (64, 1024), (128, 520)])
+def test_bcsr_tf32_colmajor(lib, b, N):
+    """TF32 with column-major operands (X [N][k] in, Y [N][m] out): the plain K-major operand case,
+    bit-identical to the row-major result (same products, same order)."""
+    a = wl.bcsr_sweep(500 + b, m=512, k=768, b=b, density=0.3, dtype="tf32")
+    Bs = wl.dense(11, a["k"], N, ("normal", 0.0, 1.0), "tf32")
+    h0 = lib.spmm_bcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "tf32", b)
+    h1 = lib.spmm_bcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "tf32", b, layout=lib.COLMAJOR)
+    try:
+        C0 = run_gpu(lib, h0, Bs, a["m"], N)
+        C1 = run_gpu_variant(lib, h1, Bs, a["m"], N, "tf32", col_major=True)
+        Cr, S = reference(a, Bs, "tf32")
+        assert_close(C1, Cr, S, "tf32", "bcsr tf32 column-major b=%d" % b)
+        assert np.array_equal(C0, C1)
+    finally:
+        lib.spmm_destroy(h0)
+        lib.spmm_destroy(h1)
 
 
 def test_bcsr_all_empty_and_identity(lib):

@@ -42,7 +42,7 @@ def _bits(a):
 
 BCSR_CASES = [
     ("bf16", 512, 512, 64), ("fp16", 300, 410, 16), ("fp16", 257, 129, 32),
-    ("bf16", 640, 384, 128), ("fp16", 64, 64, 64),
+    ("bf16", 640, 384, 128), ("fp16", 64, 64, 64), ("tf32", 300, 260, 64), ("tf32", 130, 513, 16),
 ]
 
 
@@ -65,7 +65,7 @@ def test_bcsr_format_is_bit_exact(lib, dtype, m, k, b):
         assert info["n_empty"] == int((np.diff(f["block_row_ptr"]) == 0).sum()) >= 1
         assert info["flops_stored"] == 2.0 * nnzb * b * b * 256
         rows_touched = min(k, np.unique(f["block_col_idx"]).shape[0] * b)
-        assert info["bytes_b_touched"] == rows_touched * 256 * 2
+        assert info["bytes_b_touched"] == rows_touched * 256 * wl.elem_size(dtype)
         assert info["bytes_c"] == m * 256 * 4
         with pytest.raises(lib.SpmmError) as e:
             lib.spmm_run(h, 16, 16, 256)
@@ -319,8 +319,9 @@ def test_malformed_input_is_rejected(lib):
     assert code(mk, 2, 4, np.array([0, 3, 2], np.int64), np.array([0, 1, 2], np.int32), v, "fp16", 16,
                 host_only=True) == lib.SPMM_ERR_INVALID_ARG
     assert code(mk, 2, 4, rp, np.array([0, 1, 2], np.int32), v, "fp16", 48, host_only=True) == lib.SPMM_ERR_UNSUPPORTED
+    # TF32 BCSR: static schedule only
     assert code(mk, 2, 4, rp, np.array([0, 1, 2], np.int32), np.ones(3, np.float32), "tf32", 16,
-                host_only=True) == lib.SPMM_ERR_UNSUPPORTED
+                host_only=True, schedule=lib.SCHED_DYNAMIC) == lib.SPMM_ERR_UNSUPPORTED
     mw = lib.spmm_wcsr_create_csr
     assert code(mw, 2, 4, rp, np.array([0, 1, 2], np.int32), v, "fp16", 8, host_only=True) == lib.SPMM_ERR_UNSUPPORTED
     assert code(mw, 2, 4, rp, np.array([0, 1, 2], np.int32), v, "fp16", 16, split_cols=24,
