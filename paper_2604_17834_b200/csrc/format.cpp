@@ -285,7 +285,33 @@ int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost*
         }
     }
 
+    wcsr_reuse_classes(out->window_col_idx.data(), P, a.k, &out->grp_class);
     return plan_wcsr(out, T, n_bins, a.es);
+}
+
+void wcsr_reuse_classes(const int32_t* window_col_idx, int64_t P, int64_t k, std::vector<uint8_t>* grp_class) {
+    // gathers per B row = windows whose column list holds it
+    std::vector<int32_t> refs(static_cast<size_t>(k), 0);
+    for (int64_t q = 0; q < P; ++q)
+        if (window_col_idx[q] >= 0) refs[window_col_idx[q]]++;
+    // rows gathered more than once, most gathered first (ties: lower index first)
+    std::vector<int32_t> order;
+    for (int64_t c = 0; c < k; ++c)
+        if (refs[c] > 1) order.push_back(static_cast<int32_t>(c));
+    std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return refs[x] > refs[y]; });
+    std::vector<uint8_t> cls(static_cast<size_t>(k), 0);
+    for (size_t r = 0; r < order.size(); ++r) {
+        int level = 7;
+        for (size_t lim = kWcsrTopClassRows; level > 0 && r >= lim; lim *= 2) --level;
+        if (level == 0) break;
+        cls[order[r]] = static_cast<uint8_t>(level);
+    }
+    grp_class->assign(static_cast<size_t>(P / 4), 0);
+    for (int64_t q = 0; q < P; ++q)
+        if (window_col_idx[q] >= 0) {
+            uint8_t& g = (*grp_class)[static_cast<size_t>(q >> 2)];
+            g = std::max(g, cls[window_col_idx[q]]);
+        }
 }
 
 // Largest bin load of the longest-processing-time assignment when windows are cut into chunks of T.

@@ -103,6 +103,13 @@ struct WcsrHost {
     // the same for the narrow-operand kernel variant (stages of kWcsrNarrowCols columns); empty
     // unless the value type is 2 bytes wide and the window height 16
     std::vector<int32_t> fills_narrow, bin_fill_narrow;
+    // Device-private gather hint (no effect on results): reuse class of every group of four
+    // consecutive padded columns, one byte each.  A column's class says how high its B row ranks
+    // by the number of windows that gather it: 7 = among the 16 Ki most gathered rows, 6 = 32 Ki,
+    // ... 1 = 1 Mi, 0 = below that or gathered once; a group takes the highest class of its four
+    // columns.  At run time the rows whose class reaches the level that fits half of L2 at the
+    // dense width in use are gathered with the evict-last priority, the others with evict-first.
+    std::vector<uint8_t> grp_class;       // [P / 4]
     // finalisation lists: windows whose C rows the merge kernel writes
     std::vector<int32_t> merge_window;    // split windows then empty windows
     std::vector<int32_t> merge_first;     // first slot (split) or -1 (empty)
@@ -146,6 +153,9 @@ constexpr int kStackTileFixedCost = 8;
 // best of the four: as few split windows as the balance allows.
 int default_split_cols(const std::vector<int32_t>& window_row_ptr, int64_t nwin, int64_t P, int n_bins);
 int build_wcsr(const CsrView& a, int wh, int b_col, int T, int n_bins, WcsrHost* out);
+// Reuse classes of the column groups (WcsrHost::grp_class) from window_col_idx [P] and k.
+constexpr int kWcsrTopClassRows = 16384;   // rows in class 7; every class below doubles it
+void wcsr_reuse_classes(const int32_t* window_col_idx, int64_t P, int64_t k, std::vector<uint8_t>* grp_class);
 // Second half of build_wcsr: split plan, bins, fills and merge lists from out->window_row_ptr / out->P.
 int plan_wcsr(WcsrHost* out, int T, int n_bins, int es);
 // The WCSR format arrays built on the GPU from a CSR matrix in device memory (format_gpu.cu):

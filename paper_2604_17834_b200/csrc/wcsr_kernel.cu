@@ -248,15 +248,20 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
         // ------------------------------------------------------------------ gather producers
         // Lane l of the owning warp issues gather u = l (+32 per round): row group u / kSegs
         // (rows 4*rg .. 4*rg+3 of the fill), 128-byte segment u % kSegs of those rows.
-        auto load_idx = [&](const int2 d, int4 (&idx)[Cfg::kRounds]) {
+        // (with gather hints: also the reuse class of the four columns, one byte)
+        const bool hints = p.grp_class != nullptr;
+        auto load_idx = [&](const int2 d, int4 (&idx)[Cfg::kRounds], int (&cls)[Cfg::kRounds]) {
             const int cnt = d.y & 0xFFFF;
 #pragma unroll
             for (int r = 0; r < Cfg::kRounds; ++r) {
                 const int rg = (lane + 32 * r) / Cfg::kSegs;
                 idx[r] = (rg * 4 < cnt) ? __ldg(reinterpret_cast<const int4*>(p.col_idx + d.x) + rg)
                                         : make_int4(-1, -1, -1, -1);
+                cls[r] = (hints && rg * 4 < cnt) ? __ldg(p.grp_class + (d.x >> 2) + rg) : 0;
             }
         };
+        // B rows that many windows gather stay in L2 in preference to everything that streams through
+        const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
 
         SegIter seg;
         seg.init();
@@ -267,6 +272,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
         // column indices of this warp's current fill and of its next two fills (requested two
         // fills ahead, so their latency never sits in the issue loop)
         int4 idx_cur[Cfg::kRounds], idx_n1[Cfg::kRounds], idx_n2[Cfg::kRounds];
+        int cls_cur[Cfg::kRounds], cls_n1[Cfg::kRounds], cls_n2[Cfg::kRounds];
         bool rdy0 = false, rdy1 = false;
         while (ok && seg.next(p)) {
             const int f0 = __ldg(p.bin_fill + seg.b), f1 = __ldg(p.bin_fill + seg.b + 1);
@@ -291,9 +297,9 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     d1.y = __shfl_sync(0xffffffffu, j1 < 32 ? win.y : nwin.y, j1 & 31);
                     d2.x = __shfl_sync(0xffffffffu, j2 < 32 ? win.x : nwin.x, j2 & 31);
                     d2.y = __shfl_sync(0xffffffffu, j2 < 32 ? win.y : nwin.y, j2 & 31);
-                    if (!rdy0) load_idx(d, idx_cur);
-                    if (have1 && !rdy1) load_idx(d1, idx_n1);
-                    if (have2) load_idx(d2, idx_n2);
+                    if (!rdy0) load_idx(d, idx_cur, cls_cur);
+                    if (have1 && !rdy1) load_idx(d1, idx_n1, cls_n1);
+                    if (have2) load_idx(d2, idx_n2, cls_n2);
 
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
@@ -304,8 +310,9 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     if (lane == 0) {
                         const uint32_t abytes = (cnt / Cfg::kKStep) * (kWH * 32);
                         mbar_arrive_expect_tx(full_bar(s), abytes + (cnt / 4) * nseg * 512);
-                        bulk_load_1d(sb + Cfg::kDenseBytes,
-                                     p.packed + static_cast<size_t>(q / Cfg::kKStep) * (kWH * 32), abytes, full_bar(s));
+                        const uint8_t* asrc = p.packed + static_cast<size_t>(q / Cfg::kKStep) * (kWH * 32);
+                        if (p.hint_flags & 1) bulk_load_1d_hint(sb + Cfg::kDenseBytes, asrc, abytes, full_bar(s), pol_stream);
+                        else bulk_load_1d(sb + Cfg::kDenseBytes, asrc, abytes, full_bar(s));
                     }
                     __syncwarp();
                     ++n_issued;
@@ -314,14 +321,22 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     for (int r = 0; r < Cfg::kRounds; ++r) {
                         const int u = lane + 32 * r;
                         const int rg = u / Cfg::kSegs, sg = u % Cfg::kSegs;
-                        if (rg * 4 < cnt && sg < nseg)
-                            tma_gather4_2d(sb + sg * Cfg::kAtomStride + rg * 512, &tmB, full_bar(s),
-                                           n0 + sg * (128 / ES), idx_cur[r].x, idx_cur[r].y, idx_cur[r].z, idx_cur[r].w);
+                        if (rg * 4 < cnt && sg < nseg) {
+                            if (hints)
+                                tma_gather4_2d_hint(sb + sg * Cfg::kAtomStride + rg * 512, &tmB, full_bar(s), n0 + sg * (128 / ES),
+                                                    idx_cur[r].x, idx_cur[r].y, idx_cur[r].z, idx_cur[r].w,
+                                                    cls_cur[r] >= p.hot_min ? pol_keep : pol_stream);
+                            else
+                                tma_gather4_2d(sb + sg * Cfg::kAtomStride + rg * 512, &tmB, full_bar(s),
+                                               n0 + sg * (128 / ES), idx_cur[r].x, idx_cur[r].y, idx_cur[r].z, idx_cur[r].w);
+                        }
                     }
 #pragma unroll
                     for (int r = 0; r < Cfg::kRounds; ++r) {
                         idx_cur[r] = idx_n1[r];
                         idx_n1[r] = idx_n2[r];
+                        cls_cur[r] = cls_n1[r];
+                        cls_n1[r] = cls_n2[r];
                     }
                     rdy0 = have1;
                     rdy1 = have2;
@@ -413,6 +428,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
     } else {
         // ------------------------------------------------------------------ epilogue warps
         const int qd = warp & 3;
+        const uint64_t pol_stream_c = l2_policy_evict_first();
         SegIter seg;
         seg.init();
         uint32_t item = 0;
@@ -463,7 +479,18 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     if (lane == 0) mbar_arrive(acce_bar(acc));
                     const int n = n0 + qd * 32 + lane;
                     if (n < N) {
-                        if (sizeof(CElem) == 4 || slot >= 0) {
+                        if (p.hint_flags & 2) {
+                            // C is written once and not read again by this kernel: let it leave L2 first
+                            if (sizeof(CElem) == 4 || slot >= 0) {
+#pragma unroll
+                                for (int jr = 0; jr < kWH; ++jr)
+                                    if (jr < rows) st_global_hint(out + static_cast<int64_t>(jr) * N + n, v[jr], pol_stream_c);
+                            } else {
+#pragma unroll
+                                for (int jr = 0; jr < kWH; ++jr)
+                                    if (jr < rows) st_global_hint(outc + static_cast<int64_t>(jr) * N + n, from_f32<CElem>(v[jr]), pol_stream_c);
+                            }
+                        } else if (sizeof(CElem) == 4 || slot >= 0) {
 #pragma unroll
                             for (int jr = 0; jr < kWH; ++jr)
                                 if (jr < rows) out[static_cast<int64_t>(jr) * N + n] = v[jr];
