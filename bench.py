@@ -144,6 +144,16 @@ def workload_table():
             w["opts"] = dict(w.get("opts", {}), gather=1)
             return w
         return f
+    def ksplit(base):
+        """Same workload with outlier block-rows cut into parts (opts.k_split)."""
+        def f():
+            w = base()
+            w["opts"] = dict(w.get("opts", {}), k_split=1)
+            return w
+        return f
+    for d in (0.1, 0.01):
+        t["cfg4_bcsr_sweep_b64_d%g_ksplit" % d] = ("configs[3] b=64 skewed rows, keep %g, long block-rows cut into parts" % d,
+                                                    ksplit(cfg4(64, d)))
     def tf32_sweep(b, d):
         """configs[3] shape in the value type of the paper's own BCSR evaluation (Sec. 4.1: TF32)."""
         def f():
@@ -191,6 +201,7 @@ ALL_OTHERS = DEFAULT_OTHERS + [
     "cfg2_wcsr_irregular_lsu_gather", "cfg5_wcsr_rmat_n128_lsu_gather",
     "cfg4_bcsr_sweep_b64_d0.1_dyn", "cfg4_bcsr_sweep_b16_d0.1_plain", "cfg4_bcsr_sweep_b32_d0.1_plain",
     "cfg4_bcsr_sweep_b16_d0.5", "cfg4_bcsr_sweep_b32_d0.5",
+    "cfg4_bcsr_sweep_b64_d0.1_ksplit", "cfg4_bcsr_sweep_b64_d0.01_ksplit",
     "cfg4_bcsr_sweep_b16_d0.1_tf32", "cfg4_bcsr_sweep_b32_d0.1_tf32", "cfg4_bcsr_sweep_b64_d0.1_tf32", "cfg4_bcsr_sweep_b128_d0.1_tf32"]
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures whose
@@ -353,6 +364,8 @@ def time_workload(torch, lib, w, steps, warmup, flush):
         torch.cuda.synchronize()
         ms_warm = float(np.mean([a.elapsed_time(b) for a, b in wevs]))
         launches = 1 + (1 if (w["kind"] == "wcsr" and (info["n_split"] + info["n_empty"]) > 0) else 0)
+        if w["kind"] == "bcsr" and info["n_slots"] > 0:
+            launches = 2                                   # K-split: the SpMM kernel and the merge of the parts
         if w["kind"] == "bcsr" and info["n_stacked_rows"] > 0:
             # row groups: their own launch, then the remaining block-rows (if any)
             if lib.spmm_export(h, lib.X_BCSR_STACK_TILES, np.int32).size > 0:

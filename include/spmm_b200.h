@@ -147,7 +147,16 @@ typedef struct {
                             exported format arrays and nnz_stored are unaffected.  Ignored for
                             b = 128 and the dynamic schedule.                                 */
     int32_t gather;      /* spmm_gather_t; WCSR only (a BCSR handle ignores it)              */
-    int32_t reserved[7];
+    int32_t k_split;     /* BCSR: 1 = a block-row whose stored blocks exceed a quarter of one
+                            CTA's mean load for the dense width at hand is cut into contiguous
+                            ranges of its stored blocks; each part computes a partial tile and
+                            a second kernel adds the parts in order (the same rule as the WCSR
+                            merge: run-to-run identical).  The optional counterpart of
+                            Sec. 3.3's task split for the structured path, where Sec. 3.5 - 3.6
+                            report the imbalance.  Static schedule, fp32 row-major C, no row
+                            groups in use.  0 = off (default: the uncut plan measured faster on
+                            the benchmark configurations).                                    */
+    int32_t reserved[6];
 } spmm_opts_t;
 
 typedef struct {
@@ -161,17 +170,19 @@ typedef struct {
     double  fill_ratio;      /* nnz / stored_values (Sec. 2.3)                                */
     int64_t n_rows_units;    /* BCSR: block-rows; WCSR: windows                               */
     int64_t n_empty;         /* empty block-rows / windows                                    */
-    int64_t n_tasks;         /* WCSR sub-tasks (0 for BCSR)                                   */
-    int64_t n_split;         /* WCSR windows cut into more than one task                      */
-    int64_t n_slots;         /* WCSR partial-sum tiles                                        */
-    int32_t split_cols;      /* WCSR T in effect                                              */
+    int64_t n_tasks;         /* WCSR sub-tasks; BCSR: K-split units of the current plan (0 if no
+                                block-row is cut)                                             */
+    int64_t n_split;         /* WCSR windows / BCSR block-rows cut into more than one part    */
+    int64_t n_slots;         /* partial-sum tiles (WCSR sub-tasks of split windows; BCSR parts) */
+    int32_t split_cols;      /* WCSR T in effect; BCSR: the K-split cap in stored blocks      */
     int32_t n_ctas;          /* grid size the schedule was built for                          */
     int64_t distinct_b_rows; /* rows of B that A touches (distinct stored columns)            */
     /* bytes the roofline model charges for one spmm_run at the given N: */
     double  bytes_a, bytes_idx, bytes_b_touched, bytes_c;
     double  bytes_gather;    /* B bytes that must enter shared memory (no reuse assumed)      */
     double  flops_stored;    /* 2 * stored_values * N                                         */
-    int64_t workspace_bytes; /* device scratch spmm_run needs at this N (WCSR partial tiles)  */
+    int64_t workspace_bytes; /* device scratch spmm_run needs at this N (partial tiles; for BCSR
+                                at the planned N)                                             */
     /* BCSR tile schedule currently held (spmm_bcsr_plan or the last spmm_run); 0 if none:   */
     int64_t plan_n;          /* dense width it was built for                                  */
     int32_t plan_token_tile; /* columns of B per tile: 128, 256 or 512                        */
@@ -198,6 +209,11 @@ typedef enum {
     SPMM_X_BCSR_STACK_TILE_PTR = 9, /* int32 [n_ctas+1]: per-CTA ranges of STACK_TILES (needs a
                                        plan)                                                  */
     SPMM_X_BCSR_STACK_TILES = 20,   /* int32 [n][2]: row group, 256-column token tile; CTA-major */
+    SPMM_X_BCSR_UNITS = 21,         /* int32 [n_units][4]: block-row, first stored block, end
+                                       stored block, partial slot (-1: the unit is a whole block-row
+                                       and writes C).  Empty unless the plan cut a block-row
+                                       (opts.k_split); TILES[.][0] then indexes this array instead
+                                       of naming a block-row                                    */
     SPMM_X_WCSR_WINDOW_ROW_PTR = 10,/* int32 [ceil(m/h)+1], in columns                        */
     SPMM_X_WCSR_WINDOW_COL_IDX = 11,/* int32 [P], -1 on padding                               */
     SPMM_X_WCSR_VALUES = 12,        /* dtype [h][P] row-major                                 */
@@ -298,6 +314,8 @@ int spmm_bcsr_plan(spmm_handle_t h, int64_t N);
  * Split windows are merged by a fixed-order sum, so results are run-to-run identical.
  * A BCSR handle with row groups launches its kernel twice (groups, then the other block-rows;
  * the second launch starts on the SMs the first leaves idle and does not finish before it).
+ * A BCSR plan that cuts long block-rows (opts.k_split) keeps the parts' partial tiles in a
+ * workspace of the handle as well (allocated with the plan) and adds a small merge kernel.
  */
 int spmm_run(spmm_handle_t h, const void *B_dev, void *C_dev, int64_t N, void *stream);
 

@@ -307,6 +307,51 @@ def bcsr_tile_schedule(block_row_ptr, n_tt, slab_w, n_ctas, fixed_cost=4, units=
     return cta_ptr.astype(np.int32), tiles
 
 
+def bcsr_k_split(block_row_ptr, n_tt, n_ctas, fixed_cost=4, min_cap=8):
+    """K-split of outlier block-rows (the static-schedule answer to the imbalance Sec. 3.5 / 3.6
+    discuss: a block-row far longer than the rest makes tiles that no assignment can balance).
+
+    cap = max(min_cap, ceil(n_tt * sum over all block-rows of (stored blocks + fixed_cost) /
+    (4 * n_ctas))): a quarter of one CTA's mean load.  A block-row with more stored blocks than cap is
+    cut into parts = ceil(len / cap) contiguous ranges of its stored blocks, part j = blocks
+    [floor(j * len / parts), floor((j + 1) * len / parts)) of the row; every part computes a partial
+    C tile and the parts are summed in part order afterwards.
+
+    Returns None when no block-row exceeds cap, else int32 [n_units, 4] rows (block-row, first
+    stored block, end stored block, slot): block-rows in bcsr_row_order, parts in order; slot = -1
+    for an unsplit row, else the running index of the part counted over the split rows in ascending
+    block-row index (parts ascending).
+    """
+    brp = np.asarray(block_row_ptr, dtype=np.int64)
+    lens = np.diff(brp)
+    total = int((lens + fixed_cost).sum()) * n_tt
+    cap = max(min_cap, -(-total // (4 * n_ctas)))
+    if lens.size == 0 or int(lens.max()) <= cap:
+        return None
+    first_slot = {}
+    nslots = 0
+    for I in range(lens.shape[0]):
+        if lens[I] > cap:
+            first_slot[I] = nslots
+            nslots += -(-int(lens[I]) // cap)
+    units = []
+    for I in bcsr_row_order(brp).tolist():
+        L = int(lens[I])
+        if L <= cap:
+            units.append((I, int(brp[I]), int(brp[I + 1]), -1))
+        else:
+            parts = -(-L // cap)
+            for j in range(parts):
+                units.append((I, int(brp[I]) + j * L // parts, int(brp[I]) + (j + 1) * L // parts, first_slot[I] + j))
+    return np.asarray(units, dtype=np.int32).reshape(-1, 4)
+
+
+def bcsr_k_split_order(units):
+    """Schedule order of the K-split units: most stored blocks first, stable."""
+    ln = (units[:, 2] - units[:, 1]).astype(np.int64)
+    return np.argsort(-ln, kind="stable").astype(np.int32)
+
+
 def bcsr_row_groups(block_row_ptr, block_col_idx, b, min_fill_pct):
     """Row groups of the BCSR kernel (a device-side regrouping with no counterpart in the
     paper, whose BCSR blocks are all b x b, Sec. 2.3): R = 128 // b block-rows that store

@@ -41,6 +41,7 @@ SPMM_ERR_DEV_UNDRAINED = -11
 X_BCSR_BLOCK_ROW_PTR, X_BCSR_BLOCK_COL_IDX, X_BCSR_BLOCKS, X_BCSR_ROW_ORDER = 0, 1, 2, 3
 X_BCSR_TILE_PTR, X_BCSR_TILES = 4, 5
 X_BCSR_STACK_ROWS, X_BCSR_STACK_PTR, X_BCSR_STACK_COL_IDX, X_BCSR_STACK_TILE_PTR, X_BCSR_STACK_TILES = 6, 7, 8, 9, 20
+X_BCSR_UNITS = 21
 X_WCSR_WINDOW_ROW_PTR, X_WCSR_WINDOW_COL_IDX, X_WCSR_VALUES, X_WCSR_TASKS = 10, 11, 12, 13
 X_WCSR_BIN_PTR, X_WCSR_BIN_TASKS = 14, 15
 
@@ -55,7 +56,8 @@ EXPORTED_SYMBOLS = (
 class SpmmOpts(ctypes.Structure):
     _fields_ = [("b_col", ctypes.c_int32), ("split_cols", ctypes.c_int32), ("host_only", ctypes.c_int32),
                 ("n_ctas", ctypes.c_int32), ("c_type", ctypes.c_int32), ("layout", ctypes.c_int32),
-                ("schedule", ctypes.c_int32), ("stack_min_fill", ctypes.c_int32), ("gather", ctypes.c_int32), ("reserved", ctypes.c_int32 * 7)]
+                ("schedule", ctypes.c_int32), ("stack_min_fill", ctypes.c_int32), ("gather", ctypes.c_int32), ("k_split", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 6)]
 
 
 class SpmmInfo(ctypes.Structure):
@@ -123,13 +125,14 @@ GATHER_TMA, GATHER_LSU = 0, 1
 
 
 def _opts(b_col=0, split_cols=0, host_only=False, n_ctas=0, c_type=C_FP32, layout=ROWMAJOR, schedule=SCHED_STATIC,
-          stack_min_fill=0, gather=GATHER_TMA):
+          stack_min_fill=0, gather=GATHER_TMA, k_split=0):
     """Keyword options of the create functions -> spmm_opts_t (zero = the library's default; the
     header documents every field).  stack_min_fill: BCSR row groups, 0 = default threshold,
     -1 = off, 1..100 = minimum percentage of stored sub-blocks for a group to be formed."""
     o = SpmmOpts()
     o.stack_min_fill = int(stack_min_fill)
     o.gather = int(gather)
+    o.k_split = int(k_split)
     o.b_col, o.split_cols, o.host_only, o.n_ctas = b_col, split_cols, int(bool(host_only)), n_ctas
     o.c_type, o.layout, o.schedule = int(c_type), int(layout), int(schedule)
     return o

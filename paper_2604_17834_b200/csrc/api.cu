@@ -118,6 +118,11 @@ struct spmm_handle_s {
     CUtensorMap tmAs;                // map of d_svals
     CUtensorMap tmB3s;               // whole-tile map of B for the stacked launch's 256-token tile
     bool tmB3s_ok = false;
+    int k_split = 0;                 // opts.k_split (1: cut outlier block-rows into parts)
+    int32_t* d_kmerge = nullptr;     // K-split merge lists: row | first slot | parts, each [n_kmerge]
+    int n_kmerge = 0;
+    CUtensorMap tmP;                 // store map of the K-split partial tiles
+    bool tmP_ok = false;
     int32_t* d_tiles = nullptr;      // {block-row, token tile} pairs (the exported schedule)
     int32_t* d_tile_recs = nullptr;  // the kernel's records: {block-row, token tile, first block, end block}
     int32_t* d_cta_ptr = nullptr;
@@ -173,6 +178,7 @@ void free_handle(spmm_handle_s* h) {
         cudaFree(h->d_tiles);
         cudaFree(h->d_tile_recs);
         cudaFree(h->d_cta_ptr);
+        cudaFree(h->d_kmerge);
         cudaFree(h->d_sidx);
         cudaFree(h->d_srows);
         cudaFree(h->d_svals);
@@ -257,6 +263,7 @@ int new_bcsr_handle(spmm_handle_s** hp, int64_t m, int64_t k, int dtype, int blo
     h->col_major = opts && opts->layout == SPMM_COLMAJOR;
     h->dynamic = opts && opts->schedule == SPMM_SCHED_DYNAMIC;
     h->stack_min_fill = opts ? opts->stack_min_fill : 0;
+    h->k_split = opts ? opts->k_split : 0;
     if (h->stack_min_fill > 100) { delete h; return SPMM_ERR_INVALID_ARG; }
     if (h->dynamic && (h->c16 || h->col_major)) { delete h; return SPMM_ERR_UNSUPPORTED; }
     // column-major operands: rows of X (k elements) and of Y (m elements) must be multiples of
@@ -658,7 +665,24 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
         const int64_t n_tt_groups = (N + 128 * kStackGroups - 1) / (128 * kStackGroups);
         const bool use_groups = st.ng > 0 && (f.b <= 32 || st.ng * n_tt_groups >= h->n_ctas);
         if (!use_groups) {
-            rc = build_bcsr_schedule(f, n_tt, static_cast<int>(sw), h->dynamic ? 1 : h->n_ctas, &sc);
+            // K-split of outlier block-rows: static schedule, fp32 row-major C (the parts' partial
+            // tiles are fp32 and go through the same epilogue as C)
+            rc = SPMM_OK;
+            // (opt-in: measured 2 - 7 % slower than the uncut plan on the skewed sweep -- the parts'
+            // extra epilogues and the merge launch cost more than the better balance returns)
+            if (!h->dynamic && !h->c16 && !h->col_major && h->k_split > 0)
+                rc = build_bcsr_ksplit(f, n_tt, h->n_ctas, &sc.units, &sc.n_slots, &sc.cap);
+            if (!rc && !sc.units.empty()) {
+                const int32_t nu = static_cast<int32_t>(sc.units.size() / 4);
+                std::vector<int32_t> order(static_cast<size_t>(nu)), lens(static_cast<size_t>(nu));
+                for (int32_t u = 0; u < nu; ++u) order[u] = u;
+                auto ulen = [&](int32_t u) { return sc.units[4 * u + 2] - sc.units[4 * u + 1]; };
+                std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return ulen(x) > ulen(y); });
+                for (int32_t r = 0; r < nu; ++r) lens[r] = ulen(order[r]);
+                rc = build_tile_schedule(order, lens, kTileFixedCost, n_tt, static_cast<int>(sw), h->n_ctas, &sc);
+            } else if (!rc) {
+                rc = build_bcsr_schedule(f, n_tt, static_cast<int>(sw), h->dynamic ? 1 : h->n_ctas, &sc);
+            }
         } else {
             // The row groups get a launch and a schedule of their own; the launch of the remaining
             // block-rows starts on the SMs the first one leaves idle, CTA after CTA as they free up.
@@ -707,7 +731,10 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
             cudaFree(h->d_cta_ptr);
             cudaFree(h->d_stile_recs);
             cudaFree(h->d_scta_ptr);
-            h->d_tiles = h->d_tile_recs = h->d_cta_ptr = h->d_stile_recs = h->d_scta_ptr = nullptr;
+            cudaFree(h->d_kmerge);
+            h->d_tiles = h->d_tile_recs = h->d_cta_ptr = h->d_stile_recs = h->d_scta_ptr = h->d_kmerge = nullptr;
+            h->n_kmerge = 0;
+            h->tmP_ok = false;
         }
         rc = upload(&h->d_tiles, sc.tiles.data(), sc.tiles.size() * 4);
         if (!rc) {
@@ -715,13 +742,63 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
             const size_t nt = sc.tiles.size() / 2;
             std::vector<int32_t> recs(4 * nt);
             for (size_t i = 0; i < nt; ++i) {
-                const int32_t I = sc.tiles[2 * i];
-                recs[4 * i] = I;
                 recs[4 * i + 1] = sc.tiles[2 * i + 1];
-                recs[4 * i + 2] = f.block_row_ptr[I];
-                recs[4 * i + 3] = f.block_row_ptr[I + 1];
+                if (sc.units.empty()) {
+                    const int32_t I = sc.tiles[2 * i];
+                    recs[4 * i] = I;
+                    recs[4 * i + 2] = f.block_row_ptr[I];
+                    recs[4 * i + 3] = f.block_row_ptr[I + 1];
+                } else {
+                    // K-split: the tile names a unit {block-row, first block, end block, slot}; a part
+                    // carries -1 - slot in place of the block-row
+                    const int32_t* u = &sc.units[4 * static_cast<size_t>(sc.tiles[2 * i])];
+                    recs[4 * i] = u[3] < 0 ? u[0] : -1 - u[3];
+                    recs[4 * i + 2] = u[1];
+                    recs[4 * i + 3] = u[2];
+                }
             }
             rc = upload(&h->d_tile_recs, recs.data(), recs.size() * 4);
+        }
+        if (!rc && sc.n_slots > 0) {
+            // merge lists (split block-rows in ascending order: their slots are consecutive), the
+            // partial tiles' workspace and its store map
+            std::vector<int32_t> rows, firsts, parts;
+            for (size_t u = 0; u < sc.units.size() / 4; ++u) {
+                const int32_t I = sc.units[4 * u], slot = sc.units[4 * u + 3];
+                if (slot < 0) continue;
+                size_t j = 0;
+                while (j < rows.size() && rows[j] != I) ++j;
+                if (j == rows.size()) { rows.push_back(I); firsts.push_back(slot); parts.push_back(0); }
+                firsts[j] = std::min(firsts[j], slot);
+                parts[j]++;
+            }
+            std::vector<int32_t> mg;
+            mg.insert(mg.end(), rows.begin(), rows.end());
+            mg.insert(mg.end(), firsts.begin(), firsts.end());
+            mg.insert(mg.end(), parts.begin(), parts.end());
+            h->n_kmerge = static_cast<int>(rows.size());
+            rc = upload(&h->d_kmerge, mg.data(), mg.size() * 4);
+            const size_t need = static_cast<size_t>(sc.n_slots) * f.b * static_cast<size_t>(N) * 4;
+            if (!rc && need > h->partial_bytes) {
+                cudaFree(h->d_partial);
+                h->d_partial = nullptr;
+                h->partial_bytes = 0;
+                if (cudaMalloc(reinterpret_cast<void**>(&h->d_partial), need) != cudaSuccess) rc = SPMM_ERR_ALLOC;
+                else h->partial_bytes = need;
+            }
+            if (!rc) {
+                EncodeTiledFn fn = get_encode_fn();
+                const cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(sc.n_slots) * f.b};
+                const cuuint64_t strides[1] = {static_cast<cuuint64_t>(N) * 4};
+                const cuuint32_t box[2] = {32, static_cast<cuuint32_t>(bcsr_epi_cols(f.b, false, false))};
+                const cuuint32_t estr[2] = {1, 1};
+                if (!fn || fn(&h->tmP, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, h->d_partial, dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                    rc = SPMM_ERR_CUDA;
+                else
+                    h->tmP_ok = true;
+            }
         }
         if (!rc) rc = upload(&h->d_cta_ptr, sc.cta_ptr.data(), sc.cta_ptr.size() * 4);
         if (!rc && !ss.tiles.empty()) {
@@ -783,7 +860,7 @@ int run_bcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t s
         ps.use_3d = h->tmB3s_ok ? 1 : 0;
         ps.overlap = 1;
         p.overlap = 2;
-        cudaError_t es = launch_bcsr_stacked(h->dtype, f.b, h->c16, h->col_major, h->tmAs, h->tmB, h->tmB3s, h->tmC, ps,
+        cudaError_t es = launch_bcsr_stacked(h->dtype, f.b, h->c16, h->col_major, h->tmAs, h->tmB, h->tmB3s, h->tmC, h->tmC, ps,
                                              h->n_ctas, stream);
         if (es != cudaSuccess) return SPMM_ERR_CUDA;
         if (h->sched.tiles.empty()) return SPMM_OK;
@@ -791,9 +868,25 @@ int run_bcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t s
     // dynamic: one CTA per tile, the schedule was built as a single list in the global order
     const int grid = h->dynamic ? static_cast<int>(h->sched.tiles.size() / 2) : h->n_ctas;
     if (grid <= 0) return SPMM_OK;
+    const bool ksplit = h->sched.n_slots > 0 && h->tmP_ok;
+    if (ksplit) p.overlap = 1;          // the merge kernel's CTAs may be placed while this grid runs
     cudaError_t e = launch_bcsr(h->dtype, f.b, h->sched.groups, h->c16, h->col_major, h->dynamic, tmA, h->tmB, h->tmB3,
-                                h->tmC, p, grid, stream);
-    return e == cudaSuccess ? SPMM_OK : SPMM_ERR_CUDA;
+                                h->tmC, ksplit ? h->tmP : h->tmC, p, grid, stream);
+    if (e != cudaSuccess) return SPMM_ERR_CUDA;
+    if (ksplit) {
+        BcsrMergeParams mp;
+        mp.row = h->d_kmerge;
+        mp.first = h->d_kmerge + h->n_kmerge;
+        mp.nparts = h->d_kmerge + 2 * h->n_kmerge;
+        mp.partial = h->d_partial;
+        mp.C = static_cast<float*>(C);
+        mp.m = h->m;
+        mp.N = N;
+        mp.n = h->n_kmerge;
+        mp.b = f.b;
+        if (launch_bcsr_merge(mp, stream) != cudaSuccess) return SPMM_ERR_CUDA;
+    }
+    return SPMM_OK;
 }
 
 int64_t wcsr_workspace_bytes(const spmm_handle_s* h, int64_t N) {
@@ -1136,6 +1229,17 @@ int spmm_get_info(spmm_handle_t h, int64_t N, spmm_info_t* info) {
         info->n_stacked_rows = static_cast<int32_t>(h->stack.rows.size());
         info->n_stack_blocks = h->stack.ns;
         if (h->sched.N >= 0) {
+            info->n_slots = h->sched.n_slots;
+            info->n_split = h->n_kmerge;
+            if (h->host_only && h->sched.n_slots > 0) {
+                int64_t ns = 0, last = -1;
+                for (size_t u = 0; u < h->sched.units.size() / 4; ++u)
+                    if (h->sched.units[4 * u + 3] >= 0 && h->sched.units[4 * u] != last) { last = h->sched.units[4 * u]; ++ns; }
+                info->n_split = ns;
+            }
+            info->n_tasks = static_cast<int64_t>(h->sched.units.size() / 4);
+            info->split_cols = h->sched.cap;
+            info->workspace_bytes = h->sched.n_slots * f.b * h->sched.N * 4;
             info->plan_n = h->sched.N;
             info->plan_token_tile = 128 * h->sched.groups;
             info->plan_slab_tiles = h->sched.slab_w;
@@ -1187,6 +1291,9 @@ int spmm_export(spmm_handle_t h, int which, void* host_dst, size_t cap, size_t* 
             case SPMM_X_BCSR_TILES:
                 if (h->sched.N < 0) return SPMM_ERR_INVALID_ARG;
                 bytes = h->sched.tiles.size() * 4; dev_src = h->d_tiles; host_src = h->sched.tiles.data(); break;
+            case SPMM_X_BCSR_UNITS:
+                if (h->sched.N < 0) return SPMM_ERR_INVALID_ARG;
+                bytes = h->sched.units.size() * 4; host_src = h->sched.units.data(); host_copy = true; break;
             // the row-group plan lives on the host in every mode
             case SPMM_X_BCSR_STACK_ROWS: bytes = h->stack.rows.size() * 4; host_src = h->stack.rows.data(); host_copy = true; break;
             case SPMM_X_BCSR_STACK_PTR: bytes = h->stack.ptr.size() * 4; host_src = h->stack.ptr.data(); host_copy = true; break;

@@ -116,7 +116,8 @@ constexpr int kSchedDepth = 4;      // tile indices fetched ahead by the dynamic
 template <int B, int H, int GROUPS, int STAGES, int FMT, int CT, int CM, int DYN>
 __global__ void __launch_bounds__(DYN ? 224 : 192, 1)
 bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                 const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ CUtensorMap tmC, const BcsrParams p) {
+                 const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ CUtensorMap tmC,
+                 const __grid_constant__ CUtensorMap tmP, const BcsrParams p) {
     constexpr int ES = FMT == 3 ? 1 : (FMT == 2 ? 4 : 2);
     static_assert(ES != 1 || CM, "8-bit inputs: column-major operands only");
     static_assert(FMT != 2 || (!CT && !DYN && H == B), "TF32: fp32 C, static schedule, no row groups");
@@ -158,6 +159,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         prefetch_tmap(&tmB);
         prefetch_tmap(&tmB3);
         prefetch_tmap(&tmC);
+        prefetch_tmap(&tmP);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);
@@ -406,7 +408,11 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if constexpr (H != B) member = lane < H / B ? __ldg(p.stack_rows + tI * (H / B) + lane) : 0;
             if (!__all_sync(0xffffffffu, mbar_wait(accf_bar(acc), aph, ctl, 4))) { ok = false; break; }
             tc_fence_after_sync();
-            const int64_t row0 = static_cast<int64_t>(tI) * B;
+            // K-split: a tile of one part of a long block-row (record x = -1 - slot) writes its fp32
+            // partial tile, rows slot * b .. of the partial array, instead of C (fp32 row-major C only)
+            const bool part = tI < 0;
+            const int64_t row0 = static_cast<int64_t>(part ? -1 - tI : tI) * B;
+            const CUtensorMap* tm_out = part ? &tmP : &tmC;
             constexpr int W = Cfg::kEpiCols;                // accumulator columns per staging tile
             for (int g = 0; g < ngrp; ++g) {
                 const int nw = n0 + g * 128 + qd * 32;          // first token of this warp
@@ -473,8 +479,8 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (lane == 0) {
                         // row-major: box = 32 tokens x W rows at (token, row); column-major: box =
                         // W columns x 32 tokens at (column, token).  Out-of-range parts are clipped.
-                        if constexpr (!CM) tma_store_2d(&tmC, stg, nw, crow);
-                        else tma_store_2d(&tmC, stg, crow, nw);
+                        if constexpr (!CM) tma_store_2d(tm_out, stg, nw, crow);
+                        else tma_store_2d(tm_out, stg, crow, nw);
                         bulk_commit_group();
                     }
                 }
@@ -532,7 +538,7 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 // CAP = the deepest ring the shape is given; the ring actually used also leaves room for the
 // epilogue's staging tiles (bcsr_fit_stages).
 template <int B, int H, int GROUPS, int CAP, int FMT, int CT, int CM, int DYN>
-cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p,
+cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const CUtensorMap& tmP, const BcsrParams& p,
                        int grid, cudaStream_t stream) {
     constexpr int ES = FMT == 3 ? 1 : (FMT == 2 ? 4 : 2);
     constexpr int CS = static_cast<int>(sizeof(typename CType<FMT, CT>::type));
@@ -565,27 +571,27 @@ cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUt
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, kfn, tmA, tmB, tmB3, tmC, p);
+        return cudaLaunchKernelEx(&cfg, kfn, tmA, tmB, tmB3, tmC, tmP, p);
     }
-    kfn<<<grid, DYN ? 224 : 192, Cfg::kSmemBytes, stream>>>(tmA, tmB, tmB3, tmC, p);
+    kfn<<<grid, DYN ? 224 : 192, Cfg::kSmemBytes, stream>>>(tmA, tmB, tmB3, tmC, tmP, p);
     return cudaGetLastError();
 }
 
 template <int FMT, int CT, int CM, int DYN>
 cudaError_t launch_shape(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
-                         const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
+                         const CUtensorMap& tmC, const CUtensorMap& tmP, const BcsrParams& p, int grid, cudaStream_t stream) {
     switch (b * 10 + groups) {
-        case 161: return launch_one<16, 16, 1, 10, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 162: return launch_one<16, 16, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 164: return launch_one<16, 16, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 321: return launch_one<32, 32, 1, 10, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 322: return launch_one<32, 32, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 324: return launch_one<32, 32, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 641: return launch_one<64, 64, 1, 8, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 642: return launch_one<64, 64, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 644: return launch_one<64, 64, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 1281: return launch_one<128, 128, 1, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 1282: return launch_one<128, 128, 2, 2, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 161: return launch_one<16, 16, 1, 10, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 162: return launch_one<16, 16, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 164: return launch_one<16, 16, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 321: return launch_one<32, 32, 1, 10, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 322: return launch_one<32, 32, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 324: return launch_one<32, 32, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 641: return launch_one<64, 64, 1, 8, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 642: return launch_one<64, 64, 2, 5, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 644: return launch_one<64, 64, 4, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 1281: return launch_one<128, 128, 1, 3, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 1282: return launch_one<128, 128, 2, 2, FMT, CT, CM, DYN>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -593,37 +599,37 @@ cudaError_t launch_shape(int b, int groups, const CUtensorMap& tmA, const CUtens
 // Stacked blocks (row groups): 128 rows x b, token tile 256, four stages of 48 KB.
 template <int FMT, int CT, int CM>
 cudaError_t launch_stack_shape(int b, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
-                               const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
+                               const CUtensorMap& tmC, const CUtensorMap& tmP, const BcsrParams& p, int grid, cudaStream_t stream) {
     switch (b) {
-        case 16: return launch_one<16, 128, 2, 4, FMT, CT, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 32: return launch_one<32, 128, 2, 4, FMT, CT, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 64: return launch_one<64, 128, 2, 4, FMT, CT, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 16: return launch_one<16, 128, 2, 4, FMT, CT, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 32: return launch_one<32, 128, 2, 4, FMT, CT, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 64: return launch_one<64, 128, 2, 4, FMT, CT, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
         default: return cudaErrorInvalidValue;
     }
 }
 
 template <int FMT>
 cudaError_t launch_stack_fmt(int b, int c16, int cm, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
-                             const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
-    if (cm) return c16 ? launch_stack_shape<FMT, 1, 1>(b, tmA, tmB, tmB3, tmC, p, grid, stream)
-                       : launch_stack_shape<FMT, 0, 1>(b, tmA, tmB, tmB3, tmC, p, grid, stream);
-    return c16 ? launch_stack_shape<FMT, 1, 0>(b, tmA, tmB, tmB3, tmC, p, grid, stream)
-               : launch_stack_shape<FMT, 0, 0>(b, tmA, tmB, tmB3, tmC, p, grid, stream);
+                             const CUtensorMap& tmC, const CUtensorMap& tmP, const BcsrParams& p, int grid, cudaStream_t stream) {
+    if (cm) return c16 ? launch_stack_shape<FMT, 1, 1>(b, tmA, tmB, tmB3, tmC, tmP, p, grid, stream)
+                       : launch_stack_shape<FMT, 0, 1>(b, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+    return c16 ? launch_stack_shape<FMT, 1, 0>(b, tmA, tmB, tmB3, tmC, tmP, p, grid, stream)
+               : launch_stack_shape<FMT, 0, 0>(b, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
 }
 
 // E4M3 inputs: column-major operands, fp32 C, static schedule; b = 32, 64 or 128 (a block row
 // must hold at least one 32-element K step).  Stages are half the bytes of the 16-bit ones.
 cudaError_t launch_fp8(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
-                       const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
+                       const CUtensorMap& tmC, const CUtensorMap& tmP, const BcsrParams& p, int grid, cudaStream_t stream) {
     switch (b * 10 + groups) {
-        case 321: return launch_one<32, 32, 1, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 322: return launch_one<32, 32, 2, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 324: return launch_one<32, 32, 4, 6, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 641: return launch_one<64, 64, 1, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 642: return launch_one<64, 64, 2, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 644: return launch_one<64, 64, 4, 5, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 1281: return launch_one<128, 128, 1, 6, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 1282: return launch_one<128, 128, 2, 4, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 321: return launch_one<32, 32, 1, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 322: return launch_one<32, 32, 2, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 324: return launch_one<32, 32, 4, 6, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 641: return launch_one<64, 64, 1, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 642: return launch_one<64, 64, 2, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 644: return launch_one<64, 64, 4, 5, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 1281: return launch_one<128, 128, 1, 6, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 1282: return launch_one<128, 128, 2, 4, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -631,30 +637,30 @@ cudaError_t launch_fp8(int b, int groups, const CUtensorMap& tmA, const CUtensor
 // TF32 (fp32 storage): fp32 C, static schedule; the deepest rings the stage sizes allow.
 template <int CM>
 cudaError_t launch_tf32(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
-                        const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
+                        const CUtensorMap& tmC, const CUtensorMap& tmP, const BcsrParams& p, int grid, cudaStream_t stream) {
     switch (b * 10 + groups) {
-        case 161: return launch_one<16, 16, 1, 5, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 162: return launch_one<16, 16, 2, 3, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 321: return launch_one<32, 32, 1, 5, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 322: return launch_one<32, 32, 2, 3, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 641: return launch_one<64, 64, 1, 8, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 642: return launch_one<64, 64, 2, 5, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 644: return launch_one<64, 64, 4, 3, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 1281: return launch_one<128, 128, 1, 6, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        case 1282: return launch_one<128, 128, 2, 4, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        case 161: return launch_one<16, 16, 1, 5, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 162: return launch_one<16, 16, 2, 3, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 321: return launch_one<32, 32, 1, 5, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 322: return launch_one<32, 32, 2, 3, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 641: return launch_one<64, 64, 1, 8, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 642: return launch_one<64, 64, 2, 5, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 644: return launch_one<64, 64, 4, 3, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 1281: return launch_one<128, 128, 1, 6, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 1282: return launch_one<128, 128, 2, 4, 2, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
         default: return cudaErrorInvalidValue;
     }
 }
 
 template <int FMT>
 cudaError_t launch_fmt(int b, int groups, int c16, int cm, int dyn, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                       const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p, int grid, cudaStream_t stream) {
+                       const CUtensorMap& tmB3, const CUtensorMap& tmC, const CUtensorMap& tmP, const BcsrParams& p, int grid, cudaStream_t stream) {
     // dynamic scheduling is built for the default output (fp32, row-major) only
-    if (dyn) return (c16 || cm) ? cudaErrorInvalidValue : launch_shape<FMT, 0, 0, 1>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
-    if (cm) return c16 ? launch_shape<FMT, 1, 1, 0>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream)
-                       : launch_shape<FMT, 0, 1, 0>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
-    return c16 ? launch_shape<FMT, 1, 0, 0>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream)
-               : launch_shape<FMT, 0, 0, 0>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
+    if (dyn) return (c16 || cm) ? cudaErrorInvalidValue : launch_shape<FMT, 0, 0, 1>(b, groups, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+    if (cm) return c16 ? launch_shape<FMT, 1, 1, 0>(b, groups, tmA, tmB, tmB3, tmC, tmP, p, grid, stream)
+                       : launch_shape<FMT, 0, 1, 0>(b, groups, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+    return c16 ? launch_shape<FMT, 1, 0, 0>(b, groups, tmA, tmB, tmB3, tmC, tmP, p, grid, stream)
+               : launch_shape<FMT, 0, 0, 0>(b, groups, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
 }
 
 }  // namespace
@@ -672,31 +678,88 @@ int bcsr_token_groups_max(int dtype, int b, int c16, int col_major) {
 }
 
 cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, int dynamic, const CUtensorMap& tmA,
-                        const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p,
+                        const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const CUtensorMap& tmP, const BcsrParams& p,
                         int grid, cudaStream_t stream) {
-    if (dtype == 1) return launch_fmt<0>(b, groups, c16, col_major, dynamic, tmA, tmB, tmB3, tmC, p, grid, stream);   // fp16
-    if (dtype == 0) return launch_fmt<1>(b, groups, c16, col_major, dynamic, tmA, tmB, tmB3, tmC, p, grid, stream);   // bf16
+    if (dtype == 1) return launch_fmt<0>(b, groups, c16, col_major, dynamic, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);   // fp16
+    if (dtype == 0) return launch_fmt<1>(b, groups, c16, col_major, dynamic, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);   // bf16
     if (dtype == 3) return (c16 || !col_major || dynamic) ? cudaErrorInvalidValue
-                                                           : launch_fp8(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
+                                                           : launch_fp8(b, groups, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
     if (dtype == 2) {
         if (c16 || dynamic) return cudaErrorInvalidValue;
-        return col_major ? launch_tf32<1>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream)
-                         : launch_tf32<0>(b, groups, tmA, tmB, tmB3, tmC, p, grid, stream);
+        return col_major ? launch_tf32<1>(b, groups, tmA, tmB, tmB3, tmC, tmP, p, grid, stream)
+                         : launch_tf32<0>(b, groups, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
     }
     return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_bcsr_stacked(int dtype, int b, int c16, int col_major, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                                const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p, int grid,
+                                const CUtensorMap& tmB3, const CUtensorMap& tmC, const CUtensorMap& tmP, const BcsrParams& p, int grid,
                                 cudaStream_t stream) {
-    if (dtype == 1) return launch_stack_fmt<0>(b, c16, col_major, tmA, tmB, tmB3, tmC, p, grid, stream);   // fp16
-    if (dtype == 0) return launch_stack_fmt<1>(b, c16, col_major, tmA, tmB, tmB3, tmC, p, grid, stream);   // bf16
+    if (dtype == 1) return launch_stack_fmt<0>(b, c16, col_major, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);   // fp16
+    if (dtype == 0) return launch_stack_fmt<1>(b, c16, col_major, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);   // bf16
     if (dtype == 3 && !c16 && col_major) {
         // E4M3: half the bytes per stage, twice the ring depth
-        if (b == 32) return launch_one<32, 128, 2, 8, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
-        if (b == 64) return launch_one<64, 128, 2, 8, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, p, grid, stream);
+        if (b == 32) return launch_one<32, 128, 2, 8, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        if (b == 64) return launch_one<64, 128, 2, 8, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
     }
     return cudaErrorInvalidValue;
+}
+
+namespace {
+
+// One CTA per (split block-row, run of 1024 four-column pieces of its b x N output); a thread sums
+// four pieces over the parts, in part order (run-to-run identical results), all loads of a
+// piece in flight together.
+constexpr int kMergePieces = 4;
+__global__ void __launch_bounds__(256) bcsr_merge_kernel(const BcsrMergeParams p) {
+    const int i = blockIdx.x;
+    const int I = p.row[i], first = p.first[i], nparts = p.nparts[i];
+    // the partial tiles belong to the SpMM kernel launched just before on the same stream
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int64_t N = p.N, n4 = N >> 2;                 // N is a multiple of 4 (16-byte rows)
+    const int64_t row0 = static_cast<int64_t>(I) * p.b;
+    const int64_t rows = min_i64(p.b, p.m - row0);
+    const int64_t total = rows * n4;
+    const float4* part = reinterpret_cast<const float4*>(p.partial) + static_cast<int64_t>(first) * p.b * n4;
+    float4* out = reinterpret_cast<float4*>(p.C + row0 * N);
+    const int64_t slot_stride = static_cast<int64_t>(p.b) * n4;
+    const int64_t e0 = static_cast<int64_t>(blockIdx.y) * (256 * kMergePieces) + threadIdx.x;
+    float4 acc[kMergePieces];
+#pragma unroll
+    for (int k = 0; k < kMergePieces; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < nparts; ++s) {
+#pragma unroll
+        for (int k = 0; k < kMergePieces; ++k) {
+            const int64_t e = e0 + k * 256;
+            if (e < total) {
+                const float4 v = __ldg(part + s * slot_stride + e);
+                acc[k].x += v.x; acc[k].y += v.y; acc[k].z += v.z; acc[k].w += v.w;
+            }
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < kMergePieces; ++k) {
+        const int64_t e = e0 + k * 256;
+        if (e < total) out[e] = acc[k];
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_bcsr_merge(const BcsrMergeParams& p, cudaStream_t stream) {
+    if (p.n <= 0) return cudaSuccess;
+    cudaLaunchConfig_t cfg = {};
+    const int64_t pieces = static_cast<int64_t>(p.b) * (p.N >> 2);
+    cfg.gridDim = dim3(static_cast<unsigned>(p.n), static_cast<unsigned>((pieces + 256 * kMergePieces - 1) / (256 * kMergePieces)));
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, bcsr_merge_kernel, p);
 }
 
 }  // namespace spmm

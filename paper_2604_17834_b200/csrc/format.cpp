@@ -2,6 +2,7 @@
 #include "format.h"
 
 #include <algorithm>
+#include <climits>
 #include <cstring>
 #include <numeric>
 #include <queue>
@@ -176,6 +177,49 @@ int build_bcsr_schedule(const BcsrHost& f, int n_tt, int slab_w, int n_ctas, Bcs
         lens[r] = f.block_row_ptr[I + 1] - f.block_row_ptr[I];
     }
     return build_tile_schedule(f.row_order, lens, kTileFixedCost, n_tt, slab_w, n_ctas, out);
+}
+
+int build_bcsr_ksplit(const BcsrHost& f, int n_tt, int n_ctas, std::vector<int32_t>* units, int64_t* n_slots, int32_t* cap_out) {
+    units->clear();
+    *n_slots = 0;
+    int64_t total = 0;
+    int32_t longest = 0;
+    for (int64_t I = 0; I < f.nbr; ++I) {
+        const int32_t len = f.block_row_ptr[I + 1] - f.block_row_ptr[I];
+        total += len + kTileFixedCost;
+        longest = std::max(longest, len);
+    }
+    total *= n_tt;
+    const int64_t quarter = (total + 4 * int64_t{n_ctas} - 1) / (4 * int64_t{n_ctas});
+    const int32_t cap = static_cast<int32_t>(std::min<int64_t>(std::max<int64_t>(kKSplitMinCap, quarter), INT32_MAX));
+    *cap_out = cap;
+    if (longest <= cap) return SPMM_OK;
+    // slots: split block-rows in ascending index, parts ascending
+    std::vector<int32_t> first_slot(static_cast<size_t>(f.nbr), -1);
+    int64_t slots = 0;
+    for (int64_t I = 0; I < f.nbr; ++I) {
+        const int32_t len = f.block_row_ptr[I + 1] - f.block_row_ptr[I];
+        if (len > cap) {
+            first_slot[I] = static_cast<int32_t>(slots);
+            slots += (len + cap - 1) / cap;
+        }
+    }
+    if (slots >= (int64_t{1} << 30)) return SPMM_ERR_TOO_LARGE;
+    for (int64_t r = 0; r < f.nbr; ++r) {
+        const int32_t I = f.row_order[r];
+        const int32_t p0 = f.block_row_ptr[I];
+        const int64_t len = f.block_row_ptr[I + 1] - p0;
+        if (len <= cap) {
+            units->insert(units->end(), {I, p0, static_cast<int32_t>(p0 + len), -1});
+            continue;
+        }
+        const int64_t parts = (len + cap - 1) / cap;
+        for (int64_t j = 0; j < parts; ++j)
+            units->insert(units->end(), {I, static_cast<int32_t>(p0 + j * len / parts), static_cast<int32_t>(p0 + (j + 1) * len / parts),
+                                         static_cast<int32_t>(first_slot[I] + j)});
+    }
+    *n_slots = slots;
+    return SPMM_OK;
 }
 
 int build_bcsr_stack(const BcsrHost& f, int min_fill_pct, BcsrStack* out) {

@@ -68,8 +68,22 @@ struct BcsrSchedule {
     int64_t N = -1;
     int groups = 0, n_tt = 0, slab_w = 0, n_ctas = 0;
     std::vector<int32_t> cta_ptr;    // [n_ctas+1]
-    std::vector<int32_t> tiles;      // 2 * n_tiles: {block-row, token tile}, CTA-major
+    std::vector<int32_t> tiles;      // 2 * n_tiles: {block-row (or K-split unit, below), token tile}, CTA-major
+    // K-split of outlier block-rows (empty when no block-row exceeds the cap): 4 * n_units
+    // {block-row, first stored block, end stored block, slot}; tiles[] then names units.
+    std::vector<int32_t> units;
+    int64_t n_slots = 0;             // partial tiles (one per part of a split block-row)
+    int32_t cap = 0;
 };
+// K-split: a block-row with more stored blocks than cap = max(kKSplitMinCap, ceil(n_tt * sum over
+// all block-rows of (stored blocks + kTileFixedCost) / (4 * n_ctas))) -- a quarter of a CTA's mean
+// load -- is cut into ceil(len / cap) contiguous ranges of its stored blocks, part j = blocks
+// [j * len / parts, (j + 1) * len / parts).  Each part computes a partial C tile (fp32, slot =
+// running index over the parts of split block-rows in ascending block-row order); the parts are
+// summed in part order by the merge kernel.  Units are listed block-rows in row_order, parts in
+// order; they are scheduled most stored blocks first (stable).  Returns the units (empty: no split).
+constexpr int kKSplitMinCap = 8;
+int build_bcsr_ksplit(const BcsrHost& f, int n_tt, int n_ctas, std::vector<int32_t>* units, int64_t* n_slots, int32_t* cap);
 // a tile's fixed cost in stored-block units: its epilogue writes b x BN x 4 bytes of C, a stored
 // block brings b x BN x 2 bytes of B (measured best of 2 / 4 / 6 / 10 on the skewed sweep)
 constexpr int kTileFixedCost = 4;

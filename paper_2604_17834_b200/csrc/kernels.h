@@ -44,15 +44,28 @@ struct BcsrParams {
 // dynamic: the grid is one CTA per tile (grid = number of tiles, p.tiles in the schedule's global
 // order, p.cta_ptr unused) and CTAs steal tiles through Cluster Launch Control; fp32 row-major only.
 cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, int dynamic, const CUtensorMap& tmA,
-                        const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p,
-                        int grid, cudaStream_t stream);
+                        const CUtensorMap& tmB, const CUtensorMap& tmB3, const CUtensorMap& tmC, const CUtensorMap& tmP,
+                        const BcsrParams& p, int grid, cudaStream_t stream);
 // Row groups: the same kernel with 128 x b stacked blocks (MMA N = 128) and a 256-token tile.
 // tmA: the stacked values as [blocks * 128][b], box 128 x b; tmB3 built for groups = 2; b = 16, 32, 64.
 constexpr int kStackRows = 128;
 constexpr int kStackGroups = 2;
 cudaError_t launch_bcsr_stacked(int dtype, int b, int c16, int col_major, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                                const CUtensorMap& tmB3, const CUtensorMap& tmC, const BcsrParams& p, int grid,
-                                cudaStream_t stream);
+                                const CUtensorMap& tmB3, const CUtensorMap& tmC, const CUtensorMap& tmP, const BcsrParams& p,
+                                int grid, cudaStream_t stream);
+// K-split: tmP = the partial tiles as [slots * b][N] fp32, box as tmC's (the tile record of a
+// part holds -1 - slot in place of the block-row); pass tmC where the plan has no parts.
+// The merge: C rows of every split block-row = sum of its parts' partial tiles in part order.
+struct BcsrMergeParams {
+    const int32_t* row;      // [n] split block-rows
+    const int32_t* first;    // first slot
+    const int32_t* nparts;
+    const float* partial;    // [slots][b][N]
+    float* C;                // [m][N]
+    int64_t m, N;
+    int32_t n, b;
+};
+cudaError_t launch_bcsr_merge(const BcsrMergeParams& p, cudaStream_t stream);
 int bcsr_token_groups_max(int dtype, int b, int c16, int col_major);
 // Accumulator columns (= rows of A's block) an epilogue warp handles at a time: it stages them
 // in a 2 KB (1 KB for b = 16 with 16-bit C) shared-memory tile and stores the tile with one TMA

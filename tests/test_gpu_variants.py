@@ -451,3 +451,31 @@ def test_wcsr_lsu_gather_argument_errors(lib):
     with pytest.raises(lib.SpmmError) as e:
         lib.spmm_wcsr_create_csr(256, 256, a["row_ptr"], a["col_idx"], a["vals"], "fp16", 16, gather=7)
     assert e.value.code == lib.SPMM_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("dtype,b,m,k,N", [("fp16", 64, 2048, 4096, 1024), ("bf16", 128, 1000, 4096, 1000),
+                                           ("tf32", 64, 1536, 2048, 520), ("fp16", 32, 2048, 2048, 768)])
+def test_bcsr_k_split_of_long_block_rows(lib, dtype, b, m, k, N):
+    """A few full block-rows among short ones: the plan cuts them into parts whose partial tiles a
+    second kernel adds in order.  Same oracle bound as the uncut plan, run-to-run identical bits, and
+    (parts only regroup the fp32 sum) agreement with the uncut result to fp32 rounding."""
+    a = wl.bcsr_sweep(700 + b, m=m, k=k, b=b, density=0.05, dtype=dtype)
+    Bs = wl.dense(41, k, N, ("normal", 0.0, 1.0), dtype)
+    h1 = lib.spmm_bcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, b, stack_min_fill=-1, k_split=1)
+    h0 = lib.spmm_bcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, b, stack_min_fill=-1)
+    try:
+        C1 = run_gpu(lib, h1, Bs, m, N)
+        info = lib.spmm_get_info(h1, N)
+        assert info["n_slots"] > 0 and info["n_split"] > 0 and info["workspace_bytes"] == info["n_slots"] * b * N * 4
+        units = lib.spmm_export(h1, lib.X_BCSR_UNITS, np.int32).reshape(-1, 4)
+        assert (units[:, 2] - units[:, 1]).max() <= info["split_cols"]
+        C0 = run_gpu(lib, h0, Bs, m, N)
+        assert lib.spmm_get_info(h0, N)["n_slots"] == 0
+        Cr, S = reference(a, Bs, dtype)
+        assert_close(C1, Cr, S, dtype, "bcsr with K-split %s b=%d" % (dtype, b))
+        assert_close(C0, Cr, S, dtype, "bcsr without K-split %s b=%d" % (dtype, b))
+        assert np.array_equal(C1, run_gpu(lib, h1, Bs, m, N))            # fixed summation order
+        assert np.max(np.abs(C1 - C0)) <= 1e-4 * max(1.0, float(S.max()))
+    finally:
+        lib.spmm_destroy(h0)
+        lib.spmm_destroy(h1)

@@ -91,11 +91,13 @@ def test_bcsr_workload_generators_round_trip(lib):
     lib.spmm_destroy(h)
 
 
-@pytest.mark.parametrize("b,N,n_ctas", [(64, 4096, 148), (16, 1024, 7), (128, 640, 5), (32, 200, 3)])
-def test_bcsr_tile_schedule_is_bit_exact_and_balanced(lib, b, N, n_ctas):
+@pytest.mark.parametrize("b,N,n_ctas,k_split", [(64, 4096, 148, 0), (16, 1024, 7, 0), (128, 640, 5, 0), (32, 200, 3, 0),
+                                                (64, 4096, 148, 1), (64, 1024, 148, 1), (128, 4096, 148, 1), (16, 4096, 148, 1),
+                                                (16, 1024, 7, 1)])
+def test_bcsr_tile_schedule_is_bit_exact_and_balanced(lib, b, N, n_ctas, k_split):
     s = wl.bcsr_sweep(55 + b, m=4096, k=2048, b=b, density=0.1)
     h = lib.spmm_bcsr_create_csr(4096, 2048, s["row_ptr"], s["col_idx"], s["vals"], "fp16", b, host_only=True,
-                                 n_ctas=n_ctas, stack_min_fill=-1)
+                                 n_ctas=n_ctas, stack_min_fill=-1, k_split=k_split)
     try:
         with pytest.raises(lib.SpmmError):
             lib.spmm_export(h, lib.X_BCSR_TILES, np.int32)          # no plan yet
@@ -105,16 +107,40 @@ def test_bcsr_tile_schedule_is_bit_exact_and_balanced(lib, b, N, n_ctas):
         bnt = info["plan_token_tile"]
         n_tt = -(-N // bnt)
         f = F.bcsr_from_csr(4096, 2048, s["row_ptr"], s["col_idx"], s["vals"], b)
-        want_ptr, want_tiles = F.bcsr_tile_schedule(f["block_row_ptr"], n_tt, info["plan_slab_tiles"], n_ctas)
+        brp = f["block_row_ptr"]
+        nbr = brp.shape[0] - 1
         got_ptr = lib.spmm_export(h, lib.X_BCSR_TILE_PTR, np.int32)
         got_tiles = lib.spmm_export(h, lib.X_BCSR_TILES, np.int32).reshape(-1, 2)
-        assert np.array_equal(got_ptr, want_ptr) and np.array_equal(got_tiles, want_tiles)
-        # every (block-row, token tile) exactly once
-        nbr = f["block_row_ptr"].shape[0] - 1
-        keys = got_tiles[:, 0].astype(np.int64) * n_tt + got_tiles[:, 1]
-        assert np.array_equal(np.sort(keys), np.arange(nbr * n_tt))
+        got_units = lib.spmm_export(h, lib.X_BCSR_UNITS, np.int32).reshape(-1, 4)
+        units = None if k_split <= 0 else F.bcsr_k_split(brp, n_tt, n_ctas)
+        if units is None:
+            assert got_units.size == 0 and info["n_slots"] == 0
+            want_ptr, want_tiles = F.bcsr_tile_schedule(brp, n_tt, info["plan_slab_tiles"], n_ctas)
+            assert np.array_equal(got_ptr, want_ptr) and np.array_equal(got_tiles, want_tiles)
+            # every (block-row, token tile) exactly once
+            keys = got_tiles[:, 0].astype(np.int64) * n_tt + got_tiles[:, 1]
+            assert np.array_equal(np.sort(keys), np.arange(nbr * n_tt))
+            cost = np.diff(brp)[got_tiles[:, 0]].astype(np.int64) + 4     # stored blocks + the fixed cost per tile
+        else:
+            # long block-rows cut into parts: the units, their schedule order and the tiles over them
+            assert np.array_equal(got_units, units)
+            order = F.bcsr_k_split_order(units)
+            ulen = (units[:, 2] - units[:, 1]).astype(np.int64)
+            want_ptr, want_tiles = F.bcsr_tile_schedule(None, n_tt, info["plan_slab_tiles"], n_ctas, units=order, lens=ulen[order])
+            assert np.array_equal(got_ptr, want_ptr) and np.array_equal(got_tiles, want_tiles)
+            assert info["n_slots"] == int((units[:, 3] >= 0).sum()) == units[:, 3].max() + 1
+            assert info["n_split"] == np.unique(units[units[:, 3] >= 0, 0]).shape[0] and info["n_tasks"] == units.shape[0]
+            assert info["workspace_bytes"] == info["n_slots"] * b * N * 4
+            # every (stored block, token tile) exactly once, and every empty block-row's tile as well
+            seen = np.zeros((int(brp[-1]), n_tt), dtype=np.int32)
+            rows_seen = np.zeros((nbr, n_tt), dtype=np.int32)
+            for u, t in got_tiles:
+                seen[units[u, 1]:units[u, 2], t] += 1
+                rows_seen[units[u, 0], t] += 1
+            assert np.all(seen == 1) and np.all(rows_seen >= 1)
+            cost = ulen[got_tiles[:, 0]] + 4
+            assert cost.max() - 4 <= info["split_cols"]            # no tile longer than the cap
         # greedy longest-first bound: no CTA exceeds the lightest by more than the heaviest tile
-        cost = np.diff(f["block_row_ptr"])[got_tiles[:, 0]].astype(np.int64) + 4     # stored blocks + the fixed cost per tile
         loads = np.array([cost[got_ptr[c]:got_ptr[c + 1]].sum() for c in range(n_ctas)])
         assert loads.max() - loads.min() <= cost.max()
         if N % 512 == 0 and b != 128 and nbr * (N // 512) >= 8 * n_ctas:

@@ -273,6 +273,80 @@ def test_default_split_cols_matches_plain_loops(seed, n_bins):
     assert F.default_split_cols(wp, 8) == _brute_split_size(wp, 8) < 4608
 
 
+def _brute_k_split(brp, n_tt, n_ctas, fixed=4, min_cap=8):
+    """K-split written with plain loops: cap, parts per long block-row, slots in ascending
+    block-row order, units in schedule order of the block-rows."""
+    lens = [brp[i + 1] - brp[i] for i in range(len(brp) - 1)]
+    total = n_tt * sum(l + fixed for l in lens)
+    cap = max(min_cap, (total + 4 * n_ctas - 1) // (4 * n_ctas))
+    if not lens or max(lens) <= cap:
+        return cap, None
+    slot_of, ns = {}, 0
+    for i, l in enumerate(lens):
+        if l > cap:
+            slot_of[i] = ns
+            ns += (l + cap - 1) // cap
+    order = sorted(range(len(lens)), key=lambda i: (-lens[i], i))
+    units = []
+    for i in order:
+        l = lens[i]
+        if l <= cap:
+            units.append((i, brp[i], brp[i + 1], -1))
+        else:
+            parts = (l + cap - 1) // cap
+            for j in range(parts):
+                units.append((i, brp[i] + j * l // parts, brp[i] + (j + 1) * l // parts, slot_of[i] + j))
+    return cap, units
+
+
+@pytest.mark.parametrize("seed,n_tt,n_ctas", [(1, 4, 16), (2, 1, 3), (3, 16, 148), (4, 2, 40), (5, 8, 148)])
+def test_k_split_matches_brute_force_and_tiles_the_rows(seed, n_tt, n_ctas):
+    rng = np.random.default_rng(seed)
+    lens = rng.choice([0, 0, 1, 2, 3, 5, 9, 17, 64, 64, 128], size=70)
+    brp = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    cap, want = _brute_k_split(brp.tolist(), n_tt, n_ctas)
+    got = F.bcsr_k_split(brp, n_tt, n_ctas)
+    if want is None:
+        assert got is None
+        return
+    assert got.dtype == np.int32 and [tuple(r) for r in got.tolist()] == want
+    # the parts of a block-row tile its stored blocks in order, none longer than cap, sizes within one of each other
+    for I in np.unique(got[:, 0]):
+        u = got[got[:, 0] == I]
+        assert u[0, 1] == brp[I] and u[-1, 2] == brp[I + 1] and np.all(u[1:, 1] == u[:-1, 2])
+        ln = u[:, 2] - u[:, 1]
+        assert ln.max() <= cap and ln.max() - ln.min() <= 1
+        assert (u.shape[0] == 1) == (u[0, 3] == -1)
+        if u.shape[0] > 1:
+            assert np.all(np.diff(u[:, 3]) == 1)
+    # slots number the parts of split rows in ascending block-row order
+    parts = got[got[:, 3] >= 0]
+    by_row = parts[np.lexsort((parts[:, 1], parts[:, 0]))]
+    assert np.array_equal(by_row[:, 3], np.arange(by_row.shape[0]))
+    # no unit longer than a quarter of a CTA's mean load (or the minimum cap)
+    total = n_tt * int((np.diff(brp) + 4).sum())
+    assert cap == max(8, -(-total // (4 * n_ctas)))
+    # schedule order: most stored blocks first, stable
+    o = F.bcsr_k_split_order(got)
+    ln = (got[:, 2] - got[:, 1])[o]
+    assert np.all(np.diff(ln) <= 0)
+    for a, b in zip(o[:-1], o[1:]):
+        if got[a, 2] - got[a, 1] == got[b, 2] - got[b, 1]:
+            assert a < b
+
+
+def test_k_split_special_cases():
+    # equal rows: nothing exceeds a quarter of the mean load unless there are very few of them
+    brp = np.arange(0, 65 * 10, 10, dtype=np.int32)
+    assert F.bcsr_k_split(brp, 4, 8) is None
+    # one row of 100 blocks among 99 single-block rows on 100 CTAs: cap = max(8, ceil(2 * 599 / 400)) = 8 -> 13 parts
+    brp = np.concatenate([[0], np.cumsum([100] + [1] * 99)]).astype(np.int32)
+    u = F.bcsr_k_split(brp, 2, 100)
+    parts = u[u[:, 0] == 0]
+    assert parts.shape[0] == 13 and parts[:, 3].tolist() == list(range(13))
+    assert (parts[:, 2] - parts[:, 1]).sum() == 100 and np.all(u[u[:, 0] > 0][:, 3] == -1)
+
+
 def test_generators_are_deterministic_and_shaped():
     a1, a2 = wl.bcsr_tiny(), wl.bcsr_tiny()
     assert np.array_equal(a1["col_idx"], a2["col_idx"]) and np.array_equal(a1["vals"], a2["vals"])
