@@ -132,6 +132,13 @@ def workload_table():
         return f
     t["cfg3_bcsr_llm_gate_cm_fp8"] = ("configs[2] gate shape with E4M3 weights and activations, X [N][k] in, fp32 Y [N][m] out",
                                       fp8_linear(18944, 3584, 1003))
+    def fp8_rowmajor(m, k, seed):
+        def f():
+            return dict(kind="bcsr", a=wl.bcsr_llm(seed=seed, m=m, k=k, dtype="fp8", std=0.5), dtype="fp8", size=64, N=65536,
+                        Bdist=("normal", 0.0, 1.0))
+        return f
+    t["cfg3_bcsr_llm_gate_fp8"] = ("configs[2] gate shape with E4M3 weights and activations, row-major operands, fp32 C",
+                                   fp8_rowmajor(18944, 3584, 1003))
     t["cfg3_bcsr_llm_down_cm_fp8"] = ("configs[2] down shape with E4M3 weights and activations, X [N][k] in, fp32 Y [N][m] out",
                                       fp8_linear(3584, 18944, 1013))
     t["cfg5_wcsr_rmat_s19_n128"] = ("configs[4] recipe at 2^19 rows (a profiling-sized case: B 134 MB), N=128",
@@ -197,7 +204,7 @@ ALL_OTHERS = DEFAULT_OTHERS + [
     "cfg4_bcsr_sweep_b64_d0.05", "cfg4_bcsr_sweep_b64_d0.01", "cfg4_bcsr_flat_b64_d0.05", "cfg4_bcsr_flat_b64_d0.01",
     "cfg3_bcsr_llm_gate_c16", "cfg3_bcsr_llm_gate_cm", "cfg3_bcsr_llm_gate_cm_c16",
     "cfg3_bcsr_llm_down_cm_c16", "cfg5_wcsr_rmat_n128_c16",
-    "cfg3_bcsr_llm_gate_cm_fp8", "cfg3_bcsr_llm_down_cm_fp8", "cfg2_wcsr_irregular_wh64", "cfg5_wcsr_rmat_n128_wh64",
+    "cfg3_bcsr_llm_gate_cm_fp8", "cfg3_bcsr_llm_down_cm_fp8", "cfg3_bcsr_llm_gate_fp8", "cfg2_wcsr_irregular_wh64", "cfg5_wcsr_rmat_n128_wh64",
     "cfg2_wcsr_irregular_lsu_gather", "cfg5_wcsr_rmat_n128_lsu_gather",
     "cfg4_bcsr_sweep_b64_d0.1_dyn", "cfg4_bcsr_sweep_b16_d0.1_plain", "cfg4_bcsr_sweep_b32_d0.1_plain",
     "cfg4_bcsr_sweep_b16_d0.5", "cfg4_bcsr_sweep_b32_d0.5",

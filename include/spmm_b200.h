@@ -70,8 +70,10 @@ typedef enum {
                                     both layouts; C is fp32, the BCSR schedule static, and
                                     BCSR row groups are not formed.                           */
     SPMM_FP8_E4M3 = 3            /* 1-byte E4M3 storage (Sec. 5 names 8-bit inputs as the next
-                                    step).  BCSR with SPMM_COLMAJOR only, fp32 C, block 32,
-                                    64 or 128, k % 16 == 0.                                   */
+                                    step).  BCSR only, fp32 C, static schedule, block 32, 64 or
+                                    128; row-major operands need N >= 128 and N % 16 == 0,
+                                    SPMM_COLMAJOR needs k % 16 == 0 (row groups are formed with
+                                    SPMM_COLMAJOR only).                                      */
 } spmm_dtype_t;
 
 /* Element type of C (opts.c_type).  Accumulation is fp32 either way. */

@@ -244,11 +244,11 @@ int new_bcsr_handle(spmm_handle_s** hp, int64_t m, int64_t k, int dtype, int blo
     // TF32 (Sec. 3.1's k8 shape, the type of Sec. 4.1's BCSR evaluation): static schedule only
     if (dtype == SPMM_TF32 && opts && opts->schedule != SPMM_SCHED_STATIC) return SPMM_ERR_UNSUPPORTED;
     if (dtype == SPMM_FP8_E4M3) {
-        // 8-bit inputs: the K-major (column-major operand) path only, fp32 C, static schedule; a block
-        // row must hold a whole 32-element K step; rows of X are k bytes and must be multiples of 16
-        if (!opts || opts->layout != SPMM_COLMAJOR || opts->c_type != SPMM_C_FP32 || opts->schedule != SPMM_SCHED_STATIC)
-            return SPMM_ERR_UNSUPPORTED;
-        if (block < 32 || k % 16 != 0) return SPMM_ERR_UNSUPPORTED;
+        // 8-bit inputs: fp32 C, static schedule; a block row must hold a whole 32-element K step;
+        // with column-major operands the rows of X are k bytes and must be multiples of 16
+        if (opts && (opts->c_type != SPMM_C_FP32 || opts->schedule != SPMM_SCHED_STATIC)) return SPMM_ERR_UNSUPPORTED;
+        if (block < 32) return SPMM_ERR_UNSUPPORTED;
+        if (opts && opts->layout == SPMM_COLMAJOR && k % 16 != 0) return SPMM_ERR_UNSUPPORTED;
     }
     spmm_handle_s* h = new (std::nothrow) spmm_handle_s;
     if (!h) return SPMM_ERR_ALLOC;
@@ -295,7 +295,9 @@ int encode_tmA(spmm_handle_s* h) {
 int setup_stack(spmm_handle_s* h) {
     const BcsrHost& f = h->bcsr;
     // static schedule only; b = 128 blocks already are 128 rows high
-    const bool eligible = !h->dynamic && f.b < 128 && h->stack_min_fill >= 0 && h->dtype != SPMM_TF32;
+    // (row groups exist for the 16-bit types, and for E4M3 with column-major operands)
+    const bool eligible = !h->dynamic && f.b < 128 && h->stack_min_fill >= 0 && h->dtype != SPMM_TF32 &&
+                          !(h->dtype == SPMM_FP8_E4M3 && !h->col_major);
     int rc = build_bcsr_stack(f, eligible ? h->stack_min_fill : -1, &h->stack);
     if (rc || h->host_only || h->stack.ng == 0) return rc;
     const BcsrStack& st = h->stack;
@@ -823,7 +825,8 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
 
 int run_bcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t stream) {
     const BcsrHost& f = h->bcsr;
-    if (N < (h->col_major ? 128 : 64)) return SPMM_ERR_UNSUPPORTED;   // the box is 64 (128) tokens wide
+    // the box of the dense operand is 64 tokens wide (128 with column-major operands or 1-byte values)
+    if (N < ((h->col_major || h->es == 1) ? 128 : 64)) return SPMM_ERR_UNSUPPORTED;
     if (f.nbr == 0) return SPMM_OK;
     int rc = ensure_schedule(h, N);
     if (rc) return rc;
@@ -1073,7 +1076,7 @@ int spmm_bcsr_plan(spmm_handle_t h, int64_t N) {
     NvtxRange nvtx_range("spmm_bcsr_plan");
     if (!h || N <= 0) return SPMM_ERR_INVALID_ARG;
     if (h->format != 0) return SPMM_ERR_INVALID_ARG;
-    if (N < (h->col_major ? 128 : 64) || (!h->col_major && (N * h->es) % 16 != 0)) return SPMM_ERR_UNSUPPORTED;
+    if (N < ((h->col_major || h->es == 1) ? 128 : 64) || (!h->col_major && (N * h->es) % 16 != 0)) return SPMM_ERR_UNSUPPORTED;
     return ensure_schedule(h, N);
 }
 

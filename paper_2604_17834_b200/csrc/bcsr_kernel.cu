@@ -119,7 +119,6 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ CUtensorMap tmC,
                  const __grid_constant__ CUtensorMap tmP, const BcsrParams p) {
     constexpr int ES = FMT == 3 ? 1 : (FMT == 2 ? 4 : 2);
-    static_assert(ES != 1 || CM, "8-bit inputs: column-major operands only");
     static_assert(FMT != 2 || (!CT && !DYN && H == B), "TF32: fp32 C, static schedule, no row groups");
     static_assert(H == B || !DYN, "stacked blocks: static schedule only");
     using CElem = typename CType<FMT, CT>::type;
@@ -617,19 +616,20 @@ cudaError_t launch_stack_fmt(int b, int c16, int cm, const CUtensorMap& tmA, con
                : launch_stack_shape<FMT, 0, 0>(b, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
 }
 
-// E4M3 inputs: column-major operands, fp32 C, static schedule; b = 32, 64 or 128 (a block row
-// must hold at least one 32-element K step).  Stages are half the bytes of the 16-bit ones.
+// E4M3 inputs: fp32 C, static schedule; b = 32, 64 or 128 (a block row must hold at least one
+// 32-element K step).  Stages are half the bytes of the 16-bit ones.
+template <int CM>
 cudaError_t launch_fp8(int b, int groups, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB3,
                        const CUtensorMap& tmC, const CUtensorMap& tmP, const BcsrParams& p, int grid, cudaStream_t stream) {
     switch (b * 10 + groups) {
-        case 321: return launch_one<32, 32, 1, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
-        case 322: return launch_one<32, 32, 2, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
-        case 324: return launch_one<32, 32, 4, 6, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
-        case 641: return launch_one<64, 64, 1, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
-        case 642: return launch_one<64, 64, 2, 10, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
-        case 644: return launch_one<64, 64, 4, 5, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
-        case 1281: return launch_one<128, 128, 1, 6, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
-        case 1282: return launch_one<128, 128, 2, 4, 3, 0, 1, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 321: return launch_one<32, 32, 1, 10, 3, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 322: return launch_one<32, 32, 2, 10, 3, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 324: return launch_one<32, 32, 4, 6, 3, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 641: return launch_one<64, 64, 1, 10, 3, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 642: return launch_one<64, 64, 2, 10, 3, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 644: return launch_one<64, 64, 4, 5, 3, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 1281: return launch_one<128, 128, 1, 6, 3, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+        case 1282: return launch_one<128, 128, 2, 4, 3, 0, CM, 0>(tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -682,8 +682,11 @@ cudaError_t launch_bcsr(int dtype, int b, int groups, int c16, int col_major, in
                         int grid, cudaStream_t stream) {
     if (dtype == 1) return launch_fmt<0>(b, groups, c16, col_major, dynamic, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);   // fp16
     if (dtype == 0) return launch_fmt<1>(b, groups, c16, col_major, dynamic, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);   // bf16
-    if (dtype == 3) return (c16 || !col_major || dynamic) ? cudaErrorInvalidValue
-                                                           : launch_fp8(b, groups, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+    if (dtype == 3) {
+        if (c16 || dynamic) return cudaErrorInvalidValue;
+        return col_major ? launch_fp8<1>(b, groups, tmA, tmB, tmB3, tmC, tmP, p, grid, stream)
+                         : launch_fp8<0>(b, groups, tmA, tmB, tmB3, tmC, tmP, p, grid, stream);
+    }
     if (dtype == 2) {
         if (c16 || dynamic) return cudaErrorInvalidValue;
         return col_major ? launch_tf32<1>(b, groups, tmA, tmB, tmB3, tmC, tmP, p, grid, stream)

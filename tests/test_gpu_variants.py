@@ -479,3 +479,25 @@ def test_bcsr_k_split_of_long_block_rows(lib, dtype, b, m, k, N):
     finally:
         lib.spmm_destroy(h0)
         lib.spmm_destroy(h1)
+
+
+@pytest.mark.parametrize("b,N", [(32, 640), (64, 1024), (128, 400), (64, 128)])
+def test_bcsr_fp8_e4m3_rowmajor(lib, b, N):
+    """E4M3 inputs with the default row-major operands (B [k][N] as the token-major tensor-core
+    operand of 1-byte elements): oracle bound, and the same bits as the column-major path (same
+    products, same order)."""
+    a = wl.bcsr_sweep(950 + b, m=1024, k=768, b=b, density=0.2, dtype="fp8")
+    Bs = wl.dense(43, a["k"], N, ("uniform", -1.0, 1.0), "fp8")
+    h0 = lib.spmm_bcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "fp8", b)
+    h1 = lib.spmm_bcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "fp8", b, layout=lib.COLMAJOR,
+                                  stack_min_fill=-1)
+    try:
+        C0 = run_gpu_variant(lib, h0, Bs, a["m"], N, "fp8")
+        Cr, S = reference(a, Bs, "fp8")
+        assert_close(C0, Cr, S, "fp8", "bcsr fp8 row-major b=%d N=%d" % (b, N))
+        assert np.array_equal(C0, run_gpu_variant(lib, h0, Bs, a["m"], N, "fp8"))
+        C1 = run_gpu_variant(lib, h1, Bs, a["m"], N, "fp8", col_major=True)
+        assert np.array_equal(C0, C1)
+    finally:
+        lib.spmm_destroy(h0)
+        lib.spmm_destroy(h1)
