@@ -95,6 +95,9 @@ struct MixArgs {
     int hot;               // 1: every warp rewrites its own tile (stays in L2); 0: streams through C
     int c_rows, c_cols;    // the fp32 array the stores go to
     int roles;             // 0: every CTA loads and stores; 1: even CTAs load, odd CTAs store
+    int mma_n;             // > 0: a sixth warp issues mma_count MMAs (M = 128, N = mma_n, K = 16) on the ring's memory
+    int mma_count;
+    long long* mma_clk;    // [grid] cycles the MMA warp took
     float* C;
 };
 
@@ -118,18 +121,47 @@ __device__ __forceinline__ void store_loop(const CUtensorMap* tmS, const MixArgs
     if (lane == 0) bulk_wait_all<false>();
 }
 
-__global__ void __launch_bounds__(160, 1)
+__global__ void __launch_bounds__(192, 1)
 mix_kernel(const __grid_constant__ CUtensorMap tmL, const __grid_constant__ CUtensorMap tmS, const MixArgs a, int* err) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    __shared__ uint64_t bar[16];
+    __shared__ uint64_t bar[17];
+    __shared__ uint32_t tslot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int slot_bytes = a.load_boxes * 8192;
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 16; ++i) mbar_init(smem_u32(&bar[i]), 1);
+        for (int i = 0; i < 17; ++i) mbar_init(smem_u32(&bar[i]), 1);
         fence_mbar_init();
     }
+    if (warp == 5 && a.mma_n > 0) { tmem_alloc(smem_u32(&tslot), 512); tmem_relinquish(); }
+    tc_fence_before_sync();
     __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 5) {
+        if (a.mma_n > 0) {
+            // operands: the token tile of ring slot 0 (M side, as the SpMM kernel reads it) and 8 KB of
+            // slot 1 as the stored block (N side); the data is whatever the loads leave there
+            const uint32_t tm = tslot;
+            const uint32_t idesc = make_idesc(1, 128, a.mma_n, 1, 0);
+            const uint64_t ad = make_smem_desc(base, 8192, 1024, SWZ_128B);
+            const uint64_t bd = make_smem_desc(base + slot_bytes, 16, 1024, SWZ_128B);
+            const int acc_mask = 512 / a.mma_n - 1;
+            const long long t0 = clock64();
+            if (elect_one()) {
+#pragma unroll 8
+                for (int i = 0; i < a.mma_count; ++i) umma_ss<false>(tm + (i & acc_mask) * a.mma_n, ad + ((i & 3) * 128), bd, idesc, 1);
+                tc_commit(smem_u32(&bar[16]));
+            }
+            __syncwarp();
+            wait_bounded(smem_u32(&bar[16]), 0, err);
+            if (lane == 0) a.mma_clk[blockIdx.x] = clock64() - t0;
+            tc_fence_before_sync();
+            __syncwarp();
+            tc_fence_after_sync();
+            tmem_dealloc(tm, 512);
+        }
+        return;
+    }
     const bool loads = a.load_slots > 0 && (a.roles == 0 || (blockIdx.x & 1) == 0);
     const bool stores = a.store_mode != 0 && (a.roles == 0 || (blockIdx.x & 1) == 1);
     if (warp == 0) {
@@ -216,7 +248,7 @@ void run_mix(Ctx& cx, const char* name, MixArgs a) {
     float best = 1e30f;
     for (int rep = 0; rep < 3; ++rep) {
         CK(cudaEventRecord(e0));
-        mix_kernel<<<cx.sms, 160, smem>>>(tmL, tmS, a, cx.err);
+        mix_kernel<<<cx.sms, 192, smem>>>(tmL, tmS, a, cx.err);
         CK(cudaEventRecord(e1));
         CK(cudaDeviceSynchronize());
         float ms;
@@ -230,6 +262,20 @@ void run_mix(Ctx& cx, const char* name, MixArgs a) {
     const double lb = double(loaders) * a.load_iters * a.load_boxes * 8192.0;
     const double sb = double(storers) * 4.0 * a.store_iters * a.tile_rows * (a.store_mode == 2 ? 32 : a.tile_cols) * 4.0;
     const double s = best * 1e-3;
+    if (a.mma_n > 0) {
+        std::vector<long long> clk(cx.sms);
+        CK(cudaMemcpy(clk.data(), a.mma_clk, cx.sms * sizeof(long long), cudaMemcpyDeviceToHost));
+        double sum = 0;
+        for (long long c : clk) sum += double(c);
+        std::printf("{\"case\": \"%s\", \"ms\": %.4f, \"load_tbs\": %.2f, \"load_B_per_clk_sm\": %.1f, \"mma_n\": %d, "
+                    "\"clk_per_mma\": %.1f, \"wait_ran_out\": %d}\n",
+                    name, best, lb / s / 1e12, loaders ? lb / s / loaders / (cx.clk_ghz * 1e9) : 0.0, a.mma_n,
+                    sum / cx.sms / a.mma_count, herr);
+        std::fflush(stdout);
+        CK(cudaEventDestroy(e0));
+        CK(cudaEventDestroy(e1));
+        return;
+    }
     std::printf("{\"case\": \"%s\", \"ms\": %.4f, \"load_tbs\": %.2f, \"store_tbs\": %.2f, \"load_B_per_clk_sm\": %.1f, "
                 "\"store_B_per_clk_sm\": %.1f, \"loading_sms\": %d, \"storing_sms\": %d, \"wait_ran_out\": %d}\n",
                 name, best, lb / s / 1e12, sb / s / 1e12, loaders ? lb / s / loaders / (cx.clk_ghz * 1e9) : 0.0,
@@ -298,6 +344,26 @@ int main(int argc, char** argv) {
         MixArgs a = base;
         a.load_boxes = 4; a.load_slots = 4; a.load_iters = 3000;
         run_mix(cx, "load_only_4x32KB", a);
+    }
+
+    // ---- MMAs beside the loads: do operand reads and TMA writes share shared-memory bandwidth?
+    {
+        long long* dclk;
+        CK(cudaMalloc(&dclk, cx.sms * sizeof(long long)));
+        for (int n : {64, 128}) {
+            for (int with_loads : {0, 1}) {
+                MixArgs a = base;
+                a.load_slots = 2;                               // the ring's memory holds the operands either way
+                a.load_iters = with_loads ? 1500 : 0;
+                a.mma_n = n;
+                a.mma_count = n == 64 ? 28000 : 21000;          // about as long as the loads alone
+                a.mma_clk = dclk;
+                char nm[64];
+                std::snprintf(nm, sizeof nm, "mma_n%d%s", n, with_loads ? "_with_loads_2x64KB" : "_alone_all_sms");
+                run_mix(cx, nm, a);
+            }
+        }
+        CK(cudaFree(dclk));
     }
 
     // ---- stores alone and beside loads, per box shape
