@@ -117,7 +117,7 @@ struct WcsrParams {
     const int32_t* col_idx;      // window_col_idx [P]
     const uint8_t* grp_class;    // reuse class of every four padded columns [P / 4], or null: no gather hints
     int32_t hot_min;             // groups of this class and above are gathered with the evict-last priority
-    int32_t hint_flags;          // 1: the packed A tiles are fetched evict-first; 2: C and partial tiles are stored evict-first
+    int32_t hint_flags;          // 1: the packed A tiles are fetched evict-first
     const uint8_t* packed;       // packed A values
     const void* B;               // k x N row-major
     void* C;                     // [m][N] fp32, or the input's 16-bit type

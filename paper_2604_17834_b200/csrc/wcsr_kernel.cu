@@ -428,7 +428,6 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
     } else {
         // ------------------------------------------------------------------ epilogue warps
         const int qd = warp & 3;
-        const uint64_t pol_stream_c = l2_policy_evict_first();
         SegIter seg;
         seg.init();
         uint32_t item = 0;
@@ -479,18 +478,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     if (lane == 0) mbar_arrive(acce_bar(acc));
                     const int n = n0 + qd * 32 + lane;
                     if (n < N) {
-                        if (p.hint_flags & 2) {
-                            // C is written once and not read again by this kernel: let it leave L2 first
-                            if (sizeof(CElem) == 4 || slot >= 0) {
-#pragma unroll
-                                for (int jr = 0; jr < kWH; ++jr)
-                                    if (jr < rows) st_global_hint(out + static_cast<int64_t>(jr) * N + n, v[jr], pol_stream_c);
-                            } else {
-#pragma unroll
-                                for (int jr = 0; jr < kWH; ++jr)
-                                    if (jr < rows) st_global_hint(outc + static_cast<int64_t>(jr) * N + n, from_f32<CElem>(v[jr]), pol_stream_c);
-                            }
-                        } else if (sizeof(CElem) == 4 || slot >= 0) {
+                        if (sizeof(CElem) == 4 || slot >= 0) {
 #pragma unroll
                             for (int jr = 0; jr < kWH; ++jr)
                                 if (jr < rows) out[static_cast<int64_t>(jr) * N + n] = v[jr];
