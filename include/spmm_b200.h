@@ -222,8 +222,12 @@ typedef enum {
     SPMM_X_WCSR_TASKS = 13,         /* int32 [n_tasks][4]: window, first col in window,
                                        column count, partial slot (-1 = writes C directly)    */
     SPMM_X_WCSR_BIN_PTR = 14,       /* int32 [n_bins+1]: ranges of BIN_TASKS, n_bins = 2*n_ctas */
-    SPMM_X_WCSR_BIN_TASKS = 15      /* int32 [n_tasks]: task indices bin by bin (the static
+    SPMM_X_WCSR_BIN_TASKS = 15,     /* int32 [n_tasks]: task indices bin by bin (the static
                                        schedule: CTA c runs bins c, c + grid, ...)            */
+    SPMM_X_WCSR_GROUP_CLASS = 16    /* uint8 [P / 4]: reuse class of every four padded columns
+                                       (7 = among the 16 Ki most gathered rows of B, each class
+                                       below twice as many, 0 = the rest): the kernel's L2
+                                       hint for the gathers, no effect on results             */
 } spmm_export_t;
 
 /*

@@ -43,7 +43,7 @@ X_BCSR_TILE_PTR, X_BCSR_TILES = 4, 5
 X_BCSR_STACK_ROWS, X_BCSR_STACK_PTR, X_BCSR_STACK_COL_IDX, X_BCSR_STACK_TILE_PTR, X_BCSR_STACK_TILES = 6, 7, 8, 9, 20
 X_BCSR_UNITS = 21
 X_WCSR_WINDOW_ROW_PTR, X_WCSR_WINDOW_COL_IDX, X_WCSR_VALUES, X_WCSR_TASKS = 10, 11, 12, 13
-X_WCSR_BIN_PTR, X_WCSR_BIN_TASKS = 14, 15
+X_WCSR_BIN_PTR, X_WCSR_BIN_TASKS, X_WCSR_GROUP_CLASS = 14, 15, 16
 
 EXPORTED_SYMBOLS = (
     "spmm_bcsr_create_csr", "spmm_bcsr_create_csr_device", "spmm_bcsr_create_coo", "spmm_wcsr_create_csr",

@@ -495,7 +495,7 @@ int create_wcsr_device(spmm_handle_t* out, int64_t m, int64_t k, const int64_t* 
     try {
         rc = build_wcsr_device(m, k, d_row_ptr, d_col_idx, static_cast<const uint8_t*>(d_vals), h->es, wh, b_col, T,
                                h->n_ctas * wcsr_bins_per_sm(h->es, wh), stream, &h->wcsr, &h->nnz, &h->d_ptr, &h->d_idx,
-                               &h->d_vals);
+                               &h->d_vals, &h->d_grp_class);
         if (!rc) rc = upload_wcsr_plan(h);
     } catch (const std::bad_alloc&) {
         rc = SPMM_ERR_ALLOC;
@@ -1318,6 +1318,7 @@ int spmm_export(spmm_handle_t h, int which, void* host_dst, size_t cap, size_t* 
             case SPMM_X_WCSR_TASKS: bytes = f.tasks.size() * 16; break;
             case SPMM_X_WCSR_BIN_PTR: bytes = f.bin_ptr.size() * 4; dev_src = h->d_bin_ptr; host_src = f.bin_ptr.data(); break;
             case SPMM_X_WCSR_BIN_TASKS: bytes = f.bin_tasks.size() * 4; dev_src = h->d_bin_tasks; host_src = f.bin_tasks.data(); break;
+            case SPMM_X_WCSR_GROUP_CLASS: bytes = static_cast<size_t>(f.P / 4); dev_src = h->d_grp_class; host_src = f.grp_class.data(); break;
             default: return SPMM_ERR_INVALID_ARG;
         }
     }

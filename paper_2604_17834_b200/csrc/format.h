@@ -174,11 +174,13 @@ void wcsr_reuse_classes(const int32_t* window_col_idx, int64_t P, int64_t k, std
 int plan_wcsr(WcsrHost* out, int T, int n_bins, int es);
 // The WCSR format arrays built on the GPU from a CSR matrix in device memory (format_gpu.cu):
 // validates the CSR, allocates and fills window_row_ptr, window_col_idx and the packed values on
-// the device (owned by the caller afterwards), leaves window_row_ptr, P and distinct_cols in *out
-// (out->window_col_idx and out->packed stay empty) and runs plan_wcsr.  Synchronises `stream`.
+// the device (owned by the caller afterwards) together with the column groups' reuse classes
+// (*d_grp_class, the rule of wcsr_reuse_classes), leaves window_row_ptr, P and distinct_cols in *out
+// (out->window_col_idx, out->packed and out->grp_class stay empty) and runs plan_wcsr.
+// Synchronises `stream`.
 int build_wcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int32_t* d_col_idx, const uint8_t* d_vals,
                       int es, int wh, int b_col, int T, int n_bins, cudaStream_t stream, WcsrHost* out, int64_t* nnz_out,
-                      int32_t** d_window_row_ptr, int32_t** d_window_col_idx, uint8_t** d_packed);
+                      int32_t** d_window_row_ptr, int32_t** d_window_col_idx, uint8_t** d_packed, uint8_t** d_grp_class);
 
 // Byte offset of element (row r, padded column q) inside the packed WCSR value array.
 #ifdef __CUDACC__

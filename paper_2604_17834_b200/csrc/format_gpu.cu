@@ -423,11 +423,91 @@ __global__ void wcsr_values_kernel(int64_t m, int wh, int b_col, const int64_t* 
     }
 }
 
+// ---- reuse classes of the column groups (gather hints; the host rule of wcsr_reuse_classes)
+
+__global__ void wcsr_refs_kernel(const int32_t* __restrict__ col_idx, int64_t P, int32_t* __restrict__ refs) {
+    for (int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; q < P; q += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int32_t c = col_idx[q];
+        if (c >= 0) atomicAdd(refs + c, 1);
+    }
+}
+
+__global__ void iota_kernel(int32_t* __restrict__ x, int64_t n) {
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += static_cast<int64_t>(gridDim.x) * blockDim.x)
+        x[i] = static_cast<int32_t>(i);
+}
+
+// rows in descending order of their gather count (stable: ties by index): rank r -> class
+__global__ void wcsr_class_kernel(const int32_t* __restrict__ sorted_refs, const int32_t* __restrict__ order, int64_t k,
+                                  uint8_t* __restrict__ cls) {
+    for (int64_t r = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; r < k; r += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        int level = 0;
+        if (sorted_refs[r] > 1) {
+            level = 7;
+            for (int64_t lim = kWcsrTopClassRows; level > 0 && r >= lim; lim *= 2) --level;
+        }
+        cls[order[r]] = static_cast<uint8_t>(level);
+    }
+}
+
+__global__ void wcsr_group_class_kernel(const int32_t* __restrict__ col_idx, int64_t n_groups, const uint8_t* __restrict__ cls,
+                                        uint8_t* __restrict__ grp_class) {
+    for (int64_t g = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; g < n_groups; g += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int4 c = reinterpret_cast<const int4*>(col_idx)[g];
+        int best = 0;
+        if (c.x >= 0) best = max(best, static_cast<int>(cls[c.x]));
+        if (c.y >= 0) best = max(best, static_cast<int>(cls[c.y]));
+        if (c.z >= 0) best = max(best, static_cast<int>(cls[c.z]));
+        if (c.w >= 0) best = max(best, static_cast<int>(cls[c.w]));
+        grp_class[g] = static_cast<uint8_t>(best);
+    }
+}
+
+// Allocates and fills *d_grp_class [P / 4] from the device copy of window_col_idx.
+int wcsr_reuse_classes_device(const int32_t* d_window_col_idx, int64_t P, int64_t k, cudaStream_t st, uint8_t** d_grp_class) {
+    *d_grp_class = nullptr;
+    if (P <= 0 || k <= 0) return SPMM_OK;
+    int32_t *refs = nullptr, *refs_sorted = nullptr, *ids = nullptr, *order = nullptr;
+    uint8_t* cls = nullptr;
+    void* temp = nullptr;
+    auto release = [&]() { cudaFree(refs); cudaFree(refs_sorted); cudaFree(ids); cudaFree(order); cudaFree(cls); cudaFree(temp); };
+    const size_t kb = static_cast<size_t>(k) * 4;
+    if (cudaMalloc(reinterpret_cast<void**>(&refs), kb) != cudaSuccess || cudaMalloc(reinterpret_cast<void**>(&refs_sorted), kb) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&ids), kb) != cudaSuccess || cudaMalloc(reinterpret_cast<void**>(&order), kb) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&cls), static_cast<size_t>(k)) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(d_grp_class), static_cast<size_t>(P / 4)) != cudaSuccess) {
+        release();
+        cudaFree(*d_grp_class);
+        *d_grp_class = nullptr;
+        return SPMM_ERR_ALLOC;
+    }
+    cudaMemsetAsync(refs, 0, kb, st);
+    wcsr_refs_kernel<<<2048, 256, 0, st>>>(d_window_col_idx, P, refs);
+    iota_kernel<<<static_cast<unsigned>(std::min<int64_t>((k + 255) / 256, 2048)), 256, 0, st>>>(ids, k);
+    size_t tb = 0;
+    cub::DeviceRadixSort::SortPairsDescending(nullptr, tb, refs, refs_sorted, ids, order, static_cast<int>(k), 0, 32, st);
+    bool ok = cudaMalloc(&temp, tb ? tb : 16) == cudaSuccess &&
+              cub::DeviceRadixSort::SortPairsDescending(temp, tb, refs, refs_sorted, ids, order, static_cast<int>(k), 0, 32, st) == cudaSuccess;
+    if (ok) {
+        wcsr_class_kernel<<<static_cast<unsigned>(std::min<int64_t>((k + 255) / 256, 2048)), 256, 0, st>>>(refs_sorted, order, k, cls);
+        wcsr_group_class_kernel<<<2048, 256, 0, st>>>(d_window_col_idx, P / 4, cls, *d_grp_class);
+        ok = cudaStreamSynchronize(st) == cudaSuccess && cudaGetLastError() == cudaSuccess;
+    }
+    release();
+    if (!ok) {
+        cudaFree(*d_grp_class);
+        *d_grp_class = nullptr;
+        return SPMM_ERR_CUDA;
+    }
+    return SPMM_OK;
+}
+
 }  // namespace
 
 int build_wcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int32_t* d_col_idx, const uint8_t* d_vals,
                       int es, int wh, int b_col, int T, int n_bins, cudaStream_t st, WcsrHost* out, int64_t* nnz_out,
-                      int32_t** d_window_row_ptr, int32_t** d_window_col_idx, uint8_t** d_packed) {
+                      int32_t** d_window_row_ptr, int32_t** d_window_col_idx, uint8_t** d_packed, uint8_t** d_grp_class) {
+    *d_grp_class = nullptr;
     if (wh != 16 && wh != 64) return SPMM_ERR_UNSUPPORTED;
     if ((es != 2 && es != 4) || b_col * es != 32) return SPMM_ERR_UNSUPPORTED;
     if (T < 0 || T % b_col != 0 || n_bins <= 0) return SPMM_ERR_INVALID_ARG;
@@ -544,10 +624,11 @@ int build_wcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int3
     }
     if (cudaStreamSynchronize(st) != cudaSuccess || cudaGetLastError() != cudaSuccess) return fail(SPMM_ERR_CUDA);
     release();
-    const int rc = plan_wcsr(out, T, n_bins, es);
+    int rc = wcsr_reuse_classes_device(*d_window_col_idx, P, k, st, d_grp_class);
+    if (!rc) rc = plan_wcsr(out, T, n_bins, es);
     if (rc) {
-        cudaFree(*d_window_row_ptr); cudaFree(*d_window_col_idx); cudaFree(*d_packed);
-        *d_window_row_ptr = nullptr; *d_window_col_idx = nullptr; *d_packed = nullptr;
+        cudaFree(*d_window_row_ptr); cudaFree(*d_window_col_idx); cudaFree(*d_packed); cudaFree(*d_grp_class);
+        *d_window_row_ptr = nullptr; *d_window_col_idx = nullptr; *d_packed = nullptr; *d_grp_class = nullptr;
     }
     return rc;
 }

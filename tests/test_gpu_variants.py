@@ -251,6 +251,8 @@ def test_wcsr_built_on_the_gpu_is_bit_exact(lib, dtype, wh, m, k, dens):
                               f["values"].view(bits).ravel())
         for which in (lib.X_WCSR_TASKS, lib.X_WCSR_BIN_PTR, lib.X_WCSR_BIN_TASKS):
             assert np.array_equal(lib.spmm_export(h, which, np.int32), lib.spmm_export(h0, which, np.int32))
+        # the gather hints (reuse class per four padded columns): same bytes from both builders
+        assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_GROUP_CLASS, np.uint8), lib.spmm_export(h0, lib.X_WCSR_GROUP_CLASS, np.uint8))
         i1, i0 = lib.spmm_get_info(h, 128), lib.spmm_get_info(h0, 128)
         assert i1 == i0
         N = 136

@@ -398,3 +398,28 @@ def test_bcsr_row_major_needs_at_least_64_columns(lib):
         assert lib.spmm_get_info(h, 64)["plan_n"] == 64
     finally:
         lib.spmm_destroy(h)
+
+
+def test_wcsr_reuse_classes_of_the_gather_hints(lib):
+    """Device-private hint, checked against its rule written out with numpy: B rows ranked by the
+    number of windows that gather them (ties: lower index), class 7 for the first 16 Ki, one class
+    down per doubling, 0 beyond 1 Mi and for rows gathered once; a group of four padded columns
+    takes the highest class among its columns."""
+    a = wl.rmat(seed=5, scale=16, edge_factor=12)                     # 65,536 columns, skewed popularity
+    h = lib.spmm_wcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], "fp16", 16, host_only=True)
+    try:
+        got = lib.spmm_export(h, lib.X_WCSR_GROUP_CLASS, np.uint8)
+        wcol = lib.spmm_export(h, lib.X_WCSR_WINDOW_COL_IDX, np.int32)
+    finally:
+        lib.spmm_destroy(h)
+    refs = np.bincount(wcol[wcol >= 0], minlength=a["k"])
+    order = np.argsort(-refs, kind="stable")
+    rank = np.empty(a["k"], dtype=np.int64)
+    rank[order] = np.arange(a["k"])
+    level = np.clip(7 - np.floor(np.log2(np.maximum(rank, 1) / 16384.0) + 1).astype(np.int64), 0, 7)
+    level = np.where(rank < 16384, 7, level)
+    cls = np.where(refs > 1, level, 0)
+    per_col = np.where(wcol >= 0, cls[np.maximum(wcol, 0)], 0).reshape(-1, 4)
+    assert got.shape[0] == wcol.shape[0] // 4
+    assert np.array_equal(got, per_col.max(axis=1).astype(np.uint8))
+    assert got.max() == 7 and (got == 6).any() and (got == 0).any()
