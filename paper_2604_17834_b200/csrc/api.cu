@@ -764,15 +764,13 @@ int ensure_schedule(spmm_handle_s* h, int64_t N) {
         if (!rc && sc.n_slots > 0) {
             // merge lists (split block-rows in ascending order: their slots are consecutive), the
             // partial tiles' workspace and its store map
+            // (the parts of a block-row are consecutive units, in part order)
             std::vector<int32_t> rows, firsts, parts;
             for (size_t u = 0; u < sc.units.size() / 4; ++u) {
                 const int32_t I = sc.units[4 * u], slot = sc.units[4 * u + 3];
                 if (slot < 0) continue;
-                size_t j = 0;
-                while (j < rows.size() && rows[j] != I) ++j;
-                if (j == rows.size()) { rows.push_back(I); firsts.push_back(slot); parts.push_back(0); }
-                firsts[j] = std::min(firsts[j], slot);
-                parts[j]++;
+                if (rows.empty() || rows.back() != I) { rows.push_back(I); firsts.push_back(slot); parts.push_back(0); }
+                parts.back()++;
             }
             std::vector<int32_t> mg;
             mg.insert(mg.end(), rows.begin(), rows.end());

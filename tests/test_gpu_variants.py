@@ -301,7 +301,8 @@ def test_variant_argument_errors(lib):
         lib.spmm_wcsr_create_csr(*args, 16, schedule=lib.SCHED_DYNAMIC)
     assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
     a8 = wl.bcsr_sweep(5, m=256, k=256, b=32, density=0.3, dtype="fp8")
-    for kw in (dict(), dict(layout=lib.COLMAJOR, c_type=lib.C_SAME_AS_INPUT)):    # E4M3: column-major, fp32 C only
+    for kw in (dict(c_type=lib.C_SAME_AS_INPUT), dict(layout=lib.COLMAJOR, c_type=lib.C_SAME_AS_INPUT),
+               dict(schedule=lib.SCHED_DYNAMIC)):                                  # E4M3: fp32 C, static schedule only
         with pytest.raises(lib.SpmmError) as e:
             lib.spmm_bcsr_create_csr(256, 256, a8["row_ptr"], a8["col_idx"], a8["vals"], "fp8", 32, **kw)
         assert e.value.code == lib.SPMM_ERR_UNSUPPORTED
