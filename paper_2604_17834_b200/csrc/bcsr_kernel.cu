@@ -16,12 +16,17 @@
 //   warp 1      MMA issuer: one thread issues tcgen05.mma into one of two TMEM accumulator
 //               buffers; tcgen05.commit frees the ring slot / publishes the accumulator.
 //   warps 2-5   epilogue: tcgen05.ld -> registers -> one of the warp's staging tiles in shared
-//               memory (up to 64 C rows x 32 tokens = 8 KB of fp32; a ring of 2 or more tiles
-//               per warp, so that the warp fills the next tile while earlier TMA stores are
-//               still reading theirs) -> one TMA store per tile, which also clips at the edges
-//               of C (zeros for empty block-rows); overlaps the next tile's MMAs thanks to the
-//               second TMEM buffer.
-// Two optional variants, both template parameters:
+//               memory (16 fp32 or 32 16-bit C rows x 32 tokens = 2 KB; a ring of as many tiles
+//               per warp as fit beside the stage ring, so that the warp fills the next tile
+//               while earlier TMA stores are still reading theirs) -> one TMA store per tile,
+//               which also clips at the edges of C (zeros for empty block-rows); overlaps the
+//               next tile's MMAs thanks to the second TMEM buffer.
+// Value types (FMT): fp16, bf16 (K = 16 per MMA), TF32 (fp32 storage, K = 8; the token tile then
+// uses the 128-byte swizzle with 32-byte atoms, and blocks wider than 32 columns pass through the
+// ring in 32-column slices), E4M3 (K = 32): a K step is 32 bytes of an operand row in all of them.
+// A tile of one part of a K-split block-row (record x < 0) stores an fp32 partial tile through
+// tmP instead of C; bcsr_merge_kernel adds the parts in order.
+// Optional variants, all template parameters:
 //   CT = 1   C is written in the input's 16-bit type instead of fp32.
 //   CM = 1   "column-major" operands (the layout of the paper's BCSR kernel, Sec. 3.2, and of a
 //            linear layer Y = X W^T, Sec. 4.4): B is given as X[N][k] (one row per token, k
