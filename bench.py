@@ -184,6 +184,13 @@ def workload_table():
                 "configs[3] b=%d skewed rows, keep %g, dynamic tile scheduling" % (b, d), variant(cfg4(b, d), dyn=True))
         t["cfg4_bcsr_sweep_b%d_d0.1_plain" % b] = ("configs[3] b=%d skewed rows, keep 0.1, row groups switched off" % b,
                                                     plain(cfg4(b, 0.1)))
+        if b < 128:
+            def fam(b=b):
+                return dict(kind="bcsr", a=wl.bcsr_families(1300 + b, b=b), dtype="fp16", size=b, N=4096,
+                            Bdist=("uniform", -1.0, 1.0))
+            t["cfg4_bcsr_families_b%d" % b] = (
+                "configs[3] shape, b=%d, block-rows in 32 scattered families (keep 0.1, 10 %% dropped per row)" % b, fam)
+            t["cfg4_bcsr_families_b%d_plain" % b] = ("the same, row groups switched off", plain(fam))
         for d in (0.05, 0.01):
             t["cfg4_bcsr_flat_b%d_d%g" % (b, d)] = (
                 "configs[3] BCSR 8192x8192 fp16 b=%d flat Bernoulli(%g), N=4096" % (b, d), cfg4(b, d, False))
@@ -208,6 +215,7 @@ ALL_OTHERS = DEFAULT_OTHERS + [
     "cfg2_wcsr_irregular_lsu_gather", "cfg5_wcsr_rmat_n128_lsu_gather",
     "cfg4_bcsr_sweep_b64_d0.1_dyn", "cfg4_bcsr_sweep_b16_d0.1_plain", "cfg4_bcsr_sweep_b32_d0.1_plain",
     "cfg4_bcsr_sweep_b16_d0.5", "cfg4_bcsr_sweep_b32_d0.5",
+    "cfg4_bcsr_families_b16", "cfg4_bcsr_families_b16_plain", "cfg4_bcsr_families_b32", "cfg4_bcsr_families_b32_plain",
     "cfg4_bcsr_sweep_b64_d0.1_ksplit", "cfg4_bcsr_sweep_b64_d0.01_ksplit",
     "cfg4_bcsr_sweep_b16_d0.1_tf32", "cfg4_bcsr_sweep_b32_d0.1_tf32", "cfg4_bcsr_sweep_b64_d0.1_tf32", "cfg4_bcsr_sweep_b128_d0.1_tf32"]
 

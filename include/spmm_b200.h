@@ -141,9 +141,12 @@ typedef struct {
                             block-rows store blocks in mostly the same block columns, the
                             kernel computes them together from 128-row stacked blocks (absent
                             sub-blocks zero), so that each slice of the dense operand is staged
-                            once for all of them.  Candidates are runs of 128 / b consecutive
-                            non-empty block-rows in ROW_ORDER; one is taken when at least this
-                            percentage of its sub-blocks is stored.  0 = default (30 / 45 / 75
+                            once for all of them.  Grouping is by similarity: in ROW_ORDER, every
+                            block-row not yet grouped is offered the 128 / b - 1 ungrouped
+                            block-rows that share the most block columns with it (they may
+                            lie anywhere in the matrix); the candidate is taken when at least
+                            this percentage of its sub-blocks is stored (the search is capped
+                            at 2^27 visited stored blocks).  0 = default (30 / 45 / 75
                             for b = 16 / 32 / 64), -1 = off, 1..100 = threshold.  A private
                             second copy of the grouped rows' values is kept on the device; the
                             exported format arrays and nnz_stored are unaffected.  Ignored for

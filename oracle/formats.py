@@ -352,32 +352,66 @@ def bcsr_k_split_order(units):
     return np.argsort(-ln, kind="stable").astype(np.int32)
 
 
+BCSR_GROUP_WORK_LIMIT = 1 << 27
+
+
 def bcsr_row_groups(block_row_ptr, block_col_idx, b, min_fill_pct):
     """Row groups of the BCSR kernel (a device-side regrouping with no counterpart in the
     paper, whose BCSR blocks are all b x b, Sec. 2.3): R = 128 // b block-rows that store
     blocks in mostly the same block columns are computed together, one 128-row stacked block
     per block column of their union.
 
-    Rule: walk bcsr_row_order (most stored blocks first, stable); every run of R consecutive
-    block-rows in that order is a candidate while its last row is non-empty; a candidate is
-    accepted when 100 * (stored blocks of its rows) >= min_fill_pct * R * |union of their
-    block columns|.  Returns (rows int32 [ng, R], ptr int32 [ng+1], col_idx int32 [ns]):
-    member rows in row order, and per group the ascending union of block columns.
+    Rule (grouping by similarity): walk bcsr_row_order (most stored blocks first, stable).  A
+    block-row that is non-empty and not yet in a group is a seed; its partners are the R - 1 other
+    free non-empty block-rows that share the most block columns with it (at least one; ties: the
+    one earlier in the order); with fewer than R - 1 such rows the seed forms no group.  The
+    candidate (seed and partners, listed in the order) is accepted when 100 * (stored blocks of
+    its rows) >= min_fill_pct * R * |union of their block columns|; its rows then leave the free
+    set, otherwise all of them stay free (the seed is not tried again as a seed, but may become a
+    partner).  The search stops for good once the work it has charged -- per seed, the sum over
+    the seed's block columns of the number of block-rows that store that column -- would pass
+    BCSR_GROUP_WORK_LIMIT.  Returns (rows int32 [ng, R], ptr int32 [ng+1], col_idx int32 [ns]):
+    member rows in the order, and per group the ascending union of block columns.
     """
     brp = np.asarray(block_row_ptr, dtype=np.int64)
     bci = np.asarray(block_col_idx, dtype=np.int64)
     R = 128 // b
+    nbr = brp.shape[0] - 1
     order = bcsr_row_order(brp)
+    pos = np.empty(nbr, dtype=np.int64)
+    pos[order] = np.arange(nbr)
+    colsets = [set(bci[brp[I]:brp[I + 1]].tolist()) for I in range(nbr)]
+    degree = np.bincount(bci, minlength=int(bci.max()) + 1 if bci.size else 1)
+    by_col = {}
+    for I in range(nbr):
+        for J in colsets[I]:
+            by_col.setdefault(J, []).append(I)
+    free = [len(colsets[I]) > 0 for I in range(nbr)]
     rows, ptr, cols = [], [0], []
-    for r0 in range(0, len(order) - R + 1, R):
-        cand = order[r0:r0 + R]
-        if brp[cand[-1] + 1] == brp[cand[-1]]:
+    work = 0
+    for s in order.tolist():
+        if not free[s]:
+            continue
+        w = int(sum(degree[J] for J in colsets[s]))
+        if work + w > BCSR_GROUP_WORK_LIMIT:
             break
-        stored = int(sum(brp[I + 1] - brp[I] for I in cand))
-        union = np.unique(np.concatenate([bci[brp[I]:brp[I + 1]] for I in cand]))
+        work += w
+        overlap = {}
+        for J in colsets[s]:
+            for r in by_col[J]:
+                if r != s and free[r]:
+                    overlap[r] = overlap.get(r, 0) + 1
+        if len(overlap) < R - 1:
+            continue
+        partners = sorted(overlap, key=lambda r: (-overlap[r], pos[r]))[:R - 1]
+        members = sorted([s] + partners, key=lambda r: pos[r])
+        stored = sum(len(colsets[r]) for r in members)
+        union = sorted(set().union(*[colsets[r] for r in members]))
         if 100 * stored >= min_fill_pct * R * len(union):
-            rows.append([int(I) for I in cand])
-            cols.extend(union.tolist())
+            for r in members:
+                free[r] = False
+            rows.append(members)
+            cols.extend(union)
             ptr.append(len(cols))
     return (np.asarray(rows, dtype=np.int32).reshape(-1, R), np.asarray(ptr, dtype=np.int32),
             np.asarray(cols, dtype=np.int32))

@@ -231,11 +231,53 @@ int build_bcsr_stack(const BcsrHost& f, int min_fill_pct, BcsrStack* out) {
     out->min_fill_pct = min_fill_pct > 0 ? min_fill_pct : bcsr_stack_default_fill(f.b);
     out->ptr.push_back(0);
     std::vector<int32_t> cursor(static_cast<size_t>(R));
-    for (int64_t r0 = 0; r0 + R <= f.nbr; r0 += R) {
-        // the candidate's rows; row_order lists empty block-rows last, so the walk can stop there
-        const int32_t* rows = f.row_order.data() + r0;
-        const int32_t last = rows[R - 1];
-        if (f.block_row_ptr[last + 1] == f.block_row_ptr[last]) break;
+    // block-rows per block column (ascending), position of every block-row in row_order
+    std::vector<int64_t> col_ptr(static_cast<size_t>(f.nbc) + 1, 0);
+    for (int64_t q = 0; q < f.nnzb; ++q) ++col_ptr[f.block_col_idx[q] + 1];
+    for (int64_t J = 0; J < f.nbc; ++J) col_ptr[J + 1] += col_ptr[J];
+    std::vector<int32_t> col_rows(static_cast<size_t>(f.nnzb));
+    {
+        std::vector<int64_t> fill(col_ptr.begin(), col_ptr.end() - 1);
+        for (int64_t I = 0; I < f.nbr; ++I)
+            for (int32_t q = f.block_row_ptr[I]; q < f.block_row_ptr[I + 1]; ++q) col_rows[fill[f.block_col_idx[q]]++] = static_cast<int32_t>(I);
+    }
+    std::vector<int32_t> pos(static_cast<size_t>(f.nbr));
+    std::vector<uint8_t> is_free(static_cast<size_t>(f.nbr));
+    for (int64_t r = 0; r < f.nbr; ++r) {
+        pos[f.row_order[r]] = static_cast<int32_t>(r);
+        is_free[r] = f.block_row_ptr[r + 1] > f.block_row_ptr[r];
+    }
+    std::vector<int32_t> shared(static_cast<size_t>(f.nbr), 0), touched, rows(static_cast<size_t>(R));
+    int64_t work = 0;
+    for (int64_t r0 = 0; r0 < f.nbr; ++r0) {
+        const int32_t seed = f.row_order[r0];
+        if (f.block_row_ptr[seed + 1] == f.block_row_ptr[seed]) break;      // row_order lists empty block-rows last
+        if (!is_free[seed]) continue;
+        int64_t w = 0;
+        for (int32_t q = f.block_row_ptr[seed]; q < f.block_row_ptr[seed + 1]; ++q)
+            w += col_ptr[f.block_col_idx[q] + 1] - col_ptr[f.block_col_idx[q]];
+        if (work + w > kBcsrGroupWorkLimit) break;
+        work += w;
+        // block columns shared with the seed, per free block-row
+        touched.clear();
+        for (int32_t q = f.block_row_ptr[seed]; q < f.block_row_ptr[seed + 1]; ++q) {
+            const int32_t J = f.block_col_idx[q];
+            for (int64_t t = col_ptr[J]; t < col_ptr[J + 1]; ++t) {
+                const int32_t r = col_rows[t];
+                if (r == seed || !is_free[r]) continue;
+                if (shared[r]++ == 0) touched.push_back(r);
+            }
+        }
+        const bool enough = static_cast<int64_t>(touched.size()) >= R - 1;
+        if (enough)
+            std::partial_sort(touched.begin(), touched.begin() + (R - 1), touched.end(), [&](int32_t x, int32_t y) {
+                return shared[x] != shared[y] ? shared[x] > shared[y] : pos[x] < pos[y];
+            });
+        rows[0] = seed;
+        for (int i = 1; enough && i < R; ++i) rows[i] = touched[i - 1];
+        for (int32_t r : touched) shared[r] = 0;
+        if (!enough) continue;
+        std::sort(rows.begin(), rows.end(), [&](int32_t x, int32_t y) { return pos[x] < pos[y]; });
         int64_t stored = 0;
         for (int i = 0; i < R; ++i) {
             cursor[i] = f.block_row_ptr[rows[i]];
@@ -259,6 +301,7 @@ int build_bcsr_stack(const BcsrHost& f, int min_fill_pct, BcsrStack* out) {
             for (int i = 0; i < R; ++i) {
                 out->rows.push_back(rows[i]);
                 out->stacked[rows[i]] = 1;
+                is_free[rows[i]] = 0;
             }
             out->ptr.push_back(static_cast<int32_t>(out->col_idx.size()));
         } else {

@@ -41,9 +41,13 @@ struct BcsrHost {
 // as one "row group": for every block column of the union one stacked block of 128 rows x b
 // (absent sub-blocks zero), so that the slice of the token tile is fetched once for all R rows
 // and one MMA with N = 128 replaces R MMAs with N = b.
-// Rule (a pure function of the index arrays): walk row_order (most stored blocks first); every
-// run of R consecutive non-empty block-rows in that order is a candidate, accepted when
-// 100 * (stored blocks of the R rows) >= min_fill_pct * R * (block columns in their union).
+// Rule (a pure function of the index arrays; grouping by similarity): walk row_order (most stored
+// blocks first).  A non-empty block-row not yet in a group is a seed; its partners are the R - 1
+// other free block-rows that share the most block columns with it (at least one; ties: the one
+// earlier in row_order).  The candidate is accepted when
+// 100 * (stored blocks of the R rows) >= min_fill_pct * R * (block columns in their union);
+// a rejected candidate leaves all its rows free.  The search stops once the work charged -- per
+// seed, the number of stored blocks in the seed's block columns -- would pass kBcsrGroupWorkLimit.
 struct BcsrStack {
     int R = 0;                          // block-rows per group; 0: no stacking for this handle
     int min_fill_pct = 0;
@@ -56,6 +60,7 @@ struct BcsrStack {
 };
 // default acceptance threshold per block size, from the bytes a stacked and an unstacked block
 // bring into shared memory per unit of work (and measured on the Bernoulli sweep)
+constexpr int64_t kBcsrGroupWorkLimit = int64_t{1} << 27;
 constexpr int bcsr_stack_default_fill(int b) { return b == 16 ? 30 : (b == 32 ? 45 : 75); }
 int build_bcsr_stack(const BcsrHost& f, int min_fill_pct, BcsrStack* out);
 

@@ -200,6 +200,26 @@ def bcsr_sweep(seed, m=8192, k=8192, b=64, density=0.1, skewed=True, dtype="fp16
     return dict(m=m, k=k, dtype=dtype, row_ptr=row_ptr, col_idx=col_idx, vals=vals, block=b)
 
 
+def bcsr_families(seed, m=8192, k=8192, b=16, density=0.1, n_families=32, drop=0.1, dtype="fp16"):
+    """Block-sparse matrix whose block-rows come in families scattered over the row range (the
+    pattern structured pruning leaves when channels that are pruned together are not adjacent).
+
+    Every family has a Bernoulli(density) mask over the block columns; every block-row is
+    assigned a family uniformly at random, takes that family's mask and drops each kept block
+    with probability ``drop``.  Kept blocks are dense U[-1,1].
+    Draw order: family masks (row-major), family of every block-row, drop mask (row-major, all
+    blocks), values in CSR order.
+    """
+    rng = np.random.default_rng(seed)
+    nbr, nbc = -(-m // b), -(-k // b)
+    fam_mask = rng.random((n_families, nbc)) < density
+    fam = rng.integers(0, n_families, size=nbr)
+    mask = fam_mask[fam] & (rng.random((nbr, nbc)) >= drop)
+    row_ptr, col_idx = csr_from_block_mask(mask, b, m, k)
+    vals = _draw_vals(rng, col_idx.shape[0], ("uniform", -1.0, 1.0), dtype)
+    return dict(m=m, k=k, dtype=dtype, row_ptr=row_ptr, col_idx=col_idx, vals=vals, block=b)
+
+
 # --------------------------------------------------------------------------- irregular matrices
 
 

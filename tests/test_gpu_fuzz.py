@@ -104,8 +104,8 @@ def test_bcsr_tf32_random_case(lib, seed):
 
 @pytest.mark.parametrize("seed", range(40))
 def test_bcsr_row_groups_random_case(lib, seed):
-    """Row groups forced on (every run of 128 / b non-empty block-rows is stacked, however few of its
-    sub-blocks are stored) or left to the default threshold, over ragged shapes and all output options."""
+    """Row groups forced on (every candidate of 128 / b block-rows that share columns is stacked, however
+    few of its sub-blocks are stored) or left to the default threshold, over ragged shapes and all output options."""
     import torch
     rng = np.random.default_rng(11000 + seed)
     dtype = ["bf16", "fp16", "fp8"][seed % 3]

@@ -417,6 +417,35 @@ def test_bcsr_row_groups_from_the_gpu_builder(lib):
         lib.spmm_destroy(h)
 
 
+@pytest.mark.parametrize("b,dtype", [(16, "fp16"), (32, "bf16")])
+def test_bcsr_row_groups_find_scattered_families(lib, b, dtype):
+    """Block-rows of one family are far apart in the index range and in the length order: the
+    groups must still be (mostly) families, i.e. far fewer stacked blocks than R neighbours' union
+    would need, and the product must match the oracle."""
+    from oracle import formats as F
+    m, k, N = 2048, 2048, 384
+    a = wl.bcsr_families(55 + b, m=m, k=k, b=b, density=0.15, n_families=8, drop=0.1, dtype=dtype)
+    Bs = wl.dense(56 + b, k, N, ("uniform", -1.0, 1.0), dtype)
+    Cr, S = reference(a, Bs, dtype)
+    f = F.bcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], b)
+    rows, ptr, cols = F.bcsr_row_groups(f["block_row_ptr"], f["block_col_idx"], b, {16: 30, 32: 45}[b])
+    R = 128 // b
+    stored = np.diff(f["block_row_ptr"].astype(np.int64))[rows].sum()
+    assert rows.shape[0] >= (m // b) // R * 3 // 4, "most block-rows must end up in a group"
+    # (a group of one family is ~90 % full; the leftovers of every family mix; unrelated rows at this
+    # density would give ~20 %)
+    assert stored >= 0.65 * R * cols.size, "groups must be made of rows of one family"
+    h = lib.spmm_bcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, b)
+    try:
+        info = lib.spmm_get_info(h, N)
+        assert info["n_stacked_rows"] == rows.size and info["n_stack_blocks"] == cols.size
+        assert np.array_equal(lib.spmm_export(h, lib.X_BCSR_STACK_ROWS, np.int32).reshape(-1, R), rows)
+        got = run_gpu_variant(lib, h, Bs, m, N, dtype)
+        assert_close(got, Cr, S, dtype, "families b=%d" % b)
+    finally:
+        lib.spmm_destroy(h)
+
+
 # --------------------------------------------------------------------------- the paper's own gather (load/store units)
 
 

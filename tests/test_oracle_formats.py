@@ -420,17 +420,26 @@ def test_tile_schedule_matches_brute_force(seed, n_ctas, n_tt, slab_w):
 
 
 def _brute_groups(rows_cols, R, min_fill_pct):
-    """rows_cols: list of sets of block columns per block-row."""
+    """rows_cols: list of sets of block columns per block-row.  The similarity rule with plain
+    set intersections against every other free block-row (no inverted index)."""
     order = sorted(range(len(rows_cols)), key=lambda i: (-len(rows_cols[i]), i))
+    pos = {r: i for i, r in enumerate(order)}
+    free = {i for i in range(len(rows_cols)) if rows_cols[i]}
     out = []
-    for r0 in range(0, len(order) - R + 1, R):
-        cand = order[r0:r0 + R]
-        if not rows_cols[cand[-1]]:
-            break
+    for s in order:
+        if s not in free:
+            continue
+        ov = [(len(rows_cols[s] & rows_cols[r]), r) for r in free if r != s]
+        ov = [(n, r) for n, r in ov if n > 0]
+        if len(ov) < R - 1:
+            continue
+        ov.sort(key=lambda x: (-x[0], pos[x[1]]))
+        cand = sorted([s] + [r for _, r in ov[:R - 1]], key=lambda r: pos[r])
         union = set().union(*[rows_cols[i] for i in cand])
         stored = sum(len(rows_cols[i]) for i in cand)
         if 100 * stored >= min_fill_pct * R * len(union):
             out.append((cand, sorted(union)))
+            free -= set(cand)
     return out
 
 
@@ -460,11 +469,29 @@ def test_row_groups_special_cases():
     bci = np.tile(cols, 8)
     rows, ptr, gcols = F.bcsr_row_groups(brp, bci, b, 100)
     assert rows.tolist() == [[0, 1, 2, 3], [4, 5, 6, 7]] and ptr.tolist() == [0, 4, 8] and gcols.tolist() == cols.tolist() * 2
-    # block-diagonal: the union of R rows has R columns for R stored blocks, fill 100 / R %
+    # block-diagonal: no two block-rows share a block column, so nothing is similar to anything
     brp = np.arange(9, dtype=np.int32)
     bci = np.arange(8, dtype=np.int32)
-    assert F.bcsr_row_groups(brp, bci, b, 100 // R)[0].shape[0] == 2
-    assert F.bcsr_row_groups(brp, bci, b, 100 // R + 1)[0].shape[0] == 0
+    assert F.bcsr_row_groups(brp, bci, b, 1)[0].shape[0] == 0
+    # families scattered over the index range (block-row i belongs to family i % 3, all members of a
+    # family store the same columns, all lengths equal): neighbours in the order belong to different
+    # families, the groups are the families
+    fam = [np.array([0, 1, 2, 3]), np.array([10, 11, 12, 13]), np.array([20, 21, 22, 23])]
+    bci = np.concatenate([fam[i % 3] for i in range(12)]).astype(np.int32)
+    brp = np.arange(0, 4 * 13, 4, dtype=np.int32)
+    rows, ptr, gcols = F.bcsr_row_groups(brp, bci, b, 100)
+    assert rows.tolist() == [[0, 3, 6, 9], [1, 4, 7, 10], [2, 5, 8, 11]]
+    assert gcols.tolist() == fam[0].tolist() + fam[1].tolist() + fam[2].tolist()
+    # partners are the most similar rows, not the next ones in the order: row 0 = {0..7} (longest),
+    # rows 1-3 = {0}, rows 4-6 = {0, 1}.  Seed 0 takes rows 4, 5, 6 (overlap 2 beats overlap 1):
+    # fill (8 + 6) / (4 * 8) = 44 %.  At 50 % that group is rejected, row 0 stays free, and the
+    # seeds 4, 5, 6 each pick row 0 again (overlap 2, earliest in the order): rejected as well
+    bci = np.array(list(range(8)) + [0] * 3 + [0, 1] * 3, dtype=np.int32)
+    brp = np.array([0, 8, 9, 10, 11, 13, 15, 17], dtype=np.int32)
+    rows, ptr, gcols = F.bcsr_row_groups(brp, bci, b, 40)
+    assert rows.tolist() == [[0, 4, 5, 6]]
+    rows, ptr, gcols = F.bcsr_row_groups(brp, bci, b, 50)
+    assert rows.tolist() == []
     # fewer non-empty block-rows than a group needs: nothing to group
     brp = np.array([0, 3, 3, 3, 6, 6, 6, 6, 6], dtype=np.int32)
     bci = np.array([0, 1, 2, 0, 1, 2], dtype=np.int32)
