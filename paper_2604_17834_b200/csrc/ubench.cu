@@ -10,6 +10,9 @@
 //            streaming through a large array; and of st.global from registers.
 //   mix      both at once on every SM, or loads on the even SMs and stores on the odd ones: how
 //            much the two streams slow each other down, and whether that happens inside an SM.
+//   gather   aggregate rate of TMA row gathers (tile::gather4: four rows x 128 bytes per request,
+//            random rows of an L2-resident array), the operand stream of the WCSR kernel, for
+//            several numbers of resident CTAs, issuing warps and 16 KB stages in flight.
 //
 // Every wait is bounded (an iteration limit; on expiry the thread records an error and leaves),
 // device memory stays below 1 GB and each case runs for about a millisecond.  Output: one JSON
@@ -202,6 +205,45 @@ mix_kernel(const __grid_constant__ CUtensorMap tmL, const __grid_constant__ CUte
     }
 }
 
+// ----------------------------------------------------------------------------- row gather
+
+// Every warp owns `slots` stages and refills a stage as soon as its data has landed: lane l < lanes
+// requests rows 4 * (l / 2) .. + 3, 128-byte segment l % 2, as the WCSR kernel's producers do (all
+// 32 lanes: 64 gathered rows x 256 bytes = 16 KB, the kernel's stage for 2-byte types).  Rows are
+// pseudo-random.
+__global__ void __launch_bounds__(384, 1)
+gather_kernel(const __grid_constant__ CUtensorMap tmG, int slots, int lanes, int iters, int n_rows, int n_col_segs, int* err) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    __shared__ uint64_t bar[16 * 4];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warps = blockDim.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < warps * slots; ++i) mbar_init(smem_u32(&bar[i]), 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    uint32_t seed = (blockIdx.x * 64u + threadIdx.x / 2) * 2654435761u + 777u;
+    const int rg = lane >> 1, sg = lane & 1;
+    bool ok = true;
+    for (int i = 0; i < iters + slots && ok; ++i) {
+        const int sl = i % slots;
+        const uint32_t b = smem_u32(&bar[warp * slots + sl]);
+        if (i >= slots) ok = __all_sync(0xffffffffu, wait_bounded(b, ((i / slots) - 1) & 1, err));
+        if (ok && i < iters) {
+            const uint32_t sb = base + (warp * slots + sl) * (lanes * 512);
+            if (lane == 0) mbar_arrive_expect_tx(b, lanes * 512);
+            __syncwarp();
+            int r[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { seed = seed * 1664525u + 1013904223u; r[k] = static_cast<int>((seed >> 8) % static_cast<uint32_t>(n_rows)); }
+            seed = seed * 1664525u + 1013904223u;
+            const int x = static_cast<int>((seed >> 10) % static_cast<uint32_t>(n_col_segs / 2)) * 128 + sg * 64;
+            if (lane < lanes) tma_gather4_2d(sb + sg * (lanes * 256) + rg * 512, &tmG, b, x, r[0], r[1], r[2], r[3]);
+        }
+    }
+}
+
 struct Ctx {
     EncodeTiledFn fn = nullptr;
     void* src = nullptr;        // bf16 [K][N], L2 resident
@@ -285,6 +327,49 @@ void run_mix(Ctx& cx, const char* name, MixArgs a) {
     CK(cudaEventDestroy(e1));
 }
 
+void run_gather(Ctx& cx, const char* name, int ctas_per_sm, int warps, int slots, int lanes, int iters) {
+    CUtensorMap tmG;
+    const cuuint64_t dims[2] = {Ctx::N, Ctx::K};
+    const cuuint64_t strides[1] = {Ctx::N * 2};
+    const cuuint32_t box[2] = {64, 1};
+    const cuuint32_t es[2] = {1, 1};
+    if (cx.fn(&tmG, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, cx.src, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+        std::printf("{\"error\": \"gather map\"}\n");
+        std::exit(1);
+    }
+    const int smem = warps * slots * lanes * 512 + 1024;
+    if (warps > 12 || warps * slots > 64 || ctas_per_sm * (smem + 1024) > 227 * 1024) {
+        std::printf("{\"case\": \"%s\", \"error\": \"shape\"}\n", name);
+        return;
+    }
+    CK(cudaFuncSetAttribute(gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    cudaEvent_t e0, e1;
+    CK(cudaEventCreate(&e0));
+    CK(cudaEventCreate(&e1));
+    float best = 1e30f;
+    for (int rep = 0; rep < 3; ++rep) {
+        CK(cudaEventRecord(e0));
+        gather_kernel<<<cx.sms * ctas_per_sm, warps * 32, smem>>>(tmG, slots, lanes, iters, static_cast<int>(Ctx::K), static_cast<int>(Ctx::N / 64), cx.err);
+        CK(cudaEventRecord(e1));
+        CK(cudaDeviceSynchronize());
+        float ms;
+        CK(cudaEventElapsedTime(&ms, e0, e1));
+        if (rep > 0 && ms < best) best = ms;
+    }
+    int herr = 0;
+    CK(cudaMemcpy(&herr, cx.err, 4, cudaMemcpyDeviceToHost));
+    const double bytes = double(cx.sms) * ctas_per_sm * warps * iters * (lanes * 512.0);
+    const double sec = best * 1e-3;
+    std::printf("{\"case\": \"%s\", \"ms\": %.4f, \"gather_tbs\": %.2f, \"gather_B_per_clk_sm\": %.1f, \"clk_per_request_sm\": %.1f, "
+                "\"ctas_per_sm\": %d, \"warps\": %d, \"stages_per_warp\": %d, \"requests_per_stage\": %d, \"KB_in_flight_per_sm\": %d, \"wait_ran_out\": %d}\n",
+                name, best, bytes / sec / 1e12, bytes / sec / cx.sms / (cx.clk_ghz * 1e9),
+                512.0 / (bytes / sec / cx.sms / (cx.clk_ghz * 1e9)), ctas_per_sm, warps, slots, lanes, ctas_per_sm * warps * slots * lanes / 2, herr);
+    std::fflush(stdout);
+    CK(cudaEventDestroy(e0));
+    CK(cudaEventDestroy(e1));
+}
+
 }  // namespace
 
 int main(int argc, char** argv) {
@@ -333,7 +418,7 @@ int main(int argc, char** argv) {
     base.store_depth = 2;
     base.tile_cols = 32;
     base.tile_rows = 64;
-    for (int slots : {1, 2, 3}) {
+    for (int slots : {1, 2}) {
         MixArgs a = base;
         a.load_slots = slots;
         char nm[64];
@@ -344,6 +429,18 @@ int main(int argc, char** argv) {
         MixArgs a = base;
         a.load_boxes = 4; a.load_slots = 4; a.load_iters = 3000;
         run_mix(cx, "load_only_4x32KB", a);
+    }
+
+    // ---- row gathers: {resident CTAs per SM, issuing warps per CTA, 16 KB stages per warp}
+    {
+        struct G { int ctas, warps, slots, lanes; };
+        const G gs[] = {{1, 1, 1, 32}, {1, 1, 4, 32}, {1, 4, 1, 32}, {1, 4, 3, 32}, {1, 12, 1, 32}, {3, 4, 1, 32}, {2, 6, 1, 32},
+                        {3, 8, 1, 16}, {2, 12, 1, 16}, {3, 12, 1, 8}, {3, 12, 1, 10}, {3, 4, 2, 16}, {3, 8, 2, 8}};
+        for (const G& g : gs) {
+            char nm[96];
+            std::snprintf(nm, sizeof nm, "gather4_%dcta_%dwarps_x%dstages_of_%dreq", g.ctas, g.warps, g.slots, g.lanes);
+            run_gather(cx, nm, g.ctas, g.warps, g.slots, g.lanes, 6000 * 32 / (g.ctas * g.warps * g.lanes));      // ~100 MB per SM
+        }
     }
 
     // ---- MMAs beside the loads: do operand reads and TMA writes share shared-memory bandwidth?
