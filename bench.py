@@ -173,6 +173,11 @@ def workload_table():
     t["cfg2_wcsr_irregular_lsu_gather"] = ("configs[1], B rows gathered with 16-byte cp.async instead of TMA", lsu(cfg2))
     t["cfg5_wcsr_rmat_n128_lsu_gather"] = ("configs[4] N=128, B rows gathered with 16-byte cp.async instead of TMA", lsu(cfg5(128)))
     t["cfg2_wcsr_irregular_wh64"] = ("configs[1] with 64-row windows", tall(cfg2))
+    def cfg5_fp8():
+        if "rmat_fp8" not in _CACHE:
+            _CACHE["rmat_fp8"] = wl.rmat(dtype="fp8")
+        return dict(kind="wcsr", a=_CACHE["rmat_fp8"], dtype="fp8", size=16, N=128, Bdist=("normal", 0.0, 1.0))
+    t["cfg5_wcsr_rmat_n128_fp8"] = ("configs[4] N=128 with E4M3 values (windows padded to 32 columns)", cfg5_fp8)
     t["cfg5_wcsr_rmat_n128_wh64"] = ("configs[4] N=128 with 64-row windows", tall(cfg5(128)))
     t["cfg3_bcsr_llm_gate_dyn"] = ("configs[2] gate, dynamic tile scheduling", variant(cfg3_gate, dyn=True))
     t["cfg3_bcsr_llm_down_dyn"] = ("configs[2] down, dynamic tile scheduling", variant(cfg3_down, dyn=True))
@@ -215,6 +220,7 @@ ALL_OTHERS = DEFAULT_OTHERS + [
     "cfg2_wcsr_irregular_lsu_gather", "cfg5_wcsr_rmat_n128_lsu_gather",
     "cfg4_bcsr_sweep_b64_d0.1_dyn", "cfg4_bcsr_sweep_b16_d0.1_plain", "cfg4_bcsr_sweep_b32_d0.1_plain",
     "cfg4_bcsr_sweep_b16_d0.5", "cfg4_bcsr_sweep_b32_d0.5",
+    "cfg5_wcsr_rmat_n128_fp8",
     "cfg4_bcsr_families_b16", "cfg4_bcsr_families_b16_plain", "cfg4_bcsr_families_b32", "cfg4_bcsr_families_b32_plain",
     "cfg4_bcsr_sweep_b64_d0.1_ksplit", "cfg4_bcsr_sweep_b64_d0.01_ksplit",
     "cfg4_bcsr_sweep_b16_d0.1_tf32", "cfg4_bcsr_sweep_b32_d0.1_tf32", "cfg4_bcsr_sweep_b64_d0.1_tf32", "cfg4_bcsr_sweep_b128_d0.1_tf32"]

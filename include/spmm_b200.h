@@ -70,10 +70,11 @@ typedef enum {
                                     both layouts; C is fp32, the BCSR schedule static, and
                                     BCSR row groups are not formed.                           */
     SPMM_FP8_E4M3 = 3            /* 1-byte E4M3 storage (Sec. 5 names 8-bit inputs as the next
-                                    step).  BCSR only, fp32 C, static schedule, block 32, 64 or
+                                    step); fp32 C.  BCSR: static schedule, block 32, 64 or
                                     128; row-major operands need N >= 128 and N % 16 == 0,
                                     SPMM_COLMAJOR needs k % 16 == 0 (row groups are formed with
-                                    SPMM_COLMAJOR only).                                      */
+                                    SPMM_COLMAJOR only).  WCSR: windows padded to 32 columns
+                                    (b_col = 32), the TMA gather, N % 16 == 0.                */
 } spmm_dtype_t;
 
 /* Element type of C (opts.c_type).  Accumulation is fp32 either way. */
@@ -121,8 +122,8 @@ typedef enum {
 typedef struct {
     int32_t b_col;       /* WCSR: pad every window to a multiple of this many columns.
                             Default (and only supported value): 16 for 2-byte types, 8 for
-                            TF32 -- the K extent of one tensor-core instruction (Sec. 2.3,
-                            Sec. 4.1 uses 8 with TF32).                                      */
+                            TF32, 32 for E4M3 -- the K extent of one tensor-core instruction
+                            (Sec. 2.3, Sec. 4.1 uses 8 with TF32).                           */
     int32_t split_cols;  /* WCSR: sub-task size T in columns (Sec. 3.3); multiple of b_col.
                             Default: the largest of one bin's share of the padded columns, its
                             half, quarter and eighth (rounded down to a multiple of 64, clamped

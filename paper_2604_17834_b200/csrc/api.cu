@@ -423,9 +423,11 @@ int upload_wcsr_plan(spmm_handle_s* h) {
 
 // Option and size checks shared by the host and the device builder; on success *hp is a fresh handle.
 int new_wcsr_handle(spmm_handle_s** hp, int64_t m, int64_t k, int dtype, const spmm_opts_t* opts, int* b_col_out, int* T_out) {
-    if (dtype != SPMM_BF16 && dtype != SPMM_FP16 && dtype != SPMM_TF32) return SPMM_ERR_UNSUPPORTED;
+    if (dtype != SPMM_BF16 && dtype != SPMM_FP16 && dtype != SPMM_TF32 && dtype != SPMM_FP8_E4M3) return SPMM_ERR_UNSUPPORTED;
     if (int orc = check_opts(opts)) return orc;
     if (opts && opts->layout == SPMM_COLMAJOR) return SPMM_ERR_UNSUPPORTED;   // BCSR only
+    // 8-bit inputs: fp32 C, the TMA gather
+    if (dtype == SPMM_FP8_E4M3 && opts && (opts->c_type != SPMM_C_FP32 || opts->gather != SPMM_GATHER_TMA)) return SPMM_ERR_UNSUPPORTED;
     if (opts && opts->schedule == SPMM_SCHED_DYNAMIC) return SPMM_ERR_UNSUPPORTED;
     const int es = elem_size(dtype);
     const int b_col_default = 32 / es;
@@ -524,13 +526,12 @@ int make_view(CsrView* v, int64_t m, int64_t k, const int64_t* row_ptr, const in
 int encode_gather_map(CUtensorMap* map, int dtype, const void* base, uint64_t rows, uint64_t cols) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return SPMM_ERR_CUDA;
-    const uint32_t es = dtype == SPMM_TF32 ? 4 : 2;
+    const uint32_t es = static_cast<uint32_t>(elem_size(dtype));
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {cols * es};
     const cuuint32_t box[2] = {128 / es, 1};
     const cuuint32_t estr[2] = {1, 1};
-    const CUtensorMapDataType dt = dtype == SPMM_TF32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
-                                 : (dtype == SPMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
+    const CUtensorMapDataType dt = tmap_dtype(dtype);
     const CUtensorMapSwizzle swz = dtype == SPMM_TF32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B;
     const CUtensorMapL2promotion promo = cols * es >= 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_NONE;
     CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,

@@ -313,8 +313,6 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                 }
             }
-            if (lane == 0) {
-            }
             if (!ok && lane == 0) {
                 // leave no bulk copy in flight: wait (bounded) for the fills already issued
                 const uint32_t first = it > STAGES ? it - STAGES : 0;
@@ -387,8 +385,6 @@ bcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (pe > pb) tc_commit(accf_bar(acc));
                     else mbar_arrive(accf_bar(acc));
                 }
-            }
-            if (lane == 0) {
             }
         }
     } else if (warp < 6) {

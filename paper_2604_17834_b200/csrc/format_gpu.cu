@@ -417,7 +417,8 @@ __global__ void wcsr_values_kernel(int64_t m, int wh, int b_col, const int64_t* 
             }
             uint8_t* dst = packed + wcsr_packed_offset(wh, b_col, ES, r, base + lo);
             const uint8_t* src = vals + static_cast<size_t>(p) * ES;
-            if constexpr (ES == 2) *reinterpret_cast<uint16_t*>(dst) = *reinterpret_cast<const uint16_t*>(src);
+            if constexpr (ES == 1) *dst = *src;
+            else if constexpr (ES == 2) *reinterpret_cast<uint16_t*>(dst) = *reinterpret_cast<const uint16_t*>(src);
             else *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(src);
         }
     }
@@ -509,7 +510,7 @@ int build_wcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int3
                       int32_t** d_window_row_ptr, int32_t** d_window_col_idx, uint8_t** d_packed, uint8_t** d_grp_class) {
     *d_grp_class = nullptr;
     if (wh != 16 && wh != 64) return SPMM_ERR_UNSUPPORTED;
-    if ((es != 2 && es != 4) || b_col * es != 32) return SPMM_ERR_UNSUPPORTED;
+    if ((es != 1 && es != 2 && es != 4) || b_col * es != 32) return SPMM_ERR_UNSUPPORTED;
     if (T < 0 || T % b_col != 0 || n_bins <= 0) return SPMM_ERR_INVALID_ARG;
     if (m < 0 || k < 0 || !d_row_ptr) return SPMM_ERR_INVALID_ARG;
     const int64_t nwin = (m + wh - 1) / wh;
@@ -617,7 +618,9 @@ int build_wcsr_device(int64_t m, int64_t k, const int64_t* d_row_ptr, const int3
     if (n > 0) {
         wcsr_cols_kernel<<<2048, 256, 0, st>>>(d_keys, d_flags + 2, d_ustart, *d_window_row_ptr, *d_window_col_idx);
         const unsigned vgrid = static_cast<unsigned>(std::min<int64_t>((m + 7) / 8, 8192));
-        if (es == 2)
+        if (es == 1)
+            wcsr_values_kernel<1><<<vgrid, 256, 0, st>>>(m, wh, b_col, d_row_ptr, d_col_idx, d_vals, d_cnt, *d_window_row_ptr, *d_window_col_idx, *d_packed);
+        else if (es == 2)
             wcsr_values_kernel<2><<<vgrid, 256, 0, st>>>(m, wh, b_col, d_row_ptr, d_col_idx, d_vals, d_cnt, *d_window_row_ptr, *d_window_col_idx, *d_packed);
         else
             wcsr_values_kernel<4><<<vgrid, 256, 0, st>>>(m, wh, b_col, d_row_ptr, d_col_idx, d_vals, d_cnt, *d_window_row_ptr, *d_window_col_idx, *d_packed);

@@ -129,7 +129,7 @@ struct WcsrParams {
     uint64_t wait_limit_ns;
 };
 
-// dtype: 0 bf16, 1 fp16, 2 tf32.  groups: 1 or 2.  tmB: 2-D map of B (k rows x N), box = 128
+// dtype: 0 bf16, 1 fp16, 2 tf32, 3 E4M3 (fp32 C).  tmB: 2-D map of B (k rows x N), box = 128
 // bytes x 1 row, 128-byte swizzle (32-byte atoms for tf32), used in row-gather mode.
 // narrow: the N <= 64 variant for 2-byte types at window height 16 (p.fills / p.bin_fill cut to kWcsrNarrowCols).
 // lsu_gather: the comparison variant whose producers gather B rows with 16-byte cp.async copies through the

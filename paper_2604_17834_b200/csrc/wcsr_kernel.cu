@@ -356,11 +356,12 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
         // ------------------------------------------------------------------ MMA issuer
         // The whole warp walks the fill list (descriptor windows via shuffles) and waits for
         // stages and accumulators; one elected lane issues the MMAs and commits.
-        constexpr uint32_t idesc = make_idesc(FMT, 128, kWH, 1, 0);
+        // (8-bit floats: format code 0 = E4M3 in both operand fields)
+        constexpr uint32_t idesc = make_idesc(FMT == 3 ? 0 : FMT, 128, kWH, 1, 0);
         // narrow variant: only the first 64-token atom is staged; the MMA's second atom is made to
         // alias it (atom stride 0) so that no address outside the stage is read; its TMEM lanes
         // (tokens 64..127) are never stored
-        const uint64_t adesc0 = make_smem_desc(0, NARROW ? 0 : Cfg::kAtomStride, ES == 2 ? 1024 : 512, ES == 2 ? SWZ_128B : SWZ_128B_BASE32B);
+        const uint64_t adesc0 = make_smem_desc(0, NARROW ? 0 : Cfg::kAtomStride, ES == 4 ? 512 : 1024, ES == 4 ? SWZ_128B_BASE32B : SWZ_128B);
         const uint64_t bdesc0 = make_smem_desc(0, kWH * 16, 128, SWZ_NONE);
         const bool leader = elect_one();
         SegIter seg;
@@ -402,7 +403,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                         auto issue = [&](int ks) {
                             // the item's first MMA overwrites the accumulator: no zeroing pass
                             if (leader)
-                                umma_ss<FMT == 2>(d0, a0 + ((ks * (Cfg::kKStep / 8) * 1024) >> 4),
+                                umma_kind<FMT == 3 ? 2 : (FMT == 2 ? 1 : 0)>(d0, a0 + ((ks * (Cfg::kKStep / 8) * 1024) >> 4),
                                                   b0 + ((ks * (kWH * 32)) >> 4), idesc, (ks > 0 || !fresh) ? 1u : 0u);
                         };
                         constexpr int kFullSteps = KT / Cfg::kKStep;
@@ -583,6 +584,7 @@ cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cud
 template <int WH>
 cudaError_t launch_wh(int dtype, int c16, const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
     if (dtype == 2) return launch_one<4, 2, WH, 0>(tmB, p, sms, stream);
+    if (dtype == 3) return c16 ? cudaErrorInvalidValue : launch_one<1, 3, WH, 0>(tmB, p, sms, stream);   // E4M3: fp32 C
     if (dtype == 1) return c16 ? launch_one<2, 0, WH, 1>(tmB, p, sms, stream) : launch_one<2, 0, WH, 0>(tmB, p, sms, stream);
     if (dtype == 0) return c16 ? launch_one<2, 1, WH, 1>(tmB, p, sms, stream) : launch_one<2, 1, WH, 0>(tmB, p, sms, stream);
     return cudaErrorInvalidValue;

@@ -114,11 +114,11 @@ def _wcsr_case(lib, a, dtype, N, T=0, Bdist=("normal", 0.0, 1.0), seed=19):
     Bs = wl.dense(seed, a["k"], N, Bdist, dtype)
     h = lib.spmm_wcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], dtype, 16, split_cols=T)
     try:
-        b_col = 8 if dtype == "tf32" else 16
+        b_col = 32 // wl.elem_size(dtype)
         info = lib.spmm_get_info(h, N)
         f = F.wcsr_from_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], 16, b_col)
         np_dt = wl.storage_np_dtype(dtype)
-        bits = np.uint32 if dtype == "tf32" else np.uint16
+        bits = {4: np.uint32, 2: np.uint16, 1: np.uint8}[wl.elem_size(dtype)]
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_ROW_PTR, np.int32), f["window_row_ptr"])
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_COL_IDX, np.int32), f["window_col_idx"])
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_VALUES, np_dt).view(bits), f["values"].view(bits).ravel())
@@ -142,6 +142,15 @@ def _wcsr_case(lib, a, dtype, N, T=0, Bdist=("normal", 0.0, 1.0), seed=19):
 def test_wcsr_small(lib, dtype, N):
     a = wl.random_csr(51, 1000, 900, 0.02, dtype, empty_rows=tuple(range(32, 64)))
     _, info = _wcsr_case(lib, a, dtype, N, T=64)
+    assert info["n_split"] > 0 and info["n_empty"] >= 2
+
+
+@pytest.mark.parametrize("N", [128, 32, 256, 80, 336])     # 80: ragged single tile; 336: three tiles, ragged tail
+def test_wcsr_fp8_e4m3_small(lib, N):
+    """E4M3 values (Sec. 5 names 8-bit inputs as the next step): windows padded to 32 columns = one
+    K step of the 8-bit MMA, 128 gathered rows of 128 bytes per stage, fp32 C."""
+    a = wl.random_csr(53, 1000, 900, 0.03, "fp8", empty_rows=tuple(range(32, 64)))
+    _, info = _wcsr_case(lib, a, "fp8", N, T=64, Bdist=("uniform", -1.0, 1.0))
     assert info["n_split"] > 0 and info["n_empty"] >= 2
 
 

@@ -100,8 +100,8 @@ def test_wcsr_c16(lib, dtype, N):
         lib.spmm_destroy(h)
 
 
-@pytest.mark.parametrize("dtype", ["tf32", "fp16", "bf16"])
-@pytest.mark.parametrize("N", [128, 72, 328])
+@pytest.mark.parametrize("dtype", ["tf32", "fp16", "bf16", "fp8"])
+@pytest.mark.parametrize("N", [128, 80, 336])
 def test_wcsr_window_height_64(lib, dtype, N):
     """The paper's own window height (Sec. 4.1): 64-row windows, MMA N = 64.  Format arrays
     bit-exact against the format oracle, result against the SpMM oracle, split + empty windows."""
@@ -110,9 +110,9 @@ def test_wcsr_window_height_64(lib, dtype, N):
     Bs = wl.dense(19, 900, N, ("normal", 0.0, 1.0), dtype)
     h = lib.spmm_wcsr_create_csr(1000, 900, a["row_ptr"], a["col_idx"], a["vals"], dtype, 64, split_cols=128)
     try:
-        b_col = 8 if dtype == "tf32" else 16
+        b_col = 32 // wl.elem_size(dtype)
         f = F.wcsr_from_csr(1000, 900, a["row_ptr"], a["col_idx"], a["vals"], 64, b_col)
-        bits = np.uint32 if dtype == "tf32" else np.uint16
+        bits = {4: np.uint32, 2: np.uint16, 1: np.uint8}[wl.elem_size(dtype)]
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_ROW_PTR, np.int32), f["window_row_ptr"])
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_COL_IDX, np.int32), f["window_col_idx"])
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_VALUES, wl.storage_np_dtype(dtype)).view(bits),
@@ -228,7 +228,8 @@ def test_bcsr_built_on_the_gpu_is_bit_exact(lib, dtype, b, m, k):
 
 @pytest.mark.parametrize("dtype,wh,m,k,dens", [("tf32", 16, 1000, 900, 0.02), ("fp16", 16, 333, 517, 0.05),
                                                 ("bf16", 64, 1000, 4000, 0.01), ("fp16", 16, 5000, 70000, 0.0005),
-                                                ("tf32", 64, 130, 70, 0.2)])
+                                                ("tf32", 64, 130, 70, 0.2), ("fp8", 16, 1000, 900, 0.02),
+                                                ("fp8", 64, 400, 2000, 0.01)])
 def test_wcsr_built_on_the_gpu_is_bit_exact(lib, dtype, wh, m, k, dens):
     """Window condensation and value packing as GPU kernels (sort / unique of (window, column)
     keys): every exported array equals the format oracle's, plan and bins included, and the
@@ -242,9 +243,9 @@ def test_wcsr_built_on_the_gpu_is_bit_exact(lib, dtype, wh, m, k, dens):
     h = lib.spmm_wcsr_create_csr_device(m, k, rp.data_ptr(), ci.data_ptr(), va.data_ptr(), dtype, wh, split_cols=64)
     h0 = lib.spmm_wcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, wh, split_cols=64)
     try:
-        b_col = 8 if dtype == "tf32" else 16
+        b_col = 32 // wl.elem_size(dtype)
         f = F.wcsr_from_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], wh, b_col)
-        bits = np.uint32 if dtype == "tf32" else np.uint16
+        bits = {4: np.uint32, 2: np.uint16, 1: np.uint8}[wl.elem_size(dtype)]
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_ROW_PTR, np.int32), f["window_row_ptr"])
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_WINDOW_COL_IDX, np.int32), f["window_col_idx"])
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_VALUES, wl.storage_np_dtype(dtype)).view(bits),
@@ -255,7 +256,7 @@ def test_wcsr_built_on_the_gpu_is_bit_exact(lib, dtype, wh, m, k, dens):
         assert np.array_equal(lib.spmm_export(h, lib.X_WCSR_GROUP_CLASS, np.uint8), lib.spmm_export(h0, lib.X_WCSR_GROUP_CLASS, np.uint8))
         i1, i0 = lib.spmm_get_info(h, 128), lib.spmm_get_info(h0, 128)
         assert i1 == i0
-        N = 136
+        N = 144
         Bs = wl.dense(3, k, N, ("normal", 0.0, 1.0), dtype)
         C = run_gpu(lib, h, Bs, m, N)
         assert np.array_equal(C, run_gpu(lib, h0, Bs, m, N))

@@ -37,7 +37,7 @@ def test_library_exports_every_declared_symbol(lib):
 
 def _bits(a):
     a = np.ascontiguousarray(a)
-    return a.view({2: np.uint16, 4: np.uint32}[a.dtype.itemsize])
+    return a.view({1: np.uint8, 2: np.uint16, 4: np.uint32}[a.dtype.itemsize])
 
 
 BCSR_CASES = [
@@ -216,14 +216,14 @@ def test_bcsr_row_groups_and_their_schedules_are_bit_exact(lib, b, N, n_ctas, fi
 
 
 WCSR_CASES = [("tf32", 1000, 900, 0.01, 64), ("fp16", 333, 517, 0.05, 32), ("bf16", 160, 4000, 0.2, 128),
-              ("fp16", 16, 40, 0.5, 16)]
+              ("fp16", 16, 40, 0.5, 16), ("fp8", 700, 1300, 0.03, 96)]
 
 
 @pytest.mark.parametrize("wh", [16, 64])
 @pytest.mark.parametrize("dtype,m,k,dens,T", WCSR_CASES)
 def test_wcsr_format_plan_and_bins_are_bit_exact(lib, dtype, m, k, dens, T, wh):
     a = wl.random_csr(41 + m, m, k, dens, dtype, empty_rows=tuple(range(16, min(32, m))))
-    b_col = 8 if dtype == "tf32" else 16
+    b_col = 32 // wl.elem_size(dtype)
     h = lib.spmm_wcsr_create_csr(m, k, a["row_ptr"], a["col_idx"], a["vals"], dtype, wh, split_cols=T,
                                  host_only=True, n_ctas=5)
     try:
@@ -354,6 +354,17 @@ def test_malformed_input_is_rejected(lib):
                 host_only=True) == lib.SPMM_ERR_INVALID_ARG
     assert code(mw, 2, 4, rp, np.array([0, 1, 2], np.int32), v, "fp16", 16, b_col=8,
                 host_only=True) == lib.SPMM_ERR_UNSUPPORTED
+    # E4M3 WCSR: fp32 C and the TMA gather only; windows are padded to 32 columns
+    v8 = np.full(3, 0x38, np.uint8)
+    assert code(mw, 2, 4, rp, np.array([0, 1, 2], np.int32), v8, "fp8", 16, host_only=True,
+                c_type=lib.C_SAME_AS_INPUT) == lib.SPMM_ERR_UNSUPPORTED
+    assert code(mw, 2, 4, rp, np.array([0, 1, 2], np.int32), v8, "fp8", 16, host_only=True,
+                gather=lib.GATHER_LSU) == lib.SPMM_ERR_UNSUPPORTED
+    assert code(mw, 2, 4, rp, np.array([0, 1, 2], np.int32), v8, "fp8", 16, host_only=True,
+                b_col=16) == lib.SPMM_ERR_UNSUPPORTED
+    h8 = mw(2, 4, rp, np.array([0, 1, 2], np.int32), v8, "fp8", 16, host_only=True)
+    assert lib.spmm_export(h8, lib.X_WCSR_WINDOW_COL_IDX, np.int32).tolist() == [0, 1, 2] + [-1] * 29
+    lib.spmm_destroy(h8)
     dup_r, dup_c = np.array([0, 0], np.int32), np.array([1, 1], np.int32)
     assert code(lib.spmm_bcsr_create_coo, 2, 4, dup_r, dup_c, v[:2], "fp16", 16, host_only=True) == lib.SPMM_ERR_UNSORTED
     lib.spmm_destroy(None)                                     # NULL is accepted
