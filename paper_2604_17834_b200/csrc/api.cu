@@ -134,8 +134,6 @@ struct spmm_handle_s {
     int32_t* d_bin_fill = nullptr;
     int32_t* d_fills_narrow = nullptr;    // WCSR narrow-operand variant (2-byte types, height 16)
     int32_t* d_bin_fill_narrow = nullptr;
-    int32_t* d_fills_wide = nullptr;      // WCSR two-tile passes (2-byte types, height 16, N > 128)
-    int32_t* d_bin_fill_wide = nullptr;
     uint8_t* d_grp_class = nullptr;  // WCSR: reuse class per group of four padded columns (gather hints)
     int32_t* d_merge = nullptr;      // window | first | nparts, each [n_merge]
     int n_merge = 0;
@@ -194,8 +192,6 @@ void free_handle(spmm_handle_s* h) {
         cudaFree(h->d_bin_fill);
         cudaFree(h->d_fills_narrow);
         cudaFree(h->d_bin_fill_narrow);
-        cudaFree(h->d_fills_wide);
-        cudaFree(h->d_bin_fill_wide);
         cudaFree(h->d_grp_class);
         cudaFree(h->d_merge);
         cudaFree(h->d_status);
@@ -413,10 +409,6 @@ int upload_wcsr_plan(spmm_handle_s* h) {
     }
     if (!rc) rc = upload(&h->d_fills, f.fills.data(), f.fills.size() * 4);
     if (!rc) rc = upload(&h->d_bin_fill, f.bin_fill.data(), f.bin_fill.size() * 4);
-    if (!rc && !f.bin_fill_wide.empty()) {
-        rc = upload(&h->d_fills_wide, f.fills_wide.data(), f.fills_wide.size() * 4);
-        if (!rc) rc = upload(&h->d_bin_fill_wide, f.bin_fill_wide.data(), f.bin_fill_wide.size() * 4);
-    }
     if (!rc && !f.bin_fill_narrow.empty()) {
         rc = upload(&h->d_fills_narrow, f.fills_narrow.data(), f.fills_narrow.size() * 4);
         if (!rc) rc = upload(&h->d_bin_fill_narrow, f.bin_fill_narrow.data(), f.bin_fill_narrow.size() * 4);
@@ -905,16 +897,14 @@ int64_t wcsr_workspace_bytes(const spmm_handle_s* h, int64_t N) {
 
 int launch_wcsr_all(spmm_handle_s* h, const void* B, void* C, float* partial, int64_t N, cudaStream_t stream) {
     const WcsrHost& f = h->wcsr;
+    const int bnt = 128;                    // tokens per tile; wider B takes one pass per tile
     WcsrParams p;
     p.bin_ptr = h->d_bin_ptr;
     p.items = reinterpret_cast<const int4*>(h->d_items);
     // narrow dense operand: the variant whose stages hold more columns
     const bool narrow = h->d_bin_fill_narrow != nullptr && N <= kWcsrNarrowMaxN && !h->lsu_gather;
-    // wide dense operand: two 128-token tiles per pass over a bin
-    const bool wide = h->d_bin_fill_wide != nullptr && N > 128 && !h->lsu_gather;
-    const int bnt = wide ? 256 : 128;       // tokens per pass
-    p.fills = reinterpret_cast<const int2*>(narrow ? h->d_fills_narrow : (wide ? h->d_fills_wide : h->d_fills));
-    p.bin_fill = narrow ? h->d_bin_fill_narrow : (wide ? h->d_bin_fill_wide : h->d_bin_fill);
+    p.fills = reinterpret_cast<const int2*>(narrow ? h->d_fills_narrow : h->d_fills);
+    p.bin_fill = narrow ? h->d_bin_fill_narrow : h->d_bin_fill;
     p.col_idx = h->d_idx;
     // Gather hints: B rows whose reuse class fits half of a 126 MB L2 at this dense width are
     // fetched evict-last, everything else evict-first.  Class c holds at most
@@ -940,7 +930,7 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, void* C, float* partial, in
     if (!f.tasks.empty()) {
         int rc = ensure_tmB(h, B, N, 1);
         if (rc) return rc;
-        cudaError_t e = launch_wcsr(h->dtype, f.wh, h->c16, narrow ? 1 : 0, h->lsu_gather ? 1 : 0, wide ? 1 : 0, h->tmB, p, h->sms, stream);
+        cudaError_t e = launch_wcsr(h->dtype, f.wh, h->c16, narrow ? 1 : 0, h->lsu_gather ? 1 : 0, h->tmB, p, h->sms, stream);
         if (e != cudaSuccess) return SPMM_ERR_CUDA;
     }
     MergeParams mp;

@@ -531,9 +531,6 @@ int plan_wcsr(WcsrHost* out, int T, int n_bins, int es) {
     out->fills_narrow.clear();
     out->bin_fill_narrow.clear();
     if (!rc && es == 2 && out->wh == 16) rc = cut(kWcsrNarrowCols, &out->fills_narrow, &out->bin_fill_narrow);
-    out->fills_wide.clear();
-    out->bin_fill_wide.clear();
-    if (!rc && wcsr_wide_pass(es, out->wh)) rc = cut(out->kt / 2, &out->fills_wide, &out->bin_fill_wide);
     if (rc) return rc;
     return SPMM_OK;
 }

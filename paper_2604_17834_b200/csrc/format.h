@@ -122,7 +122,6 @@ struct WcsrHost {
     // the same for the narrow-operand kernel variant (stages of kWcsrNarrowCols columns); empty
     // unless the value type is 2 bytes wide and the window height 16
     std::vector<int32_t> fills_narrow, bin_fill_narrow;
-    std::vector<int32_t> fills_wide, bin_fill_wide;     // two token tiles per pass (N > 128): fills of half a stage's columns
     // Device-private gather hint (no effect on results): reuse class of every group of four
     // consecutive padded columns, one byte each.  A column's class says how high its B row ranks
     // by the number of windows that gather it: 7 = among the 16 Ki most gathered rows, 6 = 32 Ki,

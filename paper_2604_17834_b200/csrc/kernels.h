@@ -97,11 +97,6 @@ constexpr int wcsr_stage_cols(int es) { return WCSR_STAGE_ROW_BYTES / es; }
 // 3 KB of A): a third fewer stage hand-shakes per column, which is what bounds the narrow case.
 constexpr int kWcsrNarrowCols = 96;
 constexpr int kWcsrNarrowMaxN = 64;
-// Wide dense operands (2-byte types, window height 16, N > 128): a pass takes two 128-token tiles
-// at once -- a stage holds half as many columns (32) with 512 bytes of every gathered row, so the
-// packed A tiles and the column indices are fetched once for both tiles and the four 128-byte
-// pieces of a row of B are requested together.
-constexpr bool wcsr_wide_pass(int es, int wh) { return es == 2 && wh == 16; }
 constexpr int wcsr_stages(int es, int wh) { return wh == 64 ? 4 : (es == 4 ? 6 : 4); }
 constexpr int wcsr_producer_warps(int es, int wh) { return wh == 64 ? 4 : (es == 4 ? 6 : 4); }
 constexpr int wcsr_bins_per_sm(int es, int wh) { return wh == 64 ? 2 : (es == 4 ? 2 : 3); }
@@ -129,7 +124,7 @@ struct WcsrParams {
     float* partial;              // [n_slots][window height][N]
     int64_t m, N;
     int32_t n_bins;
-    int32_t n_tt;                // passes over a bin = ceil(N / tokens per pass) (128, or 256 in the wide variant)
+    int32_t n_tt;                // token tiles = ceil(N / (128 * groups))
     int* status;
     uint64_t wait_limit_ns;
 };
@@ -139,9 +134,7 @@ struct WcsrParams {
 // narrow: the N <= 64 variant for 2-byte types at window height 16 (p.fills / p.bin_fill cut to kWcsrNarrowCols).
 // lsu_gather: the comparison variant whose producers gather B rows with 16-byte cp.async copies through the
 // load/store units instead of TMA (window height 16, fp32 C, not narrow); tmB is then unused.
-// wide: the N > 128 variant of wcsr_wide_pass (p.fills / p.bin_fill cut to half a stage's columns,
-// p.n_tt counts passes of 256 tokens).
-cudaError_t launch_wcsr(int dtype, int wh, int c16, int narrow, int lsu_gather, int wide, const CUtensorMap& tmB, const WcsrParams& p,
+cudaError_t launch_wcsr(int dtype, int wh, int c16, int narrow, int lsu_gather, const CUtensorMap& tmB, const WcsrParams& p,
                         int sms, cudaStream_t stream);
 
 struct MergeParams {

@@ -1,8 +1,7 @@
 // WCSR SpMM kernel for sm_100a (Sec. 3.2 - 3.3 of the paper, re-designed for Blackwell).
 //
 // Work item: one sub-task of the split plan (a run of `count` condensed columns of one
-// 16-row window) times one tile of 128 columns of B ("tokens"; wider B: one pass per tile, or per
-// two tiles in the wide variant, TT = 2).  It accumulates
+// 16-row window) times one tile of 128 columns of B ("tokens"; wider B: one pass per tile).  It accumulates
 //     D[n, r] += sum_q  B[window_col_idx[q], n0 + n] * values[r, q]
 // with the tokens on the 128 TMEM lanes (MMA M side; the gathered B rows are written to
 // shared memory in the MN-major 128-byte-swizzled layout tcgen05.mma reads) and the 16
@@ -36,17 +35,13 @@ namespace {
 // tensor pipe takes a 128 x 16 MMA every 39 cycles whether or not it depends on the previous
 // one, and the extra TMEM loads lengthen the epilogue.)
 
-// TT = token tiles per pass over a bin: 1, or 2 in the wide variant (N > 128), whose stages hold
-// TT * 128 tokens of every gathered row and whose items own TT accumulator tiles.
-template <int ES, int WH, int KT, int STAGES, bool NARROW = false, int TT = 1>
+template <int ES, int WH, int KT, int STAGES, bool NARROW = false>
 struct WcsrCfg {
     static constexpr int kWH = WH;                          // window height = MMA N
     static constexpr int kKStep = 32 / ES;                  // columns per MMA (= b_col)
     static constexpr int kBnT = 128;                        // tokens per tile = TMEM lanes
-    static constexpr int kPassTok = kBnT * TT;              // tokens per pass
-    // 128-byte segments per gathered row: all tokens of the pass, or (narrow: N <= 64, 2-byte types) one
-    static constexpr int kSegsTile = kBnT * ES / 128;       // segments of one token tile
-    static constexpr int kSegs = NARROW ? 1 : TT * kSegsTile;
+    // 128-byte segments per gathered row: all 128 tokens, or (narrow: N <= 64, 2-byte types) one
+    static constexpr int kSegs = NARROW ? 1 : kBnT * ES / 128;
     static constexpr int kRowBytes = kSegs * 128;
     static constexpr int kGathers = (KT / 4) * kSegs;       // row-gather instructions per full fill
     static constexpr int kRounds = (kGathers + 31) / 32;    // per lane
@@ -60,13 +55,12 @@ struct WcsrCfg {
     static_assert(kCtasPerSm * (STAGES * kStageBytes + 1024 + 256 + 1024) <= 227 * 1024, "shared memory over-subscribed");
     // items with live accumulators
     static constexpr int kNAcc = 4;                         // items with live accumulators
-    static constexpr int kAccCols = TT * kWH;               // TMEM columns of one item
+    static constexpr int kAccCols = kWH;                    // TMEM columns of one item
     static constexpr int kTmemCols = kNAcc * kAccCols;      // 64 or 256
     static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 + 256;
     static_assert(KT % 8 == 0 && KT % kKStep == 0 && KT <= 128, "stage shape");
     static_assert(kGathers <= 32, "one gather instruction per lane and fill");
-    static_assert(!NARROW || (ES == 2 && WH == 16 && TT == 1), "narrow variant: 2-byte types, window height 16");
-    static_assert(TT == 1 || TT == 2, "one or two token tiles per pass");
+    static_assert(!NARROW || (ES == 2 && WH == 16), "narrow variant: 2-byte types, window height 16");
     static_assert(kStageBytes % 1024 == 0, "stage alignment");
 };
 
@@ -92,11 +86,10 @@ struct SegIter {
 // TMA -- the cooperative gather with 128-bit loads that Sec. 3.2 describes, here as 16-byte
 // cp.async copies that every lane of the producer warp places at the swizzled position the MMA
 // expects.  Kept as a selectable variant so that the two gathers can be measured side by side.
-template <int ES, int FMT, int WH, int KT, int STAGES, int PW, int CT, bool NARROW, bool LSU = false, int TT = 1>
-__global__ void __launch_bounds__((PW + 5) * 32, WcsrCfg<ES, WH, KT, STAGES, NARROW, TT>::kCtasPerSm)
+template <int ES, int FMT, int WH, int KT, int STAGES, int PW, int CT, bool NARROW, bool LSU = false>
+__global__ void __launch_bounds__((PW + 5) * 32, WcsrCfg<ES, WH, KT, STAGES, NARROW>::kCtasPerSm)
 wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
-    using Cfg = WcsrCfg<ES, WH, KT, STAGES, NARROW, TT>;
-    static_assert(TT == 1 || !LSU, "the load/store-unit gather takes one token tile per pass");
+    using Cfg = WcsrCfg<ES, WH, KT, STAGES, NARROW>;
     constexpr int kWH = WH;
     constexpr int kProducerWarps = PW;          // warps 0 .. PW-1; MMA warp PW; epilogue PW+1 .. PW+4
     constexpr int kMmaWarp = PW;
@@ -283,8 +276,8 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
         bool rdy0 = false, rdy1 = false;
         while (ok && seg.next(p)) {
             const int f0 = __ldg(p.bin_fill + seg.b), f1 = __ldg(p.bin_fill + seg.b + 1);
-            const int n0 = seg.tt * Cfg::kPassTok;
-            const int nvalid = static_cast<int>(min_i64(Cfg::kPassTok, N - n0));
+            const int n0 = seg.tt * Cfg::kBnT;
+            const int nvalid = static_cast<int>(min_i64(Cfg::kBnT, N - n0));
             const int nseg = (nvalid * ES + 127) >> 7;       // 128-byte segments that hold tokens < N
             int2 win = (f0 + lane < f1) ? __ldg(p.fills + f0 + lane) : kNoDesc;
             for (int wbase = f0; wbase < f1 && ok; wbase += 32) {
@@ -379,8 +372,6 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
         bool ok = true;
         while (ok && seg.next(p)) {
             const int f0 = __ldg(p.bin_fill + seg.b), f1 = __ldg(p.bin_fill + seg.b + 1);
-            // token tiles of this pass that hold tokens < N
-            const int ntile = static_cast<int>((min_i64(Cfg::kPassTok, N - static_cast<int64_t>(seg.tt) * Cfg::kPassTok) + 127) >> 7);
             int2 win = (f0 + lane < f1) ? __ldg(p.fills + f0 + lane) : kNoDesc;
             for (int wbase = f0; wbase < f1 && ok; wbase += 32) {
                 const int2 nwin = (wbase + 32 + lane < f1) ? __ldg(p.fills + wbase + 32 + lane) : kNoDesc;
@@ -411,12 +402,9 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                         const uint64_t b0 = bdesc0 + ((sb + Cfg::kDenseBytes) >> 4);
                         auto issue = [&](int ks) {
                             // the item's first MMA overwrites the accumulator: no zeroing pass
-#pragma unroll
-                            for (int t = 0; t < TT; ++t)
-                                if (leader && t < ntile)
-                                    umma_kind<FMT == 3 ? 2 : (FMT == 2 ? 1 : 0)>(d0 + t * kWH,
-                                                      a0 + ((t * Cfg::kSegsTile * Cfg::kAtomStride + ks * (Cfg::kKStep / 8) * 1024) >> 4),
-                                                      b0 + ((ks * (kWH * 32)) >> 4), idesc, (ks > 0 || !fresh) ? 1u : 0u);
+                            if (leader)
+                                umma_kind<FMT == 3 ? 2 : (FMT == 2 ? 1 : 0)>(d0, a0 + ((ks * (Cfg::kKStep / 8) * 1024) >> 4),
+                                                  b0 + ((ks * (kWH * 32)) >> 4), idesc, (ks > 0 || !fresh) ? 1u : 0u);
                         };
                         constexpr int kFullSteps = KT / Cfg::kKStep;
                         if (nks == kFullSteps) {                 // a full stage: straight-line code
@@ -447,7 +435,7 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
         bool ok = true;
         while (ok && seg.next(p)) {
             const int i0 = __ldg(p.bin_ptr + seg.b), i1 = __ldg(p.bin_ptr + seg.b + 1);
-            const int n0 = seg.tt * Cfg::kPassTok;
+            const int n0 = seg.tt * Cfg::kBnT;
             const int4 kNoItem = make_int4(0, 0, 0, 0);
             int4 win = (i0 + lane < i1) ? __ldg(p.items + i0 + lane) : kNoItem;
             for (int wbase = i0; wbase < i1 && ok; wbase += 32) {
@@ -476,36 +464,29 @@ wcsr_spmm_kernel(const __grid_constant__ CUtensorMap tmB, const WcsrParams p) {
                     const uint32_t aph = (item / Cfg::kNAcc) & 1u;
                     if (!__all_sync(0xffffffffu, mbar_wait(accf_bar(acc), aph, ctl, 14))) { ok = false; break; }
                     tc_fence_after_sync();
-                    // tile by tile: TMEM -> registers -> global; the buffer is released once the
-                    // last tile has been read
+                    float v[kWH];
                     const uint32_t tbase = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + acc * Cfg::kAccCols;
 #pragma unroll
-                    for (int t = 0; t < TT; ++t) {
-                        float v[kWH];
+                    for (int c = 0; c < kWH; c += 16) {
+                        uint32_t u[16];
+                        tmem_ld_x16(tbase + c, u);
+                        tmem_ld_wait();
 #pragma unroll
-                        for (int c = 0; c < kWH; c += 16) {
-                            uint32_t u[16];
-                            tmem_ld_x16(tbase + t * kWH + c, u);
-                            tmem_ld_wait();
+                        for (int jr = 0; jr < 16; ++jr) v[c + jr] = __uint_as_float(u[jr]);
+                    }
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(acce_bar(acc));
+                    const int n = n0 + qd * 32 + lane;
+                    if (n < N) {
+                        if (sizeof(CElem) == 4 || slot >= 0) {
 #pragma unroll
-                            for (int jr = 0; jr < 16; ++jr) v[c + jr] = __uint_as_float(u[jr]);
-                        }
-                        if (t == TT - 1) {
-                            tc_fence_before_sync();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(acce_bar(acc));
-                        }
-                        const int n = n0 + t * Cfg::kBnT + qd * 32 + lane;
-                        if (n < N) {
-                            if (sizeof(CElem) == 4 || slot >= 0) {
+                            for (int jr = 0; jr < kWH; ++jr)
+                                if (jr < rows) out[static_cast<int64_t>(jr) * N + n] = v[jr];
+                        } else {
 #pragma unroll
-                                for (int jr = 0; jr < kWH; ++jr)
-                                    if (jr < rows) out[static_cast<int64_t>(jr) * N + n] = v[jr];
-                            } else {
-#pragma unroll
-                                for (int jr = 0; jr < kWH; ++jr)
-                                    if (jr < rows) outc[static_cast<int64_t>(jr) * N + n] = from_f32<CElem>(v[jr]);
-                            }
+                            for (int jr = 0; jr < kWH; ++jr)
+                                if (jr < rows) outc[static_cast<int64_t>(jr) * N + n] = from_f32<CElem>(v[jr]);
                         }
                     }
                 }
@@ -567,12 +548,12 @@ wcsr_merge_kernel(const MergeParams p) {
     }
 }
 
-template <int ES, int FMT, int WH, int CT, bool NARROW = false, bool LSU = false, int TT = 1>
+template <int ES, int FMT, int WH, int CT, bool NARROW = false, bool LSU = false>
 cudaError_t launch_one(const CUtensorMap& tmB, const WcsrParams& p, int sms, cudaStream_t stream) {
-    constexpr int KT = NARROW ? kWcsrNarrowCols : wcsr_stage_cols(ES) / TT;
+    constexpr int KT = NARROW ? kWcsrNarrowCols : wcsr_stage_cols(ES);
     constexpr int STAGES = wcsr_stages(ES, WH), PW = wcsr_producer_warps(ES, WH);
-    using Cfg = WcsrCfg<ES, WH, KT, STAGES, NARROW, TT>;
-    auto kfn = wcsr_spmm_kernel<ES, FMT, WH, KT, STAGES, PW, CT, NARROW, LSU, TT>;
+    using Cfg = WcsrCfg<ES, WH, KT, STAGES, NARROW>;
+    auto kfn = wcsr_spmm_kernel<ES, FMT, WH, KT, STAGES, PW, CT, NARROW, LSU>;
     // resident CTAs per SM: shared memory and TMEM columns are checked in WcsrCfg; the
     // register file follows from __launch_bounds__
     static_assert(Cfg::kCtasPerSm * Cfg::kTmemCols <= 512, "TMEM over-subscribed");
@@ -611,15 +592,8 @@ cudaError_t launch_wh(int dtype, int c16, const CUtensorMap& tmB, const WcsrPara
 
 }  // namespace
 
-cudaError_t launch_wcsr(int dtype, int wh, int c16, int narrow, int lsu_gather, int wide, const CUtensorMap& tmB, const WcsrParams& p,
-                        int sms, cudaStream_t stream) {
-    if (wide) {
-        // two token tiles per pass: 2-byte types at window height 16
-        if (!wcsr_wide_pass(dtype == 2 ? 4 : (dtype == 3 ? 1 : 2), wh) || narrow || lsu_gather) return cudaErrorInvalidValue;
-        if (dtype == 1) return c16 ? launch_one<2, 0, 16, 1, false, false, 2>(tmB, p, sms, stream) : launch_one<2, 0, 16, 0, false, false, 2>(tmB, p, sms, stream);
-        if (dtype == 0) return c16 ? launch_one<2, 1, 16, 1, false, false, 2>(tmB, p, sms, stream) : launch_one<2, 1, 16, 0, false, false, 2>(tmB, p, sms, stream);
-        return cudaErrorInvalidValue;
-    }
+cudaError_t launch_wcsr(int dtype, int wh, int c16, int narrow, int lsu_gather, const CUtensorMap& tmB, const WcsrParams& p, int sms,
+                        cudaStream_t stream) {
     if (lsu_gather) {
         // the comparison variant: window height 16, fp32 C, 128-token stages
         if (wh != 16 || c16 || narrow) return cudaErrorInvalidValue;
