@@ -228,8 +228,9 @@ ALL_OTHERS = DEFAULT_OTHERS + [
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures whose
 # summaries are under profiles/ (absent where no capture of that exact launch exists).
 NCU_DRAM_TRAFFIC = {
-    "cfg2_wcsr_irregular": 131.8e6,     # profiles/wcsr_spmm_cfg2_ncu.md
+    "cfg2_wcsr_irregular": 118.5e6,     # profiles/wcsr_spmm_cfg2_ncu.md
     "cfg5_wcsr_rmat_n128": 3.525e9,     # profiles/wcsr_spmm_cfg5_n128_dram.md
+    "cfg5_wcsr_rmat_n256": 7.186e9,     # the same file, N = 256
     # captured at N = 16,384 (1.409 GB) and scaled by 4 to N = 65,536: one L2 slab is 2048
     # tokens, so traffic grows in proportion to N (profiles/bcsr_spmm_cfg3_n8192_ncu.md)
     "cfg3_bcsr_llm_gate": 5.64e9,
