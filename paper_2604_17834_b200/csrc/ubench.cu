@@ -465,7 +465,7 @@ int main(int argc, char** argv) {
 
     // ---- stores alone and beside loads, per box shape
     struct Shape { int cols, rows; };
-    const Shape shapes[] = {{32, 16}, {32, 64}, {64, 32}, {128, 16}, {256, 8}, {128, 64}};
+    const Shape shapes[] = {{32, 4}, {32, 8}, {32, 16}, {32, 64}, {64, 32}, {128, 16}, {256, 8}, {128, 64}};
     for (const Shape& sh : shapes) {
         for (int hot : {1, 0}) {
             for (int with_loads : {0, 1}) {
