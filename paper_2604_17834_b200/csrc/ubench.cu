@@ -490,6 +490,18 @@ int main(int argc, char** argv) {
             }
         }
     }
+    // ---- more stores in flight per warp: 16 x 128 B boxes with four staging tiles per warp
+    for (int hot : {1, 0})
+        for (int with_loads : {0, 1}) {
+            MixArgs a = base;
+            a.tile_cols = 32; a.tile_rows = 16; a.store_mode = 1; a.hot = hot; a.store_depth = 4;
+            a.store_iters = (24 << 20) / 4 / 2048;
+            a.load_slots = with_loads ? 2 : 0;
+            a.load_iters = with_loads ? 1200 : 0;
+            char nm[96];
+            std::snprintf(nm, sizeof nm, "tma_store_16x128B_depth4_%s%s", hot ? "hot" : "stream", with_loads ? "_with_loads" : "");
+            run_mix(cx, nm, a);
+        }
     // ---- st.global from registers
     for (int hot : {1, 0})
         for (int with_loads : {0, 1}) {
