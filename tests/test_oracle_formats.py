@@ -116,7 +116,7 @@ def test_bcsr_dense_and_block_diagonal_and_fill_ratio():
 
 
 @pytest.mark.parametrize("m,k,dens", CASES)
-@pytest.mark.parametrize("wh,b_col", [(4, 2), (16, 8), (16, 16), (1, 4)])
+@pytest.mark.parametrize("wh,b_col", [(4, 2), (16, 8), (16, 16), (1, 4), (16, 32), (64, 32)])
 def test_wcsr_matches_brute_force_and_round_trips(m, k, dens, wh, b_col):
     a = wl.random_csr(200 + m + wh, m, k, dens, "fp16", empty_rows=tuple(range(min(wh, m))))
     D, mask = _dense(a)
