@@ -149,6 +149,9 @@ mix_kernel(const __grid_constant__ CUtensorMap tmL, const __grid_constant__ CUte
             const uint64_t ad = make_smem_desc(base, 8192, 1024, SWZ_128B);
             const uint64_t bd = make_smem_desc(base + slot_bytes, 16, 1024, SWZ_128B);
             const int acc_mask = 512 / a.mma_n - 1;
+            // the ring's first loads bring the source array's values into both slots: give them time
+            const long long ts = clock64();
+            while (clock64() - ts < 30000) { }
             const long long t0 = clock64();
             if (elect_one()) {
 #pragma unroll 8
@@ -241,6 +244,15 @@ gather_kernel(const __grid_constant__ CUtensorMap tmG, int slots, int lanes, int
             const int x = static_cast<int>((seed >> 10) % static_cast<uint32_t>(n_col_segs / 2)) * 128 + sg * 64;
             if (lane < lanes) tma_gather4_2d(sb + sg * (lanes * 256) + rg * 512, &tmG, b, x, r[0], r[1], r[2], r[3]);
         }
+    }
+}
+
+// bf16 values +-[1, 2) with pseudo-random signs and mantissas
+__global__ void fill_random_kernel(uint16_t* p, size_t n) {
+    for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n; i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        uint32_t h = static_cast<uint32_t>(i) * 2654435761u;
+        h ^= h >> 15; h *= 2246822519u; h ^= h >> 13;
+        p[i] = static_cast<uint16_t>(0x3F80u | (h & 0x7Fu) | ((h >> 8) & 1u) << 15);
     }
 }
 
@@ -444,22 +456,31 @@ int main(int argc, char** argv) {
     }
 
     // ---- MMAs beside the loads: do operand reads and TMA writes share shared-memory bandwidth?
+    // And does the rate of the MMAs depend on the operand VALUES (all SMs issuing: a power question)?
     {
         long long* dclk;
         CK(cudaMalloc(&dclk, cx.sms * sizeof(long long)));
-        for (int n : {64, 128}) {
-            for (int with_loads : {0, 1}) {
-                MixArgs a = base;
-                a.load_slots = 2;                               // the ring's memory holds the operands either way
-                a.load_iters = with_loads ? 1500 : 0;
-                a.mma_n = n;
-                a.mma_count = n == 64 ? 28000 : 21000;          // about as long as the loads alone
-                a.mma_clk = dclk;
-                char nm[64];
-                std::snprintf(nm, sizeof nm, "mma_n%d%s", n, with_loads ? "_with_loads_2x64KB" : "_alone_all_sms");
-                run_mix(cx, nm, a);
+        for (int random_data : {0, 1}) {
+            if (random_data) {
+                fill_random_kernel<<<1024, 256>>>(static_cast<uint16_t*>(cx.src), Ctx::K * Ctx::N);
+                CK(cudaDeviceSynchronize());
+            }
+            for (int n : {64, 128, 256}) {
+                for (int with_loads : {0, 1}) {
+                    MixArgs a = base;
+                    a.load_slots = 2;                               // the ring's memory holds the operands either way
+                    a.load_iters = with_loads ? 1500 : 2;           // (alone: one load per slot, then nothing)
+                    a.mma_n = n;
+                    a.mma_count = n == 64 ? 28000 : (n == 128 ? 21000 : 10500);   // about as long as the loads alone
+                    a.mma_clk = dclk;
+                    char nm[96];
+                    std::snprintf(nm, sizeof nm, "mma_n%d%s_%s_operands", n, with_loads ? "_with_loads_2x64KB" : "_alone_all_sms",
+                                  random_data ? "random" : "zero");
+                    run_mix(cx, nm, a);
+                }
             }
         }
+        CK(cudaMemset(cx.src, 0, Ctx::K * Ctx::N * 2));
         CK(cudaFree(dclk));
     }
 
