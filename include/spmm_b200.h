@@ -306,6 +306,17 @@ int spmm_wcsr_create_coo(spmm_handle_t *out, int64_t m, int64_t k, int64_t nnz,
 int spmm_bcsr_plan(spmm_handle_t h, int64_t N);
 
 /*
+ * Both formats (an addition of this library): do ahead of time what the first spmm_run with a
+ * new dense width N would do besides launching -- BCSR: spmm_bcsr_plan (schedule, its device
+ * arrays, the workspace of a K-split plan); WCSR: grow the handle's partial-tile workspace to
+ * what N needs.  May allocate and synchronise the device.  Afterwards spmm_run(h, ., ., N', .)
+ * with N' = N (BCSR) or N' <= N (WCSR) makes no allocating or synchronising call of its own
+ * (the CUDA runtime may still load a kernel variant's code on that variant's first launch).
+ * Same argument rules as spmm_run for N; a host_only WCSR handle returns SPMM_OK and does nothing.
+ */
+int spmm_prepare(spmm_handle_t h, int64_t N);
+
+/*
  * C = A x B (Sec. 2.3; kernels of Sec. 3).  Asynchronous on `stream` (a cudaStream_t passed
  * as void*; NULL = the default stream); never synchronises.
  *   B_dev  device, k x N row-major, elements of the handle's dtype, 16-byte aligned.

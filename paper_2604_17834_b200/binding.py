@@ -48,7 +48,7 @@ X_WCSR_BIN_PTR, X_WCSR_BIN_TASKS, X_WCSR_GROUP_CLASS = 14, 15, 16
 EXPORTED_SYMBOLS = (
     "spmm_bcsr_create_csr", "spmm_bcsr_create_csr_device", "spmm_bcsr_create_coo", "spmm_wcsr_create_csr",
     "spmm_wcsr_create_csr_device", "spmm_wcsr_create_coo",
-    "spmm_bcsr_plan", "spmm_run", "spmm_wcsr_run_static", "spmm_run_host", "spmm_check", "spmm_get_info", "spmm_export", "spmm_destroy",
+    "spmm_bcsr_plan", "spmm_prepare", "spmm_run", "spmm_wcsr_run_static", "spmm_run_host", "spmm_check", "spmm_get_info", "spmm_export", "spmm_destroy",
     "spmm_status_string", "spmm_set_wait_limit_ns",
 )
 
@@ -92,6 +92,7 @@ _lib.spmm_bcsr_create_coo.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _vp
 _lib.spmm_wcsr_create_coo.argtypes = _lib.spmm_bcsr_create_coo.argtypes
 _lib.spmm_run.argtypes = [_vp, _vp, _vp, _i64, _vp]
 _lib.spmm_bcsr_plan.argtypes = [_vp, _i64]
+_lib.spmm_prepare.argtypes = [_vp, _i64]
 _lib.spmm_run_host.argtypes = [_vp, _vp, _vp, _i64, _vp]
 _lib.spmm_wcsr_run_static.argtypes = [_vp, _vp, _vp, _i64, _vp]
 _lib.spmm_check.argtypes = [_vp]
@@ -224,6 +225,13 @@ def spmm_bcsr_plan(h, N):
     rc = _lib.spmm_bcsr_plan(h, N)
     if rc != SPMM_OK:
         raise SpmmError(rc, "spmm_bcsr_plan")
+
+
+def spmm_prepare(h, N):
+    """Both formats: allocate and plan now what the first spmm_run at dense width N would."""
+    rc = _lib.spmm_prepare(h, N)
+    if rc != SPMM_OK:
+        raise SpmmError(rc, "spmm_prepare")
 
 
 def spmm_run(h, B_dev_ptr, C_dev_ptr, N, stream=0):

@@ -946,7 +946,8 @@ int launch_wcsr_all(spmm_handle_s* h, const void* B, void* C, float* partial, in
     return e == cudaSuccess ? SPMM_OK : SPMM_ERR_CUDA;
 }
 
-int run_wcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t stream) {
+// The handle's workspace for the partial tiles of split windows at dense width N (grown, never shrunk).
+int ensure_wcsr_workspace(spmm_handle_s* h, int64_t N) {
     const size_t need = static_cast<size_t>(wcsr_workspace_bytes(h, N));
     if (need > h->partial_bytes) {
         if (h->d_partial) {
@@ -958,6 +959,11 @@ int run_wcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t s
         if (cudaMalloc(reinterpret_cast<void**>(&h->d_partial), need) != cudaSuccess) return SPMM_ERR_ALLOC;
         h->partial_bytes = need;
     }
+    return SPMM_OK;
+}
+
+int run_wcsr(spmm_handle_s* h, const void* B, void* C, int64_t N, cudaStream_t stream) {
+    if (int rc = ensure_wcsr_workspace(h, N)) return rc;
     return launch_wcsr_all(h, B, C, h->d_partial, N, stream);
 }
 
@@ -1077,6 +1083,19 @@ int spmm_bcsr_plan(spmm_handle_t h, int64_t N) {
     if (h->format != 0) return SPMM_ERR_INVALID_ARG;
     if (N < ((h->col_major || h->es == 1) ? 128 : 64) || (!h->col_major && (N * h->es) % 16 != 0)) return SPMM_ERR_UNSUPPORTED;
     return ensure_schedule(h, N);
+}
+
+int spmm_prepare(spmm_handle_t h, int64_t N) {
+    NvtxRange nvtx_range("spmm_prepare");
+    if (!h || N <= 0) return SPMM_ERR_INVALID_ARG;
+    if (h->format == 0) return spmm_bcsr_plan(h, N);
+    if ((N * h->es) % 16 != 0) return SPMM_ERR_UNSUPPORTED;
+    if (N >= (int64_t{1} << 31)) return SPMM_ERR_TOO_LARGE;
+    if (h->host_only) return SPMM_OK;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SPMM_ERR_CUDA;
+    if (dev != h->device) return SPMM_ERR_INVALID_ARG;
+    return ensure_wcsr_workspace(h, N);
 }
 
 int spmm_wcsr_run_static(spmm_handle_t h, const void* B_dev, void* C_dev, int64_t N, void* stream) {

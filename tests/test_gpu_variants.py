@@ -447,6 +447,53 @@ def test_bcsr_row_groups_find_scattered_families(lib, b, dtype):
         lib.spmm_destroy(h)
 
 
+@pytest.mark.parametrize("kind", ["bcsr", "bcsr_ksplit", "wcsr"])
+def test_prepare_leaves_nothing_to_allocate_for_the_run(lib, kind):
+    """After spmm_prepare(h, N) the first spmm_run at that width changes neither the free device
+    memory nor the workspace the handle reports (one throw-away handle of the same kind runs first,
+    so that the kernel variant's code is already loaded)."""
+    import torch
+    dtype, N = "fp16", 512
+    st = torch.cuda.current_stream().cuda_stream
+
+    def make():
+        if kind == "wcsr":
+            a = wl.wcsr_irregular(seed=91, m=6000, dtype=dtype)
+            return a, lib.spmm_wcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], dtype, 16, split_cols=64)
+        a = wl.bcsr_sweep(93, m=2048, k=2048, b=64, density=0.05, dtype=dtype)
+        return a, lib.spmm_bcsr_create_csr(a["m"], a["k"], a["row_ptr"], a["col_idx"], a["vals"], dtype, 64,
+                                           k_split=1 if kind == "bcsr_ksplit" else 0)
+
+    a, h0 = make()
+    Bs = wl.dense(94, a["k"], N, ("normal", 0.0, 1.0), dtype)
+    Bd = to_device(Bs)
+    C = torch.empty((a["m"], N), dtype=torch.float32, device="cuda")
+    lib.spmm_run(h0, Bd.data_ptr(), C.data_ptr(), N, st)                 # loads the kernels
+    torch.cuda.synchronize()
+    want = C.cpu().numpy().copy()
+    lib.spmm_destroy(h0)
+    _, h = make()
+    try:
+        lib.spmm_prepare(h, N)
+        info = lib.spmm_get_info(h, N)
+        if kind != "bcsr":
+            assert info["workspace_bytes"] > 0, "the case must need a workspace"
+        C.fill_(float("nan"))
+        torch.cuda.synchronize()
+        free0 = torch.cuda.mem_get_info()[0]
+        lib.spmm_run(h, Bd.data_ptr(), C.data_ptr(), N, st)
+        free1 = torch.cuda.mem_get_info()[0]
+        torch.cuda.synchronize()
+        lib.spmm_check(h)
+        assert free1 == free0
+        assert lib.spmm_get_info(h, N)["workspace_bytes"] == info["workspace_bytes"]
+        assert np.array_equal(C.cpu().numpy(), want)
+        Cr, S = reference(a, Bs, dtype)
+        assert_close(C.cpu().numpy(), Cr, S, dtype, "prepared run, " + kind)
+    finally:
+        lib.spmm_destroy(h)
+
+
 # --------------------------------------------------------------------------- the paper's own gather (load/store units)
 
 

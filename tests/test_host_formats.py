@@ -365,6 +365,17 @@ def test_malformed_input_is_rejected(lib):
     h8 = mw(2, 4, rp, np.array([0, 1, 2], np.int32), v8, "fp8", 16, host_only=True)
     assert lib.spmm_export(h8, lib.X_WCSR_WINDOW_COL_IDX, np.int32).tolist() == [0, 1, 2] + [-1] * 29
     lib.spmm_destroy(h8)
+    # spmm_prepare: spmm_run's rules for N; a host-only WCSR handle has nothing to prepare
+    hp = mw(2, 4, rp, np.array([0, 1, 2], np.int32), v, "fp16", 16, host_only=True)
+    lib.spmm_prepare(hp, 128)
+    assert code(lib.spmm_prepare, hp, 100) == lib.SPMM_ERR_UNSUPPORTED          # rows of 200 bytes
+    assert code(lib.spmm_prepare, hp, 0) == lib.SPMM_ERR_INVALID_ARG
+    lib.spmm_destroy(hp)
+    hp = mk(2, 4, rp, np.array([0, 1, 2], np.int32), v, "fp16", 16, host_only=True)
+    lib.spmm_prepare(hp, 128)                                                    # = spmm_bcsr_plan
+    assert lib.spmm_get_info(hp, 128)["plan_token_tile"] > 0
+    assert code(lib.spmm_prepare, hp, 32) == lib.SPMM_ERR_UNSUPPORTED
+    lib.spmm_destroy(hp)
     dup_r, dup_c = np.array([0, 0], np.int32), np.array([1, 1], np.int32)
     assert code(lib.spmm_bcsr_create_coo, 2, 4, dup_r, dup_c, v[:2], "fp16", 16, host_only=True) == lib.SPMM_ERR_UNSORTED
     lib.spmm_destroy(None)                                     # NULL is accepted
