@@ -167,11 +167,12 @@ def test_wcsr_irregular_scaled(lib):
     assert worst < 1.0
 
 
-def test_wcsr_rmat_scaled(lib):
-    """configs[4] recipe at 2^14 rows, fp16, N = 32 / 128."""
-    a = wl.rmat(scale=14, dtype="fp16")
+@pytest.mark.parametrize("dtype", ["fp16", "fp8"])
+def test_wcsr_rmat_scaled(lib, dtype):
+    """configs[4] recipe at 2^14 rows, fp16 (and E4M3 values), N = 32 / 128."""
+    a = wl.rmat(scale=14, dtype=dtype)
     for N in (32, 128):
-        _wcsr_case(lib, a, "fp16", N, T=512)
+        _wcsr_case(lib, a, dtype, N, T=512)
 
 
 def test_wcsr_ragged_rows_and_identity(lib):
